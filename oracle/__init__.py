@@ -1,0 +1,191 @@
+"""Float64 CPU oracle for the S4C verify step (arXiv 2506.14158) -- TEST INFRASTRUCTURE ONLY.
+
+This package wraps ``s4c_oracle.c`` (plain C, float64) with ctypes and numpy.  It is the
+checker the CUDA library is compared against: it shares no code with the CUDA path and
+does not import it.  Only the tests, the smoke check and the benchmark's CPU-baseline /
+reference legs may import it; the product path never does.
+
+Functions (array layouts are row-major numpy arrays):
+
+* :func:`tree_attention`      -- Section 3.2 / Figure 3 tree mask: masked softmax attention by definition.
+* :func:`accept_greedy`       -- Section 4.1.2 greedy decoding + Section 3.2 longest accepted path.
+* :func:`accept_stochastic`   -- Section 2 speculative sampling, Eq. 11 / Eq. 12, step by step.
+* :func:`kv_compact`          -- Section 3.2 last paragraph: keep accepted tokens' K/V and features.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "s4c_oracle.c")
+_LIB = os.path.join(_HERE, "libs4c_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+SEQ_OK = 0
+SEQ_BAD_PARENT = 1
+SEQ_TOKEN_RANGE = 2
+SEQ_CAPACITY = 4
+SEQ_DEPTH = 8
+SEQ_BAD_PATH = 16
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP on the outer loops only) and return the library path."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            cmd = ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-fopenmp", "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        lib.s4c_oracle_max_threads.restype = ctypes.c_int
+        lib.s4c_oracle_set_threads.argtypes = [ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().s4c_oracle_max_threads())
+
+
+def set_threads(n: int) -> None:
+    _load().s4c_oracle_set_threads(int(n))
+
+
+def _ptr(a, ctype):
+    if a is None:
+        return None
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+def _i32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.int32)
+
+
+def tree_attention(q, k, v, cache_len, parent, n_nodes=None, scale=0.0):
+    """q [B,Hq,T,d]; k, v [B,Hkv,C,d] (tree K/V at slots L_b..L_b+T-1); returns (out f64, status[B])."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k = np.ascontiguousarray(k, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    B, Hq, T, d = q.shape
+    _, Hkv, C, _ = k.shape
+    assert k.shape == v.shape == (B, Hkv, C, d)
+    cache_len = _i32(cache_len)
+    parent = _i32(parent).reshape(B, T)
+    n_nodes = _i32(n_nodes)
+    out = np.full(q.shape, np.nan, dtype=np.float64)
+    status = np.zeros(B, dtype=np.int32)
+    dbl, i32 = ctypes.c_double, ctypes.c_int32
+    rc = _load().s4c_oracle_tree_attention(
+        _ptr(q, dbl), _ptr(k, dbl), _ptr(v, dbl), _ptr(cache_len, i32), _ptr(parent, i32),
+        _ptr(n_nodes, i32), _ptr(out, dbl), _ptr(status, i32),
+        B, T, Hq, Hkv, d, C, ctypes.c_double(scale))
+    if rc:
+        raise ValueError(f"oracle tree_attention rejected its arguments (code {rc})")
+    return out, status
+
+
+def _accept_outputs(B, max_depth):
+    return (np.full(B, -7, dtype=np.int32), np.full((B, max_depth + 1), -7, dtype=np.int32),
+            np.full(B, -7, dtype=np.int32), np.zeros(B, dtype=np.int32))
+
+
+def accept_greedy(logits, tokens, parent, n_nodes=None, max_depth=None):
+    """logits [B,T,V] f32 -> dict(accept_len[B], path[B,max_depth+1], next_token[B], status[B])."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    B, T, V = logits.shape
+    tokens = _i32(tokens).reshape(B, T)
+    parent = _i32(parent).reshape(B, T)
+    n_nodes = _i32(n_nodes)
+    if max_depth is None:
+        max_depth = T - 1
+    a, path, nxt, status = _accept_outputs(B, max_depth)
+    f32, i32 = ctypes.c_float, ctypes.c_int32
+    rc = _load().s4c_oracle_accept_greedy(
+        _ptr(logits, f32), _ptr(tokens, i32), _ptr(parent, i32), _ptr(n_nodes, i32),
+        B, T, V, max_depth, _ptr(a, i32), _ptr(path, i32), _ptr(nxt, i32), _ptr(status, i32))
+    if rc:
+        raise ValueError(f"oracle accept_greedy rejected its arguments (code {rc})")
+    return dict(accept_len=a, path=path, next_token=nxt, status=status)
+
+
+def accept_stochastic(logits, draft_probs, tokens, parent, temperature, uniforms, n_nodes=None,
+                      max_depth=None):
+    """Eq. 11 / Eq. 12 walk; returns dict(accept_len, path, next_token, near_tie[B,T], status)."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    draft_probs = np.ascontiguousarray(draft_probs, dtype=np.float32)
+    B, T, V = logits.shape
+    assert draft_probs.shape == (B, T, V)
+    tokens = _i32(tokens).reshape(B, T)
+    parent = _i32(parent).reshape(B, T)
+    uniforms = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, T)
+    n_nodes = _i32(n_nodes)
+    if max_depth is None:
+        max_depth = T - 1
+    a, path, nxt, status = _accept_outputs(B, max_depth)
+    tie = np.zeros((B, T), dtype=np.uint8)
+    f32, i32 = ctypes.c_float, ctypes.c_int32
+    rc = _load().s4c_oracle_accept_stochastic(
+        _ptr(logits, f32), _ptr(draft_probs, f32), _ptr(tokens, i32), _ptr(parent, i32),
+        _ptr(n_nodes, i32), ctypes.c_double(float(temperature)), _ptr(uniforms, f32),
+        B, T, V, max_depth, _ptr(a, i32), _ptr(path, i32), _ptr(nxt, i32),
+        _ptr(tie, ctypes.c_uint8), _ptr(status, i32))
+    if rc:
+        raise ValueError(f"oracle accept_stochastic rejected its arguments (code {rc})")
+    return dict(accept_len=a, path=path, next_token=nxt, near_tie=tie, status=status)
+
+
+def kv_compact(k_caches, v_caches, cache_len, path, accept_len, T, feat_in=None, feat_out=None):
+    """In place on lists of numpy caches [B,Hkv,C,d] (any fixed-size dtype); returns status[B].
+
+    ``T`` is the number of tree slots per sequence.  ``cache_len`` (int32 array) is updated in
+    place to L_b + a + 1; ``feat_out`` [B,max_depth+1,hid] receives rows 0..a of ``feat_in``
+    [B,T,hid] gathered along the path.
+    """
+    n_layers = len(k_caches)
+    assert len(v_caches) == n_layers
+    assert cache_len.dtype == np.int32 and cache_len.flags.c_contiguous
+    B = cache_len.shape[0]
+    path = _i32(path).reshape(B, -1)
+    max_depth = path.shape[1] - 1
+    accept_len = _i32(accept_len)
+    if n_layers:
+        _, Hkv, C, d = k_caches[0].shape
+        esz = k_caches[0].dtype.itemsize
+    else:
+        Hkv, C, d, esz = 1, 1, 1, (feat_in.dtype.itemsize if feat_in is not None else 1)
+    for c in list(k_caches) + list(v_caches):
+        assert c.flags.c_contiguous and c.shape == (B, Hkv, C, d) and c.dtype.itemsize == esz
+    u8p = ctypes.POINTER(ctypes.c_uint8)
+    karr = (u8p * max(n_layers, 1))(*[c.ctypes.data_as(u8p) for c in k_caches])
+    varr = (u8p * max(n_layers, 1))(*[c.ctypes.data_as(u8p) for c in v_caches])
+    hid = 0
+    if feat_in is not None:
+        assert feat_in.flags.c_contiguous and feat_out is not None and feat_out.flags.c_contiguous
+        assert feat_in.shape[0] == B and feat_in.shape[1] == T and feat_in.dtype.itemsize == esz
+        hid = feat_in.shape[2]
+        assert feat_out.shape == (B, max_depth + 1, hid) and feat_out.dtype == feat_in.dtype
+    status = np.zeros(B, dtype=np.int32)
+    rc = _load().s4c_oracle_kv_compact(
+        karr, varr, n_layers, _ptr(cache_len, ctypes.c_int32), _ptr(path, ctypes.c_int32),
+        _ptr(accept_len, ctypes.c_int32), max_depth,
+        None if feat_in is None else feat_in.ctypes.data_as(u8p),
+        None if feat_out is None else feat_out.ctypes.data_as(u8p),
+        B, T, Hkv, d, C, hid, esz, _ptr(status, ctypes.c_int32))
+    if rc:
+        raise ValueError(f"oracle kv_compact rejected its arguments (code {rc})")
+    return status

@@ -1,0 +1,450 @@
+/*
+ * s4c_oracle.c -- slow, plain, float64 CPU oracle for the S4C verify step.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the checker the CUDA library is
+ * compared against.  It shares no code, header, table or helper with the CUDA
+ * path and the product never calls it.  Only the tests, the smoke check and the
+ * "cpu_baseline" / "--impl reference" legs of the benchmark may load it.
+ *
+ * What it computes (each function cites the passage of the S4C paper,
+ * arXiv 2506.14158, that defines the operation):
+ *
+ *   s4c_oracle_tree_attention  Section 3.2 ("a tree mask is applied") and the
+ *                              caption of Figure 3 (tree mask matrix): every
+ *                              tree token attends the cached prefix and its own
+ *                              root path.  Written out as the definition of
+ *                              masked softmax attention; no tiling, no online
+ *                              softmax.
+ *   s4c_oracle_accept_greedy   Section 4.1.2 (all experiments decode greedily)
+ *                              and Section 3.2 (longest accepted path).
+ *   s4c_oracle_accept_stochastic
+ *                              Section 2 "Speculative Sampling" (accept with
+ *                              probability min(1, p/q), resample from
+ *                              norm(max(0, p - q))), Eq. 11 and Eq. 12 of
+ *                              Section 3.2 (the correction at fork positions).
+ *                              Taken step by step, in the paper's order.
+ *   s4c_oracle_kv_compact      Section 3.2, last paragraph (accepted tokens and
+ *                              their features are kept for the next drafting
+ *                              phase): a gather from a snapshot.
+ *
+ * Readings of silent or garbled points (symbols follow Section 2: p = target,
+ * q = draft):
+ *   - Eq. 11 prints q(x)/p(x) and then calls q the target and p the draft; with
+ *     the symbols untangled the ratio is target/draft, as in Section 2.
+ *   - Eq. 12 prints norm(max(q_c, p_c)); Section 2 gives the rule it stands for:
+ *     norm(max(0, p_target - p_draft)).
+ *   - Several siblings at one position are tried one after another in index
+ *     order; after each rejection the target distribution is replaced by the
+ *     normalised residual and the rejected token is removed from the draft
+ *     distribution, which is renormalised (the multi-candidate correction the
+ *     paper cites for trees).
+ *   - Comparison is strict (r < min(1, ratio)), as printed in Eq. 11.
+ *   - A token is always emitted at the end of the walk: from the residual at the
+ *     fork, or from the unmodified target distribution at a leaf.
+ *   - Ties in argmax go to the lowest index.
+ *
+ * Pins (see tests/test_oracle_*.py): chain tree == causal attention, star tree,
+ * path equivalence against a library SDPA, constant-V, GQA == repeated MHA;
+ * greedy verify == token-by-token greedy decoding, planted trees; exact
+ * enumeration on dyadic tiny-vocab cases and chi-square Monte-Carlo showing the
+ * emitted token follows the target distribution; compaction against a library
+ * gather.  The paper prints no worked numeric example for any of these steps,
+ * so config-level values are: parity unpinned by printed numbers (pinned by the
+ * invariants above instead).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* per-sequence status bit flags (kept numerically equal to the public header's
+ * values by a test, not by a shared include) */
+#define ORC_SEQ_OK 0
+#define ORC_SEQ_BAD_PARENT 1
+#define ORC_SEQ_TOKEN_RANGE 2
+#define ORC_SEQ_CAPACITY 4
+#define ORC_SEQ_DEPTH 8
+#define ORC_SEQ_BAD_PATH 16
+
+int s4c_oracle_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void s4c_oracle_set_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* A tree is given in topological order: parent[0] = -1, 0 <= parent[i] < i. */
+static int tree_is_valid(const int32_t* parent, int n) {
+    if (n < 1) return 0;
+    if (parent[0] != -1) return 0;
+    for (int i = 1; i < n; ++i)
+        if (parent[i] < 0 || parent[i] >= i) return 0;
+    return 1;
+}
+
+static int node_count(const int32_t* n_nodes, int b, int T) {
+    return n_nodes ? n_nodes[b] : T;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Tree-masked attention (Section 3.2; Figure 3, tree mask matrix).            */
+/*                                                                           */
+/* q      [B,Hq,T,d]   float64                                               */
+/* k, v   [B,Hkv,C,d]  float64; the tree's own K/V sit at slots L_b..L_b+T-1 */
+/* out    [B,Hq,T,d]   float64                                               */
+/* Node i of sequence b sees slots 0..L_b-1 (the committed prefix) and slot   */
+/* L_b+t for every t on the path root..i (i included).  Weights are a softmax */
+/* of scale * <q,k> over exactly that set.                                    */
+/* Rows of padding nodes (i >= n_nodes[b]) are set to zero.  A sequence with  */
+/* a malformed tree or L_b + n > C gets a status flag and its rows untouched. */
+/* ------------------------------------------------------------------------- */
+int s4c_oracle_tree_attention(const double* q, const double* k, const double* v,
+                              const int32_t* cache_len, const int32_t* parent,
+                              const int32_t* n_nodes, double* out, int32_t* status,
+                              int B, int T, int Hq, int Hkv, int d, int C, double scale) {
+    if (!q || !k || !v || !cache_len || !parent || !out) return 1;
+    if (B < 0 || T < 1 || Hq < 1 || Hkv < 1 || d < 1 || C < 1 || Hq % Hkv) return 2;
+    const int G = Hq / Hkv;
+    if (scale == 0.0) scale = 1.0 / sqrt((double)d);
+    for (int b = 0; b < B; ++b) {
+        const int n = node_count(n_nodes, b, T);
+        const int L = cache_len[b];
+        const int32_t* par = parent + (size_t)b * T;
+        int st = ORC_SEQ_OK;
+        if (n < 1 || n > T || !tree_is_valid(par, n)) st |= ORC_SEQ_BAD_PARENT;
+        if (L < 0 || (long)L + (n > 0 ? n : 0) > (long)C) st |= ORC_SEQ_CAPACITY;
+        if (status) status[b] = st;
+        if (st) continue;
+
+        /* visible[i*n + t] = 1 iff t is i or an ancestor of i */
+        unsigned char* visible = (unsigned char*)calloc((size_t)n * n, 1);
+        for (int i = 0; i < n; ++i)
+            for (int t = i; t >= 0; t = par[t]) visible[(size_t)i * n + t] = 1;
+
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic)
+#endif
+        for (int h = 0; h < Hq; ++h) {
+            const int hk = h / G;
+            const double* kb = k + ((size_t)b * Hkv + hk) * C * d;
+            const double* vb = v + ((size_t)b * Hkv + hk) * C * d;
+            double* s = (double*)malloc(sizeof(double) * (size_t)(L + n));
+            for (int i = 0; i < T; ++i) {
+                double* o = out + (((size_t)b * Hq + h) * T + i) * d;
+                for (int c = 0; c < d; ++c) o[c] = 0.0;
+                if (i >= n) continue;
+                const double* qi = q + (((size_t)b * Hq + h) * T + i) * d;
+                double mx = -INFINITY;
+                for (int j = 0; j < L + n; ++j) {
+                    if (j >= L && !visible[(size_t)i * n + (j - L)]) {
+                        s[j] = -INFINITY;
+                        continue;
+                    }
+                    double acc = 0.0;
+                    for (int c = 0; c < d; ++c) acc += qi[c] * kb[(size_t)j * d + c];
+                    s[j] = scale * acc;
+                    if (s[j] > mx) mx = s[j];
+                }
+                double den = 0.0;
+                for (int j = 0; j < L + n; ++j) {
+                    s[j] = (s[j] == -INFINITY) ? 0.0 : exp(s[j] - mx);
+                    den += s[j];
+                }
+                for (int j = 0; j < L + n; ++j) {
+                    if (s[j] == 0.0) continue;
+                    const double w = s[j] / den;
+                    for (int c = 0; c < d; ++c) o[c] += w * vb[(size_t)j * d + c];
+                }
+            }
+            free(s);
+        }
+        free(visible);
+    }
+    return 0;
+}
+
+/* depth of every node, root = 0 */
+static void tree_depths(const int32_t* par, int n, int* depth) {
+    depth[0] = 0;
+    for (int i = 1; i < n; ++i) depth[i] = depth[par[i]] + 1;
+}
+
+/* writes root..e into path (max_depth+1 entries, -1 padded); returns depth of e */
+static int write_path(const int32_t* par, int e, const int* depth, int max_depth, int32_t* path) {
+    for (int j = 0; j <= max_depth; ++j) path[j] = -1;
+    for (int t = e; t >= 0; t = par[t]) path[depth[t]] = t;
+    return depth[e];
+}
+
+static int validate_accept_inputs(const int32_t* par, const int32_t* tok, int n, int T, int V,
+                                  int max_depth, int* depth) {
+    int st = ORC_SEQ_OK;
+    if (n < 1 || n > T || !tree_is_valid(par, n)) return ORC_SEQ_BAD_PARENT;
+    for (int i = 0; i < n; ++i)
+        if (tok[i] < 0 || tok[i] >= V) st |= ORC_SEQ_TOKEN_RANGE;
+    tree_depths(par, n, depth);
+    for (int i = 0; i < n; ++i)
+        if (depth[i] > max_depth) st |= ORC_SEQ_DEPTH;
+    return st;
+}
+
+static int argmax_lowest(const float* row, int V) {
+    int best = 0;
+    for (int v = 1; v < V; ++v)
+        if (row[v] > row[best]) best = v;
+    return best;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Greedy verification (Section 4.1.2: greedy decoding; Section 3.2: longest   */
+/* accepted path).                                                           */
+/*                                                                           */
+/* g[n] = argmax_v logits[n,v].  Node i is accepted iff its parent is and    */
+/* tokens[i] == g[parent[i]]; the root is accepted by definition.  The result */
+/* is the accepted node of greatest depth (lowest index among equals), the    */
+/* path to it, and the target's own next token g[e] after it.                 */
+/* ------------------------------------------------------------------------- */
+int s4c_oracle_accept_greedy(const float* logits, const int32_t* tokens, const int32_t* parent,
+                             const int32_t* n_nodes, int B, int T, int V, int max_depth,
+                             int32_t* accept_len, int32_t* path, int32_t* next_token,
+                             int32_t* status) {
+    if (!logits || !tokens || !parent || !accept_len || !path || !next_token) return 1;
+    if (B < 0 || T < 1 || V < 1 || max_depth < 0) return 2;
+    for (int b = 0; b < B; ++b) {
+        const int n = node_count(n_nodes, b, T);
+        const int32_t* par = parent + (size_t)b * T;
+        const int32_t* tok = tokens + (size_t)b * T;
+        int32_t* pth = path + (size_t)b * (max_depth + 1);
+        int* depth = (int*)malloc(sizeof(int) * (size_t)T);
+        const int st = validate_accept_inputs(par, tok, n, T, V, max_depth, depth);
+        if (status) status[b] = st;
+        if (st) {
+            accept_len[b] = -1;
+            next_token[b] = -1;
+            for (int j = 0; j <= max_depth; ++j) pth[j] = -1;
+            free(depth);
+            continue;
+        }
+        int* g = (int*)malloc(sizeof(int) * (size_t)n);
+        unsigned char* ok = (unsigned char*)calloc((size_t)n, 1);
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic)
+#endif
+        for (int i = 0; i < n; ++i) g[i] = argmax_lowest(logits + ((size_t)b * T + i) * V, V);
+        ok[0] = 1;
+        int e = 0;
+        for (int i = 1; i < n; ++i) {
+            ok[i] = ok[par[i]] && tok[i] == g[par[i]];
+            if (ok[i] && depth[i] > depth[e]) e = i;
+        }
+        accept_len[b] = write_path(par, e, depth, max_depth, pth);
+        next_token[b] = g[e];
+        free(g);
+        free(ok);
+        free(depth);
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Stochastic verification (Section 2 "Speculative Sampling"; Eq. 11, Eq. 12). */
+/*                                                                           */
+/* logits  [B,T,V] float32: row n = target logits for the token after node n  */
+/* dprobs  [B,T,V] float32: row n = draft distribution the children of n were */
+/*                          proposed from (already at this temperature)       */
+/* uniforms[B,T]   float32 in [0,1): entry i>=1 is node i's acceptance draw,  */
+/*                          entry 0 is the draw for the final token           */
+/* Steps per sequence, cur = root:                                            */
+/*  S1  p = softmax(logits[cur]/tau), q = dprobs[cur]; children of cur in     */
+/*      index order.                                                          */
+/*  S2  for each child c with token x: ratio = p(x)/q(x) (q(x)=0: +inf if     */
+/*      p(x)>0 else 0); accept iff u_c < min(1, ratio); on accept cur = c and */
+/*      back to S1.                                                           */
+/*  S3  on reject: p <- norm(max(p-q,0)) (kept if the mass is 0); q(x) <- 0,  */
+/*      q <- q/sum(q) (if the sum is 0 no further sibling is tried).           */
+/*  S4  no child accepted: next token = smallest v whose running sum of p     */
+/*      exceeds u_0 * sum(p).                                                 */
+/* near_tie[b,i] = 1 where |ratio - u_i| < 1e-6 at node i's test.             */
+/* ------------------------------------------------------------------------- */
+int s4c_oracle_accept_stochastic(const float* logits, const float* dprobs, const int32_t* tokens,
+                                 const int32_t* parent, const int32_t* n_nodes, double tau,
+                                 const float* uniforms, int B, int T, int V, int max_depth,
+                                 int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                 uint8_t* near_tie, int32_t* status) {
+    if (!logits || !dprobs || !tokens || !parent || !uniforms || !accept_len || !path ||
+        !next_token)
+        return 1;
+    if (B < 0 || T < 1 || V < 1 || max_depth < 0 || !(tau > 0.0)) return 2;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic)
+#endif
+    for (int b = 0; b < B; ++b) {
+        const int n = node_count(n_nodes, b, T);
+        const int32_t* par = parent + (size_t)b * T;
+        const int32_t* tok = tokens + (size_t)b * T;
+        const float* u = uniforms + (size_t)b * T;
+        int32_t* pth = path + (size_t)b * (max_depth + 1);
+        uint8_t* tie = near_tie ? near_tie + (size_t)b * T : NULL;
+        if (tie) memset(tie, 0, (size_t)T);
+        int* depth = (int*)malloc(sizeof(int) * (size_t)T);
+        const int st = validate_accept_inputs(par, tok, n, T, V, max_depth, depth);
+        if (status) status[b] = st;
+        if (st) {
+            accept_len[b] = -1;
+            next_token[b] = -1;
+            for (int j = 0; j <= max_depth; ++j) pth[j] = -1;
+            free(depth);
+            continue;
+        }
+        double* p = (double*)malloc(sizeof(double) * (size_t)V);
+        double* q = (double*)malloc(sizeof(double) * (size_t)V);
+        int cur = 0;
+        for (;;) {
+            /* S1 */
+            const float* x = logits + ((size_t)b * T + cur) * V;
+            const float* dq = dprobs + ((size_t)b * T + cur) * V;
+            double mx = -INFINITY;
+            for (int v = 0; v < V; ++v)
+                if ((double)x[v] > mx) mx = (double)x[v];
+            double den = 0.0;
+            for (int v = 0; v < V; ++v) {
+                p[v] = exp(((double)x[v] - mx) / tau);
+                den += p[v];
+            }
+            for (int v = 0; v < V; ++v) {
+                p[v] /= den;
+                q[v] = (double)dq[v];
+            }
+            /* S2 / S3 */
+            int accepted = -1;
+            for (int c = cur + 1; c < n && accepted < 0; ++c) {
+                if (par[c] != cur) continue;
+                const int xt = tok[c];
+                double ratio;
+                if (q[xt] > 0.0)
+                    ratio = p[xt] / q[xt];
+                else
+                    ratio = (p[xt] > 0.0) ? INFINITY : 0.0;
+                const double uc = (double)u[c];
+                if (tie && fabs(ratio - uc) < 1e-6) tie[c] = 1;
+                const double thr = ratio < 1.0 ? ratio : 1.0;
+                if (uc < thr) {
+                    accepted = c;
+                    break;
+                }
+                double mass = 0.0;
+                for (int v = 0; v < V; ++v) {
+                    const double r = p[v] - q[v];
+                    mass += (r > 0.0) ? r : 0.0;
+                }
+                if (mass > 0.0)
+                    for (int v = 0; v < V; ++v) {
+                        const double r = p[v] - q[v];
+                        p[v] = (r > 0.0) ? r / mass : 0.0;
+                    }
+                q[xt] = 0.0;
+                double qs = 0.0;
+                for (int v = 0; v < V; ++v) qs += q[v];
+                if (!(qs > 0.0)) break;
+                for (int v = 0; v < V; ++v) q[v] /= qs;
+            }
+            if (accepted >= 0) {
+                cur = accepted;
+                continue;
+            }
+            /* S4 */
+            double tot = 0.0;
+            for (int v = 0; v < V; ++v) tot += p[v];
+            const double target = (double)u[0] * tot;
+            double run = 0.0;
+            int pick = -1, last_pos = 0;
+            for (int v = 0; v < V; ++v) {
+                if (p[v] > 0.0) last_pos = v;
+                run += p[v];
+                if (run > target) {
+                    pick = v;
+                    break;
+                }
+            }
+            next_token[b] = (pick >= 0) ? pick : last_pos;
+            break;
+        }
+        accept_len[b] = write_path(par, cur, depth, max_depth, pth);
+        free(p);
+        free(q);
+        free(depth);
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Compaction of the accepted path (Section 3.2, last paragraph: accepted     */
+/* tokens and their features are kept for the next drafting phase).            */
+/*                                                                           */
+/* Every cache is [B,Hkv,C,d] with elem_bytes per element.  For j = 0..a:     */
+/* slot L_b + j  <-  old slot L_b + path[j]  (copied from a snapshot of the   */
+/* T tree slots, so the order of the copies cannot matter);                   */
+/* feat_out[b,j,:] = feat_in[b,path[j],:]; cache_len[b] = L_b + a + 1.        */
+/* A sequence with accept_len < 0 is skipped.                                 */
+/* ------------------------------------------------------------------------- */
+int s4c_oracle_kv_compact(uint8_t* const* k_caches, uint8_t* const* v_caches, int n_layers,
+                          int32_t* cache_len, const int32_t* path, const int32_t* accept_len,
+                          int max_depth, const uint8_t* feat_in, uint8_t* feat_out, int B, int T,
+                          int Hkv, int d, int C, int hid, int elem_bytes, int32_t* status) {
+    if (!cache_len || !path || !accept_len) return 1;
+    if (n_layers > 0 && (!k_caches || !v_caches)) return 1;
+    if (B < 0 || T < 1 || Hkv < 1 || d < 1 || C < 1 || max_depth < 0 || elem_bytes < 1) return 2;
+    const size_t row = (size_t)d * elem_bytes;
+    const size_t frow = (size_t)hid * elem_bytes;
+    uint8_t* snap = (uint8_t*)malloc(row * (size_t)T);
+    for (int b = 0; b < B; ++b) {
+        const int a = accept_len[b];
+        const int L = cache_len[b];
+        const int32_t* pth = path + (size_t)b * (max_depth + 1);
+        int st = ORC_SEQ_OK;
+        if (a < 0) {
+            if (status) status[b] = st;
+            continue;
+        }
+        if (a > max_depth) st |= ORC_SEQ_DEPTH;
+        if (L < 0 || (long)L + T > (long)C) st |= ORC_SEQ_CAPACITY;
+        if (!st) {
+            for (int j = 0; j <= a; ++j) {
+                if (pth[j] < j || pth[j] >= T) st |= ORC_SEQ_BAD_PATH;
+                if (j > 0 && pth[j] <= pth[j - 1]) st |= ORC_SEQ_BAD_PATH;
+            }
+            if (pth[0] != 0) st |= ORC_SEQ_BAD_PATH;
+        }
+        if (status) status[b] = st;
+        if (st) continue;
+        for (int l = 0; l < n_layers; ++l)
+            for (int kv = 0; kv < 2; ++kv) {
+                uint8_t* cache = kv ? v_caches[l] : k_caches[l];
+                for (int h = 0; h < Hkv; ++h) {
+                    uint8_t* base = cache + (((size_t)b * Hkv + h) * C + L) * row;
+                    memcpy(snap, base, row * (size_t)T);
+                    for (int j = 0; j <= a; ++j)
+                        memcpy(base + (size_t)j * row, snap + (size_t)pth[j] * row, row);
+                }
+            }
+        if (feat_in && feat_out)
+            for (int j = 0; j <= a; ++j)
+                memcpy(feat_out + ((size_t)b * (max_depth + 1) + j) * frow,
+                       feat_in + ((size_t)b * T + pth[j]) * frow, frow);
+        cache_len[b] = L + a + 1;
+    }
+    free(snap);
+    return 0;
+}
