@@ -1,0 +1,164 @@
+/*
+ * s4c.h -- C ABI of libs4c.so: the verify step of S4C speculative decoding
+ * (arXiv 2506.14158) as hand-written CUDA kernels for NVIDIA B200 (sm_100a).
+ *
+ * One verify step of the target model over the continuous verification tree
+ * (Section 3.2) is three calls, all asynchronous on one CUDA stream:
+ *
+ *   per decoder layer:  s4c_tree_attention   tree-masked attention of the T tree tokens
+ *   once per step:      s4c_tree_accept      greedy / speculative-sampling acceptance + path walk
+ *   once per step:      s4c_kv_compact       keep the accepted path's K/V (all layers) and features
+ *
+ * Conventions for every entry point
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *     The library allocates nothing; scratch memory comes from the caller, sized by the
+ *     matching *_workspace_bytes query (a host function, no CUDA call).
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *     synchronising.  Results are never read on the host by the library.
+ *   - The return value reports host-side argument validation and launch errors only.
+ *     Data-dependent problems (a malformed tree, a token outside the vocabulary, a cache
+ *     that is too short) are reported per sequence in the caller's device array
+ *     `status[B]` (S4C_SEQ_* bit flags, 0 = fine; may be NULL): the kernels skip such a
+ *     sequence, mark its outputs (accept_len = -1) and never trap or assert.
+ *   - Base pointers of tensors must be 16-byte aligned.  All tensors are dense, row-major,
+ *     innermost dimension last.
+ *   - Tree order: node 0 is the root (the last committed token, Section 3.2: "begins with
+ *     the prefix ... as the root node"), parent[0] = -1 and 0 <= parent[i] < i.  A batch may
+ *     pad trees to T nodes; n_nodes[b] gives the real count (NULL = T everywhere).
+ *   - Limits: 1 <= T <= 128, d in {64, 128}, Hq % Hkv == 0.
+ */
+#ifndef S4C_H_
+#define S4C_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    S4C_OK = 0,
+    S4C_ERR_NULL = 1,        /* a required pointer is NULL */
+    S4C_ERR_SHAPE = 2,       /* a size is out of range or inconsistent */
+    S4C_ERR_DTYPE = 3,       /* unknown s4c_dtype */
+    S4C_ERR_ALIGN = 4,       /* a tensor base pointer is not 16-byte aligned */
+    S4C_ERR_WORKSPACE = 5,   /* workspace missing or smaller than the query says */
+    S4C_ERR_UNSUPPORTED = 6, /* valid request this build has no kernel for */
+    S4C_ERR_CUDA = 7         /* a CUDA runtime call (launch, attribute) failed */
+} s4c_status;
+
+typedef enum { S4C_F32 = 0, S4C_BF16 = 1 } s4c_dtype;
+
+/* per-sequence flags written to status[b] */
+#define S4C_SEQ_OK 0
+#define S4C_SEQ_BAD_PARENT 1  /* n_nodes out of 1..T, parent[0] != -1 or parent[i] outside [0, i) */
+#define S4C_SEQ_TOKEN_RANGE 2 /* a draft token outside [0, V) */
+#define S4C_SEQ_CAPACITY 4    /* cache_len < 0 or cache_len + tree slots > C */
+#define S4C_SEQ_DEPTH 8       /* a node deeper than max_depth / accept_len > max_depth */
+#define S4C_SEQ_BAD_PATH 16   /* path not of the form 0 = path[0] < path[1] < ... < T */
+
+typedef void* s4c_stream_t; /* a cudaStream_t */
+
+/* Library version (major * 100 + minor) and a static, NUL-terminated name for a return code (host). */
+int s4c_version(void);
+const char* s4c_status_string(s4c_status code);
+
+/* ------------------------------------------------------------------------------------------
+ * s4c_tree_attention -- Section 3.2 ("a tree mask is applied") and Figure 3 (tree mask matrix);
+ * the single target forward pass that verifies all drafts at once (Sections 1 and 2).
+ *
+ * For sequence b, query head h and tree node i the output is softmax attention of q[b,h,i,:]
+ * over the cache slots 0..L_b-1 (the committed prefix, fully visible) and the slots L_b+t of the
+ * nodes t on the path root..i (i itself included); every other tree slot is masked.  KV head of
+ * query head h is h / (Hq/Hkv).  Scores are scale * <q,k>; softmax statistics and accumulation
+ * are fp32; for S4C_BF16 the probabilities are rounded to bf16 before the PV product.
+ *
+ *   q          [B,Hq,T,d]   dt     queries of the tree tokens (after positional encoding)
+ *   k_cache    [B,Hkv,C,d]  dt     keys; the tree tokens' own keys already sit at slots L_b..L_b+T-1
+ *   v_cache    [B,Hkv,C,d]  dt     values, same layout
+ *   cache_len  [B]          int32  L_b, the committed length (tree slots not counted)
+ *   parent     [B,T]        int32
+ *   n_nodes    [B] or NULL  int32
+ *   out        [B,Hq,T,d]   dt     rows of padding nodes (i >= n_nodes[b]) are written as zeros;
+ *                                  rows of a flagged sequence are left untouched
+ *   scale      0 selects 1/sqrt(d)
+ *   status     [B] or NULL  int32  S4C_SEQ_BAD_PARENT, S4C_SEQ_CAPACITY
+ *   workspace  at least s4c_tree_attention_workspace_bytes(...) bytes, 256-byte aligned; holds the
+ *              split-KV partial results; contents are scratch, nothing needs clearing.
+ * Calls sharing a workspace must be ordered on the stream.
+ * ------------------------------------------------------------------------------------------ */
+size_t s4c_tree_attention_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt);
+
+s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                              void* out, int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt,
+                              float scale, int32_t* status, void* workspace, size_t workspace_bytes,
+                              s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * s4c_tree_accept -- Section 2 "Speculative Sampling" (accept with probability min(1, p/q), else
+ * resample from norm(max(0, p - q))), Eq. 11 and Eq. 12 of Section 3.2, the longest accepted path
+ * of Section 3.2, and greedy decoding as used in Section 4.1.2.
+ *
+ * temperature == 0: greedy.  g[n] = argmax_v target_logits[b,n,v] (lowest v on ties); node i is
+ *   accepted iff its parent is and tokens[b,i] == g[parent]; the deepest accepted node e (lowest
+ *   index among equals) ends the path and next_token = g[e].
+ * temperature > 0: speculative sampling along the tree.  At the current node (root first) with
+ *   p = softmax(target_logits[b,cur,:]/temperature) and q = draft_probs[b,cur,:], the children are
+ *   tried in index order: child c with token x is accepted iff uniforms[b,c] < min(1, p(x)/q(x))
+ *   (strict; q(x) = 0 counts as +inf when p(x) > 0, else 0).  After a rejection p becomes
+ *   norm(max(p - q, 0)) (kept if that mass is 0) and q loses x and is renormalised.  When no child
+ *   is accepted, next_token is the smallest v whose running sum of p exceeds uniforms[b,0] * sum(p).
+ *   Sums and ratios are evaluated in float64.
+ *
+ *   target_logits [B,T,V] f32   row n: the target's logits for the token that follows node n
+ *   draft_probs   [B,T,V] f32   row n: the distribution the children of n were proposed from, at this
+ *                               temperature; may be NULL iff temperature == 0
+ *   tokens        [B,T]   int32 tokens[b,0] is the root's token (committed, never tested)
+ *   uniforms      [B,T]   f32   in [0,1); entry i >= 1: acceptance draw of node i; entry 0: final-token
+ *                               draw; may be NULL iff temperature == 0
+ *   max_depth     path buffers hold max_depth+1 entries; a deeper tree is flagged S4C_SEQ_DEPTH
+ *   accept_len    [B]   int32  out: a = number of accepted draft tokens (-1 for a flagged sequence)
+ *   path          [B,max_depth+1] int32 out: node indices root..e, path[b,0] = 0, -1 beyond a
+ *   next_token    [B]   int32  out: the bonus / resampled token (-1 for a flagged sequence)
+ *   near_tie      [B,T] uint8  out or NULL: 1 where node i was tested with |p/q - u| < 1e-6
+ *   status        [B] or NULL  S4C_SEQ_BAD_PARENT, S4C_SEQ_TOKEN_RANGE, S4C_SEQ_DEPTH
+ *   workspace     at least s4c_tree_accept_workspace_bytes(B,T,V) bytes, 256-byte aligned, scratch.
+ * Returns S4C_ERR_SHAPE for temperature < 0 or NaN.
+ * ------------------------------------------------------------------------------------------ */
+size_t s4c_tree_accept_workspace_bytes(int B, int T, int V);
+
+s4c_status s4c_tree_accept(const float* target_logits, const float* draft_probs, const int32_t* tokens,
+                           const int32_t* parent, const int32_t* n_nodes, float temperature,
+                           const float* uniforms, int B, int T, int V, int max_depth,
+                           int32_t* accept_len, int32_t* path, int32_t* next_token, uint8_t* near_tie,
+                           int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * s4c_kv_compact -- Section 3.2, last paragraph: accepted tokens and their features are kept for
+ * the following drafting phase (feature reuse, Section 1; "feature" = hidden state before the
+ * LM head, Section 2 Notations).
+ *
+ * For every layer, KV head and j = 0..a (a = accept_len[b]): cache slot L_b + j receives the old
+ * contents of slot L_b + path[b,j], for K and V, in place; feat_out[b,j,:] = feat_in[b,path[b,j],:];
+ * finally cache_len[b] = L_b + a + 1.  Slots >= the new length are unspecified afterwards; slots
+ * < L_b and other sequences' rows are never written.  A sequence with accept_len[b] < 0 is skipped.
+ *
+ *   k_caches, v_caches  device arrays of n_layers device pointers, each cache [B,Hkv,C,d] dt
+ *                       (n_layers may be 0, the arrays then may be NULL)
+ *   cache_len   [B] int32  in: L_b   out: L_b + a + 1
+ *   path        [B,max_depth+1] int32, accept_len [B] int32: as written by s4c_tree_accept
+ *   feat_in     [B,T,hid] dt or NULL;  feat_out [B,max_depth+1,hid] dt or NULL (rows > a untouched)
+ *   status      [B] or NULL  S4C_SEQ_CAPACITY (L_b + T > C), S4C_SEQ_DEPTH, S4C_SEQ_BAD_PATH
+ * d * sizeof(dt) and hid * sizeof(dt) must be multiples of 16 bytes (rows move as 16-byte words).
+ * ------------------------------------------------------------------------------------------ */
+s4c_status s4c_kv_compact(void* const* k_caches, void* const* v_caches, int n_layers, int32_t* cache_len,
+                          const int32_t* path, const int32_t* accept_len, int max_depth,
+                          const void* feat_in, void* feat_out, int B, int T, int Hkv, int d, int C, int hid,
+                          s4c_dtype dt, int32_t* status, s4c_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S4C_H_ */

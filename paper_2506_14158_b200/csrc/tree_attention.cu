@@ -1,0 +1,42 @@
+// s4c_tree_attention: argument validation and kernel selection.
+#include <math.h>
+
+#include "tree_attention.cuh"
+
+namespace s4c {
+
+static s4c_status check_shapes(int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt) {
+    if (dt != S4C_F32 && dt != S4C_BF16) return S4C_ERR_DTYPE;
+    if (B < 0 || B > 65535 || T < 1 || T > S4C_MAX_T || Hq < 1 || Hkv < 1 || Hq > 65535 || Hq % Hkv != 0 || C < 1)
+        return S4C_ERR_SHAPE;
+    if (d != 64 && d != 128) return S4C_ERR_SHAPE;
+    return S4C_OK;
+}
+
+}  // namespace s4c
+
+extern "C" size_t s4c_tree_attention_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt) {
+    using namespace s4c;
+    if (check_shapes(B, T, Hq, Hkv, d, C, dt) != S4C_OK || B == 0) return 0;
+    return simt_workspace_bytes(B, T, Hq, d, C);
+}
+
+extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                                         const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                         void* out, int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt,
+                                         float scale, int32_t* status, void* workspace, size_t workspace_bytes,
+                                         s4c_stream_t stream_) {
+    using namespace s4c;
+    const s4c_status st = check_shapes(B, T, Hq, Hkv, d, C, dt);
+    if (st != S4C_OK) return st;
+    if (!q || !k_cache || !v_cache || !cache_len || !parent || !out) return S4C_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return S4C_ERR_ALIGN;
+    if (!(scale >= 0.f) || isinf(scale)) return S4C_ERR_SHAPE;
+    if (B == 0) return S4C_OK;
+    if (scale == 0.f) scale = 1.f / sqrtf((float)d);
+    const size_t need = s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt);
+    if (need > 0 && (!workspace || workspace_bytes < need || !aligned256(workspace))) return S4C_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    return tree_attention_simt(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, dt, scale,
+                               status, workspace, stream);
+}

@@ -1,0 +1,204 @@
+"""ctypes binding of ``libs4c.so`` -- argument marshalling only; every step runs in the library's CUDA kernels.
+
+The functions mirror the C ABI declared in ``include/s4c.h`` (same names, same argument meaning).  Tensors are
+torch CUDA tensors used purely as device buffers: the binding checks dtype / contiguity / device, passes raw
+pointers and the current CUDA stream, and raises :class:`S4CError` on a non-zero return code.  There is no
+CPU fallback: importing this module fails if the library has not been built, and calls fail on CPU tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+from ._build import lib_path
+
+F32, BF16 = 0, 1
+SEQ_OK, SEQ_BAD_PARENT, SEQ_TOKEN_RANGE, SEQ_CAPACITY, SEQ_DEPTH, SEQ_BAD_PATH = 0, 1, 2, 4, 8, 16
+STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WORKSPACE", "ERR_UNSUPPORTED", "ERR_CUDA"]
+
+EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
+           "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_kv_compact"]
+
+
+class S4CError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        msg = _lib.s4c_status_string(code).decode() if _lib is not None else ""
+        name = STATUS_NAMES[code] if 0 <= code < len(STATUS_NAMES) else str(code)
+        super().__init__(f"{fn} returned S4C_{name}: {msg}")
+
+
+def _load() -> ctypes.CDLL:
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(path)
+    vp, i32p, i, f, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.s4c_version.restype = i
+    lib.s4c_status_string.restype = ctypes.c_char_p
+    lib.s4c_status_string.argtypes = [i]
+    lib.s4c_tree_attention_workspace_bytes.restype = sz
+    lib.s4c_tree_attention_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
+    lib.s4c_tree_attention.restype = i
+    lib.s4c_tree_attention.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_tree_accept_workspace_bytes.restype = sz
+    lib.s4c_tree_accept_workspace_bytes.argtypes = [i, i, i]
+    lib.s4c_tree_accept.restype = i
+    lib.s4c_tree_accept.argtypes = [vp, vp, i32p, i32p, i32p, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp, sz, vp]
+    lib.s4c_kv_compact.restype = i
+    lib.s4c_kv_compact.argtypes = [vp, vp, i, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i32p, vp]
+    return lib
+
+
+_lib = None
+_lib = _load()
+
+
+def version() -> int:
+    return int(_lib.s4c_version())
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: the library takes float32 or bfloat16")
+
+
+def _dev(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+_ws_cache = {}
+
+
+def _workspace(nbytes: int, device, tag: str) -> Optional[torch.Tensor]:
+    """A cached scratch buffer per (device, call family); reused by calls ordered on one stream."""
+    if nbytes == 0:
+        return None
+    key = (str(device), tag)
+    buf = _ws_cache.get(key)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        _ws_cache[key] = buf
+    return buf
+
+
+def tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dtype) -> int:
+    dt = F32 if dtype == torch.float32 else BF16
+    return int(_lib.s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt))
+
+
+def tree_attention(q, k_cache, v_cache, cache_len, parent, n_nodes=None, out=None, scale: float = 0.0, status=None,
+                   workspace=None, stream=None):
+    """s4c_tree_attention: q [B,Hq,T,d], k_cache/v_cache [B,Hkv,C,d] -> out [B,Hq,T,d] (same dtype)."""
+    B, Hq, T, d = q.shape
+    _, Hkv, C, _ = k_cache.shape
+    if k_cache.shape != (B, Hkv, C, d) or v_cache.shape != (B, Hkv, C, d):
+        raise ValueError("k_cache / v_cache must be [B,Hkv,C,d]")
+    if k_cache.dtype != q.dtype or v_cache.dtype != q.dtype:
+        raise TypeError("q, k_cache and v_cache must share one dtype")
+    if out is None:
+        out = torch.empty_like(q)
+    dt = _dt(q)
+    need = int(_lib.s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt))
+    if workspace is None:
+        workspace = _workspace(need, q.device, "attn")
+    rc = _lib.s4c_tree_attention(
+        _dev(q, name="q"), _dev(k_cache, name="k_cache"), _dev(v_cache, name="v_cache"),
+        _dev(cache_len, torch.int32, "cache_len"), _dev(parent, torch.int32, "parent"),
+        _dev(n_nodes, torch.int32, "n_nodes"), _dev(out, q.dtype, "out"), B, T, Hq, Hkv, d, C, dt, float(scale),
+        _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+        0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_attention", rc)
+    return out
+
+
+def tree_accept_workspace_bytes(B, T, V) -> int:
+    return int(_lib.s4c_tree_accept_workspace_bytes(B, T, V))
+
+
+def tree_accept(target_logits, draft_probs, tokens, parent, temperature: float, uniforms=None, n_nodes=None,
+                max_depth: Optional[int] = None, accept_len=None, path=None, next_token=None, near_tie=None,
+                status=None, workspace=None, stream=None):
+    """s4c_tree_accept: returns dict(accept_len [B], path [B,max_depth+1], next_token [B], near_tie [B,T], status [B])."""
+    B, T, V = target_logits.shape
+    dev = target_logits.device
+    if max_depth is None:
+        max_depth = T - 1
+    i32 = dict(dtype=torch.int32, device=dev)
+    accept_len = torch.empty(B, **i32) if accept_len is None else accept_len
+    path = torch.empty(B, max_depth + 1, **i32) if path is None else path
+    next_token = torch.empty(B, **i32) if next_token is None else next_token
+    near_tie = torch.empty(B, T, dtype=torch.uint8, device=dev) if near_tie is None else near_tie
+    status = torch.empty(B, **i32) if status is None else status
+    need = int(_lib.s4c_tree_accept_workspace_bytes(B, T, V))
+    if workspace is None:
+        workspace = _workspace(need, dev, "accept")
+    rc = _lib.s4c_tree_accept(
+        _dev(target_logits, torch.float32, "target_logits"), _dev(draft_probs, torch.float32, "draft_probs"),
+        _dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"),
+        float(temperature), _dev(uniforms, torch.float32, "uniforms"), B, T, V, int(max_depth),
+        _dev(accept_len, torch.int32, "accept_len"), _dev(path, torch.int32, "path"),
+        _dev(next_token, torch.int32, "next_token"), _dev(near_tie, torch.uint8, "near_tie"),
+        _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+        0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_accept", rc)
+    return dict(accept_len=accept_len, path=path, next_token=next_token, near_tie=near_tie, status=status)
+
+
+def cache_pointer_array(caches: Sequence[torch.Tensor]) -> torch.Tensor:
+    """Device array of the layers' cache base pointers (int64), as s4c_kv_compact expects."""
+    if not caches:
+        return torch.zeros(1, dtype=torch.int64, device="cuda")
+    for c in caches:
+        _dev(c, caches[0].dtype, "cache")
+        if c.shape != caches[0].shape:
+            raise ValueError("all layer caches must share one shape")
+    return torch.tensor([c.data_ptr() for c in caches], dtype=torch.int64, device=caches[0].device)
+
+
+def kv_compact(k_ptrs, v_ptrs, n_layers: int, cache_shape, dtype, cache_len, path, accept_len, T: int,
+               feat_in=None, feat_out=None, status=None, stream=None):
+    """s4c_kv_compact.  k_ptrs / v_ptrs: device int64 arrays from :func:`cache_pointer_array`;
+    cache_shape = (B,Hkv,C,d); cache_len is updated in place.  Returns status [B]."""
+    B, Hkv, C, d = cache_shape
+    max_depth = path.shape[1] - 1
+    dt = F32 if dtype == torch.float32 else BF16
+    if status is None:
+        status = torch.empty(B, dtype=torch.int32, device=cache_len.device)
+    hid = 0
+    if feat_in is not None:
+        if feat_in.dtype != dtype or feat_out is None or feat_out.dtype != dtype:
+            raise TypeError("features must have the cache dtype")
+        if feat_in.shape[:2] != (B, T) or feat_out.shape != (B, max_depth + 1, feat_in.shape[2]):
+            raise ValueError("feat_in must be [B,T,hid] and feat_out [B,max_depth+1,hid]")
+        hid = feat_in.shape[2]
+    rc = _lib.s4c_kv_compact(
+        _dev(k_ptrs, torch.int64, "k_ptrs") if n_layers else None, _dev(v_ptrs, torch.int64, "v_ptrs") if n_layers else None,
+        int(n_layers), _dev(cache_len, torch.int32, "cache_len"), _dev(path, torch.int32, "path"),
+        _dev(accept_len, torch.int32, "accept_len"), max_depth, _dev(feat_in, name="feat_in"),
+        _dev(feat_out, name="feat_out"), B, T, Hkv, d, C, hid, dt, _dev(status, torch.int32, "status"), _stream(stream))
+    if rc:
+        raise S4CError("s4c_kv_compact", rc)
+    return status

@@ -1,0 +1,162 @@
+"""One whole S4C verify step on device buffers: n_layers x s4c_tree_attention, s4c_tree_accept, s4c_kv_compact.
+
+:class:`VerifyStep` owns nothing but references to the caller's tensors plus the small output / scratch tensors
+it allocates once.  ``run()`` enqueues the step on the current stream through the C ABI; ``capture()`` records
+the same launches into a CUDA graph so that a replay costs one host call (the step is 34 tiny launches at the
+7B shape -- launch-bound from Python otherwise).  ``run_host()`` is the end-to-end form: the step's per-step
+inputs arrive in pinned host memory, are copied in, the step runs, and the decision is copied back.
+All arithmetic happens inside libs4c's kernels.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import torch
+
+from . import s4c
+
+
+class VerifyStep:
+    def __init__(self, q: List[torch.Tensor], k_caches: List[torch.Tensor], v_caches: List[torch.Tensor],
+                 cache_len: torch.Tensor, parent: torch.Tensor, tokens: torch.Tensor, target_logits: torch.Tensor,
+                 draft_probs: Optional[torch.Tensor], uniforms: Optional[torch.Tensor], temperature: float,
+                 max_depth: int, n_nodes: Optional[torch.Tensor] = None, feat_in: Optional[torch.Tensor] = None):
+        self.n_layers = len(q)
+        assert len(k_caches) == self.n_layers and len(v_caches) == self.n_layers
+        self.q, self.k_caches, self.v_caches = q, k_caches, v_caches
+        self.cache_len0 = cache_len
+        self.parent, self.tokens, self.n_nodes = parent, tokens, n_nodes
+        self.logits, self.draft_probs, self.uniforms = target_logits, draft_probs, uniforms
+        self.temperature, self.max_depth = float(temperature), int(max_depth)
+        self.feat_in = feat_in
+        dev = cache_len.device
+        B, T, V = target_logits.shape
+        self.B, self.T, self.V = B, T, V
+        self.cache_shape = tuple(k_caches[0].shape)
+        self.dtype = k_caches[0].dtype
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.cache_len = cache_len.clone()            # working copy: the step advances it in place
+        self.attn_out = [torch.empty_like(t) for t in q]
+        self.accept_len = torch.empty(B, **i32)
+        self.path = torch.empty(B, self.max_depth + 1, **i32)
+        self.next_token = torch.empty(B, **i32)
+        self.near_tie = torch.empty(B, T, dtype=torch.uint8, device=dev)
+        self.status_attn = torch.empty(B, **i32)
+        self.status_accept = torch.empty(B, **i32)
+        self.status_compact = torch.empty(B, **i32)
+        self.feat_out = None if feat_in is None else torch.zeros(B, self.max_depth + 1, feat_in.shape[2],
+                                                                 dtype=feat_in.dtype, device=dev)
+        _, Hq, _, d = q[0].shape
+        _, Hkv, C, _ = self.cache_shape
+        self.ws_attn = torch.empty(max(1, s4c.tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, self.dtype)),
+                                   dtype=torch.uint8, device=dev)
+        self.ws_accept = torch.empty(max(1, s4c.tree_accept_workspace_bytes(B, T, V)), dtype=torch.uint8, device=dev)
+        self.k_ptrs = s4c.cache_pointer_array(k_caches)
+        self.v_ptrs = s4c.cache_pointer_array(v_caches)
+        self.graph: Optional[torch.cuda.CUDAGraph] = None
+        self._host = None
+
+    # ------------------------------------------------------------------ the three stages
+    def attention(self):
+        for l in range(self.n_layers):
+            s4c.tree_attention(self.q[l], self.k_caches[l], self.v_caches[l], self.cache_len, self.parent, self.n_nodes,
+                               out=self.attn_out[l], status=self.status_attn, workspace=self.ws_attn)
+
+    def accept(self):
+        s4c.tree_accept(self.logits, self.draft_probs, self.tokens, self.parent, self.temperature, self.uniforms,
+                        self.n_nodes, self.max_depth, self.accept_len, self.path, self.next_token, self.near_tie,
+                        self.status_accept, self.ws_accept)
+
+    def compact(self):
+        s4c.kv_compact(self.k_ptrs, self.v_ptrs, self.n_layers, self.cache_shape, self.dtype, self.cache_len, self.path,
+                       self.accept_len, self.T, self.feat_in, self.feat_out, self.status_compact)
+
+    def reset_lengths(self):
+        """Rewind the working cache length to the committed length (so that a benchmark can repeat the step)."""
+        self.cache_len.copy_(self.cache_len0)
+
+    def run(self):
+        self.reset_lengths()
+        self.attention()
+        self.accept()
+        self.compact()
+
+    # kernels launched by one run(): used by the benchmark to report its launch count
+    def launches_per_step(self, attn_launches_per_layer: int) -> int:
+        accept = 3 if self.temperature > 0 else 2
+        compact = 2 if self.n_layers > 0 else 1
+        return self.n_layers * attn_launches_per_layer + accept + compact
+
+    # ------------------------------------------------------------------ CUDA graph
+    def capture(self, what: str = "step") -> torch.cuda.CUDAGraph:
+        fn = {"step": self.run, "attention": self.attention, "accept": self.accept,
+              "compact": lambda: (self.reset_lengths(), self.compact())}[what]
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            fn()  # warm-up outside capture (first-launch module loading must not happen while capturing)
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        if what == "step":
+            self.graph = g
+        return g
+
+    # ------------------------------------------------------------------ end to end from host memory
+    def bind_host_inputs(self):
+        """Allocate pinned host mirrors of the per-step inputs and outputs; returns (inputs dict, outputs dict).
+
+        Per-step inputs: queries and the tree tokens' K/V rows of every layer, the tree, the draft tokens,
+        target logits, draft probabilities, uniforms and features.  The committed cache prefix is state that
+        lives on the device across steps and is not copied.
+        """
+        pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+        L = int(self.cache_len0.max().item())
+        assert int(self.cache_len0.min().item()) == L, "run_host expects one committed length for the batch"
+        T = self.T
+        inp = dict(q=[pin(t) for t in self.q],
+                   k_tree=[pin(c[:, :, L:L + T]) for c in self.k_caches],
+                   v_tree=[pin(c[:, :, L:L + T]) for c in self.v_caches],
+                   parent=pin(self.parent), tokens=pin(self.tokens), logits=pin(self.logits))
+        if self.draft_probs is not None:
+            inp["draft_probs"] = pin(self.draft_probs)
+            inp["uniforms"] = pin(self.uniforms)
+        if self.feat_in is not None:
+            inp["feat_in"] = pin(self.feat_in)
+        out = dict(accept_len=pin(self.accept_len), path=pin(self.path), next_token=pin(self.next_token),
+                   cache_len=pin(self.cache_len), status=pin(self.status_accept))
+        self._host = (inp, out, L)
+        nbytes = lambda x: sum(t.numel() * t.element_size() for t in (x if isinstance(x, list) else [x]))
+        self.h2d_bytes = sum(nbytes(v) for v in inp.values())
+        self.d2h_bytes = sum(nbytes(v) for v in out.values())
+        return inp, out
+
+    def run_host(self):
+        """Copy the per-step inputs in (async, pinned), run the step, copy the decision back, and wait for it."""
+        inp, out, L = self._host
+        T = self.T
+        for l in range(self.n_layers):
+            self.q[l].copy_(inp["q"][l], non_blocking=True)
+            self.k_caches[l][:, :, L:L + T].copy_(inp["k_tree"][l], non_blocking=True)
+            self.v_caches[l][:, :, L:L + T].copy_(inp["v_tree"][l], non_blocking=True)
+        self.parent.copy_(inp["parent"], non_blocking=True)
+        self.tokens.copy_(inp["tokens"], non_blocking=True)
+        self.logits.copy_(inp["logits"], non_blocking=True)
+        if self.draft_probs is not None:
+            self.draft_probs.copy_(inp["draft_probs"], non_blocking=True)
+            self.uniforms.copy_(inp["uniforms"], non_blocking=True)
+        if self.feat_in is not None:
+            self.feat_in.copy_(inp["feat_in"], non_blocking=True)
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.run()
+        out["accept_len"].copy_(self.accept_len, non_blocking=True)
+        out["path"].copy_(self.path, non_blocking=True)
+        out["next_token"].copy_(self.next_token, non_blocking=True)
+        out["cache_len"].copy_(self.cache_len, non_blocking=True)
+        out["status"].copy_(self.status_accept, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return out

@@ -1,0 +1,92 @@
+"""Host-side checks of the C ABI: the library loads, exports everything include/s4c.h declares, sizes its
+workspaces on the host and rejects bad arguments before touching CUDA.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "s4c.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(s4c_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(s4c_lib):
+    lib = ctypes.CDLL(s4c_lib)
+    names = _declared_functions()
+    assert "s4c_tree_attention" in names and "s4c_tree_accept" in names and "s4c_kv_compact" in names
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in include/s4c.h but not exported"
+    from paper_2506_14158_b200 import s4c
+
+    assert sorted(s4c.EXPORTS) == names
+    assert s4c.version() >= 100
+
+
+def test_sequence_flags_agree_between_header_binding_and_oracle(s4c_lib):
+    from paper_2506_14158_b200 import s4c
+
+    text = open(os.path.join(ROOT, "include", "s4c.h")).read()
+    flags = {k: int(v) for k, v in re.findall(r"#define\s+S4C_(SEQ_[A-Z_]+)\s+(\d+)", text)}
+    assert flags == {"SEQ_OK": 0, "SEQ_BAD_PARENT": 1, "SEQ_TOKEN_RANGE": 2, "SEQ_CAPACITY": 4, "SEQ_DEPTH": 8,
+                     "SEQ_BAD_PATH": 16}
+    for k, v in flags.items():
+        assert getattr(s4c, k) == v and getattr(oracle, k) == v
+
+
+def test_workspace_queries_are_host_functions(s4c_lib):
+    from paper_2506_14158_b200 import s4c
+
+    assert s4c.tree_accept_workspace_bytes(1, 26, 32000) > 0
+    assert s4c.tree_accept_workspace_bytes(4, 64, 128256) % 256 == 0
+    assert s4c.tree_accept_workspace_bytes(0, 1, 1) == 0
+    import torch
+
+    w = s4c.tree_attention_workspace_bytes(1, 26, 32, 32, 128, 1152, torch.bfloat16)
+    assert w > 0 and w % 256 == 0
+    assert s4c.tree_attention_workspace_bytes(1, 200, 32, 32, 128, 1152, torch.bfloat16) == 0  # T > 128: invalid
+
+
+def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
+    lib = ctypes.CDLL(s4c_lib)
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.s4c_tree_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp, vp, sz, vp]
+    lib.s4c_tree_accept.argtypes = [vp, vp, vp, vp, vp, f, vp, i, i, i, i, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.s4c_kv_compact.argtypes = [vp, vp, i, vp, vp, vp, i, vp, vp, i, i, i, i, i, i, i, vp, vp]
+    lib.s4c_status_string.restype = ctypes.c_char_p
+    P = 4096  # a fake, 16-byte aligned "pointer": rejected calls never dereference or launch
+    att = lambda **kw: lib.s4c_tree_attention(*[kw.get(k, d) for k, d in [
+        ("q", P), ("k", P), ("v", P), ("cl", P), ("par", P), ("nn", None), ("out", P), ("B", 1), ("T", 8), ("Hq", 4),
+        ("Hkv", 2), ("d", 128), ("C", 256), ("dt", 1), ("scale", 0.0), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
+    assert att(q=None) == 1                      # S4C_ERR_NULL
+    assert att(T=129) == 2 and att(T=0) == 2     # S4C_ERR_SHAPE
+    assert att(Hq=4, Hkv=3) == 2 and att(d=96) == 2
+    assert att(dt=5) == 3                        # S4C_ERR_DTYPE
+    assert att(k=P + 2) == 4                     # S4C_ERR_ALIGN
+    assert att(scale=-1.0) == 2
+    assert att(B=0) == 0
+    assert att(Hq=32, Hkv=32, C=4096, ws=None) == 5  # needs a workspace: S4C_ERR_WORKSPACE
+    acc = lambda **kw: lib.s4c_tree_accept(*[kw.get(k, d) for k, d in [
+        ("lg", P), ("dp", P), ("tok", P), ("par", P), ("nn", None), ("tau", 1.0), ("u", P), ("B", 1), ("T", 8),
+        ("V", 100), ("md", 7), ("al", P), ("path", P), ("nt", P), ("tie", None), ("st", None), ("ws", None), ("wsb", 0),
+        ("s", None)]])
+    assert acc(tau=-0.5) == 2 and acc(tau=float("nan")) == 2
+    assert acc(dp=None) == 1 and acc(u=None) == 1 and acc(lg=None) == 1
+    assert acc(T=500) == 2 and acc(V=0) == 2 and acc(md=128) == 2
+    assert acc() == 5                            # no workspace
+    assert acc(B=0) == 0
+    cmp_ = lambda **kw: lib.s4c_kv_compact(*[kw.get(k, d) for k, d in [
+        ("k", P), ("v", P), ("nl", 1), ("cl", P), ("path", P), ("al", P), ("md", 7), ("fi", None), ("fo", None), ("B", 1),
+        ("T", 8), ("Hkv", 2), ("d", 128), ("C", 256), ("hid", 0), ("dt", 1), ("st", None), ("s", None)]])
+    assert cmp_(cl=None) == 1 and cmp_(k=None) == 1
+    assert cmp_(d=100) == 2                      # rows must be whole 16-byte words
+    assert cmp_(fi=P) == 1                       # feat_in without feat_out
+    assert cmp_(dt=9) == 3
+    assert cmp_(B=0) == 0
+    assert b"workspace" in lib.s4c_status_string(5)

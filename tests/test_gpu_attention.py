@@ -1,0 +1,87 @@
+"""GPU parity: s4c_tree_attention (through the C ABI) against the float64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_14158_b200 import workloads as W
+
+from parity import ATTN_TOL, assert_attention_close, attention_both
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
+def test_named_configs(name):
+    cfg = W.CONFIGS[name]
+    q, k, v = W.make_attention_inputs(cfg)
+    parent = W.make_trees(cfg)
+    got, ref, gst, rst = attention_both(q, k, v, [cfg.L] * cfg.B, parent)
+    assert (rst == 0).all()
+    assert_attention_close(got, ref, gst, rst, ATTN_TOL[cfg.dtype])
+
+
+def _case(B, Hq, Hkv, T, d, Ls, dtype, seed, tree="random", n_nodes=None, scale=0.0, C=None):
+    rng = np.random.default_rng(seed)
+    dt = {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
+    C = C or (max(Ls) + T + 5)
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn((B, Hq, T, d), generator=g).to(dt)
+    k = torch.randn((B, Hkv, C, d), generator=g).to(dt)
+    v = torch.randn((B, Hkv, C, d), generator=g).to(dt)
+    if tree == "chain":
+        parent = np.tile(W.chain_tree(T), (B, 1))
+    elif tree == "star":
+        parent = np.tile(W.star_tree(T), (B, 1))
+    else:
+        parent = np.stack([W.random_tree(T, 8, rng) for _ in range(B)])
+    got, ref, gst, rst = attention_both(q, k, v, Ls, parent, n_nodes, scale)
+    assert_attention_close(got, ref, gst, rst, ATTN_TOL[dtype])
+    return got, ref
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [64, 128])
+def test_ragged_lengths_gqa_and_padding(dtype, d):
+    # cache lengths that are not multiples of any tile, several tiles long, one empty prefix; padded trees
+    _case(B=3, Hq=8, Hkv=2, T=37, d=d, Ls=[0, 333, 130], dtype=dtype, seed=1, n_nodes=[37, 5, 20])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("tree", ["chain", "star"])
+def test_chain_and_star_trees(dtype, tree):
+    _case(B=1, Hq=4, Hkv=4, T=33, d=128, Ls=[257], dtype=dtype, seed=2, tree=tree, scale=0.11)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_extreme_tree_sizes(dtype):
+    _case(B=2, Hq=2, Hkv=1, T=1, d=128, Ls=[64, 1], dtype=dtype, seed=3)            # plain decode
+    _case(B=1, Hq=2, Hkv=2, T=128, d=128, Ls=[700], dtype=dtype, seed=4)            # the maximum tree
+    _case(B=1, Hq=4, Hkv=1, T=128, d=64, Ls=[0], dtype=dtype, seed=5, tree="chain")  # no prefix at all
+
+
+def test_long_context_many_splits():
+    _case(B=1, Hq=8, Hkv=8, T=16, d=128, Ls=[9000], dtype="bf16", seed=6)
+
+
+def test_flagged_sequences_are_skipped_not_trapped():
+    from parity import attention_both
+
+    g = torch.Generator().manual_seed(9)
+    B, H, T, d, C = 3, 2, 6, 128, 64
+    q = torch.randn((B, H, T, d), generator=g).to(torch.bfloat16)
+    k = torch.randn((B, H, C, d), generator=g).to(torch.bfloat16)
+    v = torch.randn((B, H, C, d), generator=g).to(torch.bfloat16)
+    parent = np.tile(W.chain_tree(T), (B, 1))
+    parent[1, 3] = 4  # parent[i] >= i
+    got, ref, gst, rst = attention_both(q, k, v, [10, 10, 60], parent)  # third: 60 + 6 > 64
+    assert gst[0] == 0 and gst[1] == 1 and gst[2] == 4
+    assert_attention_close(got, ref, gst, rst, ATTN_TOL["bf16"])
+
+
+def test_results_do_not_depend_on_scheduling():
+    cfg = W.CONFIGS["c2"]
+    q, k, v = W.make_attention_inputs(cfg)
+    parent = W.make_trees(cfg)
+    a, _, _, _ = attention_both(q, k, v, [cfg.L], parent)
+    b, _, _, _ = attention_both(q, k, v, [cfg.L], parent)
+    np.testing.assert_array_equal(a, b)
