@@ -57,6 +57,7 @@ typedef enum { S4C_F32 = 0, S4C_BF16 = 1 } s4c_dtype;
 #define S4C_SEQ_CAPACITY 4    /* cache_len < 0 or cache_len + tree slots > C */
 #define S4C_SEQ_DEPTH 8       /* a node deeper than max_depth / accept_len > max_depth */
 #define S4C_SEQ_BAD_PATH 16   /* path not of the form 0 = path[0] < path[1] < ... < T */
+#define S4C_SEQ_TIMEOUT 32    /* a bounded in-kernel wait expired (OR-ed in; results of that sequence are invalid) */
 
 typedef void* s4c_stream_t; /* a cudaStream_t */
 

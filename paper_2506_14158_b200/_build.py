@@ -49,6 +49,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.wait() != 0:
             raise RuntimeError(f"nvcc failed on {src}")
     tmp = _LIB + f".tmp{os.getpid()}"
-    subprocess.run([nvcc, "-shared", "-o", tmp, *objs, "-lcudart", "-lcuda"], check=True)
+    subprocess.run([nvcc, "-shared", "-o", tmp, *objs, "-lcudart"], check=True)
     os.replace(tmp, _LIB)
     return _LIB

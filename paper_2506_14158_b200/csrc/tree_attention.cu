@@ -18,6 +18,7 @@ static s4c_status check_shapes(int B, int T, int Hq, int Hkv, int d, int C, s4c_
 extern "C" size_t s4c_tree_attention_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt) {
     using namespace s4c;
     if (check_shapes(B, T, Hq, Hkv, d, C, dt) != S4C_OK || B == 0) return 0;
+    if (tc_supported(T, Hq, Hkv, d, dt)) return tc_workspace_bytes(B, T, Hq, Hkv, d, C);
     return simt_workspace_bytes(B, T, Hq, d, C);
 }
 
@@ -37,6 +38,9 @@ extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, con
     const size_t need = s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt);
     if (need > 0 && (!workspace || workspace_bytes < need || !aligned256(workspace))) return S4C_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (tc_supported(T, Hq, Hkv, d, dt))
+        return tree_attention_tc(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, scale, status,
+                                 workspace, stream);
     return tree_attention_simt(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, dt, scale,
                                status, workspace, stream);
 }

@@ -10,4 +10,16 @@ s4c_status tree_attention_simt(const void* q, const void* k, const void* v, cons
                                const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
                                int d, int C, s4c_dtype dt, float scale, int32_t* status, void* ws, cudaStream_t stream);
 
+// Merges split partials [B*Hq*T rows][splits][d + 2] (unnormalised output, running max in base-2 units, sum).
+s4c_status tree_attention_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                  void* out, int B, int T, int Hq, int d, int C, int splits, s4c_dtype dt,
+                                  cudaStream_t stream);
+
+// Tensor-core path (bf16, d in {64, 128}): tcgen05 / TMEM / TMA.
+bool tc_supported(int T, int Hq, int Hkv, int d, s4c_dtype dt);
+size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C);
+s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
+                             const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
+                             int d, int C, float scale, int32_t* status, void* ws, cudaStream_t stream);
+
 }  // namespace s4c

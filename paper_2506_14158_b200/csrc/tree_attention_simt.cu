@@ -184,6 +184,26 @@ size_t simt_workspace_bytes(int B, int T, int Hq, int d, int C) {
 }
 
 template <typename T_, int D>
+static s4c_status launch_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                 void* out, int B, int T, int Hq, int C, int splits, cudaStream_t stream) {
+    dim3 g2(T, Hq, B);
+    tree_attention_combine_kernel<T_, D><<<g2, D, 0, stream>>>(static_cast<const float*>(ws), cache_len, parent, n_nodes,
+                                                              static_cast<T_*>(out), T, Hq, C, splits);
+    S4C_RETURN_IF_CUDA_ERROR();
+    return S4C_OK;
+}
+
+s4c_status tree_attention_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                  void* out, int B, int T, int Hq, int d, int C, int splits, s4c_dtype dt,
+                                  cudaStream_t stream) {
+    if (dt == S4C_F32)
+        return d == 64 ? launch_combine<float, 64>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream)
+                       : launch_combine<float, 128>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream);
+    return d == 64 ? launch_combine<__nv_bfloat16, 64>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream)
+                   : launch_combine<__nv_bfloat16, 128>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream);
+}
+
+template <typename T_, int D>
 static s4c_status launch_simt(const void* q, const void* k, const void* v, const int32_t* cache_len,
                               const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
                               int C, float scale, int32_t* status, void* ws, cudaStream_t stream) {
@@ -193,12 +213,7 @@ static s4c_status launch_simt(const void* q, const void* k, const void* v, const
         static_cast<const T_*>(q), static_cast<const T_*>(k), static_cast<const T_*>(v), cache_len, parent, n_nodes,
         static_cast<T_*>(out), T, Hq, Hkv, C, scale * kLog2e, status, static_cast<float*>(ws));
     S4C_RETURN_IF_CUDA_ERROR();
-    if (splits > 1) {
-        dim3 g2(T, Hq, B);
-        tree_attention_combine_kernel<T_, D><<<g2, D, 0, stream>>>(static_cast<const float*>(ws), cache_len, parent,
-                                                                  n_nodes, static_cast<T_*>(out), T, Hq, C, splits);
-        S4C_RETURN_IF_CUDA_ERROR();
-    }
+    if (splits > 1) return launch_combine<T_, D>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream);
     return S4C_OK;
 }
 
