@@ -137,6 +137,38 @@ s4c_status s4c_tree_accept(const float* target_logits, const float* draft_probs,
                            int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * s4c_tree_accept_noalloc -- the paper has no counterpart; this is a packaging variant of
+ * s4c_tree_accept for callers that cannot provide scratch memory.
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they verify a tree: a
+ * serving loop that has handed all device memory to its own pool, a plug-in running inside
+ * another framework's allocator, code on a latency path where an allocation could block or
+ * synchronise.  For them this entry point takes the same inputs and outputs as s4c_tree_accept
+ * but no workspace: its scratch is a fixed array of S4C_NOALLOC_SCRATCH_BYTES bytes compiled into
+ * the library (so every GPU that loads the library gives up that much memory until the process
+ * exits).  The call itself allocates and frees nothing, directly or through any library.
+ *
+ *   - Size limit: s4c_tree_accept_workspace_bytes(B,T,V) must not exceed
+ *     S4C_NOALLOC_SCRATCH_BYTES (about B*T*ceil(V/4096) <= 32000 row segments); a larger problem is
+ *     refused with S4C_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on each device looks up the array's device address (a host-side runtime
+ *     query, made with that device current).  Make that first call outside any stream capture.
+ *   - All calls in the process share the one array per device, and it keeps whatever the last
+ *     call left in it.  Nothing in it needs to start at zero (every value is written before it is
+ *     read), but two calls whose kernels overlap on the GPU -- different streams, or one stream per
+ *     thread -- race on it: order such calls on one stream or with events.
+ *   - Results are identical to s4c_tree_accept on the same inputs.
+ * All other arguments, outputs, status flags and return codes are those of s4c_tree_accept.
+ * ------------------------------------------------------------------------------------------ */
+#define S4C_NOALLOC_SCRATCH_BYTES (1 << 20)
+
+s4c_status s4c_tree_accept_noalloc(const float* target_logits, const float* draft_probs, const int32_t* tokens,
+                                   const int32_t* parent, const int32_t* n_nodes, float temperature,
+                                   const float* uniforms, int B, int T, int V, int max_depth,
+                                   int32_t* accept_len, int32_t* path, int32_t* next_token, uint8_t* near_tie,
+                                   int32_t* status, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * s4c_kv_compact -- Section 3.2, last paragraph: accepted tokens and their features are kept for
  * the following drafting phase (feature reuse, Section 1; "feature" = hidden state before the
  * LM head, Section 2 Notations).

@@ -525,3 +525,30 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
     S4C_RETURN_IF_CUDA_ERROR();
     return S4C_OK;
 }
+
+// ----------------------------------------------------------------------------- no-allocation variant
+// Scratch for s4c_tree_accept_noalloc lives in the library image itself: S4C_NOALLOC_SCRATCH_BYTES of device
+// memory on every GPU that loads the library, held until the process exits.  In host code the array's name
+// is only a handle for the runtime, never a device address, so the address is looked up once per device.
+static __device__ __align__(256) unsigned char g_accept_scratch[S4C_NOALLOC_SCRATCH_BYTES];
+
+extern "C" s4c_status s4c_tree_accept_noalloc(const float* target_logits, const float* draft_probs,
+                                              const int32_t* tokens, const int32_t* parent, const int32_t* n_nodes,
+                                              float temperature, const float* uniforms, int B, int T, int V,
+                                              int max_depth, int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                              uint8_t* near_tie, int32_t* status, s4c_stream_t stream) {
+    if (B < 0 || T < 1 || T > S4C_MAX_T || V < 1) return S4C_ERR_SHAPE;
+    if (B > 0 && s4c::accept_ws_layout(B, T, V, nullptr, nullptr) > (size_t)S4C_NOALLOC_SCRATCH_BYTES)
+        return S4C_ERR_WORKSPACE;  // the problem needs more scratch than the built-in array holds
+    static void* scratch_of_device[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
+    if (!scratch_of_device[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_accept_scratch) != cudaSuccess || !p) return S4C_ERR_CUDA;
+        scratch_of_device[dev] = p;
+    }
+    return s4c_tree_accept(target_logits, draft_probs, tokens, parent, n_nodes, temperature, uniforms, B, T, V,
+                           max_depth, accept_len, path, next_token, near_tie, status, scratch_of_device[dev],
+                           (size_t)S4C_NOALLOC_SCRATCH_BYTES, stream);
+}

@@ -20,7 +20,8 @@ SEQ_OK, SEQ_BAD_PARENT, SEQ_TOKEN_RANGE, SEQ_CAPACITY, SEQ_DEPTH, SEQ_BAD_PATH, 
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WORKSPACE", "ERR_UNSUPPORTED", "ERR_CUDA"]
 
 EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
-           "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_kv_compact"]
+           "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact"]
+NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
 class S4CError(RuntimeError):
@@ -49,6 +50,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_accept_workspace_bytes.argtypes = [i, i, i]
     lib.s4c_tree_accept.restype = i
     lib.s4c_tree_accept.argtypes = [vp, vp, i32p, i32p, i32p, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp, sz, vp]
+    lib.s4c_tree_accept_noalloc.restype = i
+    lib.s4c_tree_accept_noalloc.argtypes = [vp, vp, i32p, i32p, i32p, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp]
     lib.s4c_kv_compact.restype = i
     lib.s4c_kv_compact.argtypes = [vp, vp, i, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i32p, vp]
     return lib
@@ -165,6 +168,37 @@ def tree_accept(target_logits, draft_probs, tokens, parent, temperature: float, 
     if rc:
         raise S4CError("s4c_tree_accept", rc)
     return dict(accept_len=accept_len, path=path, next_token=next_token, near_tie=near_tie, status=status)
+
+
+def tree_accept_noalloc(target_logits, draft_probs, tokens, parent, temperature: float, uniforms=None, n_nodes=None,
+                        max_depth: Optional[int] = None, out: Optional[dict] = None, stream=None):
+    """s4c_tree_accept_noalloc: the acceptance step for callers that cannot allocate device memory.
+
+    Same inputs and results as :func:`tree_accept`, but the library's built-in scratch array is used instead of a
+    workspace, so the C call allocates nothing.  This wrapper allocates nothing either when ``out`` (a dict holding
+    the five output tensors ``accept_len, path, next_token, near_tie, status``) is passed; it creates them only as a
+    convenience when ``out`` is None.  Problems whose scratch need exceeds ``NOALLOC_SCRATCH_BYTES`` raise
+    :class:`S4CError` (ERR_WORKSPACE).  Calls share the one array: keep them ordered on a stream.
+    """
+    B, T, V = target_logits.shape
+    dev = target_logits.device
+    if max_depth is None:
+        max_depth = T - 1
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=dev)
+        out = dict(accept_len=torch.empty(B, **i32), path=torch.empty(B, max_depth + 1, **i32),
+                   next_token=torch.empty(B, **i32), near_tie=torch.empty(B, T, dtype=torch.uint8, device=dev),
+                   status=torch.empty(B, **i32))
+    rc = _lib.s4c_tree_accept_noalloc(
+        _dev(target_logits, torch.float32, "target_logits"), _dev(draft_probs, torch.float32, "draft_probs"),
+        _dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"),
+        float(temperature), _dev(uniforms, torch.float32, "uniforms"), B, T, V, int(max_depth),
+        _dev(out["accept_len"], torch.int32, "accept_len"), _dev(out["path"], torch.int32, "path"),
+        _dev(out["next_token"], torch.int32, "next_token"), _dev(out["near_tie"], torch.uint8, "near_tie"),
+        _dev(out["status"], torch.int32, "status"), _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_accept_noalloc", rc)
+    return out
 
 
 def cache_pointer_array(caches: Sequence[torch.Tensor]) -> torch.Tensor:
