@@ -1,17 +1,28 @@
 // Tree-masked attention on the 5th-generation tensor cores (Section 3.2 tree mask; Figure 3) for bf16 caches.
 //
-// One CTA = one KV head of one sequence x one tile of 128 query rows x one split of the cache.  The query
+// One CTA = one KV head of one sequence x NM tiles of 128 query rows x one split of the cache.  The query
 // rows of the G = Hq/Hkv heads that share the KV head are packed into the MMA M dimension (row = g*T + node),
-// so K/V stream from HBM once per KV head.  Warp-specialised:
-//   warp 0      TMA producer: Q once, then K and V tiles of 64 slots into 128B-swizzled shared-memory rings
-//   warp 1      MMA issuer: S = Q K^T (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of two TMEM
-//               score buffers, O += P V (M128 N=d K16 x 4) into a TMEM accumulator; owns the TMEM allocation
-//   warps 2..5  one thread per query row: tcgen05.ld of the scores, tree / tail masking from the per-node
-//               ancestor bitmask, online softmax in fp32 (base-2), rescale of O in TMEM when the running max
-//               moves, P rounded to bf16 into swizzled shared memory as the A operand of the PV product
-// Partial (max, sum, unnormalised O) per split go to the workspace; the combine kernel merges them in split
-// order.  Every mbarrier wait is bounded (200 ms): on expiry the CTA flags S4C_SEQ_TIMEOUT in status[b],
-// stops waiting for anything else, still frees its TMEM and returns.
+// so K/V stream from HBM once per KV head (NM = 2 covers G*T up to 256 rows, the GQA case, with one pass).
+// Warp-specialised:
+//   warp 0        TMA producer: Q once, then K and V tiles of 64 slots into 128B-swizzled shared-memory rings
+//   warp 1        MMA issuer: S = Q K^T (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of two TMEM
+//                 score buffers per row tile, O += P V (M128 N=d K16 x 4) into a TMEM accumulator per row
+//                 tile; owns the TMEM allocation
+//   warps 2..     one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
+//                 tree / tail masking from the row's ancestor bitmask (built from parent[] by the thread
+//                 itself), online softmax in fp32 (base 2; the running offset only moves when the maximum
+//                 grew by more than 2^8, so O in TMEM is rarely rescaled), P rounded to bf16 into swizzled
+//                 shared memory as the A operand of the PV product
+// Split-KV without a second launch: the splits of one (sequence, KV head, row-tile group) form a thread-block
+// cluster; every CTA parks its partial (offset, sum, unnormalised O) in its own shared memory and, after a
+// cluster barrier, CTA r merges the rows r, r + splits, ... of all partials through distributed shared memory
+// in split order (deterministic) and writes the output.  More than 8 splits fall back to a global workspace
+// and the separate combine kernel.
+// The launch carries the programmatic-dependent-launch attribute: the prologue (barriers, TMEM allocation,
+// descriptor prefetch) may overlap the tail of the previous kernel on the stream; nothing is read from or
+// written to global memory before griddepcontrol.wait.
+// Every mbarrier wait is bounded (200 ms): on expiry the CTA flags S4C_SEQ_TIMEOUT in status[b], stops
+// waiting for anything else, still takes part in the cluster barriers, frees its TMEM and returns.
 #include <cuda.h>
 #include <math.h>
 
@@ -20,23 +31,29 @@
 
 namespace s4c {
 
-constexpr int kBM = 128;       // query rows per CTA (TMEM lanes)
-constexpr int kBN = 64;        // cache slots per tile
-constexpr int kTcThreads = 192;
+constexpr int kBM = 128;  // query rows per row tile (TMEM lanes)
+constexpr int kBN = 64;   // cache slots per tile
+constexpr int kMaxClusterSplits = 8;
 constexpr uint64_t kWaitLimitNs = 200ull * 1000 * 1000;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
 
-template <int D>
+template <int D, int NM>
 struct TcCfg {
-    static constexpr int kHalves = D / 64;                    // 64-element (128-byte) swizzle atoms along d
-    static constexpr int kQBytes = kBM * D * 2;               // 32 KB (d = 128)
-    static constexpr int kTileBytes = kBN * D * 2;            // 16 KB: one K or V tile
-    static constexpr int kPBytes = kBM * kBN * 2;             // 16 KB
-    static constexpr int kStages = D == 128 ? 4 : 6;
-    static constexpr int kSmemData = kQBytes + 2 * kPBytes + 2 * kStages * kTileBytes;
-    static constexpr int kNumBars = 1 + 4 * kStages + 2 + 2 + 2 + 1;
-    static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, masks, flags*/ + S4C_MAX_T * 4 +
-                                      S4C_MAX_T * S4C_MASK_WORDS * 4;
-    static constexpr int kTmemCols = 256;                     // 2 x 64 score columns + up to 128 output columns
+    static constexpr int kHalves = D / 64;           // 64-element (128-byte) swizzle atoms along d
+    static constexpr int kQBytes = kBM * D * 2;      // one row tile of Q: 32 KB (d = 128)
+    static constexpr int kTileBytes = kBN * D * 2;   // 16 KB: one K or V tile
+    static constexpr int kPBytes = kBM * kBN * 2;    // 16 KB
+    static constexpr int kStages = D == 128 ? (NM == 1 ? 5 : 3) : 8;
+    static constexpr int kSmemData = NM * kQBytes + NM * 2 * kPBytes + 2 * kStages * kTileBytes;
+    static constexpr int kNumBars = 1 + 4 * kStages + 7 * NM;
+    static constexpr int kThreads = 64 + 128 * NM;
+    static constexpr int kPartStride = D + 4;        // floats per parked row (padding spreads the banks)
+    static constexpr int kPartBytes = NM * kBM * kPartStride * 4 + NM * kBM * 8;
+    static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
+    static constexpr int kTmemCols = NM * 128 + NM * D <= 256 ? 256 : 512;
+    static_assert(kNumBars * 8 <= 480, "barrier area");
+    static_assert(kPartBytes <= kSmemData, "parked partials reuse the tile buffers");
+    static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -80,6 +97,9 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
             return;
         }
     }
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
     asm volatile(
@@ -134,6 +154,36 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
 // Field units are 16 bytes: start address [0,14), leading byte offset [16,30), stride byte offset [32,46),
 // version [46,48) = 1, layout type [61,64) = 2 (SWIZZLE_128B).
@@ -148,6 +198,8 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, bool b_mn_m
            ((uint32_t)(M >> 4) << 24);
 }
 
+enum TcMode { kModeDirect = 0, kModeCluster = 1, kModeWorkspace = 2 };
+
 struct TcParams {
     const int32_t* cache_len;
     const int32_t* parent;
@@ -155,7 +207,7 @@ struct TcParams {
     __nv_bfloat16* out;
     float* ws;
     int32_t* status;
-    int T, Hq, Hkv, C, m_tiles, splits;
+    int T, Hq, Hkv, C, m_groups, splits, mode, q_box_rows;
     float scale_log2;
 };
 
@@ -165,287 +217,434 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, 
     t1 = (int)(((long long)n_tiles * (split + 1)) / splits);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int D, int NM>
+__global__ void __launch_bounds__(TcCfg<D, NM>::kThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const TcParams prm) {
-    using Cfg = TcCfg<D>;
+    using Cfg = TcCfg<D, NM>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
+    constexpr int PS = Cfg::kPartStride;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128B swizzle atoms need 1024-byte alignment
     unsigned char* base_ptr = smem_raw + (base - raw);
     const uint32_t sQ = base;
-    const uint32_t sP = sQ + Cfg::kQBytes;
-    const uint32_t sK = sP + 2 * Cfg::kPBytes;
+    const uint32_t sP = sQ + NM * Cfg::kQBytes;
+    const uint32_t sK = sP + NM * 2 * Cfg::kPBytes;
     const uint32_t sV = sK + S * Cfg::kTileBytes;
     unsigned char* tail = base_ptr + Cfg::kSmemData;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 512);
-    volatile int* dead = reinterpret_cast<volatile int*>(tail + 516);
-    int* flag_s = reinterpret_cast<int*>(tail + 520);
-    int32_t* par_s = reinterpret_cast<int32_t*>(tail + 1024);
-    uint32_t(*anc_s)[S4C_MASK_WORDS] = reinterpret_cast<uint32_t(*)[S4C_MASK_WORDS]>(tail + 1024 + S4C_MAX_T * 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 480);
+    volatile int* dead = reinterpret_cast<volatile int*>(tail + 484);
+    int32_t* par_s = reinterpret_cast<int32_t*>(tail + 512);  // S4C_MAX_T * 4 = 512 bytes
 
     const uint32_t bar0 = smem_u32(bars);
     auto BAR = [&](int i) { return bar0 + 8u * i; };
-    const int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + S, V_FULL = 1 + 2 * S, V_EMPTY = 1 + 3 * S, S_FULL = 1 + 4 * S,
-              S_EMPTY = S_FULL + 2, P_FULL = S_EMPTY + 2, PV_DONE = P_FULL + 2;
+    // barrier indices; the per-row-tile ones take (tile t, buffer i)
+    constexpr int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + S, V_FULL = 1 + 2 * S, V_EMPTY = 1 + 3 * S, PER_TILE = 1 + 4 * S;
+    auto S_FULL = [&](int t, int i) { return BAR(PER_TILE + 7 * t + i); };
+    auto S_EMPTY = [&](int t, int i) { return BAR(PER_TILE + 7 * t + 2 + i); };
+    auto P_FULL = [&](int t, int i) { return BAR(PER_TILE + 7 * t + 4 + i); };
+    auto PV_DONE = [&](int t) { return BAR(PER_TILE + 7 * t + 6); };
 
     const int split = blockIdx.x, splits = prm.splits;
-    const int mt = blockIdx.y % prm.m_tiles, hk = blockIdx.y / prm.m_tiles, b = blockIdx.z;
+    const int mg = blockIdx.y % prm.m_groups, hk = blockIdx.y / prm.m_groups, b = blockIdx.z;
     const int T = prm.T, G = prm.Hq / prm.Hkv, R = G * T;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int mt0 = mg * NM;  // first row tile of this CTA
+    auto rows_in = [&](int t) {  // valid query rows of row tile t of this CTA
+        const int r = R - (mt0 + t) * kBM;
+        return r < 0 ? 0 : (r > kBM ? kBM : r);
+    };
+    int nm_act = 0;  // row tiles with at least one row (they are the first ones)
+#pragma unroll
+    for (int t = 0; t < NM; ++t) nm_act += rows_in(t) > 0 ? 1 : 0;
 
-    // ---- validate the sequence, build the ancestor bitmasks (all threads)
-    const int n = prm.n_nodes ? prm.n_nodes[b] : T;
-    const int L = prm.cache_len[b];
-    for (int i = threadIdx.x; i < T; i += blockDim.x) par_s[i] = prm.parent[(size_t)b * T + i];
-    if (threadIdx.x == 0) *dead = 0;
-    __syncthreads();
-    int flags = build_ancestor_masks(par_s, n, T, anc_s, nullptr, flag_s);
-    if (L < 0 || (long long)L + (n > 0 ? n : 0) > (long long)prm.C) flags |= S4C_SEQ_CAPACITY;
-    if (split == 0 && blockIdx.y == 0 && threadIdx.x == 0 && prm.status) prm.status[b] = flags;
-    if (flags) return;
-
-    const int Ltot = L + n;
-    const int n_tiles = (Ltot + kBN - 1) / kBN;
-    int t0, t1;
-    split_range(n_tiles, splits, split, t0, t1);
-    const int nt = t1 - t0;
-
-    // ---- barriers and TMEM
+    // ---- prologue that touches no global memory: barriers, TMEM, descriptor prefetch
     if (threadIdx.x == 0) {
+        tma_prefetch_desc(&map_q), tma_prefetch_desc(&map_k), tma_prefetch_desc(&map_v);
         mbar_init(BAR(Q_FULL), 1);
         for (int s = 0; s < S; ++s) {
             mbar_init(BAR(K_FULL + s), 1), mbar_init(BAR(K_EMPTY + s), 1);
             mbar_init(BAR(V_FULL + s), 1), mbar_init(BAR(V_EMPTY + s), 1);
         }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(BAR(S_FULL + i), 1), mbar_init(BAR(S_EMPTY + i), 128);
-            mbar_init(BAR(P_FULL + i), 128);
+#pragma unroll
+        for (int t = 0; t < NM; ++t) {
+            const uint32_t active = 32u * (uint32_t)((rows_in(t) + 31) / 32);  // threads of the warps that own a valid row
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(S_FULL(t, i), 1), mbar_init(S_EMPTY(t, i), active ? active : 1);
+                mbar_init(P_FULL(t, i), active ? active : 1);
+            }
+            mbar_init(PV_DONE(t), 1);
         }
-        mbar_init(BAR(PV_DONE), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        *dead = 0;
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint32_t tmem_O = tmem + 2 * kBN;
 
-    const int q_row0 = (b * prm.Hq + hk * G) * T + mt * kBM;  // row of the [B*Hq*T, d] view of q
-    const int kv_row0 = (b * prm.Hkv + hk) * prm.C;           // row of the [B*Hkv*C, d] view of the caches
+    griddep_wait();  // everything below may depend on the previous kernel of the stream
+
+    const int n = prm.n_nodes ? prm.n_nodes[b] : T;
+    const int L = prm.cache_len[b];
+    int flags = (n < 1 || n > T) ? S4C_SEQ_BAD_PARENT : 0;
+    if (L < 0 || (long long)L + (n > 0 ? n : 0) > (long long)prm.C) flags |= S4C_SEQ_CAPACITY;
+    const int Ltot = L + n;
+    int t0 = 0, t1 = 0;
+    if (!flags) split_range((Ltot + kBN - 1) / kBN, splits, split, t0, t1);
+    const int nt = t1 - t0;  // 0 when the lengths are unusable: nothing is loaded then
+
+    const int q_row0 = (b * prm.Hq + hk * G) * T + mt0 * kBM;  // row of the [B*Hq*T, d] view of q
+    const int kv_row0 = (b * prm.Hkv + hk) * prm.C;            // row of the [B*Hkv*C, d] view of the caches
+    const uint32_t q_bytes = (uint32_t)prm.q_box_rows * 128u * NH;
+
+    auto load_tile = [&](int j) {  // TMA producer thread only
+        const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
+        mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead);
+        mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
+        for (int h = 0; h < NH; ++h)
+            tma_load_2d(sK + s * Cfg::kTileBytes + h * (kBN * 128), &map_k, BAR(K_FULL + s), h * 64, row);
+        mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead);
+        mbar_expect_tx(BAR(V_FULL + s), Cfg::kTileBytes);
+        for (int h = 0; h < NH; ++h)
+            tma_load_2d(sV + s * Cfg::kTileBytes + h * (kBN * 128), &map_v, BAR(V_FULL + s), h * 64, row);
+    };
+    const int n_first = nt < S ? nt : S;  // tiles whose ring slots are free from the start
+    if (threadIdx.x == 0 && nt > 0) {
+        // first pass of the ring before anyone else is ready: the loads only need the barriers this thread made
+        mbar_expect_tx(BAR(Q_FULL), q_bytes * nm_act);
+        for (int t = 0; t < nm_act; ++t)
+            for (int h = 0; h < NH; ++h)
+                tma_load_2d(sQ + t * Cfg::kQBytes + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0 + t * kBM);
+        for (int j = 0; j < n_first; ++j) load_tile(j);
+    }
+    int bad_parent = 0;
+    if (warp >= 2 && !flags) {  // tree check: thread i looks at node i
+        const int i = threadIdx.x - 64;
+        if (i < T) {
+            const int p = prm.parent[(size_t)b * T + i];
+            par_s[i] = p;
+            bad_parent = i < n && ((i == 0 && p != -1) || (i > 0 && (p < 0 || p >= i)));
+        }
+    }
+    tc_fence_before();
+    if (__syncthreads_or(bad_parent)) flags |= S4C_SEQ_BAD_PARENT;
+    tc_fence_after();
+    griddep_launch_dependents();
+    const bool run = flags == 0;
+    if (split == 0 && blockIdx.y == 0 && threadIdx.x == 64 && prm.status) prm.status[b] = flags;
+    const uint32_t tmem = *tmem_slot;
+    auto TM_S = [&](int t, int i) { return tmem + (uint32_t)(t * 2 * kBN + i * kBN); };
+    auto TM_O = [&](int t) { return tmem + (uint32_t)(NM * 2 * kBN + t * D); };
 
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0 && nt > 0) {
-            mbar_expect_tx(BAR(Q_FULL), Cfg::kQBytes);
-            for (int h = 0; h < NH; ++h) tma_load_2d(sQ + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0);
-            for (int j = 0; j < nt; ++j) {
-                const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
-                mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead);
-                mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
-                for (int h = 0; h < NH; ++h)
-                    tma_load_2d(sK + s * Cfg::kTileBytes + h * (kBN * 128), &map_k, BAR(K_FULL + s), h * 64, row);
-                mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead);
-                mbar_expect_tx(BAR(V_FULL + s), Cfg::kTileBytes);
-                for (int h = 0; h < NH; ++h)
-                    tma_load_2d(sV + s * Cfg::kTileBytes + h * (kBN * 128), &map_v, BAR(V_FULL + s), h * 64, row);
+            if (run) {
+                for (int j = n_first; j < nt; ++j) load_tile(j);
+            } else {  // malformed tree: nobody consumes what was requested; let it land before the CTA goes away
+                mbar_wait(BAR(Q_FULL), 0, dead);
+                for (int j = 0; j < n_first; ++j) mbar_wait(BAR(K_FULL + j), 0, dead), mbar_wait(BAR(V_FULL + j), 0, dead);
             }
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0 && nt > 0) {
+        if (lane == 0 && nt > 0 && run) {
             constexpr uint32_t idesc_qk = instr_desc_bf16(kBM, kBN, false);
             constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
             auto issue_pv = [&](int jj) {
                 const int s = jj % S, it = jj / S;
                 mbar_wait(BAR(V_FULL + s), it & 1, dead);
-                mbar_wait(BAR(P_FULL + (jj & 1)), (jj >> 1) & 1, dead);
-                tc_fence_after();
-                const uint32_t p_base = sP + (jj & 1) * Cfg::kPBytes, v_base = sV + s * Cfg::kTileBytes;
+                const uint32_t v_base = sV + s * Cfg::kTileBytes;
+                for (int t = 0; t < nm_act; ++t) {
+                    mbar_wait(P_FULL(t, jj & 1), (jj >> 1) & 1, dead);
+                    tc_fence_after();
+                    const uint32_t p_base = sP + (t * 2 + (jj & 1)) * Cfg::kPBytes;
 #pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk) {
-                    // A = P [128 rows][64 slots], K-major: 32 bytes per K step inside the 128-byte row
-                    const uint64_t ad = smem_desc_sw128(p_base + kk * 32, 16, 1024);
-                    // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
-                    const uint64_t bd = smem_desc_sw128(v_base + kk * 2048, kBN * 128, 1024);
-                    tc_mma_bf16(tmem_O, ad, bd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kBN / 16; ++kk) {
+                        // A = P [128 rows][64 slots], K-major: 32 bytes per K step inside the 128-byte row
+                        const uint64_t ad = smem_desc_sw128(p_base + kk * 32, 16, 1024);
+                        // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
+                        const uint64_t bd = smem_desc_sw128(v_base + kk * 2048, kBN * 128, 1024);
+                        tc_mma_bf16(TM_O(t), ad, bd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(PV_DONE(t));
                 }
                 tc_commit(BAR(V_EMPTY + s));
-                tc_commit(BAR(PV_DONE));
             };
             mbar_wait(BAR(Q_FULL), 0, dead);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
                 mbar_wait(BAR(K_FULL + s), it & 1, dead);
-                mbar_wait(BAR(S_EMPTY + (j & 1)), ((j >> 1) & 1) ^ 1, dead);
-                tc_fence_after();
                 const uint32_t k_base = sK + s * Cfg::kTileBytes;
+                for (int t = 0; t < nm_act; ++t) {
+                    mbar_wait(S_EMPTY(t, j & 1), ((j >> 1) & 1) ^ 1, dead);
+                    tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const int h = kk >> 2, ko = (kk & 3) * 32;  // 64-element halves along d, 32 bytes per K step
-                    const uint64_t ad = smem_desc_sw128(sQ + h * (kBM * 128) + ko, 16, 1024);
-                    const uint64_t bd = smem_desc_sw128(k_base + h * (kBN * 128) + ko, 16, 1024);
-                    tc_mma_bf16(tmem + (j & 1) * kBN, ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const int h = kk >> 2, ko = (kk & 3) * 32;  // 64-element halves along d, 32 bytes per K step
+                        const uint64_t ad = smem_desc_sw128(sQ + t * Cfg::kQBytes + h * (kBM * 128) + ko, 16, 1024);
+                        const uint64_t bd = smem_desc_sw128(k_base + h * (kBN * 128) + ko, 16, 1024);
+                        tc_mma_bf16(TM_S(t, j & 1), ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
+                    }
+                    tc_commit(S_FULL(t, j & 1));
                 }
                 tc_commit(BAR(K_EMPTY + s));
-                tc_commit(BAR(S_FULL + (j & 1)));
                 if (j > 0) issue_pv(j - 1);
             }
             issue_pv(nt - 1);
         }
-    } else {
-        // ================= softmax / correction / epilogue: one thread per query row =================
-        const int wq = warp & 3;  // TMEM lane quadrant this warp may access
+    } else if (run) {
+        // ================= softmax / correction: one thread per query row =================
+        const int t = (warp - 2) >> 2;  // row tile of this warp group
+        const int wq = warp & 3;        // TMEM lane quadrant this warp may access
         const int row = wq * 32 + lane;
-        const int gr = mt * kBM + row;
-        const bool row_valid = gr < R;
+        const int rows_t = rows_in(t);
+        const bool warp_active = wq * 32 < rows_t;
+        const bool row_ok = row < rows_t;
+        const int gr = (mt0 + t) * kBM + row;
         const int node = gr % T;
-        const bool node_valid = row_valid && node < n;
-        uint32_t am[S4C_MASK_WORDS];
-#pragma unroll
-        for (int w = 0; w < S4C_MASK_WORDS; ++w) am[w] = node_valid ? anc_s[node][w] : 0u;
+        // the row's ancestor-or-self set as a 128-bit mask, straight from parent[] (checked above: the chain ends)
+        uint64_t anc_lo = 0, anc_hi = 0;
+        if (row_ok && node < n)
+            for (int u = node, guard = 0; u >= 0 && guard <= T; u = par_s[u], ++guard) {
+                if (u < 64)
+                    anc_lo |= 1ull << u;
+                else
+                    anc_hi |= 1ull << (u - 64);
+            }
         const uint32_t lane_off = (uint32_t)(wq * 32) << 16;
-        const int sm_tid = threadIdx.x - 64;  // 0..127
-        float m = -1e30f, l = 0.f;
+        float m = -1e30f, l = 0.f;  // m: offset in use (scaled, log2 units); never -inf so that exp2(-inf - m) = 0
         const float sc = prm.scale_log2;
 
-        for (int j = 0; j < nt; ++j) {
-            const int kv0 = (t0 + j) * kBN;
-            mbar_wait(BAR(S_FULL + (j & 1)), (j >> 1) & 1, dead);
-            tc_fence_after();
-            uint32_t sr[2][32];
-            tmem_ld32(tmem + lane_off + (j & 1) * kBN, sr[0]);
-            tmem_ld32(tmem + lane_off + (j & 1) * kBN + 32, sr[1]);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(BAR(S_EMPTY + (j & 1)));
-
-            float sv[kBN];
-#pragma unroll
-            for (int c = 0; c < kBN; ++c) sv[c] = __uint_as_float(sr[c >> 5][c & 31]) * sc;
-            if (kv0 + kBN > L) {  // the tile touches tree slots or the tail: mask by index
-#pragma unroll
-                for (int c = 0; c < kBN; ++c) {
-                    const int kv = kv0 + c, t = kv - L;
-                    bool vis = kv < L;
-                    if (!vis && t < n) vis = (am[(t >> 5) & 3] >> (t & 31)) & 1u;
-                    sv[c] = vis ? sv[c] : -INFINITY;
-                }
-            }
-            float mx = sv[0];
-#pragma unroll
-            for (int c = 1; c < kBN; ++c) mx = fmaxf(mx, sv[c]);
-            const float m_new = row_valid ? fmaxf(m, mx) : m;
-            const float alpha = exp2f(m - m_new);
-            float ls = 0.f;
-            uint32_t pk[kBN / 2];
-#pragma unroll
-            for (int c = 0; c < kBN; c += 2) {
-                const float p0 = exp2f(sv[c] - m_new), p1 = exp2f(sv[c + 1] - m_new);
-                ls += p0 + p1;
-                const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-                pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-            l = l * alpha + ls;
-            m = m_new;
-
-            if (j > 0) {
-                mbar_wait(BAR(PV_DONE), (j - 1) & 1, dead);
+        if (warp_active)
+            for (int j = 0; j < nt; ++j) {
+                const int kv0 = (t0 + j) * kBN;
+                mbar_wait(S_FULL(t, j & 1), (j >> 1) & 1, dead);
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, row_valid && alpha != 1.f)) {
-#pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
-                        uint32_t o[32];
-                        tmem_ld32(tmem_O + lane_off + cc * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        tmem_st32(tmem_O + lane_off + cc * 32, o);
-                    }
-                    tmem_wait_st();
-                }
-            }
-            if (kv0 + kBN > Ltot) {
-                // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
-                // but 0 * NaN would poison O, so those V rows are cleared before the PV product reads them
-                const int s = j % S, it = j / S;
-                mbar_wait(BAR(V_FULL + s), it & 1, dead);
-                const int first = Ltot - kv0;  // 1..63
-                unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
-                for (int idx = sm_tid; idx < (kBN - first) * 8 * NH; idx += 128) {
-                    const int h = idx / ((kBN - first) * 8), rem = idx % ((kBN - first) * 8);
-                    const int r = first + rem / 8, ch = rem % 8;
-                    *reinterpret_cast<uint4*>(vt + h * (kBN * 128) + r * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
-                }
-            }
-            // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
-            {
-                unsigned char* pt = base_ptr + (sP - base) + (j & 1) * Cfg::kPBytes + row * 128;
-#pragma unroll
-                for (int ch = 0; ch < 8; ++ch)
-                    *reinterpret_cast<uint4*>(pt + ((ch ^ (row & 7)) << 4)) =
-                        make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-            }
-            fence_async_smem();
-            tc_fence_before();
-            mbar_arrive(BAR(P_FULL + (j & 1)));
-        }
+                uint32_t sr[2][32];
+                tmem_ld32(TM_S(t, j & 1) + lane_off, sr[0]);
+                tmem_ld32(TM_S(t, j & 1) + lane_off + 32, sr[1]);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(S_EMPTY(t, j & 1));
 
-        // ---- epilogue
-        if (nt > 0) {
-            mbar_wait(BAR(PV_DONE), (nt - 1) & 1, dead);
+                float sv[kBN];
+#pragma unroll
+                for (int c = 0; c < kBN; ++c) sv[c] = __uint_as_float(sr[c >> 5][c & 31]);
+                if (kv0 + kBN > L) {
+                    // the tile touches tree slots or the tail: column c is visible iff it lies in the prefix or is the
+                    // slot of a node on this row's root path
+                    const int off = L - kv0;  // prefix columns of this tile (<= 0: none)
+                    uint64_t vis;
+                    if (off >= 0) {
+                        vis = (anc_lo << off) | ((1ull << off) - 1ull);  // off < 64 here
+                    } else {
+                        const int sh = -off;  // first tree node of the tile
+                        vis = sh < 64 ? ((anc_lo >> sh) | (anc_hi << (64 - sh))) : (sh < 128 ? (anc_hi >> (sh - 64)) : 0ull);
+                    }
+                    const uint32_t v0 = (uint32_t)vis, v1 = (uint32_t)(vis >> 32);
+#pragma unroll
+                    for (int c = 0; c < kBN; ++c) {
+                        const bool on = (((c < 32 ? v0 : v1) >> (c & 31)) & 1u) != 0;
+                        sv[c] = on ? sv[c] : -INFINITY;
+                    }
+                }
+                float mx = sv[0];
+#pragma unroll
+                for (int c = 1; c < kBN; ++c) mx = fmaxf(mx, sv[c]);
+                mx *= sc;  // sc > 0
+                const bool grow = row_ok && mx > m + kRescaleThreshold;
+                const float m_new = grow ? mx : m;
+                const float alpha = grow ? exp2f(m - m_new) : 1.f;
+                float ls = 0.f;
+                uint32_t pk[kBN / 2];
+#pragma unroll
+                for (int c = 0; c < kBN; c += 2) {
+                    const float p0 = exp2f(fmaf(sv[c], sc, -m_new)), p1 = exp2f(fmaf(sv[c + 1], sc, -m_new));
+                    ls += p0 + p1;
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                    pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                }
+                l = l * alpha + ls;
+                m = m_new;
+
+                if (j > 0) {
+                    mbar_wait(PV_DONE(t), (j - 1) & 1, dead);
+                    tc_fence_after();
+                    if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+                        for (int cc = 0; cc < D / 32; ++cc) {
+                            uint32_t o[32];
+                            tmem_ld32(TM_O(t) + lane_off + cc * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            tmem_st32(TM_O(t) + lane_off + cc * 32, o);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                if (t == 0 && kv0 + kBN > Ltot) {
+                    // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
+                    // but 0 * NaN would poison O, so those V rows are cleared before the PV products read them (the
+                    // MMA thread sees P_FULL of row tile 0 before it issues any PV of this tile)
+                    const int s = j % S, it = j / S;
+                    mbar_wait(BAR(V_FULL + s), it & 1, dead);
+                    const int first = Ltot - kv0;  // 1..63
+                    unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
+                    const int stride = 32 * ((rows_t + 31) / 32);
+                    for (int idx = row; idx < (kBN - first) * 8 * NH; idx += stride) {
+                        const int h = idx / ((kBN - first) * 8), rem = idx % ((kBN - first) * 8);
+                        const int r = first + rem / 8, ch = rem % 8;
+                        *reinterpret_cast<uint4*>(vt + h * (kBN * 128) + r * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
+                {
+                    unsigned char* pt = base_ptr + (sP - base) + (t * 2 + (j & 1)) * Cfg::kPBytes + row * 128;
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch)
+                        *reinterpret_cast<uint4*>(pt + ((ch ^ (row & 7)) << 4)) =
+                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(P_FULL(t, j & 1));
+            }
+
+        // ---- this split's result for the row: (m, l, unnormalised O)
+        if (warp_active && nt > 0) {
+            mbar_wait(PV_DONE(t), (nt - 1) & 1, dead);
             tc_fence_after();
         }
-        const bool direct = splits == 1;
-        const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
-        const float inv = (node_valid && l > 0.f) ? 1.f / l : 0.f;
+        const bool node_valid = row_ok && node < n;
+        if (prm.mode == kModeCluster) {
+            // every MMA of the CTA has finished before any tile buffer is reused for the parked partials
+            named_bar_sync(1, NM * 128);
+            if (warp_active) {
+                float* po = reinterpret_cast<float*>(base_ptr) + (size_t)(t * kBM + row) * PS;
 #pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-            uint32_t o[32];
-            if (nt > 0) {
-                tmem_ld32(tmem_O + lane_off + cc * 32, o);
-                tmem_wait_ld();
-            } else {
+                for (int cc = 0; cc < D / 32; ++cc) {
+                    uint32_t o[32];
+                    if (nt > 0) {
+                        tmem_ld32(TM_O(t) + lane_off + cc * 32, o);
+                        tmem_wait_ld();
+                    } else {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) o[c] = 0u;
-            }
-            if (!row_valid) continue;
-            if (direct) {
-                uint32_t packed[16];
+                        for (int c = 0; c < 32; ++c) o[c] = 0u;
+                    }
 #pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    const __nv_bfloat162 h2 =
-                        __floats2bfloat162_rn(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
-                    packed[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                    for (int c = 0; c < 32; c += 4)
+                        *reinterpret_cast<float4*>(po + cc * 32 + c) = make_float4(
+                            __uint_as_float(o[c]), __uint_as_float(o[c + 1]), __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
                 }
-                uint4* dst = reinterpret_cast<uint4*>(prm.out + orow * D + cc * 32);
+                float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)NM * kBM * PS);
+                pml[t * kBM + row] = make_float2(m, l);
+            }
+        } else if (warp_active) {
+            const bool direct = prm.mode == kModeDirect;
+            const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
+            const float inv = (node_valid && l > 0.f) ? 1.f / l : 0.f;
 #pragma unroll
-                for (int v = 0; v < 4; ++v)
-                    dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-            } else {
-                float* w = prm.ws + (orow * splits + split) * (D + 2) + cc * 32;
-                if (!node_valid) {
+            for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t o[32];
+                if (nt > 0) {
+                    tmem_ld32(TM_O(t) + lane_off + cc * 32, o);
+                    tmem_wait_ld();
+                } else {
 #pragma unroll
                     for (int c = 0; c < 32; ++c) o[c] = 0u;
                 }
+                if (!row_ok) continue;
+                if (direct) {
+                    uint32_t packed[16];
 #pragma unroll
-                for (int c = 0; c < 32; c += 2)
-                    *reinterpret_cast<float2*>(w + c) = make_float2(__uint_as_float(o[c]), __uint_as_float(o[c + 1]));
+                    for (int c = 0; c < 32; c += 2) {
+                        const __nv_bfloat162 h2 =
+                            __floats2bfloat162_rn(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
+                        packed[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(prm.out + orow * D + cc * 32);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                } else {
+                    float* w = prm.ws + (orow * splits + split) * (D + 2) + cc * 32;
+                    if (!node_valid) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = 0u;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2)
+                        *reinterpret_cast<float2*>(w + c) = make_float2(__uint_as_float(o[c]), __uint_as_float(o[c + 1]));
+                }
             }
-        }
-        if (!direct && row_valid) {
-            float* w = prm.ws + (orow * splits + split) * (D + 2) + D;
-            *reinterpret_cast<float2*>(w) = make_float2(node_valid ? m : -INFINITY, node_valid ? l : 0.f);
+            if (!direct && row_ok) {
+                float* w = prm.ws + (orow * splits + split) * (D + 2) + D;
+                *reinterpret_cast<float2*>(w) = make_float2(node_valid ? m : -INFINITY, node_valid ? l : 0.f);
+            }
         }
         tc_fence_before();
     }
 
-    __syncthreads();
+    if (prm.mode == kModeCluster && run) {
+        // ---- merge the splits through distributed shared memory: this CTA owns rows rank, rank + splits, ...
+        __syncwarp();
+        cluster_sync_all();
+        const uint32_t rank = cluster_ctarank();
+        const uint32_t part = base, part_ml = base + (uint32_t)(NM * kBM * PS * 4);
+        constexpr int EPL = D / 32;  // output elements per lane
+        for (int idx = (int)rank + splits * warp; idx < NM * kBM; idx += splits * (Cfg::kThreads / 32)) {
+            const int t = idx / kBM, row = idx % kBM;
+            if (row >= rows_in(t)) continue;
+            const int gr = (mt0 + t) * kBM + row;
+            const bool node_valid = (gr % T) < n;
+            float ms[kMaxClusterSplits], ls[kMaxClusterSplits];
+            float M = -INFINITY;
+#pragma unroll
+            for (int s = 0; s < kMaxClusterSplits; ++s) {
+                ms[s] = -INFINITY, ls[s] = 0.f;
+                if (s < splits) {
+                    const float2 ml = ld_cluster_f2(map_to_cta(part_ml + (uint32_t)idx * 8u, (uint32_t)s));
+                    ms[s] = ml.x, ls[s] = ml.y;
+                    M = fmaxf(M, ml.x);
+                }
+            }
+            float num[4] = {0.f, 0.f, 0.f, 0.f}, den = 0.f;
+#pragma unroll
+            for (int s = 0; s < kMaxClusterSplits; ++s) {
+                if (s < splits) {
+                    const float f = exp2f(ms[s] - M);
+                    den = fmaf(f, ls[s], den);
+                    const uint32_t a = map_to_cta(part + ((uint32_t)idx * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)s);
+                    if (EPL == 4) {
+                        const float4 o = ld_cluster_f4(a);
+                        num[0] = fmaf(f, o.x, num[0]), num[1] = fmaf(f, o.y, num[1]);
+                        num[2] = fmaf(f, o.z, num[2]), num[3] = fmaf(f, o.w, num[3]);
+                    } else {
+                        const float2 o = ld_cluster_f2(a);
+                        num[0] = fmaf(f, o.x, num[0]), num[1] = fmaf(f, o.y, num[1]);
+                    }
+                }
+            }
+            const float inv = (node_valid && den > 0.f) ? 1.f / den : 0.f;
+            const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;
+            __nv_bfloat16* dst = prm.out + orow * D + lane * EPL;
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
+            if (EPL == 4) {
+                const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[2] * inv, num[3] * inv);
+                *reinterpret_cast<uint2*>(dst) =
+                    make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+            } else {
+                *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(&h0);
+            }
+        }
+        __syncwarp();
+        cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
+    } else {
+        __syncthreads();
+    }
     if (threadIdx.x == 0 && *dead && prm.status) atomicOr(prm.status + b, S4C_SEQ_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
@@ -485,42 +684,78 @@ static bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int d, in
 
 bool tc_supported(int T, int Hq, int Hkv, int d, s4c_dtype dt) { return dt == S4C_BF16 && (d == 128 || d == 64); }
 
-int tc_m_tiles(int T, int Hq, int Hkv) { return ceil_div((Hq / Hkv) * T, kBM); }
+static int tc_m_tiles(int T, int Hq, int Hkv) { return ceil_div((Hq / Hkv) * T, kBM); }
+static int tc_nm(int T, int Hq, int Hkv) { return tc_m_tiles(T, Hq, Hkv) > 1 ? 2 : 1; }
+static int tc_m_groups(int T, int Hq, int Hkv) { return ceil_div(tc_m_tiles(T, Hq, Hkv), tc_nm(T, Hq, Hkv)); }
 
-int tc_splits(int B, int T, int Hq, int Hkv, int C) {
-    const int base = B * Hkv * tc_m_tiles(T, Hq, Hkv);
-    int s = 148 / base;  // one resident CTA per SM: fill one wave
-    const int max_by_len = ceil_div(C, kBN) / 2;  // at least two tiles per split
-    if (s > max_by_len) s = max_by_len;
-    if (s > 64) s = 64;
-    return s < 1 ? 1 : s;
+// Number of splits of the cache: the smallest count that minimises (waves of one-CTA-per-SM work) / splits, with a
+// small charge per extra split for the merge; a split has at least two tiles.  Up to 8 splits merge inside a
+// cluster; a grid too small to fill the GPU even with 8 goes wider and merges through the workspace.
+static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
+    const int base = B * Hkv * tc_m_groups(T, Hq, Hkv);
+    int max_by_len = ceil_div(C, kBN) / 2;
+    if (max_by_len < 1) max_by_len = 1;
+    if (base * kMaxClusterSplits * 2 <= 148) {  // tiny grids: fill one wave through the workspace path
+        int s = 148 / base;
+        if (s > 64) s = 64;
+        return s > max_by_len ? max_by_len : s;
+    }
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= kMaxClusterSplits && s <= max_by_len; ++s) {
+        const int resident = s == 1 ? 148 : 8 * (18 / s) * s;  // clusters do not straddle the 8 GPCs (18+ SMs each)
+        const double waves = (double)ceil_div(base * s, resident);
+        const double cost = waves / s * (1.0 + 0.03 * (s - 1));
+        if (cost < best_cost - 1e-12) best_cost = cost, best = s;
+    }
+    return best;
 }
 
 size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
     const int s = tc_splits(B, T, Hq, Hkv, C);
-    return s == 1 ? 0 : round_up((size_t)B * Hq * T * s * (d + 2) * sizeof(float), 256);
+    return s <= kMaxClusterSplits ? 0 : round_up((size_t)B * Hq * T * s * (d + 2) * sizeof(float), 256);
 }
 
-template <int D>
+template <int D, int NM>
 static s4c_status launch_tc(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
-    using Cfg = TcCfg<D>;
-    static bool configured[64] = {};  // the opt-in to > 48 KB of dynamic shared memory is per device
+    using Cfg = TcCfg<D, NM>;
+    static bool configured[64] = {};  // the opt-ins (dynamic shared memory, cluster size) are per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return S4C_ERR_CUDA;
         configured[dev] = true;
     }
     CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, q, (uint64_t)B * prm.Hq * prm.T, D, kBM) ||
+    if (!make_map(&mq, q, (uint64_t)B * prm.Hq * prm.T, D, prm.q_box_rows) ||
         !make_map(&mk, k, (uint64_t)B * prm.Hkv * prm.C, D, kBN) ||
         !make_map(&mv, v, (uint64_t)B * prm.Hkv * prm.C, D, kBN))
         return S4C_ERR_CUDA;
-    dim3 grid(prm.splits, prm.m_tiles * prm.Hkv, B);
-    tree_attention_tc_kernel<D><<<grid, kTcThreads, Cfg::kSmemBytes, stream>>>(mq, mk, mv, prm);
-    S4C_RETURN_IF_CUDA_ERROR();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(prm.splits, prm.m_groups * prm.Hkv, B);
+    cfg.blockDim = dim3(Cfg::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[2];
+    int na = 0;
+    attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+    if (prm.mode == kModeCluster) {
+        attrs[na].id = cudaLaunchAttributeClusterDimension;
+        attrs[na].val.clusterDim.x = prm.splits;
+        attrs[na].val.clusterDim.y = 1;
+        attrs[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    cfg.attrs = attrs;
+    cfg.numAttrs = na;
+    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM>, mq, mk, mv, prm) != cudaSuccess) {
+        cudaGetLastError();
+        return S4C_ERR_CUDA;
+    }
     return S4C_OK;
 }
 
@@ -531,12 +766,21 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     prm.cache_len = cache_len, prm.parent = parent, prm.n_nodes = n_nodes;
     prm.out = static_cast<__nv_bfloat16*>(out), prm.ws = static_cast<float*>(ws), prm.status = status;
     prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C;
-    prm.m_tiles = tc_m_tiles(T, Hq, Hkv);
+    const int nm = tc_nm(T, Hq, Hkv);
+    prm.m_groups = tc_m_groups(T, Hq, Hkv);
     prm.splits = tc_splits(B, T, Hq, Hkv, C);
+    prm.mode = prm.splits == 1 ? kModeDirect : (prm.splits <= kMaxClusterSplits ? kModeCluster : kModeWorkspace);
+    const int R = (Hq / Hkv) * T;
+    prm.q_box_rows = R >= kBM ? kBM : (int)round_up((size_t)R, 8);
     prm.scale_log2 = scale * 1.4426950408889634f;
-    s4c_status st = d == 128 ? launch_tc<128>(q, k, v, prm, B, stream) : launch_tc<64>(q, k, v, prm, B, stream);
+    s4c_status st;
+    if (d == 128)
+        st = nm == 1 ? launch_tc<128, 1>(q, k, v, prm, B, stream) : launch_tc<128, 2>(q, k, v, prm, B, stream);
+    else
+        st = nm == 1 ? launch_tc<64, 1>(q, k, v, prm, B, stream) : launch_tc<64, 2>(q, k, v, prm, B, stream);
     if (st != S4C_OK) return st;
-    if (prm.splits > 1) return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits, S4C_BF16, stream);
+    if (prm.mode == kModeWorkspace)
+        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits, S4C_BF16, stream);
     return S4C_OK;
 }
 

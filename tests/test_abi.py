@@ -50,7 +50,9 @@ def test_workspace_queries_are_host_functions(s4c_lib):
     assert s4c.tree_accept_workspace_bytes(0, 1, 1) == 0
     import torch
 
-    w = s4c.tree_attention_workspace_bytes(1, 26, 32, 32, 128, 1152, torch.bfloat16)
+    # 32 KV heads x 4 splits merge inside a thread-block cluster: no scratch; 8 KV heads go wider than a cluster
+    assert s4c.tree_attention_workspace_bytes(1, 26, 32, 32, 128, 1152, torch.bfloat16) == 0
+    w = s4c.tree_attention_workspace_bytes(1, 16, 8, 8, 128, 9088, torch.bfloat16)
     assert w > 0 and w % 256 == 0
     assert s4c.tree_attention_workspace_bytes(1, 200, 32, 32, 128, 1152, torch.bfloat16) == 0  # T > 128: invalid
 
@@ -73,7 +75,7 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert att(k=P + 2) == 4                     # S4C_ERR_ALIGN
     assert att(scale=-1.0) == 2
     assert att(B=0) == 0
-    assert att(Hq=32, Hkv=32, C=4096, ws=None) == 5  # needs a workspace: S4C_ERR_WORKSPACE
+    assert att(Hq=8, Hkv=8, C=9088, ws=None) == 5   # a grid this small splits wider than a cluster and needs a workspace
     acc = lambda **kw: lib.s4c_tree_accept(*[kw.get(k, d) for k, d in [
         ("lg", P), ("dp", P), ("tok", P), ("par", P), ("nn", None), ("tau", 1.0), ("u", P), ("B", 1), ("T", 8),
         ("V", 100), ("md", 7), ("al", P), ("path", P), ("nt", P), ("tie", None), ("st", None), ("ws", None), ("wsb", 0),
