@@ -5,10 +5,10 @@
 // so K/V stream from HBM once per KV head (NM = 2 covers G*T up to 256 rows, the GQA case, with one pass).
 // Warp-specialised:
 //   warp 0        TMA producer: Q once, then K and V tiles of 64 slots into 128B-swizzled shared-memory rings
-//   warp 1        MMA issuer: S = Q K^T (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of two TMEM
-//                 score buffers per row tile, O += P V (M128 N=d K16 x 4) into a TMEM accumulator per row
-//                 tile; owns the TMEM allocation
-//   warps 2..     one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
+//   warps 1, 2    MMA issuers, one thread each: warp 1 issues S = Q K^T (tcgen05.mma kind::f16, M128 N64 K16 x
+//                 d/16) into one of two TMEM score buffers per row tile and owns the TMEM allocation; warp 2
+//                 issues O += P V (M128 N=d K16 x 4) into a TMEM accumulator per row tile
+//   warps 3..     one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
 //                 tree / tail masking from the row's ancestor bitmask (built from parent[] by the thread
 //                 itself), online softmax in fp32 (base 2; the running offset only moves when the maximum
 //                 grew by more than 2^8, so O in TMEM is rarely rescaled), P rounded to bf16 into swizzled
@@ -34,7 +34,7 @@ namespace s4c {
 constexpr int kBM = 128;  // query rows per row tile (TMEM lanes)
 constexpr int kBN = 64;   // cache slots per tile
 constexpr int kMaxClusterSplits = 8;
-constexpr uint64_t kWaitLimitNs = 200ull * 1000 * 1000;
+constexpr long long kWaitLimitCycles = 400ll * 1000 * 1000;  // about 200 ms at the 1.965 GHz boost clock, longer below it
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
 template <int D, int NM>
@@ -46,7 +46,7 @@ struct TcCfg {
     static constexpr int kStages = D == 128 ? (NM == 1 ? 5 : 3) : 8;
     static constexpr int kSmemData = NM * kQBytes + NM * 2 * kPBytes + 2 * kStages * kTileBytes;
     static constexpr int kNumBars = 1 + 4 * kStages + 7 * NM;
-    static constexpr int kThreads = 64 + 128 * NM;
+    static constexpr int kThreads = 96 + 128 * NM;   // TMA warp, two MMA issuer warps, four softmax warps per row tile
     static constexpr int kPartStride = D + 4;        // floats per parked row (padding spreads the banks)
     static constexpr int kPartBytes = NM * kBM * kPartStride * 4 + NM * kBM * 8;
     static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
@@ -79,24 +79,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ uint64_t global_timer() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 // Bounded wait.  `dead` (shared memory) is set by the first wait that expires; later waits then give up at once.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead) {
     if (mbar_try_wait(bar, parity)) return;
-    const uint64_t t0 = global_timer();
+    const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return;
         if (*dead) return;
-        if (global_timer() - t0 > kWaitLimitNs) {
+        if (clock64() - t0 > kWaitLimitCycles) {
             *dead = 1;
             return;
         }
     }
+}
+// Whole-warp wait: lane 0 polls the barrier, the other lanes pick the result up at the warp barrier (one poller
+// per warp instead of 32 keeps the shared-memory barrier unit free for the arrivals).
+__device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* dead) {
+    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, dead);
+    __syncwarp();
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -139,6 +140,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+// N consecutive 32-bit columns of this thread's TMEM lane (N in {16, 32, 64}); the caller waits for the load.
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[N]) {
+    static_assert(N == 16 || N == 32 || N == 64, "column count");
+    if constexpr (N == 16) {
+        tmem_ld16(taddr, r);
+    } else if constexpr (N == 32) {
+        tmem_ld32(taddr, r);
+    } else {
+        tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+    }
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
     asm volatile(
@@ -217,14 +240,22 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, 
     t1 = (int)(((long long)n_tiles * (split + 1)) / splits);
 }
 
-template <int D, int NM>
+// REP > 1 (one row tile, G*T <= 128 / REP rows): the query rows are laid into the 128 MMA rows REP times
+// (copy c at rows c*128/REP...), every copy sees the same scores and owns the columns [c*64/REP, (c+1)*64/REP)
+// of each tile: its own running offset and sum, its own slice of P (the rest of its P rows stays zero), its
+// own accumulator rows.  The copies are merged like splits.  This spreads the exponentials of a small tree
+// over all four softmax warps instead of leaving them to one.
+template <int D, int NM, int REP>
 __global__ void __launch_bounds__(TcCfg<D, NM>::kThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const TcParams prm) {
+    static_assert(NM == 1 || REP == 1, "row copies only with a single row tile");
     using Cfg = TcCfg<D, NM>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
     constexpr int PS = Cfg::kPartStride;
+    constexpr int RB = kBM / REP;  // rows per copy
+    constexpr int CW = kBN / REP;  // columns of a tile per copy
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128B swizzle atoms need 1024-byte alignment
@@ -253,9 +284,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int T = prm.T, G = prm.Hq / prm.Hkv, R = G * T;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int mt0 = mg * NM;  // first row tile of this CTA
-    auto rows_in = [&](int t) {  // valid query rows of row tile t of this CTA
+    auto rows_in = [&](int t) {  // valid query rows of row tile t of this CTA (per copy when REP > 1)
         const int r = R - (mt0 + t) * kBM;
         return r < 0 ? 0 : (r > kBM ? kBM : r);
+    };
+    auto active_threads = [&](int t) {  // softmax threads of row tile t whose warp owns at least one valid row
+        return REP > 1 ? kBM : 32 * ((rows_in(t) + 31) / 32);
     };
     int nm_act = 0;  // row tiles with at least one row (they are the first ones)
 #pragma unroll
@@ -271,7 +305,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
 #pragma unroll
         for (int t = 0; t < NM; ++t) {
-            const uint32_t active = 32u * (uint32_t)((rows_in(t) + 31) / 32);  // threads of the warps that own a valid row
+            const uint32_t active = (uint32_t)active_threads(t) / 32u;  // one arrival per active warp
             for (int i = 0; i < 2; ++i) {
                 mbar_init(S_FULL(t, i), 1), mbar_init(S_EMPTY(t, i), active ? active : 1);
                 mbar_init(P_FULL(t, i), active ? active : 1);
@@ -282,6 +316,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         *dead = 0;
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
+    if (REP > 1 && warp >= 3) {
+        // a copy only ever writes its own columns of P: the rest of both P buffers must read as zero
+        // (each thread clears the row it later writes, so its own proxy fence before P_FULL covers these stores too)
+        unsigned char* pt = base_ptr + (sP - base) + ((warp & 3) * 32 + lane) * 128;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(pt + i * Cfg::kPBytes + ch * 16) = make_uint4(0, 0, 0, 0);
+    }
 
     griddep_wait();  // everything below may depend on the previous kernel of the stream
 
@@ -312,15 +355,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int n_first = nt < S ? nt : S;  // tiles whose ring slots are free from the start
     if (threadIdx.x == 0 && nt > 0) {
         // first pass of the ring before anyone else is ready: the loads only need the barriers this thread made
-        mbar_expect_tx(BAR(Q_FULL), q_bytes * nm_act);
-        for (int t = 0; t < nm_act; ++t)
-            for (int h = 0; h < NH; ++h)
-                tma_load_2d(sQ + t * Cfg::kQBytes + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0 + t * kBM);
+        if (REP > 1) {
+            mbar_expect_tx(BAR(Q_FULL), q_bytes * REP);
+            for (int c = 0; c < REP; ++c)  // the same rows once per copy, RB rows (a whole number of swizzle atoms) apart
+                for (int h = 0; h < NH; ++h)
+                    tma_load_2d(sQ + h * (kBM * 128) + c * (RB * 128), &map_q, BAR(Q_FULL), h * 64, q_row0);
+        } else {
+            mbar_expect_tx(BAR(Q_FULL), q_bytes * nm_act);
+            for (int t = 0; t < nm_act; ++t)
+                for (int h = 0; h < NH; ++h)
+                    tma_load_2d(sQ + t * Cfg::kQBytes + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0 + t * kBM);
+        }
         for (int j = 0; j < n_first; ++j) load_tile(j);
     }
     int bad_parent = 0;
-    if (warp >= 2 && !flags) {  // tree check: thread i looks at node i
-        const int i = threadIdx.x - 64;
+    if (warp >= 3 && !flags) {  // tree check: thread i looks at node i
+        const int i = threadIdx.x - 96;
         if (i < T) {
             const int p = prm.parent[(size_t)b * T + i];
             par_s[i] = p;
@@ -332,7 +382,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     tc_fence_after();
     griddep_launch_dependents();
     const bool run = flags == 0;
-    if (split == 0 && blockIdx.y == 0 && threadIdx.x == 64 && prm.status) prm.status[b] = flags;
+    if (split == 0 && blockIdx.y == 0 && threadIdx.x == 96 && prm.status) prm.status[b] = flags;
     const uint32_t tmem = *tmem_slot;
     auto TM_S = [&](int t, int i) { return tmem + (uint32_t)(t * 2 * kBN + i * kBN); };
     auto TM_O = [&](int t) { return tmem + (uint32_t)(NM * 2 * kBN + t * D); };
@@ -348,30 +398,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer =================
+        // ================= MMA issuer 1: S = Q K^T =================
         if (lane == 0 && nt > 0 && run) {
             constexpr uint32_t idesc_qk = instr_desc_bf16(kBM, kBN, false);
-            constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
-            auto issue_pv = [&](int jj) {
-                const int s = jj % S, it = jj / S;
-                mbar_wait(BAR(V_FULL + s), it & 1, dead);
-                const uint32_t v_base = sV + s * Cfg::kTileBytes;
-                for (int t = 0; t < nm_act; ++t) {
-                    mbar_wait(P_FULL(t, jj & 1), (jj >> 1) & 1, dead);
-                    tc_fence_after();
-                    const uint32_t p_base = sP + (t * 2 + (jj & 1)) * Cfg::kPBytes;
-#pragma unroll
-                    for (int kk = 0; kk < kBN / 16; ++kk) {
-                        // A = P [128 rows][64 slots], K-major: 32 bytes per K step inside the 128-byte row
-                        const uint64_t ad = smem_desc_sw128(p_base + kk * 32, 16, 1024);
-                        // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
-                        const uint64_t bd = smem_desc_sw128(v_base + kk * 2048, kBN * 128, 1024);
-                        tc_mma_bf16(TM_O(t), ad, bd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
-                    }
-                    tc_commit(PV_DONE(t));
-                }
-                tc_commit(BAR(V_EMPTY + s));
-            };
             mbar_wait(BAR(Q_FULL), 0, dead);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
@@ -390,20 +419,46 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     tc_commit(S_FULL(t, j & 1));
                 }
                 tc_commit(BAR(K_EMPTY + s));
-                if (j > 0) issue_pv(j - 1);
             }
-            issue_pv(nt - 1);
+        }
+    } else if (warp == 2) {
+        // ================= MMA issuer 2: O += P V (its own thread, so that neither product waits for the other's
+        //                   barriers: one issuing thread spends more time per tile than the tile takes to arrive) ====
+        if (lane == 0 && nt > 0 && run) {
+            constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
+            for (int j = 0; j < nt; ++j) {
+                const int s = j % S, it = j / S;
+                mbar_wait(BAR(V_FULL + s), it & 1, dead);
+                const uint32_t v_base = sV + s * Cfg::kTileBytes;
+                for (int t = 0; t < nm_act; ++t) {
+                    mbar_wait(P_FULL(t, j & 1), (j >> 1) & 1, dead);
+                    tc_fence_after();
+                    const uint32_t p_base = sP + (t * 2 + (j & 1)) * Cfg::kPBytes;
+#pragma unroll
+                    for (int kk = 0; kk < kBN / 16; ++kk) {
+                        // A = P [128 rows][64 slots], K-major: 32 bytes per K step inside the 128-byte row
+                        const uint64_t ad = smem_desc_sw128(p_base + kk * 32, 16, 1024);
+                        // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
+                        const uint64_t bd = smem_desc_sw128(v_base + kk * 2048, kBN * 128, 1024);
+                        tc_mma_bf16(TM_O(t), ad, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(PV_DONE(t));
+                }
+                tc_commit(BAR(V_EMPTY + s));
+            }
         }
     } else if (run) {
-        // ================= softmax / correction: one thread per query row =================
-        const int t = (warp - 2) >> 2;  // row tile of this warp group
+        // ================= softmax / correction: one thread per MMA row =================
+        const int t = (warp - 3) >> 2;  // row tile of this warp group
         const int wq = warp & 3;        // TMEM lane quadrant this warp may access
         const int row = wq * 32 + lane;
+        const int copy = row / RB, lr = row % RB;  // which copy of the rows, and the row within it
         const int rows_t = rows_in(t);
-        const bool warp_active = wq * 32 < rows_t;
-        const bool row_ok = row < rows_t;
-        const int gr = (mt0 + t) * kBM + row;
+        const bool warp_active = REP > 1 || wq * 32 < rows_t;
+        const bool row_ok = lr < rows_t;
+        const int gr = (mt0 + t) * kBM + lr;
         const int node = gr % T;
+        const int c0 = copy * CW;  // first tile column of this copy
         // the row's ancestor-or-self set as a 128-bit mask, straight from parent[] (checked above: the chain ends)
         uint64_t anc_lo = 0, anc_hi = 0;
         if (row_ok && node < n)
@@ -420,18 +475,19 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         if (warp_active)
             for (int j = 0; j < nt; ++j) {
                 const int kv0 = (t0 + j) * kBN;
-                mbar_wait(S_FULL(t, j & 1), (j >> 1) & 1, dead);
+                mbar_wait_warp(S_FULL(t, j & 1), (j >> 1) & 1, dead);
                 tc_fence_after();
-                uint32_t sr[2][32];
-                tmem_ld32(TM_S(t, j & 1) + lane_off, sr[0]);
-                tmem_ld32(TM_S(t, j & 1) + lane_off + 32, sr[1]);
-                tmem_wait_ld();
-                tc_fence_before();
-                mbar_arrive(S_EMPTY(t, j & 1));
-
-                float sv[kBN];
+                float sv[CW];
+                {
+                    uint32_t sr[CW];
+                    tmem_ld_cols<CW>(TM_S(t, j & 1) + lane_off + c0, sr);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(S_EMPTY(t, j & 1));
 #pragma unroll
-                for (int c = 0; c < kBN; ++c) sv[c] = __uint_as_float(sr[c >> 5][c & 31]);
+                    for (int c = 0; c < CW; ++c) sv[c] = __uint_as_float(sr[c]);
+                }
                 if (kv0 + kBN > L) {
                     // the tile touches tree slots or the tail: column c is visible iff it lies in the prefix or is the
                     // slot of a node on this row's root path
@@ -443,40 +499,41 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         const int sh = -off;  // first tree node of the tile
                         vis = sh < 64 ? ((anc_lo >> sh) | (anc_hi << (64 - sh))) : (sh < 128 ? (anc_hi >> (sh - 64)) : 0ull);
                     }
+                    vis >>= c0;
                     const uint32_t v0 = (uint32_t)vis, v1 = (uint32_t)(vis >> 32);
 #pragma unroll
-                    for (int c = 0; c < kBN; ++c) {
+                    for (int c = 0; c < CW; ++c) {
                         const bool on = (((c < 32 ? v0 : v1) >> (c & 31)) & 1u) != 0;
                         sv[c] = on ? sv[c] : -INFINITY;
                     }
                 }
-                float mx = sv[0];
+                float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};  // four independent chains
 #pragma unroll
-                for (int c = 1; c < kBN; ++c) mx = fmaxf(mx, sv[c]);
-                mx *= sc;  // sc > 0
+                for (int c = 4; c < CW; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sv[c]);
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;  // sc > 0
                 const bool grow = row_ok && mx > m + kRescaleThreshold;
                 const float m_new = grow ? mx : m;
                 const float alpha = grow ? exp2f(m - m_new) : 1.f;
-                float ls = 0.f;
-                uint32_t pk[kBN / 2];
+                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t pk[CW / 2];
 #pragma unroll
-                for (int c = 0; c < kBN; c += 2) {
+                for (int c = 0; c < CW; c += 2) {
                     const float p0 = exp2f(fmaf(sv[c], sc, -m_new)), p1 = exp2f(fmaf(sv[c + 1], sc, -m_new));
-                    ls += p0 + p1;
+                    ls4[(c >> 1) & 3] += p0 + p1;
                     const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
                     pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
                 }
-                l = l * alpha + ls;
+                l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
                 m = m_new;
 
                 if (j > 0) {
-                    mbar_wait(PV_DONE(t), (j - 1) & 1, dead);
+                    mbar_wait_warp(PV_DONE(t), (j - 1) & 1, dead);
                     tc_fence_after();
                     if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll
                         for (int cc = 0; cc < D / 32; ++cc) {
                             uint32_t o[32];
-                            tmem_ld32(TM_O(t) + lane_off + cc * 32, o);
+                            tmem_ld_cols<32>(TM_O(t) + lane_off + cc * 32, o);
                             tmem_wait_ld();
 #pragma unroll
                             for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
@@ -490,10 +547,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     // but 0 * NaN would poison O, so those V rows are cleared before the PV products read them (the
                     // MMA thread sees P_FULL of row tile 0 before it issues any PV of this tile)
                     const int s = j % S, it = j / S;
-                    mbar_wait(BAR(V_FULL + s), it & 1, dead);
+                    mbar_wait_warp(BAR(V_FULL + s), it & 1, dead);
                     const int first = Ltot - kv0;  // 1..63
                     unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
-                    const int stride = 32 * ((rows_t + 31) / 32);
+                    const int stride = active_threads(0);
                     for (int idx = row; idx < (kBN - first) * 8 * NH; idx += stride) {
                         const int h = idx / ((kBN - first) * 8), rem = idx % ((kBN - first) * 8);
                         const int r = first + rem / 8, ch = rem % 8;
@@ -504,18 +561,19 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 {
                     unsigned char* pt = base_ptr + (sP - base) + (t * 2 + (j & 1)) * Cfg::kPBytes + row * 128;
 #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch)
-                        *reinterpret_cast<uint4*>(pt + ((ch ^ (row & 7)) << 4)) =
+                    for (int ch = 0; ch < CW / 8; ++ch)
+                        *reinterpret_cast<uint4*>(pt + (((ch + c0 / 8) ^ (row & 7)) << 4)) =
                             make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
                 }
                 fence_async_smem();
                 tc_fence_before();
-                mbar_arrive(P_FULL(t, j & 1));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(P_FULL(t, j & 1));
             }
 
-        // ---- this split's result for the row: (m, l, unnormalised O)
+        // ---- this split's (and copy's) result for the row: (m, l, unnormalised O)
         if (warp_active && nt > 0) {
-            mbar_wait(PV_DONE(t), (nt - 1) & 1, dead);
+            mbar_wait_warp(PV_DONE(t), (nt - 1) & 1, dead);
             tc_fence_after();
         }
         const bool node_valid = row_ok && node < n;
@@ -528,7 +586,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 for (int cc = 0; cc < D / 32; ++cc) {
                     uint32_t o[32];
                     if (nt > 0) {
-                        tmem_ld32(TM_O(t) + lane_off + cc * 32, o);
+                        tmem_ld_cols<32>(TM_O(t) + lane_off + cc * 32, o);
                         tmem_wait_ld();
                     } else {
 #pragma unroll
@@ -543,14 +601,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 pml[t * kBM + row] = make_float2(m, l);
             }
         } else if (warp_active) {
-            const bool direct = prm.mode == kModeDirect;
+            const bool direct = prm.mode == kModeDirect;  // REP == 1 then
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
             const float inv = (node_valid && l > 0.f) ? 1.f / l : 0.f;
+            float* wrow = prm.ws + (orow * (size_t)(splits * REP) + (size_t)(split * REP + copy)) * (D + 2);
 #pragma unroll
             for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t o[32];
                 if (nt > 0) {
-                    tmem_ld32(TM_O(t) + lane_off + cc * 32, o);
+                    tmem_ld_cols<32>(TM_O(t) + lane_off + cc * 32, o);
                     tmem_wait_ld();
                 } else {
 #pragma unroll
@@ -570,7 +629,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     for (int v = 0; v < 4; ++v)
                         dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
                 } else {
-                    float* w = prm.ws + (orow * splits + split) * (D + 2) + cc * 32;
+                    float* w = wrow + cc * 32;
                     if (!node_valid) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c) o[c] = 0u;
@@ -580,44 +639,39 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         *reinterpret_cast<float2*>(w + c) = make_float2(__uint_as_float(o[c]), __uint_as_float(o[c + 1]));
                 }
             }
-            if (!direct && row_ok) {
-                float* w = prm.ws + (orow * splits + split) * (D + 2) + D;
-                *reinterpret_cast<float2*>(w) = make_float2(node_valid ? m : -INFINITY, node_valid ? l : 0.f);
-            }
+            if (!direct && row_ok)
+                *reinterpret_cast<float2*>(wrow + D) = make_float2(node_valid ? m : -INFINITY, node_valid ? l : 0.f);
         }
         tc_fence_before();
     }
 
     if (prm.mode == kModeCluster && run) {
-        // ---- merge the splits through distributed shared memory: this CTA owns rows rank, rank + splits, ...
+        // ---- merge the splits (and copies) through distributed shared memory: this CTA owns the output rows
+        //      rank, rank + splits, ... of every row tile
         __syncwarp();
         cluster_sync_all();
         const uint32_t rank = cluster_ctarank();
         const uint32_t part = base, part_ml = base + (uint32_t)(NM * kBM * PS * 4);
         constexpr int EPL = D / 32;  // output elements per lane
-        for (int idx = (int)rank + splits * warp; idx < NM * kBM; idx += splits * (Cfg::kThreads / 32)) {
-            const int t = idx / kBM, row = idx % kBM;
-            if (row >= rows_in(t)) continue;
-            const int gr = (mt0 + t) * kBM + row;
+        for (int idx = (int)rank + splits * warp; idx < NM * RB; idx += splits * (Cfg::kThreads / 32)) {
+            const int t = idx / RB, lr = idx % RB;
+            if (lr >= rows_in(t)) continue;
+            const int gr = (mt0 + t) * kBM + lr;
             const bool node_valid = (gr % T) < n;
-            float ms[kMaxClusterSplits], ls[kMaxClusterSplits];
             float M = -INFINITY;
+            for (int s = 0; s < splits; ++s)
 #pragma unroll
-            for (int s = 0; s < kMaxClusterSplits; ++s) {
-                ms[s] = -INFINITY, ls[s] = 0.f;
-                if (s < splits) {
-                    const float2 ml = ld_cluster_f2(map_to_cta(part_ml + (uint32_t)idx * 8u, (uint32_t)s));
-                    ms[s] = ml.x, ls[s] = ml.y;
-                    M = fmaxf(M, ml.x);
-                }
-            }
+                for (int c = 0; c < REP; ++c)
+                    M = fmaxf(M, ld_cluster_f2(map_to_cta(part_ml + (uint32_t)(t * kBM + c * RB + lr) * 8u, (uint32_t)s)).x);
             float num[4] = {0.f, 0.f, 0.f, 0.f}, den = 0.f;
+            for (int s = 0; s < splits; ++s)
 #pragma unroll
-            for (int s = 0; s < kMaxClusterSplits; ++s) {
-                if (s < splits) {
-                    const float f = exp2f(ms[s] - M);
-                    den = fmaf(f, ls[s], den);
-                    const uint32_t a = map_to_cta(part + ((uint32_t)idx * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)s);
+                for (int c = 0; c < REP; ++c) {
+                    const uint32_t prow = (uint32_t)(t * kBM + c * RB + lr);
+                    const float2 ml = ld_cluster_f2(map_to_cta(part_ml + prow * 8u, (uint32_t)s));
+                    const float f = exp2f(ml.x - M);
+                    den = fmaf(f, ml.y, den);
+                    const uint32_t a = map_to_cta(part + (prow * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)s);
                     if (EPL == 4) {
                         const float4 o = ld_cluster_f4(a);
                         num[0] = fmaf(f, o.x, num[0]), num[1] = fmaf(f, o.y, num[1]);
@@ -627,7 +681,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         num[0] = fmaf(f, o.x, num[0]), num[1] = fmaf(f, o.y, num[1]);
                     }
                 }
-            }
             const float inv = (node_valid && den > 0.f) ? 1.f / den : 0.f;
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;
             __nv_bfloat16* dst = prm.out + orow * D + lane * EPL;
@@ -711,19 +764,26 @@ static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
     return best;
 }
 
-size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
-    const int s = tc_splits(B, T, Hq, Hkv, C);
-    return s <= kMaxClusterSplits ? 0 : round_up((size_t)B * Hq * T * s * (d + 2) * sizeof(float), 256);
+// Copies of the query rows inside the one row tile (see the kernel): 4 up to 32 rows, 2 up to 64, else 1.
+static int tc_rep(int T, int Hq, int Hkv) {
+    const int R = (Hq / Hkv) * T;
+    return R <= 32 ? 4 : (R <= 64 ? 2 : 1);
 }
 
-template <int D, int NM>
+size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
+    const int s = tc_splits(B, T, Hq, Hkv, C);
+    return s <= kMaxClusterSplits ? 0
+                                  : round_up((size_t)B * Hq * T * s * tc_rep(T, Hq, Hkv) * (d + 2) * sizeof(float), 256);
+}
+
+template <int D, int NM, int REP>
 static s4c_status launch_tc(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
     using Cfg = TcCfg<D, NM>;
     static bool configured[64] = {};  // the opt-ins (dynamic shared memory, cluster size) are per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return S4C_ERR_CUDA;
         configured[dev] = true;
@@ -752,7 +812,7 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
     }
     cfg.attrs = attrs;
     cfg.numAttrs = na;
-    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM>, mq, mk, mv, prm) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP>, mq, mk, mv, prm) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
@@ -769,18 +829,26 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     const int nm = tc_nm(T, Hq, Hkv);
     prm.m_groups = tc_m_groups(T, Hq, Hkv);
     prm.splits = tc_splits(B, T, Hq, Hkv, C);
-    prm.mode = prm.splits == 1 ? kModeDirect : (prm.splits <= kMaxClusterSplits ? kModeCluster : kModeWorkspace);
+    const int rep = tc_rep(T, Hq, Hkv);
+    // the copies of a row merge like splits, so a single split with copies still takes the (one-CTA) cluster path
+    prm.mode = prm.splits > kMaxClusterSplits ? kModeWorkspace : (prm.splits == 1 && rep == 1 ? kModeDirect : kModeCluster);
     const int R = (Hq / Hkv) * T;
     prm.q_box_rows = R >= kBM ? kBM : (int)round_up((size_t)R, 8);
     prm.scale_log2 = scale * 1.4426950408889634f;
     s4c_status st;
     if (d == 128)
-        st = nm == 1 ? launch_tc<128, 1>(q, k, v, prm, B, stream) : launch_tc<128, 2>(q, k, v, prm, B, stream);
+        st = nm == 2   ? launch_tc<128, 2, 1>(q, k, v, prm, B, stream)
+             : rep == 4 ? launch_tc<128, 1, 4>(q, k, v, prm, B, stream)
+             : rep == 2 ? launch_tc<128, 1, 2>(q, k, v, prm, B, stream)
+                        : launch_tc<128, 1, 1>(q, k, v, prm, B, stream);
     else
-        st = nm == 1 ? launch_tc<64, 1>(q, k, v, prm, B, stream) : launch_tc<64, 2>(q, k, v, prm, B, stream);
+        st = nm == 2   ? launch_tc<64, 2, 1>(q, k, v, prm, B, stream)
+             : rep == 4 ? launch_tc<64, 1, 4>(q, k, v, prm, B, stream)
+             : rep == 2 ? launch_tc<64, 1, 2>(q, k, v, prm, B, stream)
+                        : launch_tc<64, 1, 1>(q, k, v, prm, B, stream);
     if (st != S4C_OK) return st;
     if (prm.mode == kModeWorkspace)
-        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits, S4C_BF16, stream);
+        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits * rep, S4C_BF16, stream);
     return S4C_OK;
 }
 
