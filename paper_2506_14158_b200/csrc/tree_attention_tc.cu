@@ -195,12 +195,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 }
 __device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
     float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
     float2 v;
-    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
@@ -268,6 +268,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 480);
     volatile int* dead = reinterpret_cast<volatile int*>(tail + 484);
+    int* bad_s = reinterpret_cast<int*>(tail + 488);  // S4C_SEQ_* flags found by the softmax warps (malformed tree)
     int32_t* par_s = reinterpret_cast<int32_t*>(tail + 512);  // S4C_MAX_T * 4 = 512 bytes
 
     const uint32_t bar0 = smem_u32(bars);
@@ -295,25 +296,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
     for (int t = 0; t < NM; ++t) nm_act += rows_in(t) > 0 ? 1 : 0;
 
-    // ---- prologue that touches no global memory: barriers, TMEM, descriptor prefetch
-    if (threadIdx.x == 0) {
-        tma_prefetch_desc(&map_q), tma_prefetch_desc(&map_k), tma_prefetch_desc(&map_v);
-        mbar_init(BAR(Q_FULL), 1);
-        for (int s = 0; s < S; ++s) {
-            mbar_init(BAR(K_FULL + s), 1), mbar_init(BAR(K_EMPTY + s), 1);
-            mbar_init(BAR(V_FULL + s), 1), mbar_init(BAR(V_EMPTY + s), 1);
-        }
-#pragma unroll
-        for (int t = 0; t < NM; ++t) {
-            const uint32_t active = (uint32_t)active_threads(t) / 32u;  // one arrival per active warp
-            for (int i = 0; i < 2; ++i) {
-                mbar_init(S_FULL(t, i), 1), mbar_init(S_EMPTY(t, i), active ? active : 1);
-                mbar_init(P_FULL(t, i), active ? active : 1);
+    // ---- prologue that touches no global memory: barriers (one per lane of warp 0), TMEM, descriptor prefetch
+    if (warp == 0) {
+        for (int i = lane; i < Cfg::kNumBars; i += 32) {
+            uint32_t count = 1;  // every barrier but the two the softmax warps arrive on: one arrival per active warp
+            if (i >= PER_TILE) {
+                const int t = (i - PER_TILE) / 7, k = (i - PER_TILE) % 7;
+                const uint32_t active = (uint32_t)active_threads(t) / 32u;
+                if (k >= 2 && k < 6 && active) count = active;
             }
-            mbar_init(PV_DONE(t), 1);
+            mbar_init(BAR(i), count);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        *dead = 0;
+        if (lane == 0) {
+            tma_prefetch_desc(&map_q), tma_prefetch_desc(&map_k), tma_prefetch_desc(&map_v);
+            *dead = 0;
+            *bad_s = 0;
+        }
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
     if (REP > 1 && warp >= 3) {
@@ -325,6 +324,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(pt + i * Cfg::kPBytes + ch * 16) = make_uint4(0, 0, 0, 0);
     }
+    tc_fence_before();
+    __syncthreads();  // the only CTA-wide barrier before the results: from here on the roles run on mbarriers alone
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    auto TM_S = [&](int t, int i) { return tmem + (uint32_t)(t * 2 * kBN + i * kBN); };
+    auto TM_O = [&](int t) { return tmem + (uint32_t)(NM * 2 * kBN + t * D); };
 
     griddep_wait();  // everything below may depend on the previous kernel of the stream
 
@@ -335,71 +340,51 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int Ltot = L + n;
     int t0 = 0, t1 = 0;
     if (!flags) split_range((Ltot + kBN - 1) / kBN, splits, split, t0, t1);
-    const int nt = t1 - t0;  // 0 when the lengths are unusable: nothing is loaded then
+    const int nt = t1 - t0;  // 0 when the lengths are unusable: nothing is loaded, issued or stored then
+    griddep_launch_dependents();
 
     const int q_row0 = (b * prm.Hq + hk * G) * T + mt0 * kBM;  // row of the [B*Hq*T, d] view of q
     const int kv_row0 = (b * prm.Hkv + hk) * prm.C;            // row of the [B*Hkv*C, d] view of the caches
     const uint32_t q_bytes = (uint32_t)prm.q_box_rows * 128u * NH;
 
-    auto load_tile = [&](int j) {  // TMA producer thread only
-        const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
-        mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead);
-        mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
-        for (int h = 0; h < NH; ++h)
-            tma_load_2d(sK + s * Cfg::kTileBytes + h * (kBN * 128), &map_k, BAR(K_FULL + s), h * 64, row);
-        mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead);
-        mbar_expect_tx(BAR(V_FULL + s), Cfg::kTileBytes);
-        for (int h = 0; h < NH; ++h)
-            tma_load_2d(sV + s * Cfg::kTileBytes + h * (kBN * 128), &map_v, BAR(V_FULL + s), h * 64, row);
-    };
-    const int n_first = nt < S ? nt : S;  // tiles whose ring slots are free from the start
-    if (threadIdx.x == 0 && nt > 0) {
-        // first pass of the ring before anyone else is ready: the loads only need the barriers this thread made
-        if (REP > 1) {
-            mbar_expect_tx(BAR(Q_FULL), q_bytes * REP);
-            for (int c = 0; c < REP; ++c)  // the same rows once per copy, RB rows (a whole number of swizzle atoms) apart
-                for (int h = 0; h < NH; ++h)
-                    tma_load_2d(sQ + h * (kBM * 128) + c * (RB * 128), &map_q, BAR(Q_FULL), h * 64, q_row0);
-        } else {
-            mbar_expect_tx(BAR(Q_FULL), q_bytes * nm_act);
-            for (int t = 0; t < nm_act; ++t)
-                for (int h = 0; h < NH; ++h)
-                    tma_load_2d(sQ + t * Cfg::kQBytes + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0 + t * kBM);
-        }
-        for (int j = 0; j < n_first; ++j) load_tile(j);
-    }
-    int bad_parent = 0;
-    if (warp >= 3 && !flags) {  // tree check: thread i looks at node i
-        const int i = threadIdx.x - 96;
-        if (i < T) {
-            const int p = prm.parent[(size_t)b * T + i];
-            par_s[i] = p;
-            bad_parent = i < n && ((i == 0 && p != -1) || (i > 0 && (p < 0 || p >= i)));
-        }
-    }
-    tc_fence_before();
-    if (__syncthreads_or(bad_parent)) flags |= S4C_SEQ_BAD_PARENT;
-    tc_fence_after();
-    griddep_launch_dependents();
-    const bool run = flags == 0;
-    if (split == 0 && blockIdx.y == 0 && threadIdx.x == 96 && prm.status) prm.status[b] = flags;
-    const uint32_t tmem = *tmem_slot;
-    auto TM_S = [&](int t, int i) { return tmem + (uint32_t)(t * 2 * kBN + i * kBN); };
-    auto TM_O = [&](int t) { return tmem + (uint32_t)(NM * 2 * kBN + t * D); };
-
     if (warp == 0) {
         // ================= TMA producer =================
-        if (lane == 0 && nt > 0) {
-            if (run) {
-                for (int j = n_first; j < nt; ++j) load_tile(j);
-            } else {  // malformed tree: nobody consumes what was requested; let it land before the CTA goes away
-                mbar_wait(BAR(Q_FULL), 0, dead);
-                for (int j = 0; j < n_first; ++j) mbar_wait(BAR(K_FULL + j), 0, dead), mbar_wait(BAR(V_FULL + j), 0, dead);
+        auto load_tile = [&](int j) {
+            const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
+            mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead);
+            mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
+            for (int h = 0; h < NH; ++h)
+                tma_load_2d(sK + s * Cfg::kTileBytes + h * (kBN * 128), &map_k, BAR(K_FULL + s), h * 64, row);
+            mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead);
+            mbar_expect_tx(BAR(V_FULL + s), Cfg::kTileBytes);
+            for (int h = 0; h < NH; ++h)
+                tma_load_2d(sV + s * Cfg::kTileBytes + h * (kBN * 128), &map_v, BAR(V_FULL + s), h * 64, row);
+        };
+        if (nt > 0) {
+            // first pass of the ring, every ring slot still free: lane j requests tile j, the last lane requests Q,
+            // all at once (one thread needs about 50 ns per request)
+            if (lane == 31) {
+                if (REP > 1) {
+                    mbar_expect_tx(BAR(Q_FULL), q_bytes * REP);
+                    for (int c = 0; c < REP; ++c)  // the same rows once per copy, RB rows (whole swizzle atoms) apart
+                        for (int h = 0; h < NH; ++h)
+                            tma_load_2d(sQ + h * (kBM * 128) + c * (RB * 128), &map_q, BAR(Q_FULL), h * 64, q_row0);
+                } else {
+                    mbar_expect_tx(BAR(Q_FULL), q_bytes * nm_act);
+                    for (int t = 0; t < nm_act; ++t)
+                        for (int h = 0; h < NH; ++h)
+                            tma_load_2d(sQ + t * Cfg::kQBytes + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0 + t * kBM);
+                }
+            } else if (lane < S && lane < nt) {
+                load_tile(lane);
             }
+            __syncwarp();
+            if (lane == 0)
+                for (int j = S; j < nt; ++j) load_tile(j);
         }
     } else if (warp == 1) {
         // ================= MMA issuer 1: S = Q K^T =================
-        if (lane == 0 && nt > 0 && run) {
+        if (lane == 0 && nt > 0) {
             constexpr uint32_t idesc_qk = instr_desc_bf16(kBM, kBN, false);
             mbar_wait(BAR(Q_FULL), 0, dead);
             for (int j = 0; j < nt; ++j) {
@@ -424,7 +409,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     } else if (warp == 2) {
         // ================= MMA issuer 2: O += P V (its own thread, so that neither product waits for the other's
         //                   barriers: one issuing thread spends more time per tile than the tile takes to arrive) ====
-        if (lane == 0 && nt > 0 && run) {
+        if (lane == 0 && nt > 0) {
             constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
@@ -447,8 +432,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tc_commit(BAR(V_EMPTY + s));
             }
         }
-    } else if (run) {
+    } else {
         // ================= softmax / correction: one thread per MMA row =================
+        // tree check first: softmax thread i looks at node i; a malformed tree still runs the pipeline (with empty
+        // masks, so that no role waits for another) and only its outputs are withheld
+        if (!flags) {
+            const int i = threadIdx.x - 96;
+            if (i < T) {
+                const int p = prm.parent[(size_t)b * T + i];
+                par_s[i] = p;
+                if (i < n && ((i == 0 && p != -1) || (i > 0 && (p < 0 || p >= i)))) atomicOr(bad_s, S4C_SEQ_BAD_PARENT);
+            }
+        }
+        named_bar_sync(1, NM * 128);
+        flags |= *bad_s;
+        if (split == 0 && blockIdx.y == 0 && threadIdx.x == 96 && prm.status) prm.status[b] = flags;
+        const bool run = flags == 0;
         const int t = (warp - 3) >> 2;  // row tile of this warp group
         const int wq = warp & 3;        // TMEM lane quadrant this warp may access
         const int row = wq * 32 + lane;
@@ -461,7 +460,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const int c0 = copy * CW;  // first tile column of this copy
         // the row's ancestor-or-self set as a 128-bit mask, straight from parent[] (checked above: the chain ends)
         uint64_t anc_lo = 0, anc_hi = 0;
-        if (row_ok && node < n)
+        if (run && row_ok && node < n)
             for (int u = node, guard = 0; u >= 0 && guard <= T; u = par_s[u], ++guard) {
                 if (u < 64)
                     anc_lo |= 1ull << u;
@@ -600,7 +599,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)NM * kBM * PS);
                 pml[t * kBM + row] = make_float2(m, l);
             }
-        } else if (warp_active) {
+        } else if (warp_active && run) {
             const bool direct = prm.mode == kModeDirect;  // REP == 1 then
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
             const float inv = (node_valid && l > 0.f) ? 1.f / l : 0.f;
@@ -645,54 +644,71 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         tc_fence_before();
     }
 
-    if (prm.mode == kModeCluster && run) {
+    if (prm.mode == kModeCluster) {
         // ---- merge the splits (and copies) through distributed shared memory: this CTA owns the output rows
-        //      rank, rank + splits, ... of every row tile
+        //      rank, rank + splits, ... of every row tile; one warp per row, lane i first fetches (offset, sum) of
+        //      partial i, then every lane gathers its 4 (d = 64: 2) output columns from all partials, 8 loads in flight
         __syncwarp();
         cluster_sync_all();
+        const bool run = (flags | *bad_s) == 0;  // the same in every CTA of the cluster: it depends on the sequence only
         const uint32_t rank = cluster_ctarank();
         const uint32_t part = base, part_ml = base + (uint32_t)(NM * kBM * PS * 4);
         constexpr int EPL = D / 32;  // output elements per lane
-        for (int idx = (int)rank + splits * warp; idx < NM * RB; idx += splits * (Cfg::kThreads / 32)) {
-            const int t = idx / RB, lr = idx % RB;
-            if (lr >= rows_in(t)) continue;
-            const int gr = (mt0 + t) * kBM + lr;
-            const bool node_valid = (gr % T) < n;
-            float M = -INFINITY;
-            for (int s = 0; s < splits; ++s)
+        const int np = splits * REP;  // partials per output row (<= 32)
+        if (run)
+            for (int idx = (int)rank + splits * warp; idx < NM * RB; idx += splits * (Cfg::kThreads / 32)) {
+                const int t = idx / RB, lr = idx % RB;
+                if (lr >= rows_in(t)) continue;
+                const int gr = (mt0 + t) * kBM + lr;
+                const bool node_valid = (gr % T) < n;
+                // partial i = (split i / REP, copy i % REP)
+                float2 ml = make_float2(-INFINITY, 0.f);
+                if (lane < np)
+                    ml = ld_cluster_f2(map_to_cta(part_ml + (uint32_t)(t * kBM + (lane % REP) * RB + lr) * 8u, (uint32_t)(lane / REP)));
+                float M = ml.x;
 #pragma unroll
-                for (int c = 0; c < REP; ++c)
-                    M = fmaxf(M, ld_cluster_f2(map_to_cta(part_ml + (uint32_t)(t * kBM + c * RB + lr) * 8u, (uint32_t)s)).x);
-            float num[4] = {0.f, 0.f, 0.f, 0.f}, den = 0.f;
-            for (int s = 0; s < splits; ++s)
+                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                const float f_mine = lane < np ? exp2f(ml.x - M) : 0.f;
+                float den = f_mine * ml.y;  // summed in a fixed (butterfly) order: the same on every run
 #pragma unroll
-                for (int c = 0; c < REP; ++c) {
-                    const uint32_t prow = (uint32_t)(t * kBM + c * RB + lr);
-                    const float2 ml = ld_cluster_f2(map_to_cta(part_ml + prow * 8u, (uint32_t)s));
-                    const float f = exp2f(ml.x - M);
-                    den = fmaf(f, ml.y, den);
-                    const uint32_t a = map_to_cta(part + (prow * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)s);
-                    if (EPL == 4) {
-                        const float4 o = ld_cluster_f4(a);
-                        num[0] = fmaf(f, o.x, num[0]), num[1] = fmaf(f, o.y, num[1]);
-                        num[2] = fmaf(f, o.z, num[2]), num[3] = fmaf(f, o.w, num[3]);
-                    } else {
-                        const float2 o = ld_cluster_f2(a);
-                        num[0] = fmaf(f, o.x, num[0]), num[1] = fmaf(f, o.y, num[1]);
+                for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+                float num[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int i0 = 0; i0 < np; i0 += 8) {
+                    float4 o4[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int i = i0 + k;
+                        o4[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (i < np) {
+                            const uint32_t prow = (uint32_t)(t * kBM + (i % REP) * RB + lr);
+                            const uint32_t a = map_to_cta(part + (prow * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)(i / REP));
+                            if (EPL == 4) {
+                                o4[k] = ld_cluster_f4(a);
+                            } else {
+                                const float2 o2 = ld_cluster_f2(a);
+                                o4[k].x = o2.x, o4[k].y = o2.y;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const float f = __shfl_sync(0xffffffffu, f_mine, (i0 + k) & 31);
+                        num[0] = fmaf(f, o4[k].x, num[0]), num[1] = fmaf(f, o4[k].y, num[1]);
+                        num[2] = fmaf(f, o4[k].z, num[2]), num[3] = fmaf(f, o4[k].w, num[3]);
                     }
                 }
-            const float inv = (node_valid && den > 0.f) ? 1.f / den : 0.f;
-            const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;
-            __nv_bfloat16* dst = prm.out + orow * D + lane * EPL;
-            const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
-            if (EPL == 4) {
-                const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[2] * inv, num[3] * inv);
-                *reinterpret_cast<uint2*>(dst) =
-                    make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-            } else {
-                *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(&h0);
+                const float inv = (node_valid && den > 0.f) ? 1.f / den : 0.f;
+                const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;
+                __nv_bfloat16* dst = prm.out + orow * D + lane * EPL;
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
+                if (EPL == 4) {
+                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[2] * inv, num[3] * inv);
+                    *reinterpret_cast<uint2*>(dst) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                } else {
+                    *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(&h0);
+                }
             }
-        }
         __syncwarp();
         cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
     } else {
