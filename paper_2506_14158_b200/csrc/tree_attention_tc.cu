@@ -42,9 +42,8 @@ struct TcCfg {
     static constexpr int kHalves = D / 64;           // 64-element (128-byte) swizzle atoms along d
     static constexpr int kQBytes = kBM * D * 2;      // one row tile of Q: 32 KB (d = 128)
     static constexpr int kTileBytes = kBN * D * 2;   // 16 KB: one K or V tile
-    static constexpr int kPBytes = kBM * kBN * 2;    // 16 KB
-    static constexpr int kStages = D == 128 ? (NM == 1 ? 5 : 3) : 8;
-    static constexpr int kSmemData = NM * kQBytes + NM * 2 * kPBytes + 2 * kStages * kTileBytes;
+    static constexpr int kStages = D == 128 ? (NM == 1 ? 6 : 5) : 8;
+    static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes;
     static constexpr int kNumBars = 1 + 4 * kStages + 7 * NM;
     static constexpr int kThreads = 96 + 128 * NM;   // TMA warp, two MMA issuer warps, four softmax warps per row tile
     static constexpr int kPartStride = D + 4;        // floats per parked row (padding spreads the banks)
@@ -129,6 +128,16 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same product with the A operand in tensor memory: 128 lanes (rows) x 8 columns, each 32-bit cell two bf16 (the
+// lower K index in the lower half).
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -173,6 +182,31 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
         "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+// N consecutive 32-bit columns of this thread's TMEM lane (N in {8, 16, 32}); the caller waits for the store.
+template <int N>
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t (&r)[N]) {
+    static_assert(N == 8 || N == 16 || N == 32, "column count");
+    if constexpr (N == 8) {
+        tmem_st8(taddr, r);
+    } else if constexpr (N == 16) {
+        tmem_st16(taddr, r);
+    } else {
+        tmem_st32(taddr, r);
+    }
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -261,8 +295,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128B swizzle atoms need 1024-byte alignment
     unsigned char* base_ptr = smem_raw + (base - raw);
     const uint32_t sQ = base;
-    const uint32_t sP = sQ + NM * Cfg::kQBytes;
-    const uint32_t sK = sP + NM * 2 * Cfg::kPBytes;
+    const uint32_t sK = sQ + NM * Cfg::kQBytes;
     const uint32_t sV = sK + S * Cfg::kTileBytes;
     unsigned char* tail = base_ptr + Cfg::kSmemData;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
@@ -299,11 +332,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // ---- prologue that touches no global memory: barriers (one per lane of warp 0), TMEM, descriptor prefetch
     if (warp == 0) {
         for (int i = lane; i < Cfg::kNumBars; i += 32) {
-            uint32_t count = 1;  // every barrier but the two the softmax warps arrive on: one arrival per active warp
+            uint32_t count = 1;  // every barrier but P_FULL, which takes one arrival per active softmax warp
             if (i >= PER_TILE) {
                 const int t = (i - PER_TILE) / 7, k = (i - PER_TILE) % 7;
                 const uint32_t active = (uint32_t)active_threads(t) / 32u;
-                if (k >= 2 && k < 6 && active) count = active;
+                if (k >= 4 && k < 6 && active) count = active;
             }
             mbar_init(BAR(i), count);
         }
@@ -315,15 +348,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
-    if (REP > 1 && warp >= 3) {
-        // a copy only ever writes its own columns of P: the rest of both P buffers must read as zero
-        // (each thread clears the row it later writes, so its own proxy fence before P_FULL covers these stores too)
-        unsigned char* pt = base_ptr + (sP - base) + ((warp & 3) * 32 + lane) * 128;
-#pragma unroll
-        for (int i = 0; i < 2; ++i)
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(pt + i * Cfg::kPBytes + ch * 16) = make_uint4(0, 0, 0, 0);
-    }
     tc_fence_before();
     __syncthreads();  // the only CTA-wide barrier before the results: from here on the roles run on mbarriers alone
     tc_fence_after();
@@ -418,16 +442,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 for (int t = 0; t < nm_act; ++t) {
                     mbar_wait(P_FULL(t, j & 1), (j >> 1) & 1, dead);
                     tc_fence_after();
-                    const uint32_t p_base = sP + (t * 2 + (j & 1)) * Cfg::kPBytes;
 #pragma unroll
                     for (int kk = 0; kk < kBN / 16; ++kk) {
-                        // A = P [128 rows][64 slots], K-major: 32 bytes per K step inside the 128-byte row
-                        const uint64_t ad = smem_desc_sw128(p_base + kk * 32, 16, 1024);
+                        // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
                         // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
                         const uint64_t bd = smem_desc_sw128(v_base + kk * 2048, kBN * 128, 1024);
-                        tc_mma_bf16(TM_O(t), ad, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                        tc_mma_bf16_ts(TM_O(t), TM_S(t, j & 1) + kk * 8, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
                     }
                     tc_commit(PV_DONE(t));
+                    tc_commit(S_EMPTY(t, j & 1));  // the score buffer (and the P inside it) may be overwritten
                 }
                 tc_commit(BAR(V_EMPTY + s));
             }
@@ -481,9 +504,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     uint32_t sr[CW];
                     tmem_ld_cols<CW>(TM_S(t, j & 1) + lane_off + c0, sr);
                     tmem_wait_ld();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(S_EMPTY(t, j & 1));
 #pragma unroll
                     for (int c = 0; c < CW; ++c) sv[c] = __uint_as_float(sr[c]);
                 }
@@ -555,16 +575,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         const int r = first + rem / 8, ch = rem % 8;
                         *reinterpret_cast<uint4*>(vt + h * (kBN * 128) + r * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
                     }
+                    fence_async_smem();  // generic-proxy stores, read by the tensor core through the async proxy
                 }
-                // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
+                // P row -> tensor memory, packed two bf16 per column over the first 32 columns of this score buffer (the
+                // scores were read above).  A copy owns CW/2 of these columns and clears the others: the product runs
+                // over all 64 slots of every row.
                 {
-                    unsigned char* pt = base_ptr + (sP - base) + (t * 2 + (j & 1)) * Cfg::kPBytes + row * 128;
+                    const uint32_t p_row = TM_S(t, j & 1) + lane_off;
+                    tmem_st_cols<CW / 2>(p_row + c0 / 2, pk);
+                    if (REP > 1) {
+                        uint32_t zero[CW / 2];
 #pragma unroll
-                    for (int ch = 0; ch < CW / 8; ++ch)
-                        *reinterpret_cast<uint4*>(pt + (((ch + c0 / 8) ^ (row & 7)) << 4)) =
-                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                        for (int c = 0; c < CW / 2; ++c) zero[c] = 0u;
+#pragma unroll
+                        for (int k = 1; k < REP; ++k) tmem_st_cols<CW / 2>(p_row + ((copy + k) % REP) * (CW / 2), zero);
+                    }
+                    tmem_wait_st();
                 }
-                fence_async_smem();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(P_FULL(t, j & 1));
