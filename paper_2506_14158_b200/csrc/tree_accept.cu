@@ -44,10 +44,19 @@ struct NodeStats {
 
 static inline int accept_splits(int V) { return ceil_div(V, kSegElems); }
 
+struct NodeSummary {  // per-node result of the cluster path
+    double S;  // sum exp((x - M)/tau)
+    double Z;  // sum max(p - q, 0)
+    double Q;  // sum of q, the first child's token left out
+    float M;
+    int idx;   // lowest index attaining M
+};
+
 struct AcceptWorkspace {
     RowPartial* row;
     ResPartial* res;
     NodeStats* node;
+    NodeSummary* summary;
 };
 static inline size_t accept_ws_layout(int B, int T, int V, char* base, AcceptWorkspace* ws) {
     const size_t n = (size_t)B * T * accept_splits(V);
@@ -58,6 +67,8 @@ static inline size_t accept_ws_layout(int B, int T, int V, char* base, AcceptWor
     off += round_up(n * sizeof(ResPartial), 256);
     if (ws) ws->node = reinterpret_cast<NodeStats*>(base + off);
     off += round_up((size_t)B * T * sizeof(NodeStats), 256);
+    if (ws) ws->summary = reinterpret_cast<NodeSummary*>(base + off);
+    off += round_up((size_t)B * T * sizeof(NodeSummary), 256);
     return off;
 }
 
@@ -463,6 +474,444 @@ accept_walk_kernel(const float* __restrict__ logits, const float* __restrict__ d
     }
 }
 
+
+// ============================================================================= cluster path
+// The default path when V is a multiple of 4 and at most 8 * 1024 * 16: one thread-block cluster of 8 CTAs per
+// (sequence, node) row keeps the row's logits in registers, so every logit and every draft probability is read
+// from HBM exactly once and exponentiated exactly once; the row-wide maximum, sum and residual mass are merged
+// across the cluster through distributed shared memory in CTA-rank order (deterministic).  The walk then runs
+// as one cluster per sequence, its vocabulary-wide passes spread over the 8 CTAs.
+constexpr int kCl = 8;             // CTAs per cluster
+constexpr int kClEpt = 16;         // row elements per thread
+constexpr int kClMaxThreads = 1024;
+constexpr int kClMaxV = kCl * kClMaxThreads * kClEpt;
+
+__device__ __forceinline__ uint32_t cl_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cl_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Reads 8 bytes at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ double cl_peer_f64(const double* local, uint32_t rank) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(local);
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    double v;
+    asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(ra));
+    return v;
+}
+
+// exp(t) for t <= 0 in float64, about 1 ulp: t = (32 k + j) ln2/32 + r, exp(t) = 2^k * 2^(j/32) * e^r with |r| <=
+// ln2/64 and a degree-6 polynomial for e^r (remainder below 4e-18).  About a third of the float64 instructions of
+// the library exp, which matters because this path is otherwise bound by the float64 pipe, not by HBM.
+__device__ const double kExp2Frac[32] = {
+    0x1.0000000000000p+0, 0x1.059b0d3158574p+0, 0x1.0b5586cf9890fp+0, 0x1.11301d0125b51p+0,
+    0x1.172b83c7d517bp+0, 0x1.1d4873168b9aap+0, 0x1.2387a6e756238p+0, 0x1.29e9df51fdee1p+0,
+    0x1.306fe0a31b715p+0, 0x1.371a7373aa9cbp+0, 0x1.3dea64c123422p+0, 0x1.44e086061892dp+0,
+    0x1.4bfdad5362a27p+0, 0x1.5342b569d4f82p+0, 0x1.5ab07dd485429p+0, 0x1.6247eb03a5585p+0,
+    0x1.6a09e667f3bcdp+0, 0x1.71f75e8ec5f74p+0, 0x1.7a11473eb0187p+0, 0x1.82589994cce13p+0,
+    0x1.8ace5422aa0dbp+0, 0x1.93737b0cdc5e5p+0, 0x1.9c49182a3f090p+0, 0x1.a5503b23e255dp+0,
+    0x1.ae89f995ad3adp+0, 0x1.b7f76f2fb5e47p+0, 0x1.c199bdd85529cp+0, 0x1.cb720dcef9069p+0,
+    0x1.d5818dcfba487p+0, 0x1.dfc97337b9b5fp+0, 0x1.ea4afa2a490dap+0, 0x1.f50765b6e4540p+0};
+
+__device__ __forceinline__ double exp_nonpos(double t, const double* tab /* shared copy of kExp2Frac */) {
+    const double kd = rint(t * 0x1.71547652b82fep+5);  // t * 32/ln2
+    if (!(kd > -32000.0)) return exp(t);                // result near or below the normal range (also -inf, NaN)
+    const int k = (int)kd;
+    double r = fma(-kd, 0x1.62e42fefa39efp-6, t);       // ln2/32, high and low part
+    r = fma(-kd, 0x1.abc9e3b39803fp-61, r);
+    double pl = fma(r, 1.0 / 720.0, 1.0 / 120.0);
+    pl = fma(pl, r, 1.0 / 24.0);
+    pl = fma(pl, r, 1.0 / 6.0);
+    pl = fma(pl, r, 0.5);
+    pl = fma(pl, r, 1.0);
+    pl = pl * r;                                        // e^r - 1
+    const double tj = tab[k & 31];
+    const double y = fma(tj, pl, tj);                   // in [1, 2.05)
+    return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));  // * 2^(k >> 5), exponent stays normal
+}
+
+// Cluster-wide exchange area of one CTA: written by its thread 0, read by every peer after a cluster barrier.  Every
+// round has fields of its own, so a round never overwrites what a slower peer may still be reading.
+struct ClSlots {
+    double m, idx, s, z, qs;
+};
+
+// After a cluster barrier: all 8 CTAs' values of up to two slot fields, in rank order, into shared arrays of 8.
+// Call from every thread of every CTA of the cluster.
+__device__ __forceinline__ void cl_gather(const double* f0, double* d0, const double* f1 = nullptr, double* d1 = nullptr) {
+    cl_sync();
+    if (threadIdx.x < kCl) {
+        d0[threadIdx.x] = cl_peer_f64(f0, threadIdx.x);
+        if (f1) d1[threadIdx.x] = cl_peer_f64(f1, threadIdx.x);
+    }
+    __syncthreads();
+}
+
+template <int THREADS, bool STOCH>
+__global__ void __launch_bounds__(THREADS, THREADS == 1024 ? 1 : 2)
+accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
+                            const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                            const int32_t* __restrict__ n_nodes, int T, int V, int chunk, double inv_tau,
+                            NodeSummary* __restrict__ out) {
+    const int node = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
+    const int n = n_nodes ? n_nodes[b] : T;
+    if (node >= n || n > T) return;  // the whole cluster leaves together: nobody is left waiting at a barrier
+    const uint32_t rank = cl_rank();
+    const size_t off = ((size_t)b * T + node) * V;
+    const int c0 = (int)rank * chunk;
+
+    __shared__ ClSlots slot;
+    __shared__ double gathered[kCl], gathered2[kCl];
+    __shared__ double scratch[33];
+    __shared__ double tab[32];
+    __shared__ float wm[THREADS / 32];
+    __shared__ int wi[THREADS / 32];
+    __shared__ int first_tok;
+    if (tid < 32) tab[tid] = kExp2Frac[tid];
+    if (STOCH && tid == 32) {  // token of the first child in index order (the first one ever rejected at this node)
+        int ft = -1;
+        for (int c = node + 1; c < n; ++c)
+            if (parent[(size_t)b * T + c] == node) {
+                ft = tokens[(size_t)b * T + c];
+                break;
+            }
+        first_tok = ft;
+    }
+
+    // ---- the row segment of this thread: 4 x 16 bytes of logits (and of draft probabilities), requested up front
+    float x[kClEpt], q[kClEpt];
+#pragma unroll
+    for (int k = 0; k < kClEpt / 4; ++k) {
+        const int e = c0 + (k * THREADS + tid) * 4;
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (e < c0 + chunk && e < V) v = __ldg(reinterpret_cast<const float4*>(logits + off + e));  // V % 4 == 0
+        x[4 * k + 0] = v.x, x[4 * k + 1] = v.y, x[4 * k + 2] = v.z, x[4 * k + 3] = v.w;
+    }
+    if (STOCH) {
+#pragma unroll
+        for (int k = 0; k < kClEpt / 4; ++k) {
+            const int e = c0 + (k * THREADS + tid) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (e < c0 + chunk && e < V) v = __ldg(reinterpret_cast<const float4*>(dprobs + off + e));
+            q[4 * k + 0] = v.x, q[4 * k + 1] = v.y, q[4 * k + 2] = v.z, q[4 * k + 3] = v.w;
+        }
+    }
+    auto elem = [&](int k) { return c0 + ((k >> 2) * THREADS + tid) * 4 + (k & 3); };
+
+    auto valid = [&](int k) { return elem(k) < V && elem(k) < c0 + chunk; };
+
+    // ---- round 1: maximum and its lowest index
+    float m = -INFINITY;
+    int mi = INT_MAX;
+#pragma unroll
+    for (int k = 0; k < kClEpt; ++k)
+        if (valid(k)) argmax_combine(m, mi, x[k], elem(k));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, mi, o);
+        argmax_combine(m, mi, om, oi);
+    }
+    if ((tid & 31) == 0) wm[tid >> 5] = m, wi[tid >> 5] = mi;
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < THREADS / 32; ++w) argmax_combine(m, mi, wm[w], wi[w]);
+        slot.m = (double)m, slot.idx = (double)mi;  // float and int32 are exact in a double
+    }
+    cl_gather(&slot.m, gathered, &slot.idx, gathered2);
+    float M = -INFINITY;
+    int idx = INT_MAX;
+    for (int r = 0; r < kCl; ++r) argmax_combine(M, idx, (float)gathered[r], (int)gathered2[r]);
+    if (!STOCH) {
+        if (rank == 0 && tid == 0) {
+            NodeSummary ns;
+            ns.S = 0.0, ns.Z = 0.0, ns.Q = 0.0, ns.M = M, ns.idx = idx;
+            out[(size_t)b * T + node] = ns;
+        }
+        cl_sync();  // nobody leaves while a peer may still read its slots
+        return;
+    }
+
+    // ---- round 2: e = exp((x - M)/tau), once per element, kept in registers; S = sum e
+    double e[kClEpt];
+    const double Md = (double)M;
+    double s = 0.0;
+#pragma unroll
+    for (int k = 0; k < kClEpt; ++k) {
+        e[k] = (valid(k) && M > -INFINITY) ? exp_nonpos(((double)x[k] - Md) * inv_tau, tab) : 0.0;
+        s += e[k];
+    }
+    s = block_sum(s, scratch);
+    if (tid == 0) slot.s = s;
+    cl_gather(&slot.s, gathered);
+    double S = 0.0;
+    for (int r = 0; r < kCl; ++r) S += gathered[r];
+    const double invS = S > 0.0 ? 1.0 / S : 0.0;
+
+    // ---- round 3: first-round residual mass and the draft mass without the first child's token
+    const int ft = first_tok;
+    double z = 0.0, qs = 0.0;
+#pragma unroll
+    for (int k = 0; k < kClEpt; ++k) {
+        const double qd = (double)q[k];
+        const double r = e[k] * invS - qd;
+        z += r > 0.0 ? r : 0.0;
+        qs += (elem(k) == ft) ? 0.0 : qd;
+    }
+    z = block_sum(z, scratch);
+    qs = block_sum(qs, scratch);
+    if (tid == 0) slot.z = z, slot.qs = qs;
+    cl_gather(&slot.z, gathered, &slot.qs, gathered2);
+    double Z = 0.0, Q = 0.0;
+    for (int r = 0; r < kCl; ++r) Z += gathered[r], Q += gathered2[r];
+    if (rank == 0 && tid == 0) {
+        NodeSummary ns;
+        ns.S = S, ns.Z = Z, ns.Q = Q, ns.M = M, ns.idx = idx;
+        out[(size_t)b * T + node] = ns;
+    }
+    cl_sync();  // nobody leaves while a peer may still read its slots
+}
+
+// ---- the walk, one cluster per sequence (greedy: one CTA, no cluster, no vocabulary pass)
+struct WalkClShared {
+    WalkShared w;
+    double tab[32];
+    double slots[2][2];  // two alternating sets of (sum a, sum b): set k is rewritten two cluster barriers later
+    double ga[kCl], gb[kCl];
+};
+
+template <bool STOCH>
+__global__ void __launch_bounds__(STOCH ? 1024 : 128, 1)
+accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
+                           const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                           const int32_t* __restrict__ n_nodes, const float* __restrict__ uniforms, int T, int V,
+                           int chunk, int max_depth, double inv_tau, const NodeSummary* __restrict__ nodes,
+                           int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
+                           int32_t* __restrict__ next_token, uint8_t* __restrict__ near_tie,
+                           int32_t* __restrict__ status) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    WalkClShared& cs = *reinterpret_cast<WalkClShared*>(smem_raw);
+    WalkShared& sh = cs.w;
+    const int b = blockIdx.y, tid = threadIdx.x;
+    const uint32_t rank = STOCH ? cl_rank() : 0u;
+    const bool writer = rank == 0;  // CTA 0 writes everything except the final token, which its finder writes
+    const int n = n_nodes ? n_nodes[b] : T;
+    int32_t* pth = path + (size_t)b * (max_depth + 1);
+
+    for (int i = tid; i < T; i += blockDim.x) {
+        sh.par[i] = parent[(size_t)b * T + i];
+        sh.tok[i] = tokens[(size_t)b * T + i];
+        sh.uni[i] = (STOCH && uniforms) ? uniforms[(size_t)b * T + i] : 0.f;
+        if (near_tie && writer) near_tie[(size_t)b * T + i] = 0;
+    }
+    if (tid < 32) cs.tab[tid] = kExp2Frac[tid];
+    __syncthreads();
+    int flags = build_ancestor_masks(sh.par, n, T, sh.anc, sh.depth, &sh.flag);
+    if (!flags) {
+        for (int i = tid; i < n; i += blockDim.x) {
+            if (sh.tok[i] < 0 || sh.tok[i] >= V) atomicOr(&sh.flag, S4C_SEQ_TOKEN_RANGE);
+            if (sh.depth[i] > max_depth) atomicOr(&sh.flag, S4C_SEQ_DEPTH);
+        }
+        __syncthreads();
+        flags = sh.flag;
+    }
+    if (tid == 0 && status && writer) status[b] = flags;
+    if (flags) {  // the same in every CTA of the cluster: they all leave here, before any cluster barrier
+        if (writer) {
+            for (int j = tid; j <= max_depth; j += blockDim.x) pth[j] = -1;
+            if (tid == 0) accept_len[b] = -1, next_token[b] = -1;
+        }
+        return;
+    }
+    for (int i = tid; i < n; i += blockDim.x) {
+        const NodeSummary ns = nodes[(size_t)b * T + i];
+        sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = ns.Z, sh.nQ[i] = ns.Q;
+    }
+    __syncthreads();
+    auto write_path = [&](int end) {
+        for (int j = 0; j <= max_depth; ++j) pth[j] = -1;
+        for (int t = end; t >= 0; t = sh.par[t]) pth[sh.depth[t]] = t;
+        accept_len[b] = sh.depth[end];
+    };
+
+    if (!STOCH) {
+        if (tid == 0) {
+            // ok[] as a bitmask; parent[i] < i so one ascending sweep suffices
+            uint32_t ok[S4C_MASK_WORDS] = {1u, 0, 0, 0};
+            int e = 0;
+            for (int i = 1; i < n; ++i) {
+                const int p = sh.par[i];
+                if (((ok[p >> 5] >> (p & 31)) & 1u) && sh.tok[i] == sh.nArg[p]) {
+                    ok[i >> 5] |= 1u << (i & 31);
+                    if (sh.depth[i] > sh.depth[e]) e = i;
+                }
+            }
+            write_path(e);
+            next_token[b] = sh.nArg[e];
+        }
+        return;
+    }
+
+    // ---- speculative-sampling walk: every thread of every CTA follows the same control flow on the same scalars;
+    //      only the vocabulary-wide sums are split, CTA `rank` owning the elements [c0, c1)
+    const int c0 = (int)rank * chunk, c1 = min(V, c0 + chunk);
+    int round = 0;  // cluster-wide reductions so far (selects the slot set)
+    // two cluster-wide sums in rank order; every thread of the cluster calls this and gets the same values
+    auto cluster_sum2 = [&](double a, double bsum, double& A, double& Bs) {
+        a = block_sum(a, sh.scratch);
+        bsum = block_sum(bsum, sh.scratch);
+        double* set = cs.slots[round & 1];
+        if (tid == 0) set[0] = a, set[1] = bsum;
+        cl_sync();
+        if (tid < kCl) cs.ga[tid] = cl_peer_f64(&set[0], tid), cs.gb[tid] = cl_peer_f64(&set[1], tid);
+        __syncthreads();
+        A = 0.0, Bs = 0.0;
+        for (int r = 0; r < kCl; ++r) A += cs.ga[r], Bs += cs.gb[r];
+        __syncthreads();  // ga/gb are free again
+        ++round;
+    };
+
+    int cur = 0;
+    for (int guard = 0; guard <= T; ++guard) {
+        const float* lrow = logits + ((size_t)b * T + cur) * V;
+        const float* qrow = dprobs + ((size_t)b * T + cur) * V;
+        const double M = (double)sh.nM[cur];
+        const double invS = sh.nS[cur] > 0.0 ? 1.0 / sh.nS[cur] : 0.0;
+        auto p0_of = [&](int v) { return exp_nonpos(((double)__ldg(lrow + v) - M) * inv_tau, cs.tab) * invS; };
+        int r = 0, accepted = -1;
+        for (int c = cur + 1; c < n; ++c) {
+            if (sh.par[c] != cur) continue;
+            const int x = sh.tok[c];
+            double px, qx;
+            chain_eval(p0_of(x), (double)__ldg(qrow + x), x, r, sh, px, qx);
+            double ratio;
+            if (qx > 0.0)
+                ratio = px / qx;
+            else
+                ratio = px > 0.0 ? (double)INFINITY : 0.0;
+            const double u = (double)sh.uni[c];
+            if (tid == 0 && writer && near_tie && fabs(ratio - u) < 1e-6) near_tie[(size_t)b * T + c] = 1;
+            if (u < (ratio < 1.0 ? ratio : 1.0)) {
+                accepted = c;
+                break;
+            }
+            // rejected: residual mass and the draft mass left once x is removed
+            double Z, s;
+            if (r == 0) {
+                Z = sh.nZ[cur], s = sh.nQ[cur];
+            } else {
+                double z = 0.0, qs = 0.0;
+                for (int v = c0 + tid; v < c1; v += blockDim.x) {
+                    double pv, qv;
+                    chain_eval(p0_of(v), (double)__ldg(qrow + v), v, r, sh, pv, qv);
+                    const double res = pv - qv;
+                    z += res > 0.0 ? res : 0.0;
+                    qs += (v == x) ? 0.0 : qv;
+                }
+                cluster_sum2(z, qs, Z, s);
+            }
+            __syncthreads();  // everyone has finished reading the chain before it grows
+            if (tid == 0) {
+                sh.cx[r] = x;
+                sh.cinvZ[r] = Z > 0.0 ? 1.0 / Z : 0.0;
+                sh.cinvs[r] = s > 0.0 ? 1.0 / s : 0.0;
+            }
+            __syncthreads();
+            ++r;
+            if (!(s > 0.0)) break;
+        }
+        if (accepted >= 0) {
+            cur = accepted;
+            __syncthreads();
+            continue;
+        }
+
+        // ---- final token: inverse CDF over the current p at `cur` (Eq. 12 at a fork; plain target at a leaf).
+        //      Each warp sums a contiguous span of its CTA's range; the CTA totals are exchanged; the CTA whose
+        //      range holds the crossing scans the one span that holds it.
+        const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+        const int seg = ((chunk + nwarps - 1) / nwarps + 31) / 32 * 32;  // contiguous span per warp
+        const int w0 = c0 + warp * seg, w1 = min(c1, w0 + seg);
+        double acc = 0.0;
+        int last = -1;
+        for (int v = w0 + lane; v < w1; v += 32) {
+            double pv, qv;
+            chain_eval(p0_of(v), (double)__ldg(qrow + v), v, r, sh, pv, qv);
+            acc += pv;
+            if (pv > 0.0) last = v;
+        }
+        acc = warp_sum(acc);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+        if (lane == 0) sh.wsum[warp] = acc, sh.wlast[warp] = last;
+        __syncthreads();
+        double* set = cs.slots[round & 1];
+        if (tid == 0) {
+            double tot = 0.0;
+            int lastpos = -1;
+            for (int w = 0; w < nwarps; ++w) tot += sh.wsum[w], lastpos = max(lastpos, sh.wlast[w]);
+            set[0] = tot, set[1] = (double)lastpos;
+        }
+        cl_sync();
+        if (tid < kCl) cs.ga[tid] = cl_peer_f64(&set[0], tid), cs.gb[tid] = cl_peer_f64(&set[1], tid);
+        __syncthreads();
+        double total = 0.0;
+        int lastpos = 0;
+        for (int rr = 0; rr < kCl; ++rr) total += cs.ga[rr], lastpos = max(lastpos, (int)cs.gb[rr]);
+        const double target = (double)sh.uni[0] * total;
+        double before = 0.0;  // mass of the ranks before the one that holds the crossing
+        int rstar = -1;
+        for (int rr = 0; rr < kCl; ++rr) {
+            if (before + cs.ga[rr] > target) {
+                rstar = rr;
+                break;
+            }
+            before += cs.ga[rr];
+        }
+        if (rstar < 0) {  // the running sum never exceeds the target (u * total rounds up to the total): last token with mass
+            if (writer && tid == 0) {
+                next_token[b] = lastpos;
+                write_path(cur);
+            }
+        } else if ((int)rank == rstar && warp == 0) {
+            double run = before;
+            int wstar = 0;
+            for (; wstar < nwarps - 1; ++wstar) {
+                if (run + sh.wsum[wstar] > target) break;
+                run += sh.wsum[wstar];
+            }
+            int pick = -1;
+            for (int base = c0 + wstar * seg; base < c1 && pick < 0; base += 32) {
+                const int v = base + lane;
+                double pv = 0.0, qv;
+                if (v < c1) chain_eval(p0_of(v), (double)__ldg(qrow + v), v, r, sh, pv, qv);
+                double scan = pv;  // inclusive prefix within the group of 32
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double t = __shfl_up_sync(0xffffffffu, scan, o);
+                    if (lane >= o) scan += t;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, v < c1 && run + scan > target);
+                if (hit) pick = base + __ffs(hit) - 1;
+                run += __shfl_sync(0xffffffffu, scan, 31);
+            }
+            if (lane == 0) {
+                // a crossing lost to the different summation order of the scan: this CTA's last token with mass
+                next_token[b] = pick >= 0 ? pick : (int)cs.gb[rstar];
+                write_path(cur);
+            }
+        }
+        cl_sync();  // nobody leaves while a peer may still read its slots
+        return;
+    }
+    cl_sync();
+}
+
 }  // namespace s4c
 
 extern "C" size_t s4c_tree_accept_workspace_bytes(int B, int T, int V) {
@@ -495,6 +944,57 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
     dim3 grid(splits, T, B);
 
     const size_t walk_smem = sizeof(WalkShared);  // ~11 KB, below the 48 KB default limit
+
+    if (vec && V <= kClMaxV) {
+        // ---- cluster path: one 8-CTA cluster per row, then one cluster (greedy: one CTA) per sequence
+        const int chunk = (int)round_up((size_t)ceil_div(V, kCl), 4);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kCl, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kCl, T, B);
+        cfg.stream = stream;
+        cfg.attrs = attr, cfg.numAttrs = 1;
+        cudaError_t err;
+#define S4C_LAUNCH_STATS(THREADS)                                                                                      \
+    do {                                                                                                               \
+        cfg.blockDim = dim3(THREADS, 1, 1);                                                                            \
+        err = stoch ? cudaLaunchKernelEx(&cfg, accept_stats_cluster_kernel<THREADS, true>, target_logits, draft_probs, \
+                                         tokens, parent, n_nodes, T, V, chunk, inv_tau, ws.summary)                    \
+                    : cudaLaunchKernelEx(&cfg, accept_stats_cluster_kernel<THREADS, false>, target_logits,            \
+                                         draft_probs, tokens, parent, n_nodes, T, V, chunk, inv_tau, ws.summary);     \
+    } while (0)
+        if (chunk <= 256 * kClEpt)
+            S4C_LAUNCH_STATS(256);
+        else if (chunk <= 512 * kClEpt)
+            S4C_LAUNCH_STATS(512);
+        else
+            S4C_LAUNCH_STATS(1024);
+#undef S4C_LAUNCH_STATS
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            return S4C_ERR_CUDA;
+        }
+        const NodeSummary* summary = ws.summary;
+        if (stoch) {
+            cfg.gridDim = dim3(kCl, B, 1);
+            cfg.blockDim = dim3(1024, 1, 1);
+            cfg.dynamicSmemBytes = sizeof(WalkClShared);
+            err = cudaLaunchKernelEx(&cfg, accept_walk_cluster_kernel<true>, target_logits, draft_probs, tokens, parent,
+                                     n_nodes, uniforms, T, V, chunk, max_depth, inv_tau, summary, accept_len, path,
+                                     next_token, near_tie, status);
+            if (err != cudaSuccess) {
+                cudaGetLastError();
+                return S4C_ERR_CUDA;
+            }
+        } else {
+            accept_walk_cluster_kernel<false><<<dim3(1, B), 128, sizeof(WalkClShared), stream>>>(
+                target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, max_depth, inv_tau, summary,
+                accept_len, path, next_token, near_tie, status);
+            S4C_RETURN_IF_CUDA_ERROR();
+        }
+        return S4C_OK;
+    }
 
     if (stoch) {
         if (vec)

@@ -37,7 +37,7 @@ def _synthetic(B, T, V, seed, sigma=2.0, noise=1.0, tau=1.0, mode="sampled", max
     return cfg, parent, x
 
 
-@pytest.mark.parametrize("V", [1, 3, 257, 4096, 4099, 33333])
+@pytest.mark.parametrize("V", [1, 3, 4, 8, 36, 257, 4096, 4099, 33333, 33336])
 def test_odd_vocabulary_sizes(V):
     T = min(9, max(2, V))
     cfg, parent, x = _synthetic(8, T, V, seed=V % 97, tau=0.9)
