@@ -5,10 +5,11 @@
 // so K/V stream from HBM once per KV head (NM = 2 covers G*T up to 256 rows, the GQA case, with one pass).
 // Warp-specialised:
 //   warp 0        TMA producer: Q once, then K and V tiles of 64 slots into 128B-swizzled shared-memory rings
-//   warps 1, 2    MMA issuers, one thread each: warp 1 issues S = Q K^T (tcgen05.mma kind::f16, M128 N64 K16 x
-//                 d/16) into one of two TMEM score buffers per row tile and owns the TMEM allocation; warp 2
-//                 issues O += P V (M128 N=d K16 x 4) into a TMEM accumulator per row tile
-//   warps 3..     one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
+//   next 2 x NM   MMA issuers, one warp (one thread) per product and row tile: the QK issuers send S = Q K^T
+//                 (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of two TMEM score buffers of their row
+//                 tile, the PV issuers O += P V (M128 N=d K16 x 4) into its TMEM accumulator; warp 1 owns the
+//                 TMEM allocation
+//   then          one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
 //                 tree / tail masking from the row's ancestor bitmask (built from parent[] by the thread
 //                 itself), online softmax in fp32 (base 2; the running offset only moves when the maximum
 //                 grew by more than 2^8, so O in TMEM is rarely rescaled), P rounded to bf16 into swizzled
@@ -45,7 +46,8 @@ struct TcCfg {
     static constexpr int kStages = D == 128 ? (NM == 1 ? 6 : 5) : 8;
     static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes;
     static constexpr int kNumBars = 1 + 4 * kStages + 7 * NM;
-    static constexpr int kThreads = 96 + 128 * NM;   // TMA warp, two MMA issuer warps, four softmax warps per row tile
+    static constexpr int kRoleWarps = 1 + 2 * NM;    // TMA warp, then a QK issuer and a PV issuer warp per row tile
+    static constexpr int kThreads = 32 * kRoleWarps + 128 * NM;  // ... and four softmax warps per row tile
     static constexpr int kPartStride = D + 4;        // floats per parked row (padding spreads the banks)
     static constexpr int kPartBytes = NM * kBM * kPartStride * 4 + NM * kBM * 8;
     static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
@@ -332,7 +334,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // ---- prologue that touches no global memory: barriers (one per lane of warp 0), TMEM, descriptor prefetch
     if (warp == 0) {
         for (int i = lane; i < Cfg::kNumBars; i += 32) {
-            uint32_t count = 1;  // every barrier but P_FULL, which takes one arrival per active softmax warp
+            uint32_t count = 1;  // but: P_FULL takes one arrival per active softmax warp, the EMPTY barriers of
+                                 // the ring one commit per active row tile (each has issuer threads of its own)
+            if ((i >= K_EMPTY && i < K_EMPTY + S) || (i >= V_EMPTY && i < V_EMPTY + S)) count = (uint32_t)nm_act;
             if (i >= PER_TILE) {
                 const int t = (i - PER_TILE) / 7, k = (i - PER_TILE) % 7;
                 const uint32_t active = (uint32_t)active_threads(t) / 32u;
@@ -406,52 +410,51 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (lane == 0)
                 for (int j = S; j < nt; ++j) load_tile(j);
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer 1: S = Q K^T =================
-        if (lane == 0 && nt > 0) {
+    } else if (warp <= NM) {
+        // ================= QK issuer of row tile t: S = Q K^T =================
+        // (one issuing thread per product and row tile: a single thread spends more time issuing a tile's
+        //  instructions and polling its barriers than the tile takes to arrive)
+        const int t = warp - 1;
+        if (lane == 0 && nt > 0 && t < nm_act) {
             constexpr uint32_t idesc_qk = instr_desc_bf16(kBM, kBN, false);
+            uint64_t a_desc[D / 16];  // the Q operand never moves: one descriptor per K step, made once
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk)  // 64-element halves along d, 32 bytes per K step inside a half
+                a_desc[kk] = smem_desc_sw128(sQ + t * Cfg::kQBytes + (kk >> 2) * (kBM * 128) + (kk & 3) * 32, 16, 1024);
             mbar_wait(BAR(Q_FULL), 0, dead);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
                 mbar_wait(BAR(K_FULL + s), it & 1, dead);
-                const uint32_t k_base = sK + s * Cfg::kTileBytes;
-                for (int t = 0; t < nm_act; ++t) {
-                    mbar_wait(S_EMPTY(t, j & 1), ((j >> 1) & 1) ^ 1, dead);
-                    tc_fence_after();
+                const uint64_t k_desc = smem_desc_sw128(sK + s * Cfg::kTileBytes, 16, 1024);
+                mbar_wait(S_EMPTY(t, j & 1), ((j >> 1) & 1) ^ 1, dead);
+                tc_fence_after();
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const int h = kk >> 2, ko = (kk & 3) * 32;  // 64-element halves along d, 32 bytes per K step
-                        const uint64_t ad = smem_desc_sw128(sQ + t * Cfg::kQBytes + h * (kBM * 128) + ko, 16, 1024);
-                        const uint64_t bd = smem_desc_sw128(k_base + h * (kBN * 128) + ko, 16, 1024);
-                        tc_mma_bf16(TM_S(t, j & 1), ad, bd, idesc_qk, kk > 0 ? 1u : 0u);
-                    }
-                    tc_commit(S_FULL(t, j & 1));
-                }
+                for (int kk = 0; kk < D / 16; ++kk)  // the start-address field counts 16-byte units
+                    tc_mma_bf16(TM_S(t, j & 1), a_desc[kk], k_desc + (uint64_t)(((kk >> 2) * (kBN * 128) + (kk & 3) * 32) >> 4),
+                                idesc_qk, kk > 0 ? 1u : 0u);
+                tc_commit(S_FULL(t, j & 1));
                 tc_commit(BAR(K_EMPTY + s));
             }
         }
-    } else if (warp == 2) {
-        // ================= MMA issuer 2: O += P V (its own thread, so that neither product waits for the other's
-        //                   barriers: one issuing thread spends more time per tile than the tile takes to arrive) ====
-        if (lane == 0 && nt > 0) {
+    } else if (warp <= 2 * NM) {
+        // ================= PV issuer of row tile t: O += P V =================
+        const int t = warp - 1 - NM;
+        if (lane == 0 && nt > 0 && t < nm_act) {
             constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
                 mbar_wait(BAR(V_FULL + s), it & 1, dead);
-                const uint32_t v_base = sV + s * Cfg::kTileBytes;
-                for (int t = 0; t < nm_act; ++t) {
-                    mbar_wait(P_FULL(t, j & 1), (j >> 1) & 1, dead);
-                    tc_fence_after();
+                // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
+                const uint64_t v_desc = smem_desc_sw128(sV + s * Cfg::kTileBytes, kBN * 128, 1024);
+                mbar_wait(P_FULL(t, j & 1), (j >> 1) & 1, dead);
+                tc_fence_after();
 #pragma unroll
-                    for (int kk = 0; kk < kBN / 16; ++kk) {
-                        // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
-                        // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
-                        const uint64_t bd = smem_desc_sw128(v_base + kk * 2048, kBN * 128, 1024);
-                        tc_mma_bf16_ts(TM_O(t), TM_S(t, j & 1) + kk * 8, bd, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
-                    }
-                    tc_commit(PV_DONE(t));
-                    tc_commit(S_EMPTY(t, j & 1));  // the score buffer (and the P inside it) may be overwritten
-                }
+                for (int kk = 0; kk < kBN / 16; ++kk)
+                    // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
+                    tc_mma_bf16_ts(TM_O(t), TM_S(t, j & 1) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv,
+                                   (j > 0 || kk > 0) ? 1u : 0u);
+                tc_commit(PV_DONE(t));
+                tc_commit(S_EMPTY(t, j & 1));  // the score buffer (and the P inside it) may be overwritten
                 tc_commit(BAR(V_EMPTY + s));
             }
         }
@@ -460,7 +463,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // tree check first: softmax thread i looks at node i; a malformed tree still runs the pipeline (with empty
         // masks, so that no role waits for another) and only its outputs are withheld
         if (!flags) {
-            const int i = threadIdx.x - 96;
+            const int i = threadIdx.x - 32 * Cfg::kRoleWarps;
             if (i < T) {
                 const int p = prm.parent[(size_t)b * T + i];
                 par_s[i] = p;
@@ -469,9 +472,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
         named_bar_sync(1, NM * 128);
         flags |= *bad_s;
-        if (split == 0 && blockIdx.y == 0 && threadIdx.x == 96 && prm.status) prm.status[b] = flags;
+        if (split == 0 && blockIdx.y == 0 && threadIdx.x == 32 * Cfg::kRoleWarps && prm.status) prm.status[b] = flags;
         const bool run = flags == 0;
-        const int t = (warp - 3) >> 2;  // row tile of this warp group
+        const int t = (warp - Cfg::kRoleWarps) >> 2;  // row tile of this warp group
         const int wq = warp & 3;        // TMEM lane quadrant this warp may access
         const int row = wq * 32 + lane;
         const int copy = row / RB, lr = row % RB;  // which copy of the rows, and the row within it
@@ -561,15 +564,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         tmem_wait_st();
                     }
                 }
-                if (t == 0 && kv0 + kBN > Ltot) {
+                if (kv0 + kBN > Ltot) {
                     // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
-                    // but 0 * NaN would poison O, so those V rows are cleared before the PV products read them (the
-                    // MMA thread sees P_FULL of row tile 0 before it issues any PV of this tile)
+                    // but 0 * NaN would poison O, so those V rows are cleared before the PV product reads them.  Every
+                    // row tile's group clears them (the same zeros) before it releases its own P: each PV issuer
+                    // only waits for its own group.
                     const int s = j % S, it = j / S;
                     mbar_wait_warp(BAR(V_FULL + s), it & 1, dead);
                     const int first = Ltot - kv0;  // 1..63
                     unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
-                    const int stride = active_threads(0);
+                    const int stride = active_threads(t);
                     for (int idx = row; idx < (kBN - first) * 8 * NH; idx += stride) {
                         const int h = idx / ((kBN - first) * 8), rem = idx % ((kBN - first) * 8);
                         const int r = first + rem / 8, ch = rem % 8;
