@@ -109,6 +109,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -381,12 +387,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
             mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead);
             mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
-            for (int h = 0; h < NH; ++h)
-                tma_load_2d(sK + s * Cfg::kTileBytes + h * (kBN * 128), &map_k, BAR(K_FULL + s), h * 64, row);
+            if (NH == 2) {  // one request per tile: the map's third dimension is the 64-column half
+                tma_load_3d(sK + s * Cfg::kTileBytes, &map_k, BAR(K_FULL + s), 0, row, 0);
+            } else {
+                tma_load_2d(sK + s * Cfg::kTileBytes, &map_k, BAR(K_FULL + s), 0, row);
+            }
             mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead);
             mbar_expect_tx(BAR(V_FULL + s), Cfg::kTileBytes);
-            for (int h = 0; h < NH; ++h)
-                tma_load_2d(sV + s * Cfg::kTileBytes + h * (kBN * 128), &map_v, BAR(V_FULL + s), h * 64, row);
+            if (NH == 2) {
+                tma_load_3d(sV + s * Cfg::kTileBytes, &map_v, BAR(V_FULL + s), 0, row, 0);
+            } else {
+                tma_load_2d(sV + s * Cfg::kTileBytes, &map_v, BAR(V_FULL + s), 0, row);
+            }
         };
         if (nt > 0) {
             // first pass of the ring, every ring slot still free: lane j requests tile j, the last lane requests Q,
@@ -782,6 +794,21 @@ static bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int d, in
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same [rows, 128] matrix seen as [2 halves][rows][64 columns]: one box of 64 columns x box_rows x 2 halves lands in
+// shared memory half by half, each half a stack of 128-byte rows -- the layout the K-major / MN-major operand
+// descriptors of the kernel expect -- so a whole K or V tile takes one request.
+static bool make_map_halves(CUtensorMap* map, const void* ptr, uint64_t rows, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, 2};
+    const cuuint64_t strides[2] = {256, 128};  // bytes: next row, next half
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool tc_supported(int T, int Hq, int Hkv, int d, s4c_dtype dt) { return dt == S4C_BF16 && (d == 128 || d == 64); }
 
 static int tc_m_tiles(int T, int Hq, int Hkv) { return ceil_div((Hq / Hkv) * T, kBM); }
@@ -837,8 +864,8 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
     }
     CUtensorMap mq, mk, mv;
     if (!make_map(&mq, q, (uint64_t)B * prm.Hq * prm.T, D, prm.q_box_rows) ||
-        !make_map(&mk, k, (uint64_t)B * prm.Hkv * prm.C, D, kBN) ||
-        !make_map(&mv, v, (uint64_t)B * prm.Hkv * prm.C, D, kBN))
+        !(D == 128 ? make_map_halves(&mk, k, (uint64_t)B * prm.Hkv * prm.C, kBN) : make_map(&mk, k, (uint64_t)B * prm.Hkv * prm.C, D, kBN)) ||
+        !(D == 128 ? make_map_halves(&mv, v, (uint64_t)B * prm.Hkv * prm.C, kBN) : make_map(&mv, v, (uint64_t)B * prm.Hkv * prm.C, D, kBN)))
         return S4C_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(prm.splits, prm.m_groups * prm.Hkv, B);
