@@ -25,7 +25,6 @@ namespace s4c {
 constexpr int kRowThreads = 256;
 constexpr int kElemsPerThread = 16;
 constexpr int kSegElems = kRowThreads * kElemsPerThread;  // 4096 logits per CTA
-constexpr int kWalkThreads = 1024;
 
 struct RowPartial {  // one vocab segment of one row
     double S;        // sum exp((x - M)/tau) over the segment (sampling only)
@@ -102,14 +101,74 @@ __device__ __forceinline__ double block_sum(double v, double* scratch) {
     return scratch[32];
 }
 
+// exp(t) for t <= 0 in float64, about 1 ulp: t = (32 k + j) ln2/32 + r, exp(t) = 2^k * 2^(j/32) * e^r with |r| <=
+// ln2/64 and a degree-6 polynomial for e^r (remainder below 4e-18).  About a third of the float64 instructions of
+// the library exp, which matters because this path is otherwise bound by the float64 pipe, not by HBM.
+__device__ const double kExp2Frac[32] = {
+    0x1.0000000000000p+0, 0x1.059b0d3158574p+0, 0x1.0b5586cf9890fp+0, 0x1.11301d0125b51p+0,
+    0x1.172b83c7d517bp+0, 0x1.1d4873168b9aap+0, 0x1.2387a6e756238p+0, 0x1.29e9df51fdee1p+0,
+    0x1.306fe0a31b715p+0, 0x1.371a7373aa9cbp+0, 0x1.3dea64c123422p+0, 0x1.44e086061892dp+0,
+    0x1.4bfdad5362a27p+0, 0x1.5342b569d4f82p+0, 0x1.5ab07dd485429p+0, 0x1.6247eb03a5585p+0,
+    0x1.6a09e667f3bcdp+0, 0x1.71f75e8ec5f74p+0, 0x1.7a11473eb0187p+0, 0x1.82589994cce13p+0,
+    0x1.8ace5422aa0dbp+0, 0x1.93737b0cdc5e5p+0, 0x1.9c49182a3f090p+0, 0x1.a5503b23e255dp+0,
+    0x1.ae89f995ad3adp+0, 0x1.b7f76f2fb5e47p+0, 0x1.c199bdd85529cp+0, 0x1.cb720dcef9069p+0,
+    0x1.d5818dcfba487p+0, 0x1.dfc97337b9b5fp+0, 0x1.ea4afa2a490dap+0, 0x1.f50765b6e4540p+0};
+
+__device__ __forceinline__ double exp_nonpos(double t, const double* tab /* shared copy of kExp2Frac */) {
+    if (!(t > -700.0)) return exp(t);  // result near or below the normal range (also -inf, NaN): library path
+    // k = round(t * 32/ln2) by adding 1.5 * 2^52: the integer sits in the low word of the sum (no conversion or
+    // rounding instruction: those run at a quarter of the float64 FMA rate)
+    const double z = fma(t, 0x1.71547652b82fep+5, 6755399441055744.0);
+    const int k = __double2loint(z);
+    const double kd = z - 6755399441055744.0;
+    double r = fma(-kd, 0x1.62e42fefa39efp-6, t);  // ln2/32, high and low part
+    r = fma(-kd, 0x1.abc9e3b39803fp-61, r);
+    double pl = fma(r, 1.0 / 720.0, 1.0 / 120.0);
+    pl = fma(pl, r, 1.0 / 24.0);
+    pl = fma(pl, r, 1.0 / 6.0);
+    pl = fma(pl, r, 0.5);
+    pl = fma(pl, r, 1.0);
+    pl = pl * r;  // e^r - 1
+    const double tj = tab[k & 31];
+    const double y = fma(tj, pl, tj);  // in [1, 2.05)
+    return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));  // * 2^(k >> 5), exponent stays normal
+}
+
+// exp_nonpos without the range test, for -700 < t <= 0.  The statistics kernels raise every logit to at least
+// M - 690 tau first (one float max): a term that small is below 1e-299 of the row sum either way, so neither the sum
+// nor the residual mass can tell the difference, and the inner loop loses a compare and a branch per element.
+// `tab32` is a copy of the table with every entry repeated once per lane (entry j of lane l at [j * 32 + l]): the 32
+// lanes of a warp then always read 32 different banks pairs, whatever entries they need.
+__device__ __forceinline__ double exp_fast(double t, const double* tab32) {
+    const double z = fma(t, 0x1.71547652b82fep+5, 6755399441055744.0);
+    const int k = __double2loint(z);
+    const double kd = z - 6755399441055744.0;
+    double r = fma(-kd, 0x1.62e42fefa39efp-6, t);
+    r = fma(-kd, 0x1.abc9e3b39803fp-61, r);
+    double pl = fma(r, 1.0 / 720.0, 1.0 / 120.0);
+    pl = fma(pl, r, 1.0 / 24.0);
+    pl = fma(pl, r, 1.0 / 6.0);
+    pl = fma(pl, r, 0.5);
+    pl = fma(pl, r, 1.0);
+    pl = pl * r;
+    const double tj = tab32[((k & 31) << 5) + (threadIdx.x & 31)];
+    const double y = fma(tj, pl, tj);
+    return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));
+}
+constexpr float kExpFloorSpan = 690.f;  // in units of tau
+__device__ __forceinline__ void fill_exp_table(double* tab32) {  // every thread of the CTA; the caller synchronises
+    for (int i = threadIdx.x; i < 1024; i += blockDim.x) tab32[i] = kExp2Frac[i >> 5];
+}
+
 // ----------------------------------------------------------------------------- kernel 1
-template <bool VEC>
+template <bool VEC, bool ZERO_FILL = false>
 __device__ __forceinline__ void load_segment(const float* __restrict__ row, int s0, int V, float (&x)[kElemsPerThread]) {
+    const float fill = ZERO_FILL ? 0.f : -INFINITY;
     if (VEC) {
 #pragma unroll
         for (int k = 0; k < kElemsPerThread / 4; ++k) {
             const int e = s0 + (k * kRowThreads + threadIdx.x) * 4;
-            float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            float4 v = make_float4(fill, fill, fill, fill);
             if (e < V) v = __ldg(reinterpret_cast<const float4*>(row + e));  // V % 4 == 0 here
             x[4 * k + 0] = v.x, x[4 * k + 1] = v.y, x[4 * k + 2] = v.z, x[4 * k + 3] = v.w;
         }
@@ -117,7 +176,7 @@ __device__ __forceinline__ void load_segment(const float* __restrict__ row, int 
 #pragma unroll
         for (int k = 0; k < kElemsPerThread; ++k) {
             const int e = s0 + k * kRowThreads + threadIdx.x;
-            x[k] = e < V ? __ldg(row + e) : -INFINITY;
+            x[k] = e < V ? __ldg(row + e) : fill;
         }
     }
 }
@@ -129,53 +188,61 @@ __device__ __forceinline__ int elem_index(int s0, int k) {
 template <bool STOCH, bool VEC>
 __global__ void __launch_bounds__(kRowThreads)
 accept_rowstats_kernel(const float* __restrict__ logits, const int32_t* __restrict__ n_nodes, int T, int V,
-                       double inv_tau, RowPartial* __restrict__ out) {
+                       double inv_tau, float floor_span, RowPartial* __restrict__ out) {
     const int split = blockIdx.x, node = blockIdx.y, b = blockIdx.z;
     if (n_nodes && node >= n_nodes[b]) return;
     const float* row = logits + ((size_t)b * T + node) * V;
     const int s0 = split * kSegElems;
     float x[kElemsPerThread];
-    load_segment<VEC>(row, s0, V, x);
+    load_segment<VEC>(row, s0, V, x);  // -inf beyond the row
 
-    float m = -INFINITY;
-    int mi = INT_MAX;
-#pragma unroll
-    for (int k = 0; k < kElemsPerThread; ++k) {
-        const int e = elem_index<VEC>(s0, k);
-        if (e < V) argmax_combine(m, mi, x[k], e);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, mi, o);
-        argmax_combine(m, mi, om, oi);
-    }
     __shared__ float sm[kRowThreads / 32];
-    __shared__ int si[kRowThreads / 32];
+    __shared__ int idx_s;
     __shared__ double scratch[33];
+    __shared__ double tab[STOCH ? 1024 : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) sm[warp] = m, si[warp] = mi;
-    __syncthreads();
-    m = sm[0], mi = si[0];
+    if (STOCH) fill_exp_table(tab);
+    if (threadIdx.x == 32) idx_s = INT_MAX;
+
+    // maximum first (one instruction per element); its lowest index is then looked up by the few threads that hold it
+    float mt = x[0];
 #pragma unroll
-    for (int w = 1; w < kRowThreads / 32; ++w) argmax_combine(m, mi, sm[w], si[w]);
+    for (int k = 1; k < kElemsPerThread; ++k) mt = fmaxf(mt, x[k]);
+    float m = mt;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) sm[warp] = m;
+    __syncthreads();
+    m = sm[0];
+#pragma unroll
+    for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, sm[w]);
+    if (mt == m) {
+#pragma unroll
+        for (int k = 0; k < kElemsPerThread; ++k) {  // a thread's element indices ascend with k
+            const int e = elem_index<VEC>(s0, k);
+            if (x[k] == m && e < V) {
+                atomicMin(&idx_s, e);
+                break;
+            }
+        }
+    }
 
     double S = 0.0;
     if (STOCH) {
         double s = 0.0;
         if (m > -INFINITY) {
-            const double md = (double)m;
+            const float x_floor = m - floor_span;
+            const double c = -(double)m * inv_tau;
 #pragma unroll
-            for (int k = 0; k < kElemsPerThread; ++k) {
-                const int e = elem_index<VEC>(s0, k);
-                if (e < V) s += exp(((double)x[k] - md) * inv_tau);
-            }
+            for (int k = 0; k < kElemsPerThread; ++k) s += exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab);
         }
         S = block_sum(s, scratch);
+    } else {
+        __syncthreads();  // idx_s
     }
     if (threadIdx.x == 0) {
         RowPartial r;
-        r.S = S, r.M = m, r.idx = mi;
+        r.S = S, r.M = m, r.idx = idx_s;
         out[((size_t)b * T + node) * gridDim.x + split] = r;
     }
 }
@@ -197,7 +264,7 @@ template <bool VEC>
 __global__ void __launch_bounds__(kRowThreads)
 accept_residual_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
                        const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
-                       const int32_t* __restrict__ n_nodes, int T, int V, double inv_tau,
+                       const int32_t* __restrict__ n_nodes, int T, int V, double inv_tau, float floor_span,
                        const RowPartial* __restrict__ rowp, ResPartial* __restrict__ resp,
                        NodeStats* __restrict__ nodes) {
     const int split = blockIdx.x, node = blockIdx.y, b = blockIdx.z, splits = gridDim.x;
@@ -206,9 +273,30 @@ accept_residual_kernel(const float* __restrict__ logits, const float* __restrict
     __shared__ NodeStats ns;
     __shared__ int first_tok;
     __shared__ double scratch[33];
-    if (threadIdx.x == 0) {
-        ns = merge_row(rowp + ((size_t)b * T + node) * splits, splits, inv_tau, true);
-        if (split == 0) nodes[(size_t)b * T + node] = ns;
+    __shared__ double tab[1024];
+    fill_exp_table(tab);
+    if (threadIdx.x < 32) {
+        // the row's statistics from its segments, by one warp: lane s (and s + 32, ...) takes segment s; the maximum
+        // and the sum then go through fixed-order butterflies (the same on every run and in every CTA of the row)
+        const RowPartial* part = rowp + ((size_t)b * T + node) * splits;
+        float M = -INFINITY;
+        int idx = INT_MAX;
+        for (int s = threadIdx.x; s < splits; s += 32) argmax_combine(M, idx, part[s].M, part[s].idx);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, M, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+            argmax_combine(M, idx, om, oi);
+        }
+        double S = 0.0;
+        if (M > -INFINITY)
+            for (int s = threadIdx.x; s < splits; s += 32)
+                if (part[s].M > -INFINITY) S += part[s].S * exp(((double)part[s].M - (double)M) * inv_tau);
+        S = warp_sum(S);
+        if (threadIdx.x == 0) {
+            ns.S = S, ns.M = M, ns.idx = idx;
+            if (split == 0) nodes[(size_t)b * T + node] = ns;
+        }
     }
     if (threadIdx.x == 32) {  // token of the first child in index order (the first one ever rejected here)
         int ft = -1;
@@ -219,26 +307,32 @@ accept_residual_kernel(const float* __restrict__ logits, const float* __restrict
             }
         first_tok = ft;
     }
-    __syncthreads();
-    const double M = (double)ns.M, invS = ns.S > 0.0 ? 1.0 / ns.S : 0.0;
-    const int ft = first_tok;
     const size_t off = ((size_t)b * T + node) * V;
     const int s0 = split * kSegElems;
-    float x[kElemsPerThread], q[kElemsPerThread];
+    float x[kElemsPerThread], q[kElemsPerThread];  // requested before the barrier: in flight while thread 0 merges
     load_segment<VEC>(logits + off, s0, V, x);
-    load_segment<VEC>(dprobs + off, s0, V, q);
+    load_segment<VEC, true>(dprobs + off, s0, V, q);  // 0 beyond the row
+    __syncthreads();
+    const double invS = ns.S > 0.0 ? 1.0 / ns.S : 0.0;
+    const int ft = first_tok;
     double z = 0.0, qs = 0.0;
+    if (ns.M > -INFINITY) {
+        const float x_floor = ns.M - floor_span;
+        const double c = -(double)ns.M * inv_tau;
 #pragma unroll
-    for (int k = 0; k < kElemsPerThread; ++k) {
-        const int e = elem_index<VEC>(s0, k);
-        if (e < V) {
-            const double p = exp(((double)x[k] - M) * inv_tau) * invS;
+        for (int k = 0; k < kElemsPerThread; ++k) {
+            const double p = exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab) * invS;
             const double qd = (double)q[k];
             const double r = p - qd;
-            z += r > 0.0 ? r : 0.0;
-            qs += (e == ft) ? 0.0 : qd;
+            if (r > 0.0) z += r;
+            qs += qd;
         }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kElemsPerThread; ++k) qs += (double)q[k];
     }
+    // the first child's token does not count towards the draft mass that is left: its owner takes it out again
+    if (threadIdx.x == 0 && ft >= s0 && ft < s0 + kSegElems && ft < V) qs -= (double)__ldg(dprobs + off + ft);
     z = block_sum(z, scratch);
     qs = block_sum(qs, scratch);
     if (threadIdx.x == 0) {
@@ -265,8 +359,8 @@ struct WalkShared {
     double cinvZ[S4C_MAX_T];  // 1/Z_j, or 0 when Z_j == 0 (p kept)
     double cinvs[S4C_MAX_T];  // 1/s_j
     double scratch[33];
-    double wsum[kWalkThreads / 32];
-    int wlast[kWalkThreads / 32];
+    double wsum[32];  // per warp of a 1024-thread CTA
+    int wlast[32];
     int flag;
     int result_tok;
 };
@@ -285,196 +379,6 @@ __device__ __forceinline__ void chain_eval(double p0, double q0, int v, int r, c
     }
 }
 
-template <bool STOCH>
-__global__ void __launch_bounds__(kWalkThreads)
-accept_walk_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
-                   const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
-                   const int32_t* __restrict__ n_nodes, const float* __restrict__ uniforms, int T, int V,
-                   int max_depth, double inv_tau, int splits, const RowPartial* __restrict__ rowp,
-                   const ResPartial* __restrict__ resp, const NodeStats* __restrict__ nodes,
-                   int32_t* __restrict__ accept_len, int32_t* __restrict__ path, int32_t* __restrict__ next_token,
-                   uint8_t* __restrict__ near_tie, int32_t* __restrict__ status) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    WalkShared& sh = *reinterpret_cast<WalkShared*>(smem_raw);
-    const int b = blockIdx.x, tid = threadIdx.x;
-    const int n = n_nodes ? n_nodes[b] : T;
-    int32_t* pth = path + (size_t)b * (max_depth + 1);
-
-    for (int i = tid; i < T; i += blockDim.x) {
-        sh.par[i] = parent[(size_t)b * T + i];
-        sh.tok[i] = tokens[(size_t)b * T + i];
-        sh.uni[i] = (STOCH && uniforms) ? uniforms[(size_t)b * T + i] : 0.f;
-        if (near_tie) near_tie[(size_t)b * T + i] = 0;
-    }
-    __syncthreads();
-    int flags = build_ancestor_masks(sh.par, n, T, sh.anc, sh.depth, &sh.flag);
-    if (!flags) {
-        for (int i = tid; i < n; i += blockDim.x) {
-            if (sh.tok[i] < 0 || sh.tok[i] >= V) atomicOr(&sh.flag, S4C_SEQ_TOKEN_RANGE);
-            if (sh.depth[i] > max_depth) atomicOr(&sh.flag, S4C_SEQ_DEPTH);
-        }
-        __syncthreads();
-        flags = sh.flag;
-    }
-    if (tid == 0 && status) status[b] = flags;
-    if (flags) {
-        for (int j = tid; j <= max_depth; j += blockDim.x) pth[j] = -1;
-        if (tid == 0) accept_len[b] = -1, next_token[b] = -1;
-        return;
-    }
-
-    // per-node statistics
-    for (int i = tid; i < n; i += blockDim.x) {
-        if (STOCH) {
-            const NodeStats ns = nodes[(size_t)b * T + i];
-            double z = 0.0, q = 0.0;
-            const ResPartial* rp = resp + ((size_t)b * T + i) * splits;
-            for (int s = 0; s < splits; ++s) z += rp[s].Z, q += rp[s].Q;
-            sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = z, sh.nQ[i] = q;
-        } else {
-            const NodeStats ns = merge_row(rowp + ((size_t)b * T + i) * splits, splits, inv_tau, false);
-            sh.nArg[i] = ns.idx;
-        }
-    }
-    __syncthreads();
-
-    if (!STOCH) {
-        if (tid == 0) {
-            // ok[] as a bitmask; parent[i] < i so one ascending sweep suffices
-            uint32_t ok[S4C_MASK_WORDS] = {1u, 0, 0, 0};
-            int e = 0;
-            for (int i = 1; i < n; ++i) {
-                const int p = sh.par[i];
-                if (((ok[p >> 5] >> (p & 31)) & 1u) && sh.tok[i] == sh.nArg[p]) {
-                    ok[i >> 5] |= 1u << (i & 31);
-                    if (sh.depth[i] > sh.depth[e]) e = i;
-                }
-            }
-            for (int j = 0; j <= max_depth; ++j) pth[j] = -1;
-            for (int t = e; t >= 0; t = sh.par[t]) pth[sh.depth[t]] = t;
-            accept_len[b] = sh.depth[e];
-            next_token[b] = sh.nArg[e];
-        }
-        return;
-    }
-
-    // ---- speculative-sampling walk: every thread follows the same control flow on the same scalars
-    int cur = 0;
-    for (int guard = 0; guard <= T; ++guard) {
-        const float* lrow = logits + ((size_t)b * T + cur) * V;
-        const float* qrow = dprobs + ((size_t)b * T + cur) * V;
-        const double M = (double)sh.nM[cur];
-        const double invS = sh.nS[cur] > 0.0 ? 1.0 / sh.nS[cur] : 0.0;
-        int r = 0, accepted = -1;
-        for (int c = cur + 1; c < n; ++c) {
-            if (sh.par[c] != cur) continue;
-            const int x = sh.tok[c];
-            double px, qx;
-            chain_eval(exp(((double)__ldg(lrow + x) - M) * inv_tau) * invS, (double)__ldg(qrow + x), x, r, sh, px, qx);
-            double ratio;
-            if (qx > 0.0)
-                ratio = px / qx;
-            else
-                ratio = px > 0.0 ? (double)INFINITY : 0.0;
-            const double u = (double)sh.uni[c];
-            if (tid == 0 && near_tie && fabs(ratio - u) < 1e-6) near_tie[(size_t)b * T + c] = 1;
-            if (u < (ratio < 1.0 ? ratio : 1.0)) {
-                accepted = c;
-                break;
-            }
-            // rejected: residual mass and the draft mass left once x is removed
-            double Z, s;
-            if (r == 0) {
-                Z = sh.nZ[cur], s = sh.nQ[cur];
-            } else {
-                double z = 0.0, qs = 0.0;
-                for (int v = tid; v < V; v += blockDim.x) {
-                    double pv, qv;
-                    chain_eval(exp(((double)__ldg(lrow + v) - M) * inv_tau) * invS, (double)__ldg(qrow + v), v, r, sh,
-                               pv, qv);
-                    const double res = pv - qv;
-                    z += res > 0.0 ? res : 0.0;
-                    qs += (v == x) ? 0.0 : qv;
-                }
-                Z = block_sum(z, sh.scratch);
-                s = block_sum(qs, sh.scratch);
-            }
-            __syncthreads();  // everyone has finished reading the chain before it grows
-            if (tid == 0) {
-                sh.cx[r] = x;
-                sh.cinvZ[r] = Z > 0.0 ? 1.0 / Z : 0.0;
-                sh.cinvs[r] = s > 0.0 ? 1.0 / s : 0.0;
-            }
-            __syncthreads();
-            ++r;
-            if (!(s > 0.0)) break;
-        }
-        if (accepted >= 0) {
-            cur = accepted;
-            __syncthreads();
-            continue;
-        }
-
-        // ---- final token: inverse CDF over the current p at `cur` (Eq. 12 at a fork; plain target at a leaf)
-        const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-        const int seg = ((V + nwarps - 1) / nwarps + 31) / 32 * 32;  // contiguous span per warp
-        const int w0 = warp * seg, w1 = min(V, w0 + seg);
-        double acc = 0.0;
-        int last = -1;
-        for (int v = w0 + lane; v < w1; v += 32) {
-            double pv, qv;
-            chain_eval(exp(((double)__ldg(lrow + v) - M) * inv_tau) * invS, (double)__ldg(qrow + v), v, r, sh, pv, qv);
-            acc += pv;
-            if (pv > 0.0) last = v;
-        }
-        acc = warp_sum(acc);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
-        if (lane == 0) sh.wsum[warp] = acc, sh.wlast[warp] = last;
-        __syncthreads();
-        if (warp == 0) {
-            double tot = 0.0;
-            int lastpos = 0;
-            for (int w = 0; w < nwarps; ++w) {
-                tot += sh.wsum[w];
-                lastpos = max(lastpos, sh.wlast[w]);
-            }
-            const double target = (double)sh.uni[0] * tot;
-            double run = 0.0;
-            int wstar = 0;
-            for (; wstar < nwarps - 1; ++wstar) {
-                if (run + sh.wsum[wstar] > target) break;
-                run += sh.wsum[wstar];
-            }
-            int pick = -1;
-            for (int base = wstar * seg; base < V && pick < 0; base += 32) {
-                const int v = base + lane;
-                double pv = 0.0, qv;
-                if (v < V)
-                    chain_eval(exp(((double)__ldg(lrow + v) - M) * inv_tau) * invS, (double)__ldg(qrow + v), v, r, sh,
-                               pv, qv);
-                double scan = pv;  // inclusive prefix within the group of 32
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const double t = __shfl_up_sync(0xffffffffu, scan, o);
-                    if (lane >= o) scan += t;
-                }
-                const unsigned hit = __ballot_sync(0xffffffffu, v < V && run + scan > target);
-                if (hit) pick = base + __ffs(hit) - 1;
-                run += __shfl_sync(0xffffffffu, scan, 31);
-            }
-            if (lane == 0) {
-                next_token[b] = pick >= 0 ? pick : lastpos;
-                for (int j = 0; j <= max_depth; ++j) pth[j] = -1;
-                for (int t = cur; t >= 0; t = sh.par[t]) pth[sh.depth[t]] = t;
-                accept_len[b] = sh.depth[cur];
-            }
-        }
-        return;
-    }
-}
-
-
 // ============================================================================= cluster path
 // The default path when V is a multiple of 4 and at most 8 * 1024 * 16: one thread-block cluster of 8 CTAs per
 // (sequence, node) row keeps the row's logits in registers, so every logit and every draft probability is read
@@ -485,6 +389,7 @@ constexpr int kCl = 8;             // CTAs per cluster
 constexpr int kClEpt = 16;         // row elements per thread
 constexpr int kClMaxThreads = 1024;
 constexpr int kClMaxV = kCl * kClMaxThreads * kClEpt;
+constexpr size_t kSegStatsMinElems = (size_t)8 << 20;  // B*T*V above which the segment kernels win (measured)
 
 __device__ __forceinline__ uint32_t cl_rank() {
     uint32_t r;
@@ -503,36 +408,6 @@ __device__ __forceinline__ double cl_peer_f64(const double* local, uint32_t rank
     double v;
     asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(ra));
     return v;
-}
-
-// exp(t) for t <= 0 in float64, about 1 ulp: t = (32 k + j) ln2/32 + r, exp(t) = 2^k * 2^(j/32) * e^r with |r| <=
-// ln2/64 and a degree-6 polynomial for e^r (remainder below 4e-18).  About a third of the float64 instructions of
-// the library exp, which matters because this path is otherwise bound by the float64 pipe, not by HBM.
-__device__ const double kExp2Frac[32] = {
-    0x1.0000000000000p+0, 0x1.059b0d3158574p+0, 0x1.0b5586cf9890fp+0, 0x1.11301d0125b51p+0,
-    0x1.172b83c7d517bp+0, 0x1.1d4873168b9aap+0, 0x1.2387a6e756238p+0, 0x1.29e9df51fdee1p+0,
-    0x1.306fe0a31b715p+0, 0x1.371a7373aa9cbp+0, 0x1.3dea64c123422p+0, 0x1.44e086061892dp+0,
-    0x1.4bfdad5362a27p+0, 0x1.5342b569d4f82p+0, 0x1.5ab07dd485429p+0, 0x1.6247eb03a5585p+0,
-    0x1.6a09e667f3bcdp+0, 0x1.71f75e8ec5f74p+0, 0x1.7a11473eb0187p+0, 0x1.82589994cce13p+0,
-    0x1.8ace5422aa0dbp+0, 0x1.93737b0cdc5e5p+0, 0x1.9c49182a3f090p+0, 0x1.a5503b23e255dp+0,
-    0x1.ae89f995ad3adp+0, 0x1.b7f76f2fb5e47p+0, 0x1.c199bdd85529cp+0, 0x1.cb720dcef9069p+0,
-    0x1.d5818dcfba487p+0, 0x1.dfc97337b9b5fp+0, 0x1.ea4afa2a490dap+0, 0x1.f50765b6e4540p+0};
-
-__device__ __forceinline__ double exp_nonpos(double t, const double* tab /* shared copy of kExp2Frac */) {
-    const double kd = rint(t * 0x1.71547652b82fep+5);  // t * 32/ln2
-    if (!(kd > -32000.0)) return exp(t);                // result near or below the normal range (also -inf, NaN)
-    const int k = (int)kd;
-    double r = fma(-kd, 0x1.62e42fefa39efp-6, t);       // ln2/32, high and low part
-    r = fma(-kd, 0x1.abc9e3b39803fp-61, r);
-    double pl = fma(r, 1.0 / 720.0, 1.0 / 120.0);
-    pl = fma(pl, r, 1.0 / 24.0);
-    pl = fma(pl, r, 1.0 / 6.0);
-    pl = fma(pl, r, 0.5);
-    pl = fma(pl, r, 1.0);
-    pl = pl * r;                                        // e^r - 1
-    const double tj = tab[k & 31];
-    const double y = fma(tj, pl, tj);                   // in [1, 2.05)
-    return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));  // * 2^(k >> 5), exponent stays normal
 }
 
 // Cluster-wide exchange area of one CTA: written by its thread 0, read by every peer after a cluster barrier.  Every
@@ -557,7 +432,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == 1024 ? 1 : 2)
 accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
                             const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
                             const int32_t* __restrict__ n_nodes, int T, int V, int chunk, double inv_tau,
-                            NodeSummary* __restrict__ out) {
+                            float floor_span, NodeSummary* __restrict__ out) {
     const int node = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
     const int n = n_nodes ? n_nodes[b] : T;
     if (node >= n || n > T) return;  // the whole cluster leaves together: nobody is left waiting at a barrier
@@ -568,11 +443,11 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     __shared__ ClSlots slot;
     __shared__ double gathered[kCl], gathered2[kCl];
     __shared__ double scratch[33];
-    __shared__ double tab[32];
+    __shared__ double tab[STOCH ? 1024 : 1];
     __shared__ float wm[THREADS / 32];
     __shared__ int wi[THREADS / 32];
     __shared__ int first_tok;
-    if (tid < 32) tab[tid] = kExp2Frac[tid];
+    if (STOCH) fill_exp_table(tab);
     if (STOCH && tid == 32) {  // token of the first child in index order (the first one ever rejected at this node)
         int ft = -1;
         for (int c = node + 1; c < n; ++c)
@@ -605,24 +480,28 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
 
     auto valid = [&](int k) { return elem(k) < V && elem(k) < c0 + chunk; };
 
-    // ---- round 1: maximum and its lowest index
-    float m = -INFINITY;
-    int mi = INT_MAX;
+    // ---- round 1: maximum (one instruction per element), then its lowest index from the few threads that hold it
+    float mt = x[0];
 #pragma unroll
-    for (int k = 0; k < kClEpt; ++k)
-        if (valid(k)) argmax_combine(m, mi, x[k], elem(k));
+    for (int k = 1; k < kClEpt; ++k) mt = fmaxf(mt, x[k]);
+    float m = mt;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, mi, o);
-        argmax_combine(m, mi, om, oi);
-    }
-    if ((tid & 31) == 0) wm[tid >> 5] = m, wi[tid >> 5] = mi;
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((tid & 31) == 0) wm[tid >> 5] = m;
+    if (tid == 0) wi[0] = INT_MAX;
     __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < THREADS / 32; ++w) argmax_combine(m, mi, wm[w], wi[w]);
-        slot.m = (double)m, slot.idx = (double)mi;  // float and int32 are exact in a double
+    m = wm[0];
+    for (int w = 1; w < THREADS / 32; ++w) m = fmaxf(m, wm[w]);
+    if (mt == m) {
+#pragma unroll
+        for (int k = 0; k < kClEpt; ++k)  // a thread's element indices ascend with k
+            if (x[k] == m && valid(k)) {
+                atomicMin(&wi[0], elem(k));
+                break;
+            }
     }
+    __syncthreads();
+    if (tid == 0) slot.m = (double)m, slot.idx = (double)wi[0];  // float and int32 are exact in a double
     cl_gather(&slot.m, gathered, &slot.idx, gathered2);
     float M = -INFINITY;
     int idx = INT_MAX;
@@ -639,12 +518,17 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
 
     // ---- round 2: e = exp((x - M)/tau), once per element, kept in registers; S = sum e
     double e[kClEpt];
-    const double Md = (double)M;
     double s = 0.0;
+    {
+        // elements beyond the row were loaded as -inf: raised to the floor like any other far-away logit, they add
+        // less than 1e-299 of the row sum
+        const float x_floor = M - floor_span;
+        const double c = -(double)M * inv_tau;
 #pragma unroll
-    for (int k = 0; k < kClEpt; ++k) {
-        e[k] = (valid(k) && M > -INFINITY) ? exp_nonpos(((double)x[k] - Md) * inv_tau, tab) : 0.0;
-        s += e[k];
+        for (int k = 0; k < kClEpt; ++k) {
+            e[k] = M > -INFINITY ? exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab) : 0.0;
+            s += e[k];
+        }
     }
     s = block_sum(s, scratch);
     if (tid == 0) slot.s = s;
@@ -660,9 +544,11 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     for (int k = 0; k < kClEpt; ++k) {
         const double qd = (double)q[k];
         const double r = e[k] * invS - qd;
-        z += r > 0.0 ? r : 0.0;
-        qs += (elem(k) == ft) ? 0.0 : qd;
+        if (r > 0.0) z += r;
+        qs += qd;
     }
+    // the first child's token does not count towards the draft mass that is left: one thread takes it out again
+    if (tid == 0 && ft >= c0 && ft < c0 + chunk && ft < V) qs -= (double)__ldg(dprobs + off + ft);
     z = block_sum(z, scratch);
     qs = block_sum(qs, scratch);
     if (tid == 0) slot.z = z, slot.qs = qs;
@@ -683,6 +569,8 @@ struct WalkClShared {
     double tab[32];
     double slots[2][2];  // two alternating sets of (sum a, sum b): set k is rewritten two cluster barriers later
     double ga[kCl], gb[kCl];
+    double tp0[S4C_MAX_T], tq0[S4C_MAX_T];  // node i's token under its parent's row: target and draft probability
+    double pa[33], pb[33];                  // scratch of the paired block reduction
 };
 
 template <bool STOCH>
@@ -691,7 +579,8 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                            const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
                            const int32_t* __restrict__ n_nodes, const float* __restrict__ uniforms, int T, int V,
                            int chunk, int max_depth, double inv_tau, const NodeSummary* __restrict__ nodes,
-                           int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
+                           const NodeStats* __restrict__ seg_nodes, const ResPartial* __restrict__ seg_res, int seg_splits,
+                           const RowPartial* __restrict__ seg_row, int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
                            int32_t* __restrict__ next_token, uint8_t* __restrict__ near_tie,
                            int32_t* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -729,9 +618,35 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         return;
     }
     for (int i = tid; i < n; i += blockDim.x) {
-        const NodeSummary ns = nodes[(size_t)b * T + i];
-        sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = ns.Z, sh.nQ[i] = ns.Q;
+        if (seg_row) {  // statistics came per vocabulary segment: merge them in segment order
+            if (STOCH) {
+                const NodeStats ns = seg_nodes[(size_t)b * T + i];
+                double z = 0.0, q = 0.0;
+                const ResPartial* rp = seg_res + ((size_t)b * T + i) * seg_splits;
+                for (int s = 0; s < seg_splits; ++s) z += rp[s].Z, q += rp[s].Q;
+                sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = z, sh.nQ[i] = q;
+            } else {
+                sh.nArg[i] = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, false).idx;
+            }
+        } else {
+            const NodeSummary ns = nodes[(size_t)b * T + i];
+            sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = ns.Z, sh.nQ[i] = ns.Q;
+        }
     }
+    if (STOCH)  // what the walk will need of the big rows, fetched by all threads at once instead of one test at a time
+        for (int i = 1 + tid; i < n; i += blockDim.x) {
+            const int pr = sh.par[i], x = sh.tok[i];
+            const size_t at = ((size_t)b * T + pr) * V + x;
+            cs.tq0[i] = (double)__ldg(dprobs + at);
+            cs.tp0[i] = (double)__ldg(logits + at);  // turned into a probability below, once the parent's statistics are in
+        }
+    __syncthreads();
+    if (STOCH)
+        for (int i = 1 + tid; i < n; i += blockDim.x) {
+            const int pr = sh.par[i];
+            const double invS = sh.nS[pr] > 0.0 ? 1.0 / sh.nS[pr] : 0.0;
+            cs.tp0[i] = exp_nonpos((cs.tp0[i] - (double)sh.nM[pr]) * inv_tau, cs.tab) * invS;
+        }
     __syncthreads();
     auto write_path = [&](int end) {
         for (int j = 0; j <= max_depth; ++j) pth[j] = -1;
@@ -763,10 +678,17 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
     int round = 0;  // cluster-wide reductions so far (selects the slot set)
     // two cluster-wide sums in rank order; every thread of the cluster calls this and gets the same values
     auto cluster_sum2 = [&](double a, double bsum, double& A, double& Bs) {
-        a = block_sum(a, sh.scratch);
-        bsum = block_sum(bsum, sh.scratch);
+        // both sums through one pair of CTA barriers, each in a fixed order
+        a = warp_sum(a), bsum = warp_sum(bsum);
+        if ((tid & 31) == 0) cs.pa[tid >> 5] = a, cs.pb[tid >> 5] = bsum;
+        __syncthreads();
+        if (tid < 32) {
+            double ta = tid < (int)(blockDim.x >> 5) ? cs.pa[tid] : 0.0, tb = tid < (int)(blockDim.x >> 5) ? cs.pb[tid] : 0.0;
+            ta = warp_sum(ta), tb = warp_sum(tb);
+            double* set = cs.slots[round & 1];
+            if (tid == 0) set[0] = ta, set[1] = tb;
+        }
         double* set = cs.slots[round & 1];
-        if (tid == 0) set[0] = a, set[1] = bsum;
         cl_sync();
         if (tid < kCl) cs.ga[tid] = cl_peer_f64(&set[0], tid), cs.gb[tid] = cl_peer_f64(&set[1], tid);
         __syncthreads();
@@ -782,13 +704,29 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         const float* qrow = dprobs + ((size_t)b * T + cur) * V;
         const double M = (double)sh.nM[cur];
         const double invS = sh.nS[cur] > 0.0 ? 1.0 / sh.nS[cur] : 0.0;
-        auto p0_of = [&](int v) { return exp_nonpos(((double)__ldg(lrow + v) - M) * inv_tau, cs.tab) * invS; };
+        auto p0_from = [&](float logit) { return exp_nonpos(((double)logit - M) * inv_tau, cs.tab) * invS; };
+        // (p, q) after r rejections of up to four vocabulary entries start, start + step, ...; the loads go out
+        // first (these passes are bound by the latency of the loads, not by their volume)
+        auto eval4 = [&](int start, int step, int end, int rr, double (&pv)[4], double (&qv)[4]) {
+            float xl[4], ql[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int v = start + u * step;
+                xl[u] = v < end ? __ldg(lrow + v) : 0.f, ql[u] = v < end ? __ldg(qrow + v) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int v = start + u * step;
+                pv[u] = 0.0, qv[u] = 0.0;
+                if (v < end) chain_eval(p0_from(xl[u]), (double)ql[u], v, rr, sh, pv[u], qv[u]);
+            }
+        };
         int r = 0, accepted = -1;
         for (int c = cur + 1; c < n; ++c) {
             if (sh.par[c] != cur) continue;
             const int x = sh.tok[c];
             double px, qx;
-            chain_eval(p0_of(x), (double)__ldg(qrow + x), x, r, sh, px, qx);
+            chain_eval(cs.tp0[c], cs.tq0[c], x, r, sh, px, qx);
             double ratio;
             if (qx > 0.0)
                 ratio = px / qx;
@@ -806,12 +744,15 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                 Z = sh.nZ[cur], s = sh.nQ[cur];
             } else {
                 double z = 0.0, qs = 0.0;
-                for (int v = c0 + tid; v < c1; v += blockDim.x) {
-                    double pv, qv;
-                    chain_eval(p0_of(v), (double)__ldg(qrow + v), v, r, sh, pv, qv);
-                    const double res = pv - qv;
-                    z += res > 0.0 ? res : 0.0;
-                    qs += (v == x) ? 0.0 : qv;
+                for (int v0 = c0 + tid; v0 < c1; v0 += 4 * blockDim.x) {
+                    double pv[4], qv[4];
+                    eval4(v0, blockDim.x, c1, r, pv, qv);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {  // entries past the end come back as (0, 0)
+                        const double res = pv[u] - qv[u];
+                        z += res > 0.0 ? res : 0.0;
+                        qs += (v0 + u * (int)blockDim.x == x) ? 0.0 : qv[u];
+                    }
                 }
                 cluster_sum2(z, qs, Z, s);
             }
@@ -839,11 +780,14 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         const int w0 = c0 + warp * seg, w1 = min(c1, w0 + seg);
         double acc = 0.0;
         int last = -1;
-        for (int v = w0 + lane; v < w1; v += 32) {
-            double pv, qv;
-            chain_eval(p0_of(v), (double)__ldg(qrow + v), v, r, sh, pv, qv);
-            acc += pv;
-            if (pv > 0.0) last = v;
+        for (int v0 = w0 + lane; v0 < w1; v0 += 128) {
+            double pv[4], qv[4];
+            eval4(v0, 32, w1, r, pv, qv);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                acc += pv[u];
+                if (pv[u] > 0.0) last = v0 + 32 * u;
+            }
         }
         acc = warp_sum(acc);
 #pragma unroll
@@ -886,19 +830,23 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                 run += sh.wsum[wstar];
             }
             int pick = -1;
-            for (int base = c0 + wstar * seg; base < c1 && pick < 0; base += 32) {
-                const int v = base + lane;
-                double pv = 0.0, qv;
-                if (v < c1) chain_eval(p0_of(v), (double)__ldg(qrow + v), v, r, sh, pv, qv);
-                double scan = pv;  // inclusive prefix within the group of 32
+            for (int base4 = c0 + wstar * seg; base4 < c1 && pick < 0; base4 += 128) {
+                double pv4[4], qv4[4];  // four groups of 32 consecutive entries, fetched together, scanned in order
+                eval4(base4 + lane, 32, c1, r, pv4, qv4);
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const double t = __shfl_up_sync(0xffffffffu, scan, o);
-                    if (lane >= o) scan += t;
+                for (int u = 0; u < 4; ++u) {
+                    const int base = base4 + 32 * u, v = base + lane;
+                    if (pick >= 0 || base >= c1) continue;  // warp-uniform
+                    double scan = pv4[u];  // inclusive prefix within the group of 32
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const double t = __shfl_up_sync(0xffffffffu, scan, o);
+                        if (lane >= o) scan += t;
+                    }
+                    const unsigned hit = __ballot_sync(0xffffffffu, v < c1 && run + scan > target);
+                    if (hit) pick = base + __ffs(hit) - 1;
+                    run += __shfl_sync(0xffffffffu, scan, 31);
                 }
-                const unsigned hit = __ballot_sync(0xffffffffu, v < c1 && run + scan > target);
-                if (hit) pick = base + __ffs(hit) - 1;
-                run += __shfl_sync(0xffffffffu, scan, 31);
             }
             if (lane == 0) {
                 // a crossing lost to the different summation order of the scan: this CTA's last token with mass
@@ -943,26 +891,51 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
     const double inv_tau = stoch ? 1.0 / (double)temperature : 1.0;
     dim3 grid(splits, T, B);
 
-    const size_t walk_smem = sizeof(WalkShared);  // ~11 KB, below the 48 KB default limit
-
-    if (vec && V <= kClMaxV) {
-        // ---- cluster path: one 8-CTA cluster per row, then one cluster (greedy: one CTA) per sequence
-        const int chunk = (int)round_up((size_t)ceil_div(V, kCl), 4);
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = kCl, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
-        cudaLaunchConfig_t cfg = {};
+    // ---- per-node statistics: row-in-registers clusters for small problems (one launch, latency-bound), vocabulary
+    //      segments of 4096 with many CTAs per SM for large ones (two launches, throughput-bound)
+#ifdef S4C_EXP_FORCE_SEG
+    const bool seg_stats = S4C_EXP_FORCE_SEG;
+#else
+    const bool seg_stats = !(vec && V <= kClMaxV) || (size_t)B * T * V > kSegStatsMinElems;
+#endif
+    const int chunk = (int)round_up((size_t)ceil_div(V, kCl), 4);
+    const float floor_span = kExpFloorSpan * (stoch ? temperature : 1.f);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kCl, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = stream;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    cudaError_t err = cudaSuccess;
+    if (seg_stats) {
+        if (stoch) {
+            if (vec)
+                accept_rowstats_kernel<true, true><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
+            else
+                accept_rowstats_kernel<true, false><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
+            S4C_RETURN_IF_CUDA_ERROR();
+            if (vec)
+                accept_residual_kernel<true><<<grid, kRowThreads, 0, stream>>>(target_logits, draft_probs, tokens, parent, n_nodes,
+                                                                              T, V, inv_tau, floor_span, ws.row, ws.res, ws.node);
+            else
+                accept_residual_kernel<false><<<grid, kRowThreads, 0, stream>>>(target_logits, draft_probs, tokens, parent, n_nodes,
+                                                                               T, V, inv_tau, floor_span, ws.row, ws.res, ws.node);
+        } else {
+            if (vec)
+                accept_rowstats_kernel<false, true><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
+            else
+                accept_rowstats_kernel<false, false><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
+        }
+        S4C_RETURN_IF_CUDA_ERROR();
+    } else {
         cfg.gridDim = dim3(kCl, T, B);
-        cfg.stream = stream;
-        cfg.attrs = attr, cfg.numAttrs = 1;
-        cudaError_t err;
 #define S4C_LAUNCH_STATS(THREADS)                                                                                      \
     do {                                                                                                               \
         cfg.blockDim = dim3(THREADS, 1, 1);                                                                            \
         err = stoch ? cudaLaunchKernelEx(&cfg, accept_stats_cluster_kernel<THREADS, true>, target_logits, draft_probs, \
-                                         tokens, parent, n_nodes, T, V, chunk, inv_tau, ws.summary)                    \
+                                         tokens, parent, n_nodes, T, V, chunk, inv_tau, floor_span, ws.summary)                    \
                     : cudaLaunchKernelEx(&cfg, accept_stats_cluster_kernel<THREADS, false>, target_logits,            \
-                                         draft_probs, tokens, parent, n_nodes, T, V, chunk, inv_tau, ws.summary);     \
+                                         draft_probs, tokens, parent, n_nodes, T, V, chunk, inv_tau, floor_span, ws.summary);     \
     } while (0)
         if (chunk <= 256 * kClEpt)
             S4C_LAUNCH_STATS(256);
@@ -975,54 +948,29 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
             cudaGetLastError();
             return S4C_ERR_CUDA;
         }
-        const NodeSummary* summary = ws.summary;
-        if (stoch) {
-            cfg.gridDim = dim3(kCl, B, 1);
-            cfg.blockDim = dim3(1024, 1, 1);
-            cfg.dynamicSmemBytes = sizeof(WalkClShared);
-            err = cudaLaunchKernelEx(&cfg, accept_walk_cluster_kernel<true>, target_logits, draft_probs, tokens, parent,
-                                     n_nodes, uniforms, T, V, chunk, max_depth, inv_tau, summary, accept_len, path,
-                                     next_token, near_tie, status);
-            if (err != cudaSuccess) {
-                cudaGetLastError();
-                return S4C_ERR_CUDA;
-            }
-        } else {
-            accept_walk_cluster_kernel<false><<<dim3(1, B), 128, sizeof(WalkClShared), stream>>>(
-                target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, max_depth, inv_tau, summary,
-                accept_len, path, next_token, near_tie, status);
-            S4C_RETURN_IF_CUDA_ERROR();
-        }
-        return S4C_OK;
     }
-
+    // ---- the walk: one cluster per sequence (greedy: one CTA, no vocabulary pass)
+    const NodeSummary* summary = seg_stats ? nullptr : ws.summary;
+    const NodeStats* seg_nodes = seg_stats ? ws.node : nullptr;
+    const ResPartial* seg_res = seg_stats ? ws.res : nullptr;
+    const RowPartial* seg_row = seg_stats ? ws.row : nullptr;
     if (stoch) {
-        if (vec)
-            accept_rowstats_kernel<true, true><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, ws.row);
-        else
-            accept_rowstats_kernel<true, false><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, ws.row);
-        S4C_RETURN_IF_CUDA_ERROR();
-        if (vec)
-            accept_residual_kernel<true><<<grid, kRowThreads, 0, stream>>>(target_logits, draft_probs, tokens, parent, n_nodes,
-                                                                          T, V, inv_tau, ws.row, ws.res, ws.node);
-        else
-            accept_residual_kernel<false><<<grid, kRowThreads, 0, stream>>>(target_logits, draft_probs, tokens, parent, n_nodes,
-                                                                           T, V, inv_tau, ws.row, ws.res, ws.node);
-        S4C_RETURN_IF_CUDA_ERROR();
-        accept_walk_kernel<true><<<B, kWalkThreads, walk_smem, stream>>>(
-            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, max_depth, inv_tau, splits, ws.row, ws.res,
-            ws.node, accept_len, path, next_token, near_tie, status);
+        cfg.gridDim = dim3(kCl, B, 1);
+        cfg.blockDim = dim3(1024, 1, 1);
+        cfg.dynamicSmemBytes = sizeof(WalkClShared);
+        err = cudaLaunchKernelEx(&cfg, accept_walk_cluster_kernel<true>, target_logits, draft_probs, tokens, parent, n_nodes,
+                                 uniforms, T, V, chunk, max_depth, inv_tau, summary, seg_nodes, seg_res, splits, seg_row,
+                                 accept_len, path, next_token, near_tie, status);
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            return S4C_ERR_CUDA;
+        }
     } else {
-        if (vec)
-            accept_rowstats_kernel<false, true><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, ws.row);
-        else
-            accept_rowstats_kernel<false, false><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, ws.row);
+        accept_walk_cluster_kernel<false><<<dim3(1, B), 128, sizeof(WalkClShared), stream>>>(
+            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, max_depth, inv_tau, summary, seg_nodes,
+            seg_res, splits, seg_row, accept_len, path, next_token, near_tie, status);
         S4C_RETURN_IF_CUDA_ERROR();
-        accept_walk_kernel<false><<<B, 128, walk_smem, stream>>>(
-            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, max_depth, inv_tau, splits, ws.row, ws.res,
-            ws.node, accept_len, path, next_token, near_tie, status);
     }
-    S4C_RETURN_IF_CUDA_ERROR();
     return S4C_OK;
 }
 
