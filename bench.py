@@ -64,6 +64,29 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
 
 
+# ----------------------------------------------------------------------------- DRAM traffic seen by ncu
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu capture summarised
+# under profiles/ (the file named here).  It only describes the kernel it was taken on: the value is reported while
+# the kernel source still has the recorded hash, otherwise null.
+NCU_TRAFFIC = {
+    "c2x32": dict(bytes=None, sha256="", profile="profiles/tree_attention_tc_c2x32_ncu_full.md"),
+}
+
+
+def ncu_traffic(workload):
+    import hashlib
+
+    rec = NCU_TRAFFIC.get(workload)
+    if not rec or rec["bytes"] is None:
+        return None
+    src = os.path.join(ROOT, "paper_2506_14158_b200", "csrc", "tree_attention_tc.cu")
+    try:
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    return rec["bytes"] if sha == rec["sha256"] else None
+
+
 # ----------------------------------------------------------------------------- algorithmic bytes
 def algorithmic_bytes(cfg, temperature, accept_lens):
     """Bytes the method must move per step: K/V of the visible slots and Q/O once per layer; every logits row
@@ -337,7 +360,8 @@ def run_ours(args):
                       frac_of_measured_peak=ab["total"] / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
                       frac_of_nominal_8tbs=ab["total"] / (ms * 1e-3) / 1e9 / 8000.0),
         roofline=dict(kernel="tree_attention (one layer)", bound="hbm", achieved=achieved, peak=pk["hbm_gbs"],
-                      unit="GB/s", frac=achieved / pk["hbm_gbs"], peak_source=pk["source"], traffic=None,
+                      unit="GB/s", frac=achieved / pk["hbm_gbs"], peak_source=pk["source"] + " copy bandwidth",
+                      traffic=ncu_traffic(cfg.name), algorithmic_bytes_per_launch=ab["attention_per_layer"],
                       us_per_launch=attn_launch_ms * 1e3, tensor_tflops=flops_layer / (attn_launch_ms * 1e-3) / 1e12),
         breakdown_ms=dict(attention_all_layers=ms_attn, accept=ms_acc, compact=ms_cmp),
         e2e=dict(value=nodes / (ms_e2e * 1e-3), unit=UNIT, h2d_bytes_per_step=step.h2d_bytes,
