@@ -227,12 +227,9 @@ def build_step(cfg, temperature, device, seed_shift=0):
     from paper_2506_14158_b200 import workloads as W
     from paper_2506_14158_b200.verify import VerifyStep
 
-    if seed_shift:
-        from dataclasses import replace
+    from paper_2506_14158_b200 import replicas
 
-        cfg_gen = replace(cfg, config_id=cfg.config_id + 20 * seed_shift)
-    else:
-        cfg_gen = cfg
+    cfg_gen = replicas.rank_config(cfg, seed_shift)  # every replica verifies its own seeded batch
     parent = W.make_trees(cfg_gen)
     x = W.make_accept_inputs(cfg_gen, parent, temperature, token_mode="topk")
     kv_bytes = 2 * cfg.n_layers * cfg.B * cfg.Hkv * cfg.C * cfg.d * (2 if cfg.dtype == "bf16" else 4)
@@ -271,9 +268,9 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2506_14158_b200 import replicas
+
+    rank, world, local = replicas.env_rank_world()
     if world != args.gpus:
         if world == 1 and args.gpus > 1:
             raise SystemExit("launch with torchrun for --gpus > 1")
@@ -296,8 +293,7 @@ def run_ours(args):
     g_cmp = step.capture("compact")
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     for _ in range(Wm):
@@ -331,10 +327,7 @@ def run_ours(args):
     ms_e2e = e0.elapsed_time(e1) / Ke
     accept_lens = step.accept_len.cpu().tolist()
 
-    tt = torch.tensor([ms, ms_attn, ms_e2e], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    ms, ms_attn, ms_e2e = (float(x) for x in tt.tolist())
+    ms, ms_attn, ms_e2e = replicas.max_over_ranks([ms, ms_attn, ms_e2e], device=device)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -348,7 +341,7 @@ def run_ours(args):
     flops_layer = 4.0 * cfg.B * cfg.Hq * cfg.T * (cfg.L + cfg.T) * cfg.d
     attn_kernels = attn_kernels_per_layer(cfg)
     line = dict(
-        metric=METRIC, value=nodes / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=Wm, ms_per_step=ms,
+        metric=METRIC, value=replicas.aggregate_nodes_per_second(cfg.B * cfg.T, world, ms), unit=UNIT, n_gpus=world, steps=K, warmup=Wm, ms_per_step=ms,
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if cfg.dtype == "bf16" else "f32",
         data="synthetic (seeded)",
         config=dict(workload=cfg.name, B=cfg.B, T=cfg.T, L=cfg.L, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, V=cfg.V,
