@@ -38,20 +38,21 @@ constexpr int kMaxClusterSplits = 8;
 constexpr long long kWaitLimitCycles = 400ll * 1000 * 1000;  // about 200 ms at the 1.965 GHz boost clock, longer below it
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
-template <int D, int NM>
+template <int D, int NM, int TC = 1>
 struct TcCfg {
     static constexpr int kHalves = D / 64;           // 64-element (128-byte) swizzle atoms along d
     static constexpr int kQBytes = kBM * D * 2;      // one row tile of Q: 32 KB (d = 128)
     static constexpr int kTileBytes = kBN * D * 2;   // 16 KB: one K or V tile
     static constexpr int kStages = D == 128 ? (NM == 1 ? 6 : 5) : 8;
     static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes;
-    static constexpr int kNumBars = 1 + 4 * kStages + 7 * NM;
+    static constexpr int kScoreBufs = 2 * TC;         // TMEM score buffers per row tile (two per softmax group)
+    static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM;
     static constexpr int kRoleWarps = 1 + 2 * NM;    // TMA warp, then a QK issuer and a PV issuer warp per row tile
-    static constexpr int kThreads = 32 * kRoleWarps + 128 * NM;  // ... and four softmax warps per row tile
+    static constexpr int kThreads = 32 * kRoleWarps + 128 * NM * TC;  // ... and four softmax warps per row tile (and turn)
     static constexpr int kPartStride = D + 4;        // floats per parked row (padding spreads the banks)
-    static constexpr int kPartBytes = NM * kBM * kPartStride * 4 + NM * kBM * 8;
+    static constexpr int kPartBytes = NM * TC * kBM * kPartStride * 4 + NM * TC * kBM * 8;
     static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
-    static constexpr int kTmemCols = NM * 128 + NM * D <= 256 ? 256 : 512;
+    static constexpr int kTmemCols = NM * kScoreBufs * kBN + NM * TC * D <= 256 ? 256 : 512;
     static_assert(kNumBars * 8 <= 480, "barrier area");
     static_assert(kPartBytes <= kSmemData, "parked partials reuse the tile buffers");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
@@ -287,12 +288,16 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, 
 // of each tile: its own running offset and sum, its own slice of P (the rest of its P rows stays zero), its
 // own accumulator rows.  The copies are merged like splits.  This spreads the exponentials of a small tree
 // over all four softmax warps instead of leaving them to one.
-template <int D, int NM, int REP>
-__global__ void __launch_bounds__(TcCfg<D, NM>::kThreads, 1)
+// TC == 2 (one row tile of 65..128 rows, no row copies): two softmax groups take turns, group c owning the tiles
+// j = c, c+2, ... with score buffer c and an accumulator of its own -- a full 128-row tile keeps one softmax group
+// busy for longer than a tile takes to arrive, two groups do not.  The two accumulators merge like splits.
+template <int D, int NM, int REP, int TC>
+__global__ void __launch_bounds__(TcCfg<D, NM, TC>::kThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const TcParams prm) {
     static_assert(NM == 1 || REP == 1, "row copies only with a single row tile");
-    using Cfg = TcCfg<D, NM>;
+    static_assert(TC == 1 || (NM == 1 && REP == 1), "turns only with a single row tile and no row copies");
+    using Cfg = TcCfg<D, NM, TC>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
     constexpr int PS = Cfg::kPartStride;
@@ -316,10 +321,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     auto BAR = [&](int i) { return bar0 + 8u * i; };
     // barrier indices; the per-row-tile ones take (tile t, buffer i)
     constexpr int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + S, V_FULL = 1 + 2 * S, V_EMPTY = 1 + 3 * S, PER_TILE = 1 + 4 * S;
-    auto S_FULL = [&](int t, int i) { return BAR(PER_TILE + 7 * t + i); };
-    auto S_EMPTY = [&](int t, int i) { return BAR(PER_TILE + 7 * t + 2 + i); };
-    auto P_FULL = [&](int t, int i) { return BAR(PER_TILE + 7 * t + 4 + i); };
-    auto PV_DONE = [&](int t) { return BAR(PER_TILE + 7 * t + 6); };
+    constexpr int NB = Cfg::kScoreBufs, PT = 3 * NB + TC;  // score buffers and barriers per row tile; tile j uses buffer j % NB
+    auto S_FULL = [&](int t, int i) { return BAR(PER_TILE + PT * t + i); };
+    auto S_EMPTY = [&](int t, int i) { return BAR(PER_TILE + PT * t + NB + i); };
+    auto P_FULL = [&](int t, int i) { return BAR(PER_TILE + PT * t + 2 * NB + i); };
+    auto PV_DONE = [&](int t, int c) { return BAR(PER_TILE + PT * t + 3 * NB + c); };  // c: the softmax group whose tile it was
 
     const int split = blockIdx.x, splits = prm.splits;
     const int mg = blockIdx.y % prm.m_groups, hk = blockIdx.y / prm.m_groups, b = blockIdx.z;
@@ -344,9 +350,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                                  // the ring one commit per active row tile (each has issuer threads of its own)
             if ((i >= K_EMPTY && i < K_EMPTY + S) || (i >= V_EMPTY && i < V_EMPTY + S)) count = (uint32_t)nm_act;
             if (i >= PER_TILE) {
-                const int t = (i - PER_TILE) / 7, k = (i - PER_TILE) % 7;
+                const int t = (i - PER_TILE) / PT, k = (i - PER_TILE) % PT;
                 const uint32_t active = (uint32_t)active_threads(t) / 32u;
-                if (k >= 4 && k < 6 && active) count = active;
+                if (k >= 2 * NB && k < 3 * NB && active) count = active;
             }
             mbar_init(BAR(i), count);
         }
@@ -362,8 +368,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     __syncthreads();  // the only CTA-wide barrier before the results: from here on the roles run on mbarriers alone
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    auto TM_S = [&](int t, int i) { return tmem + (uint32_t)(t * 2 * kBN + i * kBN); };
-    auto TM_O = [&](int t) { return tmem + (uint32_t)(NM * 2 * kBN + t * D); };
+    auto TM_S = [&](int t, int i) { return tmem + (uint32_t)((t * NB + i) * kBN); };
+    auto TM_O = [&](int t, int c) { return tmem + (uint32_t)(NM * NB * kBN + (t * TC + c) * D); };
 
     griddep_wait();  // everything below may depend on the previous kernel of the stream
 
@@ -438,13 +444,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const int s = j % S, it = j / S;
                 mbar_wait(BAR(K_FULL + s), it & 1, dead);
                 const uint64_t k_desc = smem_desc_sw128(sK + s * Cfg::kTileBytes, 16, 1024);
-                mbar_wait(S_EMPTY(t, j & 1), ((j >> 1) & 1) ^ 1, dead);
+                mbar_wait(S_EMPTY(t, j % NB), ((j / NB) & 1) ^ 1, dead);
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)  // the start-address field counts 16-byte units
-                    tc_mma_bf16(TM_S(t, j & 1), a_desc[kk], k_desc + (uint64_t)(((kk >> 2) * (kBN * 128) + (kk & 3) * 32) >> 4),
+                    tc_mma_bf16(TM_S(t, j % NB), a_desc[kk], k_desc + (uint64_t)(((kk >> 2) * (kBN * 128) + (kk & 3) * 32) >> 4),
                                 idesc_qk, kk > 0 ? 1u : 0u);
-                tc_commit(S_FULL(t, j & 1));
+                tc_commit(S_FULL(t, j % NB));
                 tc_commit(BAR(K_EMPTY + s));
             }
         }
@@ -458,15 +464,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 mbar_wait(BAR(V_FULL + s), it & 1, dead);
                 // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
                 const uint64_t v_desc = smem_desc_sw128(sV + s * Cfg::kTileBytes, kBN * 128, 1024);
-                mbar_wait(P_FULL(t, j & 1), (j >> 1) & 1, dead);
+                mbar_wait(P_FULL(t, j % NB), (j / NB) & 1, dead);
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kBN / 16; ++kk)
                     // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
-                    tc_mma_bf16_ts(TM_O(t), TM_S(t, j & 1) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv,
-                                   (j > 0 || kk > 0) ? 1u : 0u);
-                tc_commit(PV_DONE(t));
-                tc_commit(S_EMPTY(t, j & 1));  // the score buffer (and the P inside it) may be overwritten
+                    tc_mma_bf16_ts(TM_O(t, TC == 2 ? (j & 1) : 0), TM_S(t, j % NB) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4),
+                                   idesc_pv, (j >= TC || kk > 0) ? 1u : 0u);
+                tc_commit(PV_DONE(t, TC == 2 ? (j & 1) : 0));
+                tc_commit(S_EMPTY(t, j % NB));  // the score buffer (and the P inside it) may be overwritten
                 tc_commit(BAR(V_EMPTY + s));
             }
         }
@@ -482,11 +488,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 if (i < n && ((i == 0 && p != -1) || (i > 0 && (p < 0 || p >= i)))) atomicOr(bad_s, S4C_SEQ_BAD_PARENT);
             }
         }
-        named_bar_sync(1, NM * 128);
+        named_bar_sync(1, NM * TC * 128);
         flags |= *bad_s;
         if (split == 0 && blockIdx.y == 0 && threadIdx.x == 32 * Cfg::kRoleWarps && prm.status) prm.status[b] = flags;
         const bool run = flags == 0;
-        const int t = (warp - Cfg::kRoleWarps) >> 2;  // row tile of this warp group
+        const int grp = (warp - Cfg::kRoleWarps) >> 2;  // this warp group: a row tile, or (TC == 2) a turn on the one row tile
+        const int t = TC == 2 ? 0 : grp, tc = TC == 2 ? grp : 0;
+        const int n_own = nt > tc ? (nt - tc + TC - 1) / TC : 0;  // tiles this group takes: tc, tc + TC, ...
         const int wq = warp & 3;        // TMEM lane quadrant this warp may access
         const int row = wq * 32 + lane;
         const int copy = row / RB, lr = row % RB;  // which copy of the rows, and the row within it
@@ -510,14 +518,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const float sc = prm.scale_log2;
 
         if (warp_active)
-            for (int j = 0; j < nt; ++j) {
+            for (int j = tc; j < nt; j += TC) {
                 const int kv0 = (t0 + j) * kBN;
-                mbar_wait_warp(S_FULL(t, j & 1), (j >> 1) & 1, dead);
+                mbar_wait_warp(S_FULL(t, j % NB), (j / NB) & 1, dead);
                 tc_fence_after();
                 float sv[CW];
                 {
                     uint32_t sr[CW];
-                    tmem_ld_cols<CW>(TM_S(t, j & 1) + lane_off + c0, sr);
+                    tmem_ld_cols<CW>(TM_S(t, j % NB) + lane_off + c0, sr);
                     tmem_wait_ld();
 #pragma unroll
                     for (int c = 0; c < CW; ++c) sv[c] = __uint_as_float(sr[c]);
@@ -560,18 +568,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
                 m = m_new;
 
-                if (j > 0) {
-                    mbar_wait_warp(PV_DONE(t), (j - 1) & 1, dead);
+                if (j >= TC) {  // this group's previous product: number (j - tc) / TC - 1 on its own barrier
+                    mbar_wait_warp(PV_DONE(t, tc), ((j - tc) / TC - 1) & 1, dead);
                     tc_fence_after();
                     if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll
                         for (int cc = 0; cc < D / 32; ++cc) {
                             uint32_t o[32];
-                            tmem_ld_cols<32>(TM_O(t) + lane_off + cc * 32, o);
+                            tmem_ld_cols<32>(TM_O(t, tc) + lane_off + cc * 32, o);
                             tmem_wait_ld();
 #pragma unroll
                             for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                            tmem_st32(TM_O(t) + lane_off + cc * 32, o);
+                            tmem_st32(TM_O(t, tc) + lane_off + cc * 32, o);
                         }
                         tmem_wait_st();
                     }
@@ -597,7 +605,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 // scores were read above).  A copy owns CW/2 of these columns and clears the others: the product runs
                 // over all 64 slots of every row.
                 {
-                    const uint32_t p_row = TM_S(t, j & 1) + lane_off;
+                    const uint32_t p_row = TM_S(t, j % NB) + lane_off;
                     tmem_st_cols<CW / 2>(p_row + c0 / 2, pk);
                     if (REP > 1) {
                         uint32_t zero[CW / 2];
@@ -610,25 +618,25 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(P_FULL(t, j & 1));
+                if (lane == 0) mbar_arrive(P_FULL(t, j % NB));
             }
 
         // ---- this split's (and copy's) result for the row: (m, l, unnormalised O)
-        if (warp_active && nt > 0) {
-            mbar_wait_warp(PV_DONE(t), (nt - 1) & 1, dead);
+        if (warp_active && n_own > 0) {
+            mbar_wait_warp(PV_DONE(t, tc), (n_own - 1) & 1, dead);
             tc_fence_after();
         }
         const bool node_valid = row_ok && node < n;
         if (prm.mode == kModeCluster) {
             // every MMA of the CTA has finished before any tile buffer is reused for the parked partials
-            named_bar_sync(1, NM * 128);
+            named_bar_sync(1, NM * TC * 128);
             if (warp_active) {
-                float* po = reinterpret_cast<float*>(base_ptr) + (size_t)(t * kBM + row) * PS;
+                float* po = reinterpret_cast<float*>(base_ptr) + (size_t)((t * TC + tc) * kBM + row) * PS;
 #pragma unroll
                 for (int cc = 0; cc < D / 32; ++cc) {
                     uint32_t o[32];
-                    if (nt > 0) {
-                        tmem_ld_cols<32>(TM_O(t) + lane_off + cc * 32, o);
+                    if (n_own > 0) {
+                        tmem_ld_cols<32>(TM_O(t, tc) + lane_off + cc * 32, o);
                         tmem_wait_ld();
                     } else {
 #pragma unroll
@@ -639,19 +647,20 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         *reinterpret_cast<float4*>(po + cc * 32 + c) = make_float4(
                             __uint_as_float(o[c]), __uint_as_float(o[c + 1]), __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
                 }
-                float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)NM * kBM * PS);
-                pml[t * kBM + row] = make_float2(m, l);
+                float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)NM * TC * kBM * PS);
+                pml[(t * TC + tc) * kBM + row] = make_float2(m, l);
             }
         } else if (warp_active && run) {
             const bool direct = prm.mode == kModeDirect;  // REP == 1 then
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
             const float inv = (node_valid && l > 0.f) ? 1.f / l : 0.f;
-            float* wrow = prm.ws + (orow * (size_t)(splits * REP) + (size_t)(split * REP + copy)) * (D + 2);
+            // workspace: every (split, row copy or turn) is one partial of the row
+            float* wrow = prm.ws + (orow * (size_t)(splits * REP * TC) + (size_t)(split * REP * TC + (TC == 2 ? tc : copy))) * (D + 2);
 #pragma unroll
             for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t o[32];
-                if (nt > 0) {
-                    tmem_ld_cols<32>(TM_O(t) + lane_off + cc * 32, o);
+                if (n_own > 0) {
+                    tmem_ld_cols<32>(TM_O(t, tc) + lane_off + cc * 32, o);
                     tmem_wait_ld();
                 } else {
 #pragma unroll
@@ -695,9 +704,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         cluster_sync_all();
         const bool run = (flags | *bad_s) == 0;  // the same in every CTA of the cluster: it depends on the sequence only
         const uint32_t rank = cluster_ctarank();
-        const uint32_t part = base, part_ml = base + (uint32_t)(NM * kBM * PS * 4);
+        const uint32_t part = base, part_ml = base + (uint32_t)(NM * TC * kBM * PS * 4);
         constexpr int EPL = D / 32;  // output elements per lane
-        const int np = splits * REP;  // partials per output row (<= 32)
+        constexpr int NC = REP * TC;  // partials per split: row copies or turns
+        const int np = splits * NC;   // partials per output row (<= 32)
+        // shared-memory row of partial i of output row (t, lr): i / NC is the split, i % NC the copy or turn
+        auto part_row = [&](int t, int lr, int i) {
+            const int w = i % NC;
+            return (uint32_t)((t * TC + (TC == 2 ? w : 0)) * kBM + (REP > 1 ? w * RB : 0) + lr);
+        };
         if (run)
             for (int idx = (int)rank + splits * warp; idx < NM * RB; idx += splits * (Cfg::kThreads / 32)) {
                 const int t = idx / RB, lr = idx % RB;
@@ -707,7 +722,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 // partial i = (split i / REP, copy i % REP)
                 float2 ml = make_float2(-INFINITY, 0.f);
                 if (lane < np)
-                    ml = ld_cluster_f2(map_to_cta(part_ml + (uint32_t)(t * kBM + (lane % REP) * RB + lr) * 8u, (uint32_t)(lane / REP)));
+                    ml = ld_cluster_f2(map_to_cta(part_ml + part_row(t, lr, lane) * 8u, (uint32_t)(lane / NC)));
                 float M = ml.x;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
@@ -723,8 +738,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         const int i = i0 + k;
                         o4[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                         if (i < np) {
-                            const uint32_t prow = (uint32_t)(t * kBM + (i % REP) * RB + lr);
-                            const uint32_t a = map_to_cta(part + (prow * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)(i / REP));
+                            const uint32_t prow = part_row(t, lr, i);
+                            const uint32_t a = map_to_cta(part + (prow * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)(i / NC));
                             if (EPL == 4) {
                                 o4[k] = ld_cluster_f4(a);
                             } else {
@@ -844,20 +859,30 @@ static int tc_rep(int T, int Hq, int Hkv) {
     return R <= 32 ? 4 : (R <= 64 ? 2 : 1);
 }
 
+// Turns (see the kernel): a single row tile of 65..128 rows with enough tiles per CTA is shared by two softmax groups.
+static int tc_turns(int B, int T, int Hq, int Hkv, int C) {
+    const int R = (Hq / Hkv) * T;
+    if (R <= 64 || R > kBM) return 1;
+    const int tiles_per_cta = ceil_div(ceil_div(C, kBN), tc_splits(B, T, Hq, Hkv, C));
+    return tiles_per_cta >= 8 ? 2 : 1;
+}
+
 size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
     const int s = tc_splits(B, T, Hq, Hkv, C);
     return s <= kMaxClusterSplits ? 0
-                                  : round_up((size_t)B * Hq * T * s * tc_rep(T, Hq, Hkv) * (d + 2) * sizeof(float), 256);
+                                  : round_up((size_t)B * Hq * T * s * tc_rep(T, Hq, Hkv) * tc_turns(B, T, Hq, Hkv, C) *
+                                                 (d + 2) * sizeof(float),
+                                             256);
 }
 
-template <int D, int NM, int REP>
+template <int D, int NM, int REP, int TC>
 static s4c_status launch_tc(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
-    using Cfg = TcCfg<D, NM>;
+    using Cfg = TcCfg<D, NM, TC>;
     static bool configured[64] = {};  // the opt-ins (dynamic shared memory, cluster size) are per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return S4C_ERR_CUDA;
         configured[dev] = true;
@@ -886,7 +911,7 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
     }
     cfg.attrs = attrs;
     cfg.numAttrs = na;
-    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP>, mq, mk, mv, prm) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP, TC>, mq, mk, mv, prm) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
@@ -903,26 +928,30 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     const int nm = tc_nm(T, Hq, Hkv);
     prm.m_groups = tc_m_groups(T, Hq, Hkv);
     prm.splits = tc_splits(B, T, Hq, Hkv, C);
-    const int rep = tc_rep(T, Hq, Hkv);
-    // the copies of a row merge like splits, so a single split with copies still takes the (one-CTA) cluster path
-    prm.mode = prm.splits > kMaxClusterSplits ? kModeWorkspace : (prm.splits == 1 && rep == 1 ? kModeDirect : kModeCluster);
+    const int rep = tc_rep(T, Hq, Hkv), turns = tc_turns(B, T, Hq, Hkv, C);
+    // copies and turns merge like splits, so a single split with either still takes the (one-CTA) cluster path
+    prm.mode = prm.splits > kMaxClusterSplits ? kModeWorkspace
+                                              : (prm.splits == 1 && rep == 1 && turns == 1 ? kModeDirect : kModeCluster);
     const int R = (Hq / Hkv) * T;
     prm.q_box_rows = R >= kBM ? kBM : (int)round_up((size_t)R, 8);
     prm.scale_log2 = scale * 1.4426950408889634f;
     s4c_status st;
     if (d == 128)
-        st = nm == 2   ? launch_tc<128, 2, 1>(q, k, v, prm, B, stream)
-             : rep == 4 ? launch_tc<128, 1, 4>(q, k, v, prm, B, stream)
-             : rep == 2 ? launch_tc<128, 1, 2>(q, k, v, prm, B, stream)
-                        : launch_tc<128, 1, 1>(q, k, v, prm, B, stream);
+        st = nm == 2      ? launch_tc<128, 2, 1, 1>(q, k, v, prm, B, stream)
+             : rep == 4   ? launch_tc<128, 1, 4, 1>(q, k, v, prm, B, stream)
+             : rep == 2   ? launch_tc<128, 1, 2, 1>(q, k, v, prm, B, stream)
+             : turns == 2 ? launch_tc<128, 1, 1, 2>(q, k, v, prm, B, stream)
+                          : launch_tc<128, 1, 1, 1>(q, k, v, prm, B, stream);
     else
-        st = nm == 2   ? launch_tc<64, 2, 1>(q, k, v, prm, B, stream)
-             : rep == 4 ? launch_tc<64, 1, 4>(q, k, v, prm, B, stream)
-             : rep == 2 ? launch_tc<64, 1, 2>(q, k, v, prm, B, stream)
-                        : launch_tc<64, 1, 1>(q, k, v, prm, B, stream);
+        st = nm == 2      ? launch_tc<64, 2, 1, 1>(q, k, v, prm, B, stream)
+             : rep == 4   ? launch_tc<64, 1, 4, 1>(q, k, v, prm, B, stream)
+             : rep == 2   ? launch_tc<64, 1, 2, 1>(q, k, v, prm, B, stream)
+             : turns == 2 ? launch_tc<64, 1, 1, 2>(q, k, v, prm, B, stream)
+                          : launch_tc<64, 1, 1, 1>(q, k, v, prm, B, stream);
     if (st != S4C_OK) return st;
     if (prm.mode == kModeWorkspace)
-        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits * rep, S4C_BF16, stream);
+        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits * rep * turns, S4C_BF16,
+                                      stream);
     return S4C_OK;
 }
 

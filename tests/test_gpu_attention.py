@@ -85,3 +85,13 @@ def test_results_do_not_depend_on_scheduling():
     a, _, _, _ = attention_both(q, k, v, [cfg.L], parent)
     b, _, _, _ = attention_both(q, k, v, [cfg.L], parent)
     np.testing.assert_array_equal(a, b)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_full_row_tile_with_two_softmax_groups_taking_turns(d):
+    # 65..128 rows and a long cache: two softmax groups alternate over the tiles, merged inside the cluster ...
+    _case(B=1, Hq=16, Hkv=16, T=100, d=d, Ls=[6000], dtype="bf16", seed=11)
+    # ... an odd number of tiles per split, GQA rows (2 heads x 50 nodes), padded trees ...
+    _case(B=2, Hq=16, Hkv=8, T=50, d=d, Ls=[5000, 4321], dtype="bf16", seed=12, n_nodes=[50, 33])
+    # ... and through the workspace when the grid is too small for clusters
+    _case(B=1, Hq=4, Hkv=4, T=100, d=d, Ls=[20000], dtype="bf16", seed=13)
