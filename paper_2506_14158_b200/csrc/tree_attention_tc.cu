@@ -650,6 +650,36 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)NM * TC * kBM * PS);
                 pml[(t * TC + tc) * kBM + row] = make_float2(m, l);
             }
+            if (REP > 1) {
+                // The copies of a row are merged here, inside the CTA, before the splits are merged across the
+                // cluster: distributed shared memory moves only ~16 bytes per clock and SM, so it should carry one
+                // partial per split and row, not REP.  Merged rows go behind the parked ones.
+                named_bar_sync(1, 128);
+                const float* pin = reinterpret_cast<const float*>(base_ptr);
+                const float2* pml_in = reinterpret_cast<const float2*>(pin + (size_t)kBM * PS);
+                float* mout = reinterpret_cast<float*>(base_ptr) + (size_t)kBM * PS + 2 * kBM;
+                float2* mml = reinterpret_cast<float2*>(mout + (size_t)RB * PS);
+                constexpr int EPLm = D / 32;
+                for (int r = warp - Cfg::kRoleWarps; r < rows_t; r += 4) {
+                    float mc[REP], M = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < REP; ++c) mc[c] = pml_in[c * RB + r].x, M = fmaxf(M, mc[c]);
+                    float den = 0.f, num[EPLm];
+#pragma unroll
+                    for (int e = 0; e < EPLm; ++e) num[e] = 0.f;
+#pragma unroll
+                    for (int c = 0; c < REP; ++c) {  // copy order: the same on every run
+                        const float f = exp2f(mc[c] - M);
+                        den = fmaf(f, pml_in[c * RB + r].y, den);
+                        const float* src = pin + (size_t)(c * RB + r) * PS + lane * EPLm;
+#pragma unroll
+                        for (int e = 0; e < EPLm; ++e) num[e] = fmaf(f, src[e], num[e]);
+                    }
+#pragma unroll
+                    for (int e = 0; e < EPLm; ++e) mout[(size_t)r * PS + lane * EPLm + e] = num[e];
+                    if (lane == 0) mml[r] = make_float2(M, den);
+                }
+            }
         } else if (warp_active && run) {
             const bool direct = prm.mode == kModeDirect;  // REP == 1 then
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
@@ -704,15 +734,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         cluster_sync_all();
         const bool run = (flags | *bad_s) == 0;  // the same in every CTA of the cluster: it depends on the sequence only
         const uint32_t rank = cluster_ctarank();
-        const uint32_t part = base, part_ml = base + (uint32_t)(NM * TC * kBM * PS * 4);
+        // row copies were merged inside their CTA (rows behind the parked ones); turns are merged here with the splits
+        const uint32_t part = REP > 1 ? base + (uint32_t)((kBM * PS + 2 * kBM) * 4) : base;
+        const uint32_t part_ml = REP > 1 ? part + (uint32_t)(RB * PS * 4) : base + (uint32_t)(NM * TC * kBM * PS * 4);
         constexpr int EPL = D / 32;  // output elements per lane
-        constexpr int NC = REP * TC;  // partials per split: row copies or turns
-        const int np = splits * NC;   // partials per output row (<= 32)
-        // shared-memory row of partial i of output row (t, lr): i / NC is the split, i % NC the copy or turn
-        auto part_row = [&](int t, int lr, int i) {
-            const int w = i % NC;
-            return (uint32_t)((t * TC + (TC == 2 ? w : 0)) * kBM + (REP > 1 ? w * RB : 0) + lr);
-        };
+        constexpr int NC = TC;       // partials per split
+        const int np = splits * NC;  // partials per output row (<= 16)
+        // shared-memory row of partial i of output row (t, lr): i / NC is the split, i % NC the turn
+        auto part_row = [&](int t, int lr, int i) { return (uint32_t)((t * TC + i % NC) * kBM + lr); };
         if (run)
             for (int idx = (int)rank + splits * warp; idx < NM * RB; idx += splits * (Cfg::kThreads / 32)) {
                 const int t = idx / RB, lr = idx % RB;
