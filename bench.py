@@ -233,7 +233,7 @@ def build_step(cfg, temperature, device, seed_shift=0):
     parent = W.make_trees(cfg_gen)
     x = W.make_accept_inputs(cfg_gen, parent, temperature, token_mode="topk")
     kv_bytes = 2 * cfg.n_layers * cfg.B * cfg.Hkv * cfg.C * cfg.d * (2 if cfg.dtype == "bf16" else 4)
-    on_device = kv_bytes > (4 << 30)
+    on_device = kv_bytes > (1 << 30)
     qs, ks, vs = [], [], []
     dt = {"f32": torch.float32, "bf16": torch.bfloat16}[cfg.dtype]
     for l in range(cfg.n_layers):
@@ -306,6 +306,7 @@ def run_ours(args):
     t1 = time.time()
     clocks = sampler.stop(t0, t1) if sampler else None
     # dominant-kernel leg: the n_layers attention launches alone, same buffers, same stream, CUDA events
+    step.reset_lengths()  # the step's compaction advanced the lengths: attention is timed on the committed ones
     for _ in range(3):
         g_attn.replay()
     torch.cuda.synchronize()
@@ -376,6 +377,54 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep_all(args):
+    """Config 5, every point: the 7B layer shape x 32 layers with an independent cache per layer, context 512..32768,
+    trees of 16..128 nodes, batch 1/4/16.  One JSON line per point (nodes/s, HBM GB/s of the step and of the attention
+    launches); points whose 32 caches do not fit the device are recorded as such, never aliased."""
+    import gc
+
+    import torch
+
+    import __graft_entry__ as entry
+    from paper_2506_14158_b200 import workloads as W
+
+    entry.build()
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    pk = peaks()
+    free_b, total_b = torch.cuda.mem_get_info()
+    for B in (1, 4, 16):
+        for T in (16, 32, 64, 128):
+            for L in (512, 1024, 2048, 4096, 8192, 16384, 32768):
+                cfg = W.sweep_config(L, T, B, args.layers)
+                kv = 2 * cfg.n_layers * cfg.B * cfg.Hkv * cfg.C * cfg.d * 2
+                point = dict(workload=cfg.name, B=B, T=T, L=L, n_layers=cfg.n_layers, kv_gb=round(kv / 1e9, 2))
+                if kv > 0.8 * total_b:
+                    point["result"] = "exceeds device memory"
+                    print(json.dumps(point), flush=True)
+                    continue
+                step = build_step(cfg, args.temperature, device)
+                g_step, g_attn = step.capture("step"), step.capture("attention")
+                iters = 20 if kv < (8 << 30) else 5
+                for _ in range(3):
+                    g_step.replay()
+                torch.cuda.synchronize()
+                ms = time_graph(g_step, iters, torch)
+                step.reset_lengths()  # attention alone is timed on the committed lengths
+                torch.cuda.synchronize()
+                ms_attn = time_graph(g_attn, iters, torch)
+                ab = algorithmic_bytes(cfg, args.temperature, step.accept_len.cpu().tolist())
+                point.update(ms_per_step=round(ms, 4), nodes_per_s=round(B * T / (ms * 1e-3), 1),
+                             step_gbs=round(ab["total"] / (ms * 1e-3) / 1e9, 1),
+                             attn_us_per_layer=round(ms_attn / cfg.n_layers * 1e3, 2),
+                             attn_gbs=round(ab["attention"] / (ms_attn * 1e-3) / 1e9, 1),
+                             attn_frac_of_measured_peak=round(ab["attention"] / (ms_attn * 1e-3) / 1e9 / pk["hbm_gbs"], 3))
+                print(json.dumps(point), flush=True)
+                del step, g_step, g_attn
+                gc.collect()
+                torch.cuda.empty_cache()
+
+
 def attn_kernels_per_layer(cfg):
     from paper_2506_14158_b200 import s4c
     import torch
@@ -386,7 +435,9 @@ def attn_kernels_per_layer(cfg):
 
 if __name__ == "__main__":
     a = parse_args()
-    if a.impl == "reference":
+    if a.workload == "sweep-all":
+        run_sweep_all(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_ours(a)
