@@ -38,13 +38,15 @@ constexpr int kMaxClusterSplits = 8;
 constexpr long long kWaitLimitCycles = 400ll * 1000 * 1000;  // about 200 ms at the 1.965 GHz boost clock, longer below it
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
-template <int D, int NM, int TC = 1>
+template <int D, int NM, int TC = 1, int PUSH = 0>
 struct TcCfg {
     static constexpr int kHalves = D / 64;           // 64-element (128-byte) swizzle atoms along d
     static constexpr int kQBytes = kBM * D * 2;      // one row tile of Q: 32 KB (d = 128)
     static constexpr int kTileBytes = kBN * D * 2;   // 16 KB: one K or V tile
-    static constexpr int kStages = D == 128 ? (NM == 1 ? 6 : 5) : 8;
-    static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes;
+    // PUSH: 32 KB at the end of the tile area are set aside to receive the other splits' partials (see the kernel)
+    static constexpr int kRecvBytes = PUSH ? 32768 : 0;
+    static constexpr int kStages = (D == 128 ? (NM == 1 ? 6 : 5) : 8) - kRecvBytes / (2 * kTileBytes);
+    static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes + kRecvBytes;
     static constexpr int kScoreBufs = 2 * TC;         // TMEM score buffers per row tile (two per softmax group)
     static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM;
     static constexpr int kRoleWarps = 1 + 2 * NM;    // TMA warp, then a QK issuer and a PV issuer warp per row tile
@@ -231,6 +233,12 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void st_cluster_f4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
@@ -291,13 +299,17 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, 
 // TC == 2 (one row tile of 65..128 rows, no row copies): two softmax groups take turns, group c owning the tiles
 // j = c, c+2, ... with score buffer c and an accumulator of its own -- a full 128-row tile keeps one softmax group
 // busy for longer than a tile takes to arrive, two groups do not.  The two accumulators merge like splits.
-template <int D, int NM, int REP, int TC>
-__global__ void __launch_bounds__(TcCfg<D, NM, TC>::kThreads, 1)
+// PUSH (one row tile, no turns, few rows): instead of parking partials for the peers to fetch, every CTA stores its
+// (copy-merged) rows into a receive area of the row's owner that is used for nothing else, so no barrier has to say
+// "my tile buffers are dead" first; after one cluster barrier the owner merges from its own shared memory and leaves.
+template <int D, int NM, int REP, int TC, int PUSH>
+__global__ void __launch_bounds__(TcCfg<D, NM, TC, PUSH>::kThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const TcParams prm) {
     static_assert(NM == 1 || REP == 1, "row copies only with a single row tile");
     static_assert(TC == 1 || (NM == 1 && REP == 1), "turns only with a single row tile and no row copies");
-    using Cfg = TcCfg<D, NM, TC>;
+    static_assert(PUSH == 0 || (NM == 1 && TC == 1), "pushed partials only with a single row tile and no turns");
+    using Cfg = TcCfg<D, NM, TC, PUSH>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
     constexpr int PS = Cfg::kPartStride;
@@ -680,6 +692,32 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     if (lane == 0) mml[r] = make_float2(M, den);
                 }
             }
+            if (PUSH) {
+                // this CTA's (copy-merged) partial of row r goes to CTA r % splits, slot (r / splits) * splits + split
+                // of its receive area: 32 lanes x 16 (d = 64: 8) bytes per row, (offset, sum) into the row's padding
+                if (REP > 1)
+                    __syncwarp();  // a warp pushes the rows it merged itself
+                else
+                    named_bar_sync(1, 128);  // rows were parked one per thread
+                const float* rows_src = reinterpret_cast<const float*>(base_ptr) + (REP > 1 ? (size_t)kBM * PS + 2 * kBM : 0);
+                const float2* ml_src = reinterpret_cast<const float2*>(
+                    REP > 1 ? rows_src + (size_t)RB * PS : reinterpret_cast<const float*>(base_ptr) + (size_t)kBM * PS);
+                const uint32_t recv = base + (uint32_t)(Cfg::kQBytes + 2 * S * Cfg::kTileBytes);
+                constexpr int EPLp = D / 32;
+                if (run)
+                    for (int r = warp - Cfg::kRoleWarps; r < rows_t; r += 4) {
+                        const uint32_t dst = map_to_cta(recv + (uint32_t)(((r / splits) * splits + split) * PS * 4), (uint32_t)(r % splits));
+                        const float* src = rows_src + (size_t)r * PS + lane * EPLp;
+                        if (EPLp == 4) {
+                            const float4 o = *reinterpret_cast<const float4*>(src);
+                            st_cluster_f4(dst + (uint32_t)(lane * EPLp * 4), o.x, o.y, o.z, o.w);
+                        } else {
+                            const float2 o = *reinterpret_cast<const float2*>(src);
+                            st_cluster_f2(dst + (uint32_t)(lane * EPLp * 4), o.x, o.y);
+                        }
+                        if (lane == 0) st_cluster_f2(dst + (uint32_t)(D * 4), ml_src[r].x, ml_src[r].y);
+                    }
+            }
         } else if (warp_active && run) {
             const bool direct = prm.mode == kModeDirect;  // REP == 1 then
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
@@ -726,7 +764,49 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         tc_fence_before();
     }
 
-    if (prm.mode == kModeCluster) {
+    if (PUSH && prm.mode == kModeCluster) {
+        // ---- every split's partial of this CTA's rows (rank, rank + splits, ...) has been stored into its receive area
+        __syncwarp();
+        cluster_sync_all();
+        const bool run = (flags | *bad_s) == 0;
+        const uint32_t rank = cluster_ctarank();
+        const float* recv = reinterpret_cast<const float*>(base_ptr + Cfg::kQBytes + 2 * S * Cfg::kTileBytes);
+        constexpr int EPL = D / 32;
+        const int rows = rows_in(0);
+        if (run)
+            for (int k = warp; (int)rank + splits * k < rows; k += Cfg::kThreads / 32) {
+                const int lr = (int)rank + splits * k;
+                const float* prow = recv + (size_t)k * splits * PS;
+                float2 ml = make_float2(-INFINITY, 0.f);
+                if (lane < splits) ml = *reinterpret_cast<const float2*>(prow + (size_t)lane * PS + D);
+                float M = ml.x;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                const float f_mine = lane < splits ? exp2f(ml.x - M) : 0.f;
+                float den = f_mine * ml.y;  // fixed (butterfly) order: the same on every run
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+                float num[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int i = 0; i < splits; ++i) {  // split order
+                    const float f = __shfl_sync(0xffffffffu, f_mine, i);
+                    const float* src = prow + (size_t)i * PS + lane * EPL;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) num[e] = fmaf(f, src[e], num[e]);
+                }
+                const int gr = mt0 * kBM + lr;
+                const float inv = ((gr % T) < n && den > 0.f) ? 1.f / den : 0.f;
+                __nv_bfloat16* dst = prm.out + ((size_t)(b * prm.Hq + hk * G) * T + gr) * D + lane * EPL;
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
+                if (EPL == 4) {
+                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[2] * inv, num[3] * inv);
+                    *reinterpret_cast<uint2*>(dst) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                } else {
+                    *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(&h0);
+                }
+            }
+        __syncthreads();  // warp 1 frees the tensor memory below: every warp is done
+    } else if (prm.mode == kModeCluster) {
         // ---- merge the splits (and copies) through distributed shared memory: this CTA owns the output rows
         //      rank, rank + splits, ... of every row tile; one warp per row, lane i first fetches (offset, sum) of
         //      partial i, then every lane gathers its 4 (d = 64: 2) output columns from all partials, 8 loads in flight
@@ -904,14 +984,14 @@ size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
                                              256);
 }
 
-template <int D, int NM, int REP, int TC>
+template <int D, int NM, int REP, int TC, int PUSH>
 static s4c_status launch_tc(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
-    using Cfg = TcCfg<D, NM, TC>;
+    using Cfg = TcCfg<D, NM, TC, PUSH>;
     static bool configured[64] = {};  // the opt-ins (dynamic shared memory, cluster size) are per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP, TC, PUSH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return S4C_ERR_CUDA;
         configured[dev] = true;
@@ -940,7 +1020,7 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
     }
     cfg.attrs = attrs;
     cfg.numAttrs = na;
-    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP, TC>, mq, mk, mv, prm) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP, TC, PUSH>, mq, mk, mv, prm) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
@@ -965,18 +1045,20 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     prm.q_box_rows = R >= kBM ? kBM : (int)round_up((size_t)R, 8);
     prm.scale_log2 = scale * 1.4426950408889634f;
     s4c_status st;
-    if (d == 128)
-        st = nm == 2      ? launch_tc<128, 2, 1, 1>(q, k, v, prm, B, stream)
-             : rep == 4   ? launch_tc<128, 1, 4, 1>(q, k, v, prm, B, stream)
-             : rep == 2   ? launch_tc<128, 1, 2, 1>(q, k, v, prm, B, stream)
-             : turns == 2 ? launch_tc<128, 1, 1, 2>(q, k, v, prm, B, stream)
-                          : launch_tc<128, 1, 1, 1>(q, k, v, prm, B, stream);
-    else
-        st = nm == 2      ? launch_tc<64, 2, 1, 1>(q, k, v, prm, B, stream)
-             : rep == 4   ? launch_tc<64, 1, 4, 1>(q, k, v, prm, B, stream)
-             : rep == 2   ? launch_tc<64, 1, 2, 1>(q, k, v, prm, B, stream)
-             : turns == 2 ? launch_tc<64, 1, 1, 2>(q, k, v, prm, B, stream)
-                          : launch_tc<64, 1, 1, 1>(q, k, v, prm, B, stream);
+    // pushed partials (see the kernel): few rows, few tiles per CTA -- where the end of a launch, not its streaming, decides
+    const int tiles_per_cta = ceil_div(ceil_div(C, kBN), prm.splits);
+    const bool push = prm.mode == kModeCluster && nm == 1 && turns == 1 && tiles_per_cta <= 16 &&
+                      ceil_div(R, prm.splits) * prm.splits * (d + 4) * 4 <= 32768;
+#define S4C_TC_DISPATCH(DD)                                                                    \
+    (nm == 2      ? launch_tc<DD, 2, 1, 1, 0>(q, k, v, prm, B, stream)                          \
+     : turns == 2 ? launch_tc<DD, 1, 1, 2, 0>(q, k, v, prm, B, stream)                          \
+     : rep == 4   ? (push ? launch_tc<DD, 1, 4, 1, 1>(q, k, v, prm, B, stream)                  \
+                          : launch_tc<DD, 1, 4, 1, 0>(q, k, v, prm, B, stream))                 \
+     : rep == 2   ? (push ? launch_tc<DD, 1, 2, 1, 1>(q, k, v, prm, B, stream)                  \
+                          : launch_tc<DD, 1, 2, 1, 0>(q, k, v, prm, B, stream))                 \
+                  : launch_tc<DD, 1, 1, 1, 0>(q, k, v, prm, B, stream)) /* more than 64 rows never fit the receive area */
+    st = d == 128 ? S4C_TC_DISPATCH(128) : S4C_TC_DISPATCH(64);
+#undef S4C_TC_DISPATCH
     if (st != S4C_OK) return st;
     if (prm.mode == kModeWorkspace)
         return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits * rep * turns, S4C_BF16,
