@@ -43,9 +43,13 @@ struct TcCfg {
     static constexpr int kHalves = D / 64;           // 64-element (128-byte) swizzle atoms along d
     static constexpr int kQBytes = kBM * D * 2;      // one row tile of Q: 32 KB (d = 128)
     static constexpr int kTileBytes = kBN * D * 2;   // 16 KB: one K or V tile
-    // PUSH: 32 KB at the end of the tile area are set aside to receive the other splits' partials (see the kernel)
-    static constexpr int kRecvBytes = PUSH ? 32768 : 0;
-    static constexpr int kStages = (D == 128 ? (NM == 1 ? 6 : 5) : 8) - kRecvBytes / (2 * kTileBytes);
+    // PUSH == 1: 32 KB at the end of the tile area are set aside to receive the other splits' partials (see the kernel)
+    // PUSH == 2: half an SM per CTA (two K/V stages at d = 128), so that two CTAs of a grid of several waves share an
+    //            SM and one streams while the other starts or finishes
+    static constexpr int kRecvBytes = PUSH == 1 ? 32768 : 0;
+    static constexpr int kCtasPerSm = PUSH == 2 ? 2 : 1;
+    static constexpr int kStages =
+        PUSH == 2 ? (D == 128 ? 2 : 4) : (D == 128 ? (NM == 1 ? 6 : 5) : 8) - kRecvBytes / (2 * kTileBytes);
     static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes + kRecvBytes;
     static constexpr int kScoreBufs = 2 * TC;         // TMEM score buffers per row tile (two per softmax group)
     static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM;
@@ -56,7 +60,7 @@ struct TcCfg {
     static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
     static constexpr int kTmemCols = NM * kScoreBufs * kBN + NM * TC * D <= 256 ? 256 : 512;
     static_assert(kNumBars * 8 <= 480, "barrier area");
-    static_assert(kPartBytes <= kSmemData, "parked partials reuse the tile buffers");
+    static_assert(PUSH == 2 || kPartBytes <= kSmemData, "parked partials reuse the tile buffers (half-SM CTAs never merge)");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
@@ -303,12 +307,12 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, 
 // (copy-merged) rows into a receive area of the row's owner that is used for nothing else, so no barrier has to say
 // "my tile buffers are dead" first; after one cluster barrier the owner merges from its own shared memory and leaves.
 template <int D, int NM, int REP, int TC, int PUSH>
-__global__ void __launch_bounds__(TcCfg<D, NM, TC, PUSH>::kThreads, 1)
+__global__ void __launch_bounds__(TcCfg<D, NM, TC, PUSH>::kThreads, TcCfg<D, NM, TC, PUSH>::kCtasPerSm)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const TcParams prm) {
     static_assert(NM == 1 || REP == 1, "row copies only with a single row tile");
     static_assert(TC == 1 || (NM == 1 && REP == 1), "turns only with a single row tile and no row copies");
-    static_assert(PUSH == 0 || (NM == 1 && TC == 1), "pushed partials only with a single row tile and no turns");
+    static_assert(PUSH == 0 || (NM == 1 && TC == 1), "pushed partials and half-SM CTAs only with a single row tile and no turns");
     using Cfg = TcCfg<D, NM, TC, PUSH>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
@@ -665,12 +669,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (REP > 1) {
                 // The copies of a row are merged here, inside the CTA, before the splits are merged across the
                 // cluster: distributed shared memory moves only ~16 bytes per clock and SM, so it should carry one
-                // partial per split and row, not REP.  Merged rows go behind the parked ones.
+                // partial per split and row, not REP.  The merged row replaces copy 0's parked row (the warp that
+                // merges row r is the only one that touches its copies).
                 named_bar_sync(1, 128);
-                const float* pin = reinterpret_cast<const float*>(base_ptr);
-                const float2* pml_in = reinterpret_cast<const float2*>(pin + (size_t)kBM * PS);
-                float* mout = reinterpret_cast<float*>(base_ptr) + (size_t)kBM * PS + 2 * kBM;
-                float2* mml = reinterpret_cast<float2*>(mout + (size_t)RB * PS);
+                float* pin = reinterpret_cast<float*>(base_ptr);
+                float2* pml_in = reinterpret_cast<float2*>(pin + (size_t)kBM * PS);
+                float* mout = pin;
+                float2* mml = pml_in;
                 constexpr int EPLm = D / 32;
                 for (int r = warp - Cfg::kRoleWarps; r < rows_t; r += 4) {
                     float mc[REP], M = -INFINITY;
@@ -687,21 +692,21 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                         for (int e = 0; e < EPLm; ++e) num[e] = fmaf(f, src[e], num[e]);
                     }
+                    __syncwarp();  // every lane has read the copies' (offset, sum) before lane 0 overwrites copy 0's
 #pragma unroll
                     for (int e = 0; e < EPLm; ++e) mout[(size_t)r * PS + lane * EPLm + e] = num[e];
                     if (lane == 0) mml[r] = make_float2(M, den);
                 }
             }
-            if (PUSH) {
+            if (PUSH == 1) {
                 // this CTA's (copy-merged) partial of row r goes to CTA r % splits, slot (r / splits) * splits + split
                 // of its receive area: 32 lanes x 16 (d = 64: 8) bytes per row, (offset, sum) into the row's padding
                 if (REP > 1)
                     __syncwarp();  // a warp pushes the rows it merged itself
                 else
                     named_bar_sync(1, 128);  // rows were parked one per thread
-                const float* rows_src = reinterpret_cast<const float*>(base_ptr) + (REP > 1 ? (size_t)kBM * PS + 2 * kBM : 0);
-                const float2* ml_src = reinterpret_cast<const float2*>(
-                    REP > 1 ? rows_src + (size_t)RB * PS : reinterpret_cast<const float*>(base_ptr) + (size_t)kBM * PS);
+                const float* rows_src = reinterpret_cast<const float*>(base_ptr);  // parked, or merged in place
+                const float2* ml_src = reinterpret_cast<const float2*>(rows_src + (size_t)kBM * PS);
                 const uint32_t recv = base + (uint32_t)(Cfg::kQBytes + 2 * S * Cfg::kTileBytes);
                 constexpr int EPLp = D / 32;
                 if (run)
@@ -764,7 +769,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         tc_fence_before();
     }
 
-    if (PUSH && prm.mode == kModeCluster) {
+    if (PUSH == 1 && prm.mode == kModeCluster) {
         // ---- every split's partial of this CTA's rows (rank, rank + splits, ...) has been stored into its receive area
         __syncwarp();
         cluster_sync_all();
@@ -814,9 +819,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         cluster_sync_all();
         const bool run = (flags | *bad_s) == 0;  // the same in every CTA of the cluster: it depends on the sequence only
         const uint32_t rank = cluster_ctarank();
-        // row copies were merged inside their CTA (rows behind the parked ones); turns are merged here with the splits
-        const uint32_t part = REP > 1 ? base + (uint32_t)((kBM * PS + 2 * kBM) * 4) : base;
-        const uint32_t part_ml = REP > 1 ? part + (uint32_t)(RB * PS * 4) : base + (uint32_t)(NM * TC * kBM * PS * 4);
+        // row copies were merged inside their CTA (into copy 0's rows); turns are merged here with the splits
+        const uint32_t part = base, part_ml = base + (uint32_t)(NM * TC * kBM * PS * 4);
         constexpr int EPL = D / 32;  // output elements per lane
         constexpr int NC = TC;       // partials per split
         const int np = splits * NC;  // partials per output row (<= 16)
@@ -939,12 +943,14 @@ static int tc_m_tiles(int T, int Hq, int Hkv) { return ceil_div((Hq / Hkv) * T, 
 static int tc_nm(int T, int Hq, int Hkv) { return tc_m_tiles(T, Hq, Hkv) > 1 ? 2 : 1; }
 static int tc_m_groups(int T, int Hq, int Hkv) { return ceil_div(tc_m_tiles(T, Hq, Hkv), tc_nm(T, Hq, Hkv)); }
 
-// Number of splits of the cache: the smallest count that minimises (waves of one-CTA-per-SM work) / splits, with a
-// small charge per extra split for the merge; a split has at least two tiles.  Up to 8 splits merge inside a
-// cluster; a grid too small to fill the GPU even with 8 goes wider and merges through the workspace.
+// Number of splits of the cache: the count that minimises waves x (fixed cost of a CTA + its tiles), with a small
+// charge per extra split for the merge; a split has at least two tiles.  The fixed cost (set-up, first tile's latency,
+// merge, measured at 5-6 us) is worth about ten tiles.  Up to 8 splits merge inside a cluster; a grid too small to
+// fill the GPU even with 8 goes wider and merges through the workspace.
 static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
     const int base = B * Hkv * tc_m_groups(T, Hq, Hkv);
-    int max_by_len = ceil_div(C, kBN) / 2;
+    const int tiles = ceil_div(C, kBN);
+    int max_by_len = tiles / 2;
     if (max_by_len < 1) max_by_len = 1;
     if (base * kMaxClusterSplits * 2 <= 148) {  // tiny grids: fill one wave through the workspace path
         int s = 148 / base;
@@ -956,7 +962,7 @@ static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
     for (int s = 1; s <= kMaxClusterSplits && s <= max_by_len; ++s) {
         const int resident = s == 1 ? 148 : 8 * (18 / s) * s;  // clusters do not straddle the 8 GPCs (18+ SMs each)
         const double waves = (double)ceil_div(base * s, resident);
-        const double cost = waves / s * (1.0 + 0.03 * (s - 1));
+        const double cost = waves * (10.0 + ceil_div(tiles, s)) * (1.0 + 0.03 * (s - 1));
         if (cost < best_cost - 1e-12) best_cost = cost, best = s;
     }
     return best;
@@ -1049,8 +1055,13 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     const int tiles_per_cta = ceil_div(ceil_div(C, kBN), prm.splits);
     const bool push = prm.mode == kModeCluster && nm == 1 && turns == 1 && tiles_per_cta <= 16 &&
                       ceil_div(R, prm.splits) * prm.splits * (d + 4) * 4 <= 32768;
+    // half-SM CTAs: grids of at least two CTAs per SM that need no merge
+    const bool half = prm.splits == 1 && nm == 1 && turns == 1 && B * Hkv * prm.m_groups >= 2 * 148;
 #define S4C_TC_DISPATCH(DD)                                                                    \
-    (nm == 2      ? launch_tc<DD, 2, 1, 1, 0>(q, k, v, prm, B, stream)                          \
+    (half         ? (rep == 4   ? launch_tc<DD, 1, 4, 1, 2>(q, k, v, prm, B, stream)            \
+                     : rep == 2 ? launch_tc<DD, 1, 2, 1, 2>(q, k, v, prm, B, stream)            \
+                                : launch_tc<DD, 1, 1, 1, 2>(q, k, v, prm, B, stream))           \
+     : nm == 2    ? launch_tc<DD, 2, 1, 1, 0>(q, k, v, prm, B, stream)                          \
      : turns == 2 ? launch_tc<DD, 1, 1, 2, 0>(q, k, v, prm, B, stream)                          \
      : rep == 4   ? (push ? launch_tc<DD, 1, 4, 1, 1>(q, k, v, prm, B, stream)                  \
                           : launch_tc<DD, 1, 4, 1, 0>(q, k, v, prm, B, stream))                 \

@@ -95,3 +95,9 @@ def test_full_row_tile_with_two_softmax_groups_taking_turns(d):
     _case(B=2, Hq=16, Hkv=8, T=50, d=d, Ls=[5000, 4321], dtype="bf16", seed=12, n_nodes=[50, 33])
     # ... and through the workspace when the grid is too small for clusters
     _case(B=1, Hq=4, Hkv=4, T=100, d=d, Ls=[20000], dtype="bf16", seed=13)
+
+
+@pytest.mark.parametrize("T", [20, 50, 100])
+def test_grids_of_several_waves_share_an_sm_between_two_ctas(T):
+    # 320 CTAs on 148 SMs: the launch takes the half-SM configuration (with 4, 2 and no row copies)
+    _case(B=10, Hq=32, Hkv=32, T=T, d=128, Ls=[300, 17, 0, 640, 129, 300, 64, 511, 1, 77], dtype="bf16", seed=21 + T)
