@@ -69,7 +69,10 @@ def peaks():
 # under profiles/ (the file named here).  It only describes the kernel it was taken on: the value is reported while
 # the kernel source still has the recorded hash, otherwise null.
 NCU_TRAFFIC = {
-    "c2x32": dict(bytes=None, sha256="", profile="profiles/tree_attention_tc_c2x32_ncu_full.md"),
+    "c2x32": dict(bytes=18114816, sha256="5e21b2aae631293d69434b0a8765523dd49f3f44e3469c6dce069964dac636d1",
+                  profile="profiles/tree_attention_tc_c2x32_ncu_full.md"),
+    "c4x32": dict(bytes=72254464, sha256="5e21b2aae631293d69434b0a8765523dd49f3f44e3469c6dce069964dac636d1",
+                  profile="profiles/tree_attention_tc_c4x32_ncu_full.md"),
 }
 
 
