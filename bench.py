@@ -237,8 +237,13 @@ def build_step(cfg, temperature, device, seed_shift=0):
     x = W.make_accept_inputs(cfg_gen, parent, temperature, token_mode="topk")
     kv_bytes = 2 * cfg.n_layers * cfg.B * cfg.Hkv * cfg.C * cfg.d * (2 if cfg.dtype == "bf16" else 4)
     on_device = kv_bytes > (1 << 30)
-    qs, ks, vs = [], [], []
     dt = {"f32": torch.float32, "bf16": torch.bfloat16}[cfg.dtype]
+    # every layer's tensors are views of three big ones (still an independent cache per layer): the host-buffer leg
+    # then needs three copies per step, not three per layer
+    q_all = torch.empty((cfg.n_layers, cfg.B, cfg.Hq, cfg.T, cfg.d), dtype=dt, device=device)
+    k_all = torch.empty((cfg.n_layers, cfg.B, cfg.Hkv, cfg.C, cfg.d), dtype=dt, device=device)
+    v_all = torch.empty((cfg.n_layers, cfg.B, cfg.Hkv, cfg.C, cfg.d), dtype=dt, device=device)
+    qs, ks, vs = list(q_all.unbind(0)), list(k_all.unbind(0)), list(v_all.unbind(0))
     for l in range(cfg.n_layers):
         if on_device:  # very large sweeps: draw the caches on the device (values are N(0,1) either way)
             g = torch.Generator(device=device).manual_seed(W.stream_seed(cfg_gen.config_id, "kv", l))
@@ -247,13 +252,14 @@ def build_step(cfg, temperature, device, seed_shift=0):
             v = torch.randn((cfg.B, cfg.Hkv, cfg.C, cfg.d), generator=g, device=device).to(dt)
         else:
             q, k, v = (t.to(device) for t in W.make_attention_inputs(cfg_gen, l))
-        qs.append(q), ks.append(k), vs.append(v)
+        qs[l].copy_(q), ks[l].copy_(k), vs[l].copy_(v)
+        del q, k, v
     to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
     stoch = temperature > 0
     step = VerifyStep(qs, ks, vs, torch.full((cfg.B,), cfg.L, dtype=torch.int32, device=device), to(parent),
                       to(x["tokens"]), to(x["logits"]), to(x["draft_probs"]) if stoch else None,
                       to(x["uniforms"]) if stoch else None, temperature, cfg.max_depth,
-                      feat_in=W.make_features(cfg_gen).to(device))
+                      feat_in=W.make_features(cfg_gen).to(device), stacked=(q_all, k_all, v_all))
     return step
 
 

@@ -20,7 +20,11 @@ class VerifyStep:
     def __init__(self, q: List[torch.Tensor], k_caches: List[torch.Tensor], v_caches: List[torch.Tensor],
                  cache_len: torch.Tensor, parent: torch.Tensor, tokens: torch.Tensor, target_logits: torch.Tensor,
                  draft_probs: Optional[torch.Tensor], uniforms: Optional[torch.Tensor], temperature: float,
-                 max_depth: int, n_nodes: Optional[torch.Tensor] = None, feat_in: Optional[torch.Tensor] = None):
+                 max_depth: int, n_nodes: Optional[torch.Tensor] = None, feat_in: Optional[torch.Tensor] = None,
+                 stacked: Optional[tuple] = None):
+        """``stacked`` = (q_all [n_layers,B,Hq,T,d], k_all, v_all [n_layers,B,Hkv,C,d]) when the per-layer tensors are
+        views of three big ones: the host-buffer path then moves a step's inputs with three copies instead of three
+        per layer."""
         self.n_layers = len(q)
         assert len(k_caches) == self.n_layers and len(v_caches) == self.n_layers
         self.q, self.k_caches, self.v_caches = q, k_caches, v_caches
@@ -53,6 +57,7 @@ class VerifyStep:
         self.ws_accept = torch.empty(max(1, s4c.tree_accept_workspace_bytes(B, T, V)), dtype=torch.uint8, device=dev)
         self.k_ptrs = s4c.cache_pointer_array(k_caches)
         self.v_ptrs = s4c.cache_pointer_array(v_caches)
+        self.stacked = stacked
         self.graph: Optional[torch.cuda.CUDAGraph] = None
         self._host = None
 
@@ -93,7 +98,9 @@ class VerifyStep:
     # ------------------------------------------------------------------ CUDA graph
     def capture(self, what: str = "step") -> torch.cuda.CUDAGraph:
         fn = {"step": self.run, "attention": self.attention, "accept": self.accept,
-              "compact": lambda: (self.reset_lengths(), self.compact())}[what]
+              "compact": lambda: (self.reset_lengths(), self.compact()),
+              "head": lambda: (self.reset_lengths(), self.attention()),
+              "tail": lambda: (self.accept(), self.compact())}[what]
         s = torch.cuda.Stream()
         s.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(s):
@@ -119,9 +126,13 @@ class VerifyStep:
         L = int(self.cache_len0.max().item())
         assert int(self.cache_len0.min().item()) == L, "run_host expects one committed length for the batch"
         T = self.T
-        inp = dict(q=[pin(t) for t in self.q],
-                   k_tree=[pin(c[:, :, L:L + T]) for c in self.k_caches],
-                   v_tree=[pin(c[:, :, L:L + T]) for c in self.v_caches],
+        if self.stacked is not None:  # one pinned buffer per kind for all layers
+            q_all, k_all, v_all = self.stacked
+            layers = dict(q=[pin(q_all)], k_tree=[pin(k_all[:, :, :, L:L + T])], v_tree=[pin(v_all[:, :, :, L:L + T])])
+        else:
+            layers = dict(q=[pin(t) for t in self.q], k_tree=[pin(c[:, :, L:L + T]) for c in self.k_caches],
+                          v_tree=[pin(c[:, :, L:L + T]) for c in self.v_caches])
+        inp = dict(**layers,
                    parent=pin(self.parent), tokens=pin(self.tokens), logits=pin(self.logits))
         if self.draft_probs is not None:
             inp["draft_probs"] = pin(self.draft_probs)
@@ -132,6 +143,9 @@ class VerifyStep:
                    cache_len=pin(self.cache_len), status=pin(self.status_accept))
         self._host = (inp, out, L)
         nbytes = lambda x: sum(t.numel() * t.element_size() for t in (x if isinstance(x, list) else [x]))
+        if self.graph is not None:  # the step as two graphs, so that the second half of the inputs can arrive meanwhile
+            self._side_stream = torch.cuda.Stream()
+            self.graph_head, self.graph_tail = self.capture("head"), self.capture("tail")
         self.h2d_bytes = sum(nbytes(v) for v in inp.values())
         self.d2h_bytes = sum(nbytes(v) for v in out.values())
         return inp, out
@@ -140,19 +154,37 @@ class VerifyStep:
         """Copy the per-step inputs in (async, pinned), run the step, copy the decision back, and wait for it."""
         inp, out, L = self._host
         T = self.T
-        for l in range(self.n_layers):
-            self.q[l].copy_(inp["q"][l], non_blocking=True)
-            self.k_caches[l][:, :, L:L + T].copy_(inp["k_tree"][l], non_blocking=True)
-            self.v_caches[l][:, :, L:L + T].copy_(inp["v_tree"][l], non_blocking=True)
+        if self.stacked is not None:
+            q_all, k_all, v_all = self.stacked
+            q_all.copy_(inp["q"][0], non_blocking=True)
+            k_all[:, :, :, L:L + T].copy_(inp["k_tree"][0], non_blocking=True)
+            v_all[:, :, :, L:L + T].copy_(inp["v_tree"][0], non_blocking=True)
+        else:
+            for l in range(self.n_layers):
+                self.q[l].copy_(inp["q"][l], non_blocking=True)
+                self.k_caches[l][:, :, L:L + T].copy_(inp["k_tree"][l], non_blocking=True)
+                self.v_caches[l][:, :, L:L + T].copy_(inp["v_tree"][l], non_blocking=True)
         self.parent.copy_(inp["parent"], non_blocking=True)
-        self.tokens.copy_(inp["tokens"], non_blocking=True)
-        self.logits.copy_(inp["logits"], non_blocking=True)
-        if self.draft_probs is not None:
-            self.draft_probs.copy_(inp["draft_probs"], non_blocking=True)
-            self.uniforms.copy_(inp["uniforms"], non_blocking=True)
-        if self.feat_in is not None:
-            self.feat_in.copy_(inp["feat_in"], non_blocking=True)
-        if self.graph is not None:
+        split = self.graph is not None and getattr(self, "graph_head", None) is not None
+        main = torch.cuda.current_stream()
+        # what only acceptance and compaction read (logits, draft probabilities, ...) travels on a second stream while
+        # the attention layers run; the tail of the step waits for it
+        side = self._side_stream if split else main
+        if split:
+            side.wait_stream(main)
+        with torch.cuda.stream(side):
+            self.tokens.copy_(inp["tokens"], non_blocking=True)
+            self.logits.copy_(inp["logits"], non_blocking=True)
+            if self.draft_probs is not None:
+                self.draft_probs.copy_(inp["draft_probs"], non_blocking=True)
+                self.uniforms.copy_(inp["uniforms"], non_blocking=True)
+            if self.feat_in is not None:
+                self.feat_in.copy_(inp["feat_in"], non_blocking=True)
+        if split:
+            self.graph_head.replay()
+            main.wait_stream(side)
+            self.graph_tail.replay()
+        elif self.graph is not None:
             self.graph.replay()
         else:
             self.run()
