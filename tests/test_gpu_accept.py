@@ -113,3 +113,12 @@ def test_greedy_ties_take_the_lowest_index():
     x["logits"][:] = np.round(x["logits"])  # many exact ties in every row
     got, ref = accept_both(x, parent, 0.0, max_depth=cfg.max_tree_depth)
     assert assert_accept_equal(got, ref, False) == 0
+
+
+@pytest.mark.parametrize("B,T,tau", [(16, 128, 1.0), (16, 64, 0.0), (4, 32, 0.7)])
+def test_sweep_sized_batches_match_bit_for_bit(B, T, tau):
+    # the acceptance problem of the full-depth sweep at its largest batch: V = 32000, trees of depth <= 8; 65 M logits take
+    # the segment kernels, the smaller ones the row-in-registers clusters
+    cfg, parent, x = _synthetic(B, T, 32000, seed=B + T, sigma=3.0, tau=max(tau, 0.5), mode="topk", max_tree_depth=8)
+    got, ref = accept_both(x, parent, tau, max_depth=cfg.max_tree_depth)
+    assert assert_accept_equal(got, ref, tau > 0) == 0

@@ -101,3 +101,45 @@ def test_full_row_tile_with_two_softmax_groups_taking_turns(d):
 def test_grids_of_several_waves_share_an_sm_between_two_ctas(T):
     # 320 CTAs on 148 SMs: the launch takes the half-SM configuration (with 4, 2 and no row copies)
     _case(B=10, Hq=32, Hkv=32, T=T, d=128, Ls=[300, 17, 0, 640, 129, 300, 64, 511, 1, 77], dtype="bf16", seed=21 + T)
+
+
+def _sampled_heads_case(B, Hq, Hkv, T, L, seed, kv_heads, seqs):
+    """The launch runs at full size (the grid, splits and kernel variant the benchmark times); the oracle checks the
+    sampled (sequence, KV head) pairs, all their query heads and all their tree nodes, element by element."""
+    from paper_2506_14158_b200 import s4c
+    import oracle
+
+    d, G = 128, Hq // Hkv
+    C = (L + T + 127) // 128 * 128
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    q = torch.randn((B, Hq, T, d), generator=g, device="cuda").bfloat16()
+    k = torch.randn((B, Hkv, C, d), generator=g, device="cuda").bfloat16()
+    v = torch.randn((B, Hkv, C, d), generator=g, device="cuda").bfloat16()
+    rng = np.random.default_rng(seed)
+    parent = np.stack([W.random_tree(T, 8, rng) for _ in range(B)])
+    cl = np.full(B, L, dtype=np.int32)
+    status = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    out = s4c.tree_attention(q, k, v, torch.from_numpy(cl).cuda(), torch.from_numpy(parent).cuda(), status=status)
+    torch.cuda.synchronize()
+    assert (status.cpu().numpy() == 0).all()
+    assert torch.isfinite(out.float()).all()
+    worst = 0.0
+    for b in seqs:
+        for hk in kv_heads:
+            qs = q[b:b + 1, hk * G:(hk + 1) * G].cpu()
+            ks, vs = k[b:b + 1, hk:hk + 1].cpu(), v[b:b + 1, hk:hk + 1].cpu()
+            ref, st = oracle.tree_attention(W.to_f64(qs), W.to_f64(ks), W.to_f64(vs), cl[b:b + 1], parent[b:b + 1])
+            got = out[b:b + 1, hk * G:(hk + 1) * G].double().cpu().numpy()
+            worst = max(worst, float(np.abs(got - ref).max()))
+    assert worst <= ATTN_TOL["bf16"], f"max-abs error {worst:.3e}"
+
+
+@pytest.mark.parametrize("name,B,Hq,Hkv,T,L,kv_heads,seqs", [
+    ("sweep B1 T64 L32768: 4 splits in a cluster, 2 row copies", 1, 32, 32, 64, 32768, [0, 13, 31], [0]),
+    ("sweep B1 T128 L32768: two softmax groups taking turns", 1, 32, 32, 128, 32768, [5, 31], [0]),
+    ("sweep B16 T32 L4096: half-SM CTAs, 512 CTAs", 16, 32, 32, 32, 4096, [0, 17], [0, 9, 15]),
+    ("sweep B4 T16 L8192: one split, 4 row copies", 4, 32, 32, 16, 8192, [3, 30], [1, 3]),
+    ("8B shape at L16384: GQA, two row tiles per CTA", 4, 32, 8, 64, 16384, [0, 7], [0, 3]),
+])
+def test_full_size_launch_configurations_on_sampled_heads(name, B, Hq, Hkv, T, L, kv_heads, seqs):
+    _sampled_heads_case(B, Hq, Hkv, T, L, seed=len(name), kv_heads=kv_heads, seqs=seqs)
