@@ -137,9 +137,7 @@ __device__ __forceinline__ double exp_nonpos(double t, const double* tab /* shar
 // exp_nonpos without the range test, for -700 < t <= 0.  The statistics kernels raise every logit to at least
 // M - 690 tau first (one float max): a term that small is below 1e-299 of the row sum either way, so neither the sum
 // nor the residual mass can tell the difference, and the inner loop loses a compare and a branch per element.
-// `tab32` is a copy of the table with every entry repeated once per lane (entry j of lane l at [j * 32 + l]): the 32
-// lanes of a warp then always read 32 different banks pairs, whatever entries they need.
-__device__ __forceinline__ double exp_fast(double t, const double* tab32) {
+__device__ __forceinline__ double exp_fast(double t, const double* tab) {
     const double z = fma(t, 0x1.71547652b82fep+5, 6755399441055744.0);
     const int k = __double2loint(z);
     const double kd = z - 6755399441055744.0;
@@ -151,13 +149,13 @@ __device__ __forceinline__ double exp_fast(double t, const double* tab32) {
     pl = fma(pl, r, 0.5);
     pl = fma(pl, r, 1.0);
     pl = pl * r;
-    const double tj = tab32[((k & 31) << 5) + (threadIdx.x & 31)];
+    const double tj = tab[k & 31];
     const double y = fma(tj, pl, tj);
     return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));
 }
 constexpr float kExpFloorSpan = 690.f;  // in units of tau
-__device__ __forceinline__ void fill_exp_table(double* tab32) {  // every thread of the CTA; the caller synchronises
-    for (int i = threadIdx.x; i < 1024; i += blockDim.x) tab32[i] = kExp2Frac[i >> 5];
+__device__ __forceinline__ void fill_exp_table(double* tab) {  // every thread of the CTA; the caller synchronises
+    if (threadIdx.x < 32) tab[threadIdx.x] = kExp2Frac[threadIdx.x];
 }
 
 // ----------------------------------------------------------------------------- kernel 1
@@ -199,7 +197,7 @@ accept_rowstats_kernel(const float* __restrict__ logits, const int32_t* __restri
     __shared__ float sm[kRowThreads / 32];
     __shared__ int idx_s;
     __shared__ double scratch[33];
-    __shared__ double tab[STOCH ? 1024 : 1];
+    __shared__ double tab[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (STOCH) fill_exp_table(tab);
     if (threadIdx.x == 32) idx_s = INT_MAX;
@@ -273,7 +271,7 @@ accept_residual_kernel(const float* __restrict__ logits, const float* __restrict
     __shared__ NodeStats ns;
     __shared__ int first_tok;
     __shared__ double scratch[33];
-    __shared__ double tab[1024];
+    __shared__ double tab[32];
     fill_exp_table(tab);
     if (threadIdx.x < 32) {
         // the row's statistics from its segments, by one warp: lane s (and s + 32, ...) takes segment s; the maximum
@@ -324,9 +322,10 @@ accept_residual_kernel(const float* __restrict__ logits, const float* __restrict
             const double p = exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab) * invS;
             const double qd = (double)q[k];
             const double r = p - qd;
-            if (r > 0.0) z += r;
+            z += r + fabs(r);  // 2 max(r, 0), exactly; halved below
             qs += qd;
         }
+        z *= 0.5;
     } else {
 #pragma unroll
         for (int k = 0; k < kElemsPerThread; ++k) qs += (double)q[k];
@@ -443,7 +442,7 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     __shared__ ClSlots slot;
     __shared__ double gathered[kCl], gathered2[kCl];
     __shared__ double scratch[33];
-    __shared__ double tab[STOCH ? 1024 : 1];
+    __shared__ double tab[32];
     __shared__ float wm[THREADS / 32];
     __shared__ int wi[THREADS / 32];
     __shared__ int first_tok;
@@ -544,9 +543,10 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     for (int k = 0; k < kClEpt; ++k) {
         const double qd = (double)q[k];
         const double r = e[k] * invS - qd;
-        if (r > 0.0) z += r;
+        z += r + fabs(r);  // 2 max(r, 0), exactly; halved below
         qs += qd;
     }
+    z *= 0.5;
     // the first child's token does not count towards the draft mass that is left: one thread takes it out again
     if (tid == 0 && ft >= c0 && ft < c0 + chunk && ft < V) qs -= (double)__ldg(dprobs + off + ft);
     z = block_sum(z, scratch);
