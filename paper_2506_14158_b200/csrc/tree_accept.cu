@@ -578,7 +578,7 @@ __global__ void __launch_bounds__(STOCH ? 1024 : 128, 1)
 accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
                            const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
                            const int32_t* __restrict__ n_nodes, const float* __restrict__ uniforms, int T, int V,
-                           int chunk, int max_depth, double inv_tau, const NodeSummary* __restrict__ nodes,
+                           int chunk, int cache_p0, int max_depth, double inv_tau, const NodeSummary* __restrict__ nodes,
                            const NodeStats* __restrict__ seg_nodes, const ResPartial* __restrict__ seg_res, int seg_splits,
                            const RowPartial* __restrict__ seg_row, int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
                            int32_t* __restrict__ next_token, uint8_t* __restrict__ near_tie,
@@ -676,6 +676,10 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
     //      only the vocabulary-wide sums are split, CTA `rank` owning the elements [c0, c1)
     const int c0 = (int)rank * chunk, c1 = min(V, c0 + chunk);
     int round = 0;  // cluster-wide reductions so far (selects the slot set)
+    // With room in shared memory the target probabilities of this CTA's vocabulary range at the current node are kept
+    // from the first vocabulary-wide pass there to the later ones (a float64 exp per entry is most of a pass).
+    double* pc = reinterpret_cast<double*>(smem_raw + ((sizeof(WalkClShared) + 15) / 16) * 16);
+    int cached_node = -1;  // node whose probabilities pc[] holds, complete after a whole pass (the same in every thread)
     // two cluster-wide sums in rank order; every thread of the cluster calls this and gets the same values
     auto cluster_sum2 = [&](double a, double bsum, double& A, double& Bs) {
         // both sums through one pair of CTA barriers, each in a fixed order
@@ -708,17 +712,27 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         // (p, q) after r rejections of up to four vocabulary entries start, start + step, ...; the loads go out
         // first (these passes are bound by the latency of the loads, not by their volume)
         auto eval4 = [&](int start, int step, int end, int rr, double (&pv)[4], double (&qv)[4]) {
+            const bool hit = cache_p0 && cached_node == cur;
             float xl[4], ql[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int v = start + u * step;
-                xl[u] = v < end ? __ldg(lrow + v) : 0.f, ql[u] = v < end ? __ldg(qrow + v) : 0.f;
+                xl[u] = (v < end && !hit) ? __ldg(lrow + v) : 0.f, ql[u] = v < end ? __ldg(qrow + v) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int v = start + u * step;
                 pv[u] = 0.0, qv[u] = 0.0;
-                if (v < end) chain_eval(p0_from(xl[u]), (double)ql[u], v, rr, sh, pv[u], qv[u]);
+                if (v < end) {
+                    double p0;
+                    if (hit) {
+                        p0 = pc[v - c0];
+                    } else {
+                        p0 = p0_from(xl[u]);
+                        if (cache_p0) pc[v - c0] = p0;
+                    }
+                    chain_eval(p0, (double)ql[u], v, rr, sh, pv[u], qv[u]);
+                }
             }
         };
         int r = 0, accepted = -1;
@@ -755,6 +769,7 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                     }
                 }
                 cluster_sum2(z, qs, Z, s);
+                cached_node = cur;  // a whole pass at this node is behind a CTA barrier: pc[] is complete
             }
             __syncthreads();  // everyone has finished reading the chain before it grows
             if (tid == 0) {
@@ -794,6 +809,7 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
         if (lane == 0) sh.wsum[warp] = acc, sh.wlast[warp] = last;
         __syncthreads();
+        cached_node = cur;  // the sums above went over the whole range: the scan below reads pc[]
         double* set = cs.slots[round & 1];
         if (tid == 0) {
             double tot = 0.0;
@@ -957,9 +973,23 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
     if (stoch) {
         cfg.gridDim = dim3(kCl, B, 1);
         cfg.blockDim = dim3(1024, 1, 1);
-        cfg.dynamicSmemBytes = sizeof(WalkClShared);
+        // room for the range's probabilities (8 bytes per vocabulary entry of a CTA) next to the walk's state?
+        const size_t walk_state = ((sizeof(WalkClShared) + 15) / 16) * 16;
+        const int cache_p0 = walk_state + (size_t)chunk * 8 <= 200 * 1024 ? 1 : 0;
+        cfg.dynamicSmemBytes = walk_state + (cache_p0 ? (size_t)chunk * 8 : 0);
+        {
+            static bool configured[64] = {};  // the opt-in to more than 48 KB of dynamic shared memory is per device
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
+            if (!configured[dev]) {
+                if (cudaFuncSetAttribute(accept_walk_cluster_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         200 * 1024) != cudaSuccess)
+                    return S4C_ERR_CUDA;
+                configured[dev] = true;
+            }
+        }
         err = cudaLaunchKernelEx(&cfg, accept_walk_cluster_kernel<true>, target_logits, draft_probs, tokens, parent, n_nodes,
-                                 uniforms, T, V, chunk, max_depth, inv_tau, summary, seg_nodes, seg_res, splits, seg_row,
+                                 uniforms, T, V, chunk, cache_p0, max_depth, inv_tau, summary, seg_nodes, seg_res, splits, seg_row,
                                  accept_len, path, next_token, near_tie, status);
         if (err != cudaSuccess) {
             cudaGetLastError();
@@ -967,7 +997,7 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
         }
     } else {
         accept_walk_cluster_kernel<false><<<dim3(1, B), 128, sizeof(WalkClShared), stream>>>(
-            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, max_depth, inv_tau, summary, seg_nodes,
+            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, 0, max_depth, inv_tau, summary, seg_nodes,
             seg_res, splits, seg_row, accept_len, path, next_token, near_tie, status);
         S4C_RETURN_IF_CUDA_ERROR();
     }
