@@ -5,17 +5,18 @@
 // so K/V stream from HBM once per KV head (NM = 2 covers G*T up to 256 rows, the GQA case, with one pass).
 // Warp-specialised:
 //   warp 0        TMA producer: Q once, then K and V tiles of 64 slots into 128B-swizzled shared-memory rings
-//   next 2 x NM   MMA issuers, one warp (one thread) per product and row tile: the QK issuers send S = Q K^T
-//                 (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of two TMEM score buffers of their row
-//                 tile, the PV issuers O += P V (M128 N=d K16 x 4) into its TMEM accumulator; warp 1 owns the
-//                 TMEM allocation
+//   next 2 x NM   MMA issuers, one warp per product and row tile (the loop runs warp-uniformly, so that descriptors
+//                 stay in uniform registers; an elected lane issues): the QK issuers send S = Q K^T
+//                 (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of the TMEM score buffers of their row
+//                 tile, the PV issuers O += P V (M128 N=d K16 x 4, P read from tensor memory) into its TMEM
+//                 accumulator; warp 1 owns the TMEM allocation
 //   then          one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
 //                 tree / tail masking from the row's ancestor bitmask (built from parent[] by the thread
 //                 itself), online softmax in fp32 (base 2; the running offset only moves when the maximum
-//                 grew by more than 2^8, so O in TMEM is rarely rescaled), P rounded to bf16 into swizzled
-//                 shared memory as the A operand of the PV product
+//                 grew by more than 2^8, so O in TMEM is rarely rescaled), P rounded to bf16 back into the score
+//                 buffer in tensor memory, the A operand of the PV product
 // Split-KV without a second launch: the splits of one (sequence, KV head, row-tile group) form a thread-block
-// cluster; every CTA parks its partial (offset, sum, unnormalised O) in its own shared memory and, after a
+// cluster; every CTA parks its partial (offset, sum, normalised O in fp16) in its own shared memory and, after a
 // cluster barrier, CTA r merges the rows r, r + splits, ... of all partials through distributed shared memory
 // in split order (deterministic) and writes the output.  More than 8 splits fall back to a global workspace
 // and the separate combine kernel.
@@ -25,6 +26,7 @@
 // Every mbarrier wait is bounded (200 ms): on expiry the CTA flags S4C_SEQ_TIMEOUT in status[b], stops
 // waiting for anything else, still takes part in the cluster barriers, frees its TMEM and returns.
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <math.h>
 
 #include "s4c_common.cuh"
@@ -51,16 +53,23 @@ struct TcCfg {
     static constexpr int kStages =
         PUSH == 2 ? (D == 128 ? 2 : 4) : (D == 128 ? (NM == 1 ? 6 : 5) : 8) - kRecvBytes / (2 * kTileBytes);
     static constexpr int kSmemData = NM * kQBytes + 2 * kStages * kTileBytes + kRecvBytes;
-    static constexpr int kScoreBufs = 2 * TC;         // TMEM score buffers per row tile (two per softmax group)
+    // TMEM score buffers per row tile: two per softmax group; four where a single group leaves the columns free, so
+    // that a product S = Q K^T need not wait for the P V product two tiles back
+    static constexpr int kScoreBufs = (NM == 1 && TC == 1 && PUSH != 2) ? 4 : 2 * TC;
     static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM;
     static constexpr int kRoleWarps = 1 + 2 * NM;    // TMA warp, then a QK issuer and a PV issuer warp per row tile
     static constexpr int kThreads = 32 * kRoleWarps + 128 * NM * TC;  // ... and four softmax warps per row tile (and turn)
-    static constexpr int kPartStride = D + 4;        // floats per parked row (padding spreads the banks)
+    static constexpr int kPartStride = D + 4;        // floats per parked fp32 row (padding spreads the banks)
     static constexpr int kPartBytes = NM * TC * kBM * kPartStride * 4 + NM * TC * kBM * 8;
+    // A partial travels between the CTAs of a cluster as one exchange row: the normalised output row in fp16 (2^-11
+    // relative, an eighth of the bf16 rounding of the result), then (offset, sum) in fp32, padded to 16 bytes so that
+    // rows 2D + 16 bytes apart spread over the banks.  Half the bytes of fp32 rows on the slow path between SMs.
+    static constexpr int kXRowBytes = 2 * D + 16;
+    static constexpr int kXBytes = NM * TC * kBM * kXRowBytes;
     static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
     static constexpr int kTmemCols = NM * kScoreBufs * kBN + NM * TC * D <= 256 ? 256 : 512;
     static_assert(kNumBars * 8 <= 480, "barrier area");
-    static_assert(PUSH == 2 || kPartBytes <= kSmemData, "parked partials reuse the tile buffers (half-SM CTAs never merge)");
+    static_assert(PUSH == 2 || kPartBytes + kXBytes <= kSmemData, "parked partials reuse the tile buffers (half-SM CTAs never merge)");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
@@ -253,10 +262,61 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
     asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
+__device__ __forceinline__ void st_cluster_u4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint2 ld_cluster_u2(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared::cluster.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_cluster_u1(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared::cluster.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+    const __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ float2 unpack_half2(uint32_t v) { return __half22float2(*reinterpret_cast<const __half2*>(&v)); }
 __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
     float2 v;
     asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
     return v;
+}
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+// ---- packed pairs of floats (one instruction, two lanes of the FP32 pipe) and the three-input maximum
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -291,8 +351,9 @@ struct TcParams {
 
 // Tile range of a split: tiles are dealt out as evenly as whole tiles allow.
 __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, int& t0, int& t1) {
-    t0 = (int)(((long long)n_tiles * split) / splits);
-    t1 = (int)(((long long)n_tiles * (split + 1)) / splits);
+    // (at most 2^25 tiles and 64 splits: the products fit 32 bits, and a 32-bit division is a fraction of a 64-bit one)
+    t0 = (int)(((uint32_t)n_tiles * (uint32_t)split) / (uint32_t)splits);
+    t1 = (int)(((uint32_t)n_tiles * (uint32_t)(split + 1)) / (uint32_t)splits);
 }
 
 // REP > 1 (one row tile, G*T <= 128 / REP rows): the query rows are laid into the 128 MMA rows REP times
@@ -313,10 +374,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     static_assert(NM == 1 || REP == 1, "row copies only with a single row tile");
     static_assert(TC == 1 || (NM == 1 && REP == 1), "turns only with a single row tile and no row copies");
     static_assert(PUSH == 0 || (NM == 1 && TC == 1), "pushed partials and half-SM CTAs only with a single row tile and no turns");
+    static_assert(PUSH != 1 || REP > 1, "partials are pushed by the threads that merged the row copies");
     using Cfg = TcCfg<D, NM, TC, PUSH>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
     constexpr int PS = Cfg::kPartStride;
+    constexpr int XS = Cfg::kXRowBytes;
     constexpr int RB = kBM / REP;  // rows per copy
     constexpr int CW = kBN / REP;  // columns of a tile per copy
     extern __shared__ unsigned char smem_raw[];
@@ -423,22 +486,31 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
         };
         if (nt > 0) {
-            // first pass of the ring, every ring slot still free: lane j requests tile j, the last lane requests Q,
-            // all at once (one thread needs about 50 ns per request)
-            if (lane == 31) {
-                if (REP > 1) {
-                    mbar_expect_tx(BAR(Q_FULL), q_bytes * REP);
-                    for (int c = 0; c < REP; ++c)  // the same rows once per copy, RB rows (whole swizzle atoms) apart
-                        for (int h = 0; h < NH; ++h)
-                            tma_load_2d(sQ + h * (kBM * 128) + c * (RB * 128), &map_q, BAR(Q_FULL), h * 64, q_row0);
+            // Q first (the requests are served in order, and the first product needs it): one request per lane -- a row
+            // copy or row tile, and a 64-column half -- all at once; one thread needs about 50 ns per request
+            if (lane == 0) mbar_expect_tx(BAR(Q_FULL), q_bytes * (REP > 1 ? REP : nm_act));
+            if (REP > 1) {
+                if (lane < REP * NH)  // the same rows once per copy, RB rows (whole swizzle atoms) apart
+                    tma_load_2d(sQ + (lane % NH) * (kBM * 128) + (lane / NH) * (RB * 128), &map_q, BAR(Q_FULL), (lane % NH) * 64, q_row0);
+            } else if (lane < nm_act * NH) {
+                tma_load_2d(sQ + (lane / NH) * Cfg::kQBytes + (lane % NH) * (kBM * 128), &map_q, BAR(Q_FULL), (lane % NH) * 64,
+                            q_row0 + (lane / NH) * kBM);
+            }
+            __syncwarp();
+            // then the first pass of the ring, every ring slot still free: again one request per lane
+            if (lane < 2 * S && (lane >> 1) < nt) {
+                // K and V of a tile on neighbouring lanes: the requests go out as K0 V0 K1 V1 ..., so that the first
+                // product with V does not wait behind every K tile of the ring
+                const int j = lane >> 1, row = kv_row0 + (t0 + j) * kBN;
+                const uint32_t full = BAR(((lane & 1) ? V_FULL : K_FULL) + j);
+                const uint32_t dst = ((lane & 1) ? sV : sK) + j * Cfg::kTileBytes;
+                const CUtensorMap* map = (lane & 1) ? &map_v : &map_k;
+                mbar_expect_tx(full, Cfg::kTileBytes);
+                if (NH == 2) {
+                    tma_load_3d(dst, map, full, 0, row, 0);
                 } else {
-                    mbar_expect_tx(BAR(Q_FULL), q_bytes * nm_act);
-                    for (int t = 0; t < nm_act; ++t)
-                        for (int h = 0; h < NH; ++h)
-                            tma_load_2d(sQ + t * Cfg::kQBytes + h * (kBM * 128), &map_q, BAR(Q_FULL), h * 64, q_row0 + t * kBM);
+                    tma_load_2d(dst, map, full, 0, row);
                 }
-            } else if (lane < S && lane < nt) {
-                load_tile(lane);
             }
             __syncwarp();
             if (lane == 0)
@@ -446,10 +518,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
     } else if (warp <= NM) {
         // ================= QK issuer of row tile t: S = Q K^T =================
-        // (one issuing thread per product and row tile: a single thread spends more time issuing a tile's
-        //  instructions and polling its barriers than the tile takes to arrive)
+        // (one issuing warp per product and row tile: a single thread spends more time issuing a tile's
+        //  instructions and polling its barriers than the tile takes to arrive; the whole warp runs the loop so
+        //  that the descriptor arithmetic is warp-uniform, one elected lane issues)
         const int t = warp - 1;
-        if (lane == 0 && nt > 0 && t < nm_act) {
+        if (nt > 0 && t < nm_act) {
             constexpr uint32_t idesc_qk = instr_desc_bf16(kBM, kBN, false);
             uint64_t a_desc[D / 16];  // the Q operand never moves: one descriptor per K step, made once
 #pragma unroll
@@ -462,34 +535,53 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const uint64_t k_desc = smem_desc_sw128(sK + s * Cfg::kTileBytes, 16, 1024);
                 mbar_wait(S_EMPTY(t, j % NB), ((j / NB) & 1) ^ 1, dead);
                 tc_fence_after();
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)  // the start-address field counts 16-byte units
-                    tc_mma_bf16(TM_S(t, j % NB), a_desc[kk], k_desc + (uint64_t)(((kk >> 2) * (kBN * 128) + (kk & 3) * 32) >> 4),
-                                idesc_qk, kk > 0 ? 1u : 0u);
-                tc_commit(S_FULL(t, j % NB));
-                tc_commit(BAR(K_EMPTY + s));
+                    for (int kk = 0; kk < D / 16; ++kk)  // the start-address field counts 16-byte units
+                        tc_mma_bf16(TM_S(t, j % NB), a_desc[kk], k_desc + (uint64_t)(((kk >> 2) * (kBN * 128) + (kk & 3) * 32) >> 4),
+                                    idesc_qk, kk > 0 ? 1u : 0u);
+                    tc_commit(S_FULL(t, j % NB));
+                    tc_commit(BAR(K_EMPTY + s));
+                }
+                __syncwarp();
             }
         }
     } else if (warp <= 2 * NM) {
         // ================= PV issuer of row tile t: O += P V =================
         const int t = warp - 1 - NM;
-        if (lane == 0 && nt > 0 && t < nm_act) {
+        if (nt > 0 && t < nm_act) {
             constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
                 mbar_wait(BAR(V_FULL + s), it & 1, dead);
+                if ((t0 + j) * kBN + kBN > Ltot) {
+                    // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
+                    // but 0 * NaN would poison O, so those V rows are cleared before the product reads them -- here, by
+                    // the warp that waits for P anyway.  Every row tile's issuer warp clears them (the same zeros): each
+                    // only knows about its own product.
+                    const int first = Ltot - (t0 + j) * kBN;  // 1..63
+                    unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
+                    constexpr int CPR = 8 * NH;  // 16-byte chunks per slot: a lane keeps its chunk and walks down the slots
+                    for (int r = first + lane / CPR; r < kBN; r += 32 / CPR)
+                        *reinterpret_cast<uint4*>(vt + ((lane % CPR) >> 3) * (kBN * 128) + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    fence_async_smem();  // generic-proxy stores, read by the tensor core through the async proxy
+                    __syncwarp();
+                }
                 // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
                 const uint64_t v_desc = smem_desc_sw128(sV + s * Cfg::kTileBytes, kBN * 128, 1024);
                 mbar_wait(P_FULL(t, j % NB), (j / NB) & 1, dead);
                 tc_fence_after();
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk)
-                    // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
-                    tc_mma_bf16_ts(TM_O(t, TC == 2 ? (j & 1) : 0), TM_S(t, j % NB) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4),
-                                   idesc_pv, (j >= TC || kk > 0) ? 1u : 0u);
-                tc_commit(PV_DONE(t, TC == 2 ? (j & 1) : 0));
-                tc_commit(S_EMPTY(t, j % NB));  // the score buffer (and the P inside it) may be overwritten
-                tc_commit(BAR(V_EMPTY + s));
+                    for (int kk = 0; kk < kBN / 16; ++kk)
+                        // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
+                        tc_mma_bf16_ts(TM_O(t, TC == 2 ? (j & 1) : 0), TM_S(t, j % NB) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4),
+                                       idesc_pv, (j >= TC || kk > 0) ? 1u : 0u);
+                    tc_commit(PV_DONE(t, TC == 2 ? (j & 1) : 0));
+                    tc_commit(S_EMPTY(t, j % NB));  // the score buffer (and the P inside it) may be overwritten
+                    tc_commit(BAR(V_EMPTY + s));
+                }
+                __syncwarp();
             }
         }
     } else {
@@ -565,23 +657,33 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         sv[c] = on ? sv[c] : -INFINITY;
                     }
                 }
-                float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};  // four independent chains
+                float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};  // four independent chains, two columns per instruction
 #pragma unroll
-                for (int c = 4; c < CW; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sv[c]);
+                for (int c = 4; c < CW; c += 2) mx4[(c >> 1) & 3] = max3f(mx4[(c >> 1) & 3], sv[c], sv[c + 1]);
                 const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;  // sc > 0
                 const bool grow = row_ok && mx > m + kRescaleThreshold;
                 const float m_new = grow ? mx : m;
                 const float alpha = grow ? exp2f(m - m_new) : 1.f;
-                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                // exponentials and their sums in pairs
+                const uint64_t sc2 = f2_pack(sc, sc), nm2 = f2_pack(-m_new, -m_new);
+                uint64_t ls2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
                 uint32_t pk[CW / 2];
 #pragma unroll
                 for (int c = 0; c < CW; c += 2) {
-                    const float p0 = exp2f(fmaf(sv[c], sc, -m_new)), p1 = exp2f(fmaf(sv[c + 1], sc, -m_new));
-                    ls4[(c >> 1) & 3] += p0 + p1;
+                    const uint64_t x2 = f2_fma(f2_pack(sv[c], sv[c + 1]), sc2, nm2);
+                    float x0, x1;
+                    f2_unpack(x2, x0, x1);
+                    const float p0 = exp2f(x0), p1 = exp2f(x1);
+                    ls2[(c >> 1) & 1] = f2_add(ls2[(c >> 1) & 1], f2_pack(p0, p1));
                     const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
                     pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
                 }
-                l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
+                {
+                    float a0, a1, b0, b1;
+                    f2_unpack(ls2[0], a0, a1);
+                    f2_unpack(ls2[1], b0, b1);
+                    l = l * alpha + ((a0 + a1) + (b0 + b1));
+                }
                 m = m_new;
 
                 if (j >= TC) {  // this group's previous product: number (j - tc) / TC - 1 on its own barrier
@@ -599,23 +701,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         }
                         tmem_wait_st();
                     }
-                }
-                if (kv0 + kBN > Ltot) {
-                    // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
-                    // but 0 * NaN would poison O, so those V rows are cleared before the PV product reads them.  Every
-                    // row tile's group clears them (the same zeros) before it releases its own P: each PV issuer
-                    // only waits for its own group.
-                    const int s = j % S, it = j / S;
-                    mbar_wait_warp(BAR(V_FULL + s), it & 1, dead);
-                    const int first = Ltot - kv0;  // 1..63
-                    unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
-                    const int stride = active_threads(t);
-                    for (int idx = row; idx < (kBN - first) * 8 * NH; idx += stride) {
-                        const int h = idx / ((kBN - first) * 8), rem = idx % ((kBN - first) * 8);
-                        const int r = first + rem / 8, ch = rem % 8;
-                        *reinterpret_cast<uint4*>(vt + h * (kBN * 128) + r * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    fence_async_smem();  // generic-proxy stores, read by the tensor core through the async proxy
                 }
                 // P row -> tensor memory, packed two bf16 per column over the first 32 columns of this score buffer (the
                 // scores were read above).  A copy owns CW/2 of these columns and clears the others: the product runs
@@ -647,81 +732,98 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             // every MMA of the CTA has finished before any tile buffer is reused for the parked partials
             named_bar_sync(1, NM * TC * 128);
             if (warp_active) {
-                float* po = reinterpret_cast<float*>(base_ptr) + (size_t)((t * TC + tc) * kBM + row) * PS;
+                // REP == 1: the thread's row is a partial of its own and is parked as an exchange row;
+                // REP > 1: the copies are parked in fp32 and merged below
+                float* po = reinterpret_cast<float*>(base_ptr) + (size_t)row * PS;
+                unsigned char* xo = base_ptr + (size_t)((t * TC + tc) * kBM + row) * XS;
+                const float inv_l = (n_own > 0 && l > 0.f) ? 1.f / l : 0.f;
 #pragma unroll
-                for (int cc = 0; cc < D / 32; ++cc) {
-                    uint32_t o[32];
+                for (int cc = 0; cc < D / 64; ++cc) {  // 64 columns per round trip to tensor memory
+                    uint32_t o[64];
                     if (n_own > 0) {
-                        tmem_ld_cols<32>(TM_O(t, tc) + lane_off + cc * 32, o);
+                        tmem_ld_cols<64>(TM_O(t, tc) + lane_off + cc * 64, o);
                         tmem_wait_ld();
                     } else {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = 0u;
+                        for (int c = 0; c < 64; ++c) o[c] = 0u;
                     }
+                    if (REP > 1) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 4)
-                        *reinterpret_cast<float4*>(po + cc * 32 + c) = make_float4(
-                            __uint_as_float(o[c]), __uint_as_float(o[c + 1]), __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
+                        for (int c = 0; c < 64; c += 4)
+                            *reinterpret_cast<float4*>(po + cc * 64 + c) = make_float4(
+                                __uint_as_float(o[c]), __uint_as_float(o[c + 1]), __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 64; c += 8)
+                            *reinterpret_cast<uint4*>(xo + (cc * 64 + c) * 2) =
+                                make_uint4(pack_half2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l),
+                                           pack_half2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l),
+                                           pack_half2(__uint_as_float(o[c + 4]) * inv_l, __uint_as_float(o[c + 5]) * inv_l),
+                                           pack_half2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l));
+                    }
                 }
-                float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)NM * TC * kBM * PS);
-                pml[(t * TC + tc) * kBM + row] = make_float2(m, l);
+                if (REP > 1) {
+                    float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)kBM * PS);
+                    pml[row] = make_float2(m, l);
+                } else {
+                    *reinterpret_cast<float2*>(xo + 2 * D) = make_float2(m, inv_l > 0.f ? l : 0.f);
+                }
             }
             if (REP > 1) {
                 // The copies of a row are merged here, inside the CTA, before the splits are merged across the
                 // cluster: distributed shared memory moves only ~16 bytes per clock and SM, so it should carry one
-                // partial per split and row, not REP.  The merged row replaces copy 0's parked row (the warp that
-                // merges row r is the only one that touches its copies).
+                // partial per split and row, not REP.  Thread (r, q) of the 128 merges columns [q D/REP, (q+1) D/REP)
+                // of row r from all copies, in copy order (the same on every run).
                 named_bar_sync(1, 128);
                 float* pin = reinterpret_cast<float*>(base_ptr);
                 float2* pml_in = reinterpret_cast<float2*>(pin + (size_t)kBM * PS);
-                float* mout = pin;
-                float2* mml = pml_in;
-                constexpr int EPLm = D / 32;
-                for (int r = warp - Cfg::kRoleWarps; r < rows_t; r += 4) {
-                    float mc[REP], M = -INFINITY;
+                constexpr int CPT = D / REP;  // columns per thread
+                const int tid = (int)threadIdx.x - 32 * Cfg::kRoleWarps;
+                const int r = tid % RB, col0 = (tid / RB) * CPT;
+                const bool mine = r < rows_t;
+                float acc[CPT], M = -INFINITY, den = 0.f;
 #pragma unroll
-                    for (int c = 0; c < REP; ++c) mc[c] = pml_in[c * RB + r].x, M = fmaxf(M, mc[c]);
-                    float den = 0.f, num[EPLm];
+                for (int k = 0; k < CPT; ++k) acc[k] = 0.f;
+                if (mine) {
+                    float2 ml[REP];
 #pragma unroll
-                    for (int e = 0; e < EPLm; ++e) num[e] = 0.f;
+                    for (int c = 0; c < REP; ++c) ml[c] = pml_in[c * RB + r], M = fmaxf(M, ml[c].x);
 #pragma unroll
-                    for (int c = 0; c < REP; ++c) {  // copy order: the same on every run
-                        const float f = exp2f(mc[c] - M);
-                        den = fmaf(f, pml_in[c * RB + r].y, den);
-                        const float* src = pin + (size_t)(c * RB + r) * PS + lane * EPLm;
+                    for (int c = 0; c < REP; ++c) {
+                        const float f = exp2f(ml[c].x - M);
+                        den = fmaf(f, ml[c].y, den);
+                        const float* src = pin + (size_t)(c * RB + r) * PS + col0;
 #pragma unroll
-                        for (int e = 0; e < EPLm; ++e) num[e] = fmaf(f, src[e], num[e]);
-                    }
-                    __syncwarp();  // every lane has read the copies' (offset, sum) before lane 0 overwrites copy 0's
-#pragma unroll
-                    for (int e = 0; e < EPLm; ++e) mout[(size_t)r * PS + lane * EPLm + e] = num[e];
-                    if (lane == 0) mml[r] = make_float2(M, den);
-                }
-            }
-            if (PUSH == 1) {
-                // this CTA's (copy-merged) partial of row r goes to CTA r % splits, slot (r / splits) * splits + split
-                // of its receive area: 32 lanes x 16 (d = 64: 8) bytes per row, (offset, sum) into the row's padding
-                if (REP > 1)
-                    __syncwarp();  // a warp pushes the rows it merged itself
-                else
-                    named_bar_sync(1, 128);  // rows were parked one per thread
-                const float* rows_src = reinterpret_cast<const float*>(base_ptr);  // parked, or merged in place
-                const float2* ml_src = reinterpret_cast<const float2*>(rows_src + (size_t)kBM * PS);
-                const uint32_t recv = base + (uint32_t)(Cfg::kQBytes + 2 * S * Cfg::kTileBytes);
-                constexpr int EPLp = D / 32;
-                if (run)
-                    for (int r = warp - Cfg::kRoleWarps; r < rows_t; r += 4) {
-                        const uint32_t dst = map_to_cta(recv + (uint32_t)(((r / splits) * splits + split) * PS * 4), (uint32_t)(r % splits));
-                        const float* src = rows_src + (size_t)r * PS + lane * EPLp;
-                        if (EPLp == 4) {
-                            const float4 o = *reinterpret_cast<const float4*>(src);
-                            st_cluster_f4(dst + (uint32_t)(lane * EPLp * 4), o.x, o.y, o.z, o.w);
-                        } else {
-                            const float2 o = *reinterpret_cast<const float2*>(src);
-                            st_cluster_f2(dst + (uint32_t)(lane * EPLp * 4), o.x, o.y);
+                        for (int k = 0; k < CPT; k += 4) {
+                            const float4 v = *reinterpret_cast<const float4*>(src + k);
+                            acc[k] = fmaf(f, v.x, acc[k]), acc[k + 1] = fmaf(f, v.y, acc[k + 1]);
+                            acc[k + 2] = fmaf(f, v.z, acc[k + 2]), acc[k + 3] = fmaf(f, v.w, acc[k + 3]);
                         }
-                        if (lane == 0) st_cluster_f2(dst + (uint32_t)(D * 4), ml_src[r].x, ml_src[r].y);
                     }
+                }
+                // the merged partial becomes one exchange row, straight from the registers
+                const float inv_den = den > 0.f ? 1.f / den : 0.f;
+                uint32_t hx[CPT / 2];
+#pragma unroll
+                for (int k = 0; k < CPT; k += 2) hx[k >> 1] = pack_half2(acc[k] * inv_den, acc[k + 1] * inv_den);
+                if (PUSH == 1) {
+                    // ... stored to CTA r % splits, slot (r / splits) * splits + split of its receive area
+                    if (mine && run) {
+                        const uint32_t recv = base + (uint32_t)(Cfg::kQBytes + 2 * S * Cfg::kTileBytes);
+                        const uint32_t dst = map_to_cta(recv + (uint32_t)(((r / splits) * splits + split) * XS), (uint32_t)(r % splits));
+#pragma unroll
+                        for (int k = 0; k < CPT / 2; k += 4)
+                            st_cluster_u4(dst + (uint32_t)(col0 * 2 + k * 4), hx[k], hx[k + 1], hx[k + 2], hx[k + 3]);
+                        if (col0 == 0) st_cluster_f2(dst + (uint32_t)(2 * D), M, den);
+                    }
+                } else if (mine) {
+                    // ... left behind the parked copies, where the peers will fetch it
+                    unsigned char* xo = base_ptr + Cfg::kPartBytes + (size_t)r * XS;
+#pragma unroll
+                    for (int k = 0; k < CPT / 2; k += 4)
+                        *reinterpret_cast<uint4*>(xo + col0 * 2 + k * 4) = make_uint4(hx[k], hx[k + 1], hx[k + 2], hx[k + 3]);
+                    if (col0 == 0) *reinterpret_cast<float2*>(xo + 2 * D) = make_float2(M, den);
+                }
             }
         } else if (warp_active && run) {
             const bool direct = prm.mode == kModeDirect;  // REP == 1 then
@@ -775,28 +877,29 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         cluster_sync_all();
         const bool run = (flags | *bad_s) == 0;
         const uint32_t rank = cluster_ctarank();
-        const float* recv = reinterpret_cast<const float*>(base_ptr + Cfg::kQBytes + 2 * S * Cfg::kTileBytes);
+        const unsigned char* recv = base_ptr + Cfg::kQBytes + 2 * S * Cfg::kTileBytes;
         constexpr int EPL = D / 32;
         const int rows = rows_in(0);
         if (run)
             for (int k = warp; (int)rank + splits * k < rows; k += Cfg::kThreads / 32) {
                 const int lr = (int)rank + splits * k;
-                const float* prow = recv + (size_t)k * splits * PS;
-                float2 ml = make_float2(-INFINITY, 0.f);
-                if (lane < splits) ml = *reinterpret_cast<const float2*>(prow + (size_t)lane * PS + D);
-                float M = ml.x;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-                const float f_mine = lane < splits ? exp2f(ml.x - M) : 0.f;
-                float den = f_mine * ml.y;  // fixed (butterfly) order: the same on every run
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-                float num[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int i = 0; i < splits; ++i) {  // split order
-                    const float f = __shfl_sync(0xffffffffu, f_mine, i);
-                    const float* src = prow + (size_t)i * PS + lane * EPL;
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) num[e] = fmaf(f, src[e], num[e]);
+                const unsigned char* prow = recv + (size_t)k * splits * XS;
+                // every lane reads all (offset, sum) pairs itself (broadcast reads of this CTA's own shared memory):
+                // no chain of shuffles between the barrier and the stores
+                float M = -INFINITY;
+                for (int i = 0; i < splits; ++i) M = fmaxf(M, *reinterpret_cast<const float*>(prow + (size_t)i * XS + 2 * D));
+                float den = 0.f, num[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int i = 0; i < splits; ++i) {  // split order: the same on every run
+                    const float2 ml = *reinterpret_cast<const float2*>(prow + (size_t)i * XS + 2 * D);
+                    const float w = exp2f(ml.x - M) * ml.y;  // the partial's share of the softmax sum
+                    den += w;
+                    const unsigned char* src = prow + (size_t)i * XS + lane * (EPL * 2);
+                    const float2 a = unpack_half2(*reinterpret_cast<const uint32_t*>(src));
+                    num[0] = fmaf(w, a.x, num[0]), num[1] = fmaf(w, a.y, num[1]);
+                    if (EPL == 4) {
+                        const float2 c = unpack_half2(*reinterpret_cast<const uint32_t*>(src + 4));
+                        num[2] = fmaf(w, c.x, num[2]), num[3] = fmaf(w, c.y, num[3]);
+                    }
                 }
                 const int gr = mt0 * kBM + lr;
                 const float inv = ((gr % T) < n && den > 0.f) ? 1.f / den : 0.f;
@@ -812,72 +915,91 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
         __syncthreads();  // warp 1 frees the tensor memory below: every warp is done
     } else if (prm.mode == kModeCluster) {
-        // ---- merge the splits (and copies) through distributed shared memory: this CTA owns the output rows
-        //      rank, rank + splits, ... of every row tile; one warp per row, lane i first fetches (offset, sum) of
-        //      partial i, then every lane gathers its 4 (d = 64: 2) output columns from all partials, 8 loads in flight
+        // ---- merge the splits (and turns) through distributed shared memory: this CTA owns the output rows
+        //      rank, rank + splits, ... of every row tile.  One warp per row, two rows at a time: lane i fetches
+        //      (offset, sum) of partial i, every lane its 4 (d = 64: 2) output columns of up to 8 partials of both rows,
+        //      all requests in flight before the first use -- a remote read takes about a microsecond
         __syncwarp();
         cluster_sync_all();
         const bool run = (flags | *bad_s) == 0;  // the same in every CTA of the cluster: it depends on the sequence only
         const uint32_t rank = cluster_ctarank();
-        // row copies were merged inside their CTA (into copy 0's rows); turns are merged here with the splits
-        const uint32_t part = base, part_ml = base + (uint32_t)(NM * TC * kBM * PS * 4);
+        // row copies were merged inside their CTA (one exchange row per row, behind the parked copies); turns are
+        // merged here with the splits
+        const uint32_t part = base + (uint32_t)(REP > 1 ? Cfg::kPartBytes : 0);
         constexpr int EPL = D / 32;  // output elements per lane
         constexpr int NC = TC;       // partials per split
+        constexpr int U = 2;         // output rows in flight per warp
         const int np = splits * NC;  // partials per output row (<= 16)
-        // shared-memory row of partial i of output row (t, lr): i / NC is the split, i % NC the turn
-        auto part_row = [&](int t, int lr, int i) { return (uint32_t)((t * TC + i % NC) * kBM + lr); };
+        // exchange row of partial i of output row (t, lr): i / NC is the split, i % NC the turn
+        auto part_addr = [&](int t, int lr, int i) {
+            return map_to_cta(part + (uint32_t)(((t * TC + i % NC) * kBM + lr) * XS), (uint32_t)(i / NC));
+        };
+        const int stride = splits * (Cfg::kThreads / 32);
         if (run)
-            for (int idx = (int)rank + splits * warp; idx < NM * RB; idx += splits * (Cfg::kThreads / 32)) {
-                const int t = idx / RB, lr = idx % RB;
-                if (lr >= rows_in(t)) continue;
-                const int gr = (mt0 + t) * kBM + lr;
-                const bool node_valid = (gr % T) < n;
-                // partial i = (split i / REP, copy i % REP)
-                float2 ml = make_float2(-INFINITY, 0.f);
-                if (lane < np)
-                    ml = ld_cluster_f2(map_to_cta(part_ml + part_row(t, lr, lane) * 8u, (uint32_t)(lane / NC)));
-                float M = ml.x;
+            for (int idx0 = (int)rank + splits * warp; idx0 < NM * RB; idx0 += U * stride) {
+                int tt[U], lr[U];
+                bool ok[U];
+                float2 ml[U];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-                const float f_mine = lane < np ? exp2f(ml.x - M) : 0.f;
-                float den = f_mine * ml.y;  // summed in a fixed (butterfly) order: the same on every run
+                for (int u = 0; u < U; ++u) {
+                    const int idx = idx0 + u * stride;
+                    tt[u] = idx / RB, lr[u] = idx % RB;
+                    ok[u] = idx < NM * RB && lr[u] < rows_in(tt[u]);
+                    ml[u] = make_float2(-INFINITY, 0.f);
+                    if (ok[u] && lane < np) ml[u] = ld_cluster_f2(part_addr(tt[u], lr[u], lane) + (uint32_t)(2 * D));
+                }
+                float num[U][4], den[U], w_mine[U];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-                float num[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int u = 0; u < U; ++u) num[u][0] = num[u][1] = num[u][2] = num[u][3] = 0.f, den[u] = 0.f;
                 for (int i0 = 0; i0 < np; i0 += 8) {
-                    float4 o4[8];
+                    uint2 h[U][8];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const int i = i0 + k;
-                        o4[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (i < np) {
-                            const uint32_t prow = part_row(t, lr, i);
-                            const uint32_t a = map_to_cta(part + (prow * PS + (uint32_t)lane * EPL) * 4u, (uint32_t)(i / NC));
-                            if (EPL == 4) {
-                                o4[k] = ld_cluster_f4(a);
-                            } else {
-                                const float2 o2 = ld_cluster_f2(a);
-                                o4[k].x = o2.x, o4[k].y = o2.y;
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            h[u][k] = make_uint2(0u, 0u);
+                            if (ok[u] && i0 + k < np) {
+                                const uint32_t a = part_addr(tt[u], lr[u], i0 + k) + (uint32_t)(lane * EPL * 2);
+                                if (EPL == 4) {
+                                    h[u][k] = ld_cluster_u2(a);
+                                } else {
+                                    h[u][k].x = ld_cluster_u1(a);
+                                }
                             }
+                        }
+                    if (i0 == 0) {
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            float M = -INFINITY;  // independent shuffles, not a butterfly: they overlap
+                            for (int i = 0; i < np; ++i) M = fmaxf(M, __shfl_sync(0xffffffffu, ml[u].x, i));
+                            w_mine[u] = lane < np ? exp2f(ml[u].x - M) * ml[u].y : 0.f;  // the partial's share of the sum
                         }
                     }
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const float f = __shfl_sync(0xffffffffu, f_mine, (i0 + k) & 31);
-                        num[0] = fmaf(f, o4[k].x, num[0]), num[1] = fmaf(f, o4[k].y, num[1]);
-                        num[2] = fmaf(f, o4[k].z, num[2]), num[3] = fmaf(f, o4[k].w, num[3]);
-                    }
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const float w = __shfl_sync(0xffffffffu, w_mine[u], (i0 + k) & 31);  // 0 past the last partial
+                            den[u] += w;  // partial order: the same on every run
+                            const float2 a = unpack_half2(h[u][k].x), c = unpack_half2(h[u][k].y);
+                            num[u][0] = fmaf(w, a.x, num[u][0]), num[u][1] = fmaf(w, a.y, num[u][1]);
+                            num[u][2] = fmaf(w, c.x, num[u][2]), num[u][3] = fmaf(w, c.y, num[u][3]);
+                        }
                 }
-                const float inv = (node_valid && den > 0.f) ? 1.f / den : 0.f;
-                const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;
-                __nv_bfloat16* dst = prm.out + orow * D + lane * EPL;
-                const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
-                if (EPL == 4) {
-                    const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[2] * inv, num[3] * inv);
-                    *reinterpret_cast<uint2*>(dst) =
-                        make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
-                } else {
-                    *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(&h0);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (!ok[u]) continue;
+                    const int gr = (mt0 + tt[u]) * kBM + lr[u];
+                    const float inv = ((gr % T) < n && den[u] > 0.f) ? 1.f / den[u] : 0.f;
+                    __nv_bfloat16* dst = prm.out + ((size_t)(b * prm.Hq + hk * G) * T + gr) * D + lane * EPL;
+                    const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[u][0] * inv, num[u][1] * inv);
+                    if (EPL == 4) {
+                        const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[u][2] * inv, num[u][3] * inv);
+                        *reinterpret_cast<uint2*>(dst) =
+                            make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                    } else {
+                        *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(&h0);
+                    }
                 }
             }
         __syncwarp();
