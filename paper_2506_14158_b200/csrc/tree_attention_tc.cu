@@ -5,11 +5,11 @@
 // so K/V stream from HBM once per KV head (NM = 2 covers G*T up to 256 rows, the GQA case, with one pass).
 // Warp-specialised:
 //   warp 0        TMA producer: Q once, then K and V tiles of 64 slots into 128B-swizzled shared-memory rings
-//   next 2 x NM   MMA issuers, one warp per product and row tile (the loop runs warp-uniformly, so that descriptors
-//                 stay in uniform registers; an elected lane issues): the QK issuers send S = Q K^T
-//                 (tcgen05.mma kind::f16, M128 N64 K16 x d/16) into one of the TMEM score buffers of their row
-//                 tile, the PV issuers O += P V (M128 N=d K16 x 4, P read from tensor memory) into its TMEM
-//                 accumulator; warp 1 owns the TMEM allocation
+//   next NM + 1   MMA issuers (the loops run warp-uniformly, so that descriptors stay in uniform registers; an
+//                 elected lane issues): one QK issuer warp per row tile sends S = Q K^T (tcgen05.mma kind::f16,
+//                 M128 N64 K16 x d/16) into one of the TMEM score buffers of its row tile, one PV issuer warp sends
+//                 O += P V (M128 N=d K16 x 4, P read from tensor memory) into each row tile's TMEM accumulator;
+//                 warp 1 owns the TMEM allocation
 //   then          one group of four warps per row tile, one thread per query row: tcgen05.ld of the scores,
 //                 tree / tail masking from the row's ancestor bitmask (built from parent[] by the thread
 //                 itself), online softmax in fp32 (base 2; the running offset only moves when the maximum
@@ -57,11 +57,11 @@ struct TcCfg {
     // that a product S = Q K^T need not wait for the P V product two tiles back
     static constexpr int kScoreBufs = (NM == 1 && TC == 1 && PUSH != 2) ? 4 : 2 * TC;
     static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM;
-    static constexpr int kRoleWarps = 1 + 2 * NM;    // TMA warp, then a QK issuer and a PV issuer warp per row tile
+    // TMA warp, a QK issuer warp per row tile, one PV issuer warp.  (Two row tiles: 4 + 8 = 12 warps, three per scheduler,
+    // so that a thread may hold 168 registers; a 13th warp would cap every thread at 128 and spill the softmax loop.)
+    static constexpr int kRoleWarps = 2 + NM;
     static constexpr int kThreads = 32 * kRoleWarps + 128 * NM * TC;  // ... and four softmax warps per row tile (and turn)
-    static constexpr int kPartStride = D + 4;        // floats per parked fp32 row (padding spreads the banks)
-    static constexpr int kPartBytes = NM * TC * kBM * kPartStride * 4 + NM * TC * kBM * 8;
-    // A partial travels between the CTAs of a cluster as one exchange row: the normalised output row in fp16 (2^-11
+    // A partial is parked, and travels between the CTAs of a cluster, as one exchange row: the normalised output row in fp16 (2^-11
     // relative, an eighth of the bf16 rounding of the result), then (offset, sum) in fp32, padded to 16 bytes so that
     // rows 2D + 16 bytes apart spread over the banks.  Half the bytes of fp32 rows on the slow path between SMs.
     static constexpr int kXRowBytes = 2 * D + 16;
@@ -69,7 +69,7 @@ struct TcCfg {
     static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kSmemData + 1024 /*barriers, flags, parent[]*/;
     static constexpr int kTmemCols = NM * kScoreBufs * kBN + NM * TC * D <= 256 ? 256 : 512;
     static_assert(kNumBars * 8 <= 480, "barrier area");
-    static_assert(PUSH == 2 || kPartBytes + kXBytes <= kSmemData, "parked partials reuse the tile buffers (half-SM CTAs never merge)");
+    static_assert(PUSH == 2 || 2 * kXBytes <= kSmemData, "parked partials reuse the tile buffers (half-SM CTAs never merge)");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
@@ -378,7 +378,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     using Cfg = TcCfg<D, NM, TC, PUSH>;
     constexpr int S = Cfg::kStages;
     constexpr int NH = Cfg::kHalves;
-    constexpr int PS = Cfg::kPartStride;
     constexpr int XS = Cfg::kXRowBytes;
     constexpr int RB = kBM / REP;  // rows per copy
     constexpr int CW = kBN / REP;  // columns of a tile per copy
@@ -546,10 +545,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 __syncwarp();
             }
         }
-    } else if (warp <= 2 * NM) {
-        // ================= PV issuer of row tile t: O += P V =================
-        const int t = warp - 1 - NM;
-        if (nt > 0 && t < nm_act) {
+    } else if (warp == NM + 1) {
+        // ================= PV issuer: O += P V, for every row tile in turn =================
+        // (the row tiles' softmax groups finish a tile one after the other, so one warp serves them in that order)
+        if (nt > 0) {
             constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
@@ -557,8 +556,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 if ((t0 + j) * kBN + kBN > Ltot) {
                     // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
                     // but 0 * NaN would poison O, so those V rows are cleared before the product reads them -- here, by
-                    // the warp that waits for P anyway.  Every row tile's issuer warp clears them (the same zeros): each
-                    // only knows about its own product.
+                    // the warp that waits for P anyway
                     const int first = Ltot - (t0 + j) * kBN;  // 1..63
                     unsigned char* vt = base_ptr + (sV - base) + s * Cfg::kTileBytes;
                     constexpr int CPR = 8 * NH;  // 16-byte chunks per slot: a lane keeps its chunk and walks down the slots
@@ -569,19 +567,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 // B = V [64 slots][d], MN-major: 16 slots (K step) = 2048 bytes; d halves kBN*128 bytes apart
                 const uint64_t v_desc = smem_desc_sw128(sV + s * Cfg::kTileBytes, kBN * 128, 1024);
-                mbar_wait(P_FULL(t, j % NB), (j / NB) & 1, dead);
-                tc_fence_after();
-                if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < kBN / 16; ++kk)
-                        // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
-                        tc_mma_bf16_ts(TM_O(t, TC == 2 ? (j & 1) : 0), TM_S(t, j % NB) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4),
-                                       idesc_pv, (j >= TC || kk > 0) ? 1u : 0u);
-                    tc_commit(PV_DONE(t, TC == 2 ? (j & 1) : 0));
-                    tc_commit(S_EMPTY(t, j % NB));  // the score buffer (and the P inside it) may be overwritten
-                    tc_commit(BAR(V_EMPTY + s));
+                for (int t = 0; t < NM; ++t) {
+                    if (t >= nm_act) break;
+                    mbar_wait(P_FULL(t, j % NB), (j / NB) & 1, dead);
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int kk = 0; kk < kBN / 16; ++kk)
+                            // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
+                            tc_mma_bf16_ts(TM_O(t, TC == 2 ? (j & 1) : 0), TM_S(t, j % NB) + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4),
+                                           idesc_pv, (j >= TC || kk > 0) ? 1u : 0u);
+                        tc_commit(PV_DONE(t, TC == 2 ? (j & 1) : 0));
+                        tc_commit(S_EMPTY(t, j % NB));  // the score buffer (and the P inside it) may be overwritten
+                        tc_commit(BAR(V_EMPTY + s));    // (one arrival per row tile)
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
         }
     } else {
@@ -686,10 +688,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 m = m_new;
 
-                if (j >= TC) {  // this group's previous product: number (j - tc) / TC - 1 on its own barrier
-                    mbar_wait_warp(PV_DONE(t, tc), ((j - tc) / TC - 1) & 1, dead);
+                // O is rescaled (rarely) once this group's previous product, number i - 1 on its own barrier, is complete.
+                // With two score buffers per group S_FULL of tile i already says that product i - 2 is complete, so the
+                // barrier is at most one phase behind whenever it is looked at and the look can be left out when no row
+                // of the warp moves its offset -- except on the group's last tile, so that the wait after the loop
+                // finds it at most one phase behind as well.  (Four buffers: product i - 4 only; the wait stays.)
+                const int i_own = (j - tc) / TC;
+                const bool any_grow = __any_sync(0xffffffffu, grow);
+                if (i_own > 0 && (NB != 2 * TC || any_grow || i_own == n_own - 1)) {
+                    mbar_wait_warp(PV_DONE(t, tc), (i_own - 1) & 1, dead);
                     tc_fence_after();
-                    if (__any_sync(0xffffffffu, grow)) {
+                    if (any_grow) {
 #pragma unroll
                         for (int cc = 0; cc < D / 32; ++cc) {
                             uint32_t o[32];
@@ -732,9 +741,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             // every MMA of the CTA has finished before any tile buffer is reused for the parked partials
             named_bar_sync(1, NM * TC * 128);
             if (warp_active) {
-                // REP == 1: the thread's row is a partial of its own and is parked as an exchange row;
-                // REP > 1: the copies are parked in fp32 and merged below
-                float* po = reinterpret_cast<float*>(base_ptr) + (size_t)row * PS;
+                // the thread's row (of its copy, of its turn) is parked as an exchange row
                 unsigned char* xo = base_ptr + (size_t)((t * TC + tc) * kBM + row) * XS;
                 const float inv_l = (n_own > 0 && l > 0.f) ? 1.f / l : 0.f;
 #pragma unroll
@@ -747,36 +754,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                         for (int c = 0; c < 64; ++c) o[c] = 0u;
                     }
-                    if (REP > 1) {
 #pragma unroll
-                        for (int c = 0; c < 64; c += 4)
-                            *reinterpret_cast<float4*>(po + cc * 64 + c) = make_float4(
-                                __uint_as_float(o[c]), __uint_as_float(o[c + 1]), __uint_as_float(o[c + 2]), __uint_as_float(o[c + 3]));
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 64; c += 8)
-                            *reinterpret_cast<uint4*>(xo + (cc * 64 + c) * 2) =
-                                make_uint4(pack_half2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l),
-                                           pack_half2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l),
-                                           pack_half2(__uint_as_float(o[c + 4]) * inv_l, __uint_as_float(o[c + 5]) * inv_l),
-                                           pack_half2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l));
-                    }
+                    for (int c = 0; c < 64; c += 8)
+                        *reinterpret_cast<uint4*>(xo + (cc * 64 + c) * 2) =
+                            make_uint4(pack_half2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l),
+                                       pack_half2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l),
+                                       pack_half2(__uint_as_float(o[c + 4]) * inv_l, __uint_as_float(o[c + 5]) * inv_l),
+                                       pack_half2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l));
                 }
-                if (REP > 1) {
-                    float2* pml = reinterpret_cast<float2*>(reinterpret_cast<float*>(base_ptr) + (size_t)kBM * PS);
-                    pml[row] = make_float2(m, l);
-                } else {
-                    *reinterpret_cast<float2*>(xo + 2 * D) = make_float2(m, inv_l > 0.f ? l : 0.f);
-                }
+                *reinterpret_cast<float2*>(xo + 2 * D) = make_float2(m, inv_l > 0.f ? l : 0.f);
             }
             if (REP > 1) {
                 // The copies of a row are merged here, inside the CTA, before the splits are merged across the
-                // cluster: distributed shared memory moves only ~16 bytes per clock and SM, so it should carry one
-                // partial per split and row, not REP.  Thread (r, q) of the 128 merges columns [q D/REP, (q+1) D/REP)
-                // of row r from all copies, in copy order (the same on every run).
+                // cluster: distributed shared memory is slow, so it should carry one partial per split and row, not
+                // REP.  Thread (r, q) of the 128 merges columns [q D/REP, (q+1) D/REP) of row r from all copies, in
+                // copy order (the same on every run).
                 named_bar_sync(1, 128);
-                float* pin = reinterpret_cast<float*>(base_ptr);
-                float2* pml_in = reinterpret_cast<float2*>(pin + (size_t)kBM * PS);
                 constexpr int CPT = D / REP;  // columns per thread
                 const int tid = (int)threadIdx.x - 32 * Cfg::kRoleWarps;
                 const int r = tid % RB, col0 = (tid / RB) * CPT;
@@ -787,17 +780,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 if (mine) {
                     float2 ml[REP];
 #pragma unroll
-                    for (int c = 0; c < REP; ++c) ml[c] = pml_in[c * RB + r], M = fmaxf(M, ml[c].x);
+                    for (int c = 0; c < REP; ++c) {
+                        ml[c] = *reinterpret_cast<const float2*>(base_ptr + (size_t)(c * RB + r) * XS + 2 * D);
+                        M = fmaxf(M, ml[c].x);
+                    }
 #pragma unroll
                     for (int c = 0; c < REP; ++c) {
-                        const float f = exp2f(ml[c].x - M);
-                        den = fmaf(f, ml[c].y, den);
-                        const float* src = pin + (size_t)(c * RB + r) * PS + col0;
+                        const float w = exp2f(ml[c].x - M) * ml[c].y;  // the copy's share of the softmax sum
+                        den += w;
+                        const unsigned char* src = base_ptr + (size_t)(c * RB + r) * XS + col0 * 2;
 #pragma unroll
-                        for (int k = 0; k < CPT; k += 4) {
-                            const float4 v = *reinterpret_cast<const float4*>(src + k);
-                            acc[k] = fmaf(f, v.x, acc[k]), acc[k + 1] = fmaf(f, v.y, acc[k + 1]);
-                            acc[k + 2] = fmaf(f, v.z, acc[k + 2]), acc[k + 3] = fmaf(f, v.w, acc[k + 3]);
+                        for (int k = 0; k < CPT; k += 8) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(src + k * 2);
+                            const float2 a0 = unpack_half2(v.x), a1 = unpack_half2(v.y), a2 = unpack_half2(v.z), a3 = unpack_half2(v.w);
+                            acc[k] = fmaf(w, a0.x, acc[k]), acc[k + 1] = fmaf(w, a0.y, acc[k + 1]);
+                            acc[k + 2] = fmaf(w, a1.x, acc[k + 2]), acc[k + 3] = fmaf(w, a1.y, acc[k + 3]);
+                            acc[k + 4] = fmaf(w, a2.x, acc[k + 4]), acc[k + 5] = fmaf(w, a2.y, acc[k + 5]);
+                            acc[k + 6] = fmaf(w, a3.x, acc[k + 6]), acc[k + 7] = fmaf(w, a3.y, acc[k + 7]);
                         }
                     }
                 }
@@ -818,7 +817,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     }
                 } else if (mine) {
                     // ... left behind the parked copies, where the peers will fetch it
-                    unsigned char* xo = base_ptr + Cfg::kPartBytes + (size_t)r * XS;
+                    unsigned char* xo = base_ptr + Cfg::kXBytes + (size_t)r * XS;
 #pragma unroll
                     for (int k = 0; k < CPT / 2; k += 4)
                         *reinterpret_cast<uint4*>(xo + col0 * 2 + k * 4) = make_uint4(hx[k], hx[k + 1], hx[k + 2], hx[k + 3]);
@@ -925,7 +924,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const uint32_t rank = cluster_ctarank();
         // row copies were merged inside their CTA (one exchange row per row, behind the parked copies); turns are
         // merged here with the splits
-        const uint32_t part = base + (uint32_t)(REP > 1 ? Cfg::kPartBytes : 0);
+        const uint32_t part = base + (uint32_t)(REP > 1 ? Cfg::kXBytes : 0);
         constexpr int EPL = D / 32;  // output elements per lane
         constexpr int NC = TC;       // partials per split
         constexpr int U = 2;         // output rows in flight per warp
