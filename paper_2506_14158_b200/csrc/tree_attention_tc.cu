@@ -313,6 +313,31 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// 2^x for a pair on the FP32 pipe instead of the special-function unit: x is split into its nearest integer n (adding
+// 1.5 * 2^23 leaves n in the low mantissa bits) and f = x - n in [-1/2, 1/2]; a cubic (minimax, relative error 7.5e-5 --
+// the result is rounded to bf16, 3.9e-3, right after) gives 2^f and n goes into the exponent.
+__device__ __forceinline__ void exp2_pair_fma(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    f2_unpack(x2, x0, x1);
+    x0 = fmaxf(x0, -126.f), x1 = fmaxf(x1, -126.f);  // masked columns arrive as -inf
+    const uint64_t x = f2_pack(x0, x1);
+    const uint64_t magic = f2_pack(12582912.f, 12582912.f);
+    const uint64_t xr = f2_add(x, magic);
+    const uint64_t f = f2_sub(x, f2_sub(xr, magic));
+    uint64_t p = f2_fma(f2_pack(0x1.c3f760p-5f, 0x1.c3f760p-5f), f, f2_pack(0x1.f0de1ap-3f, 0x1.f0de1ap-3f));
+    p = f2_fma(p, f, f2_pack(0x1.62f31ap-1f, 0x1.62f31ap-1f));
+    p = f2_fma(p, f, f2_pack(0x1.fff692p-1f, 0x1.fff692p-1f));
+    float r0, r1, n0, n1;
+    f2_unpack(p, r0, r1);
+    f2_unpack(xr, n0, n1);
+    p0 = __uint_as_float(__float_as_uint(r0) + (__float_as_uint(n0) << 23));
+    p1 = __uint_as_float(__float_as_uint(r1) + (__float_as_uint(n1) << 23));
+}
 __device__ __forceinline__ float max3f(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -666,16 +691,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const bool grow = row_ok && mx > m + kRescaleThreshold;
                 const float m_new = grow ? mx : m;
                 const float alpha = grow ? exp2f(m - m_new) : 1.f;
-                // exponentials and their sums in pairs
+                // exponentials and their sums in pairs.  With two row tiles, two softmax warps share each scheduler's
+                // special-function unit (16 lanes per SM) and it is what a tile waits for: one pair in four goes through
+                // the FP32 pipe instead.
                 const uint64_t sc2 = f2_pack(sc, sc), nm2 = f2_pack(-m_new, -m_new);
                 uint64_t ls2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
                 uint32_t pk[CW / 2];
 #pragma unroll
                 for (int c = 0; c < CW; c += 2) {
                     const uint64_t x2 = f2_fma(f2_pack(sv[c], sv[c + 1]), sc2, nm2);
-                    float x0, x1;
-                    f2_unpack(x2, x0, x1);
-                    const float p0 = exp2f(x0), p1 = exp2f(x1);
+                    float p0, p1;
+                    if ((NM == 2) && ((c >> 1) & 3) == 3) {
+                        exp2_pair_fma(x2, p0, p1);
+                    } else {
+                        float x0, x1;
+                        f2_unpack(x2, x0, x1);
+                        p0 = exp2f(x0), p1 = exp2f(x1);
+                    }
                     ls2[(c >> 1) & 1] = f2_add(ls2[(c >> 1) & 1], f2_pack(p0, p1));
                     const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
                     pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
