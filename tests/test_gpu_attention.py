@@ -59,6 +59,38 @@ def test_extreme_tree_sizes(dtype):
     _case(B=1, Hq=4, Hkv=1, T=128, d=64, Ls=[0], dtype=dtype, seed=5, tree="chain")  # no prefix at all
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("Hq,Hkv,T", [(4, 4, 26), (8, 2, 64)])
+def test_slots_past_the_sequence_end_may_hold_anything(dtype, Hq, Hkv, T):
+    # K/V slots at and beyond L + n are not part of the sequence: NaN or Inf there must not reach the output
+    # (their scores are masked by selection, their V rows never enter the product)
+    from paper_2506_14158_b200 import s4c
+    from parity import dev
+
+    B, d, Ls, C = 2, 128, [1000, 70], 1152
+    dt = {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
+    rng = np.random.default_rng(11)
+    g = torch.Generator().manual_seed(11)
+    q = torch.randn((B, Hq, T, d), generator=g).to(dt)
+    k = torch.randn((B, Hkv, C, d), generator=g).to(dt)
+    v = torch.randn((B, Hkv, C, d), generator=g).to(dt)
+    parent = np.stack([W.random_tree(T, 8, rng) for _ in range(B)])
+    clean, ref, gst, rst = attention_both(q, k, v, Ls, parent)
+    assert_attention_close(clean, ref, gst, rst, ATTN_TOL[dtype])
+    kp, vp = k.clone(), v.clone()
+    for b in range(B):
+        kp[b, :, Ls[b] + T:] = float("nan")
+        vp[b, :, Ls[b] + T:: 2] = float("nan")
+        vp[b, :, Ls[b] + T + 1:: 2] = float("inf")
+    status = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    out = torch.full(q.shape, float("nan"), dtype=q.dtype, device="cuda")
+    s4c.tree_attention(dev(q), dev(kp), dev(vp), dev(np.asarray(Ls, dtype=np.int32)), dev(parent.astype(np.int32)), None,
+                       out=out, status=status)
+    torch.cuda.synchronize()
+    assert (status.cpu().numpy() == 0).all()
+    np.testing.assert_array_equal(out.double().cpu().numpy(), clean)
+
+
 def test_long_context_many_splits():
     _case(B=1, Hq=8, Hkv=8, T=16, d=128, Ls=[9000], dtype="bf16", seed=6)
 
