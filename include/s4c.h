@@ -149,7 +149,7 @@ s4c_status s4c_tree_accept(const float* target_logits, const float* draft_probs,
  * exits).  The call itself allocates and frees nothing, directly or through any library.
  *
  *   - Size limit: s4c_tree_accept_workspace_bytes(B,T,V) must not exceed
- *     S4C_NOALLOC_SCRATCH_BYTES (about B*T*ceil(V/4096) <= 32000 row segments); a larger problem is
+ *     S4C_NOALLOC_SCRATCH_BYTES (about B*T*(16*ceil(V/4096) + 40) bytes); a larger problem is
  *     refused with S4C_ERR_WORKSPACE and nothing is launched.
  *   - The first call on each device looks up the array's device address (a host-side runtime
  *     query, made with that device current).  Make that first call outside any stream capture.

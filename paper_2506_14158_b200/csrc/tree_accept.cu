@@ -2,17 +2,17 @@
 //   greedy (Section 4.1.2) and speculative sampling (Section 2; Eq. 11, Eq. 12), walked along
 //   root-to-leaf paths to the longest accepted path (Section 3.2).
 //
-// Three kernels, all HBM-streaming or latency-bound, no tensor cores (there is no contraction here):
-//   1. accept_rowstats_kernel   grid (vocab segments, T, B): every CTA holds one 4096-element segment of
-//      one logits row in registers (16-byte coalesced loads), reduces (max, lowest argmax) with warp
-//      shuffles and, for sampling, the segment's sum of exp((x - max_seg)/tau) in float64.
-//   2. accept_residual_kernel   (sampling only) same grid: merges the row's segment statistics, then
-//      streams the logits segment again (L2) with the draft-probability segment and reduces the
-//      first-round residual mass  Z1 = sum max(p - q, 0)  and the draft mass left after removing the
-//      first child's token -- what the walk needs after the first rejection at any node.
-//   3. accept_walk_kernel       one CTA per sequence: validates the tree, merges per-node statistics,
-//      walks root to leaf.  Second and later rejections at one node need a new residual mass; those
-//      and the final inverse-CDF draw are CTA-wide passes over that single row.
+// Kernels, all HBM-streaming or latency-bound, no tensor cores (there is no contraction here):
+//   per-node statistics, large problems: accept_rowstats_kernel, grid (vocab segments, T, B): every CTA holds one
+//      4096-element segment of one logits row in registers (16-byte coalesced loads), reduces (max, lowest argmax)
+//      with warp shuffles and, for sampling, the segment's sum of exp((x - max_seg)/tau) in float64.  The residual
+//      mass after a rejection is NOT computed ahead for every node: only the few nodes on the walked path ever
+//      need it, so the walk computes it when a rejection happens.
+//   per-node statistics, small problems: accept_stats_cluster_kernel, one 8-CTA cluster per row with the row in
+//      registers: max/argmax, sum, first-round residual mass and draft mass without the first child's token at once.
+//   accept_walk_cluster_kernel  one cluster per sequence (greedy: one CTA): validates the tree, merges per-node
+//      statistics, walks root to leaf.  Rejections at a node need a new residual mass; those and the final
+//      inverse-CDF draw are cluster-wide passes over that single row.
 // Every sum that feeds a decision is float64 with a fixed reduction order, so results do not depend on
 // scheduling and agree with a sequential float64 evaluation to rounding (~1e-15 relative).
 #include <float.h>
@@ -30,10 +30,6 @@ struct RowPartial {  // one vocab segment of one row
     double S;        // sum exp((x - M)/tau) over the segment (sampling only)
     float M;         // segment max
     int idx;         // lowest index attaining M
-};
-struct ResPartial {
-    double Z;  // sum max(p - q, 0) over the segment
-    double Q;  // sum of q over the segment, the first child's token left out
 };
 struct NodeStats {
     double S;
@@ -53,8 +49,6 @@ struct NodeSummary {  // per-node result of the cluster path
 
 struct AcceptWorkspace {
     RowPartial* row;
-    ResPartial* res;
-    NodeStats* node;
     NodeSummary* summary;
 };
 static inline size_t accept_ws_layout(int B, int T, int V, char* base, AcceptWorkspace* ws) {
@@ -62,10 +56,6 @@ static inline size_t accept_ws_layout(int B, int T, int V, char* base, AcceptWor
     size_t off = 0;
     if (ws) ws->row = reinterpret_cast<RowPartial*>(base + off);
     off += round_up(n * sizeof(RowPartial), 256);
-    if (ws) ws->res = reinterpret_cast<ResPartial*>(base + off);
-    off += round_up(n * sizeof(ResPartial), 256);
-    if (ws) ws->node = reinterpret_cast<NodeStats*>(base + off);
-    off += round_up((size_t)B * T * sizeof(NodeStats), 256);
     if (ws) ws->summary = reinterpret_cast<NodeSummary*>(base + off);
     off += round_up((size_t)B * T * sizeof(NodeSummary), 256);
     return off;
@@ -255,90 +245,6 @@ __device__ __forceinline__ NodeStats merge_row(const RowPartial* __restrict__ pa
         for (int s = 0; s < splits; ++s)
             if (part[s].M > -INFINITY) r.S += part[s].S * exp(((double)part[s].M - (double)r.M) * inv_tau);
     return r;
-}
-
-// ----------------------------------------------------------------------------- kernel 2
-template <bool VEC>
-__global__ void __launch_bounds__(kRowThreads)
-accept_residual_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs,
-                       const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
-                       const int32_t* __restrict__ n_nodes, int T, int V, double inv_tau, float floor_span,
-                       const RowPartial* __restrict__ rowp, ResPartial* __restrict__ resp,
-                       NodeStats* __restrict__ nodes) {
-    const int split = blockIdx.x, node = blockIdx.y, b = blockIdx.z, splits = gridDim.x;
-    const int n = n_nodes ? n_nodes[b] : T;
-    if (node >= n || n > T) return;
-    __shared__ NodeStats ns;
-    __shared__ int first_tok;
-    __shared__ double scratch[33];
-    __shared__ double tab[32];
-    fill_exp_table(tab);
-    if (threadIdx.x < 32) {
-        // the row's statistics from its segments, by one warp: lane s (and s + 32, ...) takes segment s; the maximum
-        // and the sum then go through fixed-order butterflies (the same on every run and in every CTA of the row)
-        const RowPartial* part = rowp + ((size_t)b * T + node) * splits;
-        float M = -INFINITY;
-        int idx = INT_MAX;
-        for (int s = threadIdx.x; s < splits; s += 32) argmax_combine(M, idx, part[s].M, part[s].idx);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float om = __shfl_xor_sync(0xffffffffu, M, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-            argmax_combine(M, idx, om, oi);
-        }
-        double S = 0.0;
-        if (M > -INFINITY)
-            for (int s = threadIdx.x; s < splits; s += 32)
-                if (part[s].M > -INFINITY) S += part[s].S * exp(((double)part[s].M - (double)M) * inv_tau);
-        S = warp_sum(S);
-        if (threadIdx.x == 0) {
-            ns.S = S, ns.M = M, ns.idx = idx;
-            if (split == 0) nodes[(size_t)b * T + node] = ns;
-        }
-    }
-    if (threadIdx.x == 32) {  // token of the first child in index order (the first one ever rejected here)
-        int ft = -1;
-        for (int c = node + 1; c < n; ++c)
-            if (parent[(size_t)b * T + c] == node) {
-                ft = tokens[(size_t)b * T + c];
-                break;
-            }
-        first_tok = ft;
-    }
-    const size_t off = ((size_t)b * T + node) * V;
-    const int s0 = split * kSegElems;
-    float x[kElemsPerThread], q[kElemsPerThread];  // requested before the barrier: in flight while thread 0 merges
-    load_segment<VEC>(logits + off, s0, V, x);
-    load_segment<VEC, true>(dprobs + off, s0, V, q);  // 0 beyond the row
-    __syncthreads();
-    const double invS = ns.S > 0.0 ? 1.0 / ns.S : 0.0;
-    const int ft = first_tok;
-    double z = 0.0, qs = 0.0;
-    if (ns.M > -INFINITY) {
-        const float x_floor = ns.M - floor_span;
-        const double c = -(double)ns.M * inv_tau;
-#pragma unroll
-        for (int k = 0; k < kElemsPerThread; ++k) {
-            const double p = exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab) * invS;
-            const double qd = (double)q[k];
-            const double r = p - qd;
-            z += r + fabs(r);  // 2 max(r, 0), exactly; halved below
-            qs += qd;
-        }
-        z *= 0.5;
-    } else {
-#pragma unroll
-        for (int k = 0; k < kElemsPerThread; ++k) qs += (double)q[k];
-    }
-    // the first child's token does not count towards the draft mass that is left: its owner takes it out again
-    if (threadIdx.x == 0 && ft >= s0 && ft < s0 + kSegElems && ft < V) qs -= (double)__ldg(dprobs + off + ft);
-    z = block_sum(z, scratch);
-    qs = block_sum(qs, scratch);
-    if (threadIdx.x == 0) {
-        ResPartial r;
-        r.Z = z, r.Q = qs;
-        resp[((size_t)b * T + node) * splits + split] = r;
-    }
 }
 
 // ----------------------------------------------------------------------------- kernel 3
@@ -579,7 +485,7 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                            const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
                            const int32_t* __restrict__ n_nodes, const float* __restrict__ uniforms, int T, int V,
                            int chunk, int cache_p0, int max_depth, double inv_tau, const NodeSummary* __restrict__ nodes,
-                           const NodeStats* __restrict__ seg_nodes, const ResPartial* __restrict__ seg_res, int seg_splits,
+                           int seg_splits,
                            const RowPartial* __restrict__ seg_row, int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
                            int32_t* __restrict__ next_token, uint8_t* __restrict__ near_tie,
                            int32_t* __restrict__ status) {
@@ -619,12 +525,9 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
     }
     for (int i = tid; i < n; i += blockDim.x) {
         if (seg_row) {  // statistics came per vocabulary segment: merge them in segment order
-            if (STOCH) {
-                const NodeStats ns = seg_nodes[(size_t)b * T + i];
-                double z = 0.0, q = 0.0;
-                const ResPartial* rp = seg_res + ((size_t)b * T + i) * seg_splits;
-                for (int s = 0; s < seg_splits; ++s) z += rp[s].Z, q += rp[s].Q;
-                sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = z, sh.nQ[i] = q;
+            if (STOCH) {  // (no residual mass ahead of time: see the first rejection below)
+                const NodeStats ns = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, true);
+                sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = 0.0, sh.nQ[i] = 0.0;
             } else {
                 sh.nArg[i] = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, false).idx;
             }
@@ -754,7 +657,7 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
             }
             // rejected: residual mass and the draft mass left once x is removed
             double Z, s;
-            if (r == 0) {
+            if (r == 0 && !seg_row) {  // small problems: the statistics kernel has them for every node
                 Z = sh.nZ[cur], s = sh.nQ[cur];
             } else {
                 double z = 0.0, qs = 0.0;
@@ -929,13 +832,6 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
                 accept_rowstats_kernel<true, true><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
             else
                 accept_rowstats_kernel<true, false><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
-            S4C_RETURN_IF_CUDA_ERROR();
-            if (vec)
-                accept_residual_kernel<true><<<grid, kRowThreads, 0, stream>>>(target_logits, draft_probs, tokens, parent, n_nodes,
-                                                                              T, V, inv_tau, floor_span, ws.row, ws.res, ws.node);
-            else
-                accept_residual_kernel<false><<<grid, kRowThreads, 0, stream>>>(target_logits, draft_probs, tokens, parent, n_nodes,
-                                                                               T, V, inv_tau, floor_span, ws.row, ws.res, ws.node);
         } else {
             if (vec)
                 accept_rowstats_kernel<false, true><<<grid, kRowThreads, 0, stream>>>(target_logits, n_nodes, T, V, inv_tau, floor_span, ws.row);
@@ -967,8 +863,6 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
     }
     // ---- the walk: one cluster per sequence (greedy: one CTA, no vocabulary pass)
     const NodeSummary* summary = seg_stats ? nullptr : ws.summary;
-    const NodeStats* seg_nodes = seg_stats ? ws.node : nullptr;
-    const ResPartial* seg_res = seg_stats ? ws.res : nullptr;
     const RowPartial* seg_row = seg_stats ? ws.row : nullptr;
     if (stoch) {
         cfg.gridDim = dim3(kCl, B, 1);
@@ -989,7 +883,7 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
             }
         }
         err = cudaLaunchKernelEx(&cfg, accept_walk_cluster_kernel<true>, target_logits, draft_probs, tokens, parent, n_nodes,
-                                 uniforms, T, V, chunk, cache_p0, max_depth, inv_tau, summary, seg_nodes, seg_res, splits, seg_row,
+                                 uniforms, T, V, chunk, cache_p0, max_depth, inv_tau, summary, splits, seg_row,
                                  accept_len, path, next_token, near_tie, status);
         if (err != cudaSuccess) {
             cudaGetLastError();
@@ -997,8 +891,8 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
         }
     } else {
         accept_walk_cluster_kernel<false><<<dim3(1, B), 128, sizeof(WalkClShared), stream>>>(
-            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, 0, max_depth, inv_tau, summary, seg_nodes,
-            seg_res, splits, seg_row, accept_len, path, next_token, near_tie, status);
+            target_logits, draft_probs, tokens, parent, n_nodes, uniforms, T, V, chunk, 0, max_depth, inv_tau, summary,
+            splits, seg_row, accept_len, path, next_token, near_tie, status);
         S4C_RETURN_IF_CUDA_ERROR();
     }
     return S4C_OK;
