@@ -88,10 +88,8 @@ class VerifyStep:
 
     # kernels launched by one run(): used by the benchmark to report its launch count
     def launches_per_step(self, attn_launches_per_layer: int) -> int:
-        # acceptance: per-node statistics (one cluster launch for small problems, two segment launches for large ones
-        # when sampling) and the walk
-        small = self.V % 4 == 0 and self.V <= 131072 and self.B * self.T * self.V <= (8 << 20)
-        accept = 2 if (self.temperature == 0 or small) else 3
+        # acceptance: per-node statistics (one launch, cluster or segment kernel) and the walk
+        accept = 2
         compact = 2 if self.n_layers > 0 else 1
         return self.n_layers * attn_launches_per_layer + accept + compact
 
