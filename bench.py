@@ -93,11 +93,15 @@ def ncu_traffic(workload):
 # ----------------------------------------------------------------------------- algorithmic bytes
 def algorithmic_bytes(cfg, temperature, accept_lens):
     """Bytes the method must move per step: K/V of the visible slots and Q/O once per layer; every logits row
-    (and draft-probability row when sampling) once; the accepted rows of every layer and the features."""
+    (and draft-probability row when sampling, see below) once; the accepted rows of every layer and the features."""
     s = 2 if cfg.dtype == "bf16" else 4
     attn_layer = 2 * cfg.B * cfg.Hkv * (cfg.L + cfg.T) * cfg.d * s + 2 * cfg.B * cfg.Hq * cfg.T * cfg.d * s
-    accept = cfg.B * cfg.T * cfg.V * (8 if temperature > 0 else 4)
     rows = sum(int(a) + 1 for a in accept_lens)
+    accept = cfg.B * cfg.T * cfg.V * (8 if temperature > 0 else 4)
+    if temperature > 0 and (cfg.B * cfg.T * cfg.V > (8 << 20) or cfg.V % 4 or cfg.V > 131072):
+        # large problems: the residual masses are computed on the walked rows only, so the draft probabilities of the
+        # other rows are never needed: every logits row once, logits and draft probabilities of the walked rows once more
+        accept = cfg.B * cfg.T * cfg.V * 4 + rows * cfg.V * 8
     compact = cfg.n_layers * 2 * 2 * cfg.Hkv * rows * cfg.d * s + 2 * rows * cfg.hid * s
     return dict(attention_per_layer=attn_layer, attention=attn_layer * cfg.n_layers, accept=accept, compact=compact,
                 total=attn_layer * cfg.n_layers + accept + compact)
