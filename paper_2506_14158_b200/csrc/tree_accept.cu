@@ -523,12 +523,32 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         }
         return;
     }
+    if (seg_row && STOCH) {
+        // statistics came per vocabulary segment: one warp per node, lane s takes segments s, s + 32, ...; the maximum
+        // and the sum go through fixed-order butterflies (the same on every run and in every CTA of the cluster)
+        const int lane = tid & 31;
+        for (int i = tid >> 5; i < n; i += blockDim.x >> 5) {
+            const RowPartial* part = seg_row + ((size_t)b * T + i) * seg_splits;
+            float M = -INFINITY;
+            int idx = INT_MAX;
+            for (int sg = lane; sg < seg_splits; sg += 32) argmax_combine(M, idx, part[sg].M, part[sg].idx);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, M, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+                argmax_combine(M, idx, om, oi);
+            }
+            double S = 0.0;
+            if (M > -INFINITY)
+                for (int sg = lane; sg < seg_splits; sg += 32)
+                    if (part[sg].M > -INFINITY) S += part[sg].S * exp(((double)part[sg].M - (double)M) * inv_tau);
+            S = warp_sum(S);
+            if (lane == 0) sh.nS[i] = S, sh.nM[i] = M, sh.nArg[i] = idx, sh.nZ[i] = 0.0, sh.nQ[i] = 0.0;
+        }
+    }
     for (int i = tid; i < n; i += blockDim.x) {
-        if (seg_row) {  // statistics came per vocabulary segment: merge them in segment order
-            if (STOCH) {  // (no residual mass ahead of time: see the first rejection below)
-                const NodeStats ns = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, true);
-                sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = 0.0, sh.nQ[i] = 0.0;
-            } else {
+        if (seg_row) {
+            if (!STOCH) {
                 sh.nArg[i] = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, false).idx;
             }
         } else {
