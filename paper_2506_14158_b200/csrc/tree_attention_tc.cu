@@ -1093,15 +1093,26 @@ static bool make_map_halves(CUtensorMap* map, const void* ptr, uint64_t rows, in
 bool tc_supported(int T, int Hq, int Hkv, int d, s4c_dtype dt) { return dt == S4C_BF16 && (d == 128 || d == 64); }
 
 static int tc_m_tiles(int T, int Hq, int Hkv) { return ceil_div((Hq / Hkv) * T, kBM); }
-static int tc_nm(int T, int Hq, int Hkv) { return tc_m_tiles(T, Hq, Hkv) > 1 ? 2 : 1; }
-static int tc_m_groups(int T, int Hq, int Hkv) { return ceil_div(tc_m_tiles(T, Hq, Hkv), tc_nm(T, Hq, Hkv)); }
+// Row tiles per CTA.  Two row tiles on one K/V stream read K/V once for all rows of a KV head.  A grid of few (sequence,
+// KV head) pairs cannot fill the GPU that way with the splits a cluster allows; one row tile per CTA then doubles the
+// CTAs, the second read of a K/V tile being served by L2 (measured at 256 rows: 1 sequence x 8 KV heads, L=1024: 21.8 ->
+// 9.2 us; 2 x 8, L=4096: 33.8 -> 18.6 us; at 1 x 8 beyond ~6k tokens the wide workspace path with two row tiles wins).
+static int tc_nm(int B, int T, int Hq, int Hkv, int C) {
+    if (tc_m_tiles(T, Hq, Hkv) <= 1) return 1;
+    const int pairs = B * Hkv;
+    if (pairs * kMaxClusterSplits >= 148) return 2;
+    return (pairs >= 12 || ceil_div(C, kBN) <= 96) ? 1 : 2;
+}
+static int tc_m_groups(int B, int T, int Hq, int Hkv, int C) {
+    return ceil_div(tc_m_tiles(T, Hq, Hkv), tc_nm(B, T, Hq, Hkv, C));
+}
 
 // Number of splits of the cache: the count that minimises waves x (fixed cost of a CTA + its tiles), with a small
 // charge per extra split for the merge; a split has at least two tiles.  The fixed cost (set-up, first tile's latency,
 // merge, measured at 5-6 us) is worth about ten tiles.  Up to 8 splits merge inside a cluster; a grid too small to
 // fill the GPU even with 8 goes wider and merges through the workspace.
 static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
-    const int base = B * Hkv * tc_m_groups(T, Hq, Hkv);
+    const int base = B * Hkv * tc_m_groups(B, T, Hq, Hkv, C);
     const int tiles = ceil_div(C, kBN);
     int max_by_len = tiles / 2;
     if (max_by_len < 1) max_by_len = 1;
@@ -1113,7 +1124,9 @@ static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
     int best = 1;
     double best_cost = 1e30;
     for (int s = 1; s <= kMaxClusterSplits && s <= max_by_len; ++s) {
-        const int resident = s == 1 ? 148 : 8 * (18 / s) * s;  // clusters do not straddle the 8 GPCs (18+ SMs each)
+        // clusters do not straddle the 8 GPCs, and not every GPC offers 18 SMs to them: clusters of 6 measured two waves
+        // for 144 CTAs, so the model packs 16 SMs per GPC
+        const int resident = s == 1 ? 148 : 8 * (16 / s) * s;
         const double waves = (double)ceil_div(base * s, resident);
         const double cost = waves * (10.0 + ceil_div(tiles, s)) * (1.0 + 0.03 * (s - 1));
         if (cost < best_cost - 1e-12) best_cost = cost, best = s;
@@ -1127,10 +1140,10 @@ static int tc_rep(int T, int Hq, int Hkv) {
     return R <= 32 ? 4 : (R <= 64 ? 2 : 1);
 }
 
-// Turns (see the kernel): a single row tile of 65..128 rows with enough tiles per CTA is shared by two softmax groups.
+// Turns (see the kernel): a single row tile per CTA, of 65..128 rows, with enough tiles per CTA is shared by two softmax groups.
 static int tc_turns(int B, int T, int Hq, int Hkv, int C) {
     const int R = (Hq / Hkv) * T;
-    if (R <= 64 || R > kBM) return 1;
+    if (R <= 64 || tc_nm(B, T, Hq, Hkv, C) == 2) return 1;
     const int tiles_per_cta = ceil_div(ceil_div(C, kBN), tc_splits(B, T, Hq, Hkv, C));
     return tiles_per_cta >= 8 ? 2 : 1;
 }
@@ -1193,8 +1206,8 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     prm.cache_len = cache_len, prm.parent = parent, prm.n_nodes = n_nodes;
     prm.out = static_cast<__nv_bfloat16*>(out), prm.ws = static_cast<float*>(ws), prm.status = status;
     prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C;
-    const int nm = tc_nm(T, Hq, Hkv);
-    prm.m_groups = tc_m_groups(T, Hq, Hkv);
+    const int nm = tc_nm(B, T, Hq, Hkv, C);
+    prm.m_groups = tc_m_groups(B, T, Hq, Hkv, C);
     prm.splits = tc_splits(B, T, Hq, Hkv, C);
     const int rep = tc_rep(T, Hq, Hkv), turns = tc_turns(B, T, Hq, Hkv, C);
     // copies and turns merge like splits, so a single split with either still takes the (one-CTA) cluster path
