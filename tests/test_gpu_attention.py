@@ -91,6 +91,14 @@ def test_slots_past_the_sequence_end_may_hold_anything(dtype, Hq, Hkv, T):
     np.testing.assert_array_equal(out.double().cpu().numpy(), clean)
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,T,L", [(1, 32, 8, 64, 1000),   # 256 rows of a KV head over two CTAs, two softmax groups each
+                                           (2, 16, 4, 40, 700),    # 160 rows: a full row tile and a partial one
+                                           (1, 16, 2, 128, 300),   # 1024 rows: eight row tiles, one per CTA
+                                           (1, 24, 24, 32, 3000)])  # 24 heads: clusters of 5, not 6
+def test_small_grids_take_one_row_tile_per_cta(B, Hq, Hkv, T, L):
+    _case(B=B, Hq=Hq, Hkv=Hkv, T=T, d=128, Ls=[L] * B, dtype="bf16", seed=21 + T)
+
+
 def test_long_context_many_splits():
     _case(B=1, Hq=8, Hkv=8, T=16, d=128, Ls=[9000], dtype="bf16", seed=6)
 
