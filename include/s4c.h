@@ -73,7 +73,9 @@ const char* s4c_status_string(s4c_status code);
  * over the cache slots 0..L_b-1 (the committed prefix, fully visible) and the slots L_b+t of the
  * nodes t on the path root..i (i itself included); every other tree slot is masked.  KV head of
  * query head h is h / (Hq/Hkv).  Scores are scale * <q,k>; softmax statistics and accumulation
- * are fp32; for S4C_BF16 the probabilities are rounded to bf16 before the PV product.
+ * are fp32; for S4C_BF16 the probabilities are rounded to bf16 before the PV product, and partial
+ * results of the splits of a long cache are exchanged as normalised fp16 rows: output entries
+ * beyond +-65504 (possible only with V entries of that size) are clamped there.
  *
  *   q          [B,Hq,T,d]   dt     queries of the tree tokens (after positional encoding)
  *   k_cache    [B,Hkv,C,d]  dt     keys; the tree tokens' own keys already sit at slots L_b..L_b+T-1

@@ -275,9 +275,13 @@ __device__ __forceinline__ uint32_t ld_cluster_u1(uint32_t addr) {
     asm volatile("ld.shared::cluster.b32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
+// Two floats to fp16 (a in the low half), saturating at the largest finite value: a normalised output row is a convex
+// combination of V rows, so only V entries beyond +-65504 can reach the limit; they are clamped there rather than turned
+// into infinities (which a zero weight would turn into NaN).
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
-    const __half2 h = __floats2half2_rn(a, b);
-    return *reinterpret_cast<const uint32_t*>(&h);
+    uint32_t r;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+    return r;
 }
 __device__ __forceinline__ float2 unpack_half2(uint32_t v) { return __half22float2(*reinterpret_cast<const __half2*>(&v)); }
 __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
