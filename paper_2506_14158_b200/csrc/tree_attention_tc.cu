@@ -1100,12 +1100,14 @@ static int tc_m_tiles(int T, int Hq, int Hkv) { return ceil_div((Hq / Hkv) * T, 
 // Row tiles per CTA.  Two row tiles on one K/V stream read K/V once for all rows of a KV head.  A grid of few (sequence,
 // KV head) pairs cannot fill the GPU that way with the splits a cluster allows; one row tile per CTA then doubles the
 // CTAs, the second read of a K/V tile being served by L2 (measured at 256 rows: 1 sequence x 8 KV heads, L=1024: 21.8 ->
-// 9.2 us; 2 x 8, L=4096: 33.8 -> 18.6 us; at 1 x 8 beyond ~6k tokens the wide workspace path with two row tiles wins).
+// 9.2 us; 2 x 8, L=4096: 33.8 -> 18.6 us; 512 rows, 1 x 8, L=8192: 48 -> 27 us).  Only a single sequence of exactly two row
+// tiles keeps both on one CTA beyond ~6k tokens (38 against 52 us at 16k).
 static int tc_nm(int B, int T, int Hq, int Hkv, int C) {
-    if (tc_m_tiles(T, Hq, Hkv) <= 1) return 1;
+    const int mt = tc_m_tiles(T, Hq, Hkv);
+    if (mt <= 1) return 1;
     const int pairs = B * Hkv;
-    if (pairs * kMaxClusterSplits >= 148) return 2;
-    return (pairs >= 12 || ceil_div(C, kBN) <= 96) ? 1 : 2;
+    if (pairs * ceil_div(mt, 2) * kMaxClusterSplits >= 148) return 2;
+    return (mt == 2 && pairs < 12 && ceil_div(C, kBN) > 96) ? 2 : 1;
 }
 static int tc_m_groups(int B, int T, int Hq, int Hkv, int C) {
     return ceil_div(tc_m_tiles(T, Hq, Hkv), tc_nm(B, T, Hq, Hkv, C));
@@ -1114,13 +1116,15 @@ static int tc_m_groups(int B, int T, int Hq, int Hkv, int C) {
 // Number of splits of the cache: the count that minimises waves x (fixed cost of a CTA + its tiles), with a small
 // charge per extra split for the merge; a split has at least two tiles.  The fixed cost (set-up, first tile's latency,
 // merge, measured at 5-6 us) is worth about ten tiles.  Up to 8 splits merge inside a cluster; a grid too small to
-// fill the GPU even with 8 goes wider and merges through the workspace.
+// fill the GPU even with 8 stays with 8 all the same -- the second launch and the fp32 partials in global memory of the
+// wide path cost more than the idle SMs (8 heads, L=2048: 26.7 -> 8.2 us; 4 heads, L=8192: 38.6 -> 12.7 us) -- except for
+// two row tiles per CTA on a very long cache, which go wider and merge through the workspace (53 against 66 us at 32k).
 static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
     const int base = B * Hkv * tc_m_groups(B, T, Hq, Hkv, C);
     const int tiles = ceil_div(C, kBN);
     int max_by_len = tiles / 2;
     if (max_by_len < 1) max_by_len = 1;
-    if (base * kMaxClusterSplits * 2 <= 148) {  // tiny grids: fill one wave through the workspace path
+    if (base * kMaxClusterSplits * 2 <= 148 && tiles >= 384 && tc_nm(B, T, Hq, Hkv, C) == 2) {  // one wave through the workspace path
         int s = 148 / base;
         if (s > 64) s = 64;
         return s > max_by_len ? max_by_len : s;

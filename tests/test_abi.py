@@ -50,9 +50,11 @@ def test_workspace_queries_are_host_functions(s4c_lib):
     assert s4c.tree_accept_workspace_bytes(0, 1, 1) == 0
     import torch
 
-    # 32 KV heads x 4 splits merge inside a thread-block cluster: no scratch; 8 KV heads go wider than a cluster
+    # splits merge inside a thread-block cluster: no scratch, also for grids of few heads; only two row tiles per CTA
+    # (256 query rows per KV head) on a very long cache of very few KV heads go wider than a cluster
     assert s4c.tree_attention_workspace_bytes(1, 26, 32, 32, 128, 1152, torch.bfloat16) == 0
-    w = s4c.tree_attention_workspace_bytes(1, 16, 8, 8, 128, 9088, torch.bfloat16)
+    assert s4c.tree_attention_workspace_bytes(1, 16, 8, 8, 128, 9088, torch.bfloat16) == 0
+    w = s4c.tree_attention_workspace_bytes(1, 64, 8, 2, 128, 24704, torch.bfloat16)
     assert w > 0 and w % 256 == 0
     assert s4c.tree_attention_workspace_bytes(1, 200, 32, 32, 128, 1152, torch.bfloat16) == 0  # T > 128: invalid
 
@@ -75,7 +77,7 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert att(k=P + 2) == 4                     # S4C_ERR_ALIGN
     assert att(scale=-1.0) == 2
     assert att(B=0) == 0
-    assert att(Hq=8, Hkv=8, C=9088, ws=None) == 5   # a grid this small splits wider than a cluster and needs a workspace
+    assert att(T=64, Hq=8, Hkv=2, C=24704, ws=None) == 5   # this grid splits wider than a cluster and needs a workspace
     acc = lambda **kw: lib.s4c_tree_accept(*[kw.get(k, d) for k, d in [
         ("lg", P), ("dp", P), ("tok", P), ("par", P), ("nn", None), ("tau", 1.0), ("u", P), ("B", 1), ("T", 8),
         ("V", 100), ("md", 7), ("al", P), ("path", P), ("nt", P), ("tie", None), ("st", None), ("ws", None), ("wsb", 0),

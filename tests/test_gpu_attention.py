@@ -133,8 +133,14 @@ def test_full_row_tile_with_two_softmax_groups_taking_turns(d):
     _case(B=1, Hq=16, Hkv=16, T=100, d=d, Ls=[6000], dtype="bf16", seed=11)
     # ... an odd number of tiles per split, GQA rows (2 heads x 50 nodes), padded trees ...
     _case(B=2, Hq=16, Hkv=8, T=50, d=d, Ls=[5000, 4321], dtype="bf16", seed=12, n_nodes=[50, 33])
-    # ... and through the workspace when the grid is too small for clusters
+    # ... and a grid of few heads, which stays with the 8 splits of a cluster
     _case(B=1, Hq=4, Hkv=4, T=100, d=d, Ls=[20000], dtype="bf16", seed=13)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_two_row_tiles_of_few_heads_on_a_long_cache_merge_through_the_workspace(d):
+    # 256 query rows per KV head, 2 KV heads, 386 tiles: 64 splits, partial results in the caller's workspace, second kernel
+    _case(B=1, Hq=8, Hkv=2, T=64, d=d, Ls=[24600], dtype="bf16", seed=14)
 
 
 @pytest.mark.parametrize("T", [20, 50, 100])
