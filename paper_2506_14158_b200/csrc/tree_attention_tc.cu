@@ -1119,22 +1119,60 @@ static int tc_m_groups(int B, int T, int Hq, int Hkv, int C) {
 // fill the GPU even with 8 stays with 8 all the same -- the second launch and the fp32 partials in global memory of the
 // wide path cost more than the idle SMs (8 heads, L=2048: 26.7 -> 8.2 us; 4 heads, L=8192: 38.6 -> 12.7 us) -- except for
 // two row tiles per CTA on a very long cache, which go wider and merge through the workspace (53 against 66 us at 32k).
+// CTAs that run at the same time when launched as clusters of s: asked of the device once (clusters do not straddle
+// GPCs, and how many SMs a GPC offers to a cluster differs between GPCs and parts: clusters of 6 and of 8 measured two
+// waves where 18 or 16 SMs per GPC would have held them in one).  Without a device the model of 16 SMs per GPC answers.
+static int tc_resident_ctas(int s) {
+    if (s == 1) return 148;
+    static int table[64][kMaxClusterSplits + 1] = {};
+    static bool asked[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        if (!asked[dev]) {
+            using Cfg = TcCfg<128, 1, 1, 0>;
+            auto kernel = tree_attention_tc_kernel<128, 1, 1, 1, 0>;
+            const bool ok = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) == cudaSuccess;
+            for (int c = 2; ok && c <= kMaxClusterSplits; ++c) {
+                cudaLaunchAttribute attr = {};
+                attr.id = cudaLaunchAttributeClusterDimension;
+                attr.val.clusterDim.x = c, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = 1;
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(c, 1, 1), cfg.blockDim = dim3(Cfg::kThreads, 1, 1), cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+                cfg.attrs = &attr, cfg.numAttrs = 1;
+                int clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) == cudaSuccess && clusters > 0) table[dev][c] = clusters * c;
+            }
+            cudaGetLastError();
+            asked[dev] = true;
+        }
+        if (table[dev][s] > 0) return table[dev][s];
+    } else {
+        cudaGetLastError();
+    }
+    return 8 * (16 / s) * s;
+}
+
+// The wide path's split count (more than a cluster holds), or 0 where the path is not taken.  Shapes only: the workspace
+// query depends on nothing else.
+static int tc_wide_splits(int B, int T, int Hq, int Hkv, int C) {
+    const int base = B * Hkv * tc_m_groups(B, T, Hq, Hkv, C);
+    const int tiles = ceil_div(C, kBN);
+    if (!(base * kMaxClusterSplits * 2 <= 148 && tiles >= 384 && tc_nm(B, T, Hq, Hkv, C) == 2)) return 0;
+    int s = 148 / base;  // one wave
+    if (s > 64) s = 64;
+    return s > tiles / 2 ? tiles / 2 : s;
+}
+
 static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
+    if (const int wide = tc_wide_splits(B, T, Hq, Hkv, C)) return wide;
     const int base = B * Hkv * tc_m_groups(B, T, Hq, Hkv, C);
     const int tiles = ceil_div(C, kBN);
     int max_by_len = tiles / 2;
     if (max_by_len < 1) max_by_len = 1;
-    if (base * kMaxClusterSplits * 2 <= 148 && tiles >= 384 && tc_nm(B, T, Hq, Hkv, C) == 2) {  // one wave through the workspace path
-        int s = 148 / base;
-        if (s > 64) s = 64;
-        return s > max_by_len ? max_by_len : s;
-    }
     int best = 1;
     double best_cost = 1e30;
     for (int s = 1; s <= kMaxClusterSplits && s <= max_by_len; ++s) {
-        // clusters do not straddle the 8 GPCs, and not every GPC offers 18 SMs to them: clusters of 6 measured two waves
-        // for 144 CTAs, so the model packs 16 SMs per GPC
-        const int resident = s == 1 ? 148 : 8 * (16 / s) * s;
+        const int resident = tc_resident_ctas(s);
         const double waves = (double)ceil_div(base * s, resident);
         const double cost = waves * (10.0 + ceil_div(tiles, s)) * (1.0 + 0.03 * (s - 1));
         if (cost < best_cost - 1e-12) best_cost = cost, best = s;
@@ -1157,11 +1195,8 @@ static int tc_turns(int B, int T, int Hq, int Hkv, int C) {
 }
 
 size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
-    const int s = tc_splits(B, T, Hq, Hkv, C);
-    return s <= kMaxClusterSplits ? 0
-                                  : round_up((size_t)B * Hq * T * s * tc_rep(T, Hq, Hkv) * tc_turns(B, T, Hq, Hkv, C) *
-                                                 (d + 2) * sizeof(float),
-                                             256);
+    const int s = tc_wide_splits(B, T, Hq, Hkv, C);  // (two row tiles per CTA: no row copies, no turns)
+    return s == 0 ? 0 : round_up((size_t)B * Hq * T * s * (d + 2) * sizeof(float), 256);
 }
 
 template <int D, int NM, int REP, int TC, int PUSH>
