@@ -1264,8 +1264,9 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     const int tiles_per_cta = ceil_div(ceil_div(C, kBN), prm.splits);
     const bool push = prm.mode == kModeCluster && nm == 1 && turns == 1 && tiles_per_cta <= 16 &&
                       ceil_div(R, prm.splits) * prm.splits * (d + 4) * 4 <= 32768;
-    // half-SM CTAs: grids of at least two CTAs per SM that need no merge
-    const bool half = prm.splits == 1 && nm == 1 && turns == 1 && B * Hkv * prm.m_groups >= 2 * 148;
+    // half-SM CTAs: grids of more CTAs than SMs that need no merge (a second wave of a few CTAs costs a whole pass;
+    // 256 CTAs at L=2048: 54.6 -> 49.6 us, 160 CTAs at L=512: 22.3 -> 17.8 us)
+    const bool half = prm.splits == 1 && nm == 1 && turns == 1 && B * Hkv * prm.m_groups > 148;
 #define S4C_TC_DISPATCH(DD)                                                                    \
     (half         ? (rep == 4   ? launch_tc<DD, 1, 4, 1, 2>(q, k, v, prm, B, stream)            \
                      : rep == 2 ? launch_tc<DD, 1, 2, 1, 2>(q, k, v, prm, B, stream)            \
