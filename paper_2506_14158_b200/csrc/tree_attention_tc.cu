@@ -1174,7 +1174,10 @@ static int tc_splits(int B, int T, int Hq, int Hkv, int C) {
     for (int s = 1; s <= kMaxClusterSplits && s <= max_by_len; ++s) {
         const int resident = tc_resident_ctas(s);
         const double waves = (double)ceil_div(base * s, resident);
-        const double cost = waves * (10.0 + ceil_div(tiles, s)) * (1.0 + 0.03 * (s - 1));
+        double cost = waves * (10.0 + ceil_div(tiles, s)) * (1.0 + 0.03 * (s - 1));
+        // an unsplit grid of more CTAs than SMs runs as half-SM CTAs where the rows allow it (see the dispatch below): two
+        // per SM at once, each streaming at half the rate
+        if (s == 1 && base > 148 && (Hq / Hkv) * T <= 64) cost = ceil_div(base, 296) * (10.0 + 2.0 * tiles);
         if (cost < best_cost - 1e-12) best_cost = cost, best = s;
     }
     return best;
