@@ -385,7 +385,7 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
 
     auto valid = [&](int k) { return elem(k) < V && elem(k) < c0 + chunk; };
 
-    // ---- round 1: maximum (one instruction per element), then its lowest index from the few threads that hold it
+    // ---- first reduction: maximum (one instruction per element), then its lowest index from the few threads that hold it
     float mt = x[0];
 #pragma unroll
     for (int k = 1; k < kClEpt; ++k) mt = fmaxf(mt, x[k]);
@@ -421,7 +421,7 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
         return;
     }
 
-    // ---- round 2: e = exp((x - M)/tau), once per element, kept in registers; S = sum e
+    // ---- second reduction: e = exp((x - M)/tau), once per element, kept in registers; S = sum e
     double e[kClEpt];
     double s = 0.0;
     {
@@ -442,7 +442,7 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     for (int r = 0; r < kCl; ++r) S += gathered[r];
     const double invS = S > 0.0 ? 1.0 / S : 0.0;
 
-    // ---- round 3: first-round residual mass and the draft mass without the first child's token
+    // ---- third reduction: first-round residual mass and the draft mass without the first child's token
     const int ft = first_tok;
     double z = 0.0, qs = 0.0;
 #pragma unroll
