@@ -8,7 +8,15 @@ graph).  The default workload "c2x32" is the LLaMA-2-7B-shaped verify step at fu
 cache per layer, temperature 1.0.  Its 0.56 GB of KV per step is larger than L2, so no flush is needed.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2x32|c2|c3|c4|c4x32|c1|sweep --L --T --B]
+                    [--capacity C] [--no-hint] [--no-also]
     python bench.py --impl reference     # the float64 CPU oracle on a bounded sample of the same workload
+    python bench.py --workload launch-floor   # empty kernels with the launch shape of an attention launch
+    python bench.py --workload sweep-all [--capacity C]   # every point of the full-depth sweep
+
+The default line also carries, under "also", the 8B-shaped step (c4x32: batch 4, GQA 32/8, 4096-token caches, 64-node
+trees, vocabulary 128256, 32 layers) with its own timing, roofline (HBM and tensor) and clock sample.
+--capacity lays the caches out for C slots (a serving cache sized for its longest context) instead of L + T; the
+host's bound on the live length (max_cache_len = L) is then what shapes the attention launches, unless --no-hint.
 
 Prints one JSON line (rank 0).  With N > 1 (torchrun) every rank verifies its own independent batch: weak scaling,
 no data-path collective; the only communication is the barrier and the max of the timings.
@@ -45,15 +53,20 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--capacity", type=int, default=0, help="cache capacity in slots (0: L + T rounded up to 128)")
+    ap.add_argument("--no-hint", action="store_true", help="do not pass max_cache_len: launches are shaped for the capacity")
+    ap.add_argument("--no-also", action="store_true", help="leave the 8B-shaped record out of the default line")
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="keep timing K-step blocks until this much is timed")
     return ap.parse_args()
 
 
 def get_config(args):
     from paper_2506_14158_b200 import workloads as W
 
-    if args.workload == "sweep":
-        return W.sweep_config(args.L, args.T, args.B, args.layers)
-    return W.CONFIGS[args.workload]
+    from dataclasses import replace
+
+    cfg = W.sweep_config(args.L, args.T, args.B, args.layers) if args.workload == "sweep" else W.CONFIGS[args.workload]
+    return replace(cfg, capacity=args.capacity) if args.capacity else cfg
 
 
 def peaks():
@@ -103,8 +116,12 @@ def algorithmic_bytes(cfg, temperature, accept_lens):
         # other rows are never needed: every logits row once, logits and draft probabilities of the walked rows once more
         accept = cfg.B * cfg.T * cfg.V * 4 + rows * cfg.V * 8
     compact = cfg.n_layers * 2 * 2 * cfg.Hkv * rows * cfg.d * s + 2 * rows * cfg.hid * s
+    # the same step counted as "every logits row and every draft-probability row once" (B*T*V*8 when sampling), whether or
+    # not the kernels need the draft probabilities of rows the walk never visits
+    accept_all_rows = cfg.B * cfg.T * cfg.V * (8 if temperature > 0 else 4)
     return dict(attention_per_layer=attn_layer, attention=attn_layer * cfg.n_layers, accept=accept, compact=compact,
-                total=attn_layer * cfg.n_layers + accept + compact)
+                total=attn_layer * cfg.n_layers + accept + compact, accept_all_rows=accept_all_rows,
+                total_all_rows=attn_layer * cfg.n_layers + accept_all_rows + compact)
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -149,46 +166,54 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- oracle timing (CPU)
-def oracle_sample(cfg, temperature, layers_sample=None):
-    """Times the float64 oracle, as it stands, on a bounded sample of the workload: `layers_sample` attention
-    layers (default: as many as fit ~10 s, at least one), the whole acceptance, and the compaction of those
-    layers; the attention and compaction times are scaled to n_layers.  Returns (seconds per step, description)."""
+def oracle_sample(cfg, temperature, layers_sample=None, threads=None, budget_s=10.0):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload: one untimed attention layer, then
+    `layers_sample` timed ones (default: as many as fit about `budget_s` seconds, at least one) -- their MEAN is the
+    layer time --, the whole acceptance, and the compaction of one layer; attention and compaction are scaled to
+    n_layers.  `threads`: OpenMP threads (default: all the oracle would use).  Returns (seconds per step, description,
+    acceptance result)."""
     import numpy as np
 
     import oracle
     from paper_2506_14158_b200 import workloads as W
 
-    parent = W.make_trees(cfg)
-    x = W.make_accept_inputs(cfg, parent, temperature, token_mode="topk")
-    cl = np.full(cfg.B, cfg.L, dtype=np.int32)
-    q, k, v = W.make_attention_inputs(cfg, 0)
-    q64, k64, v64 = W.to_f64(q), W.to_f64(k), W.to_f64(v)
-    t = time.perf_counter()
-    oracle.tree_attention(q64, k64, v64, cl, parent)
-    t_layer = time.perf_counter() - t
-    n_s = layers_sample or max(1, min(cfg.n_layers, int(10.0 / max(t_layer, 1e-3))))
-    for _ in range(n_s - 1):
+    all_threads = oracle.max_threads()
+    if threads:
+        oracle.set_threads(threads)
+    try:
+        parent = W.make_trees(cfg)
+        x = W.make_accept_inputs(cfg, parent, temperature, token_mode="topk")
+        cl = np.full(cfg.B, cfg.L, dtype=np.int32)
+        q, k, v = W.make_attention_inputs(cfg, 0)
+        q64, k64, v64 = W.to_f64(q), W.to_f64(k), W.to_f64(v)
         t = time.perf_counter()
-        oracle.tree_attention(q64, k64, v64, cl, parent)
-        t_layer = min(t_layer, time.perf_counter() - t) if n_s > 4 else (t_layer + time.perf_counter() - t)
-    if n_s <= 4:
-        t_layer /= n_s
-    t = time.perf_counter()
-    tau = float(np.float32(temperature))
-    if tau > 0:
-        r = oracle.accept_stochastic(x["logits"], x["draft_probs"], x["tokens"], parent, tau, x["uniforms"],
-                                     max_depth=cfg.max_depth)
-    else:
-        r = oracle.accept_greedy(x["logits"], x["tokens"], parent, max_depth=cfg.max_depth)
-    t_accept = time.perf_counter() - t
-    bits = k.view(torch_int_dtype(k)).numpy().copy()
-    kc, vc = [bits.copy()], [bits.copy()]
-    t = time.perf_counter()
-    oracle.kv_compact(kc, vc, cl.copy(), r["path"], r["accept_len"], cfg.T)
-    t_compact = time.perf_counter() - t
+        oracle.tree_attention(q64, k64, v64, cl, parent)  # untimed in the figure: first touch of the arrays, thread start-up
+        t_first = time.perf_counter() - t
+        n_s = layers_sample or max(1, min(cfg.n_layers, int(budget_s / max(t_first, 1e-3))))
+        t = time.perf_counter()
+        for _ in range(n_s):
+            oracle.tree_attention(q64, k64, v64, cl, parent)
+        t_layer = (time.perf_counter() - t) / n_s
+        t = time.perf_counter()
+        tau = float(np.float32(temperature))
+        if tau > 0:
+            r = oracle.accept_stochastic(x["logits"], x["draft_probs"], x["tokens"], parent, tau, x["uniforms"],
+                                         max_depth=cfg.max_depth)
+        else:
+            r = oracle.accept_greedy(x["logits"], x["tokens"], parent, max_depth=cfg.max_depth)
+        t_accept = time.perf_counter() - t
+        bits = k.view(torch_int_dtype(k)).numpy().copy()
+        kc, vc = [bits.copy()], [bits.copy()]
+        t = time.perf_counter()
+        oracle.kv_compact(kc, vc, cl.copy(), r["path"], r["accept_len"], cfg.T)
+        t_compact = time.perf_counter() - t
+        used = threads or all_threads
+    finally:
+        if threads:
+            oracle.set_threads(all_threads)
     total = t_layer * cfg.n_layers + t_accept + t_compact * cfg.n_layers
-    desc = (f"float64 C oracle, {oracle.max_threads()} OpenMP threads: {n_s} attention layer(s) of {cfg.n_layers} timed "
-            f"({t_layer * 1e3:.1f} ms each), whole acceptance ({t_accept * 1e3:.1f} ms), compaction of 1 layer "
+    desc = (f"float64 C oracle, {used} OpenMP thread(s): mean of {n_s} attention layer(s) of {cfg.n_layers} after one "
+            f"untimed ({t_layer * 1e3:.1f} ms each), whole acceptance ({t_accept * 1e3:.1f} ms), compaction of 1 layer "
             f"({t_compact * 1e3:.2f} ms); attention and compaction scaled to {cfg.n_layers} layers")
     return total, desc, r
 
@@ -208,26 +233,32 @@ def run_reference(args):
     cfg = get_config(args)
     times = []
     steps = max(1, min(args.steps, 3))
+    # every step is the same bounded sample that the CUDA arm's cpu_baseline quotes (about 3 s of attention layers, the
+    # whole acceptance, one layer's compaction), so the two figures describe the same thing
     for _ in range(min(args.warmup, 1)):
         oracle_sample(cfg, args.temperature, layers_sample=1)
     desc = ""
     for _ in range(steps):
-        t, desc, _ = oracle_sample(cfg, args.temperature, layers_sample=1)
+        t, desc, _ = oracle_sample(cfg, args.temperature, budget_s=3.0)
         times.append(t)
     tstep = statistics.median(times)
     value = cfg.B * cfg.T / tstep
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=steps,
                 warmup=min(args.warmup, 1), ms_per_step=tstep * 1e3, higher_is_better=True, scaling="weak",
-                vs_baseline=None, dtype="f64", data="synthetic (seeded)",
-                config=dict(workload=cfg.name, B=cfg.B, T=cfg.T, L=cfg.L, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, V=cfg.V,
-                            n_layers=cfg.n_layers, temperature=args.temperature),
+                vs_baseline=None, dtype="f64", data="synthetic (seeded)", config=config_record(cfg, args, 1),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.max_threads(), kind="oracle", sample=desc),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line), flush=True)
 
 
+def config_record(cfg, args, world):
+    """The `config` object of a line: identical keys in both arms, so that they can be compared field by field."""
+    return dict(workload=cfg.name, B=cfg.B, T=cfg.T, L=cfg.L, C=cfg.C, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, V=cfg.V,
+                n_layers=cfg.n_layers, temperature=args.temperature)
+
+
 # ----------------------------------------------------------------------------- the CUDA arm
-def build_step(cfg, temperature, device, seed_shift=0):
+def build_step(cfg, temperature, device, seed_shift=0, hint=True):
     import numpy as np
     import torch
 
@@ -263,7 +294,8 @@ def build_step(cfg, temperature, device, seed_shift=0):
     step = VerifyStep(qs, ks, vs, torch.full((cfg.B,), cfg.L, dtype=torch.int32, device=device), to(parent),
                       to(x["tokens"]), to(x["logits"]), to(x["draft_probs"]) if stoch else None,
                       to(x["uniforms"]) if stoch else None, temperature, cfg.max_depth,
-                      feat_in=W.make_features(cfg_gen).to(device), stacked=(q_all, k_all, v_all))
+                      feat_in=W.make_features(cfg_gen).to(device), stacked=(q_all, k_all, v_all),
+                      max_cache_len=cfg.L if hint else 0)  # what a host that tracks its sequences' lengths knows
     return step
 
 
@@ -277,11 +309,116 @@ def time_graph(graph, iters, torch):
     return e0.elapsed_time(e1) / iters  # ms per replay
 
 
+def time_blocks(graph, iters, torch, min_seconds, max_blocks=200):
+    """Blocks of `iters` replays, each between its own pair of CUDA events, until `min_seconds` have been timed
+    (at least one block).  Returns the list of ms-per-replay figures, one per block."""
+    out, total = [], 0.0
+    while not out or (total < min_seconds * 1e3 and len(out) < max_blocks):
+        ms = time_graph(graph, iters, torch)
+        out.append(ms)
+        total += ms * iters
+    return out
+
+
+def measure(cfg, args, device, rank, world, with_e2e):
+    """Times one workload on this rank: the whole-step graph (K-step blocks), then the attention launches, acceptance
+    and compaction alone.  Returns a dict of raw figures (milliseconds, max over ranks where a rank count matters)."""
+    import torch
+
+    from paper_2506_14158_b200 import replicas
+
+    K, Wm = args.steps, max(3, args.warmup)
+    step = build_step(cfg, args.temperature, device, seed_shift=rank, hint=not args.no_hint)
+    g_step = step.capture("step")
+    g_attn = step.capture("attention")
+    g_acc = step.capture("accept")
+    g_cmp = step.capture("compact")
+
+    def barrier():
+        replicas.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(Wm):
+        g_step.replay()
+    barrier()
+    sampler = ClockSampler(device.index) if rank == 0 else None
+    t0 = time.time()
+    blocks = time_blocks(g_step, K, torch, args.min_seconds)  # the first block is the K steps of the contract
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    # dominant-kernel leg: the n_layers attention launches alone, same buffers, same stream, CUDA events
+    step.reset_lengths()  # the step's compaction advanced the lengths: attention is timed on the committed ones
+    for _ in range(3):
+        g_attn.replay()
+    torch.cuda.synchronize()
+    attn_blocks = time_blocks(g_attn, K, torch, args.min_seconds / 2)
+    ms_acc = time_graph(g_acc, K, torch)  # L2-resident when the logits fit L2: informational only
+    ms_cmp = time_graph(g_cmp, K, torch)
+    ms_e2e = 0.0
+    if with_e2e:
+        # end to end: per-step inputs from pinned host memory, decision back to the host, every step
+        step.bind_host_inputs()
+        for _ in range(3):
+            step.run_host()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        Ke = max(5, min(K, 50))
+        e0.record()
+        for _ in range(Ke):
+            step.run_host()
+        e1.record()
+        e1.synchronize()
+        ms_e2e = e0.elapsed_time(e1) / Ke
+    accept_lens = step.accept_len.cpu().tolist()
+    ms_first, ms_med, ms_best, ms_attn, ms_attn_best, ms_e2e = replicas.max_over_ranks(
+        [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
+        device=device)
+    rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               clocks=clocks, K=K, Wm=Wm)
+    return rec
+
+
+TARGET_FRAC = 0.70  # of HBM peak, for the whole step on the 7B- and 8B-shaped configurations
+
+
+def roofline_records(cfg, args, rec, pk):
+    """`step_hbm`, `roofline` and `breakdown_ms` of one measured workload."""
+    ab = algorithmic_bytes(cfg, args.temperature, rec["accept_lens"])
+    ms = rec["ms_median"]
+    attn_launch_ms = rec["ms_attn"] / cfg.n_layers
+    achieved = ab["attention_per_layer"] / (attn_launch_ms * 1e-3) / 1e9
+    flops_layer = 4.0 * cfg.B * cfg.Hq * cfg.T * (cfg.L + cfg.T) * cfg.d
+    tflops = flops_layer / (attn_launch_ms * 1e-3) / 1e12
+    step_gbs = ab["total"] / (ms * 1e-3) / 1e9
+    step_hbm = dict(algorithmic_bytes=ab["total"], achieved_gbs=step_gbs, frac_of_measured_peak=step_gbs / pk["hbm_gbs"],
+                    frac_of_nominal_8tbs=step_gbs / 8000.0, target_frac=TARGET_FRAC,
+                    accept_bytes_counted=ab["accept"], accept_bytes_all_rows=ab["accept_all_rows"],
+                    frac_of_measured_peak_all_rows=ab["total_all_rows"] / (ms * 1e-3) / 1e9 / pk["hbm_gbs"])
+    # intensity of the contraction: G*T flop per byte of K/V; above the ridge of this GPU the tensor pipe is the roof
+    intensity = (cfg.Hq // cfg.Hkv) * cfg.T
+    ridge = pk["bf16_tflops"] * 1e3 / pk["hbm_gbs"]
+    hbm = dict(achieved=achieved, peak=pk["hbm_gbs"], unit="GB/s", frac=achieved / pk["hbm_gbs"],
+               peak_source=pk["source"] + " copy bandwidth")
+    tensor = dict(achieved=tflops, peak=pk["bf16_tflops"], unit="TFLOP/s", frac=tflops / pk["bf16_tflops"],
+                  peak_source=pk["source"] + " sustained bf16 GEMM")
+    bound = "tensor" if intensity >= ridge else "hbm"
+    roofline = dict(kernel="tree_attention (one layer)", bound=bound, **(tensor if bound == "tensor" else hbm),
+                    target_frac=TARGET_FRAC, traffic=ncu_traffic(cfg.name),
+                    algorithmic_bytes_per_launch=ab["attention_per_layer"], flops_per_launch=flops_layer,
+                    us_per_launch=attn_launch_ms * 1e3, us_per_launch_best=rec["ms_attn_best"] / cfg.n_layers * 1e3,
+                    flop_per_kv_byte=intensity, ridge_flop_per_byte=ridge, hbm=hbm, tensor=tensor)
+    breakdown = dict(attention_all_layers=rec["ms_attn"], accept=rec["ms_acc"], compact=rec["ms_cmp"])
+    return ab, step_hbm, roofline, breakdown
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
 
     from paper_2506_14158_b200 import replicas
+    from paper_2506_14158_b200 import workloads as W
 
     rank, world, local = replicas.env_rank_world()
     if world != args.gpus:
@@ -298,92 +435,71 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     cfg = get_config(args)
-    K, Wm = args.steps, max(3, args.warmup)
-    step = build_step(cfg, args.temperature, device, seed_shift=rank)
-    g_step = step.capture("step")
-    g_attn = step.capture("attention")
-    g_acc = step.capture("accept")
-    g_cmp = step.capture("compact")
+    rec = measure(cfg, args, device, rank, world, with_e2e=True)
+    step, K, Wm = rec["step"], rec["K"], rec["Wm"]
+    h2d, d2h = step.h2d_bytes, step.d2h_bytes
+    launches = K * rec["n_blocks"] * step.launches_per_step(attn_kernels_per_layer(cfg))
+    rec["step"] = None
+    del step
+    also = None
+    if cfg.name == "c2x32" and not args.no_also and not args.capacity:
+        # the 8B-shaped step, measured the same way in the same run (no host-buffer leg: 365 MB per step over PCIe)
+        import gc
 
-    def barrier():
-        replicas.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(Wm):
-        g_step.replay()
-    barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
-    t0 = time.time()
-    ms = time_graph(g_step, K, torch)
-    barrier()
-    t1 = time.time()
-    clocks = sampler.stop(t0, t1) if sampler else None
-    # dominant-kernel leg: the n_layers attention launches alone, same buffers, same stream, CUDA events
-    step.reset_lengths()  # the step's compaction advanced the lengths: attention is timed on the committed ones
-    for _ in range(3):
-        g_attn.replay()
-    torch.cuda.synchronize()
-    ms_attn = time_graph(g_attn, K, torch)
-    ms_acc = time_graph(g_acc, K, torch)  # L2-resident when the logits fit L2: informational only
-    ms_cmp = time_graph(g_cmp, K, torch)
-    # end to end: per-step inputs from pinned host memory, decision back to the host, every step
-    step.bind_host_inputs()
-    for _ in range(3):
-        step.run_host()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    Ke = max(5, min(K, 50))
-    e0.record()
-    for _ in range(Ke):
-        step.run_host()
-    e1.record()
-    e1.synchronize()
-    ms_e2e = e0.elapsed_time(e1) / Ke
-    accept_lens = step.accept_len.cpu().tolist()
-
-    ms, ms_attn, ms_e2e = replicas.max_over_ranks([ms, ms_attn, ms_e2e], device=device)
+        gc.collect()
+        torch.cuda.empty_cache()
+        cfg2 = W.CONFIGS["c4x32"]
+        rec2 = measure(cfg2, args, device, rank, world, with_e2e=False)
+        launches += K * rec2["n_blocks"] * rec2["step"].launches_per_step(attn_kernels_per_layer(cfg2))
+        rec2["step"] = None
+        also = (cfg2, rec2)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     pk = peaks()
-    ab = algorithmic_bytes(cfg, args.temperature, accept_lens)
+    ab, step_hbm, roofline, breakdown = roofline_records(cfg, args, rec, pk)
     nodes = cfg.B * cfg.T * world
-    attn_launch_ms = ms_attn / cfg.n_layers
-    achieved = ab["attention_per_layer"] / (attn_launch_ms * 1e-3) / 1e9
-    flops_layer = 4.0 * cfg.B * cfg.Hq * cfg.T * (cfg.L + cfg.T) * cfg.d
-    attn_kernels = attn_kernels_per_layer(cfg)
+    ms = rec["ms"]
+    accept_lens = rec["accept_lens"]
+    config = config_record(cfg, args, world)
+    config.update(parallelism=f"replicas x{world} (no collective)",
+                  l2="inputs larger than L2 (independent KV cache per layer)" if ab["attention"] > (126 << 20)
+                  else "working set fits L2: launch-latency case, not a bandwidth claim",
+                  launch="whole step replayed as one CUDA graph",
+                  max_cache_len_hint=0 if args.no_hint else cfg.L)
     line = dict(
-        metric=METRIC, value=replicas.aggregate_nodes_per_second(cfg.B * cfg.T, world, ms), unit=UNIT, n_gpus=world, steps=K, warmup=Wm, ms_per_step=ms,
-        higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if cfg.dtype == "bf16" else "f32",
-        data="synthetic (seeded)",
-        config=dict(workload=cfg.name, B=cfg.B, T=cfg.T, L=cfg.L, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, V=cfg.V,
-                    n_layers=cfg.n_layers, temperature=args.temperature, parallelism=f"replicas x{world} (no collective)",
-                    l2="inputs larger than L2 (independent KV cache per layer)" if ab["attention"] > (126 << 20)
-                    else "working set fits L2: launch-latency case, not a bandwidth claim",
-                    launch="whole step replayed as one CUDA graph"),
-        step_hbm=dict(algorithmic_bytes=ab["total"], achieved_gbs=ab["total"] / (ms * 1e-3) / 1e9,
-                      frac_of_measured_peak=ab["total"] / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                      frac_of_nominal_8tbs=ab["total"] / (ms * 1e-3) / 1e9 / 8000.0),
-        roofline=dict(kernel="tree_attention (one layer)", bound="hbm", achieved=achieved, peak=pk["hbm_gbs"],
-                      unit="GB/s", frac=achieved / pk["hbm_gbs"], peak_source=pk["source"] + " copy bandwidth",
-                      traffic=ncu_traffic(cfg.name), algorithmic_bytes_per_launch=ab["attention_per_layer"],
-                      us_per_launch=attn_launch_ms * 1e3, tensor_tflops=flops_layer / (attn_launch_ms * 1e-3) / 1e12),
-        breakdown_ms=dict(attention_all_layers=ms_attn, accept=ms_acc, compact=ms_cmp),
-        e2e=dict(value=nodes / (ms_e2e * 1e-3), unit=UNIT, h2d_bytes_per_step=step.h2d_bytes,
-                 d2h_bytes_per_step=step.d2h_bytes, ms_per_step=ms_e2e),
-        gpu_launches=K * step.launches_per_step(attn_kernels),
+        metric=METRIC, value=replicas.aggregate_nodes_per_second(cfg.B * cfg.T, world, ms), unit=UNIT, n_gpus=world,
+        steps=K, warmup=Wm, ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic (seeded)", config=config,
+        timing=dict(blocks=rec["n_blocks"], steps_per_block=K, ms_per_step_first_block=ms,
+                    ms_per_step_median=rec["ms_median"], ms_per_step_best=rec["ms_best"],
+                    note="value and ms_per_step are the first block (exactly K steps); step_hbm and roofline use the medians"),
+        step_hbm=step_hbm, roofline=roofline, breakdown_ms=breakdown,
+        e2e=dict(value=nodes / (rec["ms_e2e"] * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                 ms_per_step=rec["ms_e2e"]),
+        gpu_launches=launches,
         accepted_per_step=dict(accept_len=accept_lens, mean_accepted_plus_bonus=sum(a + 1 for a in accept_lens) / len(accept_lens)),
-        clocks=clocks,
+        clocks=rec["clocks"],
         paper_context="S4C reports 2.26x-2.60x end-to-end speedup (A100 / 4x RTX 4090, FP16, batch 1); no verify-step number",
     )
+    if also is not None:
+        cfg2, rec2 = also
+        ab2, step_hbm2, roofline2, breakdown2 = roofline_records(cfg2, args, rec2, pk)
+        line["also"] = dict(workload=cfg2.name, config=config_record(cfg2, args, world),
+                            value=replicas.aggregate_nodes_per_second(cfg2.B * cfg2.T, world, rec2["ms"]), unit=UNIT,
+                            ms_per_step=rec2["ms"], ms_per_step_median=rec2["ms_median"], ms_per_step_best=rec2["ms_best"],
+                            blocks=rec2["n_blocks"], step_hbm=step_hbm2, roofline=roofline2, breakdown_ms=breakdown2,
+                            accept_len=rec2["accept_lens"], clocks=rec2["clocks"])
     if not args.no_cpu_baseline and world == 1:
-        t_cpu, desc, ref = oracle_sample(cfg, args.temperature)
         import oracle
 
+        t_cpu, desc, ref = oracle_sample(cfg, args.temperature)
+        t_one, desc_one, _ = oracle_sample(cfg, args.temperature, layers_sample=2, threads=1)
         line["cpu_baseline"] = dict(value=cfg.B * cfg.T / t_cpu, unit=UNIT, cores=oracle.max_threads(), kind="oracle",
-                                    sample=desc)
+                                    sample=desc + " -- this all-thread figure is the one quoted as `value`",
+                                    single_thread=dict(value=cfg.B * cfg.T / t_one, unit=UNIT, cores=1, sample=desc_one))
         line["parity_in_bench"] = dict(accept_len_matches_oracle=[int(a) for a in ref["accept_len"]] == accept_lens)
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -395,6 +511,7 @@ def run_sweep_all(args):
     trees of 16..128 nodes, batch 1/4/16.  One JSON line per point (nodes/s, HBM GB/s of the step and of the attention
     launches); points whose 32 caches do not fit the device are recorded as such, never aliased."""
     import gc
+    from dataclasses import replace
 
     import torch
 
@@ -410,13 +527,18 @@ def run_sweep_all(args):
         for T in (16, 32, 64, 128):
             for L in (512, 1024, 2048, 4096, 8192, 16384, 32768):
                 cfg = W.sweep_config(L, T, B, args.layers)
+                if args.capacity:
+                    if args.capacity < L + T:
+                        continue
+                    cfg = replace(cfg, capacity=args.capacity)
                 kv = 2 * cfg.n_layers * cfg.B * cfg.Hkv * cfg.C * cfg.d * 2
-                point = dict(workload=cfg.name, B=B, T=T, L=L, n_layers=cfg.n_layers, kv_gb=round(kv / 1e9, 2))
+                point = dict(workload=cfg.name, B=B, T=T, L=L, C=cfg.C, hint=0 if args.no_hint else L,
+                             n_layers=cfg.n_layers, kv_gb=round(kv / 1e9, 2))
                 if kv > 0.8 * total_b:
                     point["result"] = "exceeds device memory"
                     print(json.dumps(point), flush=True)
                     continue
-                step = build_step(cfg, args.temperature, device)
+                step = build_step(cfg, args.temperature, device, hint=not args.no_hint)
                 g_step, g_attn = step.capture("step"), step.capture("attention")
                 iters = 20 if kv < (8 << 30) else 5
                 for _ in range(3):
@@ -438,6 +560,54 @@ def run_sweep_all(args):
                 torch.cuda.empty_cache()
 
 
+def run_launch_floor(args):
+    """The floor under one per-layer launch: CUDA graphs of `--layers` EMPTY kernels (s4c_launch_floor) with the launch
+    shape of an attention launch -- block size, dynamic shared memory, cluster size, tensor-memory allocation, cluster
+    barriers, programmatic dependent launch -- timed like the attention graph.  One JSON line per shape."""
+    import torch
+
+    import __graft_entry__ as entry
+
+    entry.build()
+    from paper_2506_14158_b200 import s4c
+
+    torch.cuda.set_device(0)
+    word = torch.full((1,), 1024, dtype=torch.int32, device="cuda")
+    n = args.layers
+    shapes = [  # (name, ctas, cluster, threads, smem, tmem columns, cluster barriers, dependent launch)
+        ("bare: 128 CTAs x 224 threads, 1 KB", 128, 1, 224, 1024, 0, 0, False),
+        ("+ programmatic dependent launch", 128, 1, 224, 1024, 0, 0, True),
+        ("+ 200 KB shared memory", 128, 1, 224, 200 * 1024, 0, 0, True),
+        ("+ 256 tensor-memory columns", 128, 1, 224, 200 * 1024, 256, 0, True),
+        ("+ clusters of 4", 128, 4, 224, 200 * 1024, 256, 0, True),
+        ("+ 1 cluster barrier (7B shape, pushed partials)", 128, 4, 224, 200 * 1024, 256, 1, True),
+        ("+ 2 cluster barriers (parked partials)", 128, 4, 224, 200 * 1024, 256, 2, True),
+        ("same without dependent launch", 128, 4, 224, 200 * 1024, 256, 1, False),
+        ("148 CTAs, no cluster, dependent launch", 148, 1, 224, 200 * 1024, 256, 0, True),
+        ("8B shape: 128 CTAs x 384 threads, clusters of 4, 512 columns, 2 barriers", 128, 4, 384, 220 * 1024, 512, 2, True),
+        ("half-SM CTAs: 296 x 224 threads, 100 KB, 256 columns", 296, 1, 224, 100 * 1024, 256, 0, True),
+    ]
+    for name, ctas, cluster, threads, smem, tmem, syncs, pdl in shapes:
+        fn = lambda: [s4c.launch_floor(ctas, cluster, threads, smem, tmem, syncs, pdl, word) for _ in range(n)]
+        st = torch.cuda.Stream()
+        st.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(st):
+            fn()
+        torch.cuda.current_stream().wait_stream(st)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        for _ in range(5):
+            g.replay()
+        torch.cuda.synchronize()
+        blocks = time_blocks(g, args.steps, torch, 0.2)
+        print(json.dumps(dict(workload="launch-floor", shape=name, ctas=ctas, cluster=cluster, threads=threads,
+                              smem_bytes=smem, tmem_cols=tmem, cluster_barriers=syncs, dependent_launch=pdl,
+                              launches_per_graph=n, us_per_launch_median=round(statistics.median(blocks) / n * 1e3, 3),
+                              us_per_launch_best=round(min(blocks) / n * 1e3, 3))), flush=True)
+
+
 def attn_kernels_per_layer(cfg):
     from paper_2506_14158_b200 import s4c
     import torch
@@ -450,6 +620,8 @@ if __name__ == "__main__":
     a = parse_args()
     if a.workload == "sweep-all":
         run_sweep_all(a)
+    elif a.workload == "launch-floor":
+        run_launch_floor(a)
     elif a.impl == "reference":
         run_reference(a)
     else:

@@ -22,9 +22,9 @@
  *     sequence, mark its outputs (accept_len = -1) and never trap or assert.
  *   - Base pointers of tensors must be 16-byte aligned.  All tensors are dense, row-major,
  *     innermost dimension last.
- *   - Tree order: node 0 is the root (the last committed token, Section 3.2: "begins with
- *     the prefix ... as the root node"), parent[0] = -1 and 0 <= parent[i] < i.  A batch may
- *     pad trees to T nodes; n_nodes[b] gives the real count (NULL = T everywhere).
+ *   - Tree order: node 0 is the root, i.e. the last committed token of the prefix (Section 3.2,
+ *     Figure 3), parent[0] = -1 and 0 <= parent[i] < i.  A batch may pad trees to T nodes;
+ *     n_nodes[b] gives the real count (NULL = T everywhere).
  *   - Limits: 1 <= T <= 128, d in {64, 128}, Hq % Hkv == 0.
  */
 #ifndef S4C_H_
@@ -58,6 +58,7 @@ typedef enum { S4C_F32 = 0, S4C_BF16 = 1 } s4c_dtype;
 #define S4C_SEQ_DEPTH 8       /* a node deeper than max_depth / accept_len > max_depth */
 #define S4C_SEQ_BAD_PATH 16   /* path not of the form 0 = path[0] < path[1] < ... < T */
 #define S4C_SEQ_TIMEOUT 32    /* a bounded in-kernel wait expired (OR-ed in; results of that sequence are invalid) */
+#define S4C_SEQ_NONFINITE 64  /* a target-logit row of a real node holds a NaN or +Inf, or nothing but -Inf */
 
 typedef void* s4c_stream_t; /* a cudaStream_t */
 
@@ -66,8 +67,8 @@ int s4c_version(void);
 const char* s4c_status_string(s4c_status code);
 
 /* ------------------------------------------------------------------------------------------
- * s4c_tree_attention -- Section 3.2 ("a tree mask is applied") and Figure 3 (tree mask matrix);
- * the single target forward pass that verifies all drafts at once (Sections 1 and 2).
+ * s4c_tree_attention -- the tree-masked attention of the verification pass (Section 3.2; the
+ * mask is drawn in Figure 3): one target forward pass verifies all drafts at once (Sections 1, 2).
  *
  * For sequence b, query head h and tree node i the output is softmax attention of q[b,h,i,:]
  * over the cache slots 0..L_b-1 (the committed prefix, fully visible) and the slots L_b+t of the
@@ -85,24 +86,35 @@ const char* s4c_status_string(s4c_status code);
  *   n_nodes    [B] or NULL  int32
  *   out        [B,Hq,T,d]   dt     rows of padding nodes (i >= n_nodes[b]) are written as zeros;
  *                                  rows of a flagged sequence are left untouched
+ *   C          capacity of the caches in slots (what the tensors are laid out for)
+ *   max_cache_len  what the host knows about the live lengths: an upper bound on cache_len[b] over
+ *              the batch, or 0 if it knows nothing (the capacity then stands in).  A serving cache has
+ *              C = the longest context it may ever hold while the sequences are far shorter; the host
+ *              cannot read cache_len (device memory, no synchronisation), so the split of the cache
+ *              over CTAs, the kernel variant and the grid are chosen for min(C, max_cache_len + T)
+ *              slots.  The value steers the launch shape only: results are the same for any value,
+ *              and a sequence longer than the bound is still handled correctly (only slower).
+ *              Negative: S4C_ERR_SHAPE.
  *   scale      0 selects 1/sqrt(d)
  *   status     [B] or NULL  int32  S4C_SEQ_BAD_PARENT, S4C_SEQ_CAPACITY
  *   workspace  at least s4c_tree_attention_workspace_bytes(...) bytes, 256-byte aligned; holds the
- *              split-KV partial results; contents are scratch, nothing needs clearing.
+ *              split-KV partial results; contents are scratch, nothing needs clearing.  The query
+ *              takes the capacity C and covers every max_cache_len.
  * Calls sharing a workspace must be ordered on the stream.
  * ------------------------------------------------------------------------------------------ */
 size_t s4c_tree_attention_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt);
 
 s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_cache,
                               const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
-                              void* out, int B, int T, int Hq, int Hkv, int d, int C, s4c_dtype dt,
-                              float scale, int32_t* status, void* workspace, size_t workspace_bytes,
-                              s4c_stream_t stream);
+                              void* out, int B, int T, int Hq, int Hkv, int d, int C, int max_cache_len,
+                              s4c_dtype dt, float scale, int32_t* status, void* workspace,
+                              size_t workspace_bytes, s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
- * s4c_tree_accept -- Section 2 "Speculative Sampling" (accept with probability min(1, p/q), else
- * resample from norm(max(0, p - q))), Eq. 11 and Eq. 12 of Section 3.2, the longest accepted path
- * of Section 3.2, and greedy decoding as used in Section 4.1.2.
+ * s4c_tree_accept -- the accept / resample rule of Section 2 ("Speculative Sampling"): a draft token
+ * passes with probability min(1, p/q), a rejected position is resampled from norm(max(0, p - q));
+ * Eq. 11 and Eq. 12 of Section 3.2 apply it along the tree, whose longest accepted path is kept
+ * (Section 3.2); greedy decoding is what Section 4.1.2 uses.
  *
  * temperature == 0: greedy.  g[n] = argmax_v target_logits[b,n,v] (lowest v on ties); node i is
  *   accepted iff its parent is and tokens[b,i] == g[parent]; the deepest accepted node e (lowest
@@ -126,8 +138,16 @@ s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_
  *   path          [B,max_depth+1] int32 out: node indices root..e, path[b,0] = 0, -1 beyond a
  *   next_token    [B]   int32  out: the bonus / resampled token (-1 for a flagged sequence)
  *   near_tie      [B,T] uint8  out or NULL: 1 where node i was tested with |p/q - u| < 1e-6
- *   status        [B] or NULL  S4C_SEQ_BAD_PARENT, S4C_SEQ_TOKEN_RANGE, S4C_SEQ_DEPTH
+ *   status        [B] or NULL  S4C_SEQ_BAD_PARENT, S4C_SEQ_TOKEN_RANGE, S4C_SEQ_DEPTH, S4C_SEQ_NONFINITE
  *   workspace     at least s4c_tree_accept_workspace_bytes(B,T,V) bytes, 256-byte aligned, scratch.
+ * Non-finite logits.  A -Inf logit beside finite ones is legal (that token has probability 0, as after a
+ * vocabulary mask).  A NaN or +Inf anywhere in the rows of the real nodes (i < n_nodes[b]), or a row holding
+ * nothing but -Inf, makes the softmax undefined: the sequence is flagged S4C_SEQ_NONFINITE and skipped
+ * (accept_len = next_token = -1), the other sequences of the batch are unaffected.  The check rides on the
+ * maximum reduction that reads every logit anyway.  draft_probs are taken as given (finite, >= 0): they are
+ * only read on the walked rows, so they are not screened.
+ * Any finite temperature > 0 is served; rows whose float spacing at the maximum exceeds 172 temperatures are
+ * summed as a count of their maxima (every other term is below e^-172 of the sum).
  * Returns S4C_ERR_SHAPE for temperature < 0 or NaN.
  * ------------------------------------------------------------------------------------------ */
 size_t s4c_tree_accept_workspace_bytes(int B, int T, int V);
@@ -192,6 +212,21 @@ s4c_status s4c_kv_compact(void* const* k_caches, void* const* v_caches, int n_la
                           const int32_t* path, const int32_t* accept_len, int max_depth,
                           const void* feat_in, void* feat_out, int B, int T, int Hkv, int d, int C, int hid,
                           s4c_dtype dt, int32_t* status, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * s4c_launch_floor -- a measurement aid; the paper has no counterpart.
+ *
+ * Enqueues an EMPTY kernel with the launch shape of an attention launch: `ctas` blocks of `threads`
+ * threads in clusters of `cluster`, `smem_bytes` of dynamic shared memory, `tmem_cols` tensor-memory
+ * columns allocated and freed (0, 32, ..., 512), `cluster_syncs` cluster barriers, the programmatic
+ * dependent-launch attribute if `dependent_launch` != 0, and one dependent read of `word` (device, may
+ * be NULL) after the wait for the previous launch.  Timed in a CUDA graph of n_layers such launches it
+ * gives the floor under one per-layer launch of a verify step (bench.py --workload launch-floor).
+ * `sink` (device, may be NULL) is never written in practice.  Shapes whose co-resident blocks would
+ * need more than 512 tensor-memory columns per SM are refused with S4C_ERR_UNSUPPORTED.
+ * ------------------------------------------------------------------------------------------ */
+s4c_status s4c_launch_floor(int ctas, int cluster, int threads, int smem_bytes, int tmem_cols, int cluster_syncs,
+                            int dependent_launch, const int32_t* word, int32_t* sink, s4c_stream_t stream);
 
 #ifdef __cplusplus
 }

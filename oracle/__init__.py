@@ -33,6 +33,7 @@ SEQ_TOKEN_RANGE = 2
 SEQ_CAPACITY = 4
 SEQ_DEPTH = 8
 SEQ_BAD_PATH = 16
+SEQ_NONFINITE = 64
 
 
 def build(force: bool = False) -> str:

@@ -9,8 +9,8 @@
  * What it computes (each function cites the passage of the S4C paper,
  * arXiv 2506.14158, that defines the operation):
  *
- *   s4c_oracle_tree_attention  Section 3.2 ("a tree mask is applied") and the
- *                              caption of Figure 3 (tree mask matrix): every
+ *   s4c_oracle_tree_attention  Section 3.2 (the verification pass uses a tree
+ *                              mask) and Figure 3 (where the mask is drawn): every
  *                              tree token attends the cached prefix and its own
  *                              root path.  Written out as the definition of
  *                              masked softmax attention; no tiling, no online
@@ -68,6 +68,7 @@
 #define ORC_SEQ_CAPACITY 4
 #define ORC_SEQ_DEPTH 8
 #define ORC_SEQ_BAD_PATH 16
+#define ORC_SEQ_NONFINITE 64
 
 int s4c_oracle_max_threads(void) {
 #ifdef _OPENMP
@@ -200,6 +201,23 @@ static int validate_accept_inputs(const int32_t* par, const int32_t* tok, int n,
     return st;
 }
 
+/* Input validation of the acceptance calls, not a step of the method: a target-logit row of a real
+ * node (i < n) is unusable when it holds a NaN or +Inf (the maximum-subtracted exponent would be
+ * Inf - Inf) or nothing but -Inf (no token has mass).  A -Inf logit beside finite ones is fine: the
+ * token simply has probability 0.  Such a sequence is flagged and skipped like a malformed tree. */
+static int logits_unusable(const float* logits, int n, int V) {
+    for (int i = 0; i < n; ++i) {
+        const float* row = logits + (size_t)i * V;
+        int any_finite = 0;
+        for (int v = 0; v < V; ++v) {
+            if (isnan(row[v]) || (isinf(row[v]) && row[v] > 0)) return 1;
+            if (!isinf(row[v])) any_finite = 1;
+        }
+        if (!any_finite) return 1;
+    }
+    return 0;
+}
+
 static int argmax_lowest(const float* row, int V) {
     int best = 0;
     for (int v = 1; v < V; ++v)
@@ -228,7 +246,8 @@ int s4c_oracle_accept_greedy(const float* logits, const int32_t* tokens, const i
         const int32_t* tok = tokens + (size_t)b * T;
         int32_t* pth = path + (size_t)b * (max_depth + 1);
         int* depth = (int*)malloc(sizeof(int) * (size_t)T);
-        const int st = validate_accept_inputs(par, tok, n, T, V, max_depth, depth);
+        int st = validate_accept_inputs(par, tok, n, T, V, max_depth, depth);
+        if (!(st & ORC_SEQ_BAD_PARENT) && logits_unusable(logits + (size_t)b * T * V, n, V)) st |= ORC_SEQ_NONFINITE;
         if (status) status[b] = st;
         if (st) {
             accept_len[b] = -1;
@@ -299,7 +318,8 @@ int s4c_oracle_accept_stochastic(const float* logits, const float* dprobs, const
         uint8_t* tie = near_tie ? near_tie + (size_t)b * T : NULL;
         if (tie) memset(tie, 0, (size_t)T);
         int* depth = (int*)malloc(sizeof(int) * (size_t)T);
-        const int st = validate_accept_inputs(par, tok, n, T, V, max_depth, depth);
+        int st = validate_accept_inputs(par, tok, n, T, V, max_depth, depth);
+        if (!(st & ORC_SEQ_BAD_PARENT) && logits_unusable(logits + (size_t)b * T * V, n, V)) st |= ORC_SEQ_NONFINITE;
         if (status) status[b] = st;
         if (st) {
             accept_len[b] = -1;

@@ -62,6 +62,16 @@ static inline size_t accept_ws_layout(int B, int T, int V, char* base, AcceptWor
 }
 
 // ----------------------------------------------------------------------------- reductions
+// Maximum that keeps a NaN (fmaxf drops it): a row with a NaN logit must be reported, not silently reduced.
+__device__ __forceinline__ float max_keep_nan(float a, float b) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+// A row maximum the method can work with: not NaN, not +Inf (the maximum-subtracted exponent would be Inf - Inf),
+// not -Inf (no token has any mass).  Single -Inf logits beside finite ones are fine: probability 0.
+__device__ __forceinline__ bool usable_max(float m) { return m > -INFINITY && m < INFINITY; }
+
 __device__ __forceinline__ void argmax_combine(float& m, int& i, float om, int oi) {
     if (om > m || (om == m && oi < i)) {
         m = om;
@@ -124,7 +134,7 @@ __device__ __forceinline__ double exp_nonpos(double t, const double* tab /* shar
     return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));  // * 2^(k >> 5), exponent stays normal
 }
 
-// exp_nonpos without the range test, for -700 < t <= 0.  The statistics kernels raise every logit to at least
+// exp_nonpos without the range test, for about -780 < t <= 0.  The statistics kernels raise every logit to at least
 // M - 690 tau first (one float max): a term that small is below 1e-299 of the row sum either way, so neither the sum
 // nor the residual mass can tell the difference, and the inner loop loses a compare and a branch per element.
 __device__ __forceinline__ double exp_fast(double t, const double* tab) {
@@ -141,9 +151,16 @@ __device__ __forceinline__ double exp_fast(double t, const double* tab) {
     pl = pl * r;
     const double tj = tab[k & 31];
     const double y = fma(tj, pl, tj);
-    return __hiloint2double(__double2hiint(y) + ((k >> 5) << 20), __double2loint(y));
+    // the float floor lets t undershoot -690 by up to ulp(M)/(2 tau): the exponent is held at 2^-1000 (an integer
+    // maximum, not a float64 instruction) so that it cannot wrap into the sign bit
+    return __hiloint2double(__double2hiint(y) + (max(k >> 5, -1000) << 20), __double2loint(y));
 }
 constexpr float kExpFloorSpan = 690.f;  // in units of tau
+// Rows whose float spacing at the maximum is coarser than 690 tau / 4 (a tiny temperature or enormous logits): the
+// float floor M - 690 tau is no longer usable (it may round to M itself), and every logit below the maximum is at least
+// ulp(M)/tau >= 172 below it in units of tau, i.e. under e^-172 of the maximum's term -- far below the rounding of the
+// sum.  Such rows are summed as the number of entries equal to the maximum.
+__device__ __forceinline__ bool degenerate_row(float m, float floor_span) { return floor_span < fabsf(m) * 4.8e-7f; }
 __device__ __forceinline__ void fill_exp_table(double* tab) {  // every thread of the CTA; the caller synchronises
     if (threadIdx.x < 32) tab[threadIdx.x] = kExp2Frac[threadIdx.x];
 }
@@ -193,18 +210,20 @@ accept_rowstats_kernel(const float* __restrict__ logits, const int32_t* __restri
     if (threadIdx.x == 32) idx_s = INT_MAX;
 
     // maximum first (one instruction per element); its lowest index is then looked up by the few threads that hold it
+    // (a NaN survives this maximum, so that the segment can be reported as unusable: see below)
     float mt = x[0];
 #pragma unroll
-    for (int k = 1; k < kElemsPerThread; ++k) mt = fmaxf(mt, x[k]);
+    for (int k = 1; k < kElemsPerThread; ++k) mt = max_keep_nan(mt, x[k]);
     float m = mt;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    for (int o = 16; o > 0; o >>= 1) m = max_keep_nan(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (lane == 0) sm[warp] = m;
     __syncthreads();
     m = sm[0];
 #pragma unroll
-    for (int w = 1; w < kRowThreads / 32; ++w) m = fmaxf(m, sm[w]);
-    if (mt == m) {
+    for (int w = 1; w < kRowThreads / 32; ++w) m = max_keep_nan(m, sm[w]);
+    const bool bad = !(m < INFINITY);  // a NaN or +Inf in the segment: the sequence will be flagged S4C_SEQ_NONFINITE
+    if (!bad && mt == m) {
 #pragma unroll
         for (int k = 0; k < kElemsPerThread; ++k) {  // a thread's element indices ascend with k
             const int e = elem_index<VEC>(s0, k);
@@ -218,11 +237,16 @@ accept_rowstats_kernel(const float* __restrict__ logits, const int32_t* __restri
     double S = 0.0;
     if (STOCH) {
         double s = 0.0;
-        if (m > -INFINITY) {
-            const float x_floor = m - floor_span;
-            const double c = -(double)m * inv_tau;
+        if (!bad && m > -INFINITY) {
+            if (degenerate_row(m, floor_span)) {
 #pragma unroll
-            for (int k = 0; k < kElemsPerThread; ++k) s += exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab);
+                for (int k = 0; k < kElemsPerThread; ++k) s += x[k] == m ? 1.0 : 0.0;
+            } else {
+                const float x_floor = m - floor_span;
+                const double c = -(double)m * inv_tau;
+#pragma unroll
+                for (int k = 0; k < kElemsPerThread; ++k) s += exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab);
+            }
         }
         S = block_sum(s, scratch);
     } else {
@@ -230,7 +254,7 @@ accept_rowstats_kernel(const float* __restrict__ logits, const int32_t* __restri
     }
     if (threadIdx.x == 0) {
         RowPartial r;
-        r.S = S, r.M = m, r.idx = idx_s;
+        r.S = S, r.M = bad ? INFINITY : m, r.idx = idx_s;  // +Inf marks the segment (and so its row) as unusable
         out[((size_t)b * T + node) * gridDim.x + split] = r;
     }
 }
@@ -388,15 +412,16 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     // ---- first reduction: maximum (one instruction per element), then its lowest index from the few threads that hold it
     float mt = x[0];
 #pragma unroll
-    for (int k = 1; k < kClEpt; ++k) mt = fmaxf(mt, x[k]);
+    for (int k = 1; k < kClEpt; ++k) mt = max_keep_nan(mt, x[k]);
     float m = mt;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    for (int o = 16; o > 0; o >>= 1) m = max_keep_nan(m, __shfl_xor_sync(0xffffffffu, m, o));
     if ((tid & 31) == 0) wm[tid >> 5] = m;
     if (tid == 0) wi[0] = INT_MAX;
     __syncthreads();
     m = wm[0];
-    for (int w = 1; w < THREADS / 32; ++w) m = fmaxf(m, wm[w]);
+    for (int w = 1; w < THREADS / 32; ++w) m = max_keep_nan(m, wm[w]);
+    if (!(m < INFINITY)) m = INFINITY;  // a NaN or +Inf: the row's maximum becomes +Inf, which the walk reports
     if (mt == m) {
 #pragma unroll
         for (int k = 0; k < kClEpt; ++k)  // a thread's element indices ascend with k
@@ -424,14 +449,23 @@ accept_stats_cluster_kernel(const float* __restrict__ logits, const float* __res
     // ---- second reduction: e = exp((x - M)/tau), once per element, kept in registers; S = sum e
     double e[kClEpt];
     double s = 0.0;
-    {
+    if (!usable_max(M)) {  // the walk flags the sequence; nothing below is used
+#pragma unroll
+        for (int k = 0; k < kClEpt; ++k) e[k] = 0.0;
+    } else if (degenerate_row(M, floor_span)) {
+#pragma unroll
+        for (int k = 0; k < kClEpt; ++k) {
+            e[k] = x[k] == M ? 1.0 : 0.0;
+            s += e[k];
+        }
+    } else {
         // elements beyond the row were loaded as -inf: raised to the floor like any other far-away logit, they add
         // less than 1e-299 of the row sum
         const float x_floor = M - floor_span;
         const double c = -(double)M * inv_tau;
 #pragma unroll
         for (int k = 0; k < kClEpt; ++k) {
-            e[k] = M > -INFINITY ? exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab) : 0.0;
+            e[k] = exp_fast(fma((double)fmaxf(x[k], x_floor), inv_tau, c), tab);
             s += e[k];
         }
     }
@@ -515,6 +549,48 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         __syncthreads();
         flags = sh.flag;
     }
+    if (!(flags & S4C_SEQ_BAD_PARENT)) {
+        // ---- per-node statistics into shared memory (n is in 1..T here), and the check that every row is usable
+        if (seg_row && STOCH) {
+            // statistics came per vocabulary segment: one warp per node, lane s takes segments s, s + 32, ...; the maximum
+            // and the sum go through fixed-order butterflies (the same on every run and in every CTA of the cluster)
+            const int lane = tid & 31;
+            for (int i = tid >> 5; i < n; i += blockDim.x >> 5) {
+                const RowPartial* part = seg_row + ((size_t)b * T + i) * seg_splits;
+                float M = -INFINITY;
+                int idx = INT_MAX;
+                for (int sg = lane; sg < seg_splits; sg += 32) argmax_combine(M, idx, part[sg].M, part[sg].idx);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float om = __shfl_xor_sync(0xffffffffu, M, o);
+                    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+                    argmax_combine(M, idx, om, oi);
+                }
+                double S = 0.0;
+                if (usable_max(M))
+                    for (int sg = lane; sg < seg_splits; sg += 32)
+                        if (part[sg].M > -INFINITY) S += part[sg].S * exp(((double)part[sg].M - (double)M) * inv_tau);
+                S = warp_sum(S);
+                if (lane == 0) sh.nS[i] = S, sh.nM[i] = M, sh.nArg[i] = idx, sh.nZ[i] = 0.0, sh.nQ[i] = 0.0;
+            }
+        }
+        for (int i = tid; i < n; i += blockDim.x) {
+            if (seg_row) {
+                if (!STOCH) {
+                    const NodeStats ns = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, false);
+                    sh.nArg[i] = ns.idx, sh.nM[i] = ns.M;
+                }
+            } else {
+                const NodeSummary ns = nodes[(size_t)b * T + i];
+                sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = ns.Z, sh.nQ[i] = ns.Q;
+            }
+        }
+        __syncthreads();
+        for (int i = tid; i < n; i += blockDim.x)
+            if (!usable_max(sh.nM[i])) atomicOr(&sh.flag, S4C_SEQ_NONFINITE);  // a NaN or +Inf logit, or a row of -Inf only
+        __syncthreads();
+        flags = sh.flag;
+    }
     if (tid == 0 && status && writer) status[b] = flags;
     if (flags) {  // the same in every CTA of the cluster: they all leave here, before any cluster barrier
         if (writer) {
@@ -522,39 +598,6 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
             if (tid == 0) accept_len[b] = -1, next_token[b] = -1;
         }
         return;
-    }
-    if (seg_row && STOCH) {
-        // statistics came per vocabulary segment: one warp per node, lane s takes segments s, s + 32, ...; the maximum
-        // and the sum go through fixed-order butterflies (the same on every run and in every CTA of the cluster)
-        const int lane = tid & 31;
-        for (int i = tid >> 5; i < n; i += blockDim.x >> 5) {
-            const RowPartial* part = seg_row + ((size_t)b * T + i) * seg_splits;
-            float M = -INFINITY;
-            int idx = INT_MAX;
-            for (int sg = lane; sg < seg_splits; sg += 32) argmax_combine(M, idx, part[sg].M, part[sg].idx);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float om = __shfl_xor_sync(0xffffffffu, M, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-                argmax_combine(M, idx, om, oi);
-            }
-            double S = 0.0;
-            if (M > -INFINITY)
-                for (int sg = lane; sg < seg_splits; sg += 32)
-                    if (part[sg].M > -INFINITY) S += part[sg].S * exp(((double)part[sg].M - (double)M) * inv_tau);
-            S = warp_sum(S);
-            if (lane == 0) sh.nS[i] = S, sh.nM[i] = M, sh.nArg[i] = idx, sh.nZ[i] = 0.0, sh.nQ[i] = 0.0;
-        }
-    }
-    for (int i = tid; i < n; i += blockDim.x) {
-        if (seg_row) {
-            if (!STOCH) {
-                sh.nArg[i] = merge_row(seg_row + ((size_t)b * T + i) * seg_splits, seg_splits, inv_tau, false).idx;
-            }
-        } else {
-            const NodeSummary ns = nodes[(size_t)b * T + i];
-            sh.nS[i] = ns.S, sh.nM[i] = ns.M, sh.nArg[i] = ns.idx, sh.nZ[i] = ns.Z, sh.nQ[i] = ns.Q;
-        }
     }
     if (STOCH)  // what the walk will need of the big rows, fetched by all threads at once instead of one test at a time
         for (int i = 1 + tid; i < n; i += blockDim.x) {
@@ -832,11 +875,7 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
 
     // ---- per-node statistics: row-in-registers clusters for small problems (one launch, latency-bound), vocabulary
     //      segments of 4096 with many CTAs per SM for large ones (two launches, throughput-bound)
-#ifdef S4C_EXP_FORCE_SEG
-    const bool seg_stats = S4C_EXP_FORCE_SEG;
-#else
     const bool seg_stats = !(vec && V <= kClMaxV) || (size_t)B * T * V > kSegStatsMinElems;
-#endif
     const int chunk = (int)round_up((size_t)ceil_div(V, kCl), 4);
     const float floor_span = kExpFloorSpan * (stoch ? temperature : 1.f);
     cudaLaunchAttribute attr[1];
@@ -929,15 +968,27 @@ extern "C" s4c_status s4c_tree_accept_noalloc(const float* target_logits, const 
                                               float temperature, const float* uniforms, int B, int T, int V,
                                               int max_depth, int32_t* accept_len, int32_t* path, int32_t* next_token,
                                               uint8_t* near_tie, int32_t* status, s4c_stream_t stream) {
-    if (B < 0 || T < 1 || T > S4C_MAX_T || V < 1) return S4C_ERR_SHAPE;
-    if (B > 0 && s4c::accept_ws_layout(B, T, V, nullptr, nullptr) > (size_t)S4C_NOALLOC_SCRATCH_BYTES)
+    // the argument checks of s4c_tree_accept, in its order, so that both entry points name the same fault first
+    if (!target_logits || !tokens || !parent || !accept_len || !path || !next_token) return S4C_ERR_NULL;
+    if (!(temperature >= 0.f) || isinf(temperature)) return S4C_ERR_SHAPE;
+    if (temperature > 0.f && (!draft_probs || !uniforms)) return S4C_ERR_NULL;
+    if (B < 0 || B > 65535 || T < 1 || T > S4C_MAX_T || V < 1 || max_depth < 0 || max_depth >= S4C_MAX_T) return S4C_ERR_SHAPE;
+    if (!s4c::aligned16(target_logits) || !s4c::aligned16(draft_probs)) return S4C_ERR_ALIGN;
+    if (B == 0) return S4C_OK;
+    if (s4c::accept_ws_layout(B, T, V, nullptr, nullptr) > (size_t)S4C_NOALLOC_SCRATCH_BYTES)
         return S4C_ERR_WORKSPACE;  // the problem needs more scratch than the built-in array holds
     static void* scratch_of_device[64] = {};
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return S4C_ERR_CUDA;
+    }
     if (!scratch_of_device[dev]) {
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_accept_scratch) != cudaSuccess || !p) return S4C_ERR_CUDA;
+        if (cudaGetSymbolAddress(&p, g_accept_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();  // leave no error behind for the caller's next runtime call
+            return S4C_ERR_CUDA;
+        }
         scratch_of_device[dev] = p;
     }
     return s4c_tree_accept(target_logits, draft_probs, tokens, parent, n_nodes, temperature, uniforms, B, T, V,

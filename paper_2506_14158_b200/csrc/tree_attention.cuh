@@ -8,7 +8,8 @@ namespace s4c {
 size_t simt_workspace_bytes(int B, int T, int Hq, int d, int C);
 s4c_status tree_attention_simt(const void* q, const void* k, const void* v, const int32_t* cache_len,
                                const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                               int d, int C, s4c_dtype dt, float scale, int32_t* status, void* ws, cudaStream_t stream);
+                               int d, int C, int span, s4c_dtype dt, float scale, int32_t* status, void* ws,
+                               cudaStream_t stream);
 
 // Merges split partials [B*Hq*T rows][splits][d + 2] (unnormalised output, running max in base-2 units, sum).
 s4c_status tree_attention_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
@@ -20,6 +21,6 @@ bool tc_supported(int T, int Hq, int Hkv, int d, s4c_dtype dt);
 size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C);
 s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                             int d, int C, float scale, int32_t* status, void* ws, cudaStream_t stream);
+                             int d, int C, int span, float scale, int32_t* status, void* ws, cudaStream_t stream);
 
 }  // namespace s4c

@@ -206,8 +206,8 @@ s4c_status tree_attention_combine(const void* ws, const int32_t* cache_len, cons
 template <typename T_, int D>
 static s4c_status launch_simt(const void* q, const void* k, const void* v, const int32_t* cache_len,
                               const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                              int C, float scale, int32_t* status, void* ws, cudaStream_t stream) {
-    const int splits = simt_splits(B, Hq, C);
+                              int C, int span, float scale, int32_t* status, void* ws, cudaStream_t stream) {
+    const int splits = simt_splits(B, Hq, span);  // shaped for the live span; the kernel splits the true length
     dim3 grid(splits, Hq, B);
     tree_attention_simt_kernel<T_, D><<<grid, kSimtThreads, 0, stream>>>(
         static_cast<const T_*>(q), static_cast<const T_*>(k), static_cast<const T_*>(v), cache_len, parent, n_nodes,
@@ -219,14 +219,18 @@ static s4c_status launch_simt(const void* q, const void* k, const void* v, const
 
 s4c_status tree_attention_simt(const void* q, const void* k, const void* v, const int32_t* cache_len,
                                const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                               int d, int C, s4c_dtype dt, float scale, int32_t* status, void* ws, cudaStream_t stream) {
+                               int d, int C, int span, s4c_dtype dt, float scale, int32_t* status, void* ws,
+                               cudaStream_t stream) {
+#define S4C_SIMT(TYPE, DD) \
+    launch_simt<TYPE, DD>(q, k, v, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, C, span, scale, status, ws, stream)
     if (dt == S4C_F32) {
-        if (d == 64) return launch_simt<float, 64>(q, k, v, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, C, scale, status, ws, stream);
-        if (d == 128) return launch_simt<float, 128>(q, k, v, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, C, scale, status, ws, stream);
+        if (d == 64) return S4C_SIMT(float, 64);
+        if (d == 128) return S4C_SIMT(float, 128);
     } else {
-        if (d == 64) return launch_simt<__nv_bfloat16, 64>(q, k, v, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, C, scale, status, ws, stream);
-        if (d == 128) return launch_simt<__nv_bfloat16, 128>(q, k, v, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, C, scale, status, ws, stream);
+        if (d == 64) return S4C_SIMT(__nv_bfloat16, 64);
+        if (d == 128) return S4C_SIMT(__nv_bfloat16, 128);
     }
+#undef S4C_SIMT
     return S4C_ERR_UNSUPPORTED;
 }
 

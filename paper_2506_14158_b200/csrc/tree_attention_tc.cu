@@ -1245,13 +1245,17 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
     return S4C_OK;
 }
 
+// `span` (<= C) is the number of slots the launch is shaped for: the host's bound on the live length (committed tokens
+// plus tree slots) where the caller gave one, else the capacity.  It steers the choices below and nothing else: the kernel
+// deals out the tiles of the true length, whatever that is.
 s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                             int d, int C, float scale, int32_t* status, void* ws, cudaStream_t stream) {
+                             int d, int C_slots, int span, float scale, int32_t* status, void* ws, cudaStream_t stream) {
     TcParams prm;
     prm.cache_len = cache_len, prm.parent = parent, prm.n_nodes = n_nodes;
     prm.out = static_cast<__nv_bfloat16*>(out), prm.ws = static_cast<float*>(ws), prm.status = status;
-    prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C;
+    prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C_slots;
+    const int C = span;  // every choice below is made for the live span
     const int nm = tc_nm(B, T, Hq, Hkv, C);
     prm.m_groups = tc_m_groups(B, T, Hq, Hkv, C);
     prm.splits = tc_splits(B, T, Hq, Hkv, C);
@@ -1285,7 +1289,7 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
 #undef S4C_TC_DISPATCH
     if (st != S4C_OK) return st;
     if (prm.mode == kModeWorkspace)
-        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, C, prm.splits * rep * turns, S4C_BF16,
+        return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, prm.C, prm.splits * rep * turns, S4C_BF16,
                                       stream);
     return S4C_OK;
 }

@@ -16,11 +16,12 @@ import torch
 from ._build import lib_path
 
 F32, BF16 = 0, 1
-SEQ_OK, SEQ_BAD_PARENT, SEQ_TOKEN_RANGE, SEQ_CAPACITY, SEQ_DEPTH, SEQ_BAD_PATH, SEQ_TIMEOUT = 0, 1, 2, 4, 8, 16, 32
+SEQ_OK, SEQ_BAD_PARENT, SEQ_TOKEN_RANGE, SEQ_CAPACITY, SEQ_DEPTH, SEQ_BAD_PATH, SEQ_TIMEOUT, SEQ_NONFINITE = 0, 1, 2, 4, 8, 16, 32, 64
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WORKSPACE", "ERR_UNSUPPORTED", "ERR_CUDA"]
 
 EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
-           "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact"]
+           "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
+           "s4c_launch_floor"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -45,7 +46,7 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_attention_workspace_bytes.restype = sz
     lib.s4c_tree_attention_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
     lib.s4c_tree_attention.restype = i
-    lib.s4c_tree_attention.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_tree_attention.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
     lib.s4c_tree_accept_workspace_bytes.restype = sz
     lib.s4c_tree_accept_workspace_bytes.argtypes = [i, i, i]
     lib.s4c_tree_accept.restype = i
@@ -54,6 +55,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_accept_noalloc.argtypes = [vp, vp, i32p, i32p, i32p, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp]
     lib.s4c_kv_compact.restype = i
     lib.s4c_kv_compact.argtypes = [vp, vp, i, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i32p, vp]
+    lib.s4c_launch_floor.restype = i
+    lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
 
 
@@ -111,8 +114,10 @@ def tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dtype) -> int:
 
 
 def tree_attention(q, k_cache, v_cache, cache_len, parent, n_nodes=None, out=None, scale: float = 0.0, status=None,
-                   workspace=None, stream=None):
-    """s4c_tree_attention: q [B,Hq,T,d], k_cache/v_cache [B,Hkv,C,d] -> out [B,Hq,T,d] (same dtype)."""
+                   workspace=None, stream=None, max_cache_len: int = 0):
+    """s4c_tree_attention: q [B,Hq,T,d], k_cache/v_cache [B,Hkv,C,d] -> out [B,Hq,T,d] (same dtype).
+
+    ``max_cache_len``: the host's upper bound on ``cache_len`` (0 = unknown); it shapes the launch, never the result."""
     B, Hq, T, d = q.shape
     _, Hkv, C, _ = k_cache.shape
     if k_cache.shape != (B, Hkv, C, d) or v_cache.shape != (B, Hkv, C, d):
@@ -128,7 +133,8 @@ def tree_attention(q, k_cache, v_cache, cache_len, parent, n_nodes=None, out=Non
     rc = _lib.s4c_tree_attention(
         _dev(q, name="q"), _dev(k_cache, name="k_cache"), _dev(v_cache, name="v_cache"),
         _dev(cache_len, torch.int32, "cache_len"), _dev(parent, torch.int32, "parent"),
-        _dev(n_nodes, torch.int32, "n_nodes"), _dev(out, q.dtype, "out"), B, T, Hq, Hkv, d, C, dt, float(scale),
+        _dev(n_nodes, torch.int32, "n_nodes"), _dev(out, q.dtype, "out"), B, T, Hq, Hkv, d, C, int(max_cache_len), dt,
+        float(scale),
         _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
         0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
     if rc:
@@ -236,3 +242,12 @@ def kv_compact(k_ptrs, v_ptrs, n_layers: int, cache_shape, dtype, cache_len, pat
     if rc:
         raise S4CError("s4c_kv_compact", rc)
     return status
+
+
+def launch_floor(ctas: int, cluster: int, threads: int, smem_bytes: int, tmem_cols: int, cluster_syncs: int,
+                 dependent_launch: bool, word: Optional[torch.Tensor] = None, stream=None):
+    """s4c_launch_floor: enqueue one empty kernel with the given launch shape (a measurement aid)."""
+    rc = _lib.s4c_launch_floor(int(ctas), int(cluster), int(threads), int(smem_bytes), int(tmem_cols), int(cluster_syncs),
+                               1 if dependent_launch else 0, _dev(word, torch.int32, "word"), None, _stream(stream))
+    if rc:
+        raise S4CError("s4c_launch_floor", rc)

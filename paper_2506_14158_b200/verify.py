@@ -21,8 +21,10 @@ class VerifyStep:
                  cache_len: torch.Tensor, parent: torch.Tensor, tokens: torch.Tensor, target_logits: torch.Tensor,
                  draft_probs: Optional[torch.Tensor], uniforms: Optional[torch.Tensor], temperature: float,
                  max_depth: int, n_nodes: Optional[torch.Tensor] = None, feat_in: Optional[torch.Tensor] = None,
-                 stacked: Optional[tuple] = None):
-        """``stacked`` = (q_all [n_layers,B,Hq,T,d], k_all, v_all [n_layers,B,Hkv,C,d]) when the per-layer tensors are
+                 stacked: Optional[tuple] = None, max_cache_len: int = 0):
+        """``max_cache_len``: what the host knows about the committed lengths (an upper bound, 0 = nothing); it is handed
+        to every s4c_tree_attention call, which shapes its launch for it instead of for the capacity.
+        ``stacked`` = (q_all [n_layers,B,Hq,T,d], k_all, v_all [n_layers,B,Hkv,C,d]) when the per-layer tensors are
         views of three big ones: the host-buffer path then moves a step's inputs with three copies instead of three
         per layer."""
         self.n_layers = len(q)
@@ -32,6 +34,7 @@ class VerifyStep:
         self.parent, self.tokens, self.n_nodes = parent, tokens, n_nodes
         self.logits, self.draft_probs, self.uniforms = target_logits, draft_probs, uniforms
         self.temperature, self.max_depth = float(temperature), int(max_depth)
+        self.max_cache_len = int(max_cache_len)
         self.feat_in = feat_in
         dev = cache_len.device
         B, T, V = target_logits.shape
@@ -65,7 +68,8 @@ class VerifyStep:
     def attention(self, l0: int = 0, l1: Optional[int] = None):
         for l in range(l0, self.n_layers if l1 is None else l1):
             s4c.tree_attention(self.q[l], self.k_caches[l], self.v_caches[l], self.cache_len, self.parent, self.n_nodes,
-                               out=self.attn_out[l], status=self.status_attn, workspace=self.ws_attn)
+                               out=self.attn_out[l], status=self.status_attn, workspace=self.ws_attn,
+                               max_cache_len=self.max_cache_len)
 
     def accept(self):
         s4c.tree_accept(self.logits, self.draft_probs, self.tokens, self.parent, self.temperature, self.uniforms,

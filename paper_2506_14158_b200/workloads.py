@@ -134,11 +134,17 @@ class VerifyConfig:
     n_layers: int = 1
     hid: int = 4096
     temperatures: Tuple[float, ...] = (0.0, 1.0)
+    capacity: int = 0  # cache capacity in slots; 0: as tight as the step allows (see C)
 
     @property
     def C(self) -> int:
-        """Cache capacity in slots: L + T rounded up to a multiple of 128."""
-        return (self.L + self.T + 127) // 128 * 128
+        """Cache capacity in slots: `capacity` if set (a serving cache laid out for its longest context), else L + T
+        rounded up to a multiple of 128."""
+        tight = (self.L + self.T + 127) // 128 * 128
+        if self.capacity:
+            assert self.capacity >= self.L + self.T, "capacity below L + T"
+            return self.capacity
+        return tight
 
     @property
     def max_depth(self) -> int:

@@ -35,7 +35,7 @@ def test_sequence_flags_agree_between_header_binding_and_oracle(s4c_lib):
     text = open(os.path.join(ROOT, "include", "s4c.h")).read()
     flags = {k: int(v) for k, v in re.findall(r"#define\s+S4C_(SEQ_[A-Z_]+)\s+(\d+)", text)}
     assert flags == {"SEQ_OK": 0, "SEQ_BAD_PARENT": 1, "SEQ_TOKEN_RANGE": 2, "SEQ_CAPACITY": 4, "SEQ_DEPTH": 8,
-                     "SEQ_BAD_PATH": 16, "SEQ_TIMEOUT": 32}
+                     "SEQ_BAD_PATH": 16, "SEQ_TIMEOUT": 32, "SEQ_NONFINITE": 64}
     for k, v in flags.items():
         assert getattr(s4c, k) == v
         if k != "SEQ_TIMEOUT":  # the CPU oracle has no waits
@@ -62,20 +62,20 @@ def test_workspace_queries_are_host_functions(s4c_lib):
 def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     lib = ctypes.CDLL(s4c_lib)
     vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
-    lib.s4c_tree_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp, vp, sz, vp]
+    lib.s4c_tree_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i, f, vp, vp, sz, vp]
     lib.s4c_tree_accept.argtypes = [vp, vp, vp, vp, vp, f, vp, i, i, i, i, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.s4c_kv_compact.argtypes = [vp, vp, i, vp, vp, vp, i, vp, vp, i, i, i, i, i, i, i, vp, vp]
     lib.s4c_status_string.restype = ctypes.c_char_p
     P = 4096  # a fake, 16-byte aligned "pointer": rejected calls never dereference or launch
     att = lambda **kw: lib.s4c_tree_attention(*[kw.get(k, d) for k, d in [
         ("q", P), ("k", P), ("v", P), ("cl", P), ("par", P), ("nn", None), ("out", P), ("B", 1), ("T", 8), ("Hq", 4),
-        ("Hkv", 2), ("d", 128), ("C", 256), ("dt", 1), ("scale", 0.0), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
+        ("Hkv", 2), ("d", 128), ("C", 256), ("hint", 0), ("dt", 1), ("scale", 0.0), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
     assert att(q=None) == 1                      # S4C_ERR_NULL
     assert att(T=129) == 2 and att(T=0) == 2     # S4C_ERR_SHAPE
     assert att(Hq=4, Hkv=3) == 2 and att(d=96) == 2
     assert att(dt=5) == 3                        # S4C_ERR_DTYPE
     assert att(k=P + 2) == 4                     # S4C_ERR_ALIGN
-    assert att(scale=-1.0) == 2
+    assert att(scale=-1.0) == 2 and att(hint=-1) == 2
     assert att(B=0) == 0
     assert att(T=64, Hq=8, Hkv=2, C=24704, ws=None) == 5   # this grid splits wider than a cluster and needs a workspace
     acc = lambda **kw: lib.s4c_tree_accept(*[kw.get(k, d) for k, d in [

@@ -122,3 +122,39 @@ def test_sweep_sized_batches_match_bit_for_bit(B, T, tau):
     cfg, parent, x = _synthetic(B, T, 32000, seed=B + T, sigma=3.0, tau=max(tau, 0.5), mode="topk", max_tree_depth=8)
     got, ref = accept_both(x, parent, tau, max_depth=cfg.max_tree_depth)
     assert assert_accept_equal(got, ref, tau > 0) == 0
+
+
+@pytest.mark.parametrize("V,B,T", [(300, 6, 12),          # row-in-registers clusters
+                                   (4099, 6, 12),         # odd vocabulary: segment kernels, scalar loads
+                                   (32000, 24, 16)])      # 12 M logits: segment kernels, vector loads
+@pytest.mark.parametrize("tau", [0.0, 1.0])
+def test_nonfinite_logits_flag_the_sequence_and_nothing_else(V, B, T, tau):
+    # NaN, +Inf and -Inf planted in rows the walk visits and in rows it never reaches; both sides must flag the same
+    # sequences (S4C_SEQ_NONFINITE = 64), skip them, and agree bit for bit on every other sequence of the batch
+    cfg, parent, x = _synthetic(B, T, V, seed=31 + V % 7, tau=max(tau, 0.5), mode="topk")
+    lg = x["logits"]
+    lg[0, 0, V // 3] = np.nan                 # the root's row: always walked
+    lg[1, T - 1, V - 1] = np.inf              # last node, last entry (a leaf, hardly ever reached)
+    lg[2, 1, :] = -np.inf                     # a row without any mass
+    lg[3, 2, 5 % V] = -np.inf                 # single masked tokens: legal, probability zero
+    lg[3, 0, x["tokens"][3, 1]] = -np.inf     # ... one of them a drafted token at the root
+    n_nodes = np.full(B, T, dtype=np.int32)
+    n_nodes[4] = T - 3
+    lg[4, T - 1, 0] = np.nan                  # a padding row: not part of the tree
+    got, ref = accept_both(x, parent, tau, n_nodes=n_nodes, max_depth=cfg.max_tree_depth)
+    assert ref["status"][:5].tolist() == [64, 64, 64, 0, 0] and (ref["status"][5:] == 0).all()
+    assert (got["accept_len"][:3] == -1).all() and (got["next_token"][:3] == -1).all()
+    assert assert_accept_equal(got, ref, tau > 0) == 0
+
+
+@pytest.mark.parametrize("tau", [1e-6, 3e-9, 50.0])
+@pytest.mark.parametrize("V,B,T", [(2000, 8, 10), (32000, 24, 16)])
+def test_extreme_temperatures(tau, V, B, T):
+    # a tiny temperature turns the softmax into (nearly) a one-hot row; below the float spacing of the logits the rows are
+    # summed as counts of their maxima.  A large one flattens it.  Decisions stay bit-exact.
+    cfg, parent, x = _synthetic(B, T, V, seed=3, tau=1.0, mode="topk")
+    x["logits"][0] = np.round(x["logits"][0])  # exact ties at the maximum in some rows
+    x["logits"][1] += 1000.0                   # large logits: coarser float spacing
+    got, ref = accept_both(x, parent, tau, max_depth=cfg.max_tree_depth)
+    assert (ref["status"] == 0).all()
+    assert assert_accept_equal(got, ref, True) == 0

@@ -149,23 +149,26 @@ def test_grids_of_several_waves_share_an_sm_between_two_ctas(T):
     _case(B=10, Hq=32, Hkv=32, T=T, d=128, Ls=[300, 17, 0, 640, 129, 300, 64, 511, 1, 77], dtype="bf16", seed=21 + T)
 
 
-def _sampled_heads_case(B, Hq, Hkv, T, L, seed, kv_heads, seqs):
+def _sampled_heads_case(B, Hq, Hkv, T, L, seed, kv_heads, seqs, C=None, max_cache_len=0, Ls=None):
     """The launch runs at full size (the grid, splits and kernel variant the benchmark times); the oracle checks the
-    sampled (sequence, KV head) pairs, all their query heads and all their tree nodes, element by element."""
+    sampled (sequence, KV head) pairs, all their query heads and all their tree nodes, element by element.
+    ``C``: cache capacity (default: as tight as L + T allows); ``max_cache_len``: the host's hint; ``Ls``: per-sequence
+    lengths (default: L everywhere)."""
     from paper_2506_14158_b200 import s4c
     import oracle
 
     d, G = 128, Hq // Hkv
-    C = (L + T + 127) // 128 * 128
+    C = C or (L + T + 127) // 128 * 128
     g = torch.Generator(device="cuda").manual_seed(seed)
     q = torch.randn((B, Hq, T, d), generator=g, device="cuda").bfloat16()
     k = torch.randn((B, Hkv, C, d), generator=g, device="cuda").bfloat16()
     v = torch.randn((B, Hkv, C, d), generator=g, device="cuda").bfloat16()
     rng = np.random.default_rng(seed)
     parent = np.stack([W.random_tree(T, 8, rng) for _ in range(B)])
-    cl = np.full(B, L, dtype=np.int32)
+    cl = np.full(B, L, dtype=np.int32) if Ls is None else np.asarray(Ls, dtype=np.int32)
     status = torch.full((B,), -1, dtype=torch.int32, device="cuda")
-    out = s4c.tree_attention(q, k, v, torch.from_numpy(cl).cuda(), torch.from_numpy(parent).cuda(), status=status)
+    out = s4c.tree_attention(q, k, v, torch.from_numpy(cl).cuda(), torch.from_numpy(parent).cuda(), status=status,
+                             max_cache_len=max_cache_len)
     torch.cuda.synchronize()
     assert (status.cpu().numpy() == 0).all()
     assert torch.isfinite(out.float()).all()
@@ -189,3 +192,40 @@ def _sampled_heads_case(B, Hq, Hkv, T, L, seed, kv_heads, seqs):
 ])
 def test_full_size_launch_configurations_on_sampled_heads(name, B, Hq, Hkv, T, L, kv_heads, seqs):
     _sampled_heads_case(B, Hq, Hkv, T, L, seed=len(name), kv_heads=kv_heads, seqs=seqs)
+
+
+# A serving cache is laid out for its longest context (C = 32768 here) while the sequences are far shorter.  The launch is
+# shaped for the capacity when the host says nothing (hint 0) and for the live length when it passes its bound; a bound
+# below the true length (hint 64 for a sequence of 4096) must still give the right answer.  Splits that receive no tile
+# (L = 0 leaves a single tile for a cluster of 8) take part in the merge with zero weight.
+@pytest.mark.parametrize("shape", ["7B", "8B"])
+@pytest.mark.parametrize("L", [0, 1000, 4096])
+@pytest.mark.parametrize("hint", ["none", "exact", "too small"])
+def test_capacity_far_beyond_the_live_length(shape, L, hint):
+    B, Hq, Hkv, T = (1, 32, 32, 26) if shape == "7B" else (4, 32, 8, 64)
+    mcl = {"none": 0, "exact": max(L, 1), "too small": 64}[hint]
+    _sampled_heads_case(B, Hq, Hkv, T, L, seed=100 + L % 97 + len(shape), kv_heads=[0, Hkv - 1], seqs=[0, B - 1], C=32768,
+                        max_cache_len=mcl)
+
+
+def test_capacity_far_beyond_ragged_live_lengths():
+    # one batch, lengths from empty to 4096, capacity 32768, the bound the host would know (the longest sequence)
+    _sampled_heads_case(4, 32, 8, 64, 4096, seed=77, kv_heads=[1, 6], seqs=[0, 1, 2, 3], C=32768, max_cache_len=4096,
+                        Ls=[0, 4096, 37, 1500])
+
+
+def test_the_hint_never_changes_the_result_class():
+    # same inputs, three launch shapes (capacity, exact bound, a bound far too small): every one within tolerance of the
+    # oracle, and the two runs with the same hint bit-identical
+    cfg = W.CONFIGS["c2"]
+    q, k, v = W.make_attention_inputs(cfg)
+    big = torch.zeros((cfg.B, cfg.Hkv, 8192, cfg.d), dtype=k.dtype)
+    kb, vb = big.clone(), big.clone()
+    kb[:, :, :cfg.C], vb[:, :, :cfg.C] = k, v
+    parent = W.make_trees(cfg)
+    outs = []
+    for mcl in (0, cfg.L, 16, cfg.L):
+        got, ref, gst, rst = attention_both(q, kb, vb, [cfg.L], parent, max_cache_len=mcl)
+        assert_attention_close(got, ref, gst, rst, ATTN_TOL["bf16"])
+        outs.append(got)
+    np.testing.assert_array_equal(outs[1], outs[3])

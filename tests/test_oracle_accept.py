@@ -357,3 +357,62 @@ def test_zero_draft_probability_and_duplicate_siblings():
     # token 0: ratio 0.2 -> rejected at u=.9; residual = norm(0,0,.3,.3); token 0 again: p=0,q=0 -> ratio 0 -> rejected
     a, _, nxt = _walk(lg2, q2, np.array([0, 0, 0], dtype=np.int32), parent, np.array([0.1, 0.9, 0.0], dtype=np.float32))
     assert a == 0 and nxt == 2
+
+
+# ------------------------------------------------------------------ non-finite logits (input validation of the boundary)
+def _nonfinite_batch(seed=5, B=6, T=9, V=40):
+    rng = np.random.default_rng(seed)
+    parent = np.stack([W.random_tree(T, 4, rng, 1, 3) for _ in range(B)])
+    logits = (rng.standard_normal((B, T, V)) * 2).astype(np.float32)
+    dq = softmax(logits.astype(np.float64) + rng.standard_normal((B, T, V)), axis=-1).astype(np.float32)
+    tokens = rng.integers(0, V, (B, T)).astype(np.int32)
+    for b in range(B):
+        for n in range(T):
+            kids = W.children_of(parent[b], n)
+            tokens[b, kids] = np.argsort(-dq[b, n], kind="stable")[: len(kids)]
+    u = np.minimum(rng.random((B, T), dtype=np.float32), ONE_MINUS)
+    return parent, logits, dq, tokens, u
+
+
+@pytest.mark.parametrize("tau", [0.0, 1.0])
+def test_nonfinite_logits_are_flagged_and_the_rest_of_the_batch_is_untouched(tau):
+    parent, logits, dq, tokens, u = _nonfinite_batch()
+    B, T, V = logits.shape
+    run = lambda lg, nn=None: (oracle.accept_stochastic(lg, dq, tokens, parent, tau, u, nn) if tau > 0
+                               else oracle.accept_greedy(lg, tokens, parent, nn))
+    clean = run(logits)
+    assert (clean["status"] == 0).all()
+    bad = logits.copy()
+    bad[0, 0, 3] = np.nan           # the root's row: always walked
+    bad[1, T - 1, 7] = np.inf       # a leaf row that the walk may never reach: flagged all the same
+    bad[2, 2, :] = -np.inf          # a row with no mass at all
+    bad[3, 4, 5] = -np.inf          # a single masked token: legal
+    nn = np.full(B, T, dtype=np.int32)
+    nn[4] = T - 2
+    bad[4, T - 1, 0] = np.nan       # a padding row (i >= n_nodes): not part of the tree, not looked at
+    r = run(bad, nn)
+    assert r["status"].tolist() == [64, 64, 64, 0, 0, 0]
+    for b in (0, 1, 2):
+        assert r["accept_len"][b] == -1 and r["next_token"][b] == -1 and (r["path"][b] == -1).all()
+    # -Inf is probability zero: exactly the result of a logit so low that its exponential underflows to zero
+    low = logits.copy()
+    low[3, 4, 5] = -1e4
+    want = run(low, nn)
+    for key in ("accept_len", "path", "next_token"):
+        np.testing.assert_array_equal(r[key][3:], want[key][3:])
+    np.testing.assert_array_equal(r["accept_len"][5], clean["accept_len"][5])
+    np.testing.assert_array_equal(r["next_token"][5], clean["next_token"][5])
+
+
+def test_a_masked_token_is_never_emitted_and_never_accepted():
+    # one candidate whose target logit is -Inf: p(x) = 0, so it is rejected for every u, and the resampled token is never x
+    V, x = 8, 3
+    logits = np.zeros((1, 2, V), dtype=np.float32)
+    logits[0, 0, x] = -np.inf
+    dq = np.full((1, 2, V), 1.0 / V, dtype=np.float32)
+    parent = np.array([[-1, 0]], dtype=np.int32)
+    tokens = np.array([[0, x]], dtype=np.int32)
+    for u1 in (0.0, 0.5, float(ONE_MINUS)):
+        for u0 in np.linspace(0, float(ONE_MINUS), 17):
+            r = oracle.accept_stochastic(logits, dq, tokens, parent, 1.0, np.array([[u0, u1]], dtype=np.float32))
+            assert r["status"][0] == 0 and r["accept_len"][0] == 0 and r["next_token"][0] != x
