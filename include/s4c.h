@@ -228,6 +228,25 @@ s4c_status s4c_kv_compact(void* const* k_caches, void* const* v_caches, int n_la
 s4c_status s4c_launch_floor(int ctas, int cluster, int threads, int smem_bytes, int tmem_cols, int cluster_syncs,
                             int dependent_launch, const int32_t* word, int32_t* sink, s4c_stream_t stream);
 
+/* ------------------------------------------------------------------------------------------
+ * s4c_selftest_attention_timeout -- checks the failure path of s4c_tree_attention; the paper has no
+ * counterpart.
+ *
+ * Every wait inside the bf16 attention kernel is bounded: when one runs out of time the CTA stops
+ * issuing copies and products, parks, merges and stores nothing, still meets its cluster's barriers,
+ * sees its own copies and products complete, frees its tensor memory and returns; status[b] gets
+ * S4C_SEQ_TIMEOUT and the context stays usable.  This call makes that happen without any fault: it is
+ * the launch of s4c_tree_attention (bf16, scale 1/sqrt(d), all trees of T nodes) in which no CTA ever
+ * requests cache tile `withhold_tile` (0-based, 64 slots each) of its own range and a wait gives up
+ * after `limit_us` microseconds (1..100000).  Afterwards status[b] holds S4C_SEQ_TIMEOUT for every
+ * sequence whose CTAs own such a tile, `out` is untouched for them, and the next call on the stream
+ * works normally.  Shapes that would merge through a workspace are refused (S4C_ERR_UNSUPPORTED).
+ * ------------------------------------------------------------------------------------------ */
+s4c_status s4c_selftest_attention_timeout(const void* q, const void* k_cache, const void* v_cache,
+                                          const int32_t* cache_len, const int32_t* parent, void* out, int B, int T,
+                                          int Hq, int Hkv, int d, int C, int max_cache_len, int withhold_tile,
+                                          int limit_us, int32_t* status, s4c_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -46,3 +46,24 @@ extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, con
     return tree_attention_simt(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, span, dt, scale,
                                status, workspace, stream);
 }
+
+// The bounded waits of the tensor-core kernel, exercised: the same launch as s4c_tree_attention, except that the copy
+// producer of every CTA never requests cache tile `withhold_tile` of its range and a wait gives up after `limit_us`
+// microseconds.  The consumers of that tile run out of time with nothing in flight, every role leaves its loop, and the
+// kernel returns normally with S4C_SEQ_TIMEOUT in status[b] and `out` untouched.
+extern "C" s4c_status s4c_selftest_attention_timeout(const void* q, const void* k_cache, const void* v_cache,
+                                                     const int32_t* cache_len, const int32_t* parent, void* out, int B,
+                                                     int T, int Hq, int Hkv, int d, int C, int max_cache_len,
+                                                     int withhold_tile, int limit_us, int32_t* status,
+                                                     s4c_stream_t stream_) {
+    using namespace s4c;
+    const s4c_status st = check_shapes(B, T, Hq, Hkv, d, C, S4C_BF16);
+    if (st != S4C_OK) return st;
+    if (!q || !k_cache || !v_cache || !cache_len || !parent || !out || !status) return S4C_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return S4C_ERR_ALIGN;
+    if (B == 0 || max_cache_len < 0 || withhold_tile < 0 || limit_us < 1 || limit_us > 100000) return S4C_ERR_SHAPE;
+    if (s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, S4C_BF16) != 0) return S4C_ERR_UNSUPPORTED;  // in-cluster merge only
+    const int span = (max_cache_len > 0 && (long long)max_cache_len + T < (long long)C) ? max_cache_len + T : C;
+    return tree_attention_tc(q, k_cache, v_cache, cache_len, parent, nullptr, out, B, T, Hq, Hkv, d, C, span,
+                             1.f / sqrtf((float)d), status, nullptr, static_cast<cudaStream_t>(stream_), limit_us, withhold_tile);
+}

@@ -21,6 +21,7 @@ bool tc_supported(int T, int Hq, int Hkv, int d, s4c_dtype dt);
 size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C);
 s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                             int d, int C, int span, float scale, int32_t* status, void* ws, cudaStream_t stream);
+                             int d, int C, int span, float scale, int32_t* status, void* ws, cudaStream_t stream,
+                             int wait_limit_us = 0 /* 0: the default of about 200 ms */, int withhold_tile = -1 /* self-test only */);
 
 }  // namespace s4c

@@ -38,6 +38,7 @@ constexpr int kBM = 128;  // query rows per row tile (TMEM lanes)
 constexpr int kBN = 64;   // cache slots per tile
 constexpr int kMaxClusterSplits = 8;
 constexpr long long kWaitLimitCycles = 400ll * 1000 * 1000;  // about 200 ms at the 1.965 GHz boost clock, longer below it
+constexpr int kDrainBars = 4;  // one per issuer warp (at most three) and a spare
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
 template <int D, int NM, int TC = 1, int PUSH = 0>
@@ -56,7 +57,7 @@ struct TcCfg {
     // TMEM score buffers per row tile: two per softmax group; four where a single group leaves the columns free, so
     // that a product S = Q K^T need not wait for the P V product two tiles back
     static constexpr int kScoreBufs = (NM == 1 && TC == 1 && PUSH != 2) ? 4 : 2 * TC;
-    static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM;
+    static constexpr int kNumBars = 1 + 4 * kStages + (3 * kScoreBufs + TC) * NM + kDrainBars;
     // TMA warp, a QK issuer warp per row tile, one PV issuer warp.  (Two row tiles: 4 + 8 = 12 warps, three per scheduler,
     // so that a thread may hold 168 registers; a 13th warp would cap every thread at 128 and spill the softmax loop.)
     static constexpr int kRoleWarps = 2 + NM;
@@ -96,25 +97,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  `dead` (shared memory) is set by the first wait that expires; later waits then give up at once.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead) {
-    if (mbar_try_wait(bar, parity)) return;
+// Bounded wait: true once the phase has completed, false when the wait was given up.  `dead` (shared memory) is set by
+// the first wait of the CTA that runs out of time; every later wait then gives up at once.  A role that gets `false`
+// leaves its loop without issuing anything further (no copy, no product, no tensor-memory store).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, long long limit) {
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return;
-        if (*dead) return;
-        if (clock64() - t0 > kWaitLimitCycles) {
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*dead) return false;
+        if (clock64() - t0 > limit) {
             *dead = 1;
-            return;
+            return false;
         }
     }
 }
 // Whole-warp wait: lane 0 polls the barrier, the other lanes pick the result up at the warp barrier (one poller
-// per warp instead of 32 keeps the shared-memory barrier unit free for the arrivals).
-__device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* dead) {
-    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, dead);
+// per warp instead of 32 keeps the shared-memory barrier unit free for the arrivals).  Whether the wait was given up
+// shows in `dead`, which the caller reads where a warp-uniform answer costs nothing.
+__device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* dead, long long limit) {
+    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, dead, limit);
     __syncwarp();
+}
+// Wait for something this CTA itself set in motion (a bulk copy, a committed product) on the way out of a CTA that has
+// given up: bounded like every wait, but not cut short by `dead`, so that nothing is still in flight into shared or
+// tensor memory when the CTA frees them.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return;
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -376,6 +388,8 @@ struct TcParams {
     int32_t* status;
     int T, Hq, Hkv, C, m_groups, splits, mode, q_box_rows;
     float scale_log2;
+    long long wait_limit;  // clock cycles a wait may take (kWaitLimitCycles; the self-test passes a short one)
+    int withhold_tile;     // -1; the self-test names one tile of every CTA that the producer does not request
 };
 
 // Tile range of a split: tiles are dealt out as evenly as whole tiles allow.
@@ -422,6 +436,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 480);
     volatile int* dead = reinterpret_cast<volatile int*>(tail + 484);
     int* bad_s = reinterpret_cast<int*>(tail + 488);  // S4C_SEQ_* flags found by the softmax warps (malformed tree)
+    int* issued_s = reinterpret_cast<int*>(tail + 492);  // tiles the producer has requested
     int32_t* par_s = reinterpret_cast<int32_t*>(tail + 512);  // S4C_MAX_T * 4 = 512 bytes
 
     const uint32_t bar0 = smem_u32(bars);
@@ -429,6 +444,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // barrier indices; the per-row-tile ones take (tile t, buffer i)
     constexpr int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + S, V_FULL = 1 + 2 * S, V_EMPTY = 1 + 3 * S, PER_TILE = 1 + 4 * S;
     constexpr int NB = Cfg::kScoreBufs, PT = 3 * NB + TC;  // score buffers and barriers per row tile; tile j uses buffer j % NB
+    constexpr int DRAIN = PER_TILE + PT * NM;               // one per issuer warp: its products are complete (used when giving up)
+    const long long limit = prm.wait_limit;
     auto S_FULL = [&](int t, int i) { return BAR(PER_TILE + PT * t + i); };
     auto S_EMPTY = [&](int t, int i) { return BAR(PER_TILE + PT * t + NB + i); };
     auto P_FULL = [&](int t, int i) { return BAR(PER_TILE + PT * t + 2 * NB + i); };
@@ -456,7 +473,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             uint32_t count = 1;  // but: P_FULL takes one arrival per active softmax warp, the EMPTY barriers of
                                  // the ring one commit per active row tile (each has issuer threads of its own)
             if ((i >= K_EMPTY && i < K_EMPTY + S) || (i >= V_EMPTY && i < V_EMPTY + S)) count = (uint32_t)nm_act;
-            if (i >= PER_TILE) {
+            if (i >= PER_TILE && i < DRAIN) {
                 const int t = (i - PER_TILE) / PT, k = (i - PER_TILE) % PT;
                 const uint32_t active = (uint32_t)active_threads(t) / 32u;
                 if (k >= 2 * NB && k < 3 * NB && active) count = active;
@@ -468,6 +485,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tma_prefetch_desc(&map_q), tma_prefetch_desc(&map_k), tma_prefetch_desc(&map_v);
             *dead = 0;
             *bad_s = 0;
+            *issued_s = 0;
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
@@ -496,22 +514,27 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
     if (warp == 0) {
         // ================= TMA producer =================
-        auto load_tile = [&](int j) {
+        auto load_tile = [&](int j) -> bool {  // false: a wait was given up, nothing further is requested
             const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
-            mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead);
+            if (j == prm.withhold_tile) return true;  // (self-test only: this tile never arrives)
+            if (!mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead, limit)) return false;
             mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
             if (NH == 2) {  // one request per tile: the map's third dimension is the 64-column half
                 tma_load_3d(sK + s * Cfg::kTileBytes, &map_k, BAR(K_FULL + s), 0, row, 0);
             } else {
                 tma_load_2d(sK + s * Cfg::kTileBytes, &map_k, BAR(K_FULL + s), 0, row);
             }
-            mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead);
+            if (!mbar_wait(BAR(V_EMPTY + s), (it & 1) ^ 1, dead, limit)) {
+                mbar_drain(BAR(K_FULL + s), it & 1, limit);  // the K half of this tile is on its way: see it in
+                return false;
+            }
             mbar_expect_tx(BAR(V_FULL + s), Cfg::kTileBytes);
             if (NH == 2) {
                 tma_load_3d(sV + s * Cfg::kTileBytes, &map_v, BAR(V_FULL + s), 0, row, 0);
             } else {
                 tma_load_2d(sV + s * Cfg::kTileBytes, &map_v, BAR(V_FULL + s), 0, row);
             }
+            return true;
         };
         if (nt > 0) {
             // Q first (the requests are served in order, and the first product needs it): one request per lane -- a row
@@ -526,7 +549,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             __syncwarp();
             // then the first pass of the ring, every ring slot still free: again one request per lane
-            if (lane < 2 * S && (lane >> 1) < nt) {
+            if (lane < 2 * S && (lane >> 1) < nt && (lane >> 1) != prm.withhold_tile) {
                 // K and V of a tile on neighbouring lanes: the requests go out as K0 V0 K1 V1 ..., so that the first
                 // product with V does not wait behind every K tile of the ring
                 const int j = lane >> 1, row = kv_row0 + (t0 + j) * kBN;
@@ -541,8 +564,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
             }
             __syncwarp();
-            if (lane == 0)
-                for (int j = S; j < nt; ++j) load_tile(j);
+            if (lane == 0) {
+                int issued = nt < S ? nt : S;
+                for (; issued < nt; ++issued)
+                    if (!load_tile(issued)) break;
+                *issued_s = issued;  // tiles requested: what a CTA that gives up has to see in before it leaves
+            }
+            __syncwarp();
         }
     } else if (warp <= NM) {
         // ================= QK issuer of row tile t: S = Q K^T =================
@@ -556,14 +584,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk)  // 64-element halves along d, 32 bytes per K step inside a half
                 a_desc[kk] = smem_desc_sw128(sQ + t * Cfg::kQBytes + (kk >> 2) * (kBM * 128) + (kk & 3) * 32, 16, 1024);
-            mbar_wait(BAR(Q_FULL), 0, dead);
+            // `ok` is this lane's own record: once one of its waits has been given up it never issues again.  (The lanes
+            // poll on their own and need not agree at the moment of giving up; the elected lane acts on what it saw
+            // itself, and every later wait of every lane ends at once.)
+            bool ok = mbar_wait(BAR(Q_FULL), 0, dead, limit);
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
-                mbar_wait(BAR(K_FULL + s), it & 1, dead);
+                ok &= mbar_wait(BAR(K_FULL + s), it & 1, dead, limit);
                 const uint64_t k_desc = smem_desc_sw128(sK + s * Cfg::kTileBytes, 16, 1024);
-                mbar_wait(S_EMPTY(t, j % NB), ((j / NB) & 1) ^ 1, dead);
+                ok &= mbar_wait(S_EMPTY(t, j % NB), ((j / NB) & 1) ^ 1, dead, limit);
                 tc_fence_after();
-                if (elect_one()) {
+                if (elect_one() && ok) {
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk)  // the start-address field counts 16-byte units
                         tc_mma_bf16(TM_S(t, j % NB), a_desc[kk], k_desc + (uint64_t)(((kk >> 2) * (kBN * 128) + (kk & 3) * 32) >> 4),
@@ -579,9 +610,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // (the row tiles' softmax groups finish a tile one after the other, so one warp serves them in that order)
         if (nt > 0) {
             constexpr uint32_t idesc_pv = instr_desc_bf16(kBM, D, true);
+            bool ok = true;  // this lane's own record, as in the QK issuer
             for (int j = 0; j < nt; ++j) {
                 const int s = j % S, it = j / S;
-                mbar_wait(BAR(V_FULL + s), it & 1, dead);
+                ok &= mbar_wait(BAR(V_FULL + s), it & 1, dead, limit);
                 if ((t0 + j) * kBN + kBN > Ltot) {
                     // last, partial tile of the sequence: rows past the end may hold anything (even NaN); P is 0 there
                     // but 0 * NaN would poison O, so those V rows are cleared before the product reads them -- here, by
@@ -599,9 +631,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                 for (int t = 0; t < NM; ++t) {
                     if (t >= nm_act) break;
-                    mbar_wait(P_FULL(t, j % NB), (j / NB) & 1, dead);
+                    ok &= mbar_wait(P_FULL(t, j % NB), (j / NB) & 1, dead, limit);
                     tc_fence_after();
-                    if (elect_one()) {
+                    if (elect_one() && ok) {
 #pragma unroll
                         for (int kk = 0; kk < kBN / 16; ++kk)
                             // A = P in tensor memory, over the first 32 columns of the score buffer: 8 columns per K step
@@ -655,17 +687,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const uint32_t lane_off = (uint32_t)(wq * 32) << 16;
         float m = -1e30f, l = 0.f;  // m: offset in use (scaled, log2 units); never -inf so that exp2(-inf - m) = 0
         const float sc = prm.scale_log2;
+        bool alive = true;  // false once this warp has seen a wait of the CTA given up
 
         if (warp_active)
             for (int j = tc; j < nt; j += TC) {
                 const int kv0 = (t0 + j) * kBN;
-                mbar_wait_warp(S_FULL(t, j % NB), (j / NB) & 1, dead);
+                mbar_wait_warp(S_FULL(t, j % NB), (j / NB) & 1, dead, limit);
                 tc_fence_after();
                 float sv[CW];
                 {
                     uint32_t sr[CW];
                     tmem_ld_cols<CW>(TM_S(t, j % NB) + lane_off + c0, sr);
+                    const int gave_up = *dead;  // one word for the whole warp, read while the scores are on their way
                     tmem_wait_ld();
+                    if (gave_up) {  // a wait of this CTA ran out: nothing further is computed or stored
+                        alive = false;
+                        break;
+                    }
 #pragma unroll
                     for (int c = 0; c < CW; ++c) sv[c] = __uint_as_float(sr[c]);
                 }
@@ -732,7 +770,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const int i_own = (j - tc) / TC;
                 const bool any_grow = __any_sync(0xffffffffu, grow);
                 if (i_own > 0 && (NB != 2 * TC || any_grow || i_own == n_own - 1)) {
-                    mbar_wait_warp(PV_DONE(t, tc), (i_own - 1) & 1, dead);
+                    mbar_wait_warp(PV_DONE(t, tc), (i_own - 1) & 1, dead, limit);
                     tc_fence_after();
                     if (any_grow) {
 #pragma unroll
@@ -769,14 +807,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
         // ---- this split's (and copy's) result for the row: (m, l, unnormalised O)
         if (warp_active && n_own > 0) {
-            mbar_wait_warp(PV_DONE(t, tc), (n_own - 1) & 1, dead);
+            mbar_wait_warp(PV_DONE(t, tc), (n_own - 1) & 1, dead, limit);
             tc_fence_after();
         }
         const bool node_valid = row_ok && node < n;
         if (prm.mode == kModeCluster) {
             // every MMA of the CTA has finished before any tile buffer is reused for the parked partials
             named_bar_sync(1, NM * TC * 128);
-            if (warp_active) {
+            // a warp that saw a wait of its CTA given up parks, merges and stores nothing (copies may still be landing in
+            // the tile buffers); it keeps taking the barriers so that nobody waits for it
+            if (warp_active && alive) {
                 // the thread's row (of its copy, of its turn) is parked as an exchange row
                 unsigned char* xo = base_ptr + (size_t)((t * TC + tc) * kBM + row) * XS;
                 const float inv_l = (n_own > 0 && l > 0.f) ? 1.f / l : 0.f;
@@ -809,7 +849,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 constexpr int CPT = D / REP;  // columns per thread
                 const int tid = (int)threadIdx.x - 32 * Cfg::kRoleWarps;
                 const int r = tid % RB, col0 = (tid / RB) * CPT;
-                const bool mine = r < rows_t;
+                const bool mine = r < rows_t && alive;
                 float acc[CPT], M = -INFINITY, den = 0.f;
 #pragma unroll
                 for (int k = 0; k < CPT; ++k) acc[k] = 0.f;
@@ -860,7 +900,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     if (col0 == 0) *reinterpret_cast<float2*>(xo + 2 * D) = make_float2(M, den);
                 }
             }
-        } else if (warp_active && run) {
+        } else if (warp_active && run && alive) {
             const bool direct = prm.mode == kModeDirect;  // REP == 1 then
             const size_t orow = (size_t)(b * prm.Hq + hk * G) * T + gr;  // row of the [B*Hq*T, d] view of out
             const float inv = (node_valid && l > 0.f) ? 1.f / l : 0.f;
@@ -911,6 +951,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         __syncwarp();
         cluster_sync_all();
         const bool run = (flags | *bad_s) == 0;
+        const int gave_up = *dead;  // (a CTA that gave up stores nothing; only the stores wait for this word)
         const uint32_t rank = cluster_ctarank();
         const unsigned char* recv = base_ptr + Cfg::kQBytes + 2 * S * Cfg::kTileBytes;
         constexpr int EPL = D / 32;
@@ -940,6 +981,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const float inv = ((gr % T) < n && den > 0.f) ? 1.f / den : 0.f;
                 __nv_bfloat16* dst = prm.out + ((size_t)(b * prm.Hq + hk * G) * T + gr) * D + lane * EPL;
                 const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
+                if (gave_up) break;
                 if (EPL == 4) {
                     const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[2] * inv, num[3] * inv);
                     *reinterpret_cast<uint2*>(dst) =
@@ -956,7 +998,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         //      all requests in flight before the first use -- a remote read takes about a microsecond
         __syncwarp();
         cluster_sync_all();
-        const bool run = (flags | *bad_s) == 0;  // the same in every CTA of the cluster: it depends on the sequence only
+        // the same in every CTA of the cluster: it depends on the sequence only
+        const bool run = (flags | *bad_s) == 0;
+        const int gave_up = *dead;  // a CTA that gave up a wait stores nothing; only the stores wait for this word
         const uint32_t rank = cluster_ctarank();
         // row copies were merged inside their CTA (one exchange row per row, behind the parked copies); turns are
         // merged here with the splits
@@ -1023,7 +1067,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    if (!ok[u]) continue;
+                    if (!ok[u] || gave_up) continue;
                     const int gr = (mt0 + tt[u]) * kBM + lr[u];
                     const float inv = ((gr % T) < n && den[u] > 0.f) ? 1.f / den[u] : 0.f;
                     __nv_bfloat16* dst = prm.out + ((size_t)(b * prm.Hq + hk * G) * T + gr) * D + lane * EPL;
@@ -1042,7 +1086,25 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     } else {
         __syncthreads();
     }
-    if (threadIdx.x == 0 && *dead && prm.status) atomicOr(prm.status + b, S4C_SEQ_TIMEOUT);
+    if (*dead) {  // read behind a CTA-wide barrier: the same in every thread
+        // A wait was given up.  Before shared and tensor memory are handed back, everything this CTA set in motion is
+        // seen to completion (bounded like every wait): a bulk copy that lands after the CTA has left would land in its
+        // successor on the SM, a product that still runs would write tensor memory that is no longer this CTA's.
+        if (warp == 0 && lane == 0 && nt > 0) {
+            const int issued = *issued_s;
+            mbar_drain(BAR(Q_FULL), 0, limit);
+            for (int j = issued > S ? issued - S : 0; j < issued; ++j)
+                if (j != prm.withhold_tile)
+                    mbar_drain(BAR(K_FULL + j % S), (j / S) & 1, limit), mbar_drain(BAR(V_FULL + j % S), (j / S) & 1, limit);
+        }
+        if (warp >= 1 && warp <= NM + 1) {  // the issuer warps: a commit covers the products its own thread issued
+            if (elect_one()) tc_commit(BAR(DRAIN + warp - 1));
+            __syncwarp();
+            mbar_drain(BAR(DRAIN + warp - 1), 0, limit);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0 && prm.status) atomicOr(prm.status + b, S4C_SEQ_TIMEOUT);
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem, Cfg::kTmemCols);
@@ -1250,11 +1312,14 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
 // deals out the tiles of the true length, whatever that is.
 s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
-                             int d, int C_slots, int span, float scale, int32_t* status, void* ws, cudaStream_t stream) {
+                             int d, int C_slots, int span, float scale, int32_t* status, void* ws, cudaStream_t stream,
+                             int wait_limit_us, int withhold_tile) {
     TcParams prm;
     prm.cache_len = cache_len, prm.parent = parent, prm.n_nodes = n_nodes;
     prm.out = static_cast<__nv_bfloat16*>(out), prm.ws = static_cast<float*>(ws), prm.status = status;
     prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C_slots;
+    prm.wait_limit = wait_limit_us > 0 ? 2000ll * wait_limit_us : kWaitLimitCycles;  // about 2 cycles per nanosecond
+    prm.withhold_tile = withhold_tile;
     const int C = span;  // every choice below is made for the live span
     const int nm = tc_nm(B, T, Hq, Hkv, C);
     prm.m_groups = tc_m_groups(B, T, Hq, Hkv, C);

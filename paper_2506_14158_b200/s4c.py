@@ -21,7 +21,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
 
 EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
-           "s4c_launch_floor"]
+           "s4c_launch_floor", "s4c_selftest_attention_timeout"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -55,6 +55,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_accept_noalloc.argtypes = [vp, vp, i32p, i32p, i32p, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp]
     lib.s4c_kv_compact.restype = i
     lib.s4c_kv_compact.argtypes = [vp, vp, i, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i32p, vp]
+    lib.s4c_selftest_attention_timeout.restype = i
+    lib.s4c_selftest_attention_timeout.argtypes = [vp, vp, vp, i32p, i32p, vp, i, i, i, i, i, i, i, i, i, i32p, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -251,3 +253,17 @@ def launch_floor(ctas: int, cluster: int, threads: int, smem_bytes: int, tmem_co
                                1 if dependent_launch else 0, _dev(word, torch.int32, "word"), None, _stream(stream))
     if rc:
         raise S4CError("s4c_launch_floor", rc)
+
+
+def selftest_attention_timeout(q, k_cache, v_cache, cache_len, parent, out, status, withhold_tile: int, limit_us: int,
+                               max_cache_len: int = 0, stream=None):
+    """s4c_selftest_attention_timeout: the attention launch with one cache tile per CTA withheld and a short wait limit."""
+    B, Hq, T, d = q.shape
+    _, Hkv, C, _ = k_cache.shape
+    rc = _lib.s4c_selftest_attention_timeout(
+        _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache"),
+        _dev(cache_len, torch.int32, "cache_len"), _dev(parent, torch.int32, "parent"), _dev(out, torch.bfloat16, "out"),
+        B, T, Hq, Hkv, d, C, int(max_cache_len), int(withhold_tile), int(limit_us), _dev(status, torch.int32, "status"),
+        _stream(stream))
+    if rc:
+        raise S4CError("s4c_selftest_attention_timeout", rc)
