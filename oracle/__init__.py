@@ -11,6 +11,8 @@ Functions (array layouts are row-major numpy arrays):
 * :func:`accept_greedy`       -- Section 4.1.2 greedy decoding + Section 3.2 longest accepted path.
 * :func:`accept_stochastic`   -- Section 2 speculative sampling, Eq. 11 / Eq. 12, step by step.
 * :func:`kv_compact`          -- Section 3.2 last paragraph: keep accepted tokens' K/V and features.
+* :func:`build_tree`          -- Section 3.2 / Figure 3: the continuous verification tree (vertical top-1 chain, then
+                                 horizontal top-k alternatives), breadth-first numbered.
 """
 from __future__ import annotations
 
@@ -190,3 +192,23 @@ def kv_compact(k_caches, v_caches, cache_len, path, accept_len, T, feat_in=None,
     if rc:
         raise ValueError(f"oracle kv_compact rejected its arguments (code {rc})")
     return status
+
+
+def build_tree(draft_probs, branching, root_token, cache_len=None):
+    """draft_probs [B,T,V] f32, branching (sequence of ints), root_token [B] -> dict(tokens, parent, position [B,T], n_nodes [B])."""
+    draft_probs = np.ascontiguousarray(draft_probs, dtype=np.float32)
+    B, T, V = draft_probs.shape
+    br = np.ascontiguousarray(branching, dtype=np.int32)
+    root_token = _i32(root_token).reshape(B)
+    cache_len = _i32(cache_len)
+    tokens = np.full((B, T), -7, dtype=np.int32)
+    parent = np.full((B, T), -7, dtype=np.int32)
+    position = np.full((B, T), -7, dtype=np.int32)
+    n_nodes = np.full(B, -7, dtype=np.int32)
+    f32, i32 = ctypes.c_float, ctypes.c_int32
+    rc = _load().s4c_oracle_build_tree(_ptr(draft_probs, f32), _ptr(br, i32), int(len(br)), _ptr(root_token, i32),
+                                       _ptr(cache_len, i32), B, T, V, _ptr(tokens, i32), _ptr(parent, i32),
+                                       _ptr(position, i32), _ptr(n_nodes, i32))
+    if rc:
+        raise ValueError(f"oracle build_tree rejected its arguments (code {rc})")
+    return dict(tokens=tokens, parent=parent, position=position, n_nodes=n_nodes)

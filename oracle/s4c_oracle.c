@@ -26,6 +26,11 @@
  *   s4c_oracle_kv_compact      Section 3.2, last paragraph (accepted tokens and
  *                              their features are kept for the next drafting
  *                              phase): a gather from a snapshot.
+ *   s4c_oracle_build_tree      Section 3.2 and Figure 3 (left): the continuous
+ *                              verification tree -- a vertical chain of top-1
+ *                              drafts, then horizontal top-k alternatives at
+ *                              every position -- built step by step as the
+ *                              section tells it, then numbered breadth-first.
  *
  * Readings of silent or garbled points (symbols follow Section 2: p = target,
  * q = draft):
@@ -48,7 +53,9 @@
  * greedy verify == token-by-token greedy decoding, planted trees; exact
  * enumeration on dyadic tiny-vocab cases and chi-square Monte-Carlo showing the
  * emitted token follows the target distribution; compaction against a library
- * gather.  The paper prints no worked numeric example for any of these steps,
+ * gather; tree construction against the example of Figure 3 as Section 3.2
+ * describes it, an independently written construction plus a library sort,
+ * and the structural facts (first sibling = top-1, rank order, breadth-first).  The paper prints no worked numeric example for any of these steps,
  * so config-level values are: parity unpinned by printed numbers (pinned by the
  * invariants above instead).
  */
@@ -466,5 +473,110 @@ int s4c_oracle_kv_compact(uint8_t* const* k_caches, uint8_t* const* v_caches, in
         cache_len[b] = L + a + 1;
     }
     free(snap);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Continuous verification tree (Section 3.2; Figure 3, left).                */
+/*                                                                           */
+/* The tree starts at the last committed token (the root).  Drafts are first  */
+/* generated "vertically": a chain of top-1 choices, one per drafting depth.  */
+/* Then the tree is extended "horizontally", depth by depth: every node at    */
+/* depth l-1 receives the top-k alternatives at its position until it has     */
+/* branching[l-1] children (its first child is the top-1 choice, the others   */
+/* the 2nd, 3rd ... most probable tokens of the same distribution).  Growth   */
+/* stops at T nodes.  Nodes are then numbered breadth-first, which makes      */
+/* parent[i] < i, keeps siblings contiguous and in rank order.                */
+/*                                                                           */
+/* draft_probs [B,T,V] float32: row n (in the final numbering) is the         */
+/*             distribution the children of node n are chosen from -- the     */
+/*             same array s4c_oracle_accept_stochastic reads.                 */
+/* branching   [D] children per node at depths 0..D-1 (>= 1 each)             */
+/* root_token  [B]; cache_len [B] or NULL                                     */
+/* tokens, parent, position [B,T]; n_nodes [B]                                */
+/*   child j (j = 1..k) of node n carries the j-th most probable token of     */
+/*   row n, ties going to the lower token index; position = cache_len + depth */
+/*   (0-based depth; just the depth when cache_len is NULL).  Entries beyond  */
+/*   n_nodes[b] are padding: parent -1, token 0, position 0.                  */
+/* The shape depends on (branching, T) only, so it is the same for every      */
+/* sequence of the batch; the tokens differ.                                  */
+/* Readings: "top-k alternatives at the same position" are the siblings of    */
+/* the top-1 token (children of the same parent), as the example of Figure 3  */
+/* has it (two continuations of the root, each with a top-1 successor and two */
+/* alternatives to that successor); nodes added horizontally are expanded at  */
+/* the next depth like the vertical ones.                                     */
+/* ------------------------------------------------------------------------- */
+int s4c_oracle_build_tree(const float* draft_probs, const int32_t* branching, int D,
+                          const int32_t* root_token, const int32_t* cache_len, int B, int T, int V,
+                          int32_t* tokens, int32_t* parent, int32_t* position, int32_t* n_nodes) {
+    if (!draft_probs || !branching || !root_token || !tokens || !parent || !position || !n_nodes) return 1;
+    if (B < 0 || T < 1 || V < 1 || D < 0) return 2;
+    for (int l = 0; l < D; ++l)
+        if (branching[l] < 1 || branching[l] > V) return 2;
+    /* ---- the shape, in creation order */
+    int* cpar = (int*)malloc(sizeof(int) * (size_t)T);
+    int* cdep = (int*)malloc(sizeof(int) * (size_t)T);
+    int* nchild = (int*)calloc((size_t)T, sizeof(int));
+    int n = 1;
+    cpar[0] = -1, cdep[0] = 0;
+    /* vertically: the chain of top-1 choices */
+    for (int l = 0, tip = 0; l < D && n < T; ++l) {
+        cpar[n] = tip, cdep[n] = l + 1, nchild[tip] += 1;
+        tip = n++;
+    }
+    /* horizontally: depth by depth, alternatives at the same position */
+    for (int l = 1; l <= D; ++l)
+        for (int node = 0; node < n; ++node) {
+            if (cdep[node] != l - 1) continue;
+            while (nchild[node] < branching[l - 1] && n < T) {
+                cpar[n] = node, cdep[n] = l, nchild[node] += 1;
+                ++n;
+            }
+        }
+    /* ---- breadth-first numbering: visit order = new index; children keep their creation order */
+    int* order = (int*)malloc(sizeof(int) * (size_t)n);   /* order[new] = creation index */
+    int* newid = (int*)malloc(sizeof(int) * (size_t)n);
+    int head = 0, tail = 0;
+    order[tail++] = 0;
+    while (head < tail) {
+        const int u = order[head++];
+        for (int c = 0; c < n; ++c)
+            if (cpar[c] == u) order[tail++] = c;
+    }
+    for (int i = 0; i < n; ++i) newid[order[i]] = i;
+    int* par = (int*)malloc(sizeof(int) * (size_t)n);
+    int* dep = (int*)malloc(sizeof(int) * (size_t)n);
+    for (int i = 0; i < n; ++i) {
+        par[i] = order[i] == 0 ? -1 : newid[cpar[order[i]]];
+        dep[i] = cdep[order[i]];
+    }
+    /* ---- tokens: the children of a node, in index order, take the 1st, 2nd, ... most probable token of its row */
+    unsigned char* taken = (unsigned char*)malloc((size_t)V);
+    for (int b = 0; b < B; ++b) {
+        int32_t* tok = tokens + (size_t)b * T;
+        int32_t* pr = parent + (size_t)b * T;
+        int32_t* pos = position + (size_t)b * T;
+        const int base = cache_len ? cache_len[b] : 0;
+        for (int i = 0; i < T; ++i) {
+            pr[i] = i < n ? par[i] : -1;
+            pos[i] = i < n ? base + dep[i] : 0;
+            tok[i] = 0;
+        }
+        tok[0] = root_token[b];
+        n_nodes[b] = n;
+        for (int u = 0; u < n; ++u) {
+            const float* row = draft_probs + ((size_t)b * T + u) * V;
+            memset(taken, 0, (size_t)V);
+            for (int c = u + 1; c < n; ++c) {
+                if (par[c] != u) continue;
+                int best = -1;  /* most probable token not taken yet; the lowest index among equals */
+                for (int v = 0; v < V; ++v)
+                    if (!taken[v] && (best < 0 || row[v] > row[best])) best = v;
+                taken[best] = 1;
+                tok[c] = best;
+            }
+        }
+    }
+    free(taken), free(par), free(dep), free(order), free(newid), free(cpar), free(cdep), free(nchild);
     return 0;
 }
