@@ -355,6 +355,13 @@ def measure(cfg, args, device, rank, world, with_e2e):
     attn_blocks = time_blocks(g_attn, K, torch, args.min_seconds / 2)
     ms_acc = time_graph(g_acc, K, torch)  # L2-resident when the logits fit L2: informational only
     ms_cmp = time_graph(g_cmp, K, torch)
+    # the tree itself, built on the device from the draft probabilities (not part of the timed step: the step takes the
+    # tree as input, as the three verify calls do); only for workloads whose tree comes from branching factors
+    ms_tree = None
+    if cfg.tree == "branching" and args.temperature > 0:
+        step.enable_tree_build(cfg.branching, step.tokens[:, 0].contiguous())
+        g_tree = step.capture("tree")
+        ms_tree = time_graph(g_tree, K, torch)
     ms_e2e = 0.0
     if with_e2e:
         # end to end: per-step inputs from pinned host memory, decision back to the host, every step
@@ -375,7 +382,7 @@ def measure(cfg, args, device, rank, world, with_e2e):
         [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
         device=device)
     rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
-               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_e2e=ms_e2e, accept_lens=accept_lens,
                clocks=clocks, K=K, Wm=Wm)
     return rec
 
@@ -410,6 +417,8 @@ def roofline_records(cfg, args, rec, pk):
                     us_per_launch=attn_launch_ms * 1e3, us_per_launch_best=rec["ms_attn_best"] / cfg.n_layers * 1e3,
                     flop_per_kv_byte=intensity, ridge_flop_per_byte=ridge, hbm=hbm, tensor=tensor)
     breakdown = dict(attention_all_layers=rec["ms_attn"], accept=rec["ms_acc"], compact=rec["ms_cmp"])
+    if rec.get("ms_tree") is not None:
+        breakdown["tree_build_not_in_step"] = rec["ms_tree"]
     return ab, step_hbm, roofline, breakdown
 
 

@@ -8,6 +8,8 @@
  *   per decoder layer:  s4c_tree_attention   tree-masked attention of the T tree tokens
  *   once per step:      s4c_tree_accept      greedy / speculative-sampling acceptance + path walk
  *   once per step:      s4c_kv_compact       keep the accepted path's K/V (all layers) and features
+ * and, before them, optionally
+ *   once per step:      s4c_tree_build       the tree itself, from the drafter's distributions
  *
  * Conventions for every entry point
  *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
@@ -212,6 +214,42 @@ s4c_status s4c_kv_compact(void* const* k_caches, void* const* v_caches, int n_la
                           const int32_t* path, const int32_t* accept_len, int max_depth,
                           const void* feat_in, void* feat_out, int B, int T, int Hkv, int d, int C, int hid,
                           s4c_dtype dt, int32_t* status, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * s4c_tree_build -- the continuous verification tree of Section 3.2 (drawn in Figure 3, left),
+ * built on the device from the drafter's distributions, in the layout the three calls above consume.
+ *
+ * Shape.  The root (node 0) is the last committed token.  Drafts are generated vertically first: a
+ * chain of top-1 choices, one per drafting depth (`depth` levels).  Then the tree is extended
+ * horizontally, depth by depth: every node at depth l (vertical or horizontal) gets the top-k
+ * alternatives at its position until it has branching[l] children -- its first child is the top-1
+ * choice, the others the 2nd, 3rd, ... most probable tokens of the same distribution.  Growth stops
+ * at T nodes.  Nodes are numbered breadth-first, so parent[i] < i, siblings are contiguous and in
+ * rank order.  The shape depends on (branching, T) only and is the same for every sequence.
+ * Tokens.  Child j (j = 1..k) of node n carries the j-th most probable token of draft_probs[b,n,:],
+ * ties going to the lower token index.
+ *
+ *   draft_probs [B,T,V] f32   row n: the drafter's distribution for the token after node n (the array
+ *                             s4c_tree_accept takes); rows of nodes without children are not read.
+ *                             Entries must not be NaN.
+ *   branching   [depth] int32, HOST memory: children per node at depths 0..depth-1, each 1..16 and <= V
+ *   root_token  [B] int32     the last committed token of each sequence
+ *   cache_len   [B] int32 or NULL
+ *   tokens, parent, position [B,T] int32  out: position[b,i] = cache_len[b] + depth of node i (the
+ *                             position id of the node's K/V slot content; just the depth if cache_len is
+ *                             NULL); entries of unused nodes (i >= n_nodes[b]): parent -1, token 0, position 0
+ *   n_nodes     [B] int32     out: nodes in use, min(T, size of the full tree)
+ *   workspace   at least s4c_tree_build_workspace_bytes(B, T, V, max over branching) bytes, 256-byte
+ *               aligned, scratch (per-segment candidates of the top-k selection)
+ * Asynchronous on `stream`; the host never reads the tree: tokens / parent / n_nodes go straight to
+ * s4c_tree_attention, s4c_tree_accept and s4c_kv_compact on the same stream.
+ * ------------------------------------------------------------------------------------------ */
+size_t s4c_tree_build_workspace_bytes(int B, int T, int V, int max_branch);
+
+s4c_status s4c_tree_build(const float* draft_probs, const int32_t* branching, int depth, const int32_t* root_token,
+                          const int32_t* cache_len, int B, int T, int V, int32_t* tokens, int32_t* parent,
+                          int32_t* position, int32_t* n_nodes, void* workspace, size_t workspace_bytes,
+                          s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
  * s4c_launch_floor -- a measurement aid; the paper has no counterpart.

@@ -21,7 +21,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
 
 EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
-           "s4c_launch_floor", "s4c_selftest_attention_timeout"]
+           "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -57,6 +57,10 @@ def _load() -> ctypes.CDLL:
     lib.s4c_kv_compact.argtypes = [vp, vp, i, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i32p, vp]
     lib.s4c_selftest_attention_timeout.restype = i
     lib.s4c_selftest_attention_timeout.argtypes = [vp, vp, vp, i32p, i32p, vp, i, i, i, i, i, i, i, i, i, i32p, vp]
+    lib.s4c_tree_build_workspace_bytes.restype = sz
+    lib.s4c_tree_build_workspace_bytes.argtypes = [i, i, i, i]
+    lib.s4c_tree_build.restype = i
+    lib.s4c_tree_build.argtypes = [vp, vp, i, i32p, i32p, i, i, i, i32p, i32p, i32p, i32p, vp, sz, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -267,3 +271,33 @@ def selftest_attention_timeout(q, k_cache, v_cache, cache_len, parent, out, stat
         _stream(stream))
     if rc:
         raise S4CError("s4c_selftest_attention_timeout", rc)
+
+
+def tree_build_workspace_bytes(B, T, V, max_branch) -> int:
+    return int(_lib.s4c_tree_build_workspace_bytes(B, T, V, max_branch))
+
+
+def tree_build(draft_probs, branching: Sequence[int], root_token, cache_len=None, tokens=None, parent=None, position=None,
+               n_nodes=None, workspace=None, stream=None):
+    """s4c_tree_build: draft_probs [B,T,V] f32, branching (host ints), root_token [B] ->
+    dict(tokens, parent, position [B,T], n_nodes [B]), all int32 on the device."""
+    B, T, V = draft_probs.shape
+    dev = draft_probs.device
+    i32 = dict(dtype=torch.int32, device=dev)
+    tokens = torch.empty(B, T, **i32) if tokens is None else tokens
+    parent = torch.empty(B, T, **i32) if parent is None else parent
+    position = torch.empty(B, T, **i32) if position is None else position
+    n_nodes = torch.empty(B, **i32) if n_nodes is None else n_nodes
+    br = (ctypes.c_int32 * max(1, len(branching)))(*[int(x) for x in branching])
+    need = int(_lib.s4c_tree_build_workspace_bytes(B, T, V, max([1] + [int(x) for x in branching])))
+    if workspace is None:
+        workspace = _workspace(need, dev, "tree")
+    rc = _lib.s4c_tree_build(
+        _dev(draft_probs, torch.float32, "draft_probs"), ctypes.cast(br, ctypes.c_void_p), len(branching),
+        _dev(root_token, torch.int32, "root_token"), _dev(cache_len, torch.int32, "cache_len"), B, T, V,
+        _dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"), _dev(position, torch.int32, "position"),
+        _dev(n_nodes, torch.int32, "n_nodes"), _dev(workspace, name="workspace"),
+        0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_build", rc)
+    return dict(tokens=tokens, parent=parent, position=position, n_nodes=n_nodes)

@@ -1,4 +1,5 @@
-"""One whole S4C verify step on device buffers: n_layers x s4c_tree_attention, s4c_tree_accept, s4c_kv_compact.
+"""One whole S4C verify step on device buffers: [s4c_tree_build,] n_layers x s4c_tree_attention, s4c_tree_accept,
+s4c_kv_compact.
 
 :class:`VerifyStep` owns nothing but references to the caller's tensors plus the small output / scratch tensors
 it allocates once.  ``run()`` enqueues the step on the current stream through the C ABI; ``capture()`` records
@@ -21,8 +22,12 @@ class VerifyStep:
                  cache_len: torch.Tensor, parent: torch.Tensor, tokens: torch.Tensor, target_logits: torch.Tensor,
                  draft_probs: Optional[torch.Tensor], uniforms: Optional[torch.Tensor], temperature: float,
                  max_depth: int, n_nodes: Optional[torch.Tensor] = None, feat_in: Optional[torch.Tensor] = None,
-                 stacked: Optional[tuple] = None, max_cache_len: int = 0):
-        """``max_cache_len``: what the host knows about the committed lengths (an upper bound, 0 = nothing); it is handed
+                 stacked: Optional[tuple] = None, max_cache_len: int = 0, branching: Optional[tuple] = None,
+                 root_token: Optional[torch.Tensor] = None):
+        """``branching`` (+ ``root_token`` [B] int32): the step then starts with s4c_tree_build, which writes the tree
+        (``tokens``, ``parent``, ``n_nodes``, position ids) from ``draft_probs`` on the device -- no host tree in the loop;
+        ``parent`` and ``tokens`` are then only buffers of the right shape.
+        ``max_cache_len``: what the host knows about the committed lengths (an upper bound, 0 = nothing); it is handed
         to every s4c_tree_attention call, which shapes its launch for it instead of for the capacity.
         ``stacked`` = (q_all [n_layers,B,Hq,T,d], k_all, v_all [n_layers,B,Hkv,C,d]) when the per-layer tensors are
         views of three big ones: the host-buffer path then moves a step's inputs with three copies instead of three
@@ -35,6 +40,7 @@ class VerifyStep:
         self.logits, self.draft_probs, self.uniforms = target_logits, draft_probs, uniforms
         self.temperature, self.max_depth = float(temperature), int(max_depth)
         self.max_cache_len = int(max_cache_len)
+        self.branching, self.root_token = None, None
         self.feat_in = feat_in
         dev = cache_len.device
         B, T, V = target_logits.shape
@@ -61,10 +67,28 @@ class VerifyStep:
         self.k_ptrs = s4c.cache_pointer_array(k_caches)
         self.v_ptrs = s4c.cache_pointer_array(v_caches)
         self.stacked = stacked
+        if branching is not None:
+            self.enable_tree_build(branching, root_token)
         self.graph: Optional[torch.cuda.CUDAGraph] = None
         self._host = None
 
-    # ------------------------------------------------------------------ the three stages
+    # ------------------------------------------------------------------ the stages
+    def enable_tree_build(self, branching, root_token: torch.Tensor):
+        """From now on ``run()`` starts with s4c_tree_build (see the constructor)."""
+        assert self.draft_probs is not None and root_token is not None, "building the tree needs draft_probs and root_token"
+        self.branching = tuple(int(x) for x in branching)
+        self.root_token = root_token
+        i32 = dict(dtype=torch.int32, device=self.cache_len.device)
+        if self.n_nodes is None:
+            self.n_nodes = torch.full((self.B,), self.T, **i32)
+        self.position = torch.empty(self.B, self.T, **i32)
+        self.ws_tree = torch.empty(max(1, s4c.tree_build_workspace_bytes(self.B, self.T, self.V, max((1,) + self.branching))),
+                                   dtype=torch.uint8, device=self.cache_len.device)
+
+    def build_tree(self):
+        s4c.tree_build(self.draft_probs, self.branching, self.root_token, self.cache_len, tokens=self.tokens,
+                       parent=self.parent, position=self.position, n_nodes=self.n_nodes, workspace=self.ws_tree)
+
     def attention(self, l0: int = 0, l1: Optional[int] = None):
         for l in range(l0, self.n_layers if l1 is None else l1):
             s4c.tree_attention(self.q[l], self.k_caches[l], self.v_caches[l], self.cache_len, self.parent, self.n_nodes,
@@ -86,6 +110,8 @@ class VerifyStep:
 
     def run(self):
         self.reset_lengths()
+        if self.branching is not None:
+            self.build_tree()
         self.attention()
         self.accept()
         self.compact()
@@ -95,7 +121,8 @@ class VerifyStep:
         # acceptance: per-node statistics (one launch, cluster or segment kernel) and the walk
         accept = 2
         compact = 2 if self.n_layers > 0 else 1
-        return self.n_layers * attn_launches_per_layer + accept + compact
+        tree = 2 if self.branching is not None else 0
+        return self.n_layers * attn_launches_per_layer + accept + compact + tree
 
     # ------------------------------------------------------------------ CUDA graph
     def capture(self, what: str = "step") -> torch.cuda.CUDAGraph:
@@ -103,7 +130,7 @@ class VerifyStep:
             l0, l1 = (int(x) for x in what.split(":")[1:])
             fn = lambda: ((self.reset_lengths() if l0 == 0 else None), self.attention(l0, l1))
         else:
-            fn = {"step": self.run, "attention": self.attention, "accept": self.accept,
+            fn = {"step": self.run, "attention": self.attention, "accept": self.accept, "tree": self.build_tree,
                   "compact": lambda: (self.reset_lengths(), self.compact()),
                   "head": lambda: (self.reset_lengths(), self.attention()),
                   "tail": lambda: (self.accept(), self.compact())}[what]

@@ -95,4 +95,20 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert cmp_(fi=P) == 1                       # feat_in without feat_out
     assert cmp_(dt=9) == 3
     assert cmp_(B=0) == 0
+    lib.s4c_tree_build.argtypes = [vp, vp, i, vp, vp, i, i, i, vp, vp, vp, vp, vp, sz, vp]
+    lib.s4c_tree_build_workspace_bytes.restype = sz
+    lib.s4c_tree_build_workspace_bytes.argtypes = [i, i, i, i]
+    br = (ctypes.c_int32 * 3)(4, 3, 2)
+    tb = lambda **kw: lib.s4c_tree_build(*[kw.get(k, d) for k, d in [
+        ("q", P), ("br", ctypes.cast(br, vp)), ("D", 3), ("root", P), ("cl", None), ("B", 1), ("T", 26), ("V", 32000),
+        ("tok", P), ("par", P), ("pos", P), ("nn", P), ("ws", None), ("wsb", 0), ("s", None)]])
+    assert tb(q=None) == 1 and tb(nn=None) == 1 and tb(br=None) == 1
+    assert tb(T=129) == 2 and tb(V=0) == 2 and tb(V=3) == 2     # V = 3: fewer tokens than the 4 children of the root
+    assert tb(q=P + 4) == 4
+    assert tb() == 5                                            # no workspace
+    assert tb(B=0) == 0
+    bad = (ctypes.c_int32 * 2)(17, 1)
+    assert tb(br=ctypes.cast(bad, vp), D=2) == 2                # more than 16 children
+    assert lib.s4c_tree_build_workspace_bytes(1, 26, 32000, 4) % 256 == 0 and lib.s4c_tree_build_workspace_bytes(1, 26, 32000, 4) > 0
+    assert lib.s4c_tree_build_workspace_bytes(1, 26, 32000, 17) == 0
     assert b"workspace" in lib.s4c_status_string(5)
