@@ -329,6 +329,7 @@ __device__ __forceinline__ void cl_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 // Reads 8 bytes at the same shared-memory offset in CTA `rank` of the cluster.
 __device__ __forceinline__ double cl_peer_f64(const double* local, uint32_t rank) {
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(local);
@@ -645,6 +646,9 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
     // With room in shared memory the target probabilities of this CTA's vocabulary range at the current node are kept
     // from the first vocabulary-wide pass there to the later ones (a float64 exp per entry is most of a pass).
     double* pc = reinterpret_cast<double*>(smem_raw + ((sizeof(WalkClShared) + 15) / 16) * 16);
+    // ... and, with still more room (cache_p0 == 2), the draft probabilities of the range beside them: a node where several
+    // siblings are rejected takes one pass per rejection, and all but the first then run from shared memory alone
+    float* qc = reinterpret_cast<float*>(pc + chunk);
     int cached_node = -1;  // node whose probabilities pc[] holds, complete after a whole pass (the same in every thread)
     // two cluster-wide sums in rank order; every thread of the cluster calls this and gets the same values
     auto cluster_sum2 = [&](double a, double bsum, double& A, double& Bs) {
@@ -683,7 +687,8 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int v = start + u * step;
-                xl[u] = (v < end && !hit) ? __ldg(lrow + v) : 0.f, ql[u] = v < end ? __ldg(qrow + v) : 0.f;
+                xl[u] = (v < end && !hit) ? __ldg(lrow + v) : 0.f;
+                ql[u] = v < end ? ((hit && cache_p0 == 2) ? qc[v - c0] : __ldg(qrow + v)) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -696,6 +701,7 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                     } else {
                         p0 = p0_from(xl[u]);
                         if (cache_p0) pc[v - c0] = p0;
+                        if (cache_p0 == 2) qc[v - c0] = ql[u];
                     }
                     chain_eval(p0, (double)ql[u], v, rr, sh, pv[u], qv[u]);
                 }
@@ -724,6 +730,10 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
                 Z = sh.nZ[cur], s = sh.nQ[cur];
             } else {
                 double z = 0.0, qs = 0.0;
+                if (!(cache_p0 && cached_node == cur))
+                    // first pass at this node: the rows come from global memory in batches of four loads per thread, each
+                    // batch a round trip; asking L2 for the later batches now leaves only the first at full latency
+                    for (int v = c0 + tid + 4 * (int)blockDim.x; v < c1; v += blockDim.x) prefetch_l2(lrow + v), prefetch_l2(qrow + v);
                 for (int v0 = c0 + tid; v0 < c1; v0 += 4 * blockDim.x) {
                     double pv[4], qv[4];
                     eval4(v0, blockDim.x, c1, r, pv, qv);
@@ -761,6 +771,8 @@ accept_walk_cluster_kernel(const float* __restrict__ logits, const float* __rest
         const int w0 = c0 + warp * seg, w1 = min(c1, w0 + seg);
         double acc = 0.0;
         int last = -1;
+        if (!(cache_p0 && cached_node == cur))  // (as above: a leaf, or a fork whose residual masses came precomputed)
+            for (int v = w0 + lane + 128; v < w1; v += 32) prefetch_l2(lrow + v), prefetch_l2(qrow + v);
         for (int v0 = w0 + lane; v0 < w1; v0 += 128) {
             double pv[4], qv[4];
             eval4(v0, 32, w1, r, pv, qv);
@@ -926,17 +938,19 @@ extern "C" s4c_status s4c_tree_accept(const float* target_logits, const float* d
     if (stoch) {
         cfg.gridDim = dim3(kCl, B, 1);
         cfg.blockDim = dim3(1024, 1, 1);
-        // room for the range's probabilities (8 bytes per vocabulary entry of a CTA) next to the walk's state?
+        // room for the range's target probabilities (8 bytes per vocabulary entry of a CTA), and for its draft
+        // probabilities too (4 more), next to the walk's state?
         const size_t walk_state = ((sizeof(WalkClShared) + 15) / 16) * 16;
-        const int cache_p0 = walk_state + (size_t)chunk * 8 <= 200 * 1024 ? 1 : 0;
-        cfg.dynamicSmemBytes = walk_state + (cache_p0 ? (size_t)chunk * 8 : 0);
+        const size_t walk_smem_max = 227 * 1024;
+        const int cache_p0 = walk_state + (size_t)chunk * 12 <= walk_smem_max ? 2 : (walk_state + (size_t)chunk * 8 <= walk_smem_max ? 1 : 0);
+        cfg.dynamicSmemBytes = walk_state + (size_t)chunk * (cache_p0 == 2 ? 12 : (cache_p0 == 1 ? 8 : 0));
         {
             static bool configured[64] = {};  // the opt-in to more than 48 KB of dynamic shared memory is per device
             int dev = 0;
             if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
             if (!configured[dev]) {
                 if (cudaFuncSetAttribute(accept_walk_cluster_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         200 * 1024) != cudaSuccess)
+                                         (int)walk_smem_max) != cudaSuccess)
                     return S4C_ERR_CUDA;
                 configured[dev] = true;
             }

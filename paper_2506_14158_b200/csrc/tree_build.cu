@@ -8,8 +8,9 @@
 // the j-th most probable token of draft row n.  That is a top-k selection over the vocabulary per expanded node -- a
 // streaming pass over the draft probabilities, bound by HBM bandwidth (every row of an expanded node is read once):
 //   tree_topk_segments_kernel  grid (vocabulary segments of 4096, expanded nodes, B): the segment sits in registers;
-//                              k rounds of a block-wide (maximum, lowest index) reduction, each round restricted to
-//                              entries that rank strictly after the previous winner, give the segment's k best
+//                              k rounds of a warp-wide (maximum, lowest index) reduction, each round restricted to
+//                              entries that rank strictly after the previous winner, give each warp's k best, and one
+//                              warp selects the segment's k best among those the same way
 //   tree_emit_kernel           grid (B): one warp per expanded node merges the segments' candidates the same way and
 //                              writes the children's tokens; the CTA also writes parent[], position ids and n_nodes
 // Ranking is (probability descending, token index ascending): ties go to the lower index, every run gives the same tree.
@@ -78,40 +79,44 @@ tree_topk_segments_kernel(const float* __restrict__ probs, const __grid_constant
 #pragma unroll
         for (int i = 0; i < kTbElems; ++i) x[i] = e[i] < V ? __ldg(row + e[i]) : -INFINITY;
     }
-    __shared__ float wp[kTbThreads / 32];
-    __shared__ int wt[kTbThreads / 32];
+    // Every warp first selects the k best of its own 512 entries (k rounds of shuffles, no CTA barrier), leaves them in
+    // shared memory, and after the one barrier warp 0 selects the segment's k best among the 8 k candidates.
+    __shared__ Cand wc[kTbThreads / 32][kMaxBranch];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float pp = INFINITY;  // previous winner: nothing ranks before (+inf, -1)
-    int pt = -1;
-    Cand* out = cand + (((size_t)b * shape.n_expanded + blockIdx.y) * gridDim.x + seg) * max_branch;
-    for (int r = 0; r < k; ++r) {
-        float bp = -INFINITY;
-        int bt = INT_MAX;  // "no entry left": ranks after every real entry
+    {
+        float pp = INFINITY;  // previous winner: nothing ranks before (+inf, -1)
+        int pt = -1;
+        for (int r = 0; r < k; ++r) {
+            float bp = -INFINITY;
+            int bt = INT_MAX;  // "no entry left": ranks after every real entry
 #pragma unroll
-        for (int i = 0; i < kTbElems; ++i)
-            if (e[i] < V && ranks_after(x[i], e[i], pp, pt) && ranks_before(x[i], e[i], bp, bt)) bp = x[i], bt = e[i];
-        warp_best(bp, bt);
-        if (lane == 0) wp[warp] = bp, wt[warp] = bt;
-        __syncthreads();
-        bp = wp[0], bt = wt[0];
-#pragma unroll
-        for (int w = 1; w < kTbThreads / 32; ++w)
-            if (ranks_before(wp[w], wt[w], bp, bt)) bp = wp[w], bt = wt[w];
-        __syncthreads();  // the arrays are rewritten in the next round
-        pp = bp, pt = bt;
-        if (threadIdx.x == 0) {
-            Cand c;
-            c.p = bp, c.tok = bt;
-            out[r] = c;
+            for (int i = 0; i < kTbElems; ++i)
+                if (e[i] < V && ranks_after(x[i], e[i], pp, pt) && ranks_before(x[i], e[i], bp, bt)) bp = x[i], bt = e[i];
+            warp_best(bp, bt);
+            pp = bp, pt = bt;
+            if (lane == 0) wc[warp][r].p = bp, wc[warp][r].tok = bt;
         }
-        if (bt == INT_MAX) {  // the segment is exhausted (the same in every thread): the remaining slots say so too
-            if (threadIdx.x == 0)
-                for (int q = r + 1; q < k; ++q) {
-                    Cand c;
-                    c.p = -INFINITY, c.tok = INT_MAX;
-                    out[q] = c;
-                }
-            break;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        Cand* out = cand + (((size_t)b * shape.n_expanded + blockIdx.y) * gridDim.x + seg) * max_branch;
+        constexpr int NW = kTbThreads / 32;
+        float pp = INFINITY;
+        int pt = -1;
+        for (int r = 0; r < k; ++r) {
+            float bp = -INFINITY;
+            int bt = INT_MAX;
+            for (int s = lane; s < NW * k; s += 32) {  // candidate (warp s / k, rank s % k)
+                const Cand v = wc[s / k][s % k];
+                if (v.tok != INT_MAX && ranks_after(v.p, v.tok, pp, pt) && ranks_before(v.p, v.tok, bp, bt)) bp = v.p, bt = v.tok;
+            }
+            warp_best(bp, bt);
+            pp = bp, pt = bt;
+            if (lane == 0) {  // an exhausted segment (fewer than k entries) leaves (-inf, INT_MAX) in the remaining slots
+                Cand c;
+                c.p = bt == INT_MAX ? -INFINITY : bp, c.tok = bt;
+                out[r] = c;
+            }
         }
     }
 }
