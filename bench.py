@@ -57,6 +57,8 @@ def parse_args():
     ap.add_argument("--no-hint", action="store_true", help="do not pass max_cache_len: launches are shaped for the capacity")
     ap.add_argument("--no-also", action="store_true", help="leave the 8B-shaped record out of the default line")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="keep timing K-step blocks until this much is timed")
+    ap.add_argument("--paged", type=int, default=0, help="page size in slots (64, 128, ...): the caches become pools of pages "
+                    "scattered at random, addressed through a block table (no host-buffer leg)")
     return ap.parse_args()
 
 
@@ -258,7 +260,7 @@ def config_record(cfg, args, world):
 
 
 # ----------------------------------------------------------------------------- the CUDA arm
-def build_step(cfg, temperature, device, seed_shift=0, hint=True):
+def build_step(cfg, temperature, device, seed_shift=0, hint=True, paged=0):
     import numpy as np
     import torch
 
@@ -290,12 +292,33 @@ def build_step(cfg, temperature, device, seed_shift=0, hint=True):
         qs[l].copy_(q), ks[l].copy_(k), vs[l].copy_(v)
         del q, k, v
     to = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    block_table = None
+    if paged:
+        # the same caches as pools of pages: page i of (sequence b, layer l) lies wherever a seeded permutation put it
+        ps = paged
+        nb = (cfg.C + ps - 1) // ps
+        n_pages = cfg.B * nb + 3
+        perm = np.random.default_rng(W.stream_seed(cfg_gen.config_id, "tree", 99)).permutation(n_pages)[: cfg.B * nb]
+        bt = torch.from_numpy(perm.reshape(cfg.B, nb).astype(np.int32)).to(device)
+        pools_k = torch.zeros((cfg.n_layers, n_pages, cfg.Hkv, ps, cfg.d), dtype=dt, device=device)
+        pools_v = torch.zeros_like(pools_k)
+        pad = nb * ps - cfg.C
+        for src, dst in ((k_all, pools_k), (v_all, pools_v)):
+            blk = torch.nn.functional.pad(src, (0, 0, 0, pad)) if pad else src                     # [n_layers,B,Hkv,nb*ps,d]
+            blk = blk.view(cfg.n_layers, cfg.B, cfg.Hkv, nb, ps, cfg.d).permute(0, 1, 3, 2, 4, 5)  # [n_layers,B,nb,Hkv,ps,d]
+            dst[:, bt.long().reshape(-1)] = blk.reshape(cfg.n_layers, cfg.B * nb, cfg.Hkv, ps, cfg.d)
+            del blk
+        ks, vs = list(pools_k.unbind(0)), list(pools_v.unbind(0))
+        del k_all, v_all
+        k_all = v_all = None
+        block_table = bt
     stoch = temperature > 0
     step = VerifyStep(qs, ks, vs, torch.full((cfg.B,), cfg.L, dtype=torch.int32, device=device), to(parent),
                       to(x["tokens"]), to(x["logits"]), to(x["draft_probs"]) if stoch else None,
                       to(x["uniforms"]) if stoch else None, temperature, cfg.max_depth,
-                      feat_in=W.make_features(cfg_gen).to(device), stacked=(q_all, k_all, v_all),
-                      max_cache_len=cfg.L if hint else 0)  # what a host that tracks its sequences' lengths knows
+                      feat_in=W.make_features(cfg_gen).to(device), stacked=None if paged else (q_all, k_all, v_all),
+                      max_cache_len=cfg.L if hint else 0,  # what a host that tracks its sequences' lengths knows
+                      block_table=block_table)
     return step
 
 
@@ -328,7 +351,8 @@ def measure(cfg, args, device, rank, world, with_e2e):
     from paper_2506_14158_b200 import replicas
 
     K, Wm = args.steps, max(3, args.warmup)
-    step = build_step(cfg, args.temperature, device, seed_shift=rank, hint=not args.no_hint)
+    step = build_step(cfg, args.temperature, device, seed_shift=rank, hint=not args.no_hint, paged=args.paged)
+    with_e2e = with_e2e and not args.paged
     g_step = step.capture("step")
     g_attn = step.capture("attention")
     g_acc = step.capture("accept")
@@ -446,12 +470,12 @@ def run_ours(args):
     cfg = get_config(args)
     rec = measure(cfg, args, device, rank, world, with_e2e=True)
     step, K, Wm = rec["step"], rec["K"], rec["Wm"]
-    h2d, d2h = step.h2d_bytes, step.d2h_bytes
+    h2d, d2h = getattr(step, "h2d_bytes", 0), getattr(step, "d2h_bytes", 0)
     launches = K * rec["n_blocks"] * step.launches_per_step(attn_kernels_per_layer(cfg))
     rec["step"] = None
     del step
     also = None
-    if cfg.name == "c2x32" and not args.no_also and not args.capacity:
+    if cfg.name == "c2x32" and not args.no_also and not args.capacity and not args.paged:
         # the 8B-shaped step, measured the same way in the same run (no host-buffer leg: 365 MB per step over PCIe)
         import gc
 
@@ -477,7 +501,8 @@ def run_ours(args):
                   l2="inputs larger than L2 (independent KV cache per layer)" if ab["attention"] > (126 << 20)
                   else "working set fits L2: launch-latency case, not a bandwidth claim",
                   launch="whole step replayed as one CUDA graph",
-                  max_cache_len_hint=0 if args.no_hint else cfg.L)
+                  max_cache_len_hint=0 if args.no_hint else cfg.L,
+                  cache_layout=f"paged, {args.paged} slots per page, pages scattered" if args.paged else "contiguous")
     line = dict(
         metric=METRIC, value=replicas.aggregate_nodes_per_second(cfg.B * cfg.T, world, ms), unit=UNIT, n_gpus=world,
         steps=K, warmup=Wm, ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -486,8 +511,8 @@ def run_ours(args):
                     ms_per_step_median=rec["ms_median"], ms_per_step_best=rec["ms_best"],
                     note="value and ms_per_step are the first block (exactly K steps); step_hbm and roofline use the medians"),
         step_hbm=step_hbm, roofline=roofline, breakdown_ms=breakdown,
-        e2e=dict(value=nodes / (rec["ms_e2e"] * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-                 ms_per_step=rec["ms_e2e"]),
+        e2e=(dict(value=nodes / (rec["ms_e2e"] * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                  ms_per_step=rec["ms_e2e"]) if rec["ms_e2e"] > 0 else None),
         gpu_launches=launches,
         accepted_per_step=dict(accept_len=accept_lens, mean_accepted_plus_bonus=sum(a + 1 for a in accept_lens) / len(accept_lens)),
         clocks=rec["clocks"],

@@ -61,6 +61,7 @@ typedef enum { S4C_F32 = 0, S4C_BF16 = 1 } s4c_dtype;
 #define S4C_SEQ_BAD_PATH 16   /* path not of the form 0 = path[0] < path[1] < ... < T */
 #define S4C_SEQ_TIMEOUT 32    /* a bounded in-kernel wait expired (OR-ed in; results of that sequence are invalid) */
 #define S4C_SEQ_NONFINITE 64  /* a target-logit row of a real node holds a NaN or +Inf, or nothing but -Inf */
+#define S4C_SEQ_BAD_PAGE 128  /* a block-table entry in use names a page outside the pool */
 
 typedef void* s4c_stream_t; /* a cudaStream_t */
 
@@ -214,6 +215,37 @@ s4c_status s4c_kv_compact(void* const* k_caches, void* const* v_caches, int n_la
                           const int32_t* path, const int32_t* accept_len, int max_depth,
                           const void* feat_in, void* feat_out, int B, int T, int Hkv, int d, int C, int hid,
                           s4c_dtype dt, int32_t* status, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * s4c_tree_attention_paged, s4c_kv_compact_paged -- the same two operations (Section 3.2: tree-masked
+ * attention of the verification pass; keeping the accepted tokens' K/V) on PAGED caches, the layout
+ * serving systems keep their caches in.  The paper does not discuss cache layouts.
+ *
+ * A cache is a pool of pages [n_pages, Hkv, page_size, d] (page_size a multiple of 64 slots; K and V
+ * pools of the same shape); block_table [B, max_blocks] int32 (device) names the page that holds
+ * slots i*page_size .. (i+1)*page_size-1 of sequence b.  Every block that holds a slot below
+ * cache_len[b] + T must be listed (the tree slots L_b..L_b+T-1 are ordinary slots of the sequence);
+ * other entries are never read.  A sequence can hold max_blocks*page_size slots (the capacity C of
+ * the contiguous calls).  A listed page outside [0, n_pages) flags the sequence S4C_SEQ_BAD_PAGE (its
+ * results are invalid; no access leaves the pool).  Results equal those of the contiguous calls on the
+ * cache the block table spells out.  s4c_tree_attention_paged serves S4C_BF16 (S4C_F32:
+ * S4C_ERR_UNSUPPORTED); its workspace is sized by s4c_tree_attention_workspace_bytes with
+ * C = max_blocks*page_size.  n_pages*Hkv*page_size must stay below 2^31.  All other arguments as in
+ * s4c_tree_attention / s4c_kv_compact (k_pages / v_pages of s4c_kv_compact_paged: device arrays of
+ * n_layers pool pointers; one block table serves all layers).
+ * ------------------------------------------------------------------------------------------ */
+s4c_status s4c_tree_attention_paged(const void* q, const void* k_pages, const void* v_pages,
+                                    const int32_t* block_table, const int32_t* cache_len, const int32_t* parent,
+                                    const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv, int d,
+                                    int n_pages, int page_size, int max_blocks, int max_cache_len, s4c_dtype dt,
+                                    float scale, int32_t* status, void* workspace, size_t workspace_bytes,
+                                    s4c_stream_t stream);
+
+s4c_status s4c_kv_compact_paged(void* const* k_pages, void* const* v_pages, int n_layers, const int32_t* block_table,
+                                int32_t* cache_len, const int32_t* path, const int32_t* accept_len, int max_depth,
+                                const void* feat_in, void* feat_out, int B, int T, int Hkv, int d, int n_pages,
+                                int page_size, int max_blocks, int hid, s4c_dtype dt, int32_t* status,
+                                s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
  * s4c_tree_build -- the continuous verification tree of Section 3.2 (drawn in Figure 3, left),

@@ -212,3 +212,26 @@ def build_tree(draft_probs, branching, root_token, cache_len=None):
     if rc:
         raise ValueError(f"oracle build_tree rejected its arguments (code {rc})")
     return dict(tokens=tokens, parent=parent, position=position, n_nodes=n_nodes)
+
+
+# ------------------------------------------------------------------ paged caches (a layout, not a step of the method)
+def pages_to_contiguous(pages, block_table):
+    """The contiguous cache [B,Hkv,max_blocks*page_size,d] that a pool of pages [n_pages,Hkv,page_size,d] spells out under
+    block_table [B,max_blocks] -- by definition of a paged cache: slot s of sequence b is slot s % page_size of page
+    block_table[b, s // page_size].  (Entries outside the pool read as page 0 here; callers only list blocks in use.)"""
+    pages = np.asarray(pages)
+    bt = np.asarray(block_table, dtype=np.int64)
+    n_pages, Hkv, ps, d = pages.shape
+    B, nb = bt.shape
+    safe = np.where((bt >= 0) & (bt < n_pages), bt, 0)
+    g = pages[safe]                                  # [B, nb, Hkv, ps, d]
+    return np.ascontiguousarray(g.transpose(0, 2, 1, 3, 4).reshape(B, Hkv, nb * ps, d))
+
+
+def scatter_to_pages(pages, block_table, contiguous, blocks_in_use):
+    """Writes the blocks in use (per sequence, a count) of a contiguous cache back into the pool, in place."""
+    n_pages, Hkv, ps, d = pages.shape
+    for b in range(contiguous.shape[0]):
+        for i in range(int(blocks_in_use[b])):
+            pages[int(block_table[b, i])] = contiguous[b, :, i * ps:(i + 1) * ps]
+    return pages

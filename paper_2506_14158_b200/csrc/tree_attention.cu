@@ -47,6 +47,33 @@ extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, con
                                status, workspace, stream);
 }
 
+// Paged caches: pages [n_pages, Hkv, page_size, d] addressed through a block table [B, max_blocks].
+extern "C" s4c_status s4c_tree_attention_paged(const void* q, const void* k_pages, const void* v_pages,
+                                               const int32_t* block_table, const int32_t* cache_len,
+                                               const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T,
+                                               int Hq, int Hkv, int d, int n_pages, int page_size, int max_blocks,
+                                               int max_cache_len, s4c_dtype dt, float scale, int32_t* status,
+                                               void* workspace, size_t workspace_bytes, s4c_stream_t stream_) {
+    using namespace s4c;
+    if (n_pages < 1 || max_blocks < 1 || page_size < 64 || page_size % 64 != 0) return S4C_ERR_SHAPE;
+    if ((long long)max_blocks * page_size > 0x7fffffffll || (long long)n_pages * Hkv * page_size > 0x7fffffffll) return S4C_ERR_SHAPE;
+    const int C = max_blocks * page_size;  // what a sequence can hold
+    const s4c_status st = check_shapes(B, T, Hq, Hkv, d, C, dt);
+    if (st != S4C_OK) return st;
+    if (!q || !k_pages || !v_pages || !block_table || !cache_len || !parent || !out) return S4C_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out)) return S4C_ERR_ALIGN;
+    if (!(scale >= 0.f) || isinf(scale) || max_cache_len < 0) return S4C_ERR_SHAPE;
+    if (dt != S4C_BF16) return S4C_ERR_UNSUPPORTED;  // paged caches are served by the tensor-core kernel only
+    if (B == 0) return S4C_OK;
+    if (scale == 0.f) scale = 1.f / sqrtf((float)d);
+    const size_t need = s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt);
+    if (need > 0 && (!workspace || workspace_bytes < need || !aligned256(workspace))) return S4C_ERR_WORKSPACE;
+    const int span = (max_cache_len > 0 && (long long)max_cache_len + T < (long long)C) ? max_cache_len + T : C;
+    const TcPaging paging = {block_table, max_blocks, page_size, n_pages};
+    return tree_attention_tc(q, k_pages, v_pages, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, span, scale, status,
+                             workspace, static_cast<cudaStream_t>(stream_), 0, -1, &paging);
+}
+
 // The bounded waits of the tensor-core kernel, exercised: the same launch as s4c_tree_attention, except that the copy
 // producer of every CTA never requests cache tile `withhold_tile` of its range and a wait gives up after `limit_us`
 // microseconds.  The consumers of that tile run out of time with nothing in flight, every role leaves its loop, and the

@@ -390,6 +390,9 @@ struct TcParams {
     float scale_log2;
     long long wait_limit;  // clock cycles a wait may take (kWaitLimitCycles; the self-test passes a short one)
     int withhold_tile;     // -1; the self-test names one tile of every CTA that the producer does not request
+    // paged caches (block_table == nullptr: one contiguous cache of C slots per sequence and KV head)
+    const int32_t* block_table;  // [B, max_blocks]: page of logical block i of sequence b
+    int max_blocks, page_tiles, n_pages;  // page_tiles = page size / 64 slots
 };
 
 // Tile range of a split: tiles are dealt out as evenly as whole tiles allow.
@@ -511,11 +514,24 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int q_row0 = (b * prm.Hq + hk * G) * T + mt0 * kBM;  // row of the [B*Hq*T, d] view of q
     const int kv_row0 = (b * prm.Hkv + hk) * prm.C;            // row of the [B*Hkv*C, d] view of the caches
     const uint32_t q_bytes = (uint32_t)prm.q_box_rows * 128u * NH;
+    // Paged caches [n_pages, Hkv, page, d]: tile g of the sequence lies in the page its block table names; a page holds
+    // whole tiles.  A page number outside the pool is flagged and replaced by page 0 (the copy stays inside the pool).
+    auto fetch_page = [&](int g) -> int { return __ldg(prm.block_table + (size_t)b * prm.max_blocks + g / prm.page_tiles); };
+    auto check_page = [&](int page) -> int {  // (apart from the fetch, so that the fetch's latency can pass behind other work)
+        if ((unsigned)page >= (unsigned)prm.n_pages) {
+            atomicOr(bad_s, S4C_SEQ_BAD_PAGE);
+            page = 0;
+        }
+        return page;
+    };
+    auto lookup_page = [&](int g) -> int { return check_page(fetch_page(g)); };
+    auto paged_row = [&](int g, int page) { return ((page * prm.Hkv + hk) * prm.page_tiles + g % prm.page_tiles) * kBN; };
+    const bool paged = prm.block_table != nullptr;
 
     if (warp == 0) {
         // ================= TMA producer =================
-        auto load_tile = [&](int j) -> bool {  // false: a wait was given up, nothing further is requested
-            const int s = j % S, it = j / S, row = kv_row0 + (t0 + j) * kBN;
+        auto load_tile = [&](int j, int row) -> bool {  // false: a wait was given up, nothing further is requested
+            const int s = j % S, it = j / S;
             if (j == prm.withhold_tile) return true;  // (self-test only: this tile never arrives)
             if (!mbar_wait(BAR(K_EMPTY + s), (it & 1) ^ 1, dead, limit)) return false;
             mbar_expect_tx(BAR(K_FULL + s), Cfg::kTileBytes);
@@ -552,7 +568,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (lane < 2 * S && (lane >> 1) < nt && (lane >> 1) != prm.withhold_tile) {
                 // K and V of a tile on neighbouring lanes: the requests go out as K0 V0 K1 V1 ..., so that the first
                 // product with V does not wait behind every K tile of the ring
-                const int j = lane >> 1, row = kv_row0 + (t0 + j) * kBN;
+                const int j = lane >> 1;
+                const int row = paged ? paged_row(t0 + j, lookup_page(t0 + j)) : kv_row0 + (t0 + j) * kBN;
                 const uint32_t full = BAR(((lane & 1) ? V_FULL : K_FULL) + j);
                 const uint32_t dst = ((lane & 1) ? sV : sK) + j * Cfg::kTileBytes;
                 const CUtensorMap* map = (lane & 1) ? &map_v : &map_k;
@@ -566,8 +583,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             __syncwarp();
             if (lane == 0) {
                 int issued = nt < S ? nt : S;
-                for (; issued < nt; ++issued)
-                    if (!load_tile(issued)) break;
+                // (paged: the page of the next tile is looked up before this tile's ring slot is waited for)
+                int page_next = (paged && issued < nt) ? fetch_page(t0 + issued) : 0, page_after = 0;
+                if (paged && issued + 1 < nt) page_after = fetch_page(t0 + issued + 1);
+                for (; issued < nt; ++issued) {  // table entries are fetched two tiles ahead and looked at when needed
+                    const int page = paged ? check_page(page_next) : 0;
+                    page_next = page_after;
+                    if (paged && issued + 2 < nt) page_after = fetch_page(t0 + issued + 2);
+                    if (!load_tile(issued, paged ? paged_row(t0 + issued, page) : kv_row0 + (t0 + issued) * kBN)) break;
+                }
                 *issued_s = issued;  // tiles requested: what a CTA that gives up has to see in before it leaves
             }
             __syncwarp();
@@ -1086,6 +1110,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     } else {
         __syncthreads();
     }
+    if (threadIdx.x == 0 && (*bad_s & S4C_SEQ_BAD_PAGE) && prm.status) atomicOr(prm.status + b, S4C_SEQ_BAD_PAGE);
     if (*dead) {  // read behind a CTA-wide barrier: the same in every thread
         // A wait was given up.  Before shared and tensor memory are handed back, everything this CTA set in motion is
         // seen to completion (bounded like every wait): a bulk copy that lands after the CTA has left would land in its
@@ -1277,9 +1302,11 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
         configured[dev] = true;
     }
     CUtensorMap mq, mk, mv;
+    // rows of the 2-D view of a cache: every slot of every (sequence, KV head), or of every (page, KV head)
+    const uint64_t kv_rows = prm.block_table ? (uint64_t)prm.n_pages * prm.Hkv * prm.page_tiles * kBN : (uint64_t)B * prm.Hkv * prm.C;
     if (!make_map(&mq, q, (uint64_t)B * prm.Hq * prm.T, D, prm.q_box_rows) ||
-        !(D == 128 ? make_map_halves(&mk, k, (uint64_t)B * prm.Hkv * prm.C, kBN) : make_map(&mk, k, (uint64_t)B * prm.Hkv * prm.C, D, kBN)) ||
-        !(D == 128 ? make_map_halves(&mv, v, (uint64_t)B * prm.Hkv * prm.C, kBN) : make_map(&mv, v, (uint64_t)B * prm.Hkv * prm.C, D, kBN)))
+        !(D == 128 ? make_map_halves(&mk, k, kv_rows, kBN) : make_map(&mk, k, kv_rows, D, kBN)) ||
+        !(D == 128 ? make_map_halves(&mv, v, kv_rows, kBN) : make_map(&mv, v, kv_rows, D, kBN)))
         return S4C_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(prm.splits, prm.m_groups * prm.Hkv, B);
@@ -1313,13 +1340,17 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
 s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
                              int d, int C_slots, int span, float scale, int32_t* status, void* ws, cudaStream_t stream,
-                             int wait_limit_us, int withhold_tile) {
+                             int wait_limit_us, int withhold_tile, const TcPaging* paging) {
     TcParams prm;
     prm.cache_len = cache_len, prm.parent = parent, prm.n_nodes = n_nodes;
     prm.out = static_cast<__nv_bfloat16*>(out), prm.ws = static_cast<float*>(ws), prm.status = status;
     prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C_slots;
     prm.wait_limit = wait_limit_us > 0 ? 2000ll * wait_limit_us : kWaitLimitCycles;  // about 2 cycles per nanosecond
     prm.withhold_tile = withhold_tile;
+    prm.block_table = paging ? paging->block_table : nullptr;
+    prm.max_blocks = paging ? paging->max_blocks : 0;
+    prm.page_tiles = paging ? paging->page_size / kBN : 1;
+    prm.n_pages = paging ? paging->n_pages : 0;
     const int C = span;  // every choice below is made for the live span
     const int nm = tc_nm(B, T, Hq, Hkv, C);
     prm.m_groups = tc_m_groups(B, T, Hq, Hkv, C);

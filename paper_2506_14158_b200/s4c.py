@@ -17,11 +17,13 @@ from ._build import lib_path
 
 F32, BF16 = 0, 1
 SEQ_OK, SEQ_BAD_PARENT, SEQ_TOKEN_RANGE, SEQ_CAPACITY, SEQ_DEPTH, SEQ_BAD_PATH, SEQ_TIMEOUT, SEQ_NONFINITE = 0, 1, 2, 4, 8, 16, 32, 64
+SEQ_BAD_PAGE = 128
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WORKSPACE", "ERR_UNSUPPORTED", "ERR_CUDA"]
 
 EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
-           "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build"]
+           "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
+           "s4c_tree_attention_paged", "s4c_kv_compact_paged"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -61,6 +63,10 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_build_workspace_bytes.argtypes = [i, i, i, i]
     lib.s4c_tree_build.restype = i
     lib.s4c_tree_build.argtypes = [vp, vp, i, i32p, i32p, i, i, i, i32p, i32p, i32p, i32p, vp, sz, vp]
+    lib.s4c_tree_attention_paged.restype = i
+    lib.s4c_tree_attention_paged.argtypes = [vp, vp, vp, i32p, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_kv_compact_paged.restype = i
+    lib.s4c_kv_compact_paged.argtypes = [vp, vp, i, i32p, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i, i, i32p, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -301,3 +307,50 @@ def tree_build(draft_probs, branching: Sequence[int], root_token, cache_len=None
     if rc:
         raise S4CError("s4c_tree_build", rc)
     return dict(tokens=tokens, parent=parent, position=position, n_nodes=n_nodes)
+
+
+def tree_attention_paged(q, k_pages, v_pages, block_table, cache_len, parent, n_nodes=None, out=None, scale: float = 0.0,
+                         status=None, workspace=None, stream=None, max_cache_len: int = 0):
+    """s4c_tree_attention_paged: q [B,Hq,T,d], k_pages / v_pages [n_pages,Hkv,page_size,d], block_table [B,max_blocks]."""
+    B, Hq, T, d = q.shape
+    n_pages, Hkv, page_size, _ = k_pages.shape
+    max_blocks = block_table.shape[1]
+    if v_pages.shape != k_pages.shape or k_pages.shape[3] != d or block_table.shape[0] != B:
+        raise ValueError("k_pages / v_pages must be [n_pages,Hkv,page_size,d] and block_table [B,max_blocks]")
+    if out is None:
+        out = torch.empty_like(q)
+    dt = _dt(q)
+    need = int(_lib.s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, max_blocks * page_size, dt))
+    if workspace is None:
+        workspace = _workspace(need, q.device, "attn")
+    rc = _lib.s4c_tree_attention_paged(
+        _dev(q, name="q"), _dev(k_pages, q.dtype, "k_pages"), _dev(v_pages, q.dtype, "v_pages"),
+        _dev(block_table, torch.int32, "block_table"), _dev(cache_len, torch.int32, "cache_len"),
+        _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"), _dev(out, q.dtype, "out"), B, T, Hq, Hkv, d,
+        n_pages, page_size, max_blocks, int(max_cache_len), dt, float(scale), _dev(status, torch.int32, "status"),
+        _dev(workspace, name="workspace"), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+        _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_attention_paged", rc)
+    return out
+
+
+def kv_compact_paged(k_ptrs, v_ptrs, n_layers: int, pool_shape, dtype, block_table, cache_len, path, accept_len, T: int,
+                     feat_in=None, feat_out=None, status=None, stream=None):
+    """s4c_kv_compact_paged.  pool_shape = (n_pages,Hkv,page_size,d); k_ptrs / v_ptrs from :func:`cache_pointer_array`."""
+    n_pages, Hkv, page_size, d = pool_shape
+    B, max_blocks = block_table.shape
+    max_depth = path.shape[1] - 1
+    dt = F32 if dtype == torch.float32 else BF16
+    if status is None:
+        status = torch.empty(B, dtype=torch.int32, device=cache_len.device)
+    hid = 0 if feat_in is None else feat_in.shape[2]
+    rc = _lib.s4c_kv_compact_paged(
+        _dev(k_ptrs, torch.int64, "k_ptrs") if n_layers else None, _dev(v_ptrs, torch.int64, "v_ptrs") if n_layers else None,
+        int(n_layers), _dev(block_table, torch.int32, "block_table"), _dev(cache_len, torch.int32, "cache_len"),
+        _dev(path, torch.int32, "path"), _dev(accept_len, torch.int32, "accept_len"), max_depth, _dev(feat_in, name="feat_in"),
+        _dev(feat_out, name="feat_out"), B, T, Hkv, d, n_pages, page_size, max_blocks, hid, dt,
+        _dev(status, torch.int32, "status"), _stream(stream))
+    if rc:
+        raise S4CError("s4c_kv_compact_paged", rc)
+    return status

@@ -23,8 +23,10 @@ class VerifyStep:
                  draft_probs: Optional[torch.Tensor], uniforms: Optional[torch.Tensor], temperature: float,
                  max_depth: int, n_nodes: Optional[torch.Tensor] = None, feat_in: Optional[torch.Tensor] = None,
                  stacked: Optional[tuple] = None, max_cache_len: int = 0, branching: Optional[tuple] = None,
-                 root_token: Optional[torch.Tensor] = None):
-        """``branching`` (+ ``root_token`` [B] int32): the step then starts with s4c_tree_build, which writes the tree
+                 root_token: Optional[torch.Tensor] = None, block_table: Optional[torch.Tensor] = None):
+        """``block_table`` [B,max_blocks] int32: the caches are paged -- every ``k_caches[l]`` / ``v_caches[l]`` is a pool
+        [n_pages,Hkv,page_size,d] and the step calls s4c_tree_attention_paged / s4c_kv_compact_paged.
+        ``branching`` (+ ``root_token`` [B] int32): the step then starts with s4c_tree_build, which writes the tree
         (``tokens``, ``parent``, ``n_nodes``, position ids) from ``draft_probs`` on the device -- no host tree in the loop;
         ``parent`` and ``tokens`` are then only buffers of the right shape.
         ``max_cache_len``: what the host knows about the committed lengths (an upper bound, 0 = nothing); it is handed
@@ -46,6 +48,7 @@ class VerifyStep:
         B, T, V = target_logits.shape
         self.B, self.T, self.V = B, T, V
         self.cache_shape = tuple(k_caches[0].shape)
+        self.block_table = block_table
         self.dtype = k_caches[0].dtype
         i32 = dict(dtype=torch.int32, device=dev)
         self.cache_len = cache_len.clone()            # working copy: the step advances it in place
@@ -61,6 +64,8 @@ class VerifyStep:
                                                                  dtype=feat_in.dtype, device=dev)
         _, Hq, _, d = q[0].shape
         _, Hkv, C, _ = self.cache_shape
+        if block_table is not None:  # a sequence can hold max_blocks pages
+            C = block_table.shape[1] * self.cache_shape[2]
         self.ws_attn = torch.empty(max(1, s4c.tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, self.dtype)),
                                    dtype=torch.uint8, device=dev)
         self.ws_accept = torch.empty(max(1, s4c.tree_accept_workspace_bytes(B, T, V)), dtype=torch.uint8, device=dev)
@@ -91,6 +96,11 @@ class VerifyStep:
 
     def attention(self, l0: int = 0, l1: Optional[int] = None):
         for l in range(l0, self.n_layers if l1 is None else l1):
+            if self.block_table is not None:
+                s4c.tree_attention_paged(self.q[l], self.k_caches[l], self.v_caches[l], self.block_table, self.cache_len,
+                                         self.parent, self.n_nodes, out=self.attn_out[l], status=self.status_attn,
+                                         workspace=self.ws_attn, max_cache_len=self.max_cache_len)
+                continue
             s4c.tree_attention(self.q[l], self.k_caches[l], self.v_caches[l], self.cache_len, self.parent, self.n_nodes,
                                out=self.attn_out[l], status=self.status_attn, workspace=self.ws_attn,
                                max_cache_len=self.max_cache_len)
@@ -101,6 +111,11 @@ class VerifyStep:
                         self.status_accept, self.ws_accept)
 
     def compact(self):
+        if self.block_table is not None:
+            s4c.kv_compact_paged(self.k_ptrs, self.v_ptrs, self.n_layers, self.cache_shape, self.dtype, self.block_table,
+                                 self.cache_len, self.path, self.accept_len, self.T, self.feat_in, self.feat_out,
+                                 self.status_compact)
+            return
         s4c.kv_compact(self.k_ptrs, self.v_ptrs, self.n_layers, self.cache_shape, self.dtype, self.cache_len, self.path,
                        self.accept_len, self.T, self.feat_in, self.feat_out, self.status_compact)
 

@@ -35,10 +35,10 @@ def test_sequence_flags_agree_between_header_binding_and_oracle(s4c_lib):
     text = open(os.path.join(ROOT, "include", "s4c.h")).read()
     flags = {k: int(v) for k, v in re.findall(r"#define\s+S4C_(SEQ_[A-Z_]+)\s+(\d+)", text)}
     assert flags == {"SEQ_OK": 0, "SEQ_BAD_PARENT": 1, "SEQ_TOKEN_RANGE": 2, "SEQ_CAPACITY": 4, "SEQ_DEPTH": 8,
-                     "SEQ_BAD_PATH": 16, "SEQ_TIMEOUT": 32, "SEQ_NONFINITE": 64}
+                     "SEQ_BAD_PATH": 16, "SEQ_TIMEOUT": 32, "SEQ_NONFINITE": 64, "SEQ_BAD_PAGE": 128}
     for k, v in flags.items():
         assert getattr(s4c, k) == v
-        if k != "SEQ_TIMEOUT":  # the CPU oracle has no waits
+        if k not in ("SEQ_TIMEOUT", "SEQ_BAD_PAGE"):  # the CPU oracle has no waits and no page tables
             assert getattr(oracle, k) == v
 
 
