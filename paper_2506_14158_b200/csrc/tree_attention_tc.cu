@@ -395,11 +395,13 @@ struct TcParams {
     int max_blocks, page_tiles, n_pages;  // page_tiles = page size / 64 slots
 };
 
-// Tile range of a split: tiles are dealt out as evenly as whole tiles allow.
+// Tile range of a split: tiles are dealt out as evenly as whole tiles allow, the odd ones to the FIRST splits -- the last
+// split holds the tree's own tiles, which cost more than a tile of the prefix (they are masked), and every split of a
+// cluster waits for the slowest.
 __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, int& t0, int& t1) {
     // (at most 2^25 tiles and 64 splits: the products fit 32 bits, and a 32-bit division is a fraction of a 64-bit one)
-    t0 = (int)(((uint32_t)n_tiles * (uint32_t)split) / (uint32_t)splits);
-    t1 = (int)(((uint32_t)n_tiles * (uint32_t)(split + 1)) / (uint32_t)splits);
+    t0 = (int)(((uint32_t)n_tiles * (uint32_t)split + (uint32_t)splits - 1u) / (uint32_t)splits);
+    t1 = (int)(((uint32_t)n_tiles * (uint32_t)(split + 1) + (uint32_t)splits - 1u) / (uint32_t)splits);
 }
 
 // REP > 1 (one row tile, G*T <= 128 / REP rows): the query rows are laid into the 128 MMA rows REP times
