@@ -10,6 +10,7 @@ Functions (array layouts are row-major numpy arrays):
 * :func:`tree_attention`      -- Section 3.2 / Figure 3 tree mask: masked softmax attention by definition.
 * :func:`accept_greedy`       -- Section 4.1.2 greedy decoding + Section 3.2 longest accepted path.
 * :func:`accept_stochastic`   -- Section 2 speculative sampling, Eq. 11 / Eq. 12, step by step.
+* :func:`accept_filtered`     -- the same against a top-k / nucleus filtered target (sampling regime of Section 4, RQ5).
 * :func:`kv_compact`          -- Section 3.2 last paragraph: keep accepted tokens' K/V and features.
 * :func:`build_tree`          -- Section 3.2 / Figure 3: the continuous verification tree (vertical top-1 chain, then
                                  horizontal top-k alternatives), breadth-first numbered.
@@ -149,6 +150,30 @@ def accept_stochastic(logits, draft_probs, tokens, parent, temperature, uniforms
         _ptr(tie, ctypes.c_uint8), _ptr(status, i32))
     if rc:
         raise ValueError(f"oracle accept_stochastic rejected its arguments (code {rc})")
+    return dict(accept_len=a, path=path, next_token=nxt, near_tie=tie, status=status)
+
+
+def accept_filtered(logits, draft_probs, tokens, parent, temperature, top_k, top_p, uniforms, n_nodes=None,
+                    max_depth=None):
+    """Speculative sampling against the top-k / nucleus filtered target distribution (steps F1-F3 of the C source)."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    draft_probs = np.ascontiguousarray(draft_probs, dtype=np.float32)
+    B, T, V = logits.shape
+    tokens = _i32(tokens).reshape(B, T)
+    parent = _i32(parent).reshape(B, T)
+    uniforms = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, T)
+    n_nodes = _i32(n_nodes)
+    if max_depth is None:
+        max_depth = T - 1
+    a, path, nxt, status = _accept_outputs(B, max_depth)
+    tie = np.zeros((B, T), dtype=np.uint8)
+    f32, i32 = ctypes.c_float, ctypes.c_int32
+    rc = _load().s4c_oracle_accept_filtered(
+        _ptr(logits, f32), _ptr(draft_probs, f32), _ptr(tokens, i32), _ptr(parent, i32), _ptr(n_nodes, i32),
+        ctypes.c_double(float(temperature)), int(top_k), ctypes.c_double(float(top_p)), _ptr(uniforms, f32),
+        B, T, V, max_depth, _ptr(a, i32), _ptr(path, i32), _ptr(nxt, i32), _ptr(tie, ctypes.c_uint8), _ptr(status, i32))
+    if rc:
+        raise ValueError(f"oracle accept_filtered rejected its arguments (code {rc})")
     return dict(accept_len=a, path=path, next_token=nxt, near_tie=tie, status=status)
 
 

@@ -23,6 +23,10 @@
  *                              norm(max(0, p - q))), Eq. 11 and Eq. 12 of
  *                              Section 3.2 (the correction at fork positions).
  *                              Taken step by step, in the paper's order.
+ *   s4c_oracle_accept_filtered the same walk against a top-k / nucleus filtered
+ *                              target distribution (the sampling regime of the
+ *                              temperature study, Section 4; the filter itself
+ *                              is this build's statement of the usual samplers).
  *   s4c_oracle_kv_compact      Section 3.2, last paragraph (accepted tokens and
  *                              their features are kept for the next drafting
  *                              phase): a gather from a snapshot.
@@ -304,15 +308,30 @@ int s4c_oracle_accept_greedy(const float* logits, const int32_t* tokens, const i
 /*      exceeds u_0 * sum(p).                                                 */
 /* near_tie[b,i] = 1 where |ratio - u_i| < 1e-6 at node i's test.             */
 /* ------------------------------------------------------------------------- */
-int s4c_oracle_accept_stochastic(const float* logits, const float* dprobs, const int32_t* tokens,
-                                 const int32_t* parent, const int32_t* n_nodes, double tau,
-                                 const float* uniforms, int B, int T, int V, int max_depth,
-                                 int32_t* accept_len, int32_t* path, int32_t* next_token,
-                                 uint8_t* near_tie, int32_t* status) {
+/*                                                                           */
+/* Filtered variant (top_k > 0): the sampling regime of the temperature study */
+/* (Section 4, RQ5) as samplers usually run it.  Between S1 and S2 the target */
+/* distribution is replaced, as by a chain of logit warpers (temperature,     */
+/* then top-k, then nucleus):                                                 */
+/*  F1  rank the tokens by target logit, higher first, equal logits by lower  */
+/*      token index; keep the first top_k;                                     */
+/*  F2  renormalise p over the kept tokens;                                    */
+/*  F3  if top_p < 1: keep the shortest prefix, in rank order, whose          */
+/*      cumulative (renormalised) probability reaches top_p; renormalise.      */
+/* Every other token gets p = 0.  top_k = 0 leaves p as it is (top_p unused). */
+/* The paper does not define filtering; F1-F3 are this build's statement of   */
+/* the usual top-k / nucleus samplers, and the accept / resample steps then    */
+/* preserve the FILTERED target distribution.                                  */
+static int accept_sampling(const float* logits, const float* dprobs, const int32_t* tokens,
+                           const int32_t* parent, const int32_t* n_nodes, double tau, int top_k, double top_p,
+                           const float* uniforms, int B, int T, int V, int max_depth,
+                           int32_t* accept_len, int32_t* path, int32_t* next_token,
+                           uint8_t* near_tie, int32_t* status) {
     if (!logits || !dprobs || !tokens || !parent || !uniforms || !accept_len || !path ||
         !next_token)
         return 1;
     if (B < 0 || T < 1 || V < 1 || max_depth < 0 || !(tau > 0.0)) return 2;
+    if (top_k < 0 || (top_k > 0 && !(top_p > 0.0 && top_p <= 1.0))) return 2;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic)
 #endif
@@ -353,6 +372,40 @@ int s4c_oracle_accept_stochastic(const float* logits, const float* dprobs, const
             for (int v = 0; v < V; ++v) {
                 p[v] /= den;
                 q[v] = (double)dq[v];
+            }
+            if (top_k > 0) {
+                /* F1: selection by repeated maximum over the tokens not taken yet */
+                const int k = top_k < V ? top_k : V;
+                int* ord = (int*)malloc(sizeof(int) * (size_t)k);
+                unsigned char* taken = (unsigned char*)calloc((size_t)V, 1);
+                for (int j = 0; j < k; ++j) {
+                    int best = -1;
+                    for (int v = 0; v < V; ++v)
+                        if (!taken[v] && (best < 0 || x[v] > x[best])) best = v;
+                    taken[best] = 1;
+                    ord[j] = best;
+                }
+                /* F2 */
+                double kept_mass = 0.0;
+                for (int j = 0; j < k; ++j) kept_mass += p[ord[j]];
+                int m = k;
+                if (top_p < 1.0) { /* F3 */
+                    double cum = 0.0;
+                    for (int j = 0; j < k; ++j) {
+                        cum += p[ord[j]] / kept_mass;
+                        if (cum >= top_p) {
+                            m = j + 1;
+                            break;
+                        }
+                    }
+                    kept_mass = 0.0;
+                    for (int j = 0; j < m; ++j) kept_mass += p[ord[j]];
+                }
+                double* keep = (double*)malloc(sizeof(double) * (size_t)m);
+                for (int j = 0; j < m; ++j) keep[j] = p[ord[j]] / kept_mass;
+                for (int v = 0; v < V; ++v) p[v] = 0.0;
+                for (int j = 0; j < m; ++j) p[ord[j]] = keep[j];
+                free(keep), free(taken), free(ord);
             }
             /* S2 / S3 */
             int accepted = -1;
@@ -414,6 +467,25 @@ int s4c_oracle_accept_stochastic(const float* logits, const float* dprobs, const
         free(depth);
     }
     return 0;
+}
+
+int s4c_oracle_accept_stochastic(const float* logits, const float* dprobs, const int32_t* tokens,
+                                 const int32_t* parent, const int32_t* n_nodes, double tau,
+                                 const float* uniforms, int B, int T, int V, int max_depth,
+                                 int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                 uint8_t* near_tie, int32_t* status) {
+    return accept_sampling(logits, dprobs, tokens, parent, n_nodes, tau, 0, 1.0, uniforms, B, T, V, max_depth,
+                           accept_len, path, next_token, near_tie, status);
+}
+
+int s4c_oracle_accept_filtered(const float* logits, const float* dprobs, const int32_t* tokens,
+                               const int32_t* parent, const int32_t* n_nodes, double tau, int top_k, double top_p,
+                               const float* uniforms, int B, int T, int V, int max_depth,
+                               int32_t* accept_len, int32_t* path, int32_t* next_token,
+                               uint8_t* near_tie, int32_t* status) {
+    if (top_k < 1) return 2;
+    return accept_sampling(logits, dprobs, tokens, parent, n_nodes, tau, top_k, top_p, uniforms, B, T, V, max_depth,
+                           accept_len, path, next_token, near_tie, status);
 }
 
 /* ------------------------------------------------------------------------- */
