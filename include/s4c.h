@@ -217,6 +217,32 @@ s4c_status s4c_kv_compact(void* const* k_caches, void* const* v_caches, int n_la
                           s4c_dtype dt, int32_t* status, s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * s4c_tree_accept_filtered -- s4c_tree_accept's speculative-sampling walk (Section 2; Eq. 11, Eq. 12;
+ * longest accepted path, Section 3.2) against a FILTERED target distribution: the sampling regime of
+ * the temperature study (Section 4, RQ5) as samplers usually run it.  The paper does not define a
+ * filter; this one is the usual chain of logit warpers:
+ *   temperature, then top-k, then nucleus.  At every node the tokens are ranked by target logit
+ *   (higher first, equal logits by lower token); the first top_k are kept and p = softmax(logit /
+ *   temperature) is renormalised over them; if top_p < 1 the shortest prefix in rank order whose
+ *   cumulative (renormalised) probability reaches top_p is kept and renormalised again.  Every
+ *   other token has target probability 0: it is never accepted and never emitted.
+ * The accept / reject / resample rules, uniforms, outputs, status flags and the NONFINITE rule are
+ * those of s4c_tree_accept with this p; the draft distribution is taken as given (a drafter that was
+ * filtered the same way passes its filtered probabilities).  top_k = 1 is greedy verification.
+ *   temperature > 0;  1 <= top_k <= 64 (values above V act as V);  0 < top_p <= 1.
+ *   workspace: at least s4c_tree_accept_filtered_workspace_bytes(B, T, V, top_k) bytes, 256-byte aligned.
+ * Cost: every logits row is read once and no exponential is taken over the vocabulary (the kept
+ * tokens are found by selection); draft rows are read only where a sibling is rejected.
+ * ------------------------------------------------------------------------------------------ */
+size_t s4c_tree_accept_filtered_workspace_bytes(int B, int T, int V, int top_k);
+
+s4c_status s4c_tree_accept_filtered(const float* target_logits, const float* draft_probs, const int32_t* tokens,
+                                    const int32_t* parent, const int32_t* n_nodes, float temperature, int top_k,
+                                    float top_p, const float* uniforms, int B, int T, int V, int max_depth,
+                                    int32_t* accept_len, int32_t* path, int32_t* next_token, uint8_t* near_tie,
+                                    int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * s4c_tree_attention_paged, s4c_kv_compact_paged -- the same two operations (Section 3.2: tree-masked
  * attention of the verification pass; keeping the accepted tokens' K/V) on PAGED caches, the layout
  * serving systems keep their caches in.  The paper does not discuss cache layouts.

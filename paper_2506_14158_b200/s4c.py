@@ -23,7 +23,8 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
 EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
-           "s4c_tree_attention_paged", "s4c_kv_compact_paged"]
+           "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
+           "s4c_tree_accept_filtered"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -67,6 +68,10 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_attention_paged.argtypes = [vp, vp, vp, i32p, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
     lib.s4c_kv_compact_paged.restype = i
     lib.s4c_kv_compact_paged.argtypes = [vp, vp, i, i32p, i32p, i32p, i32p, i, vp, vp, i, i, i, i, i, i, i, i, i, i32p, vp]
+    lib.s4c_tree_accept_filtered_workspace_bytes.restype = sz
+    lib.s4c_tree_accept_filtered_workspace_bytes.argtypes = [i, i, i, i]
+    lib.s4c_tree_accept_filtered.restype = i
+    lib.s4c_tree_accept_filtered.argtypes = [vp, vp, i32p, i32p, i32p, f, i, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp, sz, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -354,3 +359,37 @@ def kv_compact_paged(k_ptrs, v_ptrs, n_layers: int, pool_shape, dtype, block_tab
     if rc:
         raise S4CError("s4c_kv_compact_paged", rc)
     return status
+
+
+def tree_accept_filtered_workspace_bytes(B, T, V, top_k) -> int:
+    return int(_lib.s4c_tree_accept_filtered_workspace_bytes(B, T, V, top_k))
+
+
+def tree_accept_filtered(target_logits, draft_probs, tokens, parent, temperature: float, top_k: int, top_p: float, uniforms,
+                         n_nodes=None, max_depth: Optional[int] = None, accept_len=None, path=None, next_token=None,
+                         near_tie=None, status=None, workspace=None, stream=None):
+    """s4c_tree_accept_filtered: the walk of :func:`tree_accept` against the top-k / nucleus filtered target distribution."""
+    B, T, V = target_logits.shape
+    dev = target_logits.device
+    if max_depth is None:
+        max_depth = T - 1
+    i32 = dict(dtype=torch.int32, device=dev)
+    accept_len = torch.empty(B, **i32) if accept_len is None else accept_len
+    path = torch.empty(B, max_depth + 1, **i32) if path is None else path
+    next_token = torch.empty(B, **i32) if next_token is None else next_token
+    near_tie = torch.empty(B, T, dtype=torch.uint8, device=dev) if near_tie is None else near_tie
+    status = torch.empty(B, **i32) if status is None else status
+    need = int(_lib.s4c_tree_accept_filtered_workspace_bytes(B, T, V, int(top_k)))
+    if workspace is None:
+        workspace = _workspace(need, dev, "accept_filtered")
+    rc = _lib.s4c_tree_accept_filtered(
+        _dev(target_logits, torch.float32, "target_logits"), _dev(draft_probs, torch.float32, "draft_probs"),
+        _dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"),
+        float(temperature), int(top_k), float(top_p), _dev(uniforms, torch.float32, "uniforms"), B, T, V, int(max_depth),
+        _dev(accept_len, torch.int32, "accept_len"), _dev(path, torch.int32, "path"),
+        _dev(next_token, torch.int32, "next_token"), _dev(near_tie, torch.uint8, "near_tie"),
+        _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+        0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_accept_filtered", rc)
+    return dict(accept_len=accept_len, path=path, next_token=next_token, near_tie=near_tie, status=status)

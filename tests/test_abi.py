@@ -111,4 +111,22 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert tb(br=ctypes.cast(bad, vp), D=2) == 2                # more than 16 children
     assert lib.s4c_tree_build_workspace_bytes(1, 26, 32000, 4) % 256 == 0 and lib.s4c_tree_build_workspace_bytes(1, 26, 32000, 4) > 0
     assert lib.s4c_tree_build_workspace_bytes(1, 26, 32000, 17) == 0
+    lib.s4c_tree_accept_filtered.argtypes = [vp, vp, vp, vp, vp, f, i, f, vp, i, i, i, i, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.s4c_tree_accept_filtered_workspace_bytes.restype = sz
+    lib.s4c_tree_accept_filtered_workspace_bytes.argtypes = [i, i, i, i]
+    fl = lambda **kw: lib.s4c_tree_accept_filtered(*[kw.get(k, d) for k, d in [
+        ("lg", P), ("dp", P), ("tok", P), ("par", P), ("nn", None), ("tau", 1.0), ("k", 50), ("p", 0.9), ("u", P), ("B", 1),
+        ("T", 8), ("V", 100), ("md", 7), ("al", P), ("path", P), ("nt", P), ("tie", None), ("st", None), ("ws", None),
+        ("wsb", 0), ("s", None)]])
+    assert fl(lg=None) == 1 and fl(dp=None) == 1 and fl(u=None) == 1 and fl(nt=None) == 1
+    assert fl(tau=0.0) == 2 and fl(tau=float("inf")) == 2 and fl(tau=float("nan")) == 2   # greedy goes through s4c_tree_accept
+    assert fl(k=0) == 2 and fl(k=65) == 2 and fl(p=0.0) == 2 and fl(p=1.5) == 2 and fl(p=float("nan")) == 2
+    assert fl(T=129) == 2 and fl(V=0) == 2 and fl(md=128) == 2
+    assert fl(lg=P + 4) == 4
+    assert fl() == 5                                            # no workspace
+    assert fl(B=0) == 0
+    wsb = lib.s4c_tree_accept_filtered_workspace_bytes
+    assert wsb(1, 8, 32000, 50) % 256 == 0 and wsb(1, 8, 32000, 50) > 0
+    assert wsb(1, 8, 32000, 65) == 0 and wsb(1, 8, 32000, 0) == 0
+    assert wsb(1, 8, 10, 50) == wsb(1, 8, 10, 10)               # top_k is capped by the vocabulary
     assert b"workspace" in lib.s4c_status_string(5)
