@@ -386,6 +386,13 @@ def measure(cfg, args, device, rank, world, with_e2e):
         step.enable_tree_build(cfg.branching, step.tokens[:, 0].contiguous())
         g_tree = step.capture("tree")
         ms_tree = time_graph(g_tree, K, torch)
+    # the same acceptance against a top-k / nucleus filtered target (not part of the timed step either)
+    ms_filt = None
+    if args.temperature > 0:
+        step.set_filter(FILTER_TOP_K, FILTER_TOP_P)
+        ms_filt = time_graph(step.capture("accept"), K, torch)
+        step.set_filter(None)
+        g_acc.replay()  # the step's own decision is back in the output buffers
     ms_e2e = 0.0
     if with_e2e:
         # end to end: per-step inputs from pinned host memory, decision back to the host, every step
@@ -406,11 +413,12 @@ def measure(cfg, args, device, rank, world, with_e2e):
         [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
         device=device)
     rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
-               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, ms_e2e=ms_e2e, accept_lens=accept_lens,
                clocks=clocks, K=K, Wm=Wm)
     return rec
 
 
+FILTER_TOP_K, FILTER_TOP_P = 50, 0.9  # the filter the extra acceptance timing uses
 TARGET_FRAC = 0.70  # of HBM peak, for the whole step on the 7B- and 8B-shaped configurations
 
 
@@ -443,6 +451,8 @@ def roofline_records(cfg, args, rec, pk):
     breakdown = dict(attention_all_layers=rec["ms_attn"], accept=rec["ms_acc"], compact=rec["ms_cmp"])
     if rec.get("ms_tree") is not None:
         breakdown["tree_build_not_in_step"] = rec["ms_tree"]
+    if rec.get("ms_filt") is not None:
+        breakdown[f"accept_filtered_top{FILTER_TOP_K}_p{FILTER_TOP_P}_not_in_step"] = rec["ms_filt"]
     return ab, step_hbm, roofline, breakdown
 
 

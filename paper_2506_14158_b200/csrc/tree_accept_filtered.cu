@@ -2,19 +2,27 @@
 // Section 3.2) against a top-k / nucleus FILTERED target distribution -- the sampling regime of Section 4 (RQ5).
 //
 // Filtering makes the target distribution sparse: at most top_k (<= 64) tokens per node keep any mass.  So the only
-// vocabulary-wide work is finding those tokens, a selection over the logits that needs no exponential at all:
-//   filter_segments_kernel  grid (vocabulary segments of 4096, T, B): every thread sorts its 16 logits (with their token
-//                           indices, order: logit descending, token ascending), every warp merges its lanes' sorted lists
-//                           head by head into its k best, one warp merges the eight warp lists into the segment's k best
-//   filter_rows_kernel      grid (T, B), one warp: merges the segments' lists into the row's k best, turns them into
-//                           probabilities in float64 (softmax over the kept logits at the temperature), cuts the nucleus
-//                           and renormalises: per node a short list (token, probability) in rank order
-//   accept_walk_sparse_kernel  grid (B): the walk of s4c_tree_accept on these lists.  Residual masses and the final
-//                           inverse-CDF draw run over the <= 64 kept tokens of a node; only the renormalisation of the
-//                           draft distribution after a rejection needs its sum over the vocabulary, one CTA-wide pass
-//                           over the draft row of that node.
-// HBM traffic: every logits row once (the draft rows only where a rejection happens).  Ranking, sums and decisions are
-// deterministic (fixed orders); ties between equal logits go to the lower token.
+// vocabulary-wide work is finding those tokens -- a selection over the logits that needs no exponential -- and the mass
+// of every draft row (the renormalisation after a rejection needs it):
+//   filter_segments_kernel  grid (vocabulary segments of 4096, T, B), one pass over logits and draft probabilities:
+//                           the segment's k best logits by THRESHOLD SELECTION.  The k-th best of the segment is at
+//                           least the smallest of the 256 threads' maxima, so only entries at or above that value
+//                           matter (about a third of them); these are counted in a 256-bin histogram over
+//                           [that value, the segment's maximum], the bin where the count from the top reaches k is
+//                           found, the entries of the bins down to it (k plus a few) are gathered and ranked exactly
+//                           (logit descending, token ascending) by counting.  Segments that this cannot serve (more
+//                           than 256 entries in those bins: heavy ties; fewer than k threads with a finite logit) take
+//                           a slower exact path: every thread sorts its 16 entries, warps merge their lanes' lists head
+//                           by head, one warp merges the warps' lists.  Also the segment's draft mass in float64.
+//   filter_rows_kernel      grid (T, B): merges the segments' sorted lists pairwise (a bitonic merge of two lists in a
+//                           warp's registers, a tree of such merges over the lists) into the row's k best, turns them
+//                           into probabilities in float64 (softmax over the kept logits at the temperature), cuts the
+//                           nucleus and renormalises: per node a short list (token, probability, draft probability) in
+//                           rank order, and the draft row's mass
+//   accept_walk_sparse_kernel  grid (B): the walk of s4c_tree_accept on these lists, by one warp: acceptance tests,
+//                           residual masses and the final inverse-CDF draw run over the <= 64 kept tokens of a node.
+// HBM traffic: every logits row and every draft row once.  Ranking, sums and decisions are deterministic (fixed orders);
+// ties between equal logits go to the lower token.
 #include <float.h>
 #include <limits.h>
 #include <math.h>
@@ -74,42 +82,183 @@ __device__ __forceinline__ float fmax_keep_nan(float a, float b) {
     return d;
 }
 
+// order-preserving map of a float onto unsigned integers (a > b  <=>  key(a) > key(b); -0 ranks just below +0, which
+// only shifts a threshold by nothing that can be told apart: thresholds are compared as floats again)
+__device__ __forceinline__ uint32_t f_key(float x) {
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float f_unkey(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+constexpr uint32_t kKeyPosInf = 0xff800000u;  // f_key(+inf)
+constexpr uint32_t kKeyNegInf = 0x007fffffu;  // f_key(-inf)
+
+constexpr int kFsBins = 256;   // histogram bins of the threshold selection
+constexpr int kFsCap = 256;    // most candidates ranked by counting (one per thread)
+
+struct SegShared {
+    union {
+        struct {
+            FCand lists[kFsElems][kFsThreads];       // slow path: entry h of thread t at [h][t]
+            FCand wlist[kFsThreads / 32][kMaxTopK];  // slow path: the warps' k best
+        } slow;
+        struct {
+            int hist[kFsBins];
+            FCand cand[kFsCap];
+        } fast;
+    };
+    uint32_t wmax[kFsThreads / 32], wmin[kFsThreads / 32];
+    int wfin[kFsThreads / 32];
+    double wq[kFsThreads / 32];
+    int ncand;
+};
+
 template <bool VEC>
 __global__ void __launch_bounds__(kFsThreads)
-filter_segments_kernel(const float* __restrict__ logits, const int32_t* __restrict__ n_nodes, int T, int V, int k,
-                       FCand* __restrict__ cand) {
+filter_segments_kernel(const float* __restrict__ logits, const float* __restrict__ dprobs, const int32_t* __restrict__ n_nodes,
+                       int T, int V, int k, FCand* __restrict__ cand, double* __restrict__ qpart) {
     const int seg = blockIdx.x, node = blockIdx.y, b = blockIdx.z;
     if (n_nodes && node >= n_nodes[b]) return;
-    const float* row = logits + ((size_t)b * T + node) * V;
-    const int s0 = seg * kFsSeg, tid = threadIdx.x, warp = tid >> 5;
+    __shared__ SegShared sh;
+    const size_t at = (size_t)b * T + node;
+    const float* row = logits + at * V;
+    const float* qrow = dprobs + at * V;
+    const int s0 = seg * kFsSeg, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // entry i of this thread is token tok_of(i); the same map on every path
+    auto tok_of = [&](int i) { return VEC ? s0 + ((i >> 2) * kFsThreads + tid) * 4 + (i & 3) : s0 + i * kFsThreads + tid; };
     float x[kFsElems];
-    int e[kFsElems];
-#pragma unroll
-    for (int i = 0; i < kFsElems; ++i) e[i] = VEC ? s0 + ((i >> 2) * kFsThreads + tid) * 4 + (i & 3) : s0 + i * kFsThreads + tid;
-    if (VEC) {
+    double qs = 0.0;
+    if (VEC) {  // V % 4 == 0: whole 16-byte words, all requested before any is used
+        float4 lv[kFsElems / 4], qv[kFsElems / 4];
 #pragma unroll
         for (int i = 0; i < kFsElems / 4; ++i) {
-            float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-            if (e[4 * i] < V) v = __ldg(reinterpret_cast<const float4*>(row + e[4 * i]));  // V % 4 == 0 here
-            x[4 * i + 0] = v.x, x[4 * i + 1] = v.y, x[4 * i + 2] = v.z, x[4 * i + 3] = v.w;
+            lv[i] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY), qv[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (tok_of(4 * i) < V) {
+                lv[i] = __ldg(reinterpret_cast<const float4*>(row + tok_of(4 * i)));
+                qv[i] = __ldg(reinterpret_cast<const float4*>(qrow + tok_of(4 * i)));
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kFsElems / 4; ++i) {
+            x[4 * i + 0] = lv[i].x, x[4 * i + 1] = lv[i].y, x[4 * i + 2] = lv[i].z, x[4 * i + 3] = lv[i].w;
+            qs += ((double)qv[i].x + (double)qv[i].y) + ((double)qv[i].z + (double)qv[i].w);
         }
     } else {
+        float q[kFsElems];
 #pragma unroll
-        for (int i = 0; i < kFsElems; ++i) x[i] = e[i] < V ? __ldg(row + e[i]) : -INFINITY;
+        for (int i = 0; i < kFsElems; ++i) {
+            const bool in = tok_of(i) < V;
+            x[i] = in ? __ldg(row + tok_of(i)) : -INFINITY;
+            q[i] = in ? __ldg(qrow + tok_of(i)) : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < kFsElems; ++i) qs += (double)q[i];
     }
-    // a NaN or +Inf anywhere in the segment: the row is unusable (the walk flags the sequence); say so in the first slot
+    // the thread's maximum (a NaN survives), then per warp: the largest and the smallest finite thread maximum and how
+    // many threads have a finite one; the warp's draft mass
     float mx = x[0];
 #pragma unroll
     for (int i = 1; i < kFsElems; ++i) mx = fmax_keep_nan(mx, x[i]);
-    const int bad = __syncthreads_or(!(mx < INFINITY));
-    FCand* out = cand + (((size_t)b * T + node) * gridDim.x + seg) * k;
-    if (bad) {
+    const uint32_t key = mx < INFINITY ? f_key(mx) : 0xffffffffu;  // NaN (whatever its bits) and +Inf rank on top
+    const bool fin = key > kKeyNegInf;  // the thread holds something above -inf
+    const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+    const uint32_t kmin = __reduce_min_sync(0xffffffffu, fin ? key : 0xffffffffu);
+    const int nfin_w = __popc(__ballot_sync(0xffffffffu, fin));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) qs += __shfl_xor_sync(0xffffffffu, qs, o);
+    if (lane == 0) sh.wmax[warp] = kmax, sh.wmin[warp] = kmin, sh.wfin[warp] = nfin_w, sh.wq[warp] = qs;
+    sh.fast.hist[tid] = 0;  // kFsBins == kFsThreads
+    if (tid == 0) sh.ncand = 0;
+    __syncthreads();
+    uint32_t Kmax = 0, Kmin = 0xffffffffu;
+    int n_fin = 0;
+#pragma unroll
+    for (int w = 0; w < kFsThreads / 32; ++w) Kmax = max(Kmax, sh.wmax[w]), Kmin = min(Kmin, sh.wmin[w]), n_fin += sh.wfin[w];
+    if (tid == 0) {
+        double tot = 0.0;
+        for (int w = 0; w < kFsThreads / 32; ++w) tot += sh.wq[w];
+        qpart[at * gridDim.x + seg] = tot;
+    }
+    FCand* out = cand + (at * gridDim.x + seg) * k;
+    if (Kmax >= kKeyPosInf) {  // a NaN or +Inf in the segment: the row is unusable (the walk flags the sequence)
         for (int r = tid; r < k; r += kFsThreads) out[r].x = r == 0 ? INFINITY : -INFINITY, out[r].tok = r == 0 ? 0 : INT_MAX;
         return;
     }
+    const int n_valid = min(kFsSeg, V - s0);
+    // ---- which entries can be among the k best (CTA-uniform decisions)
+    int n_cand = -1;  // -1: the slow path
+    if (n_valid <= kFsCap) {  // a short tail segment: every entry is a candidate
 #pragma unroll
-    for (int i = 0; i < kFsElems; ++i)
-        if (e[i] >= V) e[i] = INT_MAX;  // entries beyond the row rank last
+        for (int i = 0; i < kFsElems; ++i)
+            if (tok_of(i) < V) {
+                const int slot = atomicAdd(&sh.ncand, 1);
+                sh.fast.cand[slot].x = x[i], sh.fast.cand[slot].tok = tok_of(i);
+            }
+        n_cand = n_valid;
+    } else if (n_fin >= k) {
+        // at least n_fin >= k entries are >= lo, so nothing below lo is among the k best; bins fall with the logit
+        // (float subtraction, multiplication by a positive constant and truncation are monotone), equal logits share a bin
+        const float M = f_unkey(Kmax), lo = f_unkey(Kmin);
+        const float inv = (float)kFsBins / (M - lo);
+        auto bin_of = [&](float v) { return min(kFsBins - 1, (int)((M - v) * inv)); };  // (int)NaN = 0: M == lo
+#pragma unroll
+        for (int i = 0; i < kFsElems; ++i)
+            if (x[i] >= lo) atomicAdd(&sh.fast.hist[bin_of(x[i])], 1);
+        __syncthreads();
+        // every warp finds the bin where the count from the top reaches k (the same scan in every warp: no broadcast)
+        int c8[8], mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c8[j] = sh.fast.hist[lane * 8 + j], mine += c8[j];
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const uint32_t reach = __ballot_sync(0xffffffffu, incl >= k);  // not empty: the bins hold >= n_fin >= k entries
+        const int L = __ffs(reach) - 1;
+        int bstar = 0, ctot = 0;
+        if (lane == L) {
+            int run = incl - mine;
+            for (int j = 0; j < 8; ++j) {
+                run += c8[j];
+                if (run >= k) {
+                    bstar = lane * 8 + j, ctot = run;
+                    break;
+                }
+            }
+        }
+        bstar = __shfl_sync(0xffffffffu, bstar, L), ctot = __shfl_sync(0xffffffffu, ctot, L);
+        if (ctot <= kFsCap) {
+#pragma unroll
+            for (int i = 0; i < kFsElems; ++i)
+                if (x[i] >= lo && bin_of(x[i]) <= bstar) {
+                    const int slot = atomicAdd(&sh.ncand, 1);
+                    sh.fast.cand[slot].x = x[i], sh.fast.cand[slot].tok = tok_of(i);
+                }
+            n_cand = ctot;
+        }
+    }
+    __syncthreads();
+    if (n_cand >= 0) {
+        // exact ranks among the candidates by counting; the order is total, so the ranks are 0 .. n_cand-1
+        if (tid < n_cand) {
+            const FCand me = sh.fast.cand[tid];
+            int r = 0;
+            for (int j = 0; j < n_cand; ++j) {
+                const FCand o = sh.fast.cand[j];
+                r += f_before(o.x, o.tok, me.x, me.tok) ? 1 : 0;
+            }
+            if (r < k) out[r] = me;
+        }
+        for (int r = n_cand + tid; r < k; r += kFsThreads) out[r].x = -INFINITY, out[r].tok = INT_MAX;
+        return;
+    }
+    // ---- the slow exact path (the barrier above: nobody reads the histogram any more, its memory is reused)
+    int e[kFsElems];
+#pragma unroll
+    for (int i = 0; i < kFsElems; ++i) e[i] = tok_of(i) < V ? tok_of(i) : INT_MAX;  // entries beyond the row rank last
     // sort the thread's 16 entries, best first (bitonic network on (logit, token) pairs; the order is total)
 #pragma unroll
     for (int size = 2; size <= kFsElems; size <<= 1)
@@ -129,44 +278,85 @@ filter_segments_kernel(const float* __restrict__ logits, const int32_t* __restri
                     }
                 }
             }
-    __shared__ FCand lists[kFsElems][kFsThreads];       // entry h of thread t at [h][t]
-    __shared__ FCand wlist[kFsThreads / 32][kMaxTopK];  // the warps' k best
 #pragma unroll
-    for (int i = 0; i < kFsElems; ++i) lists[i][tid].x = x[i], lists[i][tid].tok = e[i];
+    for (int i = 0; i < kFsElems; ++i) sh.slow.lists[i][tid].x = x[i], sh.slow.lists[i][tid].tok = e[i];
     __syncwarp();
-    merge_heads(&lists[0][warp * 32], 32, kFsElems, kFsThreads, 1, k, wlist[warp]);
+    merge_heads(&sh.slow.lists[0][warp * 32], 32, kFsElems, kFsThreads, 1, k, sh.slow.wlist[warp]);
     __syncthreads();
-    if (warp == 0) merge_heads(&wlist[0][0], kFsThreads / 32, k, 1, kMaxTopK, k, out);
+    if (warp == 0) merge_heads(&sh.slow.wlist[0][0], kFsThreads / 32, k, 1, kMaxTopK, k, out);
 }
 
 struct KeptLists {  // per (sequence, node): the filtered target distribution
     int32_t* n;     // [B*T]: kept tokens (1..top_k); -1: the row is unusable (NaN / +Inf logit, or nothing but -Inf)
     int32_t* tok;   // [B*T*k] in rank order
-    double* p;      // [B*T*k]
+    double* p;      // [B*T*k] target probabilities
+    float* q0;      // [B*T*k] the draft row's probabilities of the same tokens, as given
+    double* qtot;   // [B*T] the draft row's mass
 };
 
-__global__ void __launch_bounds__(32)
-filter_rows_kernel(const FCand* __restrict__ cand, const int32_t* __restrict__ n_nodes, int T, int segs, int k, double inv_tau,
-                   double top_p, KeptLists kept) {
-    const int node = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
-    if (n_nodes && node >= n_nodes[b]) return;
-    __shared__ FCand best[2][kMaxTopK];
-    __shared__ FCand stage[32][kMaxTopK];
-    const FCand* c = cand + ((size_t)b * T + node) * segs * k;
-    // the row's k best out of the segments' lists: 31 lists at a time, each round merged with the best so far
-    int have = 0, cur = 0;
-    for (int s0 = 0; s0 < segs; s0 += 31) {
-        const int ns = min(31, segs - s0);
-        for (int i = lane; i < ns * k; i += 32) stage[i / k][i % k] = c[(size_t)(s0 + i / k) * k + i % k];
-        if (have)
-            for (int i = lane; i < k; i += 32) stage[ns][i] = best[cur][i];
-        __syncwarp();
-        merge_heads(&stage[0][0], ns + (have ? 1 : 0), k, 1, kMaxTopK, k, best[cur ^ 1]);
-        __syncwarp();
-        cur ^= 1, have = 1;
+constexpr int kFrThreads = 512;  // 16 warps: one pair of lists each
+constexpr int kFrLists = 32;     // lists merged per round
+
+// One warp merges two sorted lists of 64 (best first; lane l holds entries l and l + 32 of the result) and keeps the
+// 64 best: entry i of the one against entry 63 - i of the other leaves the 64 best as a bitonic sequence, which five
+// shuffle stages and one in-lane stage sort.
+__device__ __forceinline__ void merge_pair(const FCand* a, const FCand* b, FCand& c0, FCand& c1) {
+    const int lane = threadIdx.x & 31;
+    const FCand a0 = a[lane], a1 = a[lane + 32], b0 = b[63 - lane], b1 = b[31 - lane];
+    c0 = f_before(b0.x, b0.tok, a0.x, a0.tok) ? b0 : a0;
+    c1 = f_before(b1.x, b1.tok, a1.x, a1.tok) ? b1 : a1;
+    if (f_before(c1.x, c1.tok, c0.x, c0.tok)) {
+        const FCand t = c0;
+        c0 = c1, c1 = t;
     }
-    const FCand* top = best[cur];
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        const bool low = (lane & s) == 0;  // the lower lane of a pair keeps the better entry
+        FCand o;
+        o.x = __shfl_xor_sync(0xffffffffu, c0.x, s), o.tok = __shfl_xor_sync(0xffffffffu, c0.tok, s);
+        if (f_before(o.x, o.tok, c0.x, c0.tok) == low) c0 = o;
+        o.x = __shfl_xor_sync(0xffffffffu, c1.x, s), o.tok = __shfl_xor_sync(0xffffffffu, c1.tok, s);
+        if (f_before(o.x, o.tok, c1.x, c1.tok) == low) c1 = o;
+    }
+}
+
+__global__ void __launch_bounds__(kFrThreads)
+filter_rows_kernel(const FCand* __restrict__ cand, const double* __restrict__ qpart, const float* __restrict__ dprobs,
+                   const int32_t* __restrict__ n_nodes, int T, int V, int segs, int k, double inv_tau, double top_p,
+                   KeptLists kept) {
+    const int node = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (n_nodes && node >= n_nodes[b]) return;
+    __shared__ FCand A[kFrLists][kMaxTopK];
     const size_t at = (size_t)b * T + node;
+    const FCand* c = cand + at * segs * k;
+    // the row's best out of the segments' lists: 32 lists at a time (later rounds: the best so far and 31 new ones),
+    // halved by pairwise merges until one is left in A[0]
+    for (int s = 0, first = 1; s < segs; first = 0) {
+        const int base = first ? 0 : 1, cnt = min(kFrLists - base, segs - s);
+        for (int i = tid; i < cnt * kMaxTopK; i += kFrThreads) {
+            const int l = i >> 6, j = i & 63;
+            FCand v;
+            v.x = -INFINITY, v.tok = INT_MAX;
+            if (j < k) v = c[(size_t)(s + l) * k + j];
+            A[base + l][j] = v;
+        }
+        __syncthreads();
+        for (int n = base + cnt; n > 1;) {
+            const int half = (n + 1) >> 1;
+            FCand c0, c1;
+            if (warp < (n >> 1))
+                merge_pair(A[2 * warp], A[2 * warp + 1], c0, c1);
+            else if (warp < half)  // n is odd: the last list moves down as it is
+                c0 = A[n - 1][lane], c1 = A[n - 1][lane + 32];
+            __syncthreads();
+            if (warp < half) A[warp][lane] = c0, A[warp][lane + 32] = c1;
+            __syncthreads();
+            n = half;
+        }
+        s += cnt;
+    }
+    if (warp != 0) return;
+    const FCand* top = A[0];
     const float M = top[0].x;
     if (!(M > -INFINITY && M < INFINITY)) {
         if (lane == 0) kept.n[at] = -1;
@@ -198,11 +388,16 @@ filter_rows_kernel(const FCand* __restrict__ cand, const int32_t* __restrict__ n
         }
         m_s = m, mass_s = mass;
         kept.n[at] = m;
+        double qt = 0.0;  // the draft row's mass: the segments' sums in segment order
+        for (int s = 0; s < segs; ++s) qt += qpart[at * segs + s];
+        kept.qtot[at] = qt;
     }
     __syncwarp();
     for (int j = lane; j < k; j += 32) {
-        kept.tok[at * k + j] = j < m_s ? top[j].tok : -1;
-        kept.p[at * k + j] = j < m_s ? ej[j] / mass_s : 0.0;
+        const bool in = j < m_s;
+        kept.tok[at * k + j] = in ? top[j].tok : -1;
+        kept.p[at * k + j] = in ? ej[j] / mass_s : 0.0;
+        kept.q0[at * k + j] = in ? __ldg(dprobs + at * V + top[j].tok) : 0.f;
     }
 }
 
@@ -213,11 +408,11 @@ struct SparseShared {
     int depth[S4C_MAX_T];
     uint32_t anc[S4C_MAX_T][S4C_MASK_WORDS];
     double tq0[S4C_MAX_T];   // draft probability of node i's token under its parent's row
-    int ktok[kMaxTopK];      // the current node's kept tokens, in TOKEN order (the order the vocabulary is scanned in)
+    int ktok[kMaxTopK];      // the current node's kept tokens, in rank order
     double kp[kMaxTopK];     // their current target probabilities
     double kq0[kMaxTopK];    // their draft probabilities as given
     int kgone[kMaxTopK];     // 1: the token was rejected here and has left the draft distribution
-    double red[kFsThreads / 32];
+    int order[kMaxTopK];     // the kept tokens' list positions in token order (the order the vocabulary is scanned in)
     int flag;
 };
 
@@ -227,7 +422,7 @@ accept_walk_sparse_kernel(const float* __restrict__ dprobs, const int32_t* __res
                           int max_depth, KeptLists kept, int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
                           int32_t* __restrict__ next_token, uint8_t* __restrict__ near_tie, int32_t* __restrict__ status) {
     __shared__ SparseShared sh;
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int n = n_nodes ? n_nodes[b] : T;
     int32_t* pth = path + (size_t)b * (max_depth + 1);
     for (int i = tid; i < T; i += blockDim.x) {
@@ -256,33 +451,25 @@ accept_walk_sparse_kernel(const float* __restrict__ dprobs, const int32_t* __res
     for (int i = 1 + tid; i < n; i += blockDim.x)
         sh.tq0[i] = (double)__ldg(dprobs + ((size_t)b * T + sh.par[i]) * V + sh.tok[i]);
     __syncthreads();
+    if (tid >= 32) return;  // the walk itself is one warp's work: lists of at most 64 entries, two per lane
 
     int cur = 0;
     for (int guard = 0; guard <= T; ++guard) {
         const size_t at = (size_t)b * T + cur;
-        const float* qrow = dprobs + at * V;
         const int m = kept.n[at];
-        // the kept tokens in token order: entry j goes to the position given by the number of smaller tokens
-        if (tid < m) {
-            const int t = kept.tok[at * k + tid];
-            int pos = 0;
-            for (int j = 0; j < m; ++j) pos += kept.tok[at * k + j] < t ? 1 : 0;
-            sh.ktok[pos] = t, sh.kp[pos] = kept.p[at * k + tid], sh.kq0[pos] = (double)__ldg(qrow + t), sh.kgone[pos] = 0;
-        }
-        __syncthreads();
-        auto find = [&](int x) {  // position of token x among the kept ones, or -1
-            for (int j = 0; j < m; ++j)
-                if (sh.ktok[j] == x) return j;
-            return -1;
-        };
-        double qscale = 1.0;   // the draft distribution is the given row times this, rejected tokens left out
-        double qtot = 0.0;     // its total mass (computed when the first rejection needs it)
-        bool have_qtot = false;
+        double qtot = kept.qtot[at];  // mass of the draft distribution as it stands
+        double qscale = 1.0;          // the draft distribution is the given row times this, rejected tokens left out
+        for (int j = lane; j < m; j += 32)
+            sh.ktok[j] = kept.tok[at * k + j], sh.kp[j] = kept.p[at * k + j], sh.kq0[j] = (double)kept.q0[at * k + j], sh.kgone[j] = 0;
+        __syncwarp();
         int accepted = -1;
         for (int c = cur + 1; c < n; ++c) {
             if (sh.par[c] != cur) continue;
             const int x = sh.tok[c];
-            const int jx = find(x);
+            // position of token x among the kept ones, or -1
+            const uint32_t h0 = __ballot_sync(0xffffffffu, lane < m && sh.ktok[lane] == x);
+            const uint32_t h1 = __ballot_sync(0xffffffffu, lane + 32 < m && sh.ktok[min(lane + 32, kMaxTopK - 1)] == x);
+            const int jx = h0 ? __ffs(h0) - 1 : (h1 ? 31 + __ffs(h1) : -1);
             const double px = jx >= 0 ? sh.kp[jx] : 0.0;
             bool gone = jx >= 0 && sh.kgone[jx];
             if (jx < 0)  // a token outside the kept set may have been rejected here before (duplicate siblings)
@@ -294,40 +481,26 @@ accept_walk_sparse_kernel(const float* __restrict__ dprobs, const int32_t* __res
             else
                 ratio = px > 0.0 ? (double)INFINITY : 0.0;
             const double u = (double)sh.uni[c];
-            if (tid == 0 && near_tie && fabs(ratio - u) < 1e-6) near_tie[(size_t)b * T + c] = 1;
+            if (lane == 0 && near_tie && fabs(ratio - u) < 1e-6) near_tie[(size_t)b * T + c] = 1;
             if (u < (ratio < 1.0 ? ratio : 1.0)) {
                 accepted = c;
                 break;
             }
             // rejected: the target becomes the normalised residual (over the kept tokens: everywhere else it is zero and
             // stays zero), the token leaves the draft distribution, which is renormalised
-            if (!have_qtot) {  // the draft row's mass: one pass of the CTA over the row, fixed order
-                double part = 0.0;
-                for (int v = tid; v < V; v += blockDim.x) part += (double)__ldg(qrow + v);
+            double r0 = 0.0, r1 = 0.0;
+            if (lane < m) r0 = fmax(sh.kp[lane] - (sh.kgone[lane] ? 0.0 : sh.kq0[lane] * qscale), 0.0);
+            if (lane + 32 < m) r1 = fmax(sh.kp[lane + 32] - (sh.kgone[lane + 32] ? 0.0 : sh.kq0[lane + 32] * qscale), 0.0);
+            double Z = r0 + r1;
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                __syncthreads();
-                if ((tid & 31) == 0) sh.red[tid >> 5] = part;
-                __syncthreads();
-                qtot = 0.0;
-                for (int w = 0; w < kFsThreads / 32; ++w) qtot += sh.red[w];
-                have_qtot = true;
+            for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, o);
+            __syncwarp();
+            if (Z > 0.0) {
+                if (lane < m) sh.kp[lane] = r0 / Z;
+                if (lane + 32 < m) sh.kp[lane + 32] = r1 / Z;
             }
-            __syncthreads();  // everyone has read the lists before thread 0 rewrites them
-            if (tid == 0) {
-                double Z = 0.0;
-                for (int j = 0; j < m; ++j) {
-                    const double r = sh.kp[j] - (sh.kgone[j] ? 0.0 : sh.kq0[j] * qscale);
-                    Z += r > 0.0 ? r : 0.0;
-                }
-                if (Z > 0.0)
-                    for (int j = 0; j < m; ++j) {
-                        const double r = sh.kp[j] - (sh.kgone[j] ? 0.0 : sh.kq0[j] * qscale);
-                        sh.kp[j] = r > 0.0 ? r / Z : 0.0;
-                    }
-                if (jx >= 0) sh.kgone[jx] = 1;
-            }
-            __syncthreads();
+            if (lane == 0 && jx >= 0) sh.kgone[jx] = 1;
+            __syncwarp();
             const double s = qtot - qx;  // mass left once x is gone
             if (!(s > 0.0)) break;
             qscale /= s;
@@ -335,17 +508,24 @@ accept_walk_sparse_kernel(const float* __restrict__ dprobs, const int32_t* __res
         }
         if (accepted >= 0) {
             cur = accepted;
-            __syncthreads();
+            __syncwarp();
             continue;
         }
         // final token: inverse CDF over the current target in vocabulary order (only kept tokens carry mass)
-        if (tid == 0) {
+        for (int j = lane; j < m; j += 32) {
+            int pos = 0;
+            for (int i = 0; i < m; ++i) pos += sh.ktok[i] < sh.ktok[j] ? 1 : 0;
+            sh.order[pos] = j;
+        }
+        __syncwarp();
+        if (lane == 0) {
             double tot = 0.0;
-            for (int j = 0; j < m; ++j) tot += sh.kp[j];
+            for (int i = 0; i < m; ++i) tot += sh.kp[sh.order[i]];
             const double target = (double)sh.uni[0] * tot;
             double run = 0.0;
-            int pick = -1, last = sh.ktok[0];
-            for (int j = 0; j < m; ++j) {
+            int pick = -1, last = sh.ktok[sh.order[0]];
+            for (int i = 0; i < m; ++i) {
+                const int j = sh.order[i];
                 if (sh.kp[j] > 0.0) last = sh.ktok[j];
                 run += sh.kp[j];
                 if (run > target) {
@@ -363,16 +543,23 @@ accept_walk_sparse_kernel(const float* __restrict__ dprobs, const int32_t* __res
 }
 
 static inline int fs_segments(int V) { return ceil_div(V, kFsSeg); }
-static inline size_t filtered_ws_layout(int B, int T, int V, int k, char* base, FCand** cand, KeptLists* kept) {
+static inline size_t filtered_ws_layout(int B, int T, int V, int k, char* base, FCand** cand, double** qpart, KeptLists* kept) {
     size_t off = 0;
+    const size_t rows = (size_t)B * T;
     if (cand) *cand = reinterpret_cast<FCand*>(base + off);
-    off += round_up((size_t)B * T * fs_segments(V) * k * sizeof(FCand), 256);
+    off += round_up(rows * fs_segments(V) * k * sizeof(FCand), 256);
+    if (qpart) *qpart = reinterpret_cast<double*>(base + off);
+    off += round_up(rows * fs_segments(V) * sizeof(double), 256);
     if (kept) kept->p = reinterpret_cast<double*>(base + off);
-    off += round_up((size_t)B * T * k * sizeof(double), 256);
+    off += round_up(rows * k * sizeof(double), 256);
+    if (kept) kept->qtot = reinterpret_cast<double*>(base + off);
+    off += round_up(rows * sizeof(double), 256);
     if (kept) kept->tok = reinterpret_cast<int32_t*>(base + off);
-    off += round_up((size_t)B * T * k * sizeof(int32_t), 256);
+    off += round_up(rows * k * sizeof(int32_t), 256);
+    if (kept) kept->q0 = reinterpret_cast<float*>(base + off);
+    off += round_up(rows * k * sizeof(float), 256);
     if (kept) kept->n = reinterpret_cast<int32_t*>(base + off);
-    off += round_up((size_t)B * T * sizeof(int32_t), 256);
+    off += round_up(rows * sizeof(int32_t), 256);
     return off;
 }
 
@@ -380,7 +567,7 @@ static inline size_t filtered_ws_layout(int B, int T, int V, int k, char* base, 
 
 extern "C" size_t s4c_tree_accept_filtered_workspace_bytes(int B, int T, int V, int top_k) {
     if (B < 1 || T < 1 || V < 1 || top_k < 1 || top_k > s4c::kMaxTopK) return 0;
-    return s4c::filtered_ws_layout(B, T, V, top_k < V ? top_k : V, nullptr, nullptr, nullptr);
+    return s4c::filtered_ws_layout(B, T, V, top_k < V ? top_k : V, nullptr, nullptr, nullptr, nullptr);
 }
 
 extern "C" s4c_status s4c_tree_accept_filtered(const float* target_logits, const float* draft_probs, const int32_t* tokens,
@@ -397,20 +584,22 @@ extern "C" s4c_status s4c_tree_accept_filtered(const float* target_logits, const
     if (!aligned16(target_logits) || !aligned16(draft_probs)) return S4C_ERR_ALIGN;
     if (B == 0) return S4C_OK;
     const int k = top_k < V ? top_k : V;
-    const size_t need = filtered_ws_layout(B, T, V, k, nullptr, nullptr, nullptr);
+    const size_t need = filtered_ws_layout(B, T, V, k, nullptr, nullptr, nullptr, nullptr);
     if (!workspace || workspace_bytes < need || !aligned256(workspace)) return S4C_ERR_WORKSPACE;
     FCand* cand;
+    double* qpart;
     KeptLists kept;
-    filtered_ws_layout(B, T, V, k, static_cast<char*>(workspace), &cand, &kept);
+    filtered_ws_layout(B, T, V, k, static_cast<char*>(workspace), &cand, &qpart, &kept);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int segs = fs_segments(V);
     dim3 grid(segs, T, B);
     if (V % 4 == 0)
-        filter_segments_kernel<true><<<grid, kFsThreads, 0, stream>>>(target_logits, n_nodes, T, V, k, cand);
+        filter_segments_kernel<true><<<grid, kFsThreads, 0, stream>>>(target_logits, draft_probs, n_nodes, T, V, k, cand, qpart);
     else
-        filter_segments_kernel<false><<<grid, kFsThreads, 0, stream>>>(target_logits, n_nodes, T, V, k, cand);
+        filter_segments_kernel<false><<<grid, kFsThreads, 0, stream>>>(target_logits, draft_probs, n_nodes, T, V, k, cand, qpart);
     S4C_RETURN_IF_CUDA_ERROR();
-    filter_rows_kernel<<<dim3(T, B), 32, 0, stream>>>(cand, n_nodes, T, segs, k, 1.0 / (double)temperature, (double)top_p, kept);
+    filter_rows_kernel<<<dim3(T, B), kFrThreads, 0, stream>>>(cand, qpart, draft_probs, n_nodes, T, V, segs, k,
+                                                              1.0 / (double)temperature, (double)top_p, kept);
     S4C_RETURN_IF_CUDA_ERROR();
     accept_walk_sparse_kernel<<<B, kFsThreads, 0, stream>>>(draft_probs, tokens, parent, n_nodes, uniforms, T, V, k, max_depth,
                                                             kept, accept_len, path, next_token, near_tie, status);

@@ -43,6 +43,7 @@ class VerifyStep:
         self.temperature, self.max_depth = float(temperature), int(max_depth)
         self.max_cache_len = int(max_cache_len)
         self.branching, self.root_token = None, None
+        self.filter = None
         self.feat_in = feat_in
         dev = cache_len.device
         B, T, V = target_logits.shape
@@ -105,7 +106,22 @@ class VerifyStep:
                                out=self.attn_out[l], status=self.status_attn, workspace=self.ws_attn,
                                max_cache_len=self.max_cache_len)
 
+    def set_filter(self, top_k: Optional[int], top_p: float = 1.0):
+        """From now on ``accept()`` verifies against the top-k / nucleus filtered target distribution
+        (s4c_tree_accept_filtered); ``top_k=None`` goes back to the unfiltered one."""
+        assert top_k is None or self.temperature > 0, "the filter belongs to stochastic acceptance"
+        self.filter = None if top_k is None else (int(top_k), float(top_p))
+        if self.filter is not None:
+            need = s4c.tree_accept_filtered_workspace_bytes(self.B, self.T, self.V, int(top_k))
+            self.ws_filter = torch.empty(max(1, need), dtype=torch.uint8, device=self.cache_len.device)
+
     def accept(self):
+        if self.filter is not None:
+            s4c.tree_accept_filtered(self.logits, self.draft_probs, self.tokens, self.parent, self.temperature,
+                                     self.filter[0], self.filter[1], self.uniforms, self.n_nodes, self.max_depth,
+                                     self.accept_len, self.path, self.next_token, self.near_tie, self.status_accept,
+                                     self.ws_filter)
+            return
         s4c.tree_accept(self.logits, self.draft_probs, self.tokens, self.parent, self.temperature, self.uniforms,
                         self.n_nodes, self.max_depth, self.accept_len, self.path, self.next_token, self.near_tie,
                         self.status_accept, self.ws_accept)
@@ -133,8 +149,9 @@ class VerifyStep:
 
     # kernels launched by one run(): used by the benchmark to report its launch count
     def launches_per_step(self, attn_launches_per_layer: int) -> int:
-        # acceptance: per-node statistics (one launch, cluster or segment kernel) and the walk
-        accept = 2
+        # acceptance: per-node statistics (one launch, cluster or segment kernel) and the walk; filtered: segment
+        # selection, row selection and the walk
+        accept = 3 if self.filter is not None else 2
         compact = 2 if self.n_layers > 0 else 1
         tree = 2 if self.branching is not None else 0
         return self.n_layers * attn_launches_per_layer + accept + compact + tree

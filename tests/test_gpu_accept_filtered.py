@@ -104,3 +104,64 @@ def test_sweep_sized_batch():
     cfg, parent, x = _synthetic(16, 128, 32000, seed=5, sigma=3.0, tau=1.0, mode="topk", max_tree_depth=8)
     got, ref = _both(x, parent, 1.0, 50, 0.9, max_depth=cfg.max_tree_depth)
     assert assert_accept_equal(got, ref, True) == 0
+
+
+def test_verify_step_with_a_filter_in_one_graph():
+    # the whole step (attention, filtered acceptance, compaction) replayed as one CUDA graph: the decision is the
+    # oracle's filtered one and the committed lengths follow it
+    from dataclasses import replace
+
+    from paper_2506_14158_b200.verify import VerifyStep
+
+    cfg = replace(W.CONFIGS["c2"], n_layers=2)
+    parent = W.make_trees(cfg)
+    x = W.make_accept_inputs(cfg, parent, 1.0, token_mode="topk")
+    qs, ks, vs = zip(*[[t.cuda() for t in W.make_attention_inputs(cfg, l)] for l in range(cfg.n_layers)])
+    step = VerifyStep(list(qs), list(ks), list(vs), torch.full((cfg.B,), cfg.L, dtype=torch.int32, device="cuda"),
+                      dev(parent), dev(x["tokens"]), dev(x["logits"]), dev(x["draft_probs"]), dev(x["uniforms"]), 1.0,
+                      cfg.max_depth, feat_in=W.make_features(cfg).cuda(), max_cache_len=cfg.L)
+    step.set_filter(20, 0.9)
+    g = step.capture("step")
+    g.replay()
+    torch.cuda.synchronize()
+    ref = oracle.accept_filtered(x["logits"], x["draft_probs"], x["tokens"], np.ascontiguousarray(parent, dtype=np.int32), 1.0,
+                                 20, float(np.float32(0.9)), x["uniforms"], None, cfg.max_depth)
+    for key in ("accept_len", "path", "next_token"):
+        np.testing.assert_array_equal(getattr(step, key).cpu().numpy(), ref[key], err_msg=key)
+    np.testing.assert_array_equal(step.cache_len.cpu().numpy(), cfg.L + ref["accept_len"] + 1)
+    plain = oracle.accept_stochastic(x["logits"], x["draft_probs"], x["tokens"], np.ascontiguousarray(parent, dtype=np.int32),
+                                     1.0, x["uniforms"], None, cfg.max_depth)
+    step.set_filter(None)
+    step.run()
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(step.accept_len.cpu().numpy(), plain["accept_len"])
+
+
+@pytest.mark.parametrize("V", [140000, 270001])
+def test_rows_wider_than_one_merge_round(V):
+    # more than 32 vocabulary segments per row: the row's best are folded over several rounds of list merges
+    cfg, parent, x = _synthetic(2, 5, V, seed=V % 89, sigma=2.5, tau=1.0, mode="topk")
+    x["logits"][0, 1, V - 3:] = 40.0    # winners in the last (ragged) segment, equal: ranked by token
+    x["logits"][1, 0, ::4096] += 30.0   # one winner in every segment
+    got, ref = _both(x, parent, 1.0, 64, 0.99, max_depth=cfg.max_tree_depth)
+    assert assert_accept_equal(got, ref, True) == 0
+
+
+@pytest.mark.parametrize("top_k,top_p", [(1, 1.0), (7, 1.0), (64, 0.9)])
+def test_segments_the_threshold_selection_cannot_serve(top_k, top_p):
+    # heavy ties and masked vocabularies: more than 256 entries at the threshold, or fewer than k finite thread maxima --
+    # those segments take the exact sort-and-merge path
+    cfg, parent, x = _synthetic(8, 6, 9000, seed=17, tau=1.0, mode="topk")
+    lg = x["logits"]
+    lg[0] = 1.25                                           # every logit equal: the k lowest tokens win
+    lg[1] = np.where(lg[1] > 0, 2.0, -1.0)                 # two values
+    lg[2] = np.round(lg[2] / 4.0)                          # a handful of values
+    keep = lg[3, :, 4090:4100].copy()
+    lg[3] = -np.inf                                        # nearly everything masked: ten finite logits across a
+    lg[3, :, 4090:4100] = keep                             # segment boundary
+    lg[4, :, :5000] = -np.inf                              # the first segment masked entirely, ties at -inf
+    lg[5] = np.minimum(lg[5], 0.5)                         # a plateau at the top
+    lg[6, :, 1:] = lg[6, :, :1]                            # every row constant, another value per row
+    got, ref = _both(x, parent, 1.0, top_k, top_p, max_depth=cfg.max_tree_depth)
+    assert (ref["status"] == 0).all()
+    assert assert_accept_equal(got, ref, True) == 0
