@@ -14,6 +14,9 @@ Functions (array layouts are row-major numpy arrays):
 * :func:`kv_compact`          -- Section 3.2 last paragraph: keep accepted tokens' K/V and features.
 * :func:`build_tree`          -- Section 3.2 / Figure 3: the continuous verification tree (vertical top-1 chain, then
                                  horizontal top-k alternatives), breadth-first numbered.
+* :func:`lm_head_greedy`      -- Eq. 6 / Section 3.2: the LM head over the tree nodes' hidden states and the greedy choice
+                                 (numpy, float64; a library matrix product is the step).
+* :func:`accept_greedy_tokens` -- the greedy walk when the target's choice per node is already known (plain Python).
 """
 from __future__ import annotations
 
@@ -260,3 +263,77 @@ def scatter_to_pages(pages, block_table, contiguous, blocks_in_use):
         for i in range(int(blocks_in_use[b])):
             pages[int(block_table[b, i])] = contiguous[b, :, i * ps:(i + 1) * ps]
     return pages
+
+
+def lm_head_greedy(hidden, weight):
+    """The LM head of the verify pass followed by the greedy choice (Eq. 6: t = Argmax(LM_head(f)); Section 3.2: the
+    target's logits at every tree node; Section 4.1: greedy decoding): logits[r, v] = sum_h hidden[r, h] * weight[v, h]
+    in float64 (a library matrix product is the step), token[r] = the first maximum of row r.
+
+    hidden [R, H], weight [V, H] (any float type: the values as given, e.g. already rounded to bf16).
+    Returns dict(token [R] int32, max_logit [R] float64, logits [R, V] float64)."""
+    h = np.asarray(hidden, dtype=np.float64)
+    w = np.asarray(weight, dtype=np.float64)
+    assert h.ndim == 2 and w.ndim == 2 and h.shape[1] == w.shape[1]
+    logits = h @ w.T
+    token = np.argmax(logits, axis=1).astype(np.int32)  # numpy returns the first of equal maxima
+    return dict(token=token, max_logit=logits[np.arange(len(h)), token], logits=logits)
+
+
+def accept_greedy_tokens(target_token, tokens, parent, n_nodes=None, max_depth=None, V=None):
+    """Greedy verification (Section 4.1; longest accepted path, Section 3.2) when the target's greedy choice at every
+    node is already known: a node is accepted when its parent is and its token is the target's choice at the parent; the
+    path ends at the accepted node of greatest depth (lowest index among equals); the token emitted after the path is
+    the target's choice at its end.
+
+    target_token [B,T] int32 (row n: the choice after node n), tokens [B,T], parent [B,T]; V (optional): tokens outside
+    [0, V) flag the sequence.  Returns dict(accept_len[B], path[B,max_depth+1] (-1 padded), next_token[B], status[B])
+    like accept_greedy."""
+    target_token = _i32(target_token)
+    B, T = target_token.shape
+    tokens = _i32(tokens).reshape(B, T)
+    parent = _i32(parent).reshape(B, T)
+    if max_depth is None:
+        max_depth = T - 1
+    a, path, nxt, status = _accept_outputs(B, max_depth)
+    for b in range(B):
+        n = T if n_nodes is None else int(n_nodes[b])
+        flags = 0
+        if n < 1 or n > T:
+            flags |= SEQ_BAD_PARENT
+        else:
+            for i in range(n):
+                p = int(parent[b, i])
+                if (i == 0 and p != -1) or (i > 0 and not (0 <= p < i)):
+                    flags |= SEQ_BAD_PARENT
+        depth = [0] * T
+        if not flags:
+            for i in range(n):
+                if i > 0:
+                    depth[i] = depth[parent[b, i]] + 1
+                if depth[i] > max_depth:
+                    flags |= SEQ_DEPTH
+                if V is not None and not (0 <= tokens[b, i] < V):
+                    flags |= SEQ_TOKEN_RANGE
+        status[b] = flags
+        if flags:
+            a[b], nxt[b], path[b, :] = -1, -1, -1
+            continue
+        ok = [False] * n
+        ok[0], end = True, 0
+        for i in range(1, n):
+            p = int(parent[b, i])
+            ok[i] = ok[p] and tokens[b, i] == target_token[b, p]
+            if ok[i] and depth[i] > depth[end]:
+                end = i
+        walked = []
+        i = end
+        while i >= 0:
+            walked.append(i)
+            i = int(parent[b, i])
+        walked.reverse()
+        a[b] = len(walked) - 1
+        path[b, :] = -1
+        path[b, :len(walked)] = walked
+        nxt[b] = target_token[b, end]
+    return dict(accept_len=a, path=path, next_token=nxt, status=status)
