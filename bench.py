@@ -393,6 +393,41 @@ def measure(cfg, args, device, rank, world, with_e2e):
         ms_filt = time_graph(step.capture("accept"), K, torch)
         step.set_filter(None)
         g_acc.replay()  # the step's own decision is back in the output buffers
+    # the LM head fused with the greedy choice, then the greedy walk on the choices: the route on which the [B,T,V] logits
+    # never exist (timed alone; the step above takes the logits as input).  Weights larger than L2 on both shapes.
+    lm = None
+    if cfg.dtype == "bf16" and not args.paged:
+        from paper_2506_14158_b200 import s4c
+        from paper_2506_14158_b200 import workloads as Wl
+
+        hid = step.feat_in.reshape(cfg.B * cfg.T, cfg.hid).contiguous()
+        wgt = Wl.make_lm_head(cfg, device)
+        choice = torch.empty(cfg.B * cfg.T, dtype=torch.int32, device=device)
+        mx = torch.empty(cfg.B * cfg.T, dtype=torch.float32, device=device)
+        st = torch.zeros(1, dtype=torch.int32, device=device)
+        ws = torch.empty(s4c.lm_head_greedy_workspace_bytes(cfg.B * cfg.T, cfg.V, cfg.hid), dtype=torch.uint8, device=device)
+        outs = [torch.empty_like(step.accept_len), torch.empty_like(step.path), torch.empty_like(step.next_token),
+                torch.empty_like(step.status_accept)]
+
+        def head_and_walk():
+            s4c.lm_head_greedy(hid, wgt, choice, mx, st, ws)
+            s4c.tree_accept_tokens(choice.view(cfg.B, cfg.T), step.tokens, step.parent, cfg.V, step.n_nodes, cfg.max_depth, *outs)
+
+        sg = torch.cuda.Stream()
+        sg.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(sg):
+            head_and_walk()
+        torch.cuda.current_stream().wait_stream(sg)
+        torch.cuda.synchronize()
+        g_lm = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_lm):
+            head_and_walk()
+        for _ in range(3):
+            g_lm.replay()
+        ms_lm = time_graph(g_lm, K, torch)
+        assert int(st.item()) == 0, "s4c_lm_head_greedy gave up a wait"
+        lm = dict(ms=ms_lm, rows=cfg.B * cfg.T, V=cfg.V, H=cfg.hid)
+        del wgt, ws
     ms_e2e = 0.0
     if with_e2e:
         # end to end: per-step inputs from pinned host memory, decision back to the host, every step
@@ -413,7 +448,7 @@ def measure(cfg, args, device, rank, world, with_e2e):
         [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
         device=device)
     rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
-               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, ms_e2e=ms_e2e, accept_lens=accept_lens,
                clocks=clocks, K=K, Wm=Wm)
     return rec
 
@@ -453,6 +488,18 @@ def roofline_records(cfg, args, rec, pk):
         breakdown["tree_build_not_in_step"] = rec["ms_tree"]
     if rec.get("ms_filt") is not None:
         breakdown[f"accept_filtered_top{FILTER_TOP_K}_p{FILTER_TOP_P}_not_in_step"] = rec["ms_filt"]
+    if rec.get("lm") is not None:
+        lm = rec["lm"]
+        breakdown["lm_head_greedy_and_walk_not_in_step"] = lm["ms"]
+        flops = 2.0 * lm["rows"] * lm["V"] * lm["H"]
+        byts = 2.0 * lm["V"] * lm["H"] + 2.0 * lm["rows"] * lm["H"]  # the weights and the hidden states once (bf16)
+        t = lm["ms"] * 1e-3
+        tensor_bound = flops / byts >= ridge
+        roofline["lm_head"] = dict(
+            kernel="lm_head_greedy_kernel (+ merge and the greedy walk on the choices)", rows=lm["rows"], V=lm["V"], H=lm["H"],
+            us=lm["ms"] * 1e3, bound="tensor" if tensor_bound else "hbm",
+            tflops=flops / t * 1e-12, frac_of_tensor_peak=flops / t * 1e-12 / pk["bf16_tflops"],
+            gbs=byts / t * 1e-9, frac_of_hbm_peak=byts / t * 1e-9 / pk["hbm_gbs"], flop_per_byte=flops / byts)
     return ab, step_hbm, roofline, breakdown
 
 

@@ -243,6 +243,38 @@ s4c_status s4c_tree_accept_filtered(const float* target_logits, const float* dra
                                     int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * s4c_lm_head_greedy -- the LM head of the verify pass fused with the greedy choice (Eq. 6:
+ * t = Argmax(LM_head(f)); Section 3.2: the target's logits at every tree node; Section 4.1: greedy
+ * decoding in all experiments): for every row r of the hidden states
+ *     logits[r, v] = sum_h hidden[r, h] * weight[v, h]      (bf16 inputs, float32 accumulation)
+ *     token[r]     = the first v that reaches max_v logits[r, v];   max_logit[r] = that maximum
+ * The [R, V] logits are not written anywhere.
+ *   hidden [R, H] bf16 (device), weight [V, H] bf16 (device, the LM head's rows), both row-major and
+ *   16-byte aligned; H a multiple of 64; any R (rows are served in groups of 256, each group reads
+ *   the weights once); token [R] int32 (device); max_logit [R] float (device) or NULL;
+ *   status: one int32 (device) or NULL, set to 0 and OR-ed with S4C_SEQ_TIMEOUT if a wait inside
+ *   the kernel was given up (results are then undefined); workspace: at least
+ *   s4c_lm_head_greedy_workspace_bytes(R, V, H) bytes, 256-byte aligned, caller-owned.
+ * Equal logits (as float32 sums in the tensor cores' order) go to the lower token; a row without any
+ * comparable logit (NaN everywhere) gets token -1.  Launches are asynchronous on `stream`.
+ *
+ * s4c_tree_accept_tokens -- greedy verification (Section 4.1; longest accepted path, Section 3.2)
+ * from the target's choice per node instead of its logits: a node is accepted when its parent is and
+ * its token equals target_token[parent]; the path ends at the accepted node of greatest depth
+ * (lowest index among equals); next_token = target_token at that node.  Arguments, outputs and
+ * status flags as s4c_tree_accept with temperature 0 (target_token [B, T] int32 replaces the logits).
+ * ------------------------------------------------------------------------------------------ */
+size_t s4c_lm_head_greedy_workspace_bytes(int R, int V, int H);
+
+s4c_status s4c_lm_head_greedy(const void* hidden, const void* weight, int R, int V, int H, int32_t* token,
+                              float* max_logit, int32_t* status, void* workspace, size_t workspace_bytes,
+                              s4c_stream_t stream);
+
+s4c_status s4c_tree_accept_tokens(const int32_t* target_token, const int32_t* tokens, const int32_t* parent,
+                                  const int32_t* n_nodes, int B, int T, int V, int max_depth, int32_t* accept_len,
+                                  int32_t* path, int32_t* next_token, int32_t* status, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * s4c_tree_attention_paged, s4c_kv_compact_paged -- the same two operations (Section 3.2: tree-masked
  * attention of the verification pass; keeping the accepted tokens' K/V) on PAGED caches, the layout
  * serving systems keep their caches in.  The paper does not discuss cache layouts.

@@ -24,7 +24,7 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
-           "s4c_tree_accept_filtered"]
+           "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -72,6 +72,12 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_accept_filtered_workspace_bytes.argtypes = [i, i, i, i]
     lib.s4c_tree_accept_filtered.restype = i
     lib.s4c_tree_accept_filtered.argtypes = [vp, vp, i32p, i32p, i32p, f, i, f, vp, i, i, i, i, i32p, i32p, i32p, vp, i32p, vp, sz, vp]
+    lib.s4c_lm_head_greedy_workspace_bytes.restype = sz
+    lib.s4c_lm_head_greedy_workspace_bytes.argtypes = [i, i, i]
+    lib.s4c_lm_head_greedy.restype = i
+    lib.s4c_lm_head_greedy.argtypes = [vp, vp, i, i, i, i32p, vp, i32p, vp, sz, vp]
+    lib.s4c_tree_accept_tokens.restype = i
+    lib.s4c_tree_accept_tokens.argtypes = [i32p, i32p, i32p, i32p, i, i, i, i, i32p, i32p, i32p, i32p, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -393,3 +399,48 @@ def tree_accept_filtered(target_logits, draft_probs, tokens, parent, temperature
     if rc:
         raise S4CError("s4c_tree_accept_filtered", rc)
     return dict(accept_len=accept_len, path=path, next_token=next_token, near_tie=near_tie, status=status)
+
+
+def lm_head_greedy_workspace_bytes(R, V, H) -> int:
+    return int(_lib.s4c_lm_head_greedy_workspace_bytes(R, V, H))
+
+
+def lm_head_greedy(hidden, weight, token=None, max_logit=None, status=None, workspace=None, stream=None):
+    """s4c_lm_head_greedy: token[r] = argmax_v sum_h hidden[r,h] * weight[v,h] (bf16 in, f32 accumulation), no logits in memory."""
+    R, H = hidden.shape
+    V = weight.shape[0]
+    dev = hidden.device
+    token = torch.empty(R, dtype=torch.int32, device=dev) if token is None else token
+    max_logit = torch.empty(R, dtype=torch.float32, device=dev) if max_logit is None else max_logit
+    status = torch.zeros(1, dtype=torch.int32, device=dev) if status is None else status
+    if workspace is None:
+        workspace = _workspace(int(_lib.s4c_lm_head_greedy_workspace_bytes(R, V, H)), dev, "lm_head")
+    rc = _lib.s4c_lm_head_greedy(_dev(hidden, torch.bfloat16, "hidden"), _dev(weight, torch.bfloat16, "weight"), R, V, H,
+                                 _dev(token, torch.int32, "token"), _dev(max_logit, torch.float32, "max_logit"),
+                                 _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+                                 workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_lm_head_greedy", rc)
+    return dict(token=token, max_logit=max_logit, status=status)
+
+
+def tree_accept_tokens(target_token, tokens, parent, V: int, n_nodes=None, max_depth: Optional[int] = None, accept_len=None,
+                       path=None, next_token=None, status=None, stream=None):
+    """s4c_tree_accept_tokens: greedy verification from the target's choice per node (target_token [B,T] int32)."""
+    B, T = target_token.shape
+    dev = target_token.device
+    if max_depth is None:
+        max_depth = T - 1
+    i32 = dict(dtype=torch.int32, device=dev)
+    accept_len = torch.empty(B, **i32) if accept_len is None else accept_len
+    path = torch.empty(B, max_depth + 1, **i32) if path is None else path
+    next_token = torch.empty(B, **i32) if next_token is None else next_token
+    status = torch.empty(B, **i32) if status is None else status
+    rc = _lib.s4c_tree_accept_tokens(_dev(target_token, torch.int32, "target_token"), _dev(tokens, torch.int32, "tokens"),
+                                     _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"), B, T, int(V),
+                                     int(max_depth), _dev(accept_len, torch.int32, "accept_len"), _dev(path, torch.int32, "path"),
+                                     _dev(next_token, torch.int32, "next_token"), _dev(status, torch.int32, "status"),
+                                     _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_accept_tokens", rc)
+    return dict(accept_len=accept_len, path=path, next_token=next_token, status=status)

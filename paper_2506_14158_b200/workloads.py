@@ -20,7 +20,7 @@ import numpy as np
 import torch
 
 BASE_SEED = 14158
-_STREAMS = {"tree": 0, "tokens": 1, "logits": 2, "noise": 3, "uniforms": 4, "q": 5, "kv": 6, "feat": 7}
+_STREAMS = {"tree": 0, "tokens": 1, "logits": 2, "noise": 3, "uniforms": 4, "q": 5, "kv": 6, "feat": 7, "lm_head": 8}
 
 
 def stream_seed(config_id: int, stream: str, extra: int = 0) -> int:
@@ -212,6 +212,15 @@ def make_attention_inputs(cfg: VerifyConfig, layer: int = 0):
 def make_features(cfg: VerifyConfig) -> torch.Tensor:
     """feat_in [B,T,hid] in the storage dtype (the hidden state before the LM head, one row per node)."""
     return _randn((cfg.B, cfg.T, cfg.hid), stream_seed(cfg.config_id, "feat"), _torch_dtype(cfg.dtype))
+
+
+def make_lm_head(cfg: VerifyConfig, device="cpu") -> torch.Tensor:
+    """The LM head's weight [V, hid] in bfloat16, entries ~ N(0, 1/hid) (random: no trained weights exist here), drawn
+    on ``device`` (the 8B-shaped head has 525 M entries) from this input's own seed."""
+    g = torch.Generator(device=device)
+    g.manual_seed(stream_seed(cfg.config_id, "lm_head"))
+    w = torch.randn((cfg.V, cfg.hid), generator=g, dtype=torch.float32, device=device)
+    return (w * (1.0 / float(cfg.hid) ** 0.5)).to(torch.bfloat16)
 
 
 def _softmax64(x: np.ndarray) -> np.ndarray:

@@ -129,4 +129,24 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert wsb(1, 8, 32000, 50) % 256 == 0 and wsb(1, 8, 32000, 50) > 0
     assert wsb(1, 8, 32000, 65) == 0 and wsb(1, 8, 32000, 0) == 0
     assert wsb(1, 8, 10, 50) == wsb(1, 8, 10, 10)               # top_k is capped by the vocabulary
+    lib.s4c_lm_head_greedy.argtypes = [vp, vp, i, i, i, vp, vp, vp, vp, sz, vp]
+    lib.s4c_lm_head_greedy_workspace_bytes.restype = sz
+    lib.s4c_lm_head_greedy_workspace_bytes.argtypes = [i, i, i]
+    lm = lambda **kw: lib.s4c_lm_head_greedy(*[kw.get(k, d) for k, d in [
+        ("h", P), ("w", P), ("R", 26), ("V", 32000), ("H", 4096), ("tok", P), ("mx", None), ("st", None), ("ws", None),
+        ("wsb", 0), ("s", None)]])
+    assert lm(h=None) == 1 and lm(w=None) == 1 and lm(tok=None) == 1
+    assert lm(H=100) == 2 and lm(H=32) == 2 and lm(V=0) == 2 and lm(R=-1) == 2   # the hidden size comes in 64-element slices
+    assert lm(w=P + 8) == 4
+    assert lm() == 5                                            # no workspace
+    assert lm(R=0) == 0
+    assert lib.s4c_lm_head_greedy_workspace_bytes(26, 32000, 4096) % 256 == 0
+    assert lib.s4c_lm_head_greedy_workspace_bytes(26, 32000, 4096) > 0 and lib.s4c_lm_head_greedy_workspace_bytes(0, 32000, 4096) == 0
+    lib.s4c_tree_accept_tokens.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, vp, vp, vp, vp]
+    tw = lambda **kw: lib.s4c_tree_accept_tokens(*[kw.get(k, d) for k, d in [
+        ("tgt", P), ("tok", P), ("par", P), ("nn", None), ("B", 1), ("T", 8), ("V", 100), ("md", 7), ("al", P), ("path", P),
+        ("nt", P), ("st", None), ("s", None)]])
+    assert tw(tgt=None) == 1 and tw(par=None) == 1 and tw(nt=None) == 1
+    assert tw(T=129) == 2 and tw(V=0) == 2 and tw(md=128) == 2 and tw(B=-1) == 2
+    assert tw(B=0) == 0
     assert b"workspace" in lib.s4c_status_string(5)
