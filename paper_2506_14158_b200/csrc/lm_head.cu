@@ -26,18 +26,20 @@ namespace s4c {
 using namespace tcp;
 
 constexpr int kLmBM = 128;        // rows per accumulator (tensor-memory lanes)
-constexpr int kLmBN = 128;        // vocabulary entries per tile
 constexpr int kLmBK = 64;         // hidden elements per stage (one 128-byte swizzled row)
 constexpr int kLmTileBytes = kLmBM * kLmBK * 2;  // 16 KB: one 128 x 64 bf16 operand tile
 constexpr int kLmThreads = 192;   // producer warp, issuer warp, four epilogue warps
 constexpr int kLmRowsPerLaunch = 2 * kLmBM;
 
+// Vocabulary entries per tile: a launch-time choice (a multiple of 32), so that the tiles spread evenly over the CTAs
+// (V = 32000 on 148 SMs: 143 tiles of 224 instead of 250 of 128 in two uneven rounds).  Two row tiles leave room for 128.
 template <int NM>
 struct LmCfg {
-    static constexpr int kStages = NM == 2 ? 4 : 6;
-    static constexpr int kStageBytes = (NM + 1) * kLmTileBytes;
-    static constexpr int kTmemCols = 2 * NM * kLmBN;  // two accumulator buffers
-    static constexpr int kBars = 2 * kStages + 5;     // full[], empty[], acc_full[2], acc_empty[2], drain
+    static constexpr int kMaxBN = NM == 2 ? 128 : 256;
+    static constexpr int kStages = 4;
+    static constexpr int kStageBytes = NM * kLmTileBytes + kMaxBN * kLmBK * 2;  // 48 KB
+    static constexpr int kTmemCols = 2 * NM * kMaxBN;  // two accumulator buffers: all 512 columns
+    static constexpr int kBars = 2 * kStages + 5;      // full[], empty[], acc_full[2], acc_empty[2], drain
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBars * 8 + 16;
 };
 
@@ -45,6 +47,7 @@ struct LmParams {
     int rows;        // rows of this launch (<= 256), starting at row0 of the hidden states
     int row0;
     int V;
+    int bn;          // vocabulary entries per tile
     int k_steps;     // H / 64
     float* part_v;   // [grid][256] the CTAs' best logits per row
     int32_t* part_t; // [grid][256] and the tokens that reach them
@@ -74,7 +77,8 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     auto sB = [&](int s) { return base + s * Cfg::kStageBytes + NM * kLmTileBytes; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = (prm.V + kLmBN - 1) / kLmBN;
+    const int bn = prm.bn;
+    const int n_tiles = (prm.V + bn - 1) / bn;
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) mbar_init(FULL(s), 1), mbar_init(EMPTY(s), 1);
         for (int b = 0; b < 2; ++b) mbar_init(ACC_FULL(b), 1), mbar_init(ACC_EMPTY(b), 4);
@@ -88,7 +92,7 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)*tmem_slot;
-    auto TM = [&](int buf, int t) { return tmem + (uint32_t)((buf * NM + t) * kLmBN); };
+    auto TM = [&](int buf, int t) { return tmem + (uint32_t)((buf * NM + t) * Cfg::kMaxBN); };
 
     if (warp == 0) {
         // ================= producer: hidden-state and weight tiles into the ring =================
@@ -100,10 +104,10 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
                     const int s = fill % S;
                     ok = mbar_wait(EMPTY(s), ((fill / S) & 1) ^ 1, dead);
                     if (!ok) break;
-                    mbar_expect_tx(FULL(s), Cfg::kStageBytes);
+                    mbar_expect_tx(FULL(s), NM * kLmTileBytes + bn * kLmBK * 2);
 #pragma unroll
                     for (int t = 0; t < NM; ++t) tma_load_2d(sA(s, t), &map_h, FULL(s), ks * kLmBK, prm.row0 + t * kLmBM);
-                    tma_load_2d(sB(s), &map_w, FULL(s), ks * kLmBK, tile * kLmBN);
+                    tma_load_2d(sB(s), &map_w, FULL(s), ks * kLmBK, tile * bn);
                 }
             *issued_s = fill;
         }
@@ -111,7 +115,7 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     } else if (warp == 1) {
         // ================= issuer: acc[t] = hidden tile t x weight tile^T over all K slices =================
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_bf16(kLmBM, kLmBN, false);
+            const uint32_t idesc = instr_desc_bf16(kLmBM, bn, false);
             int fill = 0, it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
@@ -151,11 +155,12 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int col0 = tile * kLmBN;
+            const int col0 = tile * bn;
 #pragma unroll
             for (int t = 0; t < NM; ++t) {
 #pragma unroll
-                for (int c = 0; c < kLmBN / 32; ++c) {
+                for (int c = 0; c < Cfg::kMaxBN / 32; ++c) {
+                    if (c * 32 >= bn) break;
                     uint32_t r[32];
                     tmem_ld32(TM(buf, t) + ((uint32_t)(q * 32) << 16) + c * 32, r);
                     tmem_wait_ld();
@@ -295,13 +300,13 @@ static LmEncodeTiledFn lm_encode_fn() {
     return fn;
 }
 
-// [rows, H] bf16 row-major, boxes of 128 rows x 64 elements (128 bytes), 128-byte swizzle, zero fill out of range
-static bool lm_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H) {
+// [rows, H] bf16 row-major, boxes of box_rows rows x 64 elements (128 bytes), 128-byte swizzle, zero fill out of range
+static bool lm_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H, int box_rows) {
     LmEncodeTiledFn fn = lm_encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)H, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)H * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kLmBK, (cuuint32_t)kLmBM};
+    const cuuint32_t box[2] = {(cuuint32_t)kLmBK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -321,7 +326,7 @@ static int lm_sm_count() {
 }
 
 static inline size_t lm_ws_layout(int V, char* base, float** part_v, int32_t** part_t) {
-    const size_t parts = (size_t)std::min(ceil_div(V, kLmBN), 1024);  // at most one CTA per tile, never more than this
+    const size_t parts = (size_t)std::min(ceil_div(V, 64), 1024);  // at most one CTA per tile (64 entries or more), never more than this
     size_t off = 0;
     if (part_v) *part_v = reinterpret_cast<float*>(base + off);
     off += round_up(parts * kLmRowsPerLaunch * sizeof(float), 256);
@@ -362,19 +367,31 @@ extern "C" s4c_status s4c_lm_head_greedy(const void* hidden, const void* weight,
     const size_t need = lm_ws_layout(V, nullptr, nullptr, nullptr);
     if (!workspace || workspace_bytes < need || !aligned256(workspace)) return S4C_ERR_WORKSPACE;
     lm_ws_layout(V, static_cast<char*>(workspace), &part_v, &part_t);
-    CUtensorMap map_h, map_w;
-    if (!lm_make_map(&map_h, hidden, (uint64_t)R, H) || !lm_make_map(&map_w, weight, (uint64_t)V, H)) return S4C_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
-    const int grid = std::min(std::min(ceil_div(V, kLmBN), lm_sm_count()), 1024);
+    const int sms = std::min(lm_sm_count(), 1024);
+    CUtensorMap map_h;
+    if (!lm_make_map(&map_h, hidden, (uint64_t)R, H, kLmBM)) return S4C_ERR_CUDA;
     // groups of up to 256 rows; each group streams the weights once
     for (int row0 = 0; row0 < R; row0 += kLmRowsPerLaunch) {
         LmParams prm;
         prm.rows = std::min(kLmRowsPerLaunch, R - row0), prm.row0 = row0, prm.V = V, prm.k_steps = H / kLmBK;
         prm.part_v = part_v, prm.part_t = part_t, prm.status = status;
+        // tile width: the one that costs the fewest (rounds of tiles over the CTAs) x (entries per tile)
+        prm.bn = 128;
+        if (prm.rows <= kLmBM) {
+            long long best = -1;
+            for (int bn = 64; bn <= LmCfg<1>::kMaxBN; bn += 32) {
+                const long long cost = (long long)ceil_div(ceil_div(V, bn), sms) * bn;
+                if (best < 0 || cost <= best) best = cost, prm.bn = bn;
+            }
+        }
+        const int grid = std::min(ceil_div(V, prm.bn), sms);
+        CUtensorMap map_w;
+        if (!lm_make_map(&map_w, weight, (uint64_t)V, H, prm.bn)) return S4C_ERR_CUDA;
         const s4c_status st = prm.rows > kLmBM ? lm_launch<2>(map_h, map_w, prm, grid, stream) : lm_launch<1>(map_h, map_w, prm, grid, stream);
         if (st != S4C_OK) return st;
         cudaLaunchAttribute pdl;
