@@ -42,6 +42,36 @@ def test_noalloc_entry_matches_the_workspace_entry_on_consecutive_calls():
         assert int(ref["status"].abs().sum()) == 0 and int(ref["accept_len"].min()) >= 0
 
 
+def test_noalloc_entry_leaves_device_memory_as_it_found_it():
+    # the property the entry point exists for: with the outputs preallocated, a call changes neither what the process has
+    # allocated nor what the device has free.  One problem on the cluster-statistics path, one on the segment path.
+    from dataclasses import replace
+
+    from paper_2506_14158_b200 import s4c
+
+    seg = replace(W.CONFIGS["c2"], name="noalloc_seg", config_id=81, B=4, T=128, V=32000, tree="random", max_tree_depth=8)
+    for cfg in (W.CONFIGS["c2"], seg):
+        assert s4c.tree_accept_workspace_bytes(cfg.B, cfg.T, cfg.V) <= s4c.NOALLOC_SCRATCH_BYTES
+        parent = W.make_trees(cfg)
+        x = W.make_accept_inputs(cfg, parent, 1.0, token_mode="topk")
+        args = (dev(x["logits"]), dev(x["draft_probs"]), dev(x["tokens"]), dev(parent), 1.0, dev(x["uniforms"]))
+        md = cfg.max_depth
+        ref = s4c.tree_accept(*args, max_depth=md)
+        i32 = dict(dtype=torch.int32, device="cuda")
+        out = dict(accept_len=torch.empty(cfg.B, **i32), path=torch.empty(cfg.B, md + 1, **i32),
+                   next_token=torch.empty(cfg.B, **i32), near_tie=torch.empty(cfg.B, cfg.T, dtype=torch.uint8, device="cuda"),
+                   status=torch.empty(cfg.B, **i32))
+        s4c.tree_accept_noalloc(*args, max_depth=md, out=out)  # warm-up: module loading, the symbol lookup
+        torch.cuda.synchronize()
+        held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+        for _ in range(3):
+            s4c.tree_accept_noalloc(*args, max_depth=md, out=out)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == held and torch.cuda.mem_get_info()[0] == free
+        for key in ("accept_len", "path", "next_token", "near_tie", "status"):
+            assert torch.equal(out[key], ref[key]), key
+
+
 def test_noalloc_entry_refuses_problems_beyond_its_built_in_scratch():
     from paper_2506_14158_b200 import s4c
 
