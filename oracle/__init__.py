@@ -17,6 +17,8 @@ Functions (array layouts are row-major numpy arrays):
 * :func:`lm_head_greedy`      -- Eq. 6 / Section 3.2: the LM head over the tree nodes' hidden states and the greedy choice
                                  (numpy, float64; a library matrix product is the step).
 * :func:`accept_greedy_tokens` -- the greedy walk when the target's choice per node is already known (plain Python).
+* :func:`qkv_rope`, :func:`rope_rotate` -- the verify layer's input side: q/k/v projections of the tree tokens, rotary
+                                 embedding at position cache_len + depth, k/v written into the caches' tree slots (numpy).
 """
 from __future__ import annotations
 
@@ -337,3 +339,64 @@ def accept_greedy_tokens(target_token, tokens, parent, n_nodes=None, max_depth=N
         path[b, :len(walked)] = walked
         nxt[b] = target_token[b, end]
     return dict(accept_len=a, path=path, next_token=nxt, status=status)
+
+
+def rope_rotate(x, pos, theta=10000.0):
+    """Rotary position embedding in the rotate-half form used by the LLaMA / Vicuna family (the paper's target models): for
+    a head vector x[0..d) at position pos, with x1 = x[:d/2], x2 = x[d/2:], angle_i = pos * theta**(-2i/d):
+    out[:d/2] = x1*cos - x2*sin, out[d/2:] = x2*cos + x1*sin.  float64.  x [..., d], pos broadcastable to x[..., 0]."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    assert d % 2 == 0
+    i = np.arange(d // 2, dtype=np.float64)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * theta ** (-2.0 * i / d)
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., : d // 2], x[..., d // 2:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def qkv_rope(x, w_qkv, cache_len, parent, Hq, Hkv, d, k_cache, v_cache, n_nodes=None, theta=10000.0):
+    """The verify layer's input side (Section 3.2: the target's forward pass over the T tree tokens; a decoder layer of the
+    LLaMA family): q, k, v = x W^T for every tree token (float64; a library matrix product is the step), rotary embedding of
+    q and k at position cache_len[b] + depth(node), q into a [B,Hq,T,d] array, k and v into the caches' tree slots
+    cache_len[b] + node (k_cache, v_cache [B,Hkv,C,d] float64 arrays, modified in place).
+
+    x [B,T,H]; w_qkv [(Hq+2*Hkv)*d, H]: the q heads' rows, then the k heads', then the v heads'.
+    Returns dict(q [B,Hq,T,d] float64 (rows of nodes >= n_nodes[b] and of flagged sequences are zero), status [B])."""
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(w_qkv, dtype=np.float64)
+    B, T, H = x.shape
+    assert w.shape == ((Hq + 2 * Hkv) * d, H)
+    parent = _i32(parent).reshape(B, T)
+    cache_len = _i32(cache_len)
+    C = k_cache.shape[2]
+    q = np.zeros((B, Hq, T, d))
+    status = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        n = T if n_nodes is None else int(n_nodes[b])
+        flags = 0
+        if n < 1 or n > T:
+            flags |= SEQ_BAD_PARENT
+        else:
+            for i in range(n):
+                p = int(parent[b, i])
+                if (i == 0 and p != -1) or (i > 0 and not (0 <= p < i)):
+                    flags |= SEQ_BAD_PARENT
+        L = int(cache_len[b])
+        if L < 0 or L + T > C:
+            flags |= SEQ_CAPACITY
+        status[b] = flags
+        if flags:
+            continue
+        depth = np.zeros(n, dtype=np.int64)
+        for i in range(1, n):
+            depth[i] = depth[parent[b, i]] + 1
+        proj = x[b, :n] @ w.T                                   # [n, (Hq+2Hkv)*d]
+        qh = proj[:, : Hq * d].reshape(n, Hq, d)
+        kh = proj[:, Hq * d: (Hq + Hkv) * d].reshape(n, Hkv, d)
+        vh = proj[:, (Hq + Hkv) * d:].reshape(n, Hkv, d)
+        pos = (L + depth)[:, None]
+        q[b, :, :n] = rope_rotate(qh, pos, theta).transpose(1, 0, 2)
+        k_cache[b, :, L:L + n] = rope_rotate(kh, pos, theta).transpose(1, 0, 2)
+        v_cache[b, :, L:L + n] = vh.transpose(1, 0, 2)
+    return dict(q=q, status=status)
