@@ -275,6 +275,33 @@ s4c_status s4c_tree_accept_tokens(const int32_t* target_token, const int32_t* to
                                   int32_t* path, int32_t* next_token, int32_t* status, s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * s4c_qkv_rope -- the input side of a decoder layer in the verify pass (Section 3.2: the target's
+ * forward pass over the T tree tokens; the paper's targets are LLaMA-family models): for every tree
+ * token the q, k, v projections of its hidden state (no bias), rotary embedding (rotate-half form)
+ * of q and k at position cache_len[b] + depth(node), q stored where s4c_tree_attention reads it and
+ * k, v stored straight into the caches' tree slots cache_len[b] + node:
+ *     [q | k | v](b, t) = x[b, t, :] . w_qkv^T          (bf16 inputs, float32 accumulation)
+ *     rot(u, p)[i]       = u[i] cos(p f_i) - u[i + d/2] sin(p f_i),
+ *     rot(u, p)[i + d/2] = u[i + d/2] cos(p f_i) + u[i] sin(p f_i),   f_i = rope_theta^(-2i/d), i < d/2
+ *     q_out[b, h, t, :] = rot(q_h, p);  k_cache[b, h, L_b + t, :] = rot(k_h, p);  v_cache[b, h, L_b + t, :] = v_h
+ *   x [B, T, H] bf16 (device); w_qkv [(Hq + 2 Hkv) d, H] bf16 (device): the q heads' rows, then the
+ *   k heads', then the v heads'; cache_len, parent, n_nodes as for s4c_tree_attention (node 0 is the
+ *   root, depth 0); q_out [B, Hq, T, d] bf16; k_cache, v_cache [B, Hkv, C, d] bf16 (only the tree
+ *   slots of the first n_nodes[b] nodes are written; everything else is left as it is);
+ *   d in {64, 128}; H a multiple of 64; rope_theta > 1 (10000 for the paper's models);
+ *   status [B] int32 (device) or NULL: S4C_SEQ_BAD_PARENT, S4C_SEQ_CAPACITY (L_b + T > C) -- such a
+ *   sequence is skipped (nothing of it is written) --, S4C_SEQ_TIMEOUT; workspace: at least
+ *   s4c_qkv_rope_workspace_bytes(B, T, d) bytes, 256-byte aligned.  All pointers 16-byte aligned.
+ * cos / sin are evaluated in float64 and applied in float32; results are rounded to bf16 once.
+ * ------------------------------------------------------------------------------------------ */
+size_t s4c_qkv_rope_workspace_bytes(int B, int T, int d);
+
+s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* parent,
+                        const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache, int B, int T, int H,
+                        int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status, void* workspace,
+                        size_t workspace_bytes, s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * s4c_tree_attention_paged, s4c_kv_compact_paged -- the same two operations (Section 3.2: tree-masked
  * attention of the verification pass; keeping the accepted tokens' K/V) on PAGED caches, the layout
  * serving systems keep their caches in.  The paper does not discuss cache layouts.

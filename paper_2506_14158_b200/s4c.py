@@ -24,7 +24,8 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
-           "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens"]
+           "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
+           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -78,6 +79,10 @@ def _load() -> ctypes.CDLL:
     lib.s4c_lm_head_greedy.argtypes = [vp, vp, i, i, i, i32p, vp, i32p, vp, sz, vp]
     lib.s4c_tree_accept_tokens.restype = i
     lib.s4c_tree_accept_tokens.argtypes = [i32p, i32p, i32p, i32p, i, i, i, i, i32p, i32p, i32p, i32p, vp]
+    lib.s4c_qkv_rope_workspace_bytes.restype = sz
+    lib.s4c_qkv_rope_workspace_bytes.argtypes = [i, i, i]
+    lib.s4c_qkv_rope.restype = i
+    lib.s4c_qkv_rope.argtypes = [vp, vp, i32p, i32p, i32p, vp, vp, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -444,3 +449,29 @@ def tree_accept_tokens(target_token, tokens, parent, V: int, n_nodes=None, max_d
     if rc:
         raise S4CError("s4c_tree_accept_tokens", rc)
     return dict(accept_len=accept_len, path=path, next_token=next_token, status=status)
+
+
+def qkv_rope_workspace_bytes(B, T, d) -> int:
+    return int(_lib.s4c_qkv_rope_workspace_bytes(B, T, d))
+
+
+def qkv_rope(x, w_qkv, cache_len, parent, q_out, k_cache, v_cache, n_nodes=None, rope_theta: float = 10000.0, status=None,
+             workspace=None, stream=None):
+    """s4c_qkv_rope: q/k/v projections of the tree tokens, rotary embedding at position cache_len + depth, q into
+    ``q_out`` [B,Hq,T,d], k and v into the caches' tree slots (``k_cache``, ``v_cache`` [B,Hkv,C,d], written in place)."""
+    B, T, H = x.shape
+    _, Hq, _, d = q_out.shape
+    _, Hkv, C, _ = k_cache.shape
+    dev = x.device
+    status = torch.empty(B, dtype=torch.int32, device=dev) if status is None else status
+    if workspace is None:
+        workspace = _workspace(int(_lib.s4c_qkv_rope_workspace_bytes(B, T, d)), dev, "qkv_rope")
+    bf = torch.bfloat16
+    rc = _lib.s4c_qkv_rope(_dev(x, bf, "x"), _dev(w_qkv, bf, "w_qkv"), _dev(cache_len, torch.int32, "cache_len"),
+                           _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"), _dev(q_out, bf, "q_out"),
+                           _dev(k_cache, bf, "k_cache"), _dev(v_cache, bf, "v_cache"), B, T, H, Hq, Hkv, d, C, float(rope_theta),
+                           _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+                           workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_qkv_rope", rc)
+    return dict(q=q_out, status=status)

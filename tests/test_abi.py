@@ -149,4 +149,18 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert tw(tgt=None) == 1 and tw(par=None) == 1 and tw(nt=None) == 1
     assert tw(T=129) == 2 and tw(V=0) == 2 and tw(md=128) == 2 and tw(B=-1) == 2
     assert tw(B=0) == 0
+    lib.s4c_qkv_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp, vp, sz, vp]
+    lib.s4c_qkv_rope_workspace_bytes.restype = sz
+    lib.s4c_qkv_rope_workspace_bytes.argtypes = [i, i, i]
+    qk = lambda **kw: lib.s4c_qkv_rope(*[kw.get(k, d) for k, d in [
+        ("x", P), ("w", P), ("cl", P), ("par", P), ("nn", None), ("q", P), ("k", P), ("v", P), ("B", 1), ("T", 26), ("H", 4096),
+        ("Hq", 32), ("Hkv", 8), ("d", 128), ("C", 2048), ("theta", 10000.0), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
+    assert qk(x=None) == 1 and qk(w=None) == 1 and qk(cl=None) == 1 and qk(k=None) == 1
+    assert qk(d=96) == 2 and qk(H=100) == 2 and qk(Hkv=5) == 2 and qk(T=129) == 2 and qk(C=10) == 2
+    assert qk(theta=1.0) == 2 and qk(theta=float("nan")) == 2
+    assert qk(q=P + 2) == 4
+    assert qk() == 5                                            # no workspace
+    assert qk(B=0) == 0
+    assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) % 256 == 0 and lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) > 0
+    assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 96) == 0
     assert b"workspace" in lib.s4c_status_string(5)
