@@ -322,6 +322,13 @@ def build_step(cfg, temperature, device, seed_shift=0, hint=True, paged=0):
     return step
 
 
+def replace_id(cfg, i):
+    """The same configuration with another input-stream id (another layer's random weights)."""
+    from dataclasses import replace
+
+    return replace(cfg, config_id=cfg.config_id * 37 + 11 + i)
+
+
 def time_graph(graph, iters, torch):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
@@ -428,6 +435,41 @@ def measure(cfg, args, device, rank, world, with_e2e):
         assert int(st.item()) == 0, "s4c_lm_head_greedy gave up a wait"
         lm = dict(ms=ms_lm, rows=cfg.B * cfg.T, V=cfg.V, H=cfg.hid)
         del wgt, ws
+    # the layer's input side: q/k/v projections + rotary embedding written into the attention layout and the cache's tree
+    # slots (timed alone, on buffers of its own: the step above takes q and the tree K/V as input)
+    qk = None
+    if cfg.dtype == "bf16" and not args.paged and cfg.d in (64, 128):
+        from paper_2506_14158_b200 import s4c
+        from paper_2506_14158_b200 import workloads as Wl
+
+        n_w = 4  # a few layers' weights in turn, so that the weights of a call do not sit in L2 from the call before
+        ws_qk = [Wl.make_qkv_weight(replace_id(cfg, i), device) for i in range(n_w)]
+        x_in = step.feat_in.contiguous()
+        q_buf = torch.empty_like(step.q[0])
+        kc = torch.zeros((cfg.B, cfg.Hkv, cfg.C, cfg.d), dtype=torch.bfloat16, device=device)
+        vc = torch.zeros_like(kc)
+        st_qk = torch.empty(cfg.B, dtype=torch.int32, device=device)
+        wsp = torch.empty(s4c.qkv_rope_workspace_bytes(cfg.B, cfg.T, cfg.d), dtype=torch.uint8, device=device)
+
+        def qkv_layers():
+            for w_l in ws_qk:
+                s4c.qkv_rope(x_in, w_l, step.cache_len0, step.parent, q_buf, kc, vc, step.n_nodes, 10000.0, st_qk, wsp)
+
+        sg = torch.cuda.Stream()
+        sg.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(sg):
+            qkv_layers()
+        torch.cuda.current_stream().wait_stream(sg)
+        torch.cuda.synchronize()
+        g_qk = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_qk):
+            qkv_layers()
+        for _ in range(3):
+            g_qk.replay()
+        ms_qk = time_graph(g_qk, K, torch) / n_w
+        assert int(st_qk.abs().sum().item()) == 0, "s4c_qkv_rope flagged a sequence"
+        qk = dict(ms=ms_qk, rows=cfg.B * cfg.T, N=(cfg.Hq + 2 * cfg.Hkv) * cfg.d, H=cfg.hid)
+        del ws_qk, kc, vc
     ms_e2e = 0.0
     if with_e2e:
         # end to end: per-step inputs from pinned host memory, decision back to the host, every step
@@ -448,7 +490,7 @@ def measure(cfg, args, device, rank, world, with_e2e):
         [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
         device=device)
     rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
-               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, qk=qk, ms_e2e=ms_e2e, accept_lens=accept_lens,
                clocks=clocks, K=K, Wm=Wm)
     return rec
 
@@ -500,6 +542,17 @@ def roofline_records(cfg, args, rec, pk):
             us=lm["ms"] * 1e3, bound="tensor" if tensor_bound else "hbm",
             tflops=flops / t * 1e-12, frac_of_tensor_peak=flops / t * 1e-12 / pk["bf16_tflops"],
             gbs=byts / t * 1e-9, frac_of_hbm_peak=byts / t * 1e-9 / pk["hbm_gbs"], flop_per_byte=flops / byts)
+    if rec.get("qk") is not None:
+        qk = rec["qk"]
+        breakdown["qkv_rope_one_layer_not_in_step"] = qk["ms"]
+        flops = 2.0 * qk["rows"] * qk["N"] * qk["H"]
+        byts = 2.0 * qk["N"] * qk["H"] + 2.0 * qk["rows"] * qk["H"] + 2.0 * qk["rows"] * qk["N"]  # weights, states, outputs (bf16)
+        t = qk["ms"] * 1e-3
+        roofline["qkv_rope"] = dict(
+            kernel="qkv_rope_kernel (+ the tree / rotary-table kernel in front)", rows=qk["rows"], N=qk["N"], H=qk["H"],
+            us=qk["ms"] * 1e3, bound="tensor" if flops / byts >= ridge else "hbm", tflops=flops / t * 1e-12,
+            frac_of_tensor_peak=flops / t * 1e-12 / pk["bf16_tflops"], gbs=byts / t * 1e-9,
+            frac_of_hbm_peak=byts / t * 1e-9 / pk["hbm_gbs"], flop_per_byte=flops / byts)
     return ab, step_hbm, roofline, breakdown
 
 

@@ -42,7 +42,10 @@ struct QkParams {
     int32_t* status;           // [B] (may be null)
 };
 
-// per sequence: tree and capacity checks, the rows' cache bases and the rotary table
+// Tree and capacity checks, the rows' cache bases and the rotary table.  grid (sequences, groups of kQkPrepNodes nodes):
+// every CTA of a sequence checks its tree (integer work on at most 128 nodes), then tabulates its own nodes -- the float64
+// power and sine / cosine are the expensive part and spread over the grid; a thread keeps one frequency.
+constexpr int kQkPrepNodes = 8;
 __global__ void __launch_bounds__(128)
 qkv_prep_kernel(const int32_t* __restrict__ cache_len, const int32_t* __restrict__ parent, const int32_t* __restrict__ n_nodes,
                 int T, int C, int d, double theta, int32_t* __restrict__ row_base, float2* __restrict__ rope,
@@ -53,21 +56,22 @@ qkv_prep_kernel(const int32_t* __restrict__ cache_len, const int32_t* __restrict
     __shared__ int flag;
     griddep_launch_dependents();
     const int b = blockIdx.x, tid = threadIdx.x;
+    const int t0 = blockIdx.y * kQkPrepNodes, t1 = min(T, t0 + kQkPrepNodes);
     const int n = n_nodes ? n_nodes[b] : T;
     const int L = cache_len[b];
     for (int i = tid; i < T; i += blockDim.x) par[i] = parent[(size_t)b * T + i];
     __syncthreads();
     int flags = build_ancestor_masks(par, n, T, anc, depth, &flag);
     if (L < 0 || L + T > C) flags |= S4C_SEQ_CAPACITY;
-    if (tid == 0 && status) status[b] = flags;
-    for (int t = tid; t < T; t += blockDim.x) row_base[(size_t)b * T + t] = (!flags && t < n) ? L : -1;
+    if (tid == 0 && blockIdx.y == 0 && status) status[b] = flags;
+    for (int t = t0 + tid; t < t1; t += blockDim.x) row_base[(size_t)b * T + t] = (!flags && t < n) ? L : -1;
     if (flags) return;
-    const int half = d / 2;
-    for (int idx = tid; idx < n * half; idx += blockDim.x) {
-        const int t = idx / half, i = idx - t * half;
-        const double ang = (double)(L + depth[t]) * pow(theta, -2.0 * (double)i / (double)d);
+    const int half = d / 2;  // 32 or 64: divides the block size, so a thread's pair index never changes
+    const int i = tid % half;
+    const double freq = pow(theta, -2.0 * (double)i / (double)d);
+    for (int t = t0 + tid / half; t < min(t1, n); t += blockDim.x / half) {
         double sn, cs;
-        sincos(ang, &sn, &cs);
+        sincos((double)(L + depth[t]) * freq, &sn, &cs);
         rope[((size_t)b * T + t) * half + i] = make_float2((float)cs, (float)sn);
     }
 }
@@ -109,13 +113,17 @@ qkv_rope_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     if (warp == 0) {
         // ================= producer =================
         if (lane == 0) {
+            // every CTA walks the K slices from a start of its own: the CTAs of a row tile all read the same state tiles,
+            // and in step they would all ask the same L2 lines at the same moment (the order of a sum's terms is free)
+            const int k0 = (int)((blockIdx.x * 7u + blockIdx.y * 3u) % (uint32_t)prm.k_steps);
             int fill = 0;
             for (; fill < prm.k_steps; ++fill) {
                 const int s = fill % S;
                 if (!mbar_wait(EMPTY(s), ((fill / S) & 1) ^ 1, dead)) break;
+                const int ks = fill + k0 < prm.k_steps ? fill + k0 : fill + k0 - prm.k_steps;
                 mbar_expect_tx(FULL(s), kQkBM * kQkBK * 2 + d * kQkBK * 2);
-                tma_load_2d(sX(s), &map_x, FULL(s), fill * kQkBK, mtile * kQkBM);
-                tma_load_2d(sW(s), &map_w, FULL(s), fill * kQkBK, head * d);
+                tma_load_2d(sX(s), &map_x, FULL(s), ks * kQkBK, mtile * kQkBM);
+                tma_load_2d(sW(s), &map_w, FULL(s), ks * kQkBK, head * d);
             }
             *issued_s = fill;
         }
@@ -286,7 +294,7 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
     CUtensorMap map_x, map_w;
     if (!qk_make_map(&map_x, x, (uint64_t)R, H, kQkBM) || !qk_make_map(&map_w, w_qkv, (uint64_t)heads * d, H, d)) return S4C_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    qkv_prep_kernel<<<B, 128, 0, stream>>>(cache_len, parent, n_nodes, T, C, d, (double)rope_theta, row_base, rope, status);
+    qkv_prep_kernel<<<dim3(B, ceil_div(T, kQkPrepNodes)), 128, 0, stream>>>(cache_len, parent, n_nodes, T, C, d, (double)rope_theta, row_base, rope, status);
     S4C_RETURN_IF_CUDA_ERROR();
     static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
     int dev = 0;

@@ -20,7 +20,7 @@ import numpy as np
 import torch
 
 BASE_SEED = 14158
-_STREAMS = {"tree": 0, "tokens": 1, "logits": 2, "noise": 3, "uniforms": 4, "q": 5, "kv": 6, "feat": 7, "lm_head": 8}
+_STREAMS = {"tree": 0, "tokens": 1, "logits": 2, "noise": 3, "uniforms": 4, "q": 5, "kv": 6, "feat": 7, "lm_head": 8, "qkv": 9}
 
 
 def stream_seed(config_id: int, stream: str, extra: int = 0) -> int:
@@ -220,6 +220,15 @@ def make_lm_head(cfg: VerifyConfig, device="cpu") -> torch.Tensor:
     g = torch.Generator(device=device)
     g.manual_seed(stream_seed(cfg.config_id, "lm_head"))
     w = torch.randn((cfg.V, cfg.hid), generator=g, dtype=torch.float32, device=device)
+    return (w * (1.0 / float(cfg.hid) ** 0.5)).to(torch.bfloat16)
+
+
+def make_qkv_weight(cfg: VerifyConfig, device="cpu") -> torch.Tensor:
+    """A decoder layer's stacked projection weight [(Hq + 2 Hkv) d, hid] in bfloat16 (q heads, then k, then v), entries
+    ~ N(0, 1/hid), random like the LM head's."""
+    g = torch.Generator(device=device)
+    g.manual_seed(stream_seed(cfg.config_id, "qkv"))
+    w = torch.randn(((cfg.Hq + 2 * cfg.Hkv) * cfg.d, cfg.hid), generator=g, dtype=torch.float32, device=device)
     return (w * (1.0 / float(cfg.hid) ** 0.5)).to(torch.bfloat16)
 
 
