@@ -400,3 +400,73 @@ def qkv_rope(x, w_qkv, cache_len, parent, Hq, Hkv, d, k_cache, v_cache, n_nodes=
         k_cache[b, :, L:L + n] = rope_rotate(kh, pos, theta).transpose(1, 0, 2)
         v_cache[b, :, L:L + n] = vh.transpose(1, 0, 2)
     return dict(q=q, status=status)
+
+
+def lm_head_topk(hidden, weight, k):
+    """The drafter's LM head followed by its top-k choice (Eq. 6 and Section 3.1: Argmax / top-2 of LM_head(f); Section 3.2:
+    the top-k alternatives of the verification tree): float64 logits as in :func:`lm_head_greedy`, then per row the k tokens
+    of greatest logit, greatest first, equal logits by lower token (a library sort, stable, is the step).
+
+    Returns dict(token [R, k] int32 (-1 beyond the vocabulary when k > V), logit [R, k] float64, logits [R, V])."""
+    h = np.asarray(hidden, dtype=np.float64)
+    w = np.asarray(weight, dtype=np.float64)
+    assert h.ndim == 2 and w.ndim == 2 and h.shape[1] == w.shape[1] and k >= 1
+    logits = h @ w.T
+    order = np.argsort(-logits, axis=1, kind="stable")[:, :k]
+    R, V = logits.shape
+    token = np.full((R, k), -1, dtype=np.int32)
+    logit = np.full((R, k), -np.inf)
+    token[:, : order.shape[1]] = order
+    logit[:, : order.shape[1]] = np.take_along_axis(logits, order, axis=1)
+    return dict(token=token, logit=logit, logits=logits)
+
+
+def build_tree_from_topk(topk, branching, root_token, T, cache_len=None):
+    """The continuous verification tree (Section 3.2 / Figure 3) from the drafter's ranked choices instead of its
+    distributions: the same shape as :func:`build_tree` (vertical first, then horizontal, cut at T nodes, breadth-first
+    numbering); child j of node n carries topk[b, n, j].  topk [B, T, k] int32 with k >= max(branching).
+    Returns dict(tokens, parent, position, n_nodes) like build_tree."""
+    topk = _i32(topk)
+    B, T_, k = topk.shape
+    assert T_ == T and k >= max(branching)
+    # the shape, in creation order: the vertical chain of first choices, then, depth by depth, every node of the previous
+    # depth is filled up to its branching factor, until T nodes exist
+    cpar, cdep, nchild = [-1], [0], [0]
+    tip = 0
+    for l in range(len(branching)):
+        if len(cpar) >= T:
+            break
+        cpar.append(tip), cdep.append(l + 1), nchild.append(0)
+        nchild[tip] += 1
+        tip = len(cpar) - 1
+    for l in range(1, len(branching) + 1):
+        for node in range(len(cpar)):
+            if cdep[node] != l - 1:
+                continue
+            while nchild[node] < branching[l - 1] and len(cpar) < T:
+                cpar.append(node), cdep.append(l), nchild.append(0)
+                nchild[node] += 1
+    # breadth-first numbering; a node's children keep their creation order (= rank order)
+    order, head = [0], 0
+    while head < len(order):
+        u = order[head]
+        head += 1
+        order.extend(c for c in range(len(cpar)) if cpar[c] == u)
+    newid = {c: i for i, c in enumerate(order)}
+    parent = [-1 if c == 0 else newid[cpar[c]] for c in order]
+    depth = [cdep[c] for c in order]
+    n = len(parent)
+    tokens = np.zeros((B, T), dtype=np.int32)
+    par = np.full((B, T), -1, dtype=np.int32)
+    pos = np.zeros((B, T), dtype=np.int32)
+    base = np.zeros(B, dtype=np.int64) if cache_len is None else np.asarray(cache_len, dtype=np.int64)
+    for b in range(B):
+        tokens[b, 0] = root_token[b]
+        rank = {}
+        for i in range(1, n):
+            j = rank.get(parent[i], 0)
+            rank[parent[i]] = j + 1
+            tokens[b, i] = topk[b, parent[i], j]
+        par[b, :n] = parent
+        pos[b, :n] = base[b] + np.asarray(depth)
+    return dict(tokens=tokens, parent=par, position=pos, n_nodes=np.full(B, n, dtype=np.int32))

@@ -111,3 +111,54 @@ def test_head_then_walk_equals_greedy_verification_on_materialised_logits():
     c = oracle.accept_greedy_tokens(choice, tokens, parent)
     for key in ("accept_len", "path", "next_token", "status"):
         np.testing.assert_array_equal(a[key], c[key], err_msg=key)
+
+
+# ----------------------------------------------------------------------------- top-k of the head, tree from ranked choices
+def test_topk_by_plain_loops_with_ties():
+    rng = np.random.default_rng(21)
+    R, V, H, k = 5, 11, 4, 4
+    hid = rng.integers(-2, 3, (R, H))
+    wgt = rng.integers(-2, 3, (V, H))          # few distinct integer logits: many ties
+    got = oracle.lm_head_topk(hid.astype(np.float32), wgt.astype(np.float32), k)
+    for r in range(R):
+        logit = [sum(int(hid[r, h]) * int(wgt[v, h]) for h in range(H)) for v in range(V)]
+        left = list(range(V))
+        for j in range(k):                      # selection by hand: greatest logit, the lowest token among equals
+            best = left[0]
+            for v in left:
+                if logit[v] > logit[best]:
+                    best = v
+            left.remove(best)
+            assert got["token"][r, j] == best and got["logit"][r, j] == logit[best]
+
+
+def test_topk_first_column_is_the_greedy_choice_and_rows_are_ranked():
+    rng = np.random.default_rng(22)
+    hid = rng.standard_normal((20, 16)).astype(np.float32)
+    wgt = rng.standard_normal((70, 16)).astype(np.float32)
+    top = oracle.lm_head_topk(hid, wgt, 6)
+    np.testing.assert_array_equal(top["token"][:, 0], oracle.lm_head_greedy(hid, wgt)["token"])
+    assert (np.diff(top["logit"], axis=1) <= 0).all()
+    for r in range(20):
+        assert len(set(top["token"][r])) == 6
+        rest = np.delete(top["logits"][r], top["token"][r])
+        assert rest.max() <= top["logit"][r, -1]            # nothing left out beats the last one kept
+    wide = oracle.lm_head_topk(hid[:2], wgt[:3], 5)         # k beyond the vocabulary: padded
+    assert (wide["token"][:, 3:] == -1).all() and sorted(wide["token"][0, :3]) == [0, 1, 2]
+
+
+@pytest.mark.parametrize("branching,T", [((4, 3, 2, 2, 1), 26), ((3, 2, 1), 15), ((2, 2, 2), 9), ((4, 3, 2, 2, 1), 7), ((5,), 3),
+                                         ((2, 3), 11), ((3,), 1)])
+def test_tree_from_ranked_choices_is_the_tree_from_distributions(branching, T):
+    # the separately pinned construction from draft distributions, fed with distributions whose ranking the choices are
+    rng = np.random.default_rng(len(branching) * 100 + T)
+    B, V = 3, 40
+    q = rng.random((B, T, V)).astype(np.float32)
+    q[0, :, 5] = q[0, :, 9]                                   # ties: the lower token ranks first on both routes
+    root = rng.integers(0, V, B).astype(np.int32)
+    cl = np.array([7, 0, 100], dtype=np.int32)
+    want = oracle.build_tree(q, branching, root, cl)
+    topk = np.argsort(-q, axis=2, kind="stable")[:, :, : max(branching)].astype(np.int32)
+    got = oracle.build_tree_from_topk(topk, branching, root, T, cl)
+    for key in ("tokens", "parent", "position", "n_nodes"):
+        np.testing.assert_array_equal(got[key], want[key], err_msg=key)
