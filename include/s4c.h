@@ -266,6 +266,27 @@ s4c_status s4c_tree_accept_filtered(const float* target_logits, const float* dra
  * ------------------------------------------------------------------------------------------ */
 size_t s4c_lm_head_greedy_workspace_bytes(int R, int V, int H);
 
+/* s4c_lm_head_topk -- the same contraction with the k best tokens per row instead of the best one: the
+ * drafter's LM head and its ranked choices (Section 3.1: the heads' Argmax / top-2 candidates; Section
+ * 3.2: the top-k alternatives of the verification tree).  token [R, k] int32 and logit [R, k] float
+ * (or NULL), best first, equal logits by lower token; entries beyond the vocabulary (k > V) or without
+ * a comparable logit are token -1, logit -inf.  1 <= k <= 8 (S4C_ERR_UNSUPPORTED above);
+ * s4c_lm_head_greedy is the case k = 1.  Workspace: s4c_lm_head_topk_workspace_bytes(R, V, H, k).
+ *
+ * s4c_tree_build_topk -- s4c_tree_build from ranked choices instead of distributions: the tree of
+ * Section 3.2 with the same shape and numbering; child j of node n carries topk[b, n, j]
+ * (topk [B, T, k] int32, device; k >= every branching factor).  No workspace.  With s4c_lm_head_topk
+ * in front, a drafting round needs no [B, T, V] array of probabilities at all. */
+size_t s4c_lm_head_topk_workspace_bytes(int R, int V, int H, int k);
+
+s4c_status s4c_lm_head_topk(const void* hidden, const void* weight, int R, int V, int H, int k, int32_t* token,
+                            float* logit, int32_t* status, void* workspace, size_t workspace_bytes,
+                            s4c_stream_t stream);
+
+s4c_status s4c_tree_build_topk(const int32_t* topk, int k, const int32_t* branching, int depth,
+                               const int32_t* root_token, const int32_t* cache_len, int B, int T, int32_t* tokens,
+                               int32_t* parent, int32_t* position, int32_t* n_nodes, s4c_stream_t stream);
+
 s4c_status s4c_lm_head_greedy(const void* hidden, const void* weight, int R, int V, int H, int32_t* token,
                               float* max_logit, int32_t* status, void* workspace, size_t workspace_bytes,
                               s4c_stream_t stream);

@@ -49,12 +49,12 @@ struct LmParams {
     int V;
     int bn;          // vocabulary entries per tile
     int k_steps;     // H / 64
-    float* part_v;   // [grid][256] the CTAs' best logits per row
-    int32_t* part_t; // [grid][256] and the tokens that reach them
+    float* part_v;   // [grid][256][KT] the CTAs' best logits per row, best first
+    int32_t* part_t; // [grid][256][KT] and their tokens
     int32_t* status; // one word (may be null): S4C_SEQ_TIMEOUT is OR-ed in when a wait was given up
 };
 
-template <int NM>
+template <int NM, int KT>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const LmParams prm) {
     using Cfg = LmCfg<NM>;
@@ -143,10 +143,12 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     } else {
         // ================= epilogue: running (maximum, first token) per row over this CTA's tiles =================
         const int q = warp & 3;  // the tensor-memory lanes this warp may read: 32 q .. 32 q + 31
-        float best_v[NM];
-        int best_t[NM];
+        float best_v[NM][KT];  // the KT best of the row so far, best first; equal logits: the lower token first
+        int best_t[NM][KT];
 #pragma unroll
-        for (int t = 0; t < NM; ++t) best_v[t] = -INFINITY, best_t[t] = INT_MAX;
+        for (int t = 0; t < NM; ++t)
+#pragma unroll
+            for (int j = 0; j < KT; ++j) best_v[t][j] = -INFINITY, best_t[t][j] = INT_MAX;
         int it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
@@ -168,7 +170,18 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
                     for (int j = 0; j < 32; ++j) {
                         const float v = __uint_as_float(r[j]);
                         const int col = col0 + c * 32 + j;
-                        if (col < prm.V && v > best_v[t]) best_v[t] = v, best_t[t] = col;  // ascending tokens: the first maximum stays
+                        // tokens ascend within a CTA and the comparison is strict: of equal logits the lower token stays ahead
+                        if (col < prm.V && v > best_v[t][KT - 1]) {
+                            best_v[t][KT - 1] = v, best_t[t][KT - 1] = col;
+#pragma unroll
+                            for (int j = KT - 1; j > 0; --j)
+                                if (best_v[t][j] > best_v[t][j - 1]) {
+                                    const float fv = best_v[t][j];
+                                    best_v[t][j] = best_v[t][j - 1], best_v[t][j - 1] = fv;
+                                    const int ft = best_t[t][j];
+                                    best_t[t][j] = best_t[t][j - 1], best_t[t][j - 1] = ft;
+                                }
+                        }
                     }
                 }
             }
@@ -179,8 +192,11 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
 #pragma unroll
         for (int t = 0; t < NM; ++t) {
             const int r = t * kLmBM + q * 32 + lane;
-            prm.part_v[(size_t)blockIdx.x * kLmRowsPerLaunch + r] = best_v[t];
-            prm.part_t[(size_t)blockIdx.x * kLmRowsPerLaunch + r] = best_t[t];
+#pragma unroll
+            for (int j = 0; j < KT; ++j) {
+                prm.part_v[((size_t)blockIdx.x * kLmRowsPerLaunch + r) * KT + j] = best_v[t][j];
+                prm.part_t[((size_t)blockIdx.x * kLmRowsPerLaunch + r) * KT + j] = best_t[t][j];
+            }
         }
     }
     griddep_launch_dependents();
@@ -208,21 +224,40 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     }
 }
 
-// per row: the best of the CTAs' candidates (greater logit, then lower token)
-__global__ void lm_head_merge_kernel(const float* __restrict__ part_v, const int32_t* __restrict__ part_t, int n_parts, int rows,
-                                     int32_t* __restrict__ token, float* __restrict__ max_logit) {
+// Per row: the k best of the CTAs' candidates, best first (greater logit, then lower token).  One warp per row; round j
+// takes the best candidate that ranks after round j-1's (the candidates' tokens are distinct).
+__global__ void __launch_bounds__(128)
+lm_head_merge_kernel(const float* __restrict__ part_v, const int32_t* __restrict__ part_t, int n_parts, int kt, int rows, int k,
+                     int32_t* __restrict__ token, float* __restrict__ logit) {
     griddep_wait();
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= rows) return;
-    float bv = -INFINITY;
-    int bt = INT_MAX;
-    for (int p = 0; p < n_parts; ++p) {
-        const float v = part_v[(size_t)p * kLmRowsPerLaunch + r];
-        const int t = part_t[(size_t)p * kLmRowsPerLaunch + r];
-        if (v > bv || (v == bv && t < bt)) bv = v, bt = t;
+    const int total = n_parts * kt;  // candidate c: CTA c / kt, rank c % kt
+    float pv = INFINITY;
+    int pt = -1;
+    for (int j = 0; j < k; ++j) {
+        float bv = -INFINITY;
+        int bt = INT_MAX;
+        for (int c = lane; c < total; c += 32) {
+            const size_t at = ((size_t)(c / kt) * kLmRowsPerLaunch + r) * kt + (c % kt);
+            const float v = part_v[at];
+            const int t = part_t[at];
+            const bool after = v < pv || (v == pv && t > pt);
+            if (t != INT_MAX && after && (v > bv || (v == bv && t < bt))) bv = v, bt = t;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
+            if (ov > bv || (ov == bv && ot < bt)) bv = ov, bt = ot;
+        }
+        pv = bv, pt = bt;
+        if (lane == 0) {
+            token[(size_t)r * k + j] = bt == INT_MAX ? -1 : bt;  // fewer than k comparable logits in the row (k > V, NaN)
+            if (logit) logit[(size_t)r * k + j] = bt == INT_MAX ? -INFINITY : bv;
+        }
+        if (bt == INT_MAX) pv = -INFINITY, pt = INT_MAX;  // nothing ranks after "none"
     }
-    token[r] = bt == INT_MAX ? -1 : bt;  // (no finite logit in the row: NaN everywhere)
-    if (max_logit) max_logit[r] = bv;
 }
 
 // ----------------------------------------------------------------------------- greedy walk on known choices
@@ -325,54 +360,57 @@ static int lm_sm_count() {
     return n;
 }
 
-static inline size_t lm_ws_layout(int V, char* base, float** part_v, int32_t** part_t) {
+static inline int lm_kt(int k) { return k <= 1 ? 1 : (k <= 4 ? 4 : 8); }  // candidates a thread keeps per row
+static inline size_t lm_ws_layout(int V, int k, char* base, float** part_v, int32_t** part_t) {
     const size_t parts = (size_t)std::min(ceil_div(V, 64), 1024);  // at most one CTA per tile (64 entries or more), never more than this
     size_t off = 0;
     if (part_v) *part_v = reinterpret_cast<float*>(base + off);
-    off += round_up(parts * kLmRowsPerLaunch * sizeof(float), 256);
+    off += round_up(parts * kLmRowsPerLaunch * lm_kt(k) * sizeof(float), 256);
     if (part_t) *part_t = reinterpret_cast<int32_t*>(base + off);
-    off += round_up(parts * kLmRowsPerLaunch * sizeof(int32_t), 256);
+    off += round_up(parts * kLmRowsPerLaunch * lm_kt(k) * sizeof(int32_t), 256);
     return off;
 }
 
-template <int NM>
+template <int NM, int KT>
 static s4c_status lm_launch(const CUtensorMap& map_h, const CUtensorMap& map_w, const LmParams& prm, int grid, cudaStream_t stream) {
     using Cfg = LmCfg<NM>;
-    if (cudaFuncSetAttribute(lm_head_greedy_kernel<NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+    if (cudaFuncSetAttribute(lm_head_greedy_kernel<NM, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
+        cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
-    lm_head_greedy_kernel<NM><<<grid, kLmThreads, Cfg::kSmemBytes, stream>>>(map_h, map_w, prm);
+    lm_head_greedy_kernel<NM, KT><<<grid, kLmThreads, Cfg::kSmemBytes, stream>>>(map_h, map_w, prm);
     S4C_RETURN_IF_CUDA_ERROR();
     return S4C_OK;
 }
 
 }  // namespace s4c
 
-extern "C" size_t s4c_lm_head_greedy_workspace_bytes(int R, int V, int H) {
-    if (R < 1 || V < 1 || H < 1) return 0;
-    return s4c::lm_ws_layout(V, nullptr, nullptr, nullptr);
+extern "C" size_t s4c_lm_head_topk_workspace_bytes(int R, int V, int H, int k) {
+    if (R < 1 || V < 1 || H < 1 || k < 1 || k > 8) return 0;
+    return s4c::lm_ws_layout(V, k, nullptr, nullptr, nullptr);
 }
 
-extern "C" s4c_status s4c_lm_head_greedy(const void* hidden, const void* weight, int R, int V, int H, int32_t* token,
-                                         float* max_logit, int32_t* status, void* workspace, size_t workspace_bytes,
-                                         s4c_stream_t stream_) {
+extern "C" s4c_status s4c_lm_head_topk(const void* hidden, const void* weight, int R, int V, int H, int k, int32_t* token,
+                                       float* logit, int32_t* status, void* workspace, size_t workspace_bytes,
+                                       s4c_stream_t stream_) {
     using namespace s4c;
     if (!hidden || !weight || !token) return S4C_ERR_NULL;
-    if (R < 0 || V < 1 || H < kLmBK || H % kLmBK != 0) return S4C_ERR_SHAPE;
+    if (R < 0 || V < 1 || H < kLmBK || H % kLmBK != 0 || k < 1) return S4C_ERR_SHAPE;
+    if (k > 8) return S4C_ERR_UNSUPPORTED;
     if (!aligned16(hidden) || !aligned16(weight)) return S4C_ERR_ALIGN;
     if (R == 0) return S4C_OK;
     float* part_v;
     int32_t* part_t;
-    const size_t need = lm_ws_layout(V, nullptr, nullptr, nullptr);
+    const size_t need = lm_ws_layout(V, k, nullptr, nullptr, nullptr);
     if (!workspace || workspace_bytes < need || !aligned256(workspace)) return S4C_ERR_WORKSPACE;
-    lm_ws_layout(V, static_cast<char*>(workspace), &part_v, &part_t);
+    lm_ws_layout(V, k, static_cast<char*>(workspace), &part_v, &part_t);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
-    const int sms = std::min(lm_sm_count(), 1024);
+    const int sms = std::min(lm_sm_count(), 1024), kt = lm_kt(k);
     CUtensorMap map_h;
     if (!lm_make_map(&map_h, hidden, (uint64_t)R, H, kLmBM)) return S4C_ERR_CUDA;
     // groups of up to 256 rows; each group streams the weights once
@@ -392,21 +430,32 @@ extern "C" s4c_status s4c_lm_head_greedy(const void* hidden, const void* weight,
         const int grid = std::min(ceil_div(V, prm.bn), sms);
         CUtensorMap map_w;
         if (!lm_make_map(&map_w, weight, (uint64_t)V, H, prm.bn)) return S4C_ERR_CUDA;
-        const s4c_status st = prm.rows > kLmBM ? lm_launch<2>(map_h, map_w, prm, grid, stream) : lm_launch<1>(map_h, map_w, prm, grid, stream);
+        const bool two = prm.rows > kLmBM;
+        const s4c_status st = kt == 1   ? (two ? lm_launch<2, 1>(map_h, map_w, prm, grid, stream) : lm_launch<1, 1>(map_h, map_w, prm, grid, stream))
+                              : kt == 4 ? (two ? lm_launch<2, 4>(map_h, map_w, prm, grid, stream) : lm_launch<1, 4>(map_h, map_w, prm, grid, stream))
+                                        : (two ? lm_launch<2, 8>(map_h, map_w, prm, grid, stream) : lm_launch<1, 8>(map_h, map_w, prm, grid, stream));
         if (st != S4C_OK) return st;
         cudaLaunchAttribute pdl;
         pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
         pdl.val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t cfg = {};
         cfg.stream = stream, cfg.attrs = &pdl, cfg.numAttrs = 1;
-        cfg.gridDim = dim3(ceil_div(prm.rows, 128), 1, 1), cfg.blockDim = dim3(128, 1, 1);
-        if (cudaLaunchKernelEx(&cfg, lm_head_merge_kernel, (const float*)part_v, (const int32_t*)part_t, grid, prm.rows,
-                               token + row0, max_logit ? max_logit + row0 : (float*)nullptr) != cudaSuccess) {
+        cfg.gridDim = dim3(ceil_div(prm.rows, 4), 1, 1), cfg.blockDim = dim3(128, 1, 1);  // a warp per row
+        if (cudaLaunchKernelEx(&cfg, lm_head_merge_kernel, (const float*)part_v, (const int32_t*)part_t, grid, kt, prm.rows, k,
+                               token + (size_t)row0 * k, logit ? logit + (size_t)row0 * k : (float*)nullptr) != cudaSuccess) {
             cudaGetLastError();
             return S4C_ERR_CUDA;
         }
     }
     return S4C_OK;
+}
+
+extern "C" size_t s4c_lm_head_greedy_workspace_bytes(int R, int V, int H) { return s4c_lm_head_topk_workspace_bytes(R, V, H, 1); }
+
+extern "C" s4c_status s4c_lm_head_greedy(const void* hidden, const void* weight, int R, int V, int H, int32_t* token,
+                                         float* max_logit, int32_t* status, void* workspace, size_t workspace_bytes,
+                                         s4c_stream_t stream_) {
+    return s4c_lm_head_topk(hidden, weight, R, V, H, 1, token, max_logit, status, workspace, workspace_bytes, stream_);
 }
 
 extern "C" s4c_status s4c_tree_accept_tokens(const int32_t* target_token, const int32_t* tokens, const int32_t* parent,

@@ -207,6 +207,30 @@ static void lay_out_tree(const int32_t* branching, int D, int T, TreeShape* shap
         if (shape->n_child[i]) shape->expanded[shape->n_expanded++] = (uint8_t)i;
 }
 
+// The same tree from the drafter's ranked choices (topk[b, n, j] = the j-th choice after node n) instead of its
+// distributions: nothing to select, the children copy their tokens.
+__global__ void __launch_bounds__(128)
+tree_emit_topk_kernel(const int32_t* __restrict__ topk, int k, const __grid_constant__ TreeShape shape,
+                      const int32_t* __restrict__ root_token, const int32_t* __restrict__ cache_len, int T,
+                      int32_t* __restrict__ tokens, int32_t* __restrict__ parent, int32_t* __restrict__ position,
+                      int32_t* __restrict__ n_nodes) {
+    const int b = blockIdx.x;
+    const int base = cache_len ? cache_len[b] : 0;
+    for (int i = threadIdx.x; i < T; i += blockDim.x) {
+        const bool used = i < shape.n;
+        const int p = used ? (int)shape.parent[i] : -1;
+        parent[(size_t)b * T + i] = p;
+        position[(size_t)b * T + i] = used ? base + (int)shape.depth[i] : 0;
+        int tok = 0;
+        if (i == 0)
+            tok = root_token[b];
+        else if (used)
+            tok = topk[((size_t)b * T + p) * k + (i - (int)shape.first_child[p])];  // siblings are contiguous, in rank order
+        tokens[(size_t)b * T + i] = tok;
+    }
+    if (threadIdx.x == 0) n_nodes[b] = shape.n;
+}
+
 static inline int tb_segments(int V) { return ceil_div(V, kTbSeg); }
 
 }  // namespace s4c
@@ -248,6 +272,23 @@ extern "C" s4c_status s4c_tree_build(const float* draft_probs, const int32_t* br
     }
     tree_emit_kernel<<<B, kEmitThreads, 0, stream>>>(cand, shape, root_token, cache_len, T, segs, max_branch, tokens, parent, position,
                                             n_nodes);
+    S4C_RETURN_IF_CUDA_ERROR();
+    return S4C_OK;
+}
+
+extern "C" s4c_status s4c_tree_build_topk(const int32_t* topk, int k, const int32_t* branching, int depth,
+                                          const int32_t* root_token, const int32_t* cache_len, int B, int T, int32_t* tokens,
+                                          int32_t* parent, int32_t* position, int32_t* n_nodes, s4c_stream_t stream_) {
+    using namespace s4c;
+    if (!topk || !root_token || !tokens || !parent || !position || !n_nodes || (depth > 0 && !branching)) return S4C_ERR_NULL;
+    if (B < 0 || B > 65535 || T < 1 || T > S4C_MAX_T || k < 1 || depth < 0 || depth >= S4C_MAX_T) return S4C_ERR_SHAPE;
+    for (int l = 0; l < depth; ++l)
+        if (branching[l] < 1 || branching[l] > k) return S4C_ERR_SHAPE;  // a node cannot have more children than ranked choices
+    if (B == 0) return S4C_OK;
+    TreeShape shape;
+    lay_out_tree(branching, depth, T, &shape);
+    tree_emit_topk_kernel<<<B, 128, 0, static_cast<cudaStream_t>(stream_)>>>(topk, k, shape, root_token, cache_len, T, tokens, parent,
+                                                                            position, n_nodes);
     S4C_RETURN_IF_CUDA_ERROR();
     return S4C_OK;
 }

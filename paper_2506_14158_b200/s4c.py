@@ -25,7 +25,8 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
            "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
-           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope"]
+           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
+           "s4c_tree_build_topk"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -83,6 +84,12 @@ def _load() -> ctypes.CDLL:
     lib.s4c_qkv_rope_workspace_bytes.argtypes = [i, i, i]
     lib.s4c_qkv_rope.restype = i
     lib.s4c_qkv_rope.argtypes = [vp, vp, i32p, i32p, i32p, vp, vp, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_lm_head_topk_workspace_bytes.restype = sz
+    lib.s4c_lm_head_topk_workspace_bytes.argtypes = [i, i, i, i]
+    lib.s4c_lm_head_topk.restype = i
+    lib.s4c_lm_head_topk.argtypes = [vp, vp, i, i, i, i, i32p, vp, i32p, vp, sz, vp]
+    lib.s4c_tree_build_topk.restype = i
+    lib.s4c_tree_build_topk.argtypes = [i32p, i, vp, i, i32p, i32p, i, i, i32p, i32p, i32p, i32p, vp]
     lib.s4c_launch_floor.restype = i
     lib.s4c_launch_floor.argtypes = [i, i, i, i, i, i, i, i32p, i32p, vp]
     return lib
@@ -475,3 +482,46 @@ def qkv_rope(x, w_qkv, cache_len, parent, q_out, k_cache, v_cache, n_nodes=None,
     if rc:
         raise S4CError("s4c_qkv_rope", rc)
     return dict(q=q_out, status=status)
+
+
+def lm_head_topk_workspace_bytes(R, V, H, k) -> int:
+    return int(_lib.s4c_lm_head_topk_workspace_bytes(R, V, H, k))
+
+
+def lm_head_topk(hidden, weight, k: int, token=None, logit=None, status=None, workspace=None, stream=None):
+    """s4c_lm_head_topk: the k best tokens per row of hidden @ weight^T, best first (ties to the lower token)."""
+    R, H = hidden.shape
+    V = weight.shape[0]
+    dev = hidden.device
+    token = torch.empty(R, k, dtype=torch.int32, device=dev) if token is None else token
+    logit = torch.empty(R, k, dtype=torch.float32, device=dev) if logit is None else logit
+    status = torch.zeros(1, dtype=torch.int32, device=dev) if status is None else status
+    if workspace is None:
+        workspace = _workspace(int(_lib.s4c_lm_head_topk_workspace_bytes(R, V, H, int(k))), dev, "lm_head")
+    rc = _lib.s4c_lm_head_topk(_dev(hidden, torch.bfloat16, "hidden"), _dev(weight, torch.bfloat16, "weight"), R, V, H, int(k),
+                               _dev(token, torch.int32, "token"), _dev(logit, torch.float32, "logit"),
+                               _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+                               0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_lm_head_topk", rc)
+    return dict(token=token, logit=logit, status=status)
+
+
+def tree_build_topk(topk, branching, root_token, cache_len=None, tokens=None, parent=None, position=None, n_nodes=None,
+                    stream=None):
+    """s4c_tree_build_topk: the verification tree from ranked choices topk [B,T,k] int32 (child j of node n = topk[b,n,j])."""
+    B, T, k = topk.shape
+    dev = topk.device
+    i32 = dict(dtype=torch.int32, device=dev)
+    tokens = torch.empty(B, T, **i32) if tokens is None else tokens
+    parent = torch.empty(B, T, **i32) if parent is None else parent
+    position = torch.empty(B, T, **i32) if position is None else position
+    n_nodes = torch.empty(B, **i32) if n_nodes is None else n_nodes
+    br = (ctypes.c_int32 * max(1, len(branching)))(*[int(x) for x in branching])
+    rc = _lib.s4c_tree_build_topk(_dev(topk, torch.int32, "topk"), k, ctypes.cast(br, ctypes.c_void_p), len(branching),
+                                  _dev(root_token, torch.int32, "root_token"), _dev(cache_len, torch.int32, "cache_len"), B, T,
+                                  _dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"),
+                                  _dev(position, torch.int32, "position"), _dev(n_nodes, torch.int32, "n_nodes"), _stream(stream))
+    if rc:
+        raise S4CError("s4c_tree_build_topk", rc)
+    return dict(tokens=tokens, parent=parent, position=position, n_nodes=n_nodes)

@@ -163,4 +163,22 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert qk(B=0) == 0
     assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) % 256 == 0 and lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) > 0
     assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 96) == 0
+    lib.s4c_lm_head_topk.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp, sz, vp]
+    lib.s4c_lm_head_topk_workspace_bytes.restype = sz
+    lib.s4c_lm_head_topk_workspace_bytes.argtypes = [i, i, i, i]
+    tk = lambda **kw: lib.s4c_lm_head_topk(*[kw.get(k, d) for k, d in [
+        ("h", P), ("w", P), ("R", 26), ("V", 32000), ("H", 4096), ("k", 4), ("tok", P), ("lg", None), ("st", None), ("ws", None),
+        ("wsb", 0), ("s", None)]])
+    assert tk(h=None) == 1 and tk(tok=None) == 1 and tk(k=0) == 2 and tk(H=96) == 2
+    assert tk(k=9) == 6                                         # S4C_ERR_UNSUPPORTED: at most 8 ranked choices
+    assert tk() == 5 and tk(R=0) == 0
+    assert lib.s4c_lm_head_topk_workspace_bytes(26, 32000, 4096, 8) > lib.s4c_lm_head_topk_workspace_bytes(26, 32000, 4096, 1) > 0
+    assert lib.s4c_lm_head_topk_workspace_bytes(26, 32000, 4096, 9) == 0
+    lib.s4c_tree_build_topk.argtypes = [vp, i, vp, i, vp, vp, i, i, vp, vp, vp, vp, vp]
+    tbk = lambda **kw: lib.s4c_tree_build_topk(*[kw.get(k, d) for k, d in [
+        ("topk", P), ("k", 4), ("br", ctypes.cast(br, vp)), ("D", 3), ("root", P), ("cl", None), ("B", 1), ("T", 26), ("tok", P),
+        ("par", P), ("pos", P), ("nn", P), ("s", None)]])
+    assert tbk(topk=None) == 1 and tbk(nn=None) == 1 and tbk(br=None) == 1
+    assert tbk(T=129) == 2 and tbk(k=0) == 2 and tbk(k=3) == 2  # k = 3: fewer ranked choices than the 4 children of the root
+    assert tbk(B=0) == 0
     assert b"workspace" in lib.s4c_status_string(5)

@@ -181,3 +181,85 @@ def test_head_then_walk_equals_greedy_acceptance_on_materialised_logits():
     for key in ("accept_len", "path", "next_token", "status"):
         np.testing.assert_array_equal(got[key].cpu().numpy(), want[key], err_msg=key)
     assert want["accept_len"].max() >= 2
+
+
+# ----------------------------------------------------------------------------- the k best per row; the tree from them
+def _run_topk(hid, wgt, k):
+    from paper_2506_14158_b200 import s4c
+
+    R, H = hid.shape
+    V = wgt.shape[0]
+    g = dict(token=Guarded((R, k), torch.int32, fill=-9), logit=Guarded((R, k), torch.float32, fill=-9.0),
+             status=Guarded((1,), torch.int32, fill=-9),
+             workspace=Guarded((max(256, s4c.lm_head_topk_workspace_bytes(R, V, H, k)),), torch.uint8, fill=0xCD))
+    s4c.lm_head_topk(hid.cuda(), wgt.cuda(), k, token=g["token"].t, logit=g["logit"].t, status=g["status"].t,
+                     workspace=g["workspace"].t)
+    torch.cuda.synchronize()
+    for name, buf in g.items():
+        buf.check("s4c_lm_head_topk " + name)
+    assert int(g["status"].t.item()) == 0
+    return g["token"].t.cpu().numpy(), g["logit"].t.cpu().numpy()
+
+
+@pytest.mark.parametrize("R,V,H,k", [(26, 1000, 128, 4), (130, 4099, 256, 8), (7, 333, 64, 3), (256, 32000, 192, 2),
+                                     (300, 777, 64, 5), (3, 6, 64, 8)])
+def test_topk_against_the_oracle(R, V, H, k):
+    rng = np.random.default_rng(R + V + k)
+    hid, wgt = _bf16(rng.standard_normal((R, H))), _bf16(rng.standard_normal((V, H)) * 0.5)
+    tok, lg = _run_topk(hid, wgt, k)
+    ref = oracle.lm_head_topk(hid.float().numpy(), wgt.float().numpy(), k)
+    h, w = hid.float().numpy().astype(np.float64), wgt.float().numpy().astype(np.float64)
+    bound = 4.0 * np.sqrt(H) * 2.0 ** -24 * np.linalg.norm(h, axis=1) * np.linalg.norm(w, axis=1).max() + 1e-30
+    kk = min(k, V)
+    assert (tok[:, kk:] == -1).all() and np.isneginf(lg[:, kk:]).all()
+    srt = -np.sort(-ref["logits"], axis=1)[:, : kk + 1]
+    for r in range(R):
+        assert len(set(tok[r, :kk])) == kk                                        # distinct tokens
+        mine = ref["logits"][r, tok[r, :kk]]                                      # their oracle logits
+        assert (np.abs(lg[r, :kk] - mine) <= bound[r]).all()                      # reported logits are theirs
+        assert (np.abs(mine - ref["logit"][r, :kk]) <= bound[r]).all()            # rank j holds a token as good as the oracle's
+        gaps = -np.diff(srt[r])                                                   # where neighbours are clearly apart ...
+        clear = np.ones(kk, dtype=bool)
+        clear[: len(gaps)] &= gaps[:kk] > 2 * bound[r]
+        clear[1:] &= gaps[: kk - 1] > 2 * bound[r]
+        np.testing.assert_array_equal(tok[r, :kk][clear], ref["token"][r, :kk][clear])   # ... the token is unique: equal
+
+
+def test_topk_ties_follow_the_token_order_across_tiles_and_ctas():
+    rng = np.random.default_rng(41)
+    R, V, H, k = 40, 128 * 200, 64, 8
+    hid = _bf16(rng.integers(-2, 3, (R, H)))
+    base = rng.integers(-2, 3, (30, H)).astype(np.float32)
+    wgt = _bf16(base[rng.integers(0, 30, V)])          # 30 distinct rows all over the vocabulary: exact integer logits, many ties
+    tok, lg = _run_topk(hid, wgt, k)
+    ref = oracle.lm_head_topk(hid.float().numpy(), wgt.float().numpy(), k)
+    np.testing.assert_array_equal(tok, ref["token"])
+    np.testing.assert_array_equal(lg, ref["logit"])
+
+
+def test_drafting_round_without_a_vocabulary_sized_array():
+    # drafter states -> ranked choices -> tree, against the oracle's head and its tree from ranked choices; then the
+    # tree from ranked choices equals the library's own tree from the distributions those choices rank
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(46)   # (a seed without a near tie among the first k + 1 logits of any row)
+    cfg = W.CONFIGS["c2"]
+    B, T, V, H = 3, cfg.T, 5000, 256
+    hid, wgt = _bf16(rng.standard_normal((B * T, H))), _bf16(rng.standard_normal((V, H)) * 0.3)
+    k = max(cfg.branching)
+    top = s4c.lm_head_topk(hid.cuda(), wgt.cuda(), k)
+    root = rng.integers(0, V, B).astype(np.int32)
+    cl = np.array([5, 0, 77], dtype=np.int32)
+    tree = s4c.tree_build_topk(top["token"].view(B, T, k), cfg.branching, dev(root), dev(cl))
+    torch.cuda.synchronize()
+    ref_top = oracle.lm_head_topk(hid.float().numpy(), wgt.float().numpy(), k)
+    srt = -np.sort(-ref_top["logits"], axis=1)[:, : k + 1]
+    assert (-np.diff(srt, axis=1) > 1e-3).all()      # this seed has no near tie among the first k + 1: the choices are unique
+    want = oracle.build_tree_from_topk(ref_top["token"].reshape(B, T, k), cfg.branching, root, T, cl)
+    for key in ("tokens", "parent", "position", "n_nodes"):
+        np.testing.assert_array_equal(tree[key].cpu().numpy(), want[key], err_msg=key)
+    probs = torch.softmax(torch.from_numpy(ref_top["logits"]).float(), dim=1).view(B, T, V).contiguous()
+    lib = s4c.tree_build(probs.cuda(), cfg.branching, dev(root), dev(cl))
+    torch.cuda.synchronize()
+    for key in ("tokens", "parent", "position", "n_nodes"):
+        np.testing.assert_array_equal(tree[key].cpu().numpy(), lib[key].cpu().numpy(), err_msg=key)
