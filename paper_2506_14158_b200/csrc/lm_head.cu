@@ -166,23 +166,32 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
                     uint32_t r[32];
                     tmem_ld32(TM(buf, t) + ((uint32_t)(q * 32) << 16) + c * 32, r);
                     tmem_wait_ld();
+                    // (once a row's list is full, most runs of 32 logits hold nothing that beats its last entry: one
+                    // maximum over the run settles that; NaN and columns past the vocabulary never enter)
+                    float run_max = -INFINITY;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float v = __uint_as_float(r[j]);
-                        const int col = col0 + c * 32 + j;
-                        // tokens ascend within a CTA and the comparison is strict: of equal logits the lower token stays ahead
-                        if (col < prm.V && v > best_v[t][KT - 1]) {
-                            best_v[t][KT - 1] = v, best_t[t][KT - 1] = col;
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + c * 32 + j < prm.V) run_max = fmaxf(run_max, __uint_as_float(r[j]));
+                    if (run_max > best_v[t][KT - 1]) {
 #pragma unroll
-                            for (int j = KT - 1; j > 0; --j)
-                                if (best_v[t][j] > best_v[t][j - 1]) {
-                                    const float fv = best_v[t][j];
-                                    best_v[t][j] = best_v[t][j - 1], best_v[t][j - 1] = fv;
-                                    const int ft = best_t[t][j];
-                                    best_t[t][j] = best_t[t][j - 1], best_t[t][j - 1] = ft;
-                                }
+                        for (int j = 0; j < 32; ++j) {
+                            const float v = __uint_as_float(r[j]);
+                            const int col = col0 + c * 32 + j;
+                            // tokens ascend within a CTA and the comparison is strict: of equal logits the lower token stays ahead
+                            if (col < prm.V && v > best_v[t][KT - 1]) {
+                                best_v[t][KT - 1] = v, best_t[t][KT - 1] = col;
+#pragma unroll
+                                for (int jj = KT - 1; jj > 0; --jj)
+                                    if (best_v[t][jj] > best_v[t][jj - 1]) {
+                                        const float fv = best_v[t][jj];
+                                        best_v[t][jj] = best_v[t][jj - 1], best_v[t][jj - 1] = fv;
+                                        const int ft = best_t[t][jj];
+                                        best_t[t][jj] = best_t[t][jj - 1], best_t[t][jj - 1] = ft;
+                                    }
+                            }
                         }
                     }
+                    __syncwarp();  // the lanes took different ways through the run; the next tensor-memory load is warp-wide
                 }
             }
             tc_fence_before();
