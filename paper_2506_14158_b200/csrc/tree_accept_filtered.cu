@@ -205,6 +205,68 @@ __device__ __forceinline__ int select_from_pool(SpanShared& sh, int n_pool, floa
     return min(k, n_cand);
 }
 
+// The exact path for a piece (batches batch0 .. batch1-1 of one row) that the streaming selection cannot serve: every
+// thread sorts its 16 entries of a batch, warps merge their lanes' lists head by head, one warp merges the warps' lists
+// with the k best so far.  Its own function, not inlined: it needs twice the registers of the streaming loop and runs
+// only for tie-heavy or masked pieces.  Leaves the piece's k best in sh.sorted; returns the thread's share of the draft
+// mass in *qs and whether the piece holds a NaN or +Inf.
+template <bool VEC>
+__device__ __noinline__ bool exact_piece(SpanShared& sh, const float* __restrict__ row, const float* __restrict__ qrow, int V,
+                                         int k, int batch0, int batch1, double* qs_out) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    double qs = 0.0;
+    bool unusable = false;
+    FCand* best = sh.wlist[kFsThreads / 32];
+    for (int r = tid; r < kMaxTopK; r += kFsThreads) best[r].x = -INFINITY, best[r].tok = INT_MAX;
+    for (int batch = batch0; batch < batch1 && !unusable; ++batch) {
+        const int s0 = batch * kFsSeg;
+        float x[kFsElems];
+        int e[kFsElems];
+        bool bad_here = false;
+#pragma unroll
+        for (int i = 0; i < kFsElems; ++i) {
+            const int tok = VEC ? s0 + ((i >> 2) * kFsThreads + tid) * 4 + (i & 3) : s0 + i * kFsThreads + tid;
+            const bool in = tok < V;
+            x[i] = in ? __ldg(row + tok) : -INFINITY;
+            qs += in ? (double)__ldg(qrow + tok) : 0.0;
+            e[i] = in ? tok : INT_MAX;  // slots past the row rank last
+            bad_here = bad_here || !(x[i] < INFINITY);
+        }
+        // sort the thread's 16 entries, best first (bitonic network on (logit, token) pairs; the order is total)
+#pragma unroll
+        for (int size = 2; size <= kFsElems; size <<= 1)
+#pragma unroll
+            for (int stride = size >> 1; stride > 0; stride >>= 1)
+#pragma unroll
+                for (int i = 0; i < kFsElems; ++i) {
+                    const int j = i ^ stride;
+                    if (j > i) {
+                        const bool up = (i & size) == 0;  // this block sorts best-first, its sibling worst-first
+                        const bool swap = up ? f_before(x[j], e[j], x[i], e[i]) : f_before(x[i], e[i], x[j], e[j]);
+                        if (swap) {
+                            const float tx = x[i];
+                            x[i] = x[j], x[j] = tx;
+                            const int te = e[i];
+                            e[i] = e[j], e[j] = te;
+                        }
+                    }
+                }
+#pragma unroll
+        for (int i = 0; i < kFsElems; ++i) sh.lists[i][tid].x = x[i], sh.lists[i][tid].tok = e[i];
+        __syncwarp();
+        merge_heads(&sh.lists[0][warp * 32], 32, kFsElems, kFsThreads, 1, k, sh.wlist[warp]);
+        unusable = __syncthreads_or(bad_here);
+        if (warp == 0) {  // nine lists: the warps' and the best so far; the result replaces the best so far
+            merge_heads(&sh.wlist[0][0], kFsThreads / 32 + 1, k, 1, kMaxTopK, k, sh.sorted);
+            __syncwarp();
+            for (int r = lane; r < k; r += 32) best[r] = sh.sorted[r];
+        }
+        __syncthreads();
+    }
+    *qs_out = qs;
+    return unusable;
+}
+
 // The rows' batches (4096 entries each) form one long list, cut into equal runs of `per` batches: one CTA per run, all
 // CTAs resident at once, every CTA with the same amount to read.  A run that crosses from one row into the next ends a
 // piece and starts another; a row is covered by at most pmax pieces.  For every piece: the k best logits (sorted) and the
@@ -416,54 +478,9 @@ filter_span_kernel(const float* __restrict__ logits, const float* __restrict__ d
             }
         }
         if (exact_path) {
-            // ---- the exact path, from the start of the span: every thread sorts its 16 entries of a batch, warps merge
-            // their lanes' lists head by head, one warp merges the warps' lists and the k best so far
             __syncthreads();  // nobody reads the pool any more: its memory is reused
-            qs = 0.0;
-            FCand* best = sh.wlist[kFsThreads / 32];
-            for (int r = tid; r < kMaxTopK; r += kFsThreads) best[r].x = -INFINITY, best[r].tok = INT_MAX;
-            for (int batch = batch0; batch < batch1 && !unusable; ++batch) {
-                const int s0 = batch * kFsSeg;
-                load_batch(s0);
-                int e[kFsElems];
-                bool bad_here = false;
-#pragma unroll
-                for (int i = 0; i < kFsElems; ++i) {
-                    e[i] = tok_of(s0, i) < V ? tok_of(s0, i) : INT_MAX;  // slots past the row rank last
-                    bad_here = bad_here || !(x[i] < INFINITY);
-                }
-                // sort the thread's 16 entries, best first (bitonic network on (logit, token) pairs; the order is total)
-#pragma unroll
-                for (int size = 2; size <= kFsElems; size <<= 1)
-#pragma unroll
-                    for (int stride = size >> 1; stride > 0; stride >>= 1)
-#pragma unroll
-                        for (int i = 0; i < kFsElems; ++i) {
-                            const int j = i ^ stride;
-                            if (j > i) {
-                                const bool up = (i & size) == 0;  // this block sorts best-first, its sibling worst-first
-                                const bool swap = up ? f_before(x[j], e[j], x[i], e[i]) : f_before(x[i], e[i], x[j], e[j]);
-                                if (swap) {
-                                    const float tx = x[i];
-                                    x[i] = x[j], x[j] = tx;
-                                    const int te = e[i];
-                                    e[i] = e[j], e[j] = te;
-                                }
-                            }
-                        }
-#pragma unroll
-                for (int i = 0; i < kFsElems; ++i) sh.lists[i][tid].x = x[i], sh.lists[i][tid].tok = e[i];
-                __syncwarp();
-                merge_heads(&sh.lists[0][warp * 32], 32, kFsElems, kFsThreads, 1, k, sh.wlist[warp]);
-                unusable = __syncthreads_or(bad_here);
-                if (warp == 0) {  // nine lists: the warps' and the best so far; the result replaces the best so far
-                    merge_heads(&sh.wlist[0][0], kFsThreads / 32 + 1, k, 1, kMaxTopK, k, sh.sorted);
-                    __syncwarp();
-                    for (int r = lane; r < k; r += 32) best[r] = sh.sorted[r];
-                }
-                __syncthreads();
-            }
-            kk = k;  // (empty entries at the end when the span holds fewer than k)
+            unusable = exact_piece<VEC>(sh, row, qrow, V, k, batch0, batch1, &qs);  // from the start of the piece
+            kk = k;  // (empty entries at the end when the piece holds fewer than k)
         }
         // ---- results: the piece's draft mass and its k best (or the mark of an unusable row)
 #pragma unroll
