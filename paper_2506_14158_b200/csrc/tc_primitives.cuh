@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a instructions a tensor-core kernel is built from: mbarriers with bounded waits, TMA
-// tile loads (no multicast), tensor-memory allocation and loads, tcgen05.mma issue and commit, operand and instruction
+// tile loads (each CTA fetches its own tiles), tensor-memory allocation and loads, tcgen05.mma issue and commit, operand and instruction
 // descriptors.  Device code only; used by kernels that include it (each keeps its own copy of what it needs otherwise).
 #pragma once
 #include <cuda.h>
