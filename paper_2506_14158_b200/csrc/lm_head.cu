@@ -6,7 +6,7 @@
 // accumulators in tensor memory.  One persistent CTA per SM walks over 128-token tiles of the vocabulary (tile = CTA index,
 // + grid size, ...): every weight tile leaves HBM once and meets all rows (up to 256: two 128-row accumulators side by
 // side on one weight stream); the hidden states (a few MB) are re-read from L2.  Roles: warp 0 requests tiles by TMA
-// (64-element K slices, 128-byte swizzle, a ring of 4 or 6 stages), warp 1 issues the products and commits them to the
+// (64-element K slices, 128-byte swizzle, a ring of 192 KB cut into 4 to 12 stages), warp 1 issues the products and commits them to the
 // ring's "empty" barriers and to the accumulator's "full" barrier, warps 2-5 read a finished accumulator (one row per
 // thread), keep the running (maximum, first token that reaches it) per row across the CTA's tiles while the next tile's
 // products fill the other accumulator.  A second small kernel merges the CTAs' candidates per row (greater logit, then
@@ -36,11 +36,11 @@ constexpr int kLmRowsPerLaunch = 2 * kLmBM;
 template <int NM>
 struct LmCfg {
     static constexpr int kMaxBN = NM == 2 ? 128 : 256;
-    static constexpr int kStages = 4;
-    static constexpr int kStageBytes = NM * kLmTileBytes + kMaxBN * kLmBK * 2;  // 48 KB
+    static constexpr int kRingBytes = 192 * 1024;      // cut into stages at launch: a stage holds the rows and tokens that exist
+    static constexpr int kMaxStages = 12;
     static constexpr int kTmemCols = 2 * NM * kMaxBN;  // two accumulator buffers: all 512 columns
-    static constexpr int kBars = 2 * kStages + 5;      // full[], empty[], acc_full[2], acc_empty[2], drain
-    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBars * 8 + 16;
+    static constexpr int kBars = 2 * kMaxStages + 5;   // full[], empty[], acc_full[2], acc_empty[2], drain
+    static constexpr int kSmemBytes = 1024 + kRingBytes + kBars * 8 + 16;
 };
 
 struct LmParams {
@@ -48,6 +48,8 @@ struct LmParams {
     int row0;
     int V;
     int bn;          // vocabulary entries per tile
+    int a_rows;      // rows of a hidden-state box (a multiple of 32, <= 128): 26 rows need not move 128
+    int stages;      // ring stages of a_rows * NM + bn rows of 128 bytes each
     int k_steps;     // H / 64
     float* part_v;   // [grid][256][KT] the CTAs' best logits per row, best first
     int32_t* part_t; // [grid][256][KT] and their tokens
@@ -58,23 +60,25 @@ template <int NM, int KT>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const LmParams prm) {
     using Cfg = LmCfg<NM>;
-    constexpr int S = Cfg::kStages;
+    constexpr int SM = Cfg::kMaxStages;
+    const int S = prm.stages;
+    const int a_bytes = prm.a_rows * kLmBK * 2, stage_bytes = NM * a_bytes + prm.bn * kLmBK * 2;
     extern __shared__ unsigned char lm_smem_raw[];
     const uint32_t raw = smem_u32(lm_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles start on 1024-byte boundaries
     unsigned char* gen = lm_smem_raw + (base - raw);
-    const uint32_t bars = base + S * Cfg::kStageBytes;
+    const uint32_t bars = base + Cfg::kRingBytes;
     auto FULL = [&](int s) { return bars + 8u * s; };
-    auto EMPTY = [&](int s) { return bars + 8u * (S + s); };
-    auto ACC_FULL = [&](int b) { return bars + 8u * (2 * S + b); };
-    auto ACC_EMPTY = [&](int b) { return bars + 8u * (2 * S + 2 + b); };
-    const uint32_t DRAIN = bars + 8u * (2 * S + 4);
-    volatile int* tail = reinterpret_cast<volatile int*>(gen + S * Cfg::kStageBytes + Cfg::kBars * 8);
+    auto EMPTY = [&](int s) { return bars + 8u * (SM + s); };
+    auto ACC_FULL = [&](int b) { return bars + 8u * (2 * SM + b); };
+    auto ACC_EMPTY = [&](int b) { return bars + 8u * (2 * SM + 2 + b); };
+    const uint32_t DRAIN = bars + 8u * (2 * SM + 4);
+    volatile int* tail = reinterpret_cast<volatile int*>(gen + Cfg::kRingBytes + Cfg::kBars * 8);
     volatile int* tmem_slot = tail;       // written by tcgen05.alloc
     volatile int* dead = tail + 1;        // a wait was given up
     volatile int* issued_s = tail + 2;    // stage fills the producer has requested
-    auto sA = [&](int s, int t) { return base + s * Cfg::kStageBytes + t * kLmTileBytes; };
-    auto sB = [&](int s) { return base + s * Cfg::kStageBytes + NM * kLmTileBytes; };
+    auto sA = [&](int s, int t) { return base + s * stage_bytes + t * a_bytes; };
+    auto sB = [&](int s) { return base + s * stage_bytes + NM * a_bytes; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bn = prm.bn;
@@ -97,14 +101,14 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     if (warp == 0) {
         // ================= producer: hidden-state and weight tiles into the ring =================
         if (lane == 0) {
-            int fill = 0;
+            int fill = 0, s = 0;
+            uint32_t ph = 0;  // the ring pass's parity (stage and parity are stepped, not divided out: S is not a constant)
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x)
-                for (int ks = 0; ks < prm.k_steps; ++ks, ++fill) {
-                    const int s = fill % S;
-                    ok = mbar_wait(EMPTY(s), ((fill / S) & 1) ^ 1, dead);
+                for (int ks = 0; ks < prm.k_steps; ++ks, ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                    ok = mbar_wait(EMPTY(s), ph ^ 1, dead);
                     if (!ok) break;
-                    mbar_expect_tx(FULL(s), NM * kLmTileBytes + bn * kLmBK * 2);
+                    mbar_expect_tx(FULL(s), stage_bytes);
 #pragma unroll
                     for (int t = 0; t < NM; ++t) tma_load_2d(sA(s, t), &map_h, FULL(s), ks * kLmBK, prm.row0 + t * kLmBM);
                     tma_load_2d(sB(s), &map_w, FULL(s), ks * kLmBK, tile * bn);
@@ -116,14 +120,14 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
         // ================= issuer: acc[t] = hidden tile t x weight tile^T over all K slices =================
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(kLmBM, bn, false);
-            int fill = 0, it = 0;
+            int it = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
                 const int buf = it & 1;
                 ok = mbar_wait(ACC_EMPTY(buf), ((it >> 1) & 1) ^ 1, dead);  // the epilogue has read this buffer
-                for (int ks = 0; ks < prm.k_steps && ok; ++ks, ++fill) {
-                    const int s = fill % S;
-                    ok = mbar_wait(FULL(s), (fill / S) & 1, dead);
+                for (int ks = 0; ks < prm.k_steps && ok; ++ks, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                    ok = mbar_wait(FULL(s), ph, dead);
                     if (!ok) break;
                     tc_fence_after();
                     const uint64_t b_desc = smem_desc_sw128(sB(s), 16, 1024);
@@ -420,8 +424,6 @@ extern "C" s4c_status s4c_lm_head_topk(const void* hidden, const void* weight, i
         return S4C_ERR_CUDA;
     }
     const int sms = std::min(lm_sm_count(), 1024), kt = lm_kt(k);
-    CUtensorMap map_h;
-    if (!lm_make_map(&map_h, hidden, (uint64_t)R, H, kLmBM)) return S4C_ERR_CUDA;
     // groups of up to 256 rows; each group streams the weights once
     for (int row0 = 0; row0 < R; row0 += kLmRowsPerLaunch) {
         LmParams prm;
@@ -437,9 +439,16 @@ extern "C" s4c_status s4c_lm_head_topk(const void* hidden, const void* weight, i
             }
         }
         const int grid = std::min(ceil_div(V, prm.bn), sms);
-        CUtensorMap map_w;
-        if (!lm_make_map(&map_w, weight, (uint64_t)V, H, prm.bn)) return S4C_ERR_CUDA;
         const bool two = prm.rows > kLmBM;
+        // the ring: a stage holds one K slice of the rows that exist (a box of 26 rows moves 32, not 128) and of the tile's
+        // tokens; as many stages as fit.  The product always reads 128 rows from a stage's start: one spare tile at the
+        // ring's end keeps that read inside the ring when a stage is shorter than a full tile.
+        prm.a_rows = two ? kLmBM : std::min(kLmBM, (int)round_up((size_t)prm.rows, 32));
+        const int stage_bytes = (two ? 2 : 1) * prm.a_rows * kLmBK * 2 + prm.bn * kLmBK * 2;
+        prm.stages = std::min(LmCfg<1>::kMaxStages, (LmCfg<1>::kRingBytes - (prm.a_rows < kLmBM ? kLmTileBytes : 0)) / stage_bytes);
+        CUtensorMap map_h, map_w;
+        if (!lm_make_map(&map_h, hidden, (uint64_t)R, H, prm.a_rows) || !lm_make_map(&map_w, weight, (uint64_t)V, H, prm.bn))
+            return S4C_ERR_CUDA;
         const s4c_status st = kt == 1   ? (two ? lm_launch<2, 1>(map_h, map_w, prm, grid, stream) : lm_launch<1, 1>(map_h, map_w, prm, grid, stream))
                               : kt == 4 ? (two ? lm_launch<2, 4>(map_h, map_w, prm, grid, stream) : lm_launch<1, 4>(map_h, map_w, prm, grid, stream))
                                         : (two ? lm_launch<2, 8>(map_h, map_w, prm, grid, stream) : lm_launch<1, 8>(map_h, map_w, prm, grid, stream));

@@ -7,7 +7,7 @@
 // [B*T, H] x [(Hq+2Hkv)*d, H]^T is a dense contraction: bf16 operands on the tcgen05 tensor cores, f32 accumulator in tensor
 // memory.  One CTA per (head, 128-row tile): a head's d output columns are one MMA tile, so both halves of every rotary pair
 // (j, j + d/2) sit in the same accumulator row.  Roles as in the LM-head kernel: warp 0 requests 64-element K slices by TMA
-// (128-byte swizzle, a ring of 6 stages), warp 1 issues the products, warps 2-5 read the finished accumulator (one row per
+// (128-byte swizzle, a ring of 192 KB cut into 6 to 12 stages), warp 1 issues the products, warps 2-5 read the finished accumulator (one row per
 // thread), rotate, round to bf16 and store 16 bytes at a time.  A small kernel in front checks the trees and the capacity
 // and tabulates cos / sin per (node, pair) in float64; the contraction is launched programmatically dependent on it and
 // only its epilogue waits for it.  Every wait on a barrier is bounded.
@@ -25,15 +25,16 @@ using namespace tcp;
 
 constexpr int kQkBM = 128;       // rows per CTA (tensor-memory lanes)
 constexpr int kQkBK = 64;        // hidden elements per stage (one 128-byte swizzled row)
-constexpr int kQkStages = 6;
-constexpr int kQkMaxD = 128;
-constexpr int kQkStageBytes = kQkBM * kQkBK * 2 + kQkMaxD * kQkBK * 2;  // 32 KB: a state tile and a weight tile
+constexpr int kQkMaxStages = 12;
+constexpr int kQkRingBytes = 192 * 1024;  // cut into stages at launch: a stage holds the rows that exist and the head's d weight rows
 constexpr int kQkThreads = 192;  // producer warp, issuer warp, four epilogue warps
-constexpr int kQkBars = 2 * kQkStages + 2;  // full[], empty[], acc_full, drain
-constexpr int kQkSmemBytes = 1024 + kQkStages * kQkStageBytes + kQkBars * 8 + 16;
+constexpr int kQkBars = 2 * kQkMaxStages + 2;  // full[], empty[], acc_full, drain
+constexpr int kQkSmemBytes = 1024 + kQkRingBytes + kQkBars * 8 + 16;
 
 struct QkParams {
     int R, T, Hq, Hkv, d, C, k_steps;
+    int x_rows;   // rows of a state box (a multiple of 32, <= 128): 26 rows need not move 128
+    int stages;   // ring stages of x_rows + d rows of 128 bytes each
     const int32_t* row_base;   // [R]: the row's committed length, -1 = write nothing (padding node, flagged sequence)
     const float2* rope;        // [R][d/2]: (cos, sin) of the row's position times the pair's frequency
     __nv_bfloat16* q_out;      // [B,Hq,T,d]
@@ -78,21 +79,23 @@ qkv_prep_kernel(const int32_t* __restrict__ cache_len, const int32_t* __restrict
 
 __global__ void __launch_bounds__(kQkThreads, 1)
 qkv_rope_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const QkParams prm) {
-    constexpr int S = kQkStages;
+    constexpr int SM = kQkMaxStages;
+    const int S = prm.stages;
+    const int x_bytes = prm.x_rows * kQkBK * 2, stage_bytes = x_bytes + prm.d * kQkBK * 2;
     extern __shared__ unsigned char qk_smem_raw[];
     const uint32_t raw = smem_u32(qk_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles start on 1024-byte boundaries
     unsigned char* gen = qk_smem_raw + (base - raw);
-    const uint32_t bars = base + S * kQkStageBytes;
+    const uint32_t bars = base + kQkRingBytes;
     auto FULL = [&](int s) { return bars + 8u * s; };
-    auto EMPTY = [&](int s) { return bars + 8u * (S + s); };
-    const uint32_t ACC_FULL = bars + 8u * (2 * S), DRAIN = bars + 8u * (2 * S + 1);
-    volatile int* tail = reinterpret_cast<volatile int*>(gen + S * kQkStageBytes + kQkBars * 8);
+    auto EMPTY = [&](int s) { return bars + 8u * (SM + s); };
+    const uint32_t ACC_FULL = bars + 8u * (2 * SM), DRAIN = bars + 8u * (2 * SM + 1);
+    volatile int* tail = reinterpret_cast<volatile int*>(gen + kQkRingBytes + kQkBars * 8);
     volatile int* tmem_slot = tail;  // written by tcgen05.alloc
     volatile int* dead = tail + 1;   // a wait was given up
     volatile int* issued_s = tail + 2;
-    auto sX = [&](int s) { return base + s * kQkStageBytes; };
-    auto sW = [&](int s) { return base + s * kQkStageBytes + kQkBM * kQkBK * 2; };
+    auto sX = [&](int s) { return base + s * stage_bytes; };
+    auto sW = [&](int s) { return base + s * stage_bytes + x_bytes; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int head = blockIdx.x, mtile = blockIdx.y, d = prm.d;
@@ -116,12 +119,12 @@ qkv_rope_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // every CTA walks the K slices from a start of its own: the CTAs of a row tile all read the same state tiles,
             // and in step they would all ask the same L2 lines at the same moment (the order of a sum's terms is free)
             const int k0 = (int)((blockIdx.x * 7u + blockIdx.y * 3u) % (uint32_t)prm.k_steps);
-            int fill = 0;
-            for (; fill < prm.k_steps; ++fill) {
-                const int s = fill % S;
-                if (!mbar_wait(EMPTY(s), ((fill / S) & 1) ^ 1, dead)) break;
+            int fill = 0, s = 0;
+            uint32_t ph = 0;  // the ring pass's parity (stage and parity are stepped, not divided out: S is not a constant)
+            for (; fill < prm.k_steps; ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                if (!mbar_wait(EMPTY(s), ph ^ 1, dead)) break;
                 const int ks = fill + k0 < prm.k_steps ? fill + k0 : fill + k0 - prm.k_steps;
-                mbar_expect_tx(FULL(s), kQkBM * kQkBK * 2 + d * kQkBK * 2);
+                mbar_expect_tx(FULL(s), stage_bytes);
                 tma_load_2d(sX(s), &map_x, FULL(s), ks * kQkBK, mtile * kQkBM);
                 tma_load_2d(sW(s), &map_w, FULL(s), ks * kQkBK, head * d);
             }
@@ -133,9 +136,10 @@ qkv_rope_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(kQkBM, d, false);
             bool ok = true;
-            for (int ks = 0; ks < prm.k_steps; ++ks) {
-                const int s = ks % S;
-                ok = mbar_wait(FULL(s), (ks / S) & 1, dead);
+            int s = 0;
+            uint32_t ph = 0;
+            for (int ks = 0; ks < prm.k_steps; ++ks, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                ok = mbar_wait(FULL(s), ph, dead);
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t a_desc = smem_desc_sw128(sX(s), 16, 1024), b_desc = smem_desc_sw128(sW(s), 16, 1024);
@@ -292,7 +296,13 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
     qk_ws_layout(B, T, d, static_cast<char*>(workspace), &row_base, &rope);
     const int R = B * T, heads = Hq + 2 * Hkv;
     CUtensorMap map_x, map_w;
-    if (!qk_make_map(&map_x, x, (uint64_t)R, H, kQkBM) || !qk_make_map(&map_w, w_qkv, (uint64_t)heads * d, H, d)) return S4C_ERR_CUDA;
+    // the ring: a stage holds one K slice of the rows that exist and of the head's weight rows; as many stages as fit.  The
+    // product always reads 128 rows from a stage's start: one spare tile at the ring's end keeps that read inside the ring
+    // when a stage is shorter than a full tile.
+    const int x_rows = R > kQkBM ? kQkBM : (int)round_up((size_t)R, 32);
+    const int stage_bytes = x_rows * kQkBK * 2 + d * kQkBK * 2;
+    const int stages = std::min(kQkMaxStages, (kQkRingBytes - (x_rows < kQkBM ? kQkBM * kQkBK * 2 : 0)) / stage_bytes);
+    if (!qk_make_map(&map_x, x, (uint64_t)R, H, x_rows) || !qk_make_map(&map_w, w_qkv, (uint64_t)heads * d, H, d)) return S4C_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     qkv_prep_kernel<<<dim3(B, ceil_div(T, kQkPrepNodes)), 128, 0, stream>>>(cache_len, parent, n_nodes, T, C, d, (double)rope_theta, row_base, rope, status);
     S4C_RETURN_IF_CUDA_ERROR();
@@ -308,6 +318,7 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
     }
     QkParams prm;
     prm.R = R, prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.d = d, prm.C = C, prm.k_steps = H / kQkBK;
+    prm.x_rows = x_rows, prm.stages = stages;
     prm.row_base = row_base, prm.rope = rope;
     prm.q_out = static_cast<__nv_bfloat16*>(q_out), prm.k_cache = static_cast<__nv_bfloat16*>(k_cache);
     prm.v_cache = static_cast<__nv_bfloat16*>(v_cache), prm.status = status;
