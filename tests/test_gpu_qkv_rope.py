@@ -67,7 +67,8 @@ def _compare(got, ref, x, w, cache_len, n_nodes, T):
 
 
 @pytest.mark.parametrize("B,T,H,Hq,Hkv,d,C", [(1, 1, 64, 1, 1, 64, 8), (2, 15, 128, 4, 4, 64, 160), (1, 26, 512, 8, 8, 128, 300),
-                                              (4, 64, 256, 8, 2, 128, 200), (3, 50, 192, 6, 3, 128, 512), (5, 128, 128, 2, 1, 128, 1024)])
+                                              (4, 64, 256, 8, 2, 128, 200), (3, 50, 192, 6, 3, 128, 512), (5, 128, 128, 2, 1, 128, 1024),
+                                              (2, 128, 64, 3, 1, 64, 256), (1, 33, 8192, 2, 2, 128, 64), (7, 19, 320, 5, 5, 64, 40)])
 def test_shapes_against_the_oracle(B, T, H, Hq, Hkv, d, C):
     rng = np.random.default_rng(B * 100 + T)
     parent = np.stack([W.random_tree(T, 6, rng, 1, 4) for _ in range(B)]) if T > 1 else np.full((B, 1), -1, dtype=np.int32)
