@@ -170,20 +170,41 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
                     uint32_t r[32];
                     tmem_ld32(TM(buf, t) + ((uint32_t)(q * 32) << 16) + c * 32, r);
                     tmem_wait_ld();
-                    // (once a row's list is full, most runs of 32 logits hold nothing that beats its last entry: one
-                    // maximum over the run settles that; NaN and columns past the vocabulary never enter)
-                    float run_max = -INFINITY;
+                    if (KT == 1) {
+                        // one candidate per row: compare and keep (tokens ascend within a CTA and the comparison is strict:
+                        // of equal logits the lower token stays)
+                        // (most runs of 32 hold nothing above the row's maximum so far: one maximum over the run settles that)
+                        float run_max = -INFINITY;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (col0 + c * 32 + j < prm.V) run_max = fmaxf(run_max, __uint_as_float(r[j]));
-                    if (run_max > best_v[t][KT - 1]) {
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + c * 32 + j < prm.V) run_max = fmaxf(run_max, __uint_as_float(r[j]));
+                        if (run_max > best_v[t][0]) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float v = __uint_as_float(r[j]);
+                                const int col = col0 + c * 32 + j;
+                                if (col < prm.V && v > best_v[t][0]) best_v[t][0] = v, best_t[t][0] = col;
+                            }
+                        }
+                    } else {
+                        // a ranked list per row: which of the 32 logits beat the list's last entry is one bit each; only
+                        // those (a few per run once the list has settled) are looked at again, in token order, and enter by
+                        // strict comparisons, so that of equal logits the lower token stays ahead.  NaN and columns past
+                        // the vocabulary never enter.  (The values are indexed by a run-time bit position: the compiler
+                        // keeps this copy in local memory, which the L1 serves.)
+                        float lv[32];
+                        uint32_t m = 0;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const float v = __uint_as_float(r[j]);
-                            const int col = col0 + c * 32 + j;
-                            // tokens ascend within a CTA and the comparison is strict: of equal logits the lower token stays ahead
-                            if (col < prm.V && v > best_v[t][KT - 1]) {
-                                best_v[t][KT - 1] = v, best_t[t][KT - 1] = col;
+                            lv[j] = __uint_as_float(r[j]);
+                            m |= (col0 + c * 32 + j < prm.V && lv[j] > best_v[t][KT - 1]) ? (1u << j) : 0u;
+                        }
+                        while (m) {
+                            const int j = __ffs(m) - 1;
+                            m &= m - 1;
+                            const float v = lv[j];
+                            if (v > best_v[t][KT - 1]) {
+                                best_v[t][KT - 1] = v, best_t[t][KT - 1] = col0 + c * 32 + j;
 #pragma unroll
                                 for (int jj = KT - 1; jj > 0; --jj)
                                     if (best_v[t][jj] > best_v[t][jj - 1]) {
