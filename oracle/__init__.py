@@ -19,6 +19,7 @@ Functions (array layouts are row-major numpy arrays):
 * :func:`accept_greedy_tokens` -- the greedy walk when the target's choice per node is already known (plain Python).
 * :func:`qkv_rope`, :func:`rope_rotate` -- the verify layer's input side: q/k/v projections of the tree tokens, rotary
                                  embedding at position cache_len + depth, k/v written into the caches' tree slots (numpy).
+* :func:`linear`, :func:`rmsnorm`, :func:`embed_gather` -- Eq. 3 / Eq. 6 and the decoder layer's other pieces (numpy).
 """
 from __future__ import annotations
 
@@ -470,3 +471,36 @@ def build_tree_from_topk(topk, branching, root_token, T, cache_len=None):
         par[b, :n] = parent
         pos[b, :n] = base[b] + np.asarray(depth)
     return dict(tokens=tokens, parent=par, position=pos, n_nodes=np.full(B, n, dtype=np.int32))
+
+
+def linear(x, w, x2=None, bias=None, residual=None, gate=False):
+    """A linear layer of the drafter / decoder layer in float64 (a library matrix product is the step).
+
+    y = concat[x, x2] @ w^T (+ bias): with x2 this is Eq. 3, h = Linear(concat[e, f]) -- x the embeddings, x2 the features,
+    w [N, K1 + K2].  gate=True: w holds 2N rows, the gate projection's N rows first, then the up projection's; the result is
+    silu(gate) * up, the LLaMA-family MLP's inner product (silu(z) = z / (1 + exp(-z))).  residual [R, N] is added last."""
+    xx = np.asarray(x, dtype=np.float64)
+    if x2 is not None:
+        xx = np.concatenate([xx, np.asarray(x2, dtype=np.float64)], axis=-1)
+    ww = np.asarray(w, dtype=np.float64)
+    y = xx @ ww.T
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)
+    if gate:
+        n = y.shape[-1] // 2
+        g, u = y[..., :n], y[..., n:]
+        y = g / (1.0 + np.exp(-g)) * u
+    if residual is not None:
+        y = y + np.asarray(residual, dtype=np.float64)
+    return y
+
+
+def rmsnorm(x, weight, eps=1e-6):
+    """Root-mean-square layer normalisation of the LLaMA family: x / sqrt(mean(x^2) + eps) * weight, float64."""
+    xx = np.asarray(x, dtype=np.float64)
+    return xx / np.sqrt(np.mean(xx * xx, axis=-1, keepdims=True) + eps) * np.asarray(weight, dtype=np.float64)
+
+
+def embed_gather(table, tokens):
+    """Eq. 6: e = Embedding(t): rows of the embedding table."""
+    return np.asarray(table)[np.asarray(tokens, dtype=np.int64)]
