@@ -323,6 +323,32 @@ s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_l
                         size_t workspace_bytes, s4c_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * s4c_linear, s4c_rmsnorm, s4c_embed_gather -- the pieces of the drafter's head (Section 3.1, Eq. 3-6)
+ * and of a LLaMA-family decoder layer that are not attention:
+ *   s4c_linear      out[r, n] = sum_k x1[r, k] w[n, k] + sum_k x2[r, k] w[n, K1 + k]  (+ bias[n])
+ *                   Eq. 3, h = Linear(concat[e, f]), is x1 = e, x2 = f: the concatenation is never
+ *                   formed.  gate != 0: w holds 2N rows (the gate projection's N rows, then the up
+ *                   projection's; bias likewise 2N) and out[r, n] = silu(gate_n) * up_n with
+ *                   silu(z) = z / (1 + exp(-z)).  residual [R, N] (or NULL) is added last.
+ *                   x1 [R, K1], x2 [R, K2] (NULL when K2 = 0), w [N or 2N, K1 + K2], bias, residual,
+ *                   out [R, N]: bf16, device, row-major, 16-byte aligned; K1, K2 multiples of 64,
+ *                   N a multiple of 8.  float32 accumulation, one rounding to bf16.  status: one
+ *                   int32 (device) or NULL, zeroed and OR-ed with S4C_SEQ_TIMEOUT if a wait inside
+ *                   the kernel was given up.
+ *   s4c_rmsnorm     out[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * weight   (bf16 in / out,
+ *                   float32 arithmetic; H a multiple of 8)
+ *   s4c_embed_gather out[r, :] = table[tokens[r], :]  (Eq. 6; bf16 table [V, H]; a token outside
+ *                   [0, V) yields zeros)
+ * ------------------------------------------------------------------------------------------ */
+s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
+                      void* out, int R, int K1, int K2, int N, int gate, int32_t* status, s4c_stream_t stream);
+
+s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, int R, int H, void* out, s4c_stream_t stream);
+
+s4c_status s4c_embed_gather(const void* table, const int32_t* tokens, int R, int V, int H, void* out,
+                            s4c_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * s4c_tree_attention_paged, s4c_kv_compact_paged -- the same two operations (Section 3.2: tree-masked
  * attention of the verification pass; keeping the accepted tokens' K/V) on PAGED caches, the layout
  * serving systems keep their caches in.  The paper does not discuss cache layouts.

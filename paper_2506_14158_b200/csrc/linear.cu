@@ -1,0 +1,366 @@
+// s4c_linear: the linear layers of the drafter and of a decoder layer (Eq. 3: h = Linear(concat[e, f]); Eq. 4's output
+// and MLP projections) on the tcgen05 tensor cores, with what follows them fused into the epilogue -- the second input's
+// columns (the concatenation never exists in memory), a bias, the gated form silu(gate) * up, a residual.
+// s4c_rmsnorm and s4c_embed_gather: the layer's two small row operations (root-mean-square normalisation; Eq. 6,
+// e = Embedding(t)).
+//
+// One CTA per (128-column tile of the output, 128-row tile): the pipeline of the q/k/v kernel -- warp 0 requests
+// 64-element K slices by TMA (128-byte swizzle; slices of the first input, then of the second, against consecutive column
+// ranges of the weight), warp 1 issues the products into one f32 accumulator in tensor memory, warps 2-5 read it (one row per
+// thread), apply the epilogue and store 16 bytes at a time.  Gated form: a tile's accumulator holds 64 gate columns beside
+// their 64 up columns (two 64-row boxes of the weight), as the q/k/v kernel keeps a rotary pair in one row.  Every wait on
+// a barrier is bounded.
+#include <cuda.h>
+#include <math.h>
+
+#include <algorithm>
+
+#include "s4c_common.cuh"
+#include "tc_primitives.cuh"
+
+namespace s4c {
+
+using namespace tcp;
+
+constexpr int kLnBM = 128;       // rows per CTA (tensor-memory lanes)
+constexpr int kLnBN = 128;       // accumulator columns per CTA
+constexpr int kLnBK = 64;        // K elements per stage (one 128-byte swizzled row)
+constexpr int kLnMaxStages = 12;
+constexpr int kLnRingBytes = 192 * 1024;
+constexpr int kLnThreads = 192;  // producer warp, issuer warp, four epilogue warps
+constexpr int kLnBars = 2 * kLnMaxStages + 2;  // full[], empty[], acc_full, drain
+constexpr int kLnSmemBytes = 1024 + kLnRingBytes + kLnBars * 8 + 16;
+
+struct LnParams {
+    int R, N, k1_steps, k2_steps;  // K slices of the first and of the second input
+    int gate;                      // 1: the weight holds N gate rows, then N up rows; out = silu(gate) * up
+    int x_rows, stages;            // rows of an input box (a multiple of 32, <= 128); ring stages
+    const __nv_bfloat16* bias;     // [N] or null
+    const __nv_bfloat16* residual; // [R, N] or null
+    __nv_bfloat16* out;            // [R, N]
+    int32_t* status;               // one word or null
+};
+
+__device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); }
+
+__global__ void __launch_bounds__(kLnThreads, 1)
+linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant__ CUtensorMap map_x2,
+              const __grid_constant__ CUtensorMap map_w, const LnParams prm) {
+    constexpr int SM = kLnMaxStages;
+    const int S = prm.stages;
+    const int x_bytes = prm.x_rows * kLnBK * 2, stage_bytes = x_bytes + kLnBN * kLnBK * 2;
+    extern __shared__ unsigned char ln_smem_raw[];
+    const uint32_t raw = smem_u32(ln_smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles start on 1024-byte boundaries
+    unsigned char* gen = ln_smem_raw + (base - raw);
+    const uint32_t bars = base + kLnRingBytes;
+    auto FULL = [&](int s) { return bars + 8u * s; };
+    auto EMPTY = [&](int s) { return bars + 8u * (SM + s); };
+    const uint32_t ACC_FULL = bars + 8u * (2 * SM), DRAIN = bars + 8u * (2 * SM + 1);
+    volatile int* tail = reinterpret_cast<volatile int*>(gen + kLnRingBytes + kLnBars * 8);
+    volatile int* tmem_slot = tail;  // written by tcgen05.alloc
+    volatile int* dead = tail + 1;   // a wait was given up
+    volatile int* issued_s = tail + 2;
+    auto sX = [&](int s) { return base + s * stage_bytes; };
+    auto sW = [&](int s) { return base + s * stage_bytes + x_bytes; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ntile = blockIdx.x, mtile = blockIdx.y;
+    const int k_steps = prm.k1_steps + prm.k2_steps;
+    const int n0 = ntile * (prm.gate ? kLnBN / 2 : kLnBN);  // first output column of this tile
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(FULL(s), 1), mbar_init(EMPTY(s), 1);
+        mbar_init(ACC_FULL, 1), mbar_init(DRAIN, 1);
+        mbar_fence_init();
+        *dead = 0, *issued_s = 0;
+        tma_prefetch_desc(&map_x1), tma_prefetch_desc(&map_w);
+        if (prm.k2_steps) tma_prefetch_desc(&map_x2);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<int*>(tmem_slot)), kLnBN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)*tmem_slot;
+
+    if (warp == 0) {
+        // ================= producer =================
+        if (lane == 0) {
+            // every CTA walks the K slices from a start of its own (the CTAs of a row tile read the same input tiles)
+            const int k0 = (int)((blockIdx.x * 7u + blockIdx.y * 3u) % (uint32_t)k_steps);
+            int fill = 0, s = 0;
+            uint32_t ph = 0;
+            for (; fill < k_steps; ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                if (!mbar_wait(EMPTY(s), ph ^ 1, dead)) break;
+                const int ks = fill + k0 < k_steps ? fill + k0 : fill + k0 - k_steps;
+                mbar_expect_tx(FULL(s), stage_bytes);
+                if (ks < prm.k1_steps)
+                    tma_load_2d(sX(s), &map_x1, FULL(s), ks * kLnBK, mtile * kLnBM);
+                else
+                    tma_load_2d(sX(s), &map_x2, FULL(s), (ks - prm.k1_steps) * kLnBK, mtile * kLnBM);
+                if (prm.gate) {  // 64 gate rows, then their 64 up rows
+                    tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
+                    tma_load_2d(sW(s) + (kLnBN / 2) * kLnBK * 2, &map_w, FULL(s), ks * kLnBK, prm.N + n0);
+                } else {
+                    tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
+                }
+            }
+            *issued_s = fill;
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ================= issuer: acc = input tile x (this tile's weight rows)^T =================
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_bf16(kLnBM, kLnBN, false);
+            bool ok = true;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int ks = 0; ks < k_steps; ++ks, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                ok = mbar_wait(FULL(s), ph, dead);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t a_desc = smem_desc_sw128(sX(s), 16, 1024), b_desc = smem_desc_sw128(sW(s), 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < kLnBK / 16; ++kk)  // 32 bytes per K step inside the swizzled row (field unit: 16 B)
+                    tc_mma_bf16(tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                tc_commit(EMPTY(s));
+            }
+            if (ok) tc_commit(ACC_FULL);
+        }
+        __syncwarp();
+    } else {
+        // ================= epilogue =================
+        const int q = warp & 3;  // the tensor-memory lanes this warp may read: 32 q .. 32 q + 31
+        const int r = mtile * kLnBM + q * 32 + lane;
+        bool ok = mbar_wait(ACC_FULL, 0, dead);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            const bool live = r < prm.R;
+            __nv_bfloat16* orow = prm.out + (size_t)(live ? r : 0) * prm.N;
+            const __nv_bfloat16* rrow = prm.residual ? prm.residual + (size_t)(live ? r : 0) * prm.N : nullptr;
+            const int n_chunks = prm.gate ? 2 : 4;  // runs of 32 output columns
+            for (int c = 0; c < n_chunks; ++c) {
+                uint32_t a[32], u[32];
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + c * 32, a);
+                if (prm.gate) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + kLnBN / 2 + c * 32, u);
+                tmem_wait_ld();
+                if (live) {
+#pragma unroll
+                    for (int v8 = 0; v8 < 4; ++v8) {  // eight output columns = one 16-byte store
+                        const int col = n0 + c * 32 + v8 * 8;
+                        if (col + 8 > prm.N) continue;  // (N is a multiple of 8)
+                        float y[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            y[j] = __uint_as_float(a[v8 * 8 + j]);
+                            if (prm.bias) y[j] += __bfloat162float(prm.bias[col + j]);
+                        }
+                        if (prm.gate) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float up = __uint_as_float(u[v8 * 8 + j]);
+                                if (prm.bias) up += __bfloat162float(prm.bias[prm.N + col + j]);
+                                y[j] = silu(y[j]) * up;
+                            }
+                        }
+                        if (rrow) {
+                            const uint4 rv = __ldg(reinterpret_cast<const uint4*>(rrow + col));
+                            const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 f = __bfloat1622float2(rp[j]);
+                                y[2 * j] += f.x, y[2 * j + 1] += f.y;
+                            }
+                        }
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const __nv_bfloat162 p = __floats2bfloat162_rn(y[2 * j], y[2 * j + 1]);
+                            pk[j] = *reinterpret_cast<const uint32_t*>(&p);
+                        }
+                        *reinterpret_cast<uint4*>(orow + col) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+                __syncwarp();  // the lanes took different ways; the next tensor-memory load is warp-wide
+            }
+            tc_fence_before();
+        }
+    }
+    __syncthreads();
+    if (*dead) {
+        // a wait was given up: nothing more is issued; what is still in flight lands before shared and tensor memory go
+        if (threadIdx.x == 0) {
+            const int issued = *issued_s;
+            for (int s = 0; s < S; ++s) {
+                int last = -1;
+                for (int f = s; f < issued; f += S) last = f;
+                if (last >= 0) mbar_drain(FULL(s), (last / S) & 1);
+            }
+        }
+        if (warp == 1 && lane == 0) {
+            tc_commit(DRAIN);
+            mbar_drain(DRAIN, 0);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0 && prm.status) atomicOr(prm.status, S4C_SEQ_TIMEOUT);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kLnBN);
+    }
+}
+
+// root-mean-square normalisation: one CTA per row, float32 arithmetic, one rounding to bf16
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ weight, float eps, int H,
+               __nv_bfloat16* __restrict__ out) {
+    __shared__ float red[8];
+    const size_t row = blockIdx.x;
+    const __nv_bfloat16* xr = x + row * H;
+    float ss = 0.f;
+    for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {  // H is a multiple of 8
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + i));
+        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __bfloat1622float2(p[j]);
+            ss += f.x * f.x + f.y * f.y;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float scale = rsqrtf(tot / (float)H + eps);
+    for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + i));
+        const uint4 g = __ldg(reinterpret_cast<const uint4*>(weight + i));
+        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+        const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g);
+        uint32_t pk[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __bfloat1622float2(p[j]), w2 = __bfloat1622float2(pg[j]);
+            const __nv_bfloat162 o2 = __floats2bfloat162_rn(f.x * scale * w2.x, f.y * scale * w2.y);
+            pk[j] = *reinterpret_cast<const uint32_t*>(&o2);
+        }
+        *reinterpret_cast<uint4*>(out + row * H + i) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+}
+
+// Eq. 6: rows of the embedding table; a token outside the table yields a row of zeros
+__global__ void __launch_bounds__(256)
+embed_gather_kernel(const __nv_bfloat16* __restrict__ table, const int32_t* __restrict__ tokens, int V, int H,
+                    __nv_bfloat16* __restrict__ out) {
+    const size_t row = blockIdx.x;
+    const int t = tokens[row];
+    const bool ok = t >= 0 && t < V;
+    for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (ok) v = __ldg(reinterpret_cast<const uint4*>(table + (size_t)t * H + i));
+        *reinterpret_cast<uint4*>(out + row * H + i) = v;
+    }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*LnEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static LnEncodeTiledFn ln_encode_fn() {
+    static LnEncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<LnEncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows, H] bf16 row-major, boxes of box_rows rows x 64 elements (128 bytes), 128-byte swizzle, zero fill out of range
+static bool ln_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H, int box_rows) {
+    LnEncodeTiledFn fn = ln_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)H, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)H * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kLnBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+
+}  // namespace s4c
+
+extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
+                                 void* out, int R, int K1, int K2, int N, int gate, int32_t* status, s4c_stream_t stream_) {
+    using namespace s4c;
+    if (!x1 || !w || !out || (K2 > 0 && !x2)) return S4C_ERR_NULL;
+    if (R < 0 || N < 8 || N % 8 != 0 || K1 < kLnBK || K1 % kLnBK != 0 || K2 < 0 || K2 % kLnBK != 0) return S4C_ERR_SHAPE;
+    if (!aligned16(x1) || !aligned16(w) || !aligned16(out) || (x2 && !aligned16(x2)) || (residual && !aligned16(residual)))
+        return S4C_ERR_ALIGN;
+    if (R == 0) return S4C_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) {
+        cudaGetLastError();
+        return S4C_ERR_CUDA;
+    }
+    const int x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
+    const int stage_bytes = x_rows * kLnBK * 2 + kLnBN * kLnBK * 2;
+    const int stages = std::min(kLnMaxStages, (kLnRingBytes - (x_rows < kLnBM ? kLnBM * kLnBK * 2 : 0)) / stage_bytes);
+    const int w_rows = gate ? 2 * N : N, cols_per_tile = gate ? kLnBN / 2 : kLnBN;
+    CUtensorMap map_x1, map_x2, map_w;
+    if (!ln_make_map(&map_x1, x1, (uint64_t)R, K1, x_rows) || !ln_make_map(&map_x2, K2 > 0 ? x2 : x1, (uint64_t)R, K2 > 0 ? K2 : K1, x_rows) ||
+        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, gate ? kLnBN / 2 : kLnBN))
+        return S4C_ERR_CUDA;
+    static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return S4C_ERR_CUDA;
+        }
+        configured[dev] = true;
+    }
+    LnParams prm;
+    prm.R = R, prm.N = N, prm.k1_steps = K1 / kLnBK, prm.k2_steps = K2 / kLnBK, prm.gate = gate ? 1 : 0;
+    prm.x_rows = x_rows, prm.stages = stages;
+    prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
+    prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
+    linear_kernel<<<dim3(ceil_div(N, cols_per_tile), ceil_div(R, kLnBM)), kLnThreads, kLnSmemBytes, stream>>>(map_x1, map_x2, map_w, prm);
+    S4C_RETURN_IF_CUDA_ERROR();
+    return S4C_OK;
+}
+
+extern "C" s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, int R, int H, void* out, s4c_stream_t stream_) {
+    using namespace s4c;
+    if (!x || !weight || !out) return S4C_ERR_NULL;
+    if (R < 0 || H < 8 || H % 8 != 0 || !(eps >= 0.f)) return S4C_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(weight) || !aligned16(out)) return S4C_ERR_ALIGN;
+    if (R == 0) return S4C_OK;
+    rmsnorm_kernel<<<R, 256, 0, static_cast<cudaStream_t>(stream_)>>>(static_cast<const __nv_bfloat16*>(x),
+                                                                     static_cast<const __nv_bfloat16*>(weight), eps, H,
+                                                                     static_cast<__nv_bfloat16*>(out));
+    S4C_RETURN_IF_CUDA_ERROR();
+    return S4C_OK;
+}
+
+extern "C" s4c_status s4c_embed_gather(const void* table, const int32_t* tokens, int R, int V, int H, void* out,
+                                       s4c_stream_t stream_) {
+    using namespace s4c;
+    if (!table || !tokens || !out) return S4C_ERR_NULL;
+    if (R < 0 || V < 1 || H < 8 || H % 8 != 0) return S4C_ERR_SHAPE;
+    if (!aligned16(table) || !aligned16(out)) return S4C_ERR_ALIGN;
+    if (R == 0) return S4C_OK;
+    embed_gather_kernel<<<R, 256, 0, static_cast<cudaStream_t>(stream_)>>>(static_cast<const __nv_bfloat16*>(table), tokens, V, H,
+                                                                          static_cast<__nv_bfloat16*>(out));
+    S4C_RETURN_IF_CUDA_ERROR();
+    return S4C_OK;
+}

@@ -181,4 +181,18 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert tbk(topk=None) == 1 and tbk(nn=None) == 1 and tbk(br=None) == 1
     assert tbk(T=129) == 2 and tbk(k=0) == 2 and tbk(k=3) == 2  # k = 3: fewer ranked choices than the 4 children of the root
     assert tbk(B=0) == 0
+    lib.s4c_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp]
+    ln = lambda **kw: lib.s4c_linear(*[kw.get(k, d) for k, d in [
+        ("x1", P), ("x2", None), ("w", P), ("b", None), ("res", None), ("out", P), ("R", 26), ("K1", 4096), ("K2", 0), ("N", 4096),
+        ("gate", 0), ("st", None), ("s", None)]])
+    assert ln(x1=None) == 1 and ln(w=None) == 1 and ln(out=None) == 1 and ln(K2=4096) == 1      # a second width without a second input
+    assert ln(K1=100) == 2 and ln(K2=32, x2=P) == 2 and ln(N=12) == 2 and ln(N=0) == 2 and ln(R=-1) == 2
+    assert ln(w=P + 4) == 4 and ln(res=P + 2) == 4
+    assert ln(R=0) == 0
+    lib.s4c_rmsnorm.argtypes = [vp, vp, f, i, i, vp, vp]
+    rn = lambda **kw: lib.s4c_rmsnorm(*[kw.get(k, d) for k, d in [("x", P), ("g", P), ("eps", 1e-6), ("R", 4), ("H", 4096), ("out", P), ("s", None)]])
+    assert rn(x=None) == 1 and rn(H=12) == 2 and rn(eps=-1.0) == 2 and rn(g=P + 2) == 4 and rn(R=0) == 0
+    lib.s4c_embed_gather.argtypes = [vp, vp, i, i, i, vp, vp]
+    eg = lambda **kw: lib.s4c_embed_gather(*[kw.get(k, d) for k, d in [("tab", P), ("tok", P), ("R", 4), ("V", 100), ("H", 64), ("out", P), ("s", None)]])
+    assert eg(tok=None) == 1 and eg(V=0) == 2 and eg(H=4) == 2 and eg(out=P + 8) == 4 and eg(R=0) == 0
     assert b"workspace" in lib.s4c_status_string(5)

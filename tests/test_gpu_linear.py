@@ -1,0 +1,109 @@
+"""GPU parity: s4c_linear (plain, two inputs, bias, gated, residual), s4c_rmsnorm and s4c_embed_gather against the oracle.
+
+Tolerance of the linear layer: bf16 inputs, float32 accumulation, one rounding to bf16 at the end:
+|got - want| <= 2^-8 |want| + 8 sqrt(K) 2^-24 ||x|| max ||w_n|| (for the gated form the bound of the two factors is
+propagated through silu(g) * u: |silu'| <= 1.1)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+from parity import Guarded
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16)
+
+
+def _f64(t):
+    return t.double().cpu().numpy()
+
+
+@pytest.mark.parametrize("R,K1,K2,N,bias,res", [(1, 64, 0, 8, False, False), (26, 256, 0, 384, True, False), (130, 128, 192, 200, True, True),
+                                               (256, 512, 512, 1024, False, True), (33, 64, 64, 136, True, True),
+                                               (300, 320, 0, 4096, False, False)])
+def test_linear_against_the_oracle(R, K1, K2, N, bias, res):
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(R + N)
+    K = K1 + K2
+    x1 = _bf16(rng.standard_normal((R, K1)))
+    x2 = _bf16(rng.standard_normal((R, K2))) if K2 else None
+    w = _bf16(rng.standard_normal((N, K)) / np.sqrt(K))
+    b = _bf16(rng.standard_normal(N)) if bias else None
+    rs = _bf16(rng.standard_normal((R, N))) if res else None
+    out = Guarded((R, N), torch.bfloat16, fill=-3.0)
+    st = torch.full((1,), -9, dtype=torch.int32, device="cuda")
+    s4c.linear(x1.cuda(), w.cuda(), None if x2 is None else x2.cuda(), None if b is None else b.cuda(),
+               None if rs is None else rs.cuda(), out=out.t, status=st)
+    torch.cuda.synchronize()
+    out.check("s4c_linear out")
+    assert int(st.item()) == 0
+    want = oracle.linear(_f64(x1), _f64(w), None if x2 is None else _f64(x2), None if b is None else _f64(b),
+                         None if rs is None else _f64(rs))
+    xn = np.linalg.norm(np.concatenate([_f64(x1)] + ([_f64(x2)] if K2 else []), axis=1), axis=1, keepdims=True)
+    slack = 8.0 * np.sqrt(K) * 2.0 ** -24 * xn * np.linalg.norm(_f64(w), axis=1).max()
+    assert (np.abs(_f64(out.t) - want) <= 2.0 ** -8 * np.abs(want) + slack + 1e-6).all()
+
+
+@pytest.mark.parametrize("R,K,N,res", [(26, 256, 704, False), (200, 128, 72, True), (64, 512, 1024, True)])
+def test_gated_linear_against_the_oracle(R, K, N, res):
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(R * 3 + N)
+    x, w = _bf16(rng.standard_normal((R, K))), _bf16(rng.standard_normal((2 * N, K)) / np.sqrt(K))
+    rs = _bf16(rng.standard_normal((R, N))) if res else None
+    out = Guarded((R, N), torch.bfloat16, fill=-3.0)
+    s4c.linear(x.cuda(), w.cuda(), residual=None if rs is None else rs.cuda(), gate=True, out=out.t)
+    torch.cuda.synchronize()
+    out.check("s4c_linear gated out")
+    want = oracle.linear(_f64(x), _f64(w), residual=None if rs is None else _f64(rs), gate=True)
+    y = _f64(x) @ _f64(w).T
+    g, u = y[:, :N], y[:, N:]
+    slack = 8.0 * np.sqrt(K) * 2.0 ** -24 * np.linalg.norm(_f64(x), axis=1, keepdims=True) * np.linalg.norm(_f64(w), axis=1).max()
+    bound = 2.0 ** -8 * np.abs(want) + slack * (1.1 * np.abs(u) + np.abs(g) + 1.0) + 1e-5
+    assert (np.abs(_f64(out.t) - want) <= bound).all()
+
+
+def test_concatenation_meets_the_right_columns():
+    # e = one-hot rows, f = 0: the result reads columns of the FIRST K1 columns of w; and the other way round
+    from paper_2506_14158_b200 import s4c
+
+    K1, K2, N = 64, 128, 256
+    rng = np.random.default_rng(9)
+    w = _bf16(rng.standard_normal((N, K1 + K2)))
+    e = torch.zeros(K1, K1, dtype=torch.bfloat16)
+    e[torch.arange(K1), torch.arange(K1)] = 1.0
+    got = s4c.linear(e.cuda(), w.cuda(), torch.zeros(K1, K2, dtype=torch.bfloat16).cuda())
+    np.testing.assert_array_equal(_f64(got), _f64(w)[:, :K1].T)
+    f = torch.zeros(K2, K2, dtype=torch.bfloat16)
+    f[torch.arange(K2), torch.arange(K2)] = 1.0
+    got = s4c.linear(torch.zeros(K2, K1, dtype=torch.bfloat16).cuda(), w.cuda(), f.cuda())
+    np.testing.assert_array_equal(_f64(got), _f64(w)[:, K1:].T)
+
+
+def test_rmsnorm_and_embedding():
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(10)
+    for R, H in ((1, 8), (26, 4096), (300, 5120), (7, 1000)):
+        x, g = _bf16(rng.standard_normal((R, H)) * 3.0), _bf16(1.0 + 0.1 * rng.standard_normal(H))
+        out = Guarded((R, H), torch.bfloat16, fill=-3.0)
+        s4c.rmsnorm(x.cuda(), g.cuda(), 1e-5, out=out.t)
+        torch.cuda.synchronize()
+        out.check("s4c_rmsnorm out")
+        want = oracle.rmsnorm(_f64(x), _f64(g), 1e-5)
+        assert (np.abs(_f64(out.t) - want) <= 2.0 ** -8 * np.abs(want) + 1e-5).all()
+    V, H = 1000, 256
+    table = _bf16(rng.standard_normal((V, H)))
+    tok = np.array([0, 999, 5, 5, 1000, -1, 17], dtype=np.int32)
+    out = Guarded((len(tok), H), torch.bfloat16, fill=-3.0)
+    s4c.embed_gather(table.cuda(), torch.from_numpy(tok).cuda(), out=out.t)
+    torch.cuda.synchronize()
+    out.check("s4c_embed_gather out")
+    want = oracle.embed_gather(_f64(table), np.clip(tok, 0, V - 1))
+    want[[4, 5]] = 0.0                                                  # tokens outside the table: zeros
+    np.testing.assert_array_equal(_f64(out.t), want)
