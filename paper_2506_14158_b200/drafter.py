@@ -1,0 +1,104 @@
+"""One head of the multi-head drafter (Section 3.1.1, Eq. 3-6), composed from the library's entry points.
+
+    e = Embedding(t)                                   s4c_embed_gather           (Eq. 6)
+    h = Linear(concat[e, f])                           s4c_linear, two inputs     (Eq. 3)
+    f' = Decoder_layer(h)                                                         (Eq. 4; one LLaMA-family layer)
+         a  = rmsnorm(h)                               s4c_rmsnorm
+         q, K/V tree slots = rope(a Wqkv^T)            s4c_qkv_rope
+         o  = tree attention(q, cache)                 s4c_tree_attention
+         h2 = h + o Wo^T                               s4c_linear, residual
+         f' = h2 + (silu(m Wg^T) * m Wu^T) Wd^T,  m = rmsnorm(h2)      s4c_rmsnorm, s4c_linear (gated), s4c_linear (residual)
+    ranked choices = top-k(LM_head(f'))                s4c_lm_head_topk           (Eq. 5; k = 1 is the Argmax)
+
+Only buffers, views and the order of the calls live here; every arithmetic step runs in the library's kernels.  The one
+torch operation on data is the transpose of the attention output [B,Hq,T,d] into rows [B*T, Hq*d] for the output
+projection (a copy, no arithmetic).  Weights are whatever the caller passes: this repository has no trained drafter, the
+benchmark and the tests use seeded random weights of the paper's models' shapes.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import s4c
+
+
+@dataclass
+class DrafterWeights:
+    embedding: torch.Tensor   # [V, H]       the target's embedding table
+    fc: torch.Tensor          # [H, 2H]      Eq. 3 (columns 0..H-1 meet e, H..2H-1 meet f)
+    fc_bias: Optional[torch.Tensor]  # [H] or None
+    norm1: torch.Tensor       # [H]
+    qkv: torch.Tensor         # [(Hq + 2 Hkv) d, H]
+    o: torch.Tensor           # [H, Hq d]
+    norm2: torch.Tensor       # [H]
+    gate_up: torch.Tensor     # [2 I, H]     the gate projection's rows, then the up projection's
+    down: torch.Tensor        # [H, I]
+    lm_head: torch.Tensor     # [V, H]       the target's LM head
+
+
+def random_weights(V: int, H: int, Hq: int, Hkv: int, d: int, inter: int, device, seed: int = 0) -> DrafterWeights:
+    """Seeded random weights of the given shapes (bf16; projections ~ N(0, 1/fan_in), norms near one)."""
+    g = torch.Generator(device=device).manual_seed(seed)
+    rn = lambda *shape, s=1.0: (torch.randn(*shape, generator=g, device=device, dtype=torch.float32) * s).to(torch.bfloat16)
+    return DrafterWeights(
+        embedding=rn(V, H), fc=rn(H, 2 * H, s=(2 * H) ** -0.5), fc_bias=rn(H, s=0.02), norm1=(1.0 + 0.05 * rn(H).float()).to(torch.bfloat16),
+        qkv=rn((Hq + 2 * Hkv) * d, H, s=H ** -0.5), o=rn(H, Hq * d, s=(Hq * d) ** -0.5),
+        norm2=(1.0 + 0.05 * rn(H).float()).to(torch.bfloat16), gate_up=rn(2 * inter, H, s=H ** -0.5), down=rn(H, inter, s=inter ** -0.5),
+        lm_head=rn(V, H, s=H ** -0.5))
+
+
+class DrafterHead:
+    """Buffers for one head's pass over the T positions of B sequences; ``forward`` runs the chain above and can be
+    captured in a CUDA graph (all buffers are allocated here, once)."""
+
+    def __init__(self, w: DrafterWeights, B: int, T: int, Hq: int, Hkv: int, d: int, C: int, k: int, eps: float = 1e-5,
+                 rope_theta: float = 10000.0):
+        self.w, self.B, self.T, self.Hq, self.Hkv, self.d, self.C, self.k = w, B, T, Hq, Hkv, d, C, k
+        self.eps, self.rope_theta = eps, rope_theta
+        dev = w.fc.device
+        H = w.fc.shape[0]
+        inter = w.down.shape[1]
+        R = B * T
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        self.e, self.h, self.a = torch.empty(R, H, **bf), torch.empty(R, H, **bf), torch.empty(R, H, **bf)
+        self.q = torch.empty(B, Hq, T, d, **bf)
+        self.attn = torch.empty(B, Hq, T, d, **bf)
+        self.o_in = torch.empty(R, Hq * d, **bf)
+        self.h2, self.m = torch.empty(R, H, **bf), torch.empty(R, H, **bf)
+        self.act = torch.empty(R, inter, **bf)
+        self.f_out = torch.empty(R, H, **bf)
+        self.token = torch.empty(R, k, dtype=torch.int32, device=dev)
+        self.logit = torch.empty(R, k, dtype=torch.float32, device=dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.status_qkv, self.status_attn = torch.empty(B, **i32), torch.empty(B, **i32)
+        self.status_head = torch.zeros(1, **i32)
+        V = w.lm_head.shape[0]
+        self.ws_qkv = torch.empty(max(1, s4c.qkv_rope_workspace_bytes(B, T, d)), dtype=torch.uint8, device=dev)
+        self.ws_attn = torch.empty(max(1, s4c.tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, torch.bfloat16)), dtype=torch.uint8,
+                                   device=dev)
+        self.ws_head = torch.empty(max(1, s4c.lm_head_topk_workspace_bytes(R, V, H, k)), dtype=torch.uint8, device=dev)
+
+    def forward(self, tokens: torch.Tensor, features: torch.Tensor, cache_len: torch.Tensor, parent: torch.Tensor,
+                k_cache: torch.Tensor, v_cache: torch.Tensor, n_nodes: Optional[torch.Tensor] = None, max_cache_len: int = 0):
+        """tokens [B,T] int32 (t_i), features [B*T, H] bf16 (f_i), the head's own K/V cache [B,Hkv,C,d] (tree slots are written),
+        the tree (``parent``: positions a token may look at; a chain for plain autoregressive drafting).
+        Returns dict(token [B*T,k], logit [B*T,k], features [B*T,H])."""
+        w = self.w
+        s4c.embed_gather(w.embedding, tokens.reshape(-1), out=self.e)
+        s4c.linear(self.e, w.fc, x2=features, bias=w.fc_bias, out=self.h)
+        s4c.rmsnorm(self.h, w.norm1, self.eps, out=self.a)
+        s4c.qkv_rope(self.a.view(self.B, self.T, -1), w.qkv, cache_len, parent, self.q, k_cache, v_cache, n_nodes, self.rope_theta,
+                     status=self.status_qkv, workspace=self.ws_qkv)
+        s4c.tree_attention(self.q, k_cache, v_cache, cache_len, parent, n_nodes, out=self.attn, status=self.status_attn,
+                           workspace=self.ws_attn, max_cache_len=max_cache_len)
+        self.o_in.view(self.B, self.T, self.Hq, self.d).copy_(self.attn.permute(0, 2, 1, 3))  # rows for the output projection
+        s4c.linear(self.o_in, w.o, residual=self.h, out=self.h2)
+        s4c.rmsnorm(self.h2, w.norm2, self.eps, out=self.m)
+        s4c.linear(self.m, w.gate_up, gate=True, out=self.act)
+        s4c.linear(self.act, w.down, residual=self.h2, out=self.f_out)
+        s4c.lm_head_topk(self.f_out, w.lm_head, self.k, token=self.token, logit=self.logit, status=self.status_head,
+                         workspace=self.ws_head)
+        return dict(token=self.token, logit=self.logit, features=self.f_out)
