@@ -470,6 +470,37 @@ def measure(cfg, args, device, rank, world, with_e2e):
         assert int(st_qk.abs().sum().item()) == 0, "s4c_qkv_rope flagged a sequence"
         qk = dict(ms=ms_qk, rows=cfg.B * cfg.T, N=(cfg.Hq + 2 * cfg.Hkv) * cfg.d, H=cfg.hid)
         del ws_qk, kc, vc
+    # one head of the drafter (Eq. 3-6) composed from the library's calls: embedding, Linear(concat[e, f]), one decoder layer,
+    # LM-head top-k -- random weights of the target's shapes, a cache of its own (timed alone)
+    dr = None
+    if cfg.dtype == "bf16" and not args.paged and cfg.d in (64, 128) and cfg.hid == cfg.Hq * cfg.d:
+        from paper_2506_14158_b200 import drafter
+
+        inter = {32000: 11008, 128256: 14336}.get(cfg.V, (cfg.hid * 8 // 3 + 255) // 256 * 256)  # the paper's models' MLP widths
+        kk = max(cfg.branching) if cfg.tree == "branching" else 4
+        wts = drafter.random_weights(cfg.V, cfg.hid, cfg.Hq, cfg.Hkv, cfg.d, inter, device, seed=cfg.config_id)
+        head = drafter.DrafterHead(wts, cfg.B, cfg.T, cfg.Hq, cfg.Hkv, cfg.d, cfg.C, kk)
+        kc = torch.zeros((cfg.B, cfg.Hkv, cfg.C, cfg.d), dtype=torch.bfloat16, device=device)
+        vc = torch.zeros_like(kc)
+        feats = step.feat_in.reshape(cfg.B * cfg.T, cfg.hid).contiguous()
+        run_head = lambda: head.forward(step.tokens, feats, step.cache_len0, step.parent, kc, vc, step.n_nodes, max_cache_len=cfg.L)
+        sg = torch.cuda.Stream()
+        sg.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(sg):
+            run_head()
+        torch.cuda.current_stream().wait_stream(sg)
+        torch.cuda.synchronize()
+        g_dr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_dr):
+            run_head()
+        for _ in range(3):
+            g_dr.replay()
+        ms_dr = time_graph(g_dr, K, torch)
+        assert int(head.status_head.item()) == 0 and int(head.status_qkv.abs().sum().item()) == 0
+        wbytes = sum(t.numel() * 2 for t in (wts.fc, wts.qkv, wts.o, wts.gate_up, wts.down, wts.lm_head))
+        dr = dict(ms=ms_dr, rows=cfg.B * cfg.T, weight_bytes=wbytes, inter=inter, k=kk,
+                  flops=2.0 * cfg.B * cfg.T * (wbytes / 2))
+        del wts, head, kc, vc
     ms_e2e = 0.0
     if with_e2e:
         # end to end: per-step inputs from pinned host memory, decision back to the host, every step
@@ -490,7 +521,7 @@ def measure(cfg, args, device, rank, world, with_e2e):
         [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
         device=device)
     rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
-               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, qk=qk, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, qk=qk, dr=dr, ms_e2e=ms_e2e, accept_lens=accept_lens,
                clocks=clocks, K=K, Wm=Wm)
     return rec
 
@@ -553,6 +584,16 @@ def roofline_records(cfg, args, rec, pk):
             us=qk["ms"] * 1e3, bound="tensor" if flops / byts >= ridge else "hbm", tflops=flops / t * 1e-12,
             frac_of_tensor_peak=flops / t * 1e-12 / pk["bf16_tflops"], gbs=byts / t * 1e-9,
             frac_of_hbm_peak=byts / t * 1e-9 / pk["hbm_gbs"], flop_per_byte=flops / byts)
+    if rec.get("dr") is not None:
+        dr = rec["dr"]
+        breakdown["drafter_head_not_in_step"] = dr["ms"]
+        t = dr["ms"] * 1e-3
+        roofline["drafter_head"] = dict(
+            kernel="one drafter head, Eq. 3-6: embed, Linear(concat[e,f]), decoder layer, LM-head top-k (11 launches)", rows=dr["rows"],
+            mlp_width=dr["inter"], top_k=dr["k"], us=dr["ms"] * 1e3, weight_bytes=dr["weight_bytes"],
+            bound="tensor" if dr["flops"] / dr["weight_bytes"] >= ridge else "hbm", gbs=dr["weight_bytes"] / t * 1e-9,
+            frac_of_hbm_peak=dr["weight_bytes"] / t * 1e-9 / pk["hbm_gbs"], tflops=dr["flops"] / t * 1e-12,
+            frac_of_tensor_peak=dr["flops"] / t * 1e-12 / pk["bf16_tflops"])
     return ab, step_hbm, roofline, breakdown
 
 

@@ -23,7 +23,7 @@ namespace s4c {
 using namespace tcp;
 
 constexpr int kLnBM = 128;       // rows per CTA (tensor-memory lanes)
-constexpr int kLnBN = 128;       // accumulator columns per CTA
+constexpr int kLnBN = 128;       // most accumulator columns per CTA (the launch picks 32, 64 or 128: see s4c_linear)
 constexpr int kLnBK = 64;        // K elements per stage (one 128-byte swizzled row)
 constexpr int kLnMaxStages = 12;
 constexpr int kLnRingBytes = 192 * 1024;
@@ -34,6 +34,7 @@ constexpr int kLnSmemBytes = 1024 + kLnRingBytes + kLnBars * 8 + 16;
 struct LnParams {
     int R, N, k1_steps, k2_steps;  // K slices of the first and of the second input
     int gate;                      // 1: the weight holds N gate rows, then N up rows; out = silu(gate) * up
+    int bn;                        // accumulator columns of a tile: 32, 64 or 128 (gated: half of them gate, half up)
     int x_rows, stages;            // rows of an input box (a multiple of 32, <= 128); ring stages
     const __nv_bfloat16* bias;     // [N] or null
     const __nv_bfloat16* residual; // [R, N] or null
@@ -48,7 +49,8 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
               const __grid_constant__ CUtensorMap map_w, const LnParams prm) {
     constexpr int SM = kLnMaxStages;
     const int S = prm.stages;
-    const int x_bytes = prm.x_rows * kLnBK * 2, stage_bytes = x_bytes + kLnBN * kLnBK * 2;
+    const int bn = prm.bn;
+    const int x_bytes = prm.x_rows * kLnBK * 2, stage_bytes = x_bytes + bn * kLnBK * 2;
     extern __shared__ unsigned char ln_smem_raw[];
     const uint32_t raw = smem_u32(ln_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles start on 1024-byte boundaries
@@ -67,7 +69,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ntile = blockIdx.x, mtile = blockIdx.y;
     const int k_steps = prm.k1_steps + prm.k2_steps;
-    const int n0 = ntile * (prm.gate ? kLnBN / 2 : kLnBN);  // first output column of this tile
+    const int n0 = ntile * (prm.gate ? bn / 2 : bn);  // first output column of this tile
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) mbar_init(FULL(s), 1), mbar_init(EMPTY(s), 1);
         mbar_init(ACC_FULL, 1), mbar_init(DRAIN, 1);
@@ -97,9 +99,9 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
                     tma_load_2d(sX(s), &map_x1, FULL(s), ks * kLnBK, mtile * kLnBM);
                 else
                     tma_load_2d(sX(s), &map_x2, FULL(s), (ks - prm.k1_steps) * kLnBK, mtile * kLnBM);
-                if (prm.gate) {  // 64 gate rows, then their 64 up rows
+                if (prm.gate) {  // bn / 2 gate rows, then their up rows
                     tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
-                    tma_load_2d(sW(s) + (kLnBN / 2) * kLnBK * 2, &map_w, FULL(s), ks * kLnBK, prm.N + n0);
+                    tma_load_2d(sW(s) + (bn / 2) * kLnBK * 2, &map_w, FULL(s), ks * kLnBK, prm.N + n0);
                 } else {
                     tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
                 }
@@ -110,7 +112,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     } else if (warp == 1) {
         // ================= issuer: acc = input tile x (this tile's weight rows)^T =================
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_bf16(kLnBM, kLnBN, false);
+            const uint32_t idesc = instr_desc_bf16(kLnBM, bn, false);
             bool ok = true;
             int s = 0;
             uint32_t ph = 0;
@@ -138,11 +140,11 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
             const bool live = r < prm.R;
             __nv_bfloat16* orow = prm.out + (size_t)(live ? r : 0) * prm.N;
             const __nv_bfloat16* rrow = prm.residual ? prm.residual + (size_t)(live ? r : 0) * prm.N : nullptr;
-            const int n_chunks = prm.gate ? 2 : 4;  // runs of 32 output columns
+            const int n_chunks = (prm.gate ? bn / 2 : bn) / 32;  // runs of 32 output columns
             for (int c = 0; c < n_chunks; ++c) {
                 uint32_t a[32], u[32];
                 tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + c * 32, a);
-                if (prm.gate) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + kLnBN / 2 + c * 32, u);
+                if (prm.gate) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + bn / 2 + c * 32, u);
                 tmem_wait_ld();
                 if (live) {
 #pragma unroll
@@ -312,12 +314,17 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
         return S4C_ERR_CUDA;
     }
     const int x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
-    const int stage_bytes = x_rows * kLnBK * 2 + kLnBN * kLnBK * 2;
-    const int stages = std::min(kLnMaxStages, (kLnRingBytes - (x_rows < kLnBM ? kLnBM * kLnBK * 2 : 0)) / stage_bytes);
-    const int w_rows = gate ? 2 * N : N, cols_per_tile = gate ? kLnBN / 2 : kLnBN;
+    // tile width: the widest of 128, 64, 32 accumulator columns that still gives about a CTA per SM (a narrow output such as
+    // the 4096 columns of a 7B model's projections is 32 tiles of 128: a fifth of the GPU)
+    const int m_tiles = ceil_div(R, kLnBM);
+    int bn = kLnBN;
+    while (bn > (gate ? 64 : 32) && (long long)ceil_div(gate ? 2 * N : N, bn) * m_tiles < 120) bn >>= 1;
+    const int stage_bytes = x_rows * kLnBK * 2 + bn * kLnBK * 2;
+    const int stages = std::min(kLnMaxStages, (kLnRingBytes - kLnBM * kLnBK * 2) / stage_bytes);  // (a spare tile: see the q/k/v kernel)
+    const int w_rows = gate ? 2 * N : N, cols_per_tile = gate ? bn / 2 : bn;
     CUtensorMap map_x1, map_x2, map_w;
     if (!ln_make_map(&map_x1, x1, (uint64_t)R, K1, x_rows) || !ln_make_map(&map_x2, K2 > 0 ? x2 : x1, (uint64_t)R, K2 > 0 ? K2 : K1, x_rows) ||
-        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, gate ? kLnBN / 2 : kLnBN))
+        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, gate ? bn / 2 : bn))
         return S4C_ERR_CUDA;
     static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
     int dev = 0;
@@ -331,7 +338,7 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
     }
     LnParams prm;
     prm.R = R, prm.N = N, prm.k1_steps = K1 / kLnBK, prm.k2_steps = K2 / kLnBK, prm.gate = gate ? 1 : 0;
-    prm.x_rows = x_rows, prm.stages = stages;
+    prm.x_rows = x_rows, prm.stages = stages, prm.bn = bn;
     prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
     prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
     linear_kernel<<<dim3(ceil_div(N, cols_per_tile), ceil_div(R, kLnBM)), kLnThreads, kLnSmemBytes, stream>>>(map_x1, map_x2, map_w, prm);

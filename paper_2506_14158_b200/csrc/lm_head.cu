@@ -258,24 +258,35 @@ lm_head_greedy_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_co
     }
 }
 
-// Per row: the k best of the CTAs' candidates, best first (greater logit, then lower token).  One warp per row; round j
+// Per row: the k best of the CTAs' candidates, best first (greater logit, then lower token).  One warp per row: the
+// candidates (at most 1024 CTAs x 8) come into shared memory once -- independent loads, in flight together --, then round j
 // takes the best candidate that ranks after round j-1's (the candidates' tokens are distinct).
-__global__ void __launch_bounds__(128)
+constexpr int kLmMergeRows = 4;      // rows (warps) per CTA
+constexpr int kLmMergeStage = 1184;  // candidates staged per row: 148 CTAs x 8; beyond that the rounds read global memory
+__global__ void __launch_bounds__(kLmMergeRows * 32)
 lm_head_merge_kernel(const float* __restrict__ part_v, const int32_t* __restrict__ part_t, int n_parts, int kt, int rows, int k,
                      int32_t* __restrict__ token, float* __restrict__ logit) {
+    __shared__ float sv[kLmMergeRows][kLmMergeStage];
+    __shared__ int st[kLmMergeRows][kLmMergeStage];
     griddep_wait();
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * kLmMergeRows + w;
     if (r >= rows) return;
     const int total = n_parts * kt;  // candidate c: CTA c / kt, rank c % kt
+    const bool staged = total <= kLmMergeStage;
+    auto at = [&](int c) { return ((size_t)(c / kt) * kLmRowsPerLaunch + r) * kt + (c % kt); };
+    if (staged) {
+        for (int c = lane; c < total; c += 32) sv[w][c] = part_v[at(c)], st[w][c] = part_t[at(c)];
+        __syncwarp();
+    }
     float pv = INFINITY;
     int pt = -1;
     for (int j = 0; j < k; ++j) {
         float bv = -INFINITY;
         int bt = INT_MAX;
         for (int c = lane; c < total; c += 32) {
-            const size_t at = ((size_t)(c / kt) * kLmRowsPerLaunch + r) * kt + (c % kt);
-            const float v = part_v[at];
-            const int t = part_t[at];
+            const float v = staged ? sv[w][c] : part_v[at(c)];
+            const int t = staged ? st[w][c] : part_t[at(c)];
             const bool after = v < pv || (v == pv && t > pt);
             if (t != INT_MAX && after && (v > bv || (v == bv && t < bt))) bv = v, bt = t;
         }
@@ -479,7 +490,7 @@ extern "C" s4c_status s4c_lm_head_topk(const void* hidden, const void* weight, i
         pdl.val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t cfg = {};
         cfg.stream = stream, cfg.attrs = &pdl, cfg.numAttrs = 1;
-        cfg.gridDim = dim3(ceil_div(prm.rows, 4), 1, 1), cfg.blockDim = dim3(128, 1, 1);  // a warp per row
+        cfg.gridDim = dim3(ceil_div(prm.rows, kLmMergeRows), 1, 1), cfg.blockDim = dim3(kLmMergeRows * 32, 1, 1);  // a warp per row
         if (cudaLaunchKernelEx(&cfg, lm_head_merge_kernel, (const float*)part_v, (const int32_t*)part_t, grid, kt, prm.rows, k,
                                token + (size_t)row0 * k, logit ? logit + (size_t)row0 * k : (float*)nullptr) != cudaSuccess) {
             cudaGetLastError();
