@@ -334,14 +334,22 @@ s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_l
  *                   out [R, N]: bf16, device, row-major, 16-byte aligned; K1, K2 multiples of 64,
  *                   N a multiple of 8.  float32 accumulation, one rounding to bf16.  status: one
  *                   int32 (device) or NULL, zeroed and OR-ed with S4C_SEQ_TIMEOUT if a wait inside
- *                   the kernel was given up.
+ *                   the kernel was given up.  A product with few output tiles shares each tile's
+ *                   K range out over several CTAs, whose float32 partial sums pass through
+ *                   workspace and are added in a fixed order (the result does not depend on
+ *                   timing): workspace must hold s4c_linear_workspace_bytes(R, K1, K2, N, gate)
+ *                   bytes (0 for shapes that need none; then NULL is accepted), 256-byte aligned;
+ *                   S4C_ERR_WORKSPACE otherwise.
  *   s4c_rmsnorm     out[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * weight   (bf16 in / out,
  *                   float32 arithmetic; H a multiple of 8)
  *   s4c_embed_gather out[r, :] = table[tokens[r], :]  (Eq. 6; bf16 table [V, H]; a token outside
  *                   [0, V) yields zeros)
  * ------------------------------------------------------------------------------------------ */
+size_t s4c_linear_workspace_bytes(int R, int K1, int K2, int N, int gate);
+
 s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
-                      void* out, int R, int K1, int K2, int N, int gate, int32_t* status, s4c_stream_t stream);
+                      void* out, int R, int K1, int K2, int N, int gate, int32_t* status, void* workspace,
+                      size_t workspace_bytes, s4c_stream_t stream);
 
 s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, int R, int H, void* out, s4c_stream_t stream);
 

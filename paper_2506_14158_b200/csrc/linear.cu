@@ -40,6 +40,8 @@ struct LnParams {
     const __nv_bfloat16* residual; // [R, N] or null
     __nv_bfloat16* out;            // [R, N]
     int32_t* status;               // one word or null
+    int splits;                    // CTAs that share a tile's K slices (grid.z); > 1: raw partial sums go to `partial`
+    float* partial;                // [splits][R][N or 2N] float32, read by linear_finish_kernel
 };
 
 __device__ __forceinline__ float silu(float z) { return z / (1.f + __expf(-z)); }
@@ -68,7 +70,9 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ntile = blockIdx.x, mtile = blockIdx.y;
-    const int k_steps = prm.k1_steps + prm.k2_steps;
+    const int k_all = prm.k1_steps + prm.k2_steps;
+    const int k_begin = (int)((long long)k_all * blockIdx.z / prm.splits), k_end = (int)((long long)k_all * (blockIdx.z + 1) / prm.splits);
+    const int k_steps = k_end - k_begin;  // this CTA's share of the K slices (>= 1: the launch keeps splits <= slices)
     const int n0 = ntile * (prm.gate ? bn / 2 : bn);  // first output column of this tile
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) mbar_init(FULL(s), 1), mbar_init(EMPTY(s), 1);
@@ -93,7 +97,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
             uint32_t ph = 0;
             for (; fill < k_steps; ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
                 if (!mbar_wait(EMPTY(s), ph ^ 1, dead)) break;
-                const int ks = fill + k0 < k_steps ? fill + k0 : fill + k0 - k_steps;
+                const int ks = k_begin + (fill + k0 < k_steps ? fill + k0 : fill + k0 - k_steps);
                 mbar_expect_tx(FULL(s), stage_bytes);
                 if (ks < prm.k1_steps)
                     tma_load_2d(sX(s), &map_x1, FULL(s), ks * kLnBK, mtile * kLnBM);
@@ -140,7 +144,32 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
             const bool live = r < prm.R;
             __nv_bfloat16* orow = prm.out + (size_t)(live ? r : 0) * prm.N;
             const __nv_bfloat16* rrow = prm.residual ? prm.residual + (size_t)(live ? r : 0) * prm.N : nullptr;
-            const int n_chunks = (prm.gate ? bn / 2 : bn) / 32;  // runs of 32 output columns
+            if (prm.splits > 1) {
+                // a share of the K slices: the raw sums go out as float32, column = weight row; linear_finish_kernel adds the
+                // shares in split order and applies what follows the product
+                const int w_rows = prm.gate ? 2 * prm.N : prm.N;
+                float* prow = prm.partial + ((size_t)blockIdx.z * prm.R + (live ? r : 0)) * w_rows;
+                for (int c = 0; c < bn / 32; ++c) {
+                    uint32_t a[32];
+                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + c * 32, a);
+                    tmem_wait_ld();
+                    // accumulator column -> weight row: plain n0 + column; gated: the first half are gate rows n0.., the second
+                    // half up rows N + n0..
+                    const int cc = c * 32;
+                    const int wrow = prm.gate ? (cc < bn / 2 ? n0 + cc : prm.N + n0 + cc - bn / 2) : n0 + cc;
+                    const int limit = prm.gate ? (cc < bn / 2 ? prm.N : 2 * prm.N) : prm.N;
+                    if (live) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 8; ++v4)
+                            if (wrow + v4 * 4 + 4 <= limit)
+                                *reinterpret_cast<float4*>(prow + wrow + v4 * 4) =
+                                    make_float4(__uint_as_float(a[v4 * 4]), __uint_as_float(a[v4 * 4 + 1]), __uint_as_float(a[v4 * 4 + 2]),
+                                                __uint_as_float(a[v4 * 4 + 3]));
+                    }
+                    __syncwarp();
+                }
+            }
+            const int n_chunks = prm.splits > 1 ? 0 : (prm.gate ? bn / 2 : bn) / 32;  // runs of 32 output columns
             for (int c = 0; c < n_chunks; ++c) {
                 uint32_t a[32], u[32];
                 tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + c * 32, a);
@@ -209,6 +238,46 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem, kLnBN);
+    }
+}
+
+// After a product whose K slices were shared out: per output element the shares in split order, then bias, gate,
+// residual, one rounding to bf16.  grid (rows), eight columns per thread at a time.
+__global__ void __launch_bounds__(256)
+linear_finish_kernel(const float* __restrict__ partial, int splits, int R, int N, int gate, const __nv_bfloat16* __restrict__ bias,
+                     const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ out) {
+    griddep_wait();
+    const int r = blockIdx.x;
+    const int w_rows = gate ? 2 * N : N;
+    for (int col = threadIdx.x * 8; col < N; col += blockDim.x * 8) {
+        float y[8], up[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) y[j] = 0.f, up[j] = 0.f;
+        for (int z = 0; z < splits; ++z) {
+            const float* p = partial + ((size_t)z * R + r) * w_rows;
+            const float4 a0 = *reinterpret_cast<const float4*>(p + col), a1 = *reinterpret_cast<const float4*>(p + col + 4);
+            y[0] += a0.x, y[1] += a0.y, y[2] += a0.z, y[3] += a0.w, y[4] += a1.x, y[5] += a1.y, y[6] += a1.z, y[7] += a1.w;
+            if (gate) {
+                const float4 u0 = *reinterpret_cast<const float4*>(p + N + col), u1 = *reinterpret_cast<const float4*>(p + N + col + 4);
+                up[0] += u0.x, up[1] += u0.y, up[2] += u0.z, up[3] += u0.w, up[4] += u1.x, up[5] += u1.y, up[6] += u1.z, up[7] += u1.w;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (bias) y[j] += __bfloat162float(bias[col + j]);
+            if (gate) {
+                if (bias) up[j] += __bfloat162float(bias[N + col + j]);
+                y[j] = silu(y[j]) * up[j];
+            }
+            if (residual) y[j] += __bfloat162float(residual[(size_t)r * N + col + j]);
+        }
+        uint32_t pk[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(y[2 * j], y[2 * j + 1]);
+            pk[j] = *reinterpret_cast<const uint32_t*>(&p2);
+        }
+        *reinterpret_cast<uint4*>(out + (size_t)r * N + col) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
 }
 
@@ -298,10 +367,37 @@ static bool ln_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H,
 }
 
 
+// The launch shape of a product: the widest tile (128 accumulator columns: the issuing thread spends ~140 cycles per
+// tcgen05.mma whatever its width, so a narrow tile moves fewer bytes per issue), and the K slices of a tile shared out over
+// as many CTAs as it takes to have about one per SM -- a 7B model's 4096-column projections are 32 tiles, a fifth of the GPU.
+struct LnPlan {
+    int bn, splits, x_rows, stages, cols_per_tile, m_tiles, n_tiles;
+};
+static LnPlan ln_plan(int R, int K1, int K2, int N, int gate) {
+    LnPlan p;
+    p.bn = kLnBN;
+    p.cols_per_tile = gate ? p.bn / 2 : p.bn;
+    p.m_tiles = ceil_div(R, kLnBM), p.n_tiles = ceil_div(N, p.cols_per_tile);
+    const int k_steps = (K1 + K2) / kLnBK, tiles = p.m_tiles * p.n_tiles;
+    p.splits = std::max(1, std::min(std::min(8, k_steps / 8), 148 / std::max(1, tiles)));
+    p.x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
+    const int stage_bytes = p.x_rows * kLnBK * 2 + p.bn * kLnBK * 2;
+    p.stages = std::min(kLnMaxStages, (kLnRingBytes - kLnBM * kLnBK * 2) / stage_bytes);  // (a spare tile: see the q/k/v kernel)
+    return p;
+}
+
 }  // namespace s4c
 
+extern "C" size_t s4c_linear_workspace_bytes(int R, int K1, int K2, int N, int gate) {
+    using namespace s4c;
+    if (R < 1 || N < 8 || K1 < kLnBK || K2 < 0) return 0;
+    const LnPlan p = ln_plan(R, K1, K2, N, gate);
+    return p.splits > 1 ? round_up((size_t)p.splits * R * (gate ? 2 * N : N) * sizeof(float), 256) : 0;
+}
+
 extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
-                                 void* out, int R, int K1, int K2, int N, int gate, int32_t* status, s4c_stream_t stream_) {
+                                 void* out, int R, int K1, int K2, int N, int gate, int32_t* status, void* workspace,
+                                 size_t workspace_bytes, s4c_stream_t stream_) {
     using namespace s4c;
     if (!x1 || !w || !out || (K2 > 0 && !x2)) return S4C_ERR_NULL;
     if (R < 0 || N < 8 || N % 8 != 0 || K1 < kLnBK || K1 % kLnBK != 0 || K2 < 0 || K2 % kLnBK != 0) return S4C_ERR_SHAPE;
@@ -309,22 +405,18 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
         return S4C_ERR_ALIGN;
     if (R == 0) return S4C_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const LnPlan pl = ln_plan(R, K1, K2, N, gate);
+    const size_t need = pl.splits > 1 ? round_up((size_t)pl.splits * R * (gate ? 2 * N : N) * sizeof(float), 256) : 0;
+    if (need && (!workspace || workspace_bytes < need || !aligned256(workspace))) return S4C_ERR_WORKSPACE;
     if (status && cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
-    const int x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
-    // tile width: the widest of 128, 64, 32 accumulator columns that still gives about a CTA per SM (a narrow output such as
-    // the 4096 columns of a 7B model's projections is 32 tiles of 128: a fifth of the GPU)
-    const int m_tiles = ceil_div(R, kLnBM);
-    int bn = kLnBN;
-    while (bn > (gate ? 64 : 32) && (long long)ceil_div(gate ? 2 * N : N, bn) * m_tiles < 120) bn >>= 1;
-    const int stage_bytes = x_rows * kLnBK * 2 + bn * kLnBK * 2;
-    const int stages = std::min(kLnMaxStages, (kLnRingBytes - kLnBM * kLnBK * 2) / stage_bytes);  // (a spare tile: see the q/k/v kernel)
-    const int w_rows = gate ? 2 * N : N, cols_per_tile = gate ? bn / 2 : bn;
+    const int w_rows = gate ? 2 * N : N;
     CUtensorMap map_x1, map_x2, map_w;
-    if (!ln_make_map(&map_x1, x1, (uint64_t)R, K1, x_rows) || !ln_make_map(&map_x2, K2 > 0 ? x2 : x1, (uint64_t)R, K2 > 0 ? K2 : K1, x_rows) ||
-        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, gate ? bn / 2 : bn))
+    if (!ln_make_map(&map_x1, x1, (uint64_t)R, K1, pl.x_rows) ||
+        !ln_make_map(&map_x2, K2 > 0 ? x2 : x1, (uint64_t)R, K2 > 0 ? K2 : K1, pl.x_rows) ||
+        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, gate ? pl.bn / 2 : pl.bn))
         return S4C_ERR_CUDA;
     static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
     int dev = 0;
@@ -338,11 +430,25 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
     }
     LnParams prm;
     prm.R = R, prm.N = N, prm.k1_steps = K1 / kLnBK, prm.k2_steps = K2 / kLnBK, prm.gate = gate ? 1 : 0;
-    prm.x_rows = x_rows, prm.stages = stages, prm.bn = bn;
+    prm.x_rows = pl.x_rows, prm.stages = pl.stages, prm.bn = pl.bn;
     prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
     prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
-    linear_kernel<<<dim3(ceil_div(N, cols_per_tile), ceil_div(R, kLnBM)), kLnThreads, kLnSmemBytes, stream>>>(map_x1, map_x2, map_w, prm);
+    prm.splits = pl.splits, prm.partial = static_cast<float*>(workspace);
+    linear_kernel<<<dim3(pl.n_tiles, pl.m_tiles, pl.splits), kLnThreads, kLnSmemBytes, stream>>>(map_x1, map_x2, map_w, prm);
     S4C_RETURN_IF_CUDA_ERROR();
+    if (pl.splits > 1) {
+        cudaLaunchAttribute pdl;
+        pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pdl.val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.stream = stream, cfg.attrs = &pdl, cfg.numAttrs = 1;
+        cfg.gridDim = dim3(R, 1, 1), cfg.blockDim = dim3(256, 1, 1);
+        if (cudaLaunchKernelEx(&cfg, linear_finish_kernel, (const float*)prm.partial, pl.splits, R, N, gate ? 1 : 0, prm.bias, prm.residual,
+                               prm.out) != cudaSuccess) {
+            cudaGetLastError();
+            return S4C_ERR_CUDA;
+        }
+    }
     return S4C_OK;
 }
 

@@ -80,6 +80,9 @@ class DrafterHead:
         self.ws_attn = torch.empty(max(1, s4c.tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, torch.bfloat16)), dtype=torch.uint8,
                                    device=dev)
         self.ws_head = torch.empty(max(1, s4c.lm_head_topk_workspace_bytes(R, V, H, k)), dtype=torch.uint8, device=dev)
+        ws_lin = max(s4c.linear_workspace_bytes(R, H, H, H), s4c.linear_workspace_bytes(R, Hq * d, 0, H),
+                     s4c.linear_workspace_bytes(R, H, 0, inter, True), s4c.linear_workspace_bytes(R, inter, 0, H))
+        self.ws_lin = torch.empty(max(1, ws_lin), dtype=torch.uint8, device=dev)  # the four products run one after another
 
     def forward(self, tokens: torch.Tensor, features: torch.Tensor, cache_len: torch.Tensor, parent: torch.Tensor,
                 k_cache: torch.Tensor, v_cache: torch.Tensor, n_nodes: Optional[torch.Tensor] = None, max_cache_len: int = 0):
@@ -88,17 +91,17 @@ class DrafterHead:
         Returns dict(token [B*T,k], logit [B*T,k], features [B*T,H])."""
         w = self.w
         s4c.embed_gather(w.embedding, tokens.reshape(-1), out=self.e)
-        s4c.linear(self.e, w.fc, x2=features, bias=w.fc_bias, out=self.h)
+        s4c.linear(self.e, w.fc, x2=features, bias=w.fc_bias, out=self.h, workspace=self.ws_lin)
         s4c.rmsnorm(self.h, w.norm1, self.eps, out=self.a)
         s4c.qkv_rope(self.a.view(self.B, self.T, -1), w.qkv, cache_len, parent, self.q, k_cache, v_cache, n_nodes, self.rope_theta,
                      status=self.status_qkv, workspace=self.ws_qkv)
         s4c.tree_attention(self.q, k_cache, v_cache, cache_len, parent, n_nodes, out=self.attn, status=self.status_attn,
                            workspace=self.ws_attn, max_cache_len=max_cache_len)
         self.o_in.view(self.B, self.T, self.Hq, self.d).copy_(self.attn.permute(0, 2, 1, 3))  # rows for the output projection
-        s4c.linear(self.o_in, w.o, residual=self.h, out=self.h2)
+        s4c.linear(self.o_in, w.o, residual=self.h, out=self.h2, workspace=self.ws_lin)
         s4c.rmsnorm(self.h2, w.norm2, self.eps, out=self.m)
-        s4c.linear(self.m, w.gate_up, gate=True, out=self.act)
-        s4c.linear(self.act, w.down, residual=self.h2, out=self.f_out)
+        s4c.linear(self.m, w.gate_up, gate=True, out=self.act, workspace=self.ws_lin)
+        s4c.linear(self.act, w.down, residual=self.h2, out=self.f_out, workspace=self.ws_lin)
         s4c.lm_head_topk(self.f_out, w.lm_head, self.k, token=self.token, logit=self.logit, status=self.status_head,
                          workspace=self.ws_head)
         return dict(token=self.token, logit=self.logit, features=self.f_out)

@@ -26,7 +26,7 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
            "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
            "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
-           "s4c_tree_build_topk", "s4c_linear", "s4c_rmsnorm", "s4c_embed_gather"]
+           "s4c_tree_build_topk", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_rmsnorm", "s4c_embed_gather"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -90,8 +90,10 @@ def _load() -> ctypes.CDLL:
     lib.s4c_lm_head_topk.argtypes = [vp, vp, i, i, i, i, i32p, vp, i32p, vp, sz, vp]
     lib.s4c_tree_build_topk.restype = i
     lib.s4c_tree_build_topk.argtypes = [i32p, i, vp, i, i32p, i32p, i, i, i32p, i32p, i32p, i32p, vp]
+    lib.s4c_linear_workspace_bytes.restype = sz
+    lib.s4c_linear_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.s4c_linear.restype = i
-    lib.s4c_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i32p, vp]
+    lib.s4c_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i32p, vp, sz, vp]
     lib.s4c_rmsnorm.restype = i
     lib.s4c_rmsnorm.argtypes = [vp, vp, f, i, i, vp, vp]
     lib.s4c_embed_gather.restype = i
@@ -533,16 +535,23 @@ def tree_build_topk(topk, branching, root_token, cache_len=None, tokens=None, pa
     return dict(tokens=tokens, parent=parent, position=position, n_nodes=n_nodes)
 
 
-def linear(x1, w, x2=None, bias=None, residual=None, gate: bool = False, out=None, status=None, stream=None):
+def linear_workspace_bytes(R, K1, K2, N, gate: bool = False) -> int:
+    return int(_lib.s4c_linear_workspace_bytes(R, K1, K2, N, 1 if gate else 0))
+
+
+def linear(x1, w, x2=None, bias=None, residual=None, gate: bool = False, out=None, status=None, workspace=None, stream=None):
     """s4c_linear: out = concat[x1, x2] @ w^T (+ bias) (gate: silu(gate rows) * up rows) (+ residual); bf16, f32 accumulation."""
     R, K1 = x1.shape
     K2 = 0 if x2 is None else x2.shape[1]
     N = w.shape[0] // 2 if gate else w.shape[0]
     bf = torch.bfloat16
     out = torch.empty(R, N, dtype=bf, device=x1.device) if out is None else out
+    if workspace is None:
+        workspace = _workspace(int(_lib.s4c_linear_workspace_bytes(R, K1, K2, N, 1 if gate else 0)), x1.device, "linear")
     rc = _lib.s4c_linear(_dev(x1, bf, "x1"), _dev(x2, bf, "x2"), _dev(w, bf, "w"), _dev(bias, bf, "bias"),
                          _dev(residual, bf, "residual"), _dev(out, bf, "out"), R, K1, K2, N, 1 if gate else 0,
-                         _dev(status, torch.int32, "status"), _stream(stream))
+                         _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+                         0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
     if rc:
         raise S4CError("s4c_linear", rc)
     return out

@@ -181,13 +181,19 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert tbk(topk=None) == 1 and tbk(nn=None) == 1 and tbk(br=None) == 1
     assert tbk(T=129) == 2 and tbk(k=0) == 2 and tbk(k=3) == 2  # k = 3: fewer ranked choices than the 4 children of the root
     assert tbk(B=0) == 0
-    lib.s4c_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp]
+    lib.s4c_linear_workspace_bytes.restype = ctypes.c_size_t
+    lib.s4c_linear_workspace_bytes.argtypes = [i, i, i, i, i]
+    # 26 x 4096 outputs are 32 tiles: the K range is shared out and the partial sums need room; a wide output needs none
+    assert lib.s4c_linear_workspace_bytes(26, 4096, 0, 4096, 0) >= 2 * 26 * 4096 * 4
+    assert lib.s4c_linear_workspace_bytes(26, 4096, 0, 32768, 0) == 0 and lib.s4c_linear_workspace_bytes(26, 64, 0, 4096, 0) == 0
+    lib.s4c_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp, ctypes.c_size_t, vp]
     ln = lambda **kw: lib.s4c_linear(*[kw.get(k, d) for k, d in [
         ("x1", P), ("x2", None), ("w", P), ("b", None), ("res", None), ("out", P), ("R", 26), ("K1", 4096), ("K2", 0), ("N", 4096),
-        ("gate", 0), ("st", None), ("s", None)]])
+        ("gate", 0), ("st", None), ("ws", P), ("wsb", 1 << 30), ("s", None)]])
     assert ln(x1=None) == 1 and ln(w=None) == 1 and ln(out=None) == 1 and ln(K2=4096) == 1      # a second width without a second input
     assert ln(K1=100) == 2 and ln(K2=32, x2=P) == 2 and ln(N=12) == 2 and ln(N=0) == 2 and ln(R=-1) == 2
     assert ln(w=P + 4) == 4 and ln(res=P + 2) == 4
+    assert ln(ws=None) == 5 and ln(wsb=1024) == 5 and ln(ws=P + 16) == 5  # the shared-out K range needs its workspace
     assert ln(R=0) == 0
     lib.s4c_rmsnorm.argtypes = [vp, vp, f, i, i, vp, vp]
     rn = lambda **kw: lib.s4c_rmsnorm(*[kw.get(k, d) for k, d in [("x", P), ("g", P), ("eps", 1e-6), ("R", 4), ("H", 4096), ("out", P), ("s", None)]])

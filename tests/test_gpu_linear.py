@@ -24,7 +24,10 @@ def _f64(t):
 
 @pytest.mark.parametrize("R,K1,K2,N,bias,res", [(1, 64, 0, 8, False, False), (26, 256, 0, 384, True, False), (130, 128, 192, 200, True, True),
                                                (256, 512, 512, 1024, False, True), (33, 64, 64, 136, True, True),
-                                               (300, 320, 0, 4096, False, False)])
+                                               (300, 320, 0, 4096, False, False),
+                                               # few output tiles and a long K: the K range is shared out over CTAs
+                                               (26, 2048, 2048, 520, True, True), (130, 1536, 0, 136, False, True),
+                                               (26, 4096, 0, 4096, True, False), (5, 576, 0, 8, True, True)])
 def test_linear_against_the_oracle(R, K1, K2, N, bias, res):
     from paper_2506_14158_b200 import s4c
 
@@ -49,7 +52,8 @@ def test_linear_against_the_oracle(R, K1, K2, N, bias, res):
     assert (np.abs(_f64(out.t) - want) <= 2.0 ** -8 * np.abs(want) + slack + 1e-6).all()
 
 
-@pytest.mark.parametrize("R,K,N,res", [(26, 256, 704, False), (200, 128, 72, True), (64, 512, 1024, True)])
+@pytest.mark.parametrize("R,K,N,res", [(26, 256, 704, False), (200, 128, 72, True), (64, 512, 1024, True),
+                                       (26, 1024, 200, True), (140, 2048, 328, False)])  # the last two share the K range out
 def test_gated_linear_against_the_oracle(R, K, N, res):
     from paper_2506_14158_b200 import s4c
 
@@ -66,6 +70,24 @@ def test_gated_linear_against_the_oracle(R, K, N, res):
     slack = 8.0 * np.sqrt(K) * 2.0 ** -24 * np.linalg.norm(_f64(x), axis=1, keepdims=True) * np.linalg.norm(_f64(w), axis=1).max()
     bound = 2.0 ** -8 * np.abs(want) + slack * (1.1 * np.abs(u) + np.abs(g) + 1.0) + 1e-5
     assert (np.abs(_f64(out.t) - want) <= bound).all()
+
+
+def test_shared_out_k_range_is_reproducible_and_checks_its_workspace():
+    from paper_2506_14158_b200 import s4c
+
+    R, K, N = 26, 4096, 1024
+    assert s4c.linear_workspace_bytes(R, K, 0, N) > 0 and s4c.linear_workspace_bytes(R, K, 0, 64 * 1024) == 0
+    rng = np.random.default_rng(77)
+    x, w = _bf16(rng.standard_normal((R, K))).cuda(), _bf16(rng.standard_normal((N, K)) / 64.0).cuda()
+    ws = torch.empty(s4c.linear_workspace_bytes(R, K, 0, N), dtype=torch.uint8, device="cuda")
+    first = s4c.linear(x, w, workspace=ws).clone()
+    for _ in range(5):  # partial sums are added in a fixed order: the same bits every time
+        ws.fill_(0xFF)
+        assert torch.equal(s4c.linear(x, w, workspace=ws), first)
+    with pytest.raises(s4c.S4CError):
+        s4c.linear(x, w, workspace=ws[: ws.numel() // 2])
+    with pytest.raises(s4c.S4CError):
+        s4c.linear(x, w, workspace=ws[16:])
 
 
 def test_concatenation_meets_the_right_columns():
