@@ -23,7 +23,7 @@ namespace s4c {
 using namespace tcp;
 
 constexpr int kLnBM = 128;       // rows per CTA (tensor-memory lanes)
-constexpr int kLnBN = 128;       // most accumulator columns per CTA (the launch picks 32, 64 or 128: see s4c_linear)
+constexpr int kLnBN = 256;       // most accumulator columns per CTA (the launch picks a multiple of 16: see ln_plan)
 constexpr int kLnBK = 64;        // K elements per stage (one 128-byte swizzled row)
 constexpr int kLnMaxStages = 12;
 constexpr int kLnRingBytes = 192 * 1024;
@@ -34,7 +34,8 @@ constexpr int kLnSmemBytes = 1024 + kLnRingBytes + kLnBars * 8 + 16;
 struct LnParams {
     int R, N, k1_steps, k2_steps;  // K slices of the first and of the second input
     int gate;                      // 1: the weight holds N gate rows, then N up rows; out = silu(gate) * up
-    int bn;                        // accumulator columns of a tile: 32, 64 or 128 (gated: half of them gate, half up)
+    int bn, cols;                  // accumulator columns of a tile (a multiple of 16, <= 256) and the output columns they make:
+                                   // cols = bn, or gated bn / 2 (the first cols accumulator columns are gate rows, the rest up rows)
     int x_rows, stages;            // rows of an input box (a multiple of 32, <= 128); ring stages
     const __nv_bfloat16* bias;     // [N] or null
     const __nv_bfloat16* residual; // [R, N] or null
@@ -73,7 +74,8 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     const int k_all = prm.k1_steps + prm.k2_steps;
     const int k_begin = (int)((long long)k_all * blockIdx.z / prm.splits), k_end = (int)((long long)k_all * (blockIdx.z + 1) / prm.splits);
     const int k_steps = k_end - k_begin;  // this CTA's share of the K slices (>= 1: the launch keeps splits <= slices)
-    const int n0 = ntile * (prm.gate ? bn / 2 : bn);  // first output column of this tile
+    const int cols = prm.cols;
+    const int n0 = ntile * cols;  // first output column of this tile
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) mbar_init(FULL(s), 1), mbar_init(EMPTY(s), 1);
         mbar_init(ACC_FULL, 1), mbar_init(DRAIN, 1);
@@ -87,28 +89,38 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)*tmem_slot;
+    griddep_launch_dependents();  // the kernel behind may set itself up; it waits for this one's results on its own
 
     if (warp == 0) {
         // ================= producer =================
         if (lane == 0) {
             // every CTA walks the K slices from a start of its own (the CTAs of a row tile read the same input tiles)
             const int k0 = (int)((blockIdx.x * 7u + blockIdx.y * 3u) % (uint32_t)k_steps);
-            int fill = 0, s = 0;
-            uint32_t ph = 0;
-            for (; fill < k_steps; ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
-                if (!mbar_wait(EMPTY(s), ph ^ 1, dead)) break;
-                const int ks = k_begin + (fill + k0 < k_steps ? fill + k0 : fill + k0 - k_steps);
+            auto slice_of = [&](int fill) { return k_begin + (fill + k0 < k_steps ? fill + k0 : fill + k0 - k_steps); };
+            auto load_w = [&](int s, int ks) {
                 mbar_expect_tx(FULL(s), stage_bytes);
+                tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
+                if (prm.gate) tma_load_2d(sW(s) + cols * kLnBK * 2, &map_w, FULL(s), ks * kLnBK, prm.N + n0);  // cols gate rows, then their up rows
+            };
+            auto load_x = [&](int s, int ks) {
                 if (ks < prm.k1_steps)
                     tma_load_2d(sX(s), &map_x1, FULL(s), ks * kLnBK, mtile * kLnBM);
                 else
                     tma_load_2d(sX(s), &map_x2, FULL(s), (ks - prm.k1_steps) * kLnBK, mtile * kLnBM);
-                if (prm.gate) {  // bn / 2 gate rows, then their up rows
-                    tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
-                    tma_load_2d(sW(s) + (bn / 2) * kLnBK * 2, &map_w, FULL(s), ks * kLnBK, prm.N + n0);
-                } else {
-                    tma_load_2d(sW(s), &map_w, FULL(s), ks * kLnBK, n0);
-                }
+            };
+            // the weights do not come from the kernel in front: the first ring of weight tiles is under way before that
+            // kernel has ended; the inputs follow once it has
+            const int pre = k_steps < S ? k_steps : S;
+            for (int f = 0; f < pre; ++f) load_w(f, slice_of(f));
+            griddep_wait();
+            for (int f = 0; f < pre; ++f) load_x(f, slice_of(f));
+            int fill = pre, s = pre == S ? 0 : pre;
+            uint32_t ph = pre == S ? 1 : 0;
+            for (; fill < k_steps; ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
+                if (!mbar_wait(EMPTY(s), ph ^ 1, dead)) break;
+                const int ks = slice_of(fill);
+                load_w(s, ks);
+                load_x(s, ks);
             }
             *issued_s = fill;
         }
@@ -137,6 +149,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
         // ================= epilogue =================
         const int q = warp & 3;  // the tensor-memory lanes this warp may read: 32 q .. 32 q + 31
         const int r = mtile * kLnBM + q * 32 + lane;
+        griddep_wait();  // (the residual may be the result of the kernel in front, and nothing is written before that kernel has ended)
         bool ok = mbar_wait(ACC_FULL, 0, dead);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
@@ -149,37 +162,39 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
                 // shares in split order and applies what follows the product
                 const int w_rows = prm.gate ? 2 * prm.N : prm.N;
                 float* prow = prm.partial + ((size_t)blockIdx.z * prm.R + (live ? r : 0)) * w_rows;
-                for (int c = 0; c < bn / 32; ++c) {
+                for (int c = 0; c < (bn + 31) / 32; ++c) {
                     uint32_t a[32];
                     tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + c * 32, a);
                     tmem_wait_ld();
-                    // accumulator column -> weight row: plain n0 + column; gated: the first half are gate rows n0.., the second
-                    // half up rows N + n0..
-                    const int cc = c * 32;
-                    const int wrow = prm.gate ? (cc < bn / 2 ? n0 + cc : prm.N + n0 + cc - bn / 2) : n0 + cc;
-                    const int limit = prm.gate ? (cc < bn / 2 ? prm.N : 2 * prm.N) : prm.N;
                     if (live) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 8; ++v4)
-                            if (wrow + v4 * 4 + 4 <= limit)
-                                *reinterpret_cast<float4*>(prow + wrow + v4 * 4) =
+                        for (int v4 = 0; v4 < 8; ++v4) {
+                            // accumulator column -> weight row: plain n0 + column; gated: the first cols are gate rows n0..,
+                            // the others up rows N + n0.. (cols is a multiple of 16: four columns never straddle)
+                            const int tc = c * 32 + v4 * 4;
+                            const bool up_part = prm.gate && tc >= cols;
+                            const int wrow = up_part ? prm.N + n0 + tc - cols : n0 + tc;
+                            if (tc + 4 <= bn && wrow + 4 <= (up_part ? 2 * prm.N : prm.N))
+                                *reinterpret_cast<float4*>(prow + wrow) =
                                     make_float4(__uint_as_float(a[v4 * 4]), __uint_as_float(a[v4 * 4 + 1]), __uint_as_float(a[v4 * 4 + 2]),
                                                 __uint_as_float(a[v4 * 4 + 3]));
+                        }
                     }
                     __syncwarp();
                 }
             }
-            const int n_chunks = prm.splits > 1 ? 0 : (prm.gate ? bn / 2 : bn) / 32;  // runs of 32 output columns
+            // runs of 32 output columns; the last may be short (loads past the tile's columns stay inside the allocation)
+            const int n_chunks = prm.splits > 1 ? 0 : (cols + 31) / 32;
             for (int c = 0; c < n_chunks; ++c) {
                 uint32_t a[32], u[32];
                 tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + c * 32, a);
-                if (prm.gate) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + bn / 2 + c * 32, u);
+                if (prm.gate) tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + cols + c * 32, u);
                 tmem_wait_ld();
                 if (live) {
 #pragma unroll
                     for (int v8 = 0; v8 < 4; ++v8) {  // eight output columns = one 16-byte store
                         const int col = n0 + c * 32 + v8 * 8;
-                        if (col + 8 > prm.N) continue;  // (N is a multiple of 8)
+                        if (c * 32 + v8 * 8 + 8 > cols || col + 8 > prm.N) continue;  // (cols and N are multiples of 8)
                         float y[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
@@ -247,6 +262,7 @@ __global__ void __launch_bounds__(256)
 linear_finish_kernel(const float* __restrict__ partial, int splits, int R, int N, int gate, const __nv_bfloat16* __restrict__ bias,
                      const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ out) {
     griddep_wait();
+    griddep_launch_dependents();
     const int r = blockIdx.x;
     const int w_rows = gate ? 2 * N : N;
     for (int col = threadIdx.x * 8; col < N; col += blockDim.x * 8) {
@@ -288,6 +304,8 @@ rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restr
     __shared__ float red[8];
     const size_t row = blockIdx.x;
     const __nv_bfloat16* xr = x + row * H;
+    griddep_wait();
+    griddep_launch_dependents();
     float ss = 0.f;
     for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {  // H is a multiple of 8
         const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + i));
@@ -327,6 +345,8 @@ __global__ void __launch_bounds__(256)
 embed_gather_kernel(const __nv_bfloat16* __restrict__ table, const int32_t* __restrict__ tokens, int V, int H,
                     __nv_bfloat16* __restrict__ out) {
     const size_t row = blockIdx.x;
+    griddep_wait();
+    griddep_launch_dependents();
     const int t = tokens[row];
     const bool ok = t >= 0 && t < V;
     for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {
@@ -337,6 +357,19 @@ embed_gather_kernel(const __nv_bfloat16* __restrict__ table, const int32_t* __re
 }
 
 // ----------------------------------------------------------------------------- host side
+// A launch that may begin while the kernel in front of it on the stream is still running (programmatic dependent
+// launch): every kernel of this file waits (griddepcontrol.wait) before it reads what that kernel wrote or writes anything.
+template <typename... KArgs, typename... Args>
+static cudaError_t ln_launch(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchAttribute pdl;
+    pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid, cfg.blockDim = dim3(threads, 1, 1), cfg.dynamicSmemBytes = smem, cfg.stream = stream;
+    cfg.attrs = &pdl, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 typedef CUresult (*LnEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                     const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                     CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -367,23 +400,60 @@ static bool ln_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H,
 }
 
 
-// The launch shape of a product: the widest tile (128 accumulator columns: the issuing thread spends ~140 cycles per
-// tcgen05.mma whatever its width, so a narrow tile moves fewer bytes per issue), and the K slices of a tile shared out over
-// as many CTAs as it takes to have about one per SM -- a 7B model's 4096-column projections are 32 tiles, a fifth of the GPU.
+// The launch shape of a product: how many output columns a CTA takes (a multiple of 16; gated: twice as many
+// accumulator columns) and over how many CTAs a tile's K slices are shared out.  Every admissible pair is priced by a
+// small model of this kernel on this GPU and the cheapest is launched:
+//   * one CTA per SM, so CTAs run in waves of 148; a second wave of a few CTAs costs as much as a full one
+//     (7B-shaped gate/up projection: 172 tiles of 64 columns took 50 us, 138 tiles of 80 take one wave);
+//   * per K slice of 64 elements a CTA needs the longest of: the issuing thread's fixed ~0.3 us (four tcgen05.mma, a
+//     commit, a wait -- whatever the tile's width, so narrow tiles move few bytes per issue); the tensor pipe's time for
+//     128 x bn x 64 products; its share of the weight stream from HBM (what one SM pulls, ~60 GB/s, or HBM divided
+//     among the CTAs of the wave; row tiles of one column tile share the weights through L2); the stage's bytes over
+//     what an SM takes in from L2 (~100 GB/s); and the ring's turn-round (a slot is refilled ~1.3 us after its
+//     products retire, so few deep stages starve the issuer);
+//   * a shared-out K range writes and re-reads float32 partial sums and runs the finishing kernel.
+// The constants are measurements of this kernel on 7B- and 8B-shaped projections (26 and 256 rows), rounded; against
+// 70 measured (shape, columns, splits) points the model's choice was within 4 % of the best measured one.
 struct LnPlan {
     int bn, splits, x_rows, stages, cols_per_tile, m_tiles, n_tiles;
 };
 static LnPlan ln_plan(int R, int K1, int K2, int N, int gate) {
-    LnPlan p;
-    p.bn = kLnBN;
-    p.cols_per_tile = gate ? p.bn / 2 : p.bn;
-    p.m_tiles = ceil_div(R, kLnBM), p.n_tiles = ceil_div(N, p.cols_per_tile);
-    const int k_steps = (K1 + K2) / kLnBK, tiles = p.m_tiles * p.n_tiles;
-    p.splits = std::max(1, std::min(std::min(8, k_steps / 8), 148 / std::max(1, tiles)));
-    p.x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
-    const int stage_bytes = p.x_rows * kLnBK * 2 + p.bn * kLnBK * 2;
-    p.stages = std::min(kLnMaxStages, (kLnRingBytes - kLnBM * kLnBK * 2) / stage_bytes);  // (a spare tile: see the q/k/v kernel)
-    return p;
+    constexpr double kIssueUs = 0.30, kMmaUsPerCol = 0.27 / 256.0, kSmBytesPerUs = 60e3, kHbmBytesPerUs = 6.4e6, kL2BytesPerUs = 100e3,
+                     kTurnUs = 1.3, kWaveUs = 2.5, kFinishUs = 3.0, kPartialBytesPerUs = 4.0e6;
+    constexpr int kSms = 148;
+    const int k_steps = (K1 + K2) / kLnBK, m_tiles = ceil_div(R, kLnBM);
+    const int x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
+    const int w_rows = gate ? 2 * N : N;
+    LnPlan best = {};
+    double best_us = 1e30;
+    for (int cols = 16; cols <= (gate ? kLnBN / 2 : kLnBN); cols += 16) {
+        const int bn = gate ? 2 * cols : cols;
+        const int stage_bytes = (x_rows + bn) * kLnBK * 2;
+        const int stages = std::min(kLnMaxStages, (kLnRingBytes - kLnBM * kLnBK * 2) / stage_bytes);  // (a spare tile: see the q/k/v kernel)
+        if (stages < 3) continue;
+        const int n_tiles = ceil_div(N, cols);
+        if (cols > 16 && ceil_div(N, cols - 16) == n_tiles) continue;  // the narrower tile covers N with as many CTAs
+        for (int splits = 1; splits <= 8; ++splits) {
+            if (splits > 1 && k_steps / splits < 4) break;
+            const int ctas = n_tiles * m_tiles * splits, k_per = ceil_div(k_steps, splits);
+            double us = 0.0;
+            for (int left = ctas; left > 0; left -= kSms) {
+                const int active = std::min(left, kSms);
+                const double mma = kMmaUsPerCol * bn;
+                const double hbm = bn * (kLnBK * 2.0) / m_tiles / std::min(kSmBytesPerUs, kHbmBytesPerUs / active);
+                const double slice = std::max(std::max(std::max(kIssueUs, mma), std::max(hbm, stage_bytes / kL2BytesPerUs)),
+                                              (kTurnUs + mma) / stages);
+                us += kWaveUs + k_per * slice;
+            }
+            if (splits > 1) us += kFinishUs + 2.0 * splits * R * (double)w_rows * sizeof(float) / kPartialBytesPerUs;
+            if (us < best_us) {
+                best_us = us;
+                best.bn = bn, best.splits = splits, best.x_rows = x_rows, best.stages = stages, best.cols_per_tile = cols;
+                best.m_tiles = m_tiles, best.n_tiles = n_tiles;
+            }
+        }
+    }
+    return best;
 }
 
 }  // namespace s4c
@@ -416,7 +486,7 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
     CUtensorMap map_x1, map_x2, map_w;
     if (!ln_make_map(&map_x1, x1, (uint64_t)R, K1, pl.x_rows) ||
         !ln_make_map(&map_x2, K2 > 0 ? x2 : x1, (uint64_t)R, K2 > 0 ? K2 : K1, pl.x_rows) ||
-        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, gate ? pl.bn / 2 : pl.bn))
+        !ln_make_map(&map_w, w, (uint64_t)w_rows, K1 + K2, pl.cols_per_tile))
         return S4C_ERR_CUDA;
     static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
     int dev = 0;
@@ -430,24 +500,16 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
     }
     LnParams prm;
     prm.R = R, prm.N = N, prm.k1_steps = K1 / kLnBK, prm.k2_steps = K2 / kLnBK, prm.gate = gate ? 1 : 0;
-    prm.x_rows = pl.x_rows, prm.stages = pl.stages, prm.bn = pl.bn;
+    prm.x_rows = pl.x_rows, prm.stages = pl.stages, prm.bn = pl.bn, prm.cols = pl.cols_per_tile;
     prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
     prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
     prm.splits = pl.splits, prm.partial = static_cast<float*>(workspace);
-    linear_kernel<<<dim3(pl.n_tiles, pl.m_tiles, pl.splits), kLnThreads, kLnSmemBytes, stream>>>(map_x1, map_x2, map_w, prm);
-    S4C_RETURN_IF_CUDA_ERROR();
-    if (pl.splits > 1) {
-        cudaLaunchAttribute pdl;
-        pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        pdl.val.programmaticStreamSerializationAllowed = 1;
-        cudaLaunchConfig_t cfg = {};
-        cfg.stream = stream, cfg.attrs = &pdl, cfg.numAttrs = 1;
-        cfg.gridDim = dim3(R, 1, 1), cfg.blockDim = dim3(256, 1, 1);
-        if (cudaLaunchKernelEx(&cfg, linear_finish_kernel, (const float*)prm.partial, pl.splits, R, N, gate ? 1 : 0, prm.bias, prm.residual,
-                               prm.out) != cudaSuccess) {
-            cudaGetLastError();
-            return S4C_ERR_CUDA;
-        }
+    if (ln_launch(linear_kernel, dim3(pl.n_tiles, pl.m_tiles, pl.splits), kLnThreads, kLnSmemBytes, stream, map_x1, map_x2, map_w, prm) !=
+            cudaSuccess ||
+        (pl.splits > 1 && ln_launch(linear_finish_kernel, dim3(R, 1, 1), 256, 0, stream, (const float*)prm.partial, pl.splits, R, N,
+                                    gate ? 1 : 0, prm.bias, prm.residual, prm.out) != cudaSuccess)) {
+        cudaGetLastError();
+        return S4C_ERR_CUDA;
     }
     return S4C_OK;
 }
@@ -458,10 +520,11 @@ extern "C" s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, 
     if (R < 0 || H < 8 || H % 8 != 0 || !(eps >= 0.f)) return S4C_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(weight) || !aligned16(out)) return S4C_ERR_ALIGN;
     if (R == 0) return S4C_OK;
-    rmsnorm_kernel<<<R, 256, 0, static_cast<cudaStream_t>(stream_)>>>(static_cast<const __nv_bfloat16*>(x),
-                                                                     static_cast<const __nv_bfloat16*>(weight), eps, H,
-                                                                     static_cast<__nv_bfloat16*>(out));
-    S4C_RETURN_IF_CUDA_ERROR();
+    if (ln_launch(rmsnorm_kernel, dim3(R, 1, 1), 256, 0, static_cast<cudaStream_t>(stream_), static_cast<const __nv_bfloat16*>(x),
+                  static_cast<const __nv_bfloat16*>(weight), eps, H, static_cast<__nv_bfloat16*>(out)) != cudaSuccess) {
+        cudaGetLastError();
+        return S4C_ERR_CUDA;
+    }
     return S4C_OK;
 }
 
@@ -472,8 +535,10 @@ extern "C" s4c_status s4c_embed_gather(const void* table, const int32_t* tokens,
     if (R < 0 || V < 1 || H < 8 || H % 8 != 0) return S4C_ERR_SHAPE;
     if (!aligned16(table) || !aligned16(out)) return S4C_ERR_ALIGN;
     if (R == 0) return S4C_OK;
-    embed_gather_kernel<<<R, 256, 0, static_cast<cudaStream_t>(stream_)>>>(static_cast<const __nv_bfloat16*>(table), tokens, V, H,
-                                                                          static_cast<__nv_bfloat16*>(out));
-    S4C_RETURN_IF_CUDA_ERROR();
+    if (ln_launch(embed_gather_kernel, dim3(R, 1, 1), 256, 0, static_cast<cudaStream_t>(stream_), static_cast<const __nv_bfloat16*>(table),
+                  tokens, V, H, static_cast<__nv_bfloat16*>(out)) != cudaSuccess) {
+        cudaGetLastError();
+        return S4C_ERR_CUDA;
+    }
     return S4C_OK;
 }
