@@ -589,7 +589,7 @@ def roofline_records(cfg, args, rec, pk):
         breakdown["drafter_head_not_in_step"] = dr["ms"]
         t = dr["ms"] * 1e-3
         roofline["drafter_head"] = dict(
-            kernel="one drafter head, Eq. 3-6: embed, Linear(concat[e,f]), decoder layer, LM-head top-k (11 calls)", rows=dr["rows"],
+            kernel="one drafter head, Eq. 3-6: embed, Linear(concat[e,f]), decoder layer, LM-head top-k (9 calls)", rows=dr["rows"],
             mlp_width=dr["inter"], top_k=dr["k"], us=dr["ms"] * 1e3, weight_bytes=dr["weight_bytes"],
             bound="tensor" if dr["flops"] / dr["weight_bytes"] >= ridge else "hbm", gbs=dr["weight_bytes"] / t * 1e-9,
             frac_of_hbm_peak=dr["weight_bytes"] / t * 1e-9 / pk["hbm_gbs"], tflops=dr["flops"] / t * 1e-12,

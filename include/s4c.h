@@ -340,6 +340,13 @@ s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_l
  *                   timing): workspace must hold s4c_linear_workspace_bytes(R, K1, K2, N, gate)
  *                   bytes (0 for shapes that need none; then NULL is accepted), 256-byte aligned;
  *                   S4C_ERR_WORKSPACE otherwise.
+ *   s4c_linear_rmsnorm  the ungated s4c_linear followed by norm_out[r, :] = rmsnorm(out[r, :]) with
+ *                   norm_weight [N] and eps >= 0 (norm_out [R, N] bf16, 16-byte aligned): the decoder
+ *                   layer's "projection + residual, then the next block's normalisation".  Both out
+ *                   and norm_out are written; the results equal, bit for bit, s4c_linear followed by
+ *                   s4c_rmsnorm on out.  Where the K range is shared out the finishing kernel, which
+ *                   holds whole rows, normalises them (no extra launch); otherwise the
+ *                   normalisation kernel is launched behind the product.
  *   s4c_rmsnorm     out[r, :] = x[r, :] / sqrt(mean(x[r, :]^2) + eps) * weight   (bf16 in / out,
  *                   float32 arithmetic; H a multiple of 8)
  *   s4c_embed_gather out[r, :] = table[tokens[r], :]  (Eq. 6; bf16 table [V, H]; a token outside
@@ -350,6 +357,11 @@ size_t s4c_linear_workspace_bytes(int R, int K1, int K2, int N, int gate);
 s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
                       void* out, int R, int K1, int K2, int N, int gate, int32_t* status, void* workspace,
                       size_t workspace_bytes, s4c_stream_t stream);
+
+s4c_status s4c_linear_rmsnorm(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
+                              void* out, int R, int K1, int K2, int N, const void* norm_weight, float eps,
+                              void* norm_out, int32_t* status, void* workspace, size_t workspace_bytes,
+                              s4c_stream_t stream);
 
 s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, int R, int H, void* out, s4c_stream_t stream);
 

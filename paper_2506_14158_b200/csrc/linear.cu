@@ -256,15 +256,54 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     }
 }
 
+// The root-mean-square normalisation's two steps, shared by rmsnorm_kernel and by the finishing kernel that normalises the
+// row it has just written, so that the fused and the separate form give the same bits: a thread's share of the sum of
+// squares (explicit fused multiply-adds, columns ascending), the CTA's sum (warps in order), the scaled row.
+__device__ __forceinline__ float sumsq8(float ss, const uint4& v) {
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(p[j]);
+        ss = __fmaf_rn(f.y, f.y, __fmaf_rn(f.x, f.x, ss));
+    }
+    return ss;
+}
+__device__ __forceinline__ float cta_sum_256(float ss, float* red) {  // 256 threads; red: 8 floats of shared memory
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    return tot;
+}
+__device__ __forceinline__ uint4 scale8(const uint4& v, const uint4& g, float scale) {
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+    const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g);
+    uint32_t pk[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(p[j]), w2 = __bfloat1622float2(pg[j]);
+        const __nv_bfloat162 o2 = __floats2bfloat162_rn(f.x * scale * w2.x, f.y * scale * w2.y);
+        pk[j] = *reinterpret_cast<const uint32_t*>(&o2);
+    }
+    return make_uint4(pk[0], pk[1], pk[2], pk[3]);
+}
+
 // After a product whose K slices were shared out: per output element the shares in split order, then bias, gate,
-// residual, one rounding to bf16.  grid (rows), eight columns per thread at a time.
+// residual, one rounding to bf16.  grid (rows), eight columns per thread at a time.  With norm_weight the CTA, which
+// holds the whole row, also writes its root-mean-square normalisation (of the rounded row, as a separate call would).
 __global__ void __launch_bounds__(256)
 linear_finish_kernel(const float* __restrict__ partial, int splits, int R, int N, int gate, const __nv_bfloat16* __restrict__ bias,
-                     const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ out) {
+                     const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ out,
+                     const __nv_bfloat16* __restrict__ norm_weight, float norm_eps, __nv_bfloat16* __restrict__ norm_out) {
+    __shared__ float red[8];
     griddep_wait();
     griddep_launch_dependents();
     const int r = blockIdx.x;
     const int w_rows = gate ? 2 * N : N;
+    float ss = 0.f;
     for (int col = threadIdx.x * 8; col < N; col += blockDim.x * 8) {
         float y[8], up[8];
 #pragma unroll
@@ -293,7 +332,17 @@ linear_finish_kernel(const float* __restrict__ partial, int splits, int R, int N
             const __nv_bfloat162 p2 = __floats2bfloat162_rn(y[2 * j], y[2 * j + 1]);
             pk[j] = *reinterpret_cast<const uint32_t*>(&p2);
         }
-        *reinterpret_cast<uint4*>(out + (size_t)r * N + col) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        const uint4 packed = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(out + (size_t)r * N + col) = packed;
+        ss = sumsq8(ss, packed);
+    }
+    if (norm_weight) {  // (uniform over the CTA)
+        const float scale = rsqrtf(cta_sum_256(ss, red) / (float)N + norm_eps);
+        for (int col = threadIdx.x * 8; col < N; col += blockDim.x * 8) {
+            const uint4 v = *reinterpret_cast<const uint4*>(out + (size_t)r * N + col);  // this thread's own stores
+            const uint4 g = __ldg(reinterpret_cast<const uint4*>(norm_weight + col));
+            *reinterpret_cast<uint4*>(norm_out + (size_t)r * N + col) = scale8(v, g, scale);
+        }
     }
 }
 
@@ -307,36 +356,13 @@ rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restr
     griddep_wait();
     griddep_launch_dependents();
     float ss = 0.f;
-    for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {  // H is a multiple of 8
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + i));
-        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 f = __bfloat1622float2(p[j]);
-            ss += f.x * f.x + f.y * f.y;
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
-    const float scale = rsqrtf(tot / (float)H + eps);
+    for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8)  // H is a multiple of 8
+        ss = sumsq8(ss, __ldg(reinterpret_cast<const uint4*>(xr + i)));
+    const float scale = rsqrtf(cta_sum_256(ss, red) / (float)H + eps);
     for (int i = threadIdx.x * 8; i < H; i += blockDim.x * 8) {
         const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + i));
         const uint4 g = __ldg(reinterpret_cast<const uint4*>(weight + i));
-        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
-        const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g);
-        uint32_t pk[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 f = __bfloat1622float2(p[j]), w2 = __bfloat1622float2(pg[j]);
-            const __nv_bfloat162 o2 = __floats2bfloat162_rn(f.x * scale * w2.x, f.y * scale * w2.y);
-            pk[j] = *reinterpret_cast<const uint32_t*>(&o2);
-        }
-        *reinterpret_cast<uint4*>(out + row * H + i) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(out + row * H + i) = scale8(v, g, scale);
     }
 }
 
@@ -465,13 +491,16 @@ extern "C" size_t s4c_linear_workspace_bytes(int R, int K1, int K2, int N, int g
     return p.splits > 1 ? round_up((size_t)p.splits * R * (gate ? 2 * N : N) * sizeof(float), 256) : 0;
 }
 
-extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
-                                 void* out, int R, int K1, int K2, int N, int gate, int32_t* status, void* workspace,
-                                 size_t workspace_bytes, s4c_stream_t stream_) {
-    using namespace s4c;
-    if (!x1 || !w || !out || (K2 > 0 && !x2)) return S4C_ERR_NULL;
+namespace s4c {
+// s4c_linear, and s4c_linear_rmsnorm when norm_weight is given (norm_out = rmsnorm(out))
+static s4c_status ln_run(const void* x1, const void* x2, const void* w, const void* bias, const void* residual, void* out, int R,
+                         int K1, int K2, int N, int gate, const void* norm_weight, float norm_eps, void* norm_out, int32_t* status,
+                         void* workspace, size_t workspace_bytes, s4c_stream_t stream_) {
+    if (!x1 || !w || !out || (K2 > 0 && !x2) || (norm_weight && !norm_out)) return S4C_ERR_NULL;
     if (R < 0 || N < 8 || N % 8 != 0 || K1 < kLnBK || K1 % kLnBK != 0 || K2 < 0 || K2 % kLnBK != 0) return S4C_ERR_SHAPE;
-    if (!aligned16(x1) || !aligned16(w) || !aligned16(out) || (x2 && !aligned16(x2)) || (residual && !aligned16(residual)))
+    if (norm_weight && !(norm_eps >= 0.f)) return S4C_ERR_SHAPE;
+    if (!aligned16(x1) || !aligned16(w) || !aligned16(out) || (x2 && !aligned16(x2)) || (residual && !aligned16(residual)) ||
+        (norm_weight && (!aligned16(norm_weight) || !aligned16(norm_out))))
         return S4C_ERR_ALIGN;
     if (R == 0) return S4C_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -504,14 +533,36 @@ extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, 
     prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
     prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
     prm.splits = pl.splits, prm.partial = static_cast<float*>(workspace);
-    if (ln_launch(linear_kernel, dim3(pl.n_tiles, pl.m_tiles, pl.splits), kLnThreads, kLnSmemBytes, stream, map_x1, map_x2, map_w, prm) !=
-            cudaSuccess ||
-        (pl.splits > 1 && ln_launch(linear_finish_kernel, dim3(R, 1, 1), 256, 0, stream, (const float*)prm.partial, pl.splits, R, N,
-                                    gate ? 1 : 0, prm.bias, prm.residual, prm.out) != cudaSuccess)) {
+    const __nv_bfloat16* nw = static_cast<const __nv_bfloat16*>(norm_weight);
+    __nv_bfloat16* no = static_cast<__nv_bfloat16*>(norm_out);
+    bool ok = ln_launch(linear_kernel, dim3(pl.n_tiles, pl.m_tiles, pl.splits), kLnThreads, kLnSmemBytes, stream, map_x1, map_x2, map_w,
+                        prm) == cudaSuccess;
+    if (ok && pl.splits > 1)  // the finishing kernel holds whole rows: it normalises them as well
+        ok = ln_launch(linear_finish_kernel, dim3(R, 1, 1), 256, 0, stream, (const float*)prm.partial, pl.splits, R, N, gate ? 1 : 0,
+                       prm.bias, prm.residual, prm.out, nw, norm_eps, no) == cudaSuccess;
+    else if (ok && nw)
+        ok = ln_launch(rmsnorm_kernel, dim3(R, 1, 1), 256, 0, stream, (const __nv_bfloat16*)prm.out, nw, norm_eps, N, no) == cudaSuccess;
+    if (!ok) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
     return S4C_OK;
+}
+}  // namespace s4c
+
+extern "C" s4c_status s4c_linear(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
+                                 void* out, int R, int K1, int K2, int N, int gate, int32_t* status, void* workspace,
+                                 size_t workspace_bytes, s4c_stream_t stream) {
+    return s4c::ln_run(x1, x2, w, bias, residual, out, R, K1, K2, N, gate, nullptr, 0.f, nullptr, status, workspace, workspace_bytes,
+                       stream);
+}
+
+extern "C" s4c_status s4c_linear_rmsnorm(const void* x1, const void* x2, const void* w, const void* bias, const void* residual,
+                                         void* out, int R, int K1, int K2, int N, const void* norm_weight, float eps, void* norm_out,
+                                         int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream) {
+    if (!norm_weight) return S4C_ERR_NULL;
+    return s4c::ln_run(x1, x2, w, bias, residual, out, R, K1, K2, N, 0, norm_weight, eps, norm_out, status, workspace, workspace_bytes,
+                       stream);
 }
 
 extern "C" s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, int R, int H, void* out, s4c_stream_t stream_) {

@@ -1,13 +1,13 @@
 """One head of the multi-head drafter (Section 3.1.1, Eq. 3-6), composed from the library's entry points.
 
     e = Embedding(t)                                   s4c_embed_gather           (Eq. 6)
-    h = Linear(concat[e, f])                           s4c_linear, two inputs     (Eq. 3)
+    h = Linear(concat[e, f])                           s4c_linear_rmsnorm, two inputs (Eq. 3)
     f' = Decoder_layer(h)                                                         (Eq. 4; one LLaMA-family layer)
-         a  = rmsnorm(h)                               s4c_rmsnorm
+         a  = rmsnorm(h)                               (the same call)
          q, K/V tree slots = rope(a Wqkv^T)            s4c_qkv_rope
          o  = tree attention(q, cache)                 s4c_tree_attention
-         h2 = h + o Wo^T                               s4c_linear, residual
-         f' = h2 + (silu(m Wg^T) * m Wu^T) Wd^T,  m = rmsnorm(h2)      s4c_rmsnorm, s4c_linear (gated), s4c_linear (residual)
+         h2 = h + o Wo^T,  m = rmsnorm(h2)             s4c_linear_rmsnorm, residual
+         f' = h2 + (silu(m Wg^T) * m Wu^T) Wd^T        s4c_linear (gated), s4c_linear (residual)
     ranked choices = top-k(LM_head(f'))                s4c_lm_head_topk           (Eq. 5; k = 1 is the Argmax)
 
 Only buffers, views and the order of the calls live here; every arithmetic step runs in the library's kernels.  The one
@@ -91,15 +91,14 @@ class DrafterHead:
         Returns dict(token [B*T,k], logit [B*T,k], features [B*T,H])."""
         w = self.w
         s4c.embed_gather(w.embedding, tokens.reshape(-1), out=self.e)
-        s4c.linear(self.e, w.fc, x2=features, bias=w.fc_bias, out=self.h, workspace=self.ws_lin)
-        s4c.rmsnorm(self.h, w.norm1, self.eps, out=self.a)
+        s4c.linear_rmsnorm(self.e, w.fc, w.norm1, self.eps, x2=features, bias=w.fc_bias, out=self.h, norm_out=self.a,
+                           workspace=self.ws_lin)
         s4c.qkv_rope(self.a.view(self.B, self.T, -1), w.qkv, cache_len, parent, self.q, k_cache, v_cache, n_nodes, self.rope_theta,
                      status=self.status_qkv, workspace=self.ws_qkv)
         s4c.tree_attention(self.q, k_cache, v_cache, cache_len, parent, n_nodes, out=self.attn, status=self.status_attn,
                            workspace=self.ws_attn, max_cache_len=max_cache_len)
         self.o_in.view(self.B, self.T, self.Hq, self.d).copy_(self.attn.permute(0, 2, 1, 3))  # rows for the output projection
-        s4c.linear(self.o_in, w.o, residual=self.h, out=self.h2, workspace=self.ws_lin)
-        s4c.rmsnorm(self.h2, w.norm2, self.eps, out=self.m)
+        s4c.linear_rmsnorm(self.o_in, w.o, w.norm2, self.eps, residual=self.h, out=self.h2, norm_out=self.m, workspace=self.ws_lin)
         s4c.linear(self.m, w.gate_up, gate=True, out=self.act, workspace=self.ws_lin)
         s4c.linear(self.act, w.down, residual=self.h2, out=self.f_out, workspace=self.ws_lin)
         s4c.lm_head_topk(self.f_out, w.lm_head, self.k, token=self.token, logit=self.logit, status=self.status_head,

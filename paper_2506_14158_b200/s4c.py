@@ -26,7 +26,7 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
            "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
            "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
-           "s4c_tree_build_topk", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_rmsnorm", "s4c_embed_gather"]
+           "s4c_tree_build_topk", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_linear_rmsnorm", "s4c_rmsnorm", "s4c_embed_gather"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -94,6 +94,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_linear_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.s4c_linear.restype = i
     lib.s4c_linear.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i32p, vp, sz, vp]
+    lib.s4c_linear_rmsnorm.restype = i
+    lib.s4c_linear_rmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, vp, i32p, vp, sz, vp]
     lib.s4c_rmsnorm.restype = i
     lib.s4c_rmsnorm.argtypes = [vp, vp, f, i, i, vp, vp]
     lib.s4c_embed_gather.restype = i
@@ -555,6 +557,27 @@ def linear(x1, w, x2=None, bias=None, residual=None, gate: bool = False, out=Non
     if rc:
         raise S4CError("s4c_linear", rc)
     return out
+
+
+def linear_rmsnorm(x1, w, norm_weight, eps: float = 1e-6, x2=None, bias=None, residual=None, out=None, norm_out=None, status=None,
+                   workspace=None, stream=None):
+    """s4c_linear_rmsnorm: out as s4c_linear (ungated), norm_out = rmsnorm(out) with norm_weight; returns (out, norm_out)."""
+    R, K1 = x1.shape
+    K2 = 0 if x2 is None else x2.shape[1]
+    N = w.shape[0]
+    bf = torch.bfloat16
+    out = torch.empty(R, N, dtype=bf, device=x1.device) if out is None else out
+    norm_out = torch.empty(R, N, dtype=bf, device=x1.device) if norm_out is None else norm_out
+    if workspace is None:
+        workspace = _workspace(int(_lib.s4c_linear_workspace_bytes(R, K1, K2, N, 0)), x1.device, "linear")
+    rc = _lib.s4c_linear_rmsnorm(_dev(x1, bf, "x1"), _dev(x2, bf, "x2"), _dev(w, bf, "w"), _dev(bias, bf, "bias"),
+                                 _dev(residual, bf, "residual"), _dev(out, bf, "out"), R, K1, K2, N,
+                                 _dev(norm_weight, bf, "norm_weight"), float(eps), _dev(norm_out, bf, "norm_out"),
+                                 _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
+                                 0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if rc:
+        raise S4CError("s4c_linear_rmsnorm", rc)
+    return out, norm_out
 
 
 def rmsnorm(x, weight, eps: float = 1e-6, out=None, stream=None):

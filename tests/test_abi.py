@@ -195,6 +195,12 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert ln(w=P + 4) == 4 and ln(res=P + 2) == 4
     assert ln(ws=None) == 5 and ln(wsb=1024) == 5 and ln(ws=P + 16) == 5  # the shared-out K range needs its workspace
     assert ln(R=0) == 0
+    lib.s4c_linear_rmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, f, vp, vp, vp, ctypes.c_size_t, vp]
+    lnr = lambda **kw: lib.s4c_linear_rmsnorm(*[kw.get(k, d) for k, d in [
+        ("x1", P), ("x2", None), ("w", P), ("b", None), ("res", None), ("out", P), ("R", 26), ("K1", 4096), ("K2", 0), ("N", 4096),
+        ("g", P), ("eps", 1e-5), ("no", P), ("st", None), ("ws", P), ("wsb", 1 << 30), ("s", None)]])
+    assert lnr(g=None) == 1 and lnr(no=None) == 1 and lnr(x1=None) == 1
+    assert lnr(eps=-1.0) == 2 and lnr(N=12) == 2 and lnr(g=P + 2) == 4 and lnr(no=P + 8) == 4 and lnr(ws=None) == 5 and lnr(R=0) == 0
     lib.s4c_rmsnorm.argtypes = [vp, vp, f, i, i, vp, vp]
     rn = lambda **kw: lib.s4c_rmsnorm(*[kw.get(k, d) for k, d in [("x", P), ("g", P), ("eps", 1e-6), ("R", 4), ("H", 4096), ("out", P), ("s", None)]])
     assert rn(x=None) == 1 and rn(H=12) == 2 and rn(eps=-1.0) == 2 and rn(g=P + 2) == 4 and rn(R=0) == 0

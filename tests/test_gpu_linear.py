@@ -90,6 +90,27 @@ def test_shared_out_k_range_is_reproducible_and_checks_its_workspace():
         s4c.linear(x, w, workspace=ws[16:])
 
 
+@pytest.mark.parametrize("R,K1,K2,N", [(26, 4096, 0, 1024), (26, 512, 512, 520), (140, 128, 0, 264), (3, 2048, 0, 8)])
+def test_linear_with_the_normalisation_of_its_result(R, K1, K2, N):
+    # both the row-holding finishing kernel (K range shared out) and the separate launch behind the product: the same bits as
+    # the two calls one after the other, and the oracle's two steps within the usual bound
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(R + N)
+    K = K1 + K2
+    x1, x2 = _bf16(rng.standard_normal((R, K1))).cuda(), (_bf16(rng.standard_normal((R, K2))).cuda() if K2 else None)
+    w, b = _bf16(rng.standard_normal((N, K)) / np.sqrt(K)).cuda(), _bf16(rng.standard_normal(N)).cuda()
+    rs, g = _bf16(rng.standard_normal((R, N))).cuda(), _bf16(1.0 + 0.1 * rng.standard_normal(N)).cuda()
+    out, nrm = Guarded((R, N), torch.bfloat16, fill=-3.0), Guarded((R, N), torch.bfloat16, fill=-3.0)
+    s4c.linear_rmsnorm(x1, w, g, 1e-5, x2=x2, bias=b, residual=rs, out=out.t, norm_out=nrm.t)
+    torch.cuda.synchronize()
+    out.check("s4c_linear_rmsnorm out"), nrm.check("s4c_linear_rmsnorm norm_out")
+    two = s4c.linear(x1, w, x2, b, rs)
+    assert torch.equal(out.t, two) and torch.equal(nrm.t, s4c.rmsnorm(two, g, 1e-5))
+    want = oracle.rmsnorm(_f64(out.t), _f64(g), 1e-5)   # the normalisation of the rounded row, as the two calls give it
+    assert (np.abs(_f64(nrm.t) - want) <= 2.0 ** -8 * np.abs(want) + 1e-5).all()
+
+
 def test_concatenation_meets_the_right_columns():
     # e = one-hot rows, f = 0: the result reads columns of the FIRST K1 columns of w; and the other way round
     from paper_2506_14158_b200 import s4c
