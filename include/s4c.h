@@ -339,7 +339,11 @@ s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_l
  *                   workspace and are added in a fixed order (the result does not depend on
  *                   timing): workspace must hold s4c_linear_workspace_bytes(R, K1, K2, N, gate)
  *                   bytes (0 for shapes that need none; then NULL is accepted), 256-byte aligned;
- *                   S4C_ERR_WORKSPACE otherwise.
+ *                   S4C_ERR_WORKSPACE otherwise.  Stream order: the kernels are launched programmatically
+ *                   dependent; inputs, bias, residual and outputs are touched only after the kernel
+ *                   in front has completed, but tiles of w are requested earlier -- w must not be
+ *                   the output of the kernel enqueued directly in front on the same stream (a
+ *                   weight written earlier than that, or by a copy, is fine).
  *   s4c_linear_rmsnorm  the ungated s4c_linear followed by norm_out[r, :] = rmsnorm(out[r, :]) with
  *                   norm_weight [N] and eps >= 0 (norm_out [R, N] bf16, 16-byte aligned): the decoder
  *                   layer's "projection + residual, then the next block's normalisation".  Both out
