@@ -8,7 +8,7 @@ graph).  The default workload "c2x32" is the LLaMA-2-7B-shaped verify step at fu
 cache per layer, temperature 1.0.  Its 0.56 GB of KV per step is larger than L2, so no flush is needed.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2x32|c2|c3|c4|c4x32|c1|sweep --L --T --B]
-                    [--capacity C] [--no-hint] [--no-also]
+                    [--capacity C] [--no-hint] [--no-also] [--no-verify-pass]
     python bench.py --impl reference     # the float64 CPU oracle on a bounded sample of the same workload
     python bench.py --workload launch-floor   # empty kernels with the launch shape of an attention launch
     python bench.py --workload sweep-all [--capacity C]   # every point of the full-depth sweep
@@ -56,6 +56,7 @@ def parse_args():
     ap.add_argument("--capacity", type=int, default=0, help="cache capacity in slots (0: L + T rounded up to 128)")
     ap.add_argument("--no-hint", action="store_true", help="do not pass max_cache_len: launches are shaped for the capacity")
     ap.add_argument("--no-also", action="store_true", help="leave the 8B-shaped record out of the default line")
+    ap.add_argument("--no-verify-pass", action="store_true", help="leave out the leg that runs the target's whole verify pass (all layers' weights: ~14 GB)")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="keep timing K-step blocks until this much is timed")
     ap.add_argument("--paged", type=int, default=0, help="page size in slots (64, 128, ...): the caches become pools of pages "
                     "scattered at random, addressed through a block table (no host-buffer leg)")
@@ -501,6 +502,46 @@ def measure(cfg, args, device, rank, world, with_e2e):
         dr = dict(ms=ms_dr, rows=cfg.B * cfg.T, weight_bytes=wbytes, inter=inter, k=kk,
                   flops=2.0 * cfg.B * cfg.T * (wbytes / 2))
         del wts, head, kc, vc
+    # the whole greedy verify pass of the target (Section 3.2) composed from the library's calls: embedding of the tree tokens,
+    # every decoder layer (q/k/v + rotary, tree attention, output projection, gated MLP), LM head with the greedy choice, walk,
+    # compaction of every layer's cache -- random weights of the target's shapes, caches of its own (timed alone)
+    vp = None
+    if (cfg.dtype == "bf16" and not args.paged and cfg.d in (64, 128) and cfg.hid == cfg.Hq * cfg.d and cfg.n_layers > 1
+            and not args.no_verify_pass):
+        from paper_2506_14158_b200 import target
+
+        inter = {32000: 11008, 128256: 14336}.get(cfg.V, (cfg.hid * 8 // 3 + 255) // 256 * 256)
+        tw = target.random_weights(cfg.n_layers, cfg.V, cfg.hid, cfg.Hq, cfg.Hkv, cfg.d, inter, device, seed=cfg.config_id)
+        kcs = [torch.zeros((cfg.B, cfg.Hkv, cfg.C, cfg.d), dtype=torch.bfloat16, device=device) for _ in range(cfg.n_layers)]
+        vcs = [torch.zeros_like(kcs[0]) for _ in range(cfg.n_layers)]
+        tv = target.TargetVerify(tw, cfg.B, cfg.T, cfg.Hq, cfg.Hkv, cfg.d, cfg.C, kcs, vcs, cfg.max_depth)
+        cl_run = step.cache_len0.clone()
+
+        def run_pass():
+            cl_run.copy_(step.cache_len0)  # the step commits its accepted tokens; every replay starts from the same lengths
+            tv.forward(step.tokens, cl_run, step.parent, step.n_nodes, max_cache_len=cfg.L)
+
+        sg = torch.cuda.Stream()
+        sg.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(sg):
+            run_pass()
+        torch.cuda.current_stream().wait_stream(sg)
+        torch.cuda.synchronize()
+        g_vp = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_vp):
+            run_pass()
+        for _ in range(3):
+            g_vp.replay()
+        ms_vp = time_graph(g_vp, max(3, K // 4), torch)
+        assert int(tv.status_head.item()) == 0 and int(tv.status_qkv.abs().sum().item()) == 0
+        assert int(tv.status_attn.abs().sum().item()) == 0 and int(tv.status_compact.abs().sum().item()) == 0
+        lw0 = tw.layers[0]
+        wbytes = cfg.n_layers * sum(t.numel() * 2 for t in (lw0.qkv, lw0.o, lw0.gate_up, lw0.down)) + tw.lm_head.numel() * 2
+        kv_bytes = cfg.n_layers * 2 * cfg.B * cfg.Hkv * (cfg.L + cfg.T) * cfg.d * 2
+        vp = dict(ms=ms_vp, rows=cfg.B * cfg.T, n_layers=cfg.n_layers, weight_bytes=wbytes, kv_bytes=kv_bytes, inter=inter,
+                  flops=2.0 * cfg.B * cfg.T * (wbytes / 2), calls=2 + 6 * cfg.n_layers + 3,
+                  accept_len=tv.accept_len.cpu().tolist())
+        del tw, tv, kcs, vcs
     ms_e2e = 0.0
     if with_e2e:
         # end to end: per-step inputs from pinned host memory, decision back to the host, every step
@@ -521,7 +562,7 @@ def measure(cfg, args, device, rank, world, with_e2e):
         [blocks[0], statistics.median(blocks), min(blocks), statistics.median(attn_blocks), min(attn_blocks), ms_e2e],
         device=device)
     rec = dict(step=step, ms=ms_first, ms_median=ms_med, ms_best=ms_best, n_blocks=len(blocks), ms_attn=ms_attn,
-               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, qk=qk, dr=dr, ms_e2e=ms_e2e, accept_lens=accept_lens,
+               ms_attn_best=ms_attn_best, ms_acc=ms_acc, ms_cmp=ms_cmp, ms_tree=ms_tree, ms_filt=ms_filt, lm=lm, qk=qk, dr=dr, vp=vp, ms_e2e=ms_e2e, accept_lens=accept_lens,
                clocks=clocks, K=K, Wm=Wm)
     return rec
 
@@ -594,6 +635,18 @@ def roofline_records(cfg, args, rec, pk):
             bound="tensor" if dr["flops"] / dr["weight_bytes"] >= ridge else "hbm", gbs=dr["weight_bytes"] / t * 1e-9,
             frac_of_hbm_peak=dr["weight_bytes"] / t * 1e-9 / pk["hbm_gbs"], tflops=dr["flops"] / t * 1e-12,
             frac_of_tensor_peak=dr["flops"] / t * 1e-12 / pk["bf16_tflops"])
+    if rec.get("vp") is not None:
+        vp = rec["vp"]
+        breakdown["full_verify_pass_not_in_step"] = vp["ms"]
+        t = vp["ms"] * 1e-3
+        byts = vp["weight_bytes"] + vp["kv_bytes"]
+        roofline["verify_pass"] = dict(
+            kernel="the target's whole greedy verify pass: embed, %d decoder layers (q/k/v + rotary, tree attention, projections, gated "
+                   "MLP), LM head + greedy choice, walk, compaction (%d calls)" % (vp["n_layers"], vp["calls"]),
+            rows=vp["rows"], n_layers=vp["n_layers"], mlp_width=vp["inter"], ms=vp["ms"], weight_bytes=vp["weight_bytes"],
+            kv_bytes=vp["kv_bytes"], bound="tensor" if vp["flops"] / byts >= ridge else "hbm", gbs=byts / t * 1e-9,
+            frac_of_hbm_peak=byts / t * 1e-9 / pk["hbm_gbs"], tflops=vp["flops"] / t * 1e-12,
+            frac_of_tensor_peak=vp["flops"] / t * 1e-12 / pk["bf16_tflops"], nodes_per_s=vp["rows"] / t, accept_len=vp["accept_len"])
     return ab, step_hbm, roofline, breakdown
 
 
