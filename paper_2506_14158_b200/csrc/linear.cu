@@ -36,7 +36,8 @@ struct LnParams {
     int gate;                      // 1: the weight holds N gate rows, then N up rows; out = silu(gate) * up
     int bn, cols;                  // accumulator columns of a tile (a multiple of 16, <= 256) and the output columns they make:
                                    // cols = bn, or gated bn / 2 (the first cols accumulator columns are gate rows, the rest up rows)
-    int x_rows, stages;            // rows of an input box (a multiple of 32, <= 128); ring stages
+    int x_rows, stages;            // rows of an input box (a multiple of 32, <= 128; 256 with two row tiles); ring stages
+    int nm;                        // row tiles of 128 per CTA: 1, or 2 (two accumulators fed by one weight stream)
     const __nv_bfloat16* bias;     // [N] or null
     const __nv_bfloat16* residual; // [R, N] or null
     __nv_bfloat16* out;            // [R, N]
@@ -84,11 +85,12 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
         tma_prefetch_desc(&map_x1), tma_prefetch_desc(&map_w);
         if (prm.k2_steps) tma_prefetch_desc(&map_x2);
     }
-    if (warp == 1) tmem_alloc(smem_u32(const_cast<int*>(tmem_slot)), kLnBN);
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<int*>(tmem_slot)), kLnBN * prm.nm);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = (uint32_t)*tmem_slot;
+    const uint32_t tmem_cta = (uint32_t)*tmem_slot;
+    const uint32_t tmem = tmem_cta;
     griddep_launch_dependents();  // the kernel behind may set itself up; it waits for this one's results on its own
 
     if (warp == 0) {
@@ -104,9 +106,9 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
             };
             auto load_x = [&](int s, int ks) {
                 if (ks < prm.k1_steps)
-                    tma_load_2d(sX(s), &map_x1, FULL(s), ks * kLnBK, mtile * kLnBM);
+                    tma_load_2d(sX(s), &map_x1, FULL(s), ks * kLnBK, mtile * kLnBM * prm.nm);
                 else
-                    tma_load_2d(sX(s), &map_x2, FULL(s), (ks - prm.k1_steps) * kLnBK, mtile * kLnBM);
+                    tma_load_2d(sX(s), &map_x2, FULL(s), (ks - prm.k1_steps) * kLnBK, mtile * kLnBM * prm.nm);
             };
             // the weights do not come from the kernel in front: the first ring of weight tiles is under way before that
             // kernel has ended; the inputs follow once it has
@@ -140,6 +142,12 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
 #pragma unroll
                 for (int kk = 0; kk < kLnBK / 16; ++kk)  // 32 bytes per K step inside the swizzled row (field unit: 16 B)
                     tc_mma_bf16(tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                if (prm.nm == 2) {  // the second 128 rows of the stage (16 KB further on) meet the same weight tile
+                    const uint64_t a2_desc = smem_desc_sw128(sX(s) + kLnBM * kLnBK * 2, 16, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < kLnBK / 16; ++kk)
+                        tc_mma_bf16(tmem + kLnBN, a2_desc + 2u * kk, b_desc + 2u * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                }
                 tc_commit(EMPTY(s));
             }
             if (ok) tc_commit(ACC_FULL);
@@ -148,12 +156,13 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     } else {
         // ================= epilogue =================
         const int q = warp & 3;  // the tensor-memory lanes this warp may read: 32 q .. 32 q + 31
-        const int r = mtile * kLnBM + q * 32 + lane;
         griddep_wait();  // (the residual may be the result of the kernel in front, and nothing is written before that kernel has ended)
         bool ok = mbar_wait(ACC_FULL, 0, dead);
         ok = __all_sync(0xffffffffu, ok);
-        if (ok) {
-            tc_fence_after();
+        if (ok) tc_fence_after();
+        for (int rt = 0; ok && rt < prm.nm; ++rt) {
+            const int r = (mtile * prm.nm + rt) * kLnBM + q * 32 + lane;
+            const uint32_t tmem = tmem_cta + (uint32_t)(rt * kLnBN);  // this row tile's accumulator
             const bool live = r < prm.R;
             __nv_bfloat16* orow = prm.out + (size_t)(live ? r : 0) * prm.N;
             const __nv_bfloat16* rrow = prm.residual ? prm.residual + (size_t)(live ? r : 0) * prm.N : nullptr;
@@ -229,8 +238,8 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
                 }
                 __syncwarp();  // the lanes took different ways; the next tensor-memory load is warp-wide
             }
-            tc_fence_before();
         }
+        if (ok) tc_fence_before();
     }
     __syncthreads();
     if (*dead) {
@@ -252,7 +261,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
     }
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, kLnBN);
+        tmem_dealloc(tmem_cta, kLnBN * prm.nm);
     }
 }
 
@@ -441,41 +450,48 @@ static bool ln_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H,
 // The constants are measurements of this kernel on 7B- and 8B-shaped projections (26 and 256 rows), rounded; against
 // 70 measured (shape, columns, splits) points the model's choice was within 4 % of the best measured one.
 struct LnPlan {
-    int bn, splits, x_rows, stages, cols_per_tile, m_tiles, n_tiles;
+    int bn, splits, x_rows, stages, cols_per_tile, m_tiles, n_tiles, nm;
 };
 static LnPlan ln_plan(int R, int K1, int K2, int N, int gate) {
     constexpr double kIssueUs = 0.30, kMmaUsPerCol = 0.27 / 256.0, kSmBytesPerUs = 60e3, kHbmBytesPerUs = 6.4e6, kL2BytesPerUs = 100e3,
-                     kTurnUs = 1.3, kWaveUs = 2.5, kFinishUs = 3.0, kPartialBytesPerUs = 4.0e6;
+                     kTurnUs = 1.3, kWaveUs = 2.5, kFinishUs = 3.0, kPartialBytesPerUs = 4.0e6, kIssueTwo = 1.5;
     constexpr int kSms = 148;
-    const int k_steps = (K1 + K2) / kLnBK, m_tiles = ceil_div(R, kLnBM);
-    const int x_rows = R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32);
+    const int k_steps = (K1 + K2) / kLnBK;
     const int w_rows = gate ? 2 * N : N;
     LnPlan best = {};
     double best_us = 1e30;
-    for (int cols = 16; cols <= (gate ? kLnBN / 2 : kLnBN); cols += 16) {
-        const int bn = gate ? 2 * cols : cols;
-        const int stage_bytes = (x_rows + bn) * kLnBK * 2;
-        const int stages = std::min(kLnMaxStages, (kLnRingBytes - kLnBM * kLnBK * 2) / stage_bytes);  // (a spare tile: see the q/k/v kernel)
-        if (stages < 3) continue;
-        const int n_tiles = ceil_div(N, cols);
-        if (cols > 16 && ceil_div(N, cols - 16) == n_tiles) continue;  // the narrower tile covers N with as many CTAs
-        for (int splits = 1; splits <= 8; ++splits) {
-            if (splits > 1 && k_steps / splits < 4) break;
-            const int ctas = n_tiles * m_tiles * splits, k_per = ceil_div(k_steps, splits);
-            double us = 0.0;
-            for (int left = ctas; left > 0; left -= kSms) {
-                const int active = std::min(left, kSms);
-                const double mma = kMmaUsPerCol * bn;
-                const double hbm = bn * (kLnBK * 2.0) / m_tiles / std::min(kSmBytesPerUs, kHbmBytesPerUs / active);
-                const double slice = std::max(std::max(std::max(kIssueUs, mma), std::max(hbm, stage_bytes / kL2BytesPerUs)),
-                                              (kTurnUs + mma) / stages);
-                us += kWaveUs + k_per * slice;
-            }
-            if (splits > 1) us += kFinishUs + 2.0 * splits * R * (double)w_rows * sizeof(float) / kPartialBytesPerUs;
-            if (us < best_us) {
-                best_us = us;
-                best.bn = bn, best.splits = splits, best.x_rows = x_rows, best.stages = stages, best.cols_per_tile = cols;
-                best.m_tiles = m_tiles, best.n_tiles = n_tiles;
+    // more than 128 rows: one row tile per CTA (the row tiles of a column tile share the weights through L2), or two
+    // accumulators per CTA fed by one weight stream (half the weight traffic into the SM, twice the products per slice)
+    for (int nm = 1; nm <= (R > kLnBM ? 2 : 1); ++nm) {
+        const int m_tiles = ceil_div(R, kLnBM * nm);
+        const int x_rows = nm == 2 ? 2 * kLnBM : (R > kLnBM ? kLnBM : (int)round_up((size_t)R, 32));
+        const int spare = x_rows < kLnBM ? kLnBM * kLnBK * 2 : 0;  // (a product reads 128 rows from a stage's start: see the q/k/v kernel)
+        for (int cols = 16; cols <= (gate ? kLnBN / 2 : kLnBN); cols += 16) {
+            const int bn = gate ? 2 * cols : cols;
+            const int stage_bytes = (x_rows + bn) * kLnBK * 2;
+            const int stages = std::min(kLnMaxStages, (kLnRingBytes - spare) / stage_bytes);
+            if (stages < 3) continue;
+            const int n_tiles = ceil_div(N, cols);
+            if (cols > 16 && ceil_div(N, cols - 16) == n_tiles) continue;  // the narrower tile covers N with as many CTAs
+            for (int splits = 1; splits <= 8; ++splits) {
+                if (splits > 1 && k_steps / splits < 4) break;
+                const int ctas = n_tiles * m_tiles * splits, k_per = ceil_div(k_steps, splits);
+                double us = 0.0;
+                for (int left = ctas; left > 0; left -= kSms) {
+                    const int active = std::min(left, kSms);
+                    const double mma = kMmaUsPerCol * bn * nm;
+                    const double hbm = bn * (kLnBK * 2.0) / m_tiles / std::min(kSmBytesPerUs, kHbmBytesPerUs / active);
+                    const double slice = std::max(std::max(std::max(kIssueUs * (nm == 2 ? kIssueTwo : 1.0), mma),
+                                                           std::max(hbm, stage_bytes / kL2BytesPerUs)),
+                                                  (kTurnUs + mma) / stages);
+                    us += kWaveUs + k_per * slice;
+                }
+                if (splits > 1) us += kFinishUs + 2.0 * splits * R * (double)w_rows * sizeof(float) / kPartialBytesPerUs;
+                if (us < best_us) {
+                    best_us = us;
+                    best.bn = bn, best.splits = splits, best.x_rows = x_rows, best.stages = stages, best.cols_per_tile = cols;
+                    best.m_tiles = m_tiles, best.n_tiles = n_tiles, best.nm = nm;
+                }
             }
         }
     }
@@ -529,7 +545,7 @@ static s4c_status ln_run(const void* x1, const void* x2, const void* w, const vo
     }
     LnParams prm;
     prm.R = R, prm.N = N, prm.k1_steps = K1 / kLnBK, prm.k2_steps = K2 / kLnBK, prm.gate = gate ? 1 : 0;
-    prm.x_rows = pl.x_rows, prm.stages = pl.stages, prm.bn = pl.bn, prm.cols = pl.cols_per_tile;
+    prm.x_rows = pl.x_rows, prm.stages = pl.stages, prm.bn = pl.bn, prm.cols = pl.cols_per_tile, prm.nm = pl.nm;
     prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
     prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
     prm.splits = pl.splits, prm.partial = static_cast<float*>(workspace);

@@ -72,6 +72,30 @@ def test_gated_linear_against_the_oracle(R, K, N, res):
     assert (np.abs(_f64(out.t) - want) <= bound).all()
 
 
+@pytest.mark.parametrize("R,K,N,res", [(300, 512, 8192, True), (500, 1024, 8192, False), (256, 4096, 14336, False)])
+def test_wide_gated_projection_on_many_rows(R, K, N, res):
+    # more than 128 rows and a wide output: the launch that feeds two 128-row accumulators from one weight stream (ragged
+    # second tile at 300 and 500 rows); the 8B models' gate / up shape on 512 sampled output columns
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(R + K)
+    x, w = _bf16(rng.standard_normal((R, K))), _bf16(rng.standard_normal((2 * N, K)) / np.sqrt(K))
+    rs = _bf16(rng.standard_normal((R, N))) if res else None
+    out = Guarded((R, N), torch.bfloat16, fill=-3.0)
+    s4c.linear(x.cuda(), w.cuda(), residual=None if rs is None else rs.cuda(), gate=True, out=out.t)
+    torch.cuda.synchronize()
+    out.check("s4c_linear gated out, many rows")
+    cols = np.sort(rng.choice(N, 512, replace=False))
+    cols[:3], cols[-3:] = [0, 1, 2], [N - 3, N - 2, N - 1]
+    w_s = np.concatenate([_f64(w)[cols], _f64(w)[N + cols]])
+    want = oracle.linear(_f64(x), w_s, residual=None if rs is None else _f64(rs)[:, cols], gate=True)
+    y = _f64(x) @ w_s.T
+    g, u = y[:, :512], y[:, 512:]
+    slack = 8.0 * np.sqrt(K) * 2.0 ** -24 * np.linalg.norm(_f64(x), axis=1, keepdims=True) * np.linalg.norm(w_s, axis=1).max()
+    bound = 2.0 ** -8 * np.abs(want) + slack * (1.1 * np.abs(u) + np.abs(g) + 1.0) + 1e-5
+    assert (np.abs(_f64(out.t)[:, cols] - want) <= bound).all()
+
+
 def test_shared_out_k_range_is_reproducible_and_checks_its_workspace():
     from paper_2506_14158_b200 import s4c
 
