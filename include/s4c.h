@@ -322,6 +322,17 @@ s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_l
                         int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status, void* workspace,
                         size_t workspace_bytes, s4c_stream_t stream);
 
+/* s4c_qkv_rope_same_tree -- another layer of the same verify pass (Section 3.2: one forward pass over
+ * one tree): the tree checks, the rows' cache positions and the rotary table depend on cache_len,
+ * parent, n_nodes, T, d and rope_theta alone, so the layers after the first reuse what s4c_qkv_rope
+ * left in `workspace` (same B, T, d, C; cache_len unchanged since; the workspace untouched since)
+ * and skip that kernel.  Arguments as s4c_qkv_rope.  status [B] or NULL is NOT rewritten: it keeps
+ * what it holds (the first call's flags, when the same array is passed) and gets S4C_SEQ_TIMEOUT
+ * OR-ed in; sequences the first call flagged are skipped here too. */
+s4c_status s4c_qkv_rope_same_tree(const void* x, const void* w_qkv, void* q_out, void* k_cache, void* v_cache, int B,
+                                  int T, int H, int Hq, int Hkv, int d, int C, int32_t* status, void* workspace,
+                                  size_t workspace_bytes, s4c_stream_t stream);
+
 /* ------------------------------------------------------------------------------------------
  * s4c_linear, s4c_rmsnorm, s4c_embed_gather -- the pieces of the drafter's head (Section 3.1, Eq. 3-6)
  * and of a LLaMA-family decoder layer that are not attention:

@@ -41,6 +41,7 @@ struct QkParams {
     __nv_bfloat16* k_cache;    // [B,Hkv,C,d]
     __nv_bfloat16* v_cache;
     int32_t* status;           // [B] (may be null)
+    int wait_x;                // 1: the input rows may come from the kernel directly in front (no table kernel between)
 };
 
 // Tree and capacity checks, the rows' cache bases and the rotary table.  grid (sequences, groups of kQkPrepNodes nodes):
@@ -119,11 +120,24 @@ qkv_rope_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // every CTA walks the K slices from a start of its own: the CTAs of a row tile all read the same state tiles,
             // and in step they would all ask the same L2 lines at the same moment (the order of a sum's terms is free)
             const int k0 = (int)((blockIdx.x * 7u + blockIdx.y * 3u) % (uint32_t)prm.k_steps);
+            auto slice_of = [&](int fill) { return fill + k0 < prm.k_steps ? fill + k0 : fill + k0 - prm.k_steps; };
             int fill = 0, s = 0;
             uint32_t ph = 0;  // the ring pass's parity (stage and parity are stepped, not divided out: S is not a constant)
+            if (prm.wait_x) {
+                // no table kernel in front: the weights (which no kernel of the step writes) fill the first ring while the
+                // kernel that produces the input rows is still running; the rows follow once it has ended
+                const int pre = prm.k_steps < S ? prm.k_steps : S;
+                for (int f = 0; f < pre; ++f) {
+                    mbar_expect_tx(FULL(f), stage_bytes);
+                    tma_load_2d(sW(f), &map_w, FULL(f), slice_of(f) * kQkBK, head * d);
+                }
+                griddep_wait();
+                for (int f = 0; f < pre; ++f) tma_load_2d(sX(f), &map_x, FULL(f), slice_of(f) * kQkBK, mtile * kQkBM);
+                fill = pre, s = pre == S ? 0 : pre, ph = pre == S ? 1 : 0;
+            }
             for (; fill < prm.k_steps; ++fill, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
                 if (!mbar_wait(EMPTY(s), ph ^ 1, dead)) break;
-                const int ks = fill + k0 < prm.k_steps ? fill + k0 : fill + k0 - prm.k_steps;
+                const int ks = slice_of(fill);
                 mbar_expect_tx(FULL(s), stage_bytes);
                 tma_load_2d(sX(s), &map_x, FULL(s), ks * kQkBK, mtile * kQkBM);
                 tma_load_2d(sW(s), &map_w, FULL(s), ks * kQkBK, head * d);
@@ -279,12 +293,13 @@ extern "C" size_t s4c_qkv_rope_workspace_bytes(int B, int T, int d) {
     return s4c::qk_ws_layout(B, T, d, nullptr, nullptr, nullptr);
 }
 
-extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* parent,
-                                   const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache, int B, int T, int H,
-                                   int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status, void* workspace,
-                                   size_t workspace_bytes, s4c_stream_t stream_) {
-    using namespace s4c;
-    if (!x || !w_qkv || !cache_len || !parent || !q_out || !k_cache || !v_cache) return S4C_ERR_NULL;
+namespace s4c {
+// tables: the tree / rotary-table kernel runs first (s4c_qkv_rope); otherwise the tables of the call before on this
+// workspace are used as they are (s4c_qkv_rope_same_tree)
+static s4c_status qk_run(bool tables, const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* parent,
+                         const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache, int B, int T, int H, int Hq, int Hkv, int d,
+                         int C, float rope_theta, int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream_) {
+    if (!x || !w_qkv || (tables && (!cache_len || !parent)) || !q_out || !k_cache || !v_cache) return S4C_ERR_NULL;
     if (B < 0 || T < 1 || T > S4C_MAX_T || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || (d != 64 && d != 128) || C < T) return S4C_ERR_SHAPE;
     if (H < kQkBK || H % kQkBK != 0 || !(rope_theta > 1.f) || isinf(rope_theta)) return S4C_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(q_out) || !aligned16(k_cache) || !aligned16(v_cache)) return S4C_ERR_ALIGN;
@@ -304,8 +319,10 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
     const int stages = std::min(kQkMaxStages, (kQkRingBytes - (x_rows < kQkBM ? kQkBM * kQkBK * 2 : 0)) / stage_bytes);
     if (!qk_make_map(&map_x, x, (uint64_t)R, H, x_rows) || !qk_make_map(&map_w, w_qkv, (uint64_t)heads * d, H, d)) return S4C_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    qkv_prep_kernel<<<dim3(B, ceil_div(T, kQkPrepNodes)), 128, 0, stream>>>(cache_len, parent, n_nodes, T, C, d, (double)rope_theta, row_base, rope, status);
-    S4C_RETURN_IF_CUDA_ERROR();
+    if (tables) {
+        qkv_prep_kernel<<<dim3(B, ceil_div(T, kQkPrepNodes)), 128, 0, stream>>>(cache_len, parent, n_nodes, T, C, d, (double)rope_theta, row_base, rope, status);
+        S4C_RETURN_IF_CUDA_ERROR();
+    }
     static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
@@ -322,6 +339,7 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
     prm.row_base = row_base, prm.rope = rope;
     prm.q_out = static_cast<__nv_bfloat16*>(q_out), prm.k_cache = static_cast<__nv_bfloat16*>(k_cache);
     prm.v_cache = static_cast<__nv_bfloat16*>(v_cache), prm.status = status;
+    prm.wait_x = tables ? 0 : 1;
     cudaLaunchAttribute pdl;
     pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl.val.programmaticStreamSerializationAllowed = 1;
@@ -334,4 +352,20 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
         return S4C_ERR_CUDA;
     }
     return S4C_OK;
+}
+}  // namespace s4c
+
+extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* parent,
+                                   const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache, int B, int T, int H,
+                                   int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status, void* workspace,
+                                   size_t workspace_bytes, s4c_stream_t stream) {
+    return s4c::qk_run(true, x, w_qkv, cache_len, parent, n_nodes, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C, rope_theta, status,
+                       workspace, workspace_bytes, stream);
+}
+
+extern "C" s4c_status s4c_qkv_rope_same_tree(const void* x, const void* w_qkv, void* q_out, void* k_cache, void* v_cache, int B,
+                                             int T, int H, int Hq, int Hkv, int d, int C, int32_t* status, void* workspace,
+                                             size_t workspace_bytes, s4c_stream_t stream) {
+    return s4c::qk_run(false, x, w_qkv, nullptr, nullptr, nullptr, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C, 10000.f, status,
+                       workspace, workspace_bytes, stream);
 }

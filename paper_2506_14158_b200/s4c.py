@@ -25,7 +25,7 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
            "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
-           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
+           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_qkv_rope_same_tree", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
            "s4c_tree_build_topk", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_linear_rmsnorm", "s4c_rmsnorm", "s4c_embed_gather"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_qkv_rope_workspace_bytes.argtypes = [i, i, i]
     lib.s4c_qkv_rope.restype = i
     lib.s4c_qkv_rope.argtypes = [vp, vp, i32p, i32p, i32p, vp, vp, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_qkv_rope_same_tree.restype = i
+    lib.s4c_qkv_rope_same_tree.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i32p, vp, sz, vp]
     lib.s4c_lm_head_topk_workspace_bytes.restype = sz
     lib.s4c_lm_head_topk_workspace_bytes.argtypes = [i, i, i, i]
     lib.s4c_lm_head_topk.restype = i
@@ -491,6 +493,22 @@ def qkv_rope(x, w_qkv, cache_len, parent, q_out, k_cache, v_cache, n_nodes=None,
                            workspace.numel() * workspace.element_size(), _stream(stream))
     if rc:
         raise S4CError("s4c_qkv_rope", rc)
+    return dict(q=q_out, status=status)
+
+
+def qkv_rope_same_tree(x, w_qkv, q_out, k_cache, v_cache, workspace, status=None, stream=None):
+    """s4c_qkv_rope_same_tree: another layer's projections with the tree checks, positions and rotary table that the
+    preceding :func:`qkv_rope` call left in ``workspace`` (``status``: that call's, kept and OR-ed with timeouts)."""
+    B, T, H = x.shape
+    _, Hq, _, d = q_out.shape
+    _, Hkv, C, _ = k_cache.shape
+    bf = torch.bfloat16
+    rc = _lib.s4c_qkv_rope_same_tree(_dev(x, bf, "x"), _dev(w_qkv, bf, "w_qkv"), _dev(q_out, bf, "q_out"), _dev(k_cache, bf, "k_cache"),
+                                     _dev(v_cache, bf, "v_cache"), B, T, H, Hq, Hkv, d, C, _dev(status, torch.int32, "status"),
+                                     _dev(workspace, name="workspace"), workspace.numel() * workspace.element_size(),
+                                     _stream(stream))
+    if rc:
+        raise S4CError("s4c_qkv_rope_same_tree", rc)
     return dict(q=q_out, status=status)
 
 

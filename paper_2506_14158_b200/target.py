@@ -5,7 +5,7 @@ chat models):
     x0 = Embedding(tree tokens)                                  s4c_embed_gather
     a0 = rmsnorm(x0)                                             s4c_rmsnorm
     per layer l:
-        q, K/V tree slots = rope(a_l Wqkv^T)                     s4c_qkv_rope          (position = committed length + depth)
+        q, K/V tree slots = rope(a_l Wqkv^T)                     s4c_qkv_rope / s4c_qkv_rope_same_tree (position = committed length + depth; the rotary table once per pass)
         o  = tree attention(q, cache_l)                          s4c_tree_attention    (tree mask from parent[])
         h  = x_l + o Wo^T,          m = rmsnorm(h)               s4c_linear_rmsnorm
         g  = silu(m Wg^T) * (m Wu^T)                             s4c_linear, gated
@@ -85,7 +85,7 @@ class TargetVerify:
         self.attn = [torch.empty(B, Hq, T, d, **bf) for _ in range(sets)]
         self.o_in, self.h, self.m, self.act = rows(Hq * d), rows(H), rows(H), rows(inter)
         self.sets = sets
-        self.status_qkv = torch.zeros(n, B, **i32)
+        self.status_qkv = torch.zeros(1, B, **i32)  # written by the first layer's call, timeouts of the others OR-ed in
         self.status_attn = torch.zeros(n, B, **i32)
         self.status_head = torch.zeros(1, **i32)
         self.target_token = torch.empty(R, **i32)
@@ -112,8 +112,12 @@ class TargetVerify:
         s4c.rmsnorm(self.x[0], w.layers[0].norm1, self.eps, out=self.a[0])
         for l, lw in enumerate(w.layers):
             i, i_in, i_out = l % self.sets, l % (self.sets + 1), (l + 1) % (self.sets + 1)
-            s4c.qkv_rope(self.a[i_in].view(B, T, -1), lw.qkv, cache_len, parent, self.q[i], self.k_caches[l], self.v_caches[l], n_nodes,
-                         self.rope_theta, status=self.status_qkv[l], workspace=self.ws_qkv)
+            if l == 0:  # tree checks, cache positions and the rotary table: once per pass, the other layers reuse them
+                s4c.qkv_rope(self.a[i_in].view(B, T, -1), lw.qkv, cache_len, parent, self.q[i], self.k_caches[l], self.v_caches[l], n_nodes,
+                             self.rope_theta, status=self.status_qkv[0], workspace=self.ws_qkv)
+            else:
+                s4c.qkv_rope_same_tree(self.a[i_in].view(B, T, -1), lw.qkv, self.q[i], self.k_caches[l], self.v_caches[l], self.ws_qkv,
+                                       status=self.status_qkv[0])
             s4c.tree_attention(self.q[i], self.k_caches[l], self.v_caches[l], cache_len, parent, n_nodes, out=self.attn[i],
                                status=self.status_attn[l], workspace=self.ws_attn, max_cache_len=max_cache_len)
             self.o_in[i].view(B, T, self.Hq, self.d).copy_(self.attn[i].permute(0, 2, 1, 3))  # rows for the output projection

@@ -163,6 +163,11 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert qk(B=0) == 0
     assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) % 256 == 0 and lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) > 0
     assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 96) == 0
+    lib.s4c_qkv_rope_same_tree.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp]
+    qs = lambda **kw: lib.s4c_qkv_rope_same_tree(*[kw.get(k, d) for k, d in [
+        ("x", P), ("w", P), ("q", P), ("k", P), ("v", P), ("B", 1), ("T", 26), ("H", 4096), ("Hq", 32), ("Hkv", 8), ("d", 128),
+        ("C", 2048), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
+    assert qs(x=None) == 1 and qs(v=None) == 1 and qs(d=96) == 2 and qs(Hkv=5) == 2 and qs(k=P + 2) == 4 and qs() == 5 and qs(B=0) == 0
     lib.s4c_lm_head_topk.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp, sz, vp]
     lib.s4c_lm_head_topk_workspace_bytes.restype = sz
     lib.s4c_lm_head_topk_workspace_bytes.argtypes = [i, i, i, i]

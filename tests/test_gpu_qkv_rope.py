@@ -103,6 +103,43 @@ def test_padding_flags_and_untouched_sequences():
     _compare(got, ref, x, w, cache_len, n_nodes, T)
 
 
+@pytest.mark.parametrize("B,T,H,Hq,Hkv,d,C", [(5, 20, 128, 4, 2, 128, 64), (1, 26, 512, 8, 8, 64, 200), (3, 64, 256, 8, 2, 128, 300)])
+def test_another_layer_on_the_same_tree_reuses_the_tables(B, T, H, Hq, Hkv, d, C):
+    # layer 1 with the table kernel, layer 2 (other states, other weights, other caches) on what it left in the workspace:
+    # the same bits as a full call for layer 2, flagged sequences skipped, the status array kept
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(B + T)
+    parent = np.stack([W.random_tree(T, 5, rng, 1, 4) for _ in range(B)]).astype(np.int32)
+    cache_len = rng.integers(0, C - T + 1, B).astype(np.int32)
+    n_nodes = rng.integers(1, T + 1, B).astype(np.int32)
+    if B >= 5:
+        cache_len[1] = C - T + 5   # does not fit
+        parent[2, 4] = 9           # malformed
+    mk = lambda *shape, s=1.0: _bf16(rng.standard_normal(shape) * s).cuda()
+    xs, ws_ = [mk(B, T, H), mk(B, T, H)], [mk((Hq + 2 * Hkv) * d, H, s=H ** -0.5), mk((Hq + 2 * Hkv) * d, H, s=H ** -0.5)]
+    k0, v0 = mk(B, Hkv, C, d), mk(B, Hkv, C, d)
+    wsp = torch.empty(s4c.qkv_rope_workspace_bytes(B, T, d), dtype=torch.uint8, device="cuda")
+    # the full call for layer 2's inputs: what the reuse must reproduce
+    q_full, k_full, v_full = torch.full((B, Hq, T, d), -3.0, dtype=torch.bfloat16, device="cuda"), k0.clone(), v0.clone()
+    st_full = s4c.qkv_rope(xs[1], ws_[1], dev(cache_len), dev(parent), q_full, k_full, v_full, dev(n_nodes), workspace=wsp)["status"].clone()
+    wsp.fill_(0xCD)
+    q1, k1, v1 = torch.empty_like(q_full), k0.clone(), v0.clone()
+    st = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+    s4c.qkv_rope(xs[0], ws_[0], dev(cache_len), dev(parent), q1, k1, v1, dev(n_nodes), status=st, workspace=wsp)
+    q2 = Guarded((B, Hq, T, d), torch.bfloat16, fill=-3.0)
+    k2, v2 = Guarded((B, Hkv, C, d), torch.bfloat16, src=k0), Guarded((B, Hkv, C, d), torch.bfloat16, src=v0)
+    s4c.qkv_rope_same_tree(xs[1], ws_[1], q2.t, k2.t, v2.t, wsp, status=st)
+    torch.cuda.synchronize()
+    for name, buf in (("q", q2), ("k", k2), ("v", v2)):
+        buf.check("s4c_qkv_rope_same_tree " + name)
+    assert torch.equal(st, st_full)
+    assert torch.equal(q2.t, q_full) and torch.equal(k2.t, k_full) and torch.equal(v2.t, v_full)
+    if B >= 5:
+        assert st.tolist()[1] == oracle.SEQ_CAPACITY and st.tolist()[2] == oracle.SEQ_BAD_PARENT
+        assert (q2.t[1] == -3.0).all() and torch.equal(k2.t[2], k0[2])
+
+
 def test_full_size_layer_then_attention_reads_what_was_written():
     # the 8B-shaped layer (256 rows, H = 4096, 32/8 heads x 128) in the launch the benchmark times, and the hand-over:
     # s4c_tree_attention on the q and caches this call wrote equals the oracle's attention on the oracle's q / k / v
