@@ -4,12 +4,14 @@
 // s4c_rmsnorm and s4c_embed_gather: the layer's two small row operations (root-mean-square normalisation; Eq. 6,
 // e = Embedding(t)).
 //
-// One CTA per (128-column tile of the output, 128-row tile): the pipeline of the q/k/v kernel -- warp 0 requests
-// 64-element K slices by TMA (128-byte swizzle; slices of the first input, then of the second, against consecutive column
-// ranges of the weight), warp 1 issues the products into one f32 accumulator in tensor memory, warps 2-5 read it (one row per
-// thread), apply the epilogue and store 16 bytes at a time.  Gated form: a tile's accumulator holds 64 gate columns beside
-// their 64 up columns (two 64-row boxes of the weight), as the q/k/v kernel keeps a rotary pair in one row.  Every wait on
-// a barrier is bounded.
+// One CTA per (column tile of the output, row tile, share of the K range): the pipeline of the q/k/v kernel -- warp 0
+// requests 64-element K slices by TMA (128-byte swizzle; slices of the first input, then of the second, against consecutive
+// column ranges of the weight), warp 1 issues the products into an f32 accumulator in tensor memory, warps 2-5 read it
+// (one row per thread), apply the epilogue and store 16 bytes at a time.  Gated form: a tile's accumulator holds its gate
+// columns beside the same outputs' up columns (two boxes of the weight), as the q/k/v kernel keeps a rotary pair in one row.
+// The launch shape -- tile width (a multiple of 16 columns), one or two 128-row accumulators per CTA, the number of CTAs
+// that share a tile's K range -- is chosen per call (ln_plan); shared-out K ranges meet again in linear_finish_kernel, in
+// a fixed order.  All kernels here are launched programmatically dependent.  Every wait on a barrier is bounded.
 #include <cuda.h>
 #include <math.h>
 
@@ -134,6 +136,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
             bool ok = true;
             int s = 0;
             uint32_t ph = 0;
+            griddep_wait();  // the input rows are requested only after the kernel in front has ended: the bounded waits below start then
             for (int ks = 0; ks < k_steps; ++ks, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
                 ok = mbar_wait(FULL(s), ph, dead);
                 if (!ok) break;

@@ -152,6 +152,7 @@ qkv_rope_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             bool ok = true;
             int s = 0;
             uint32_t ph = 0;
+            if (prm.wait_x) griddep_wait();  // the rows are requested only after the kernel in front has ended: the bounded waits start then
             for (int ks = 0; ks < prm.k_steps; ++ks, s = s + 1 == S ? 0 : s + 1, ph ^= (s == 0)) {
                 ok = mbar_wait(FULL(s), ph, dead);
                 if (!ok) break;
