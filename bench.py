@@ -539,7 +539,7 @@ def measure(cfg, args, device, rank, world, with_e2e):
         wbytes = cfg.n_layers * sum(t.numel() * 2 for t in (lw0.qkv, lw0.o, lw0.gate_up, lw0.down)) + tw.lm_head.numel() * 2
         kv_bytes = cfg.n_layers * 2 * cfg.B * cfg.Hkv * (cfg.L + cfg.T) * cfg.d * 2
         vp = dict(ms=ms_vp, rows=cfg.B * cfg.T, n_layers=cfg.n_layers, weight_bytes=wbytes, kv_bytes=kv_bytes, inter=inter,
-                  flops=2.0 * cfg.B * cfg.T * (wbytes / 2), calls=2 + 6 * cfg.n_layers + 3,
+                  flops=2.0 * cfg.B * cfg.T * (wbytes / 2), calls=2 + 5 * cfg.n_layers + 3,
                   accept_len=tv.accept_len.cpu().tolist())
         del tw, tv, kcs, vcs
     ms_e2e = 0.0
@@ -630,7 +630,7 @@ def roofline_records(cfg, args, rec, pk):
         breakdown["drafter_head_not_in_step"] = dr["ms"]
         t = dr["ms"] * 1e-3
         roofline["drafter_head"] = dict(
-            kernel="one drafter head, Eq. 3-6: embed, Linear(concat[e,f]), decoder layer, LM-head top-k (9 calls)", rows=dr["rows"],
+            kernel="one drafter head, Eq. 3-6: embed, Linear(concat[e,f]), decoder layer, LM-head top-k (8 calls)", rows=dr["rows"],
             mlp_width=dr["inter"], top_k=dr["k"], us=dr["ms"] * 1e3, weight_bytes=dr["weight_bytes"],
             bound="tensor" if dr["flops"] / dr["weight_bytes"] >= ridge else "hbm", gbs=dr["weight_bytes"] / t * 1e-9,
             frac_of_hbm_peak=dr["weight_bytes"] / t * 1e-9 / pk["hbm_gbs"], tflops=dr["flops"] / t * 1e-12,

@@ -126,6 +126,16 @@ s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_
                               s4c_dtype dt, float scale, int32_t* status, void* workspace,
                               size_t workspace_bytes, s4c_stream_t stream);
 
+/* s4c_tree_attention_rows -- the same attention, written as the rows the layer's output projection
+ * reads: out_rows [B, T, Hq, d] = [B*T rows, Hq*d] instead of [B, Hq, T, d] (no transposing copy
+ * between the two).  Same arguments, workspace and status; S4C_BF16 only (S4C_ERR_UNSUPPORTED
+ * otherwise).  Every element equals, bit for bit, the one s4c_tree_attention writes. */
+s4c_status s4c_tree_attention_rows(const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                   void* out_rows, int B, int T, int Hq, int Hkv, int d, int C, int max_cache_len,
+                                   s4c_dtype dt, float scale, int32_t* status, void* workspace,
+                                   size_t workspace_bytes, s4c_stream_t stream);
+
 /* ------------------------------------------------------------------------------------------
  * s4c_tree_accept -- the accept / resample rule of Section 2 ("Speculative Sampling"): a draft token
  * passes with probability min(1, p/q), a rejected position is resampled from norm(max(0, p - q));

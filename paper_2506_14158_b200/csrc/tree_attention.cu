@@ -22,17 +22,17 @@ extern "C" size_t s4c_tree_attention_workspace_bytes(int B, int T, int Hq, int H
     return simt_workspace_bytes(B, T, Hq, d, C);
 }
 
-extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_cache,
-                                         const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
-                                         void* out, int B, int T, int Hq, int Hkv, int d, int C, int max_cache_len,
-                                         s4c_dtype dt, float scale, int32_t* status, void* workspace,
-                                         size_t workspace_bytes, s4c_stream_t stream_) {
-    using namespace s4c;
+namespace s4c {
+static s4c_status attention_run(const void* q, const void* k_cache, const void* v_cache, const int32_t* cache_len,
+                                const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv, int d, int C,
+                                int max_cache_len, s4c_dtype dt, float scale, int32_t* status, void* workspace,
+                                size_t workspace_bytes, s4c_stream_t stream_, int out_rows) {
     const s4c_status st = check_shapes(B, T, Hq, Hkv, d, C, dt);
     if (st != S4C_OK) return st;
     if (!q || !k_cache || !v_cache || !cache_len || !parent || !out) return S4C_ERR_NULL;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return S4C_ERR_ALIGN;
     if (!(scale >= 0.f) || isinf(scale) || max_cache_len < 0) return S4C_ERR_SHAPE;
+    if (out_rows && !tc_supported(T, Hq, Hkv, d, dt)) return S4C_ERR_UNSUPPORTED;  // the row layout exists on the tensor-core path (bf16) only
     if (B == 0) return S4C_OK;
     if (scale == 0.f) scale = 1.f / sqrtf((float)d);
     const size_t need = s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt);
@@ -42,9 +42,28 @@ extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, con
     const int span = (max_cache_len > 0 && (long long)max_cache_len + T < (long long)C) ? max_cache_len + T : C;
     if (tc_supported(T, Hq, Hkv, d, dt))
         return tree_attention_tc(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, span, scale,
-                                 status, workspace, stream);
+                                 status, workspace, stream, 0, -1, nullptr, out_rows);
     return tree_attention_simt(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, span, dt, scale,
                                status, workspace, stream);
+}
+}  // namespace s4c
+
+extern "C" s4c_status s4c_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                                         const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                         void* out, int B, int T, int Hq, int Hkv, int d, int C, int max_cache_len,
+                                         s4c_dtype dt, float scale, int32_t* status, void* workspace,
+                                         size_t workspace_bytes, s4c_stream_t stream) {
+    return s4c::attention_run(q, k_cache, v_cache, cache_len, parent, n_nodes, out, B, T, Hq, Hkv, d, C, max_cache_len, dt, scale, status,
+                              workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" s4c_status s4c_tree_attention_rows(const void* q, const void* k_cache, const void* v_cache,
+                                              const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
+                                              void* out_rows, int B, int T, int Hq, int Hkv, int d, int C, int max_cache_len,
+                                              s4c_dtype dt, float scale, int32_t* status, void* workspace,
+                                              size_t workspace_bytes, s4c_stream_t stream) {
+    return s4c::attention_run(q, k_cache, v_cache, cache_len, parent, n_nodes, out_rows, B, T, Hq, Hkv, d, C, max_cache_len, dt, scale,
+                              status, workspace, workspace_bytes, stream, 1);
 }
 
 // Paged caches: pages [n_pages, Hkv, page_size, d] addressed through a block table [B, max_blocks].

@@ -14,7 +14,7 @@ s4c_status tree_attention_simt(const void* q, const void* k, const void* v, cons
 // Merges split partials [B*Hq*T rows][splits][d + 2] (unnormalised output, running max in base-2 units, sum).
 s4c_status tree_attention_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
                                   void* out, int B, int T, int Hq, int d, int C, int splits, s4c_dtype dt,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, int out_rows = 0 /* 1: out is [B,T,Hq,d] */);
 
 // Paged caches: pages [n_pages, Hkv, page_size, d] and a block table [B, max_blocks] (page_size a multiple of 64 slots).
 struct TcPaging {
@@ -29,6 +29,7 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
                              int d, int C, int span, float scale, int32_t* status, void* ws, cudaStream_t stream,
                              int wait_limit_us = 0 /* 0: the default of about 200 ms */, int withhold_tile = -1 /* self-test only */,
-                             const TcPaging* paging = nullptr /* nullptr: contiguous caches of C slots */);
+                             const TcPaging* paging = nullptr /* nullptr: contiguous caches of C slots */,
+                             int out_rows = 0 /* 1: out is [B,T,Hq,d] instead of [B,Hq,T,d] */);
 
 }  // namespace s4c

@@ -150,7 +150,7 @@ template <typename T_, int D>
 __global__ void __launch_bounds__(D)
 tree_attention_combine_kernel(const float* __restrict__ ws, const int32_t* __restrict__ cache_len,
                               const int32_t* __restrict__ parent, const int32_t* __restrict__ n_nodes,
-                              T_* __restrict__ out, int T, int Hq, int C, int splits) {
+                              T_* __restrict__ out, int T, int Hq, int C, int splits, int out_rows) {
     const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     __shared__ int32_t par_s[S4C_MAX_T];
     __shared__ uint32_t anc_s[S4C_MAX_T][S4C_MASK_WORDS];
@@ -168,7 +168,8 @@ tree_attention_combine_kernel(const float* __restrict__ ws, const int32_t* __res
             den = fmaf(f, w[s * (D + 2) + D + 1], den);
         }
     float r[1] = {den > 0.f ? num / den : 0.f};
-    Elem<T_>::template store<1>(out + (((size_t)b * Hq + h) * T + i) * D + threadIdx.x, r);
+    const size_t orow = out_rows ? ((size_t)b * T + i) * Hq + h : ((size_t)b * Hq + h) * T + i;
+    Elem<T_>::template store<1>(out + orow * D + threadIdx.x, r);
 }
 
 int simt_splits(int B, int Hq, int C) {
@@ -185,22 +186,22 @@ size_t simt_workspace_bytes(int B, int T, int Hq, int d, int C) {
 
 template <typename T_, int D>
 static s4c_status launch_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
-                                 void* out, int B, int T, int Hq, int C, int splits, cudaStream_t stream) {
+                                 void* out, int B, int T, int Hq, int C, int splits, cudaStream_t stream, int out_rows = 0) {
     dim3 g2(T, Hq, B);
     tree_attention_combine_kernel<T_, D><<<g2, D, 0, stream>>>(static_cast<const float*>(ws), cache_len, parent, n_nodes,
-                                                              static_cast<T_*>(out), T, Hq, C, splits);
+                                                              static_cast<T_*>(out), T, Hq, C, splits, out_rows);
     S4C_RETURN_IF_CUDA_ERROR();
     return S4C_OK;
 }
 
 s4c_status tree_attention_combine(const void* ws, const int32_t* cache_len, const int32_t* parent, const int32_t* n_nodes,
                                   void* out, int B, int T, int Hq, int d, int C, int splits, s4c_dtype dt,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, int out_rows) {
     if (dt == S4C_F32)
-        return d == 64 ? launch_combine<float, 64>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream)
-                       : launch_combine<float, 128>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream);
-    return d == 64 ? launch_combine<__nv_bfloat16, 64>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream)
-                   : launch_combine<__nv_bfloat16, 128>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream);
+        return d == 64 ? launch_combine<float, 64>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream, out_rows)
+                       : launch_combine<float, 128>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream, out_rows);
+    return d == 64 ? launch_combine<__nv_bfloat16, 64>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream, out_rows)
+                   : launch_combine<__nv_bfloat16, 128>(ws, cache_len, parent, n_nodes, out, B, T, Hq, C, splits, stream, out_rows);
 }
 
 template <typename T_, int D>

@@ -393,7 +393,16 @@ struct TcParams {
     // paged caches (block_table == nullptr: one contiguous cache of C slots per sequence and KV head)
     const int32_t* block_table;  // [B, max_blocks]: page of logical block i of sequence b
     int max_blocks, page_tiles, n_pages;  // page_tiles = page size / 64 slots
+    int out_rows;  // 0: out is [B,Hq,T,d]; 1: [B,T,Hq,d] -- rows (b, t) of width Hq*d, as the output projection reads them
 };
+
+// element offset of the output row of packed query row gr (= g * T + t, g the head within the KV head's group)
+template <int ROWS>
+__device__ __forceinline__ size_t out_row_offset(const TcParams& prm, int b, int first_head, int gr, int T, int D) {
+    if (!ROWS) return ((size_t)(b * prm.Hq + first_head) * T + gr) * D;
+    const int g = gr / T, t = gr - g * T;
+    return (((size_t)b * T + t) * prm.Hq + first_head + g) * D;
+}
 
 // Tile range of a split: tiles are dealt out as evenly as whole tiles allow, the odd ones to the FIRST splits -- the last
 // split holds the tree's own tiles, which cost more than a tile of the prefix (they are masked), and every split of a
@@ -415,7 +424,7 @@ __device__ __forceinline__ void split_range(int n_tiles, int splits, int split, 
 // PUSH (one row tile, no turns, few rows): instead of parking partials for the peers to fetch, every CTA stores its
 // (copy-merged) rows into a receive area of the row's owner that is used for nothing else, so no barrier has to say
 // "my tile buffers are dead" first; after one cluster barrier the owner merges from its own shared memory and leaves.
-template <int D, int NM, int REP, int TC, int PUSH>
+template <int D, int NM, int REP, int TC, int PUSH, int ROWS = 0 /* 1: out is [B,T,Hq,d]; a variant of its own, so that the [B,Hq,T,d] kernels stay as they are */>
 __global__ void __launch_bounds__(TcCfg<D, NM, TC, PUSH>::kThreads, TcCfg<D, NM, TC, PUSH>::kCtasPerSm)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const TcParams prm) {
@@ -951,7 +960,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             __floats2bfloat162_rn(__uint_as_float(o[c]) * inv, __uint_as_float(o[c + 1]) * inv);
                         packed[c >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
                     }
-                    uint4* dst = reinterpret_cast<uint4*>(prm.out + orow * D + cc * 32);
+                    uint4* dst = reinterpret_cast<uint4*>(prm.out + out_row_offset<ROWS>(prm, b, hk * G, gr, T, D) + cc * 32);
 #pragma unroll
                     for (int v = 0; v < 4; ++v)
                         dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
@@ -1005,7 +1014,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 const int gr = mt0 * kBM + lr;
                 const float inv = ((gr % T) < n && den > 0.f) ? 1.f / den : 0.f;
-                __nv_bfloat16* dst = prm.out + ((size_t)(b * prm.Hq + hk * G) * T + gr) * D + lane * EPL;
+                __nv_bfloat16* dst = prm.out + out_row_offset<ROWS>(prm, b, hk * G, gr, T, D) + lane * EPL;
                 const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
                 if (gave_up) break;
                 if (EPL == 4) {
@@ -1096,7 +1105,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     if (!ok[u] || gave_up) continue;
                     const int gr = (mt0 + tt[u]) * kBM + lr[u];
                     const float inv = ((gr % T) < n && den[u] > 0.f) ? 1.f / den[u] : 0.f;
-                    __nv_bfloat16* dst = prm.out + ((size_t)(b * prm.Hq + hk * G) * T + gr) * D + lane * EPL;
+                    __nv_bfloat16* dst = prm.out + out_row_offset<ROWS>(prm, b, hk * G, gr, T, D) + lane * EPL;
                     const __nv_bfloat162 h0 = __floats2bfloat162_rn(num[u][0] * inv, num[u][1] * inv);
                     if (EPL == 4) {
                         const __nv_bfloat162 h1 = __floats2bfloat162_rn(num[u][2] * inv, num[u][3] * inv);
@@ -1291,14 +1300,14 @@ size_t tc_workspace_bytes(int B, int T, int Hq, int Hkv, int d, int C) {
     return s == 0 ? 0 : round_up((size_t)B * Hq * T * s * (d + 2) * sizeof(float), 256);
 }
 
-template <int D, int NM, int REP, int TC, int PUSH>
-static s4c_status launch_tc(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
+template <int D, int NM, int REP, int TC, int PUSH, int ROWS>
+static s4c_status launch_tc_layout(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
     using Cfg = TcCfg<D, NM, TC, PUSH>;
     static bool configured[64] = {};  // the opt-ins (dynamic shared memory, cluster size) are per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return S4C_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP, TC, PUSH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(tree_attention_tc_kernel<D, NM, REP, TC, PUSH, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return S4C_ERR_CUDA;
         configured[dev] = true;
@@ -1329,11 +1338,17 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
     }
     cfg.attrs = attrs;
     cfg.numAttrs = na;
-    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP, TC, PUSH>, mq, mk, mv, prm) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<D, NM, REP, TC, PUSH, ROWS>, mq, mk, mv, prm) != cudaSuccess) {
         cudaGetLastError();
         return S4C_ERR_CUDA;
     }
     return S4C_OK;
+}
+
+template <int D, int NM, int REP, int TC, int PUSH>
+static s4c_status launch_tc(const void* q, const void* k, const void* v, const TcParams& prm, int B, cudaStream_t stream) {
+    return prm.out_rows ? launch_tc_layout<D, NM, REP, TC, PUSH, 1>(q, k, v, prm, B, stream)
+                        : launch_tc_layout<D, NM, REP, TC, PUSH, 0>(q, k, v, prm, B, stream);
 }
 
 // `span` (<= C) is the number of slots the launch is shaped for: the host's bound on the live length (committed tokens
@@ -1342,8 +1357,9 @@ static s4c_status launch_tc(const void* q, const void* k, const void* v, const T
 s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const int32_t* cache_len,
                              const int32_t* parent, const int32_t* n_nodes, void* out, int B, int T, int Hq, int Hkv,
                              int d, int C_slots, int span, float scale, int32_t* status, void* ws, cudaStream_t stream,
-                             int wait_limit_us, int withhold_tile, const TcPaging* paging) {
+                             int wait_limit_us, int withhold_tile, const TcPaging* paging, int out_rows) {
     TcParams prm;
+    prm.out_rows = out_rows;
     prm.cache_len = cache_len, prm.parent = parent, prm.n_nodes = n_nodes;
     prm.out = static_cast<__nv_bfloat16*>(out), prm.ws = static_cast<float*>(ws), prm.status = status;
     prm.T = T, prm.Hq = Hq, prm.Hkv = Hkv, prm.C = C_slots;
@@ -1388,7 +1404,7 @@ s4c_status tree_attention_tc(const void* q, const void* k, const void* v, const 
     if (st != S4C_OK) return st;
     if (prm.mode == kModeWorkspace)
         return tree_attention_combine(ws, cache_len, parent, n_nodes, out, B, T, Hq, d, prm.C, prm.splits * rep * turns, S4C_BF16,
-                                      stream);
+                                      stream, out_rows);
     return S4C_OK;
 }
 

@@ -5,14 +5,12 @@
     f' = Decoder_layer(h)                                                         (Eq. 4; one LLaMA-family layer)
          a  = rmsnorm(h)                               (the same call)
          q, K/V tree slots = rope(a Wqkv^T)            s4c_qkv_rope
-         o  = tree attention(q, cache)                 s4c_tree_attention
+         o  = tree attention(q, cache)                 s4c_tree_attention_rows (written as rows [B*T, Hq*d])
          h2 = h + o Wo^T,  m = rmsnorm(h2)             s4c_linear_rmsnorm, residual
          f' = h2 + (silu(m Wg^T) * m Wu^T) Wd^T        s4c_linear (gated), s4c_linear (residual)
     ranked choices = top-k(LM_head(f'))                s4c_lm_head_topk           (Eq. 5; k = 1 is the Argmax)
 
-Only buffers, views and the order of the calls live here; every arithmetic step runs in the library's kernels.  The one
-torch operation on data is the transpose of the attention output [B,Hq,T,d] into rows [B*T, Hq*d] for the output
-projection (a copy, no arithmetic).  Weights are whatever the caller passes: this repository has no trained drafter, the
+Only buffers, views and the order of the calls live here; every step runs in the library's kernels.  Weights are whatever the caller passes: this repository has no trained drafter, the
 benchmark and the tests use seeded random weights of the paper's models' shapes.
 """
 from __future__ import annotations
@@ -65,8 +63,7 @@ class DrafterHead:
         bf = dict(dtype=torch.bfloat16, device=dev)
         self.e, self.h, self.a = torch.empty(R, H, **bf), torch.empty(R, H, **bf), torch.empty(R, H, **bf)
         self.q = torch.empty(B, Hq, T, d, **bf)
-        self.attn = torch.empty(B, Hq, T, d, **bf)
-        self.o_in = torch.empty(R, Hq * d, **bf)
+        self.o_in = torch.empty(R, Hq * d, **bf)  # the attention output as rows [B*T, Hq*d] = [B,T,Hq,d]
         self.h2, self.m = torch.empty(R, H, **bf), torch.empty(R, H, **bf)
         self.act = torch.empty(R, inter, **bf)
         self.f_out = torch.empty(R, H, **bf)
@@ -95,9 +92,8 @@ class DrafterHead:
                            workspace=self.ws_lin)
         s4c.qkv_rope(self.a.view(self.B, self.T, -1), w.qkv, cache_len, parent, self.q, k_cache, v_cache, n_nodes, self.rope_theta,
                      status=self.status_qkv, workspace=self.ws_qkv)
-        s4c.tree_attention(self.q, k_cache, v_cache, cache_len, parent, n_nodes, out=self.attn, status=self.status_attn,
-                           workspace=self.ws_attn, max_cache_len=max_cache_len)
-        self.o_in.view(self.B, self.T, self.Hq, self.d).copy_(self.attn.permute(0, 2, 1, 3))  # rows for the output projection
+        s4c.tree_attention(self.q, k_cache, v_cache, cache_len, parent, n_nodes, out=self.o_in.view(self.B, self.T, self.Hq, self.d),
+                           status=self.status_attn, workspace=self.ws_attn, max_cache_len=max_cache_len, rows=True)
         s4c.linear_rmsnorm(self.o_in, w.o, w.norm2, self.eps, residual=self.h, out=self.h2, norm_out=self.m, workspace=self.ws_lin)
         s4c.linear(self.m, w.gate_up, gate=True, out=self.act, workspace=self.ws_lin)
         s4c.linear(self.act, w.down, residual=self.h2, out=self.f_out, workspace=self.ws_lin)

@@ -20,7 +20,7 @@ SEQ_OK, SEQ_BAD_PARENT, SEQ_TOKEN_RANGE, SEQ_CAPACITY, SEQ_DEPTH, SEQ_BAD_PATH, 
 SEQ_BAD_PAGE = 128
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WORKSPACE", "ERR_UNSUPPORTED", "ERR_CUDA"]
 
-EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention",
+EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_bytes", "s4c_tree_attention", "s4c_tree_attention_rows",
            "s4c_tree_accept_workspace_bytes", "s4c_tree_accept", "s4c_tree_accept_noalloc", "s4c_kv_compact",
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
@@ -52,6 +52,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_tree_attention_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
     lib.s4c_tree_attention.restype = i
     lib.s4c_tree_attention.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_tree_attention_rows.restype = i
+    lib.s4c_tree_attention_rows.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, i, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
     lib.s4c_tree_accept_workspace_bytes.restype = sz
     lib.s4c_tree_accept_workspace_bytes.argtypes = [i, i, i]
     lib.s4c_tree_accept.restype = i
@@ -161,10 +163,11 @@ def tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dtype) -> int:
 
 
 def tree_attention(q, k_cache, v_cache, cache_len, parent, n_nodes=None, out=None, scale: float = 0.0, status=None,
-                   workspace=None, stream=None, max_cache_len: int = 0):
+                   workspace=None, stream=None, max_cache_len: int = 0, rows: bool = False):
     """s4c_tree_attention: q [B,Hq,T,d], k_cache/v_cache [B,Hkv,C,d] -> out [B,Hq,T,d] (same dtype).
 
-    ``max_cache_len``: the host's upper bound on ``cache_len`` (0 = unknown); it shapes the launch, never the result."""
+    ``max_cache_len``: the host's upper bound on ``cache_len`` (0 = unknown); it shapes the launch, never the result.
+    ``rows``: s4c_tree_attention_rows -- out is [B,T,Hq,d], the rows the output projection reads (bf16 only)."""
     B, Hq, T, d = q.shape
     _, Hkv, C, _ = k_cache.shape
     if k_cache.shape != (B, Hkv, C, d) or v_cache.shape != (B, Hkv, C, d):
@@ -172,12 +175,12 @@ def tree_attention(q, k_cache, v_cache, cache_len, parent, n_nodes=None, out=Non
     if k_cache.dtype != q.dtype or v_cache.dtype != q.dtype:
         raise TypeError("q, k_cache and v_cache must share one dtype")
     if out is None:
-        out = torch.empty_like(q)
+        out = torch.empty(B, T, Hq, d, dtype=q.dtype, device=q.device) if rows else torch.empty_like(q)
     dt = _dt(q)
     need = int(_lib.s4c_tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, dt))
     if workspace is None:
         workspace = _workspace(need, q.device, "attn")
-    rc = _lib.s4c_tree_attention(
+    rc = (_lib.s4c_tree_attention_rows if rows else _lib.s4c_tree_attention)(
         _dev(q, name="q"), _dev(k_cache, name="k_cache"), _dev(v_cache, name="v_cache"),
         _dev(cache_len, torch.int32, "cache_len"), _dev(parent, torch.int32, "parent"),
         _dev(n_nodes, torch.int32, "n_nodes"), _dev(out, q.dtype, "out"), B, T, Hq, Hkv, d, C, int(max_cache_len), dt,
@@ -185,7 +188,7 @@ def tree_attention(q, k_cache, v_cache, cache_len, parent, n_nodes=None, out=Non
         _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
         0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
     if rc:
-        raise S4CError("s4c_tree_attention", rc)
+        raise S4CError("s4c_tree_attention_rows" if rows else "s4c_tree_attention", rc)
     return out
 
 

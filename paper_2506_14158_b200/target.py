@@ -6,7 +6,7 @@ chat models):
     a0 = rmsnorm(x0)                                             s4c_rmsnorm
     per layer l:
         q, K/V tree slots = rope(a_l Wqkv^T)                     s4c_qkv_rope / s4c_qkv_rope_same_tree (position = committed length + depth; the rotary table once per pass)
-        o  = tree attention(q, cache_l)                          s4c_tree_attention    (tree mask from parent[])
+        o  = tree attention(q, cache_l)                          s4c_tree_attention_rows (tree mask from parent[]; written as rows [B*T, Hq*d])
         h  = x_l + o Wo^T,          m = rmsnorm(h)               s4c_linear_rmsnorm
         g  = silu(m Wg^T) * (m Wu^T)                             s4c_linear, gated
         x_{l+1} = h + g Wd^T,       a_{l+1} = rmsnorm(x_{l+1})   s4c_linear_rmsnorm    (the next layer's norm, or the final norm)
@@ -14,8 +14,7 @@ chat models):
     longest accepted path, next token                            s4c_tree_accept_tokens
     accepted K/V rows of every layer -> committed slots, features of the path gathered, lengths advanced     s4c_kv_compact
 
-Only buffers and the order of the calls live here; every arithmetic step runs in the library's kernels.  The one torch
-operation on data is, per layer, the transpose of the attention output [B,Hq,T,d] into rows [B*T, Hq*d] (a copy).  The
+Only buffers and the order of the calls live here; every step runs in the library's kernels.  The
 "features" handed to the next drafting round are the last layer's output x_n (before the final norm).  Weights are the
 caller's: this repository has no trained model; tests and the benchmark use seeded random weights of the paper's
 models' shapes.
@@ -82,7 +81,6 @@ class TargetVerify:
         self.x = [torch.empty(R, H, **bf) for _ in range(sets + 1)]  # x[l]: the input of layer l (x[0]: the embeddings)
         self.a = [torch.empty(R, H, **bf) for _ in range(sets + 1)]  # its normalisation
         self.q = [torch.empty(B, Hq, T, d, **bf) for _ in range(sets)]
-        self.attn = [torch.empty(B, Hq, T, d, **bf) for _ in range(sets)]
         self.o_in, self.h, self.m, self.act = rows(Hq * d), rows(H), rows(H), rows(inter)
         self.sets = sets
         self.status_qkv = torch.zeros(1, B, **i32)  # written by the first layer's call, timeouts of the others OR-ed in
@@ -118,9 +116,9 @@ class TargetVerify:
             else:
                 s4c.qkv_rope_same_tree(self.a[i_in].view(B, T, -1), lw.qkv, self.q[i], self.k_caches[l], self.v_caches[l], self.ws_qkv,
                                        status=self.status_qkv[0])
-            s4c.tree_attention(self.q[i], self.k_caches[l], self.v_caches[l], cache_len, parent, n_nodes, out=self.attn[i],
-                               status=self.status_attn[l], workspace=self.ws_attn, max_cache_len=max_cache_len)
-            self.o_in[i].view(B, T, self.Hq, self.d).copy_(self.attn[i].permute(0, 2, 1, 3))  # rows for the output projection
+            s4c.tree_attention(self.q[i], self.k_caches[l], self.v_caches[l], cache_len, parent, n_nodes,
+                               out=self.o_in[i].view(B, T, self.Hq, self.d), status=self.status_attn[l], workspace=self.ws_attn,
+                               max_cache_len=max_cache_len, rows=True)
             s4c.linear_rmsnorm(self.o_in[i], lw.o, lw.norm2, self.eps, residual=self.x[i_in], out=self.h[i], norm_out=self.m[i],
                                workspace=self.ws_lin)
             s4c.linear(self.m[i], lw.gate_up, gate=True, out=self.act[i], workspace=self.ws_lin)

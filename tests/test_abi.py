@@ -78,6 +78,12 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert att(scale=-1.0) == 2 and att(hint=-1) == 2
     assert att(B=0) == 0
     assert att(T=64, Hq=8, Hkv=2, C=24704, ws=None) == 5   # this grid splits wider than a cluster and needs a workspace
+    lib.s4c_tree_attention_rows.argtypes = lib.s4c_tree_attention.argtypes
+    attr = lambda **kw: lib.s4c_tree_attention_rows(*[kw.get(k, d) for k, d in [
+        ("q", P), ("k", P), ("v", P), ("cl", P), ("par", P), ("nn", None), ("out", P), ("B", 1), ("T", 8), ("Hq", 4),
+        ("Hkv", 2), ("d", 128), ("C", 256), ("hint", 0), ("dt", 1), ("scale", 0.0), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
+    assert attr(out=None) == 1 and attr(T=129) == 2 and attr(k=P + 2) == 4 and attr(B=0) == 0
+    assert attr(dt=0) == 6                       # S4C_ERR_UNSUPPORTED: the row layout is written by the bf16 kernel only
     acc = lambda **kw: lib.s4c_tree_accept(*[kw.get(k, d) for k, d in [
         ("lg", P), ("dp", P), ("tok", P), ("par", P), ("nn", None), ("tau", 1.0), ("u", P), ("B", 1), ("T", 8),
         ("V", 100), ("md", 7), ("al", P), ("path", P), ("nt", P), ("tie", None), ("st", None), ("ws", None), ("wsb", 0),

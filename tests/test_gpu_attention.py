@@ -229,3 +229,41 @@ def test_the_hint_never_changes_the_result_class():
         assert_attention_close(got, ref, gst, rst, ATTN_TOL["bf16"])
         outs.append(got)
     np.testing.assert_array_equal(outs[1], outs[3])
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,T,d,Ls", [
+    (1, 32, 32, 26, 128, [1024]),            # the 7B shape: four row copies, pushed partials
+    (4, 32, 8, 64, 128, [4096, 100, 0, 2000]),  # the 8B shape: two row tiles per CTA (GQA rows packed g * T + t)
+    (2, 16, 8, 50, 64, [5000, 4321]),        # two softmax groups taking turns, GQA, d = 64
+    (1, 8, 2, 64, 128, [24600]),             # merged through the workspace by the second kernel
+    (10, 32, 32, 20, 128, [300, 17, 0, 640, 129, 300, 64, 511, 1, 77]),  # half-SM CTAs
+    (1, 16, 2, 128, 128, [300]),             # eight row tiles, one per CTA
+    (3, 4, 4, 7, 64, [5, 0, 33]),            # a single split, stored directly
+])
+def test_rows_layout_holds_the_same_values(B, Hq, Hkv, T, d, Ls):
+    # s4c_tree_attention_rows writes out[b, t, h, :]: every element equals the [B,Hq,T,d] call's, bit for bit, padding and
+    # flagged sequences included (neither call touches those rows)
+    from paper_2506_14158_b200 import s4c
+    from parity import Guarded, dev
+
+    rng = np.random.default_rng(B * 100 + T)
+    C = max(Ls) + T + 5
+    g = torch.Generator().manual_seed(B + T)
+    q = torch.randn((B, Hq, T, d), generator=g).to(torch.bfloat16).cuda()
+    k = torch.randn((B, Hkv, C, d), generator=g).to(torch.bfloat16).cuda()
+    v = torch.randn((B, Hkv, C, d), generator=g).to(torch.bfloat16).cuda()
+    parent = np.stack([W.random_tree(T, 8, rng) for _ in range(B)]).astype(np.int32)
+    n_nodes = rng.integers(max(1, T // 2), T + 1, B).astype(np.int32)
+    if B >= 3:
+        parent[1, min(3, T - 1)] = T - 1 if T > 4 else parent[1, min(3, T - 1)]   # sequence 1: malformed (a parent not before its child)
+    cl = dev(np.asarray(Ls, dtype=np.int32))
+    std = Guarded((B, Hq, T, d), torch.bfloat16, fill=-3.0)
+    rows = Guarded((B, T, Hq, d), torch.bfloat16, fill=-3.0)
+    st0, st1 = torch.empty(B, dtype=torch.int32, device="cuda"), torch.empty(B, dtype=torch.int32, device="cuda")
+    s4c.tree_attention(q, k, v, cl, dev(parent), dev(n_nodes), out=std.t, status=st0, max_cache_len=max(Ls))
+    s4c.tree_attention(q, k, v, cl, dev(parent), dev(n_nodes), out=rows.t, status=st1, max_cache_len=max(Ls), rows=True)
+    torch.cuda.synchronize()
+    std.check("s4c_tree_attention out"), rows.check("s4c_tree_attention_rows out")
+    assert torch.equal(st0, st1)
+    assert torch.equal(rows.t, std.t.permute(0, 2, 1, 3).contiguous())
+    assert (std.t != -3.0).any()
