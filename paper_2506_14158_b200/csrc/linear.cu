@@ -445,7 +445,7 @@ static bool ln_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, int H,
 //     (7B-shaped gate/up projection: 172 tiles of 64 columns took 50 us, 138 tiles of 80 take one wave);
 //   * per K slice of 64 elements a CTA needs the longest of: the issuing thread's fixed ~0.3 us (four tcgen05.mma, a
 //     commit, a wait -- whatever the tile's width, so narrow tiles move few bytes per issue); the tensor pipe's time for
-//     128 x bn x 64 products; its share of the weight stream from HBM (what one SM pulls, ~60 GB/s, or HBM divided
+//     128 x bn x 64 products; its share of the weight stream from HBM (what one SM pulls, ~55 GB/s, or HBM divided
 //     among the CTAs of the wave; row tiles of one column tile share the weights through L2); the stage's bytes over
 //     what an SM takes in from L2 (~100 GB/s); and the ring's turn-round (a slot is refilled ~1.3 us after its
 //     products retire, so few deep stages starve the issuer);
@@ -456,7 +456,7 @@ struct LnPlan {
     int bn, splits, x_rows, stages, cols_per_tile, m_tiles, n_tiles, nm;
 };
 static LnPlan ln_plan(int R, int K1, int K2, int N, int gate) {
-    constexpr double kIssueUs = 0.30, kMmaUsPerCol = 0.27 / 256.0, kSmBytesPerUs = 60e3, kHbmBytesPerUs = 6.4e6, kL2BytesPerUs = 100e3,
+    constexpr double kIssueUs = 0.30, kMmaUsPerCol = 0.27 / 256.0, kSmBytesPerUs = 55e3, kHbmBytesPerUs = 6.4e6, kL2BytesPerUs = 100e3,
                      kTurnUs = 1.3, kWaveUs = 2.5, kFinishUs = 3.0, kPartialBytesPerUs = 4.0e6, kIssueTwo = 1.5;
     constexpr int kSms = 148;
     const int k_steps = (K1 + K2) / kLnBK;
