@@ -318,6 +318,18 @@ s4c_status s4c_tree_accept_tokens(const int32_t* target_token, const int32_t* to
                                   const int32_t* n_nodes, int B, int T, int V, int max_depth, int32_t* accept_len,
                                   int32_t* path, int32_t* next_token, int32_t* status, s4c_stream_t stream);
 
+/* s4c_lm_head_logits -- the LM head when the logits themselves are wanted: verification by speculative
+ * sampling (Eq. 11-12, temperature > 0) needs the target's distribution at the walked nodes, so
+ * logits[r, v] = sum_h hidden[r, h] * weight[v, h] are written out as float32 [R, V] (the float32 sums
+ * of the bf16 products, unrounded) in the layout s4c_tree_accept reads.  hidden [R, H], weight [V, H]
+ * bf16; H a multiple of 64, V a multiple of 8; status and workspace as s4c_linear
+ * (s4c_lm_head_logits_workspace_bytes(R, V, H) bytes).  Greedy verification does not need this call:
+ * s4c_lm_head_greedy keeps the choice and writes no logits. */
+size_t s4c_lm_head_logits_workspace_bytes(int R, int V, int H);
+
+s4c_status s4c_lm_head_logits(const void* hidden, const void* weight, int R, int V, int H, float* logits,
+                              int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream);
+
 /* ------------------------------------------------------------------------------------------
  * s4c_qkv_rope -- the input side of a decoder layer in the verify pass (Section 3.2: the target's
  * forward pass over the T tree tokens; the paper's targets are LLaMA-family models): for every tree

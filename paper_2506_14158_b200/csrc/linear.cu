@@ -43,6 +43,7 @@ struct LnParams {
     const __nv_bfloat16* bias;     // [N] or null
     const __nv_bfloat16* residual; // [R, N] or null
     __nv_bfloat16* out;            // [R, N]
+    float* out_f32;                // [R, N] float32 instead of `out` (the LM head's logits), or null
     int32_t* status;               // one word or null
     int splits;                    // CTAs that share a tile's K slices (grid.z); > 1: raw partial sums go to `partial`
     float* partial;                // [splits][R][N or 2N] float32, read by linear_finish_kernel
@@ -230,6 +231,11 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x1, const __grid_constant_
                                 y[2 * j] += f.x, y[2 * j + 1] += f.y;
                             }
                         }
+                        if (prm.out_f32) {  // the sums as they are (logits)
+                            float4* dst = reinterpret_cast<float4*>(prm.out_f32 + (size_t)r * prm.N + col);
+                            dst[0] = make_float4(y[0], y[1], y[2], y[3]), dst[1] = make_float4(y[4], y[5], y[6], y[7]);
+                            continue;
+                        }
                         uint32_t pk[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -309,7 +315,8 @@ __device__ __forceinline__ uint4 scale8(const uint4& v, const uint4& g, float sc
 __global__ void __launch_bounds__(256)
 linear_finish_kernel(const float* __restrict__ partial, int splits, int R, int N, int gate, const __nv_bfloat16* __restrict__ bias,
                      const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ out,
-                     const __nv_bfloat16* __restrict__ norm_weight, float norm_eps, __nv_bfloat16* __restrict__ norm_out) {
+                     const __nv_bfloat16* __restrict__ norm_weight, float norm_eps, __nv_bfloat16* __restrict__ norm_out,
+                     float* __restrict__ out_f32) {
     __shared__ float red[8];
     griddep_wait();
     griddep_launch_dependents();
@@ -337,6 +344,11 @@ linear_finish_kernel(const float* __restrict__ partial, int splits, int R, int N
                 y[j] = silu(y[j]) * up[j];
             }
             if (residual) y[j] += __bfloat162float(residual[(size_t)r * N + col + j]);
+        }
+        if (out_f32) {  // the sums as they are (logits); no normalisation in this form
+            float4* dst = reinterpret_cast<float4*>(out_f32 + (size_t)r * N + col);
+            dst[0] = make_float4(y[0], y[1], y[2], y[3]), dst[1] = make_float4(y[4], y[5], y[6], y[7]);
+            continue;
         }
         uint32_t pk[4];
 #pragma unroll
@@ -514,7 +526,7 @@ namespace s4c {
 // s4c_linear, and s4c_linear_rmsnorm when norm_weight is given (norm_out = rmsnorm(out))
 static s4c_status ln_run(const void* x1, const void* x2, const void* w, const void* bias, const void* residual, void* out, int R,
                          int K1, int K2, int N, int gate, const void* norm_weight, float norm_eps, void* norm_out, int32_t* status,
-                         void* workspace, size_t workspace_bytes, s4c_stream_t stream_) {
+                         void* workspace, size_t workspace_bytes, s4c_stream_t stream_, bool out_is_f32 = false) {
     if (!x1 || !w || !out || (K2 > 0 && !x2) || (norm_weight && !norm_out)) return S4C_ERR_NULL;
     if (R < 0 || N < 8 || N % 8 != 0 || K1 < kLnBK || K1 % kLnBK != 0 || K2 < 0 || K2 % kLnBK != 0) return S4C_ERR_SHAPE;
     if (norm_weight && !(norm_eps >= 0.f)) return S4C_ERR_SHAPE;
@@ -550,7 +562,8 @@ static s4c_status ln_run(const void* x1, const void* x2, const void* w, const vo
     prm.R = R, prm.N = N, prm.k1_steps = K1 / kLnBK, prm.k2_steps = K2 / kLnBK, prm.gate = gate ? 1 : 0;
     prm.x_rows = pl.x_rows, prm.stages = pl.stages, prm.bn = pl.bn, prm.cols = pl.cols_per_tile, prm.nm = pl.nm;
     prm.bias = static_cast<const __nv_bfloat16*>(bias), prm.residual = static_cast<const __nv_bfloat16*>(residual);
-    prm.out = static_cast<__nv_bfloat16*>(out), prm.status = status;
+    prm.out = out_is_f32 ? nullptr : static_cast<__nv_bfloat16*>(out), prm.out_f32 = out_is_f32 ? static_cast<float*>(out) : nullptr;
+    prm.status = status;
     prm.splits = pl.splits, prm.partial = static_cast<float*>(workspace);
     const __nv_bfloat16* nw = static_cast<const __nv_bfloat16*>(norm_weight);
     __nv_bfloat16* no = static_cast<__nv_bfloat16*>(norm_out);
@@ -558,7 +571,7 @@ static s4c_status ln_run(const void* x1, const void* x2, const void* w, const vo
                         prm) == cudaSuccess;
     if (ok && pl.splits > 1)  // the finishing kernel holds whole rows: it normalises them as well
         ok = ln_launch(linear_finish_kernel, dim3(R, 1, 1), 256, 0, stream, (const float*)prm.partial, pl.splits, R, N, gate ? 1 : 0,
-                       prm.bias, prm.residual, prm.out, nw, norm_eps, no) == cudaSuccess;
+                       prm.bias, prm.residual, prm.out, nw, norm_eps, no, prm.out_f32) == cudaSuccess;
     else if (ok && nw)
         ok = ln_launch(rmsnorm_kernel, dim3(R, 1, 1), 256, 0, stream, (const __nv_bfloat16*)prm.out, nw, norm_eps, N, no) == cudaSuccess;
     if (!ok) {
@@ -582,6 +595,14 @@ extern "C" s4c_status s4c_linear_rmsnorm(const void* x1, const void* x2, const v
     if (!norm_weight) return S4C_ERR_NULL;
     return s4c::ln_run(x1, x2, w, bias, residual, out, R, K1, K2, N, 0, norm_weight, eps, norm_out, status, workspace, workspace_bytes,
                        stream);
+}
+
+extern "C" size_t s4c_lm_head_logits_workspace_bytes(int R, int V, int H) { return s4c_linear_workspace_bytes(R, H, 0, V, 0); }
+
+extern "C" s4c_status s4c_lm_head_logits(const void* hidden, const void* weight, int R, int V, int H, float* logits, int32_t* status,
+                                         void* workspace, size_t workspace_bytes, s4c_stream_t stream) {
+    return s4c::ln_run(hidden, nullptr, weight, nullptr, nullptr, logits, R, H, 0, V, 0, nullptr, 0.f, nullptr, status, workspace,
+                       workspace_bytes, stream, true);
 }
 
 extern "C" s4c_status s4c_rmsnorm(const void* x, const void* weight, float eps, int R, int H, void* out, s4c_stream_t stream_) {

@@ -26,7 +26,7 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
            "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
            "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_qkv_rope_same_tree", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
-           "s4c_tree_build_topk", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_linear_rmsnorm", "s4c_rmsnorm", "s4c_embed_gather"]
+           "s4c_tree_build_topk", "s4c_lm_head_logits_workspace_bytes", "s4c_lm_head_logits", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_linear_rmsnorm", "s4c_rmsnorm", "s4c_embed_gather"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
@@ -94,6 +94,10 @@ def _load() -> ctypes.CDLL:
     lib.s4c_lm_head_topk.argtypes = [vp, vp, i, i, i, i, i32p, vp, i32p, vp, sz, vp]
     lib.s4c_tree_build_topk.restype = i
     lib.s4c_tree_build_topk.argtypes = [i32p, i, vp, i, i32p, i32p, i, i, i32p, i32p, i32p, i32p, vp]
+    lib.s4c_lm_head_logits_workspace_bytes.restype = sz
+    lib.s4c_lm_head_logits_workspace_bytes.argtypes = [i, i, i]
+    lib.s4c_lm_head_logits.restype = i
+    lib.s4c_lm_head_logits.argtypes = [vp, vp, i, i, i, vp, i32p, vp, sz, vp]
     lib.s4c_linear_workspace_bytes.restype = sz
     lib.s4c_linear_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.s4c_linear.restype = i
@@ -449,6 +453,26 @@ def lm_head_greedy(hidden, weight, token=None, max_logit=None, status=None, work
     if rc:
         raise S4CError("s4c_lm_head_greedy", rc)
     return dict(token=token, max_logit=max_logit, status=status)
+
+
+def lm_head_logits_workspace_bytes(R, V, H) -> int:
+    return int(_lib.s4c_lm_head_logits_workspace_bytes(R, V, H))
+
+
+def lm_head_logits(hidden, weight, logits=None, status=None, workspace=None, stream=None):
+    """s4c_lm_head_logits: logits [R,V] float32 = hidden @ weight^T (bf16 in, f32 sums), for stochastic verification."""
+    R, H = hidden.shape
+    V = weight.shape[0]
+    logits = torch.empty(R, V, dtype=torch.float32, device=hidden.device) if logits is None else logits
+    if workspace is None:
+        workspace = _workspace(int(_lib.s4c_lm_head_logits_workspace_bytes(R, V, H)), hidden.device, "linear")
+    rc = _lib.s4c_lm_head_logits(_dev(hidden, torch.bfloat16, "hidden"), _dev(weight, torch.bfloat16, "weight"), R, V, H,
+                                 _dev(logits, torch.float32, "logits"), _dev(status, torch.int32, "status"),
+                                 _dev(workspace, name="workspace"), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                 _stream(stream))
+    if rc:
+        raise S4CError("s4c_lm_head_logits", rc)
+    return logits
 
 
 def tree_accept_tokens(target_token, tokens, parent, V: int, n_nodes=None, max_depth: Optional[int] = None, accept_len=None,

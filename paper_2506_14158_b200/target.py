@@ -10,8 +10,12 @@ chat models):
         h  = x_l + o Wo^T,          m = rmsnorm(h)               s4c_linear_rmsnorm
         g  = silu(m Wg^T) * (m Wu^T)                             s4c_linear, gated
         x_{l+1} = h + g Wd^T,       a_{l+1} = rmsnorm(x_{l+1})   s4c_linear_rmsnorm    (the next layer's norm, or the final norm)
+    greedy (Section 4.1):
     target token per node = Argmax(LM_head(a_n))                 s4c_lm_head_greedy    (no [B,T,V] logits in memory)
     longest accepted path, next token                            s4c_tree_accept_tokens
+    speculative sampling (Eq. 11-12, temperature > 0):
+    logits = LM_head(a_n) as float32 [B,T,V]                     s4c_lm_head_logits
+    accept / reject / residual resampling along the tree         s4c_tree_accept
     accepted K/V rows of every layer -> committed slots, features of the path gathered, lengths advanced     s4c_kv_compact
 
 Only buffers and the order of the calls live here; every step runs in the library's kernels.  The
@@ -63,7 +67,7 @@ class TargetVerify:
     ``keep`` keeps every layer's intermediate rows (for tests); otherwise two sets of row buffers alternate."""
 
     def __init__(self, w: TargetWeights, B: int, T: int, Hq: int, Hkv: int, d: int, C: int, k_caches, v_caches, max_depth: int,
-                 eps: float = 1e-5, rope_theta: float = 10000.0, keep: bool = False):
+                 eps: float = 1e-5, rope_theta: float = 10000.0, keep: bool = False, stochastic: bool = False):
         self.w, self.B, self.T, self.Hq, self.Hkv, self.d, self.C = w, B, T, Hq, Hkv, d, C
         self.eps, self.rope_theta, self.max_depth = eps, rope_theta, max_depth
         self.k_caches, self.v_caches = list(k_caches), list(v_caches)
@@ -97,13 +101,22 @@ class TargetVerify:
         self.ws_qkv = u8(s4c.qkv_rope_workspace_bytes(B, T, d))
         self.ws_attn = u8(s4c.tree_attention_workspace_bytes(B, T, Hq, Hkv, d, C, torch.bfloat16))
         self.ws_head = u8(s4c.lm_head_greedy_workspace_bytes(R, V, H))
+        self.stochastic = stochastic
+        if stochastic:  # the logits exist in memory only on this route
+            self.logits = torch.empty(B, T, V, dtype=torch.float32, device=dev)
+            self.near_tie = torch.empty(B, T, dtype=torch.uint8, device=dev)
+            self.ws_logits = u8(s4c.lm_head_logits_workspace_bytes(R, V, H))
+            self.ws_accept = u8(s4c.tree_accept_workspace_bytes(B, T, V))
         self.ws_lin = u8(max(s4c.linear_workspace_bytes(R, Hq * d, 0, H), s4c.linear_workspace_bytes(R, H, 0, inter, True),
                              s4c.linear_workspace_bytes(R, inter, 0, H)))  # the products run one after another
 
     def forward(self, tokens: torch.Tensor, cache_len: torch.Tensor, parent: torch.Tensor, n_nodes: Optional[torch.Tensor] = None,
-                max_cache_len: int = 0, compact: bool = True):
+                max_cache_len: int = 0, compact: bool = True, temperature: float = 0.0, draft_probs: Optional[torch.Tensor] = None,
+                uniforms: Optional[torch.Tensor] = None):
         """tokens, parent [B,T] int32 (the tree), cache_len [B] int32 (advanced in place when ``compact``).
-        Returns dict(accept_len, path, next_token, target_token [B,T], features [B,max_depth+1,H], status)."""
+        temperature > 0 (a pass built with ``stochastic=True``): speculative sampling against draft_probs [B,T,V] float32 (row n: the
+        drafter's distribution after node n) with the caller's uniforms (as s4c_tree_accept takes them).
+        Returns dict(accept_len, path, next_token, target_token [B,T] (greedy route), features [B,max_depth+1,H], status)."""
         w, B, T = self.w, self.B, self.T
         n = len(w.layers)
         s4c.embed_gather(w.embedding, tokens.reshape(-1), out=self.x[0])
@@ -127,9 +140,16 @@ class TargetVerify:
                                workspace=self.ws_lin)
         last = n % (self.sets + 1)
         self.last = last
-        s4c.lm_head_greedy(self.a[last], w.lm_head, self.target_token, self.max_logit, self.status_head, self.ws_head)
-        s4c.tree_accept_tokens(self.target_token.view(B, T), tokens, parent, self.V, n_nodes, self.max_depth, self.accept_len,
-                               self.path, self.next_token, self.status_accept)
+        if temperature > 0.0:
+            if not self.stochastic:
+                raise ValueError("build the pass with stochastic=True to verify by speculative sampling")
+            s4c.lm_head_logits(self.a[last], w.lm_head, self.logits.view(self.R, self.V), self.status_head, self.ws_logits)
+            s4c.tree_accept(self.logits, draft_probs, tokens, parent, temperature, uniforms, n_nodes, self.max_depth, self.accept_len,
+                            self.path, self.next_token, self.near_tie, self.status_accept, self.ws_accept)
+        else:
+            s4c.lm_head_greedy(self.a[last], w.lm_head, self.target_token, self.max_logit, self.status_head, self.ws_head)
+            s4c.tree_accept_tokens(self.target_token.view(B, T), tokens, parent, self.V, n_nodes, self.max_depth, self.accept_len,
+                                   self.path, self.next_token, self.status_accept)
         if compact:
             s4c.kv_compact(self.k_ptrs, self.v_ptrs, n, (B, self.Hkv, self.C, self.d), torch.bfloat16, cache_len, self.path,
                            self.accept_len, T, feat_in=self.x[last].view(B, T, -1), feat_out=self.feat_out,

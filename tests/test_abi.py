@@ -212,6 +212,13 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
         ("g", P), ("eps", 1e-5), ("no", P), ("st", None), ("ws", P), ("wsb", 1 << 30), ("s", None)]])
     assert lnr(g=None) == 1 and lnr(no=None) == 1 and lnr(x1=None) == 1
     assert lnr(eps=-1.0) == 2 and lnr(N=12) == 2 and lnr(g=P + 2) == 4 and lnr(no=P + 8) == 4 and lnr(ws=None) == 5 and lnr(R=0) == 0
+    lib.s4c_lm_head_logits.argtypes = [vp, vp, i, i, i, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.s4c_lm_head_logits_workspace_bytes.restype = ctypes.c_size_t
+    lib.s4c_lm_head_logits_workspace_bytes.argtypes = [i, i, i]
+    lg = lambda **kw: lib.s4c_lm_head_logits(*[kw.get(k, d) for k, d in [
+        ("h", P), ("w", P), ("R", 26), ("V", 32000), ("H", 4096), ("out", P), ("st", None), ("ws", P), ("wsb", 1 << 30), ("s", None)]])
+    assert lg(h=None) == 1 and lg(out=None) == 1 and lg(V=32001) == 2 and lg(H=100) == 2 and lg(out=P + 4) == 4 and lg(R=0) == 0
+    assert lib.s4c_lm_head_logits_workspace_bytes(26, 32000, 4096) == lib.s4c_linear_workspace_bytes(26, 4096, 0, 32000, 0)
     lib.s4c_rmsnorm.argtypes = [vp, vp, f, i, i, vp, vp]
     rn = lambda **kw: lib.s4c_rmsnorm(*[kw.get(k, d) for k, d in [("x", P), ("g", P), ("eps", 1e-6), ("R", 4), ("H", 4096), ("out", P), ("s", None)]])
     assert rn(x=None) == 1 and rn(H=12) == 2 and rn(eps=-1.0) == 2 and rn(g=P + 2) == 4 and rn(R=0) == 0

@@ -264,3 +264,23 @@ def test_drafting_round_without_a_vocabulary_sized_array():
     torch.cuda.synchronize()
     for key in ("tokens", "parent", "position", "n_nodes"):
         np.testing.assert_array_equal(tree[key].cpu().numpy(), lib[key].cpu().numpy(), err_msg=key)
+
+
+@pytest.mark.parametrize("R,V,H", [(26, 32000, 512), (256, 5000, 256), (7, 8, 64), (130, 1000, 1024), (26, 32008, 128)])
+def test_logits_written_out_for_stochastic_verification(R, V, H):
+    # s4c_lm_head_logits: the float32 sums themselves, [R, V], against the oracle's float64 logits within the accumulation bound
+    from paper_2506_14158_b200 import s4c
+    from parity import Guarded
+
+    rng = np.random.default_rng(R + V)
+    hid = torch.from_numpy(rng.standard_normal((R, H)).astype(np.float32)).to(torch.bfloat16)
+    wgt = torch.from_numpy((rng.standard_normal((V, H)) / np.sqrt(H)).astype(np.float32)).to(torch.bfloat16)
+    out = Guarded((R, V), torch.float32, fill=-3.0)
+    st = torch.full((1,), -9, dtype=torch.int32, device="cuda")
+    s4c.lm_head_logits(hid.cuda(), wgt.cuda(), out.t, st)
+    torch.cuda.synchronize()
+    out.check("s4c_lm_head_logits logits")
+    assert int(st.item()) == 0
+    want = oracle.lm_head_greedy(hid.double().numpy(), wgt.double().numpy())["logits"]
+    slack = 4.0 * np.sqrt(H) * 2.0 ** -24 * np.linalg.norm(hid.double().numpy(), axis=1, keepdims=True) * np.linalg.norm(wgt.double().numpy(), axis=1).max()
+    assert (np.abs(out.t.double().cpu().numpy() - want) <= slack + 1e-7).all()

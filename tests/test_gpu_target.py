@@ -151,3 +151,46 @@ def test_verify_step_compacts_every_layer_and_replays_as_a_graph():
     for b in range(B):
         assert torch.equal(tv.path[b, : a[b] + 1], want[2][b, : a[b] + 1])
     np.testing.assert_array_equal(cl3.cpu().numpy(), cache_len + a + 1)
+
+
+def test_verify_pass_by_speculative_sampling():
+    # temperature > 0: the pass writes float32 logits and s4c_tree_accept walks them; the oracle's walk on the GPU's logits
+    # must take the same decisions bit for bit, and the logits must be the oracle's LM head within the accumulation bound
+    n_layers, B, T, V, Hq, Hkv, d, inter, L, C, md = 2, 3, 10, 2000, 4, 2, 64, 256, 30, 48, 4
+    H = Hq * d
+    from paper_2506_14158_b200 import target
+
+    torch.manual_seed(21)
+    w = target.random_weights(n_layers, V, H, Hq, Hkv, d, inter, "cuda", seed=21)
+    kcs = [torch.randn(B, Hkv, C, d, device="cuda").to(torch.bfloat16) for _ in range(n_layers)]
+    vcs = [torch.randn(B, Hkv, C, d, device="cuda").to(torch.bfloat16) for _ in range(n_layers)]
+    tv = target.TargetVerify(w, B, T, Hq, Hkv, d, C, kcs, vcs, md, stochastic=True)
+    rng = np.random.default_rng(22)
+    parent = np.stack([W.random_tree(T, md, rng, 1, 3) for _ in range(B)]).astype(np.int32)
+    tokens = rng.integers(0, V, (B, T)).astype(np.int32)
+    dl = rng.standard_normal((B, T, V)) * 2.0
+    dp = np.exp(dl - dl.max(axis=2, keepdims=True))
+    draft_probs = (dp / dp.sum(axis=2, keepdims=True)).astype(np.float32)
+    for b in range(B):  # children carry the drafter's most probable tokens of their parent's row, best first (Section 3.2)
+        for n in range(T):
+            kids = [i for i in range(1, T) if parent[b, i] == n]
+            order = np.argsort(-draft_probs[b, n], kind="stable")
+            for j, c in enumerate(kids):
+                tokens[b, c] = order[j]
+    uniforms = rng.random((B, T)).astype(np.float32)
+    cache_len = np.asarray([L, L - 7, 3], dtype=np.int32)
+    cl = dev(cache_len.copy())
+    tau = 0.7
+    r = tv.forward(dev(tokens), cl, dev(parent), max_cache_len=L, temperature=tau, draft_probs=dev(draft_probs), uniforms=dev(uniforms))
+    torch.cuda.synchronize()
+    assert int(tv.status_head.item()) == 0 and int(tv.status_accept.abs().sum().item()) == 0
+    logits = tv.logits.cpu().numpy()
+    want = oracle.lm_head_greedy(_f64(tv.a[tv.last]), _f64(w.lm_head))["logits"].reshape(B, T, V)
+    assert np.abs(logits - want).max() <= 4.0 * np.sqrt(H) * 2.0 ** -24 * 64.0
+    ref = oracle.accept_stochastic(logits, draft_probs, tokens, parent, float(np.float32(tau)), uniforms, None, md)
+    a = ref["accept_len"]
+    np.testing.assert_array_equal(r["accept_len"].cpu().numpy(), a)
+    np.testing.assert_array_equal(r["next_token"].cpu().numpy(), ref["next_token"])
+    for b in range(B):
+        np.testing.assert_array_equal(r["path"].cpu().numpy()[b, : a[b] + 1], ref["path"][b, : a[b] + 1])
+    np.testing.assert_array_equal(cl.cpu().numpy(), cache_len + a + 1)   # compacted and advanced like the greedy route
