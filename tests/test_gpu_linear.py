@@ -96,6 +96,35 @@ def test_wide_gated_projection_on_many_rows(R, K, N, res):
     assert (np.abs(_f64(out.t)[:, cols] - want) <= bound).all()
 
 
+@pytest.mark.parametrize("R,K1,K2,N", [(26, 4096, 4096, 4096), (26, 4096, 0, 4096), (26, 11008, 0, 4096),      # 7B shapes: fc, o, down
+                                       (256, 4096, 4096, 4096), (256, 4096, 0, 4096), (256, 14336, 0, 4096)])  # 8B shapes
+def test_full_size_projections_on_sampled_columns(R, K1, K2, N):
+    # the launch shapes the benchmark's drafter head and verify pass run (shared-out K ranges, one and two row tiles), with bias,
+    # residual and the fused normalisation; 512 sampled output columns against the oracle, the normalised rows against the oracle's
+    # normalisation of the rows the GPU wrote
+    from paper_2506_14158_b200 import s4c
+
+    rng = np.random.default_rng(R + K1 + K2)
+    K = K1 + K2
+    x1 = _bf16(rng.standard_normal((R, K1)))
+    x2 = _bf16(rng.standard_normal((R, K2))) if K2 else None
+    w = _bf16(rng.standard_normal((N, K)) / np.sqrt(K))
+    b, rs, g = _bf16(0.1 * rng.standard_normal(N)), _bf16(rng.standard_normal((R, N))), _bf16(1.0 + 0.1 * rng.standard_normal(N))
+    out, nrm = Guarded((R, N), torch.bfloat16, fill=-3.0), Guarded((R, N), torch.bfloat16, fill=-3.0)
+    s4c.linear_rmsnorm(x1.cuda(), w.cuda(), g.cuda(), 1e-5, x2=None if x2 is None else x2.cuda(), bias=b.cuda(), residual=rs.cuda(),
+                       out=out.t, norm_out=nrm.t)
+    torch.cuda.synchronize()
+    out.check("s4c_linear_rmsnorm out"), nrm.check("s4c_linear_rmsnorm norm_out")
+    cols = np.sort(rng.choice(N, 512, replace=False))
+    cols[:2], cols[-2:] = [0, 1], [N - 2, N - 1]
+    xx = np.concatenate([_f64(x1)] + ([_f64(x2)] if K2 else []), axis=1)
+    want = oracle.linear(xx, _f64(w)[cols], bias=_f64(b)[cols], residual=_f64(rs)[:, cols])
+    slack = 8.0 * np.sqrt(K) * 2.0 ** -24 * np.linalg.norm(xx, axis=1, keepdims=True) * np.linalg.norm(_f64(w)[cols], axis=1).max()
+    assert (np.abs(_f64(out.t)[:, cols] - want) <= 2.0 ** -8 * np.abs(want) + slack + 1e-6).all()
+    want_n = oracle.rmsnorm(_f64(out.t), _f64(g), 1e-5)
+    assert (np.abs(_f64(nrm.t) - want_n) <= 2.0 ** -8 * np.abs(want_n) + 1e-5).all()
+
+
 def test_shared_out_k_range_is_reproducible_and_checks_its_workspace():
     from paper_2506_14158_b200 import s4c
 
