@@ -506,8 +506,8 @@ def measure(cfg, args, device, rank, world, with_e2e):
     # every decoder layer (q/k/v + rotary, tree attention, output projection, gated MLP), LM head with the greedy choice, walk,
     # compaction of every layer's cache -- random weights of the target's shapes, caches of its own (timed alone)
     vp = None
-    if (cfg.dtype == "bf16" and not args.paged and cfg.d in (64, 128) and cfg.hid == cfg.Hq * cfg.d and cfg.n_layers > 1
-            and not args.no_verify_pass):
+    if (cfg.dtype == "bf16" and not args.paged and not args.capacity and cfg.name in ("c2x32", "c4x32") and cfg.n_layers > 1
+            and not args.no_verify_pass):  # (the two named model shapes; sweeps and capacity studies time attention only)
         from paper_2506_14158_b200 import target
 
         inter = {32000: 11008, 128256: 14336}.get(cfg.V, (cfg.hid * 8 // 3 + 255) // 256 * 256)
