@@ -356,13 +356,17 @@ def rope_rotate(x, pos, theta=10000.0):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
-def qkv_rope(x, w_qkv, cache_len, parent, Hq, Hkv, d, k_cache, v_cache, n_nodes=None, theta=10000.0):
+def qkv_rope(x, w_qkv, cache_len, parent, Hq, Hkv, d, k_cache, v_cache, n_nodes=None, theta=10000.0, position_base=None):
     """The verify layer's input side (Section 3.2: the target's forward pass over the T tree tokens; a decoder layer of the
     LLaMA family): q, k, v = x W^T for every tree token (float64; a library matrix product is the step), rotary embedding of
     q and k at position cache_len[b] + depth(node), q into a [B,Hq,T,d] array, k and v into the caches' tree slots
     cache_len[b] + node (k_cache, v_cache [B,Hkv,C,d] float64 arrays, modified in place).
 
     x [B,T,H]; w_qkv [(Hq+2*Hkv)*d, H]: the q heads' rows, then the k heads', then the v heads'.
+    position_base [B] (optional): the position of a sequence's root when it is not its cache length -- a drafter head whose own
+    cache is shorter than the text (Section 3.1.1: every head keeps its own features): a node's position is then
+    position_base[b] + depth(node); its slot stays cache_len[b] + node.  A negative base flags the sequence (SEQ_CAPACITY).
+
     Returns dict(q [B,Hq,T,d] float64 (rows of nodes >= n_nodes[b] and of flagged sequences are zero), status [B])."""
     x = np.asarray(x, dtype=np.float64)
     w = np.asarray(w_qkv, dtype=np.float64)
@@ -386,6 +390,9 @@ def qkv_rope(x, w_qkv, cache_len, parent, Hq, Hkv, d, k_cache, v_cache, n_nodes=
         L = int(cache_len[b])
         if L < 0 or L + T > C:
             flags |= SEQ_CAPACITY
+        P = L if position_base is None else int(position_base[b])
+        if P < 0:
+            flags |= SEQ_CAPACITY
         status[b] = flags
         if flags:
             continue
@@ -396,7 +403,7 @@ def qkv_rope(x, w_qkv, cache_len, parent, Hq, Hkv, d, k_cache, v_cache, n_nodes=
         qh = proj[:, : Hq * d].reshape(n, Hq, d)
         kh = proj[:, Hq * d: (Hq + Hkv) * d].reshape(n, Hkv, d)
         vh = proj[:, (Hq + Hkv) * d:].reshape(n, Hkv, d)
-        pos = (L + depth)[:, None]
+        pos = (P + depth)[:, None]
         q[b, :, :n] = rope_rotate(qh, pos, theta).transpose(1, 0, 2)
         k_cache[b, :, L:L + n] = rope_rotate(kh, pos, theta).transpose(1, 0, 2)
         v_cache[b, :, L:L + n] = vh.transpose(1, 0, 2)

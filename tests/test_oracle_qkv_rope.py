@@ -99,3 +99,44 @@ def test_padding_and_flags():
     assert (kc[0][:, 2 + 4:] == 1.5).all() and (r["q"][0][:, 4:] == 0).all() and (kc[0][:, 2:6] != 1.5).any()
     full = oracle.qkv_rope(x[3:], w, cache_len[3:], parent[3:], Hq, Hkv, d, np.zeros((1, Hkv, C, d)), np.zeros((1, Hkv, C, d)))
     np.testing.assert_array_equal(full["q"][0], r["q"][3])            # sequences are independent
+
+
+def test_position_base_moves_the_rotation_and_nothing_else():
+    # a root position that is not the cache length: values are rotated for position_base + depth (checked against plain
+    # math.cos / math.sin on one element and against rope_rotate of the unrotated projection), slots stay cache_len + node,
+    # v is untouched by the base, the cache length itself as base changes nothing, a negative base flags the sequence
+    rng = np.random.default_rng(31)
+    B, T, H, Hq, Hkv, d, C = 3, 6, 16, 2, 1, 8, 20
+    x = rng.standard_normal((B, T, H))
+    w = rng.standard_normal(((Hq + 2 * Hkv) * d, H))
+    parent = np.array([[-1, 0, 0, 1, 1, 3]] * B, dtype=np.int32)
+    depth = np.array([0, 1, 1, 2, 2, 3])
+    cache_len = np.array([4, 0, 9], dtype=np.int32)
+    base = np.array([11, 0, 100], dtype=np.int32)
+    k0, v0 = rng.standard_normal((B, Hkv, C, d)), rng.standard_normal((B, Hkv, C, d))
+    ka, va, kb, vb = k0.copy(), v0.copy(), k0.copy(), v0.copy()
+    plain = oracle.qkv_rope(x, w, cache_len, parent, Hq, Hkv, d, ka, va)
+    moved = oracle.qkv_rope(x, w, cache_len, parent, Hq, Hkv, d, kb, vb, position_base=base)
+    assert (moved["status"] == 0).all()
+    np.testing.assert_array_equal(va, vb)                                        # v does not know positions
+    np.testing.assert_array_equal(moved["q"][1], plain["q"][1])                  # base == cache length (0): the same
+    same = oracle.qkv_rope(x, w, cache_len, parent, Hq, Hkv, d, k0.copy(), v0.copy(), position_base=cache_len)
+    np.testing.assert_array_equal(same["q"], plain["q"])
+    theta = 10000.0
+    for b in (0, 2):
+        proj = x[b] @ w.T
+        qh = proj[:, : Hq * d].reshape(T, Hq, d)
+        kh = proj[:, Hq * d: (Hq + Hkv) * d].reshape(T, Hkv, d)
+        pos = (base[b] + depth)[:, None]
+        np.testing.assert_allclose(moved["q"][b], oracle.rope_rotate(qh, pos, theta).transpose(1, 0, 2), atol=1e-12)
+        L = cache_len[b]
+        np.testing.assert_allclose(kb[b, :, L:L + T], oracle.rope_rotate(kh, pos, theta).transpose(1, 0, 2), atol=1e-12)   # slots: L + node
+        np.testing.assert_array_equal(kb[b, :, :L], k0[b, :, :L])
+        np.testing.assert_array_equal(kb[b, :, L + T:], k0[b, :, L + T:])
+        t, h, i = 5, 1, 2                                                        # one element by hand: node 5, depth 3
+        a = (base[b] + 3) * theta ** (-2.0 * i / d)
+        want = qh[t, h, i] * math.cos(a) - qh[t, h, i + d // 2] * math.sin(a)
+        assert moved["q"][b, h, t, i] == pytest.approx(want, abs=1e-12)
+        assert not np.allclose(moved["q"][b], plain["q"][b])                     # and it does differ from the default
+    bad = oracle.qkv_rope(x, w, cache_len, parent, Hq, Hkv, d, k0.copy(), v0.copy(), position_base=np.array([3, -1, 3]))
+    assert bad["status"].tolist() == [0, oracle.SEQ_CAPACITY, 0] and (bad["q"][1] == 0).all()
