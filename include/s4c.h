@@ -357,6 +357,16 @@ s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32_t* cache_l
                         int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status, void* workspace,
                         size_t workspace_bytes, s4c_stream_t stream);
 
+/* s4c_qkv_rope_at -- the same with the root's position given apart from the cache length: a node's
+ * position is position_base[b] + depth, its slot stays cache_len[b] + node.  For a drafter head
+ * (Section 3.1.1) whose own cache holds fewer entries than the text has tokens.  position_base [B]
+ * int32 (device); a negative entry flags the sequence S4C_SEQ_CAPACITY.  Everything else as s4c_qkv_rope
+ * (which is the case position_base = cache_len). */
+s4c_status s4c_qkv_rope_at(const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* position_base,
+                           const int32_t* parent, const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache,
+                           int B, int T, int H, int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status,
+                           void* workspace, size_t workspace_bytes, s4c_stream_t stream);
+
 /* s4c_qkv_rope_same_tree -- another layer of the same verify pass (Section 3.2: one forward pass over
  * one tree): the tree checks, the rows' cache positions and the rotary table depend on cache_len,
  * parent, n_nodes, T, d and rope_theta alone, so the layers after the first reuse what s4c_qkv_rope

@@ -50,8 +50,8 @@ struct QkParams {
 constexpr int kQkPrepNodes = 8;
 __global__ void __launch_bounds__(128)
 qkv_prep_kernel(const int32_t* __restrict__ cache_len, const int32_t* __restrict__ parent, const int32_t* __restrict__ n_nodes,
-                int T, int C, int d, double theta, int32_t* __restrict__ row_base, float2* __restrict__ rope,
-                int32_t* __restrict__ status) {
+                const int32_t* __restrict__ position_base, int T, int C, int d, double theta, int32_t* __restrict__ row_base,
+                float2* __restrict__ rope, int32_t* __restrict__ status) {
     __shared__ int32_t par[S4C_MAX_T];
     __shared__ int depth[S4C_MAX_T];
     __shared__ uint32_t anc[S4C_MAX_T][S4C_MASK_WORDS];
@@ -61,10 +61,11 @@ qkv_prep_kernel(const int32_t* __restrict__ cache_len, const int32_t* __restrict
     const int t0 = blockIdx.y * kQkPrepNodes, t1 = min(T, t0 + kQkPrepNodes);
     const int n = n_nodes ? n_nodes[b] : T;
     const int L = cache_len[b];
+    const int P = position_base ? position_base[b] : L;  // the root's position: the cache length unless the caller says otherwise
     for (int i = tid; i < T; i += blockDim.x) par[i] = parent[(size_t)b * T + i];
     __syncthreads();
     int flags = build_ancestor_masks(par, n, T, anc, depth, &flag);
-    if (L < 0 || L + T > C) flags |= S4C_SEQ_CAPACITY;
+    if (L < 0 || L + T > C || P < 0) flags |= S4C_SEQ_CAPACITY;
     if (tid == 0 && blockIdx.y == 0 && status) status[b] = flags;
     for (int t = t0 + tid; t < t1; t += blockDim.x) row_base[(size_t)b * T + t] = (!flags && t < n) ? L : -1;
     if (flags) return;
@@ -73,7 +74,7 @@ qkv_prep_kernel(const int32_t* __restrict__ cache_len, const int32_t* __restrict
     const double freq = pow(theta, -2.0 * (double)i / (double)d);
     for (int t = t0 + tid / half; t < min(t1, n); t += blockDim.x / half) {
         double sn, cs;
-        sincos((double)(L + depth[t]) * freq, &sn, &cs);
+        sincos((double)(P + depth[t]) * freq, &sn, &cs);
         rope[((size_t)b * T + t) * half + i] = make_float2((float)cs, (float)sn);
     }
 }
@@ -298,7 +299,7 @@ namespace s4c {
 // tables: the tree / rotary-table kernel runs first (s4c_qkv_rope); otherwise the tables of the call before on this
 // workspace are used as they are (s4c_qkv_rope_same_tree)
 static s4c_status qk_run(bool tables, const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* parent,
-                         const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache, int B, int T, int H, int Hq, int Hkv, int d,
+                         const int32_t* n_nodes, const int32_t* position_base, void* q_out, void* k_cache, void* v_cache, int B, int T, int H, int Hq, int Hkv, int d,
                          int C, float rope_theta, int32_t* status, void* workspace, size_t workspace_bytes, s4c_stream_t stream_) {
     if (!x || !w_qkv || (tables && (!cache_len || !parent)) || !q_out || !k_cache || !v_cache) return S4C_ERR_NULL;
     if (B < 0 || T < 1 || T > S4C_MAX_T || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || (d != 64 && d != 128) || C < T) return S4C_ERR_SHAPE;
@@ -321,7 +322,7 @@ static s4c_status qk_run(bool tables, const void* x, const void* w_qkv, const in
     if (!qk_make_map(&map_x, x, (uint64_t)R, H, x_rows) || !qk_make_map(&map_w, w_qkv, (uint64_t)heads * d, H, d)) return S4C_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (tables) {
-        qkv_prep_kernel<<<dim3(B, ceil_div(T, kQkPrepNodes)), 128, 0, stream>>>(cache_len, parent, n_nodes, T, C, d, (double)rope_theta, row_base, rope, status);
+        qkv_prep_kernel<<<dim3(B, ceil_div(T, kQkPrepNodes)), 128, 0, stream>>>(cache_len, parent, n_nodes, position_base, T, C, d, (double)rope_theta, row_base, rope, status);
         S4C_RETURN_IF_CUDA_ERROR();
     }
     static bool configured[64] = {};  // the dynamic shared memory opt-in is per device
@@ -360,13 +361,22 @@ extern "C" s4c_status s4c_qkv_rope(const void* x, const void* w_qkv, const int32
                                    const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache, int B, int T, int H,
                                    int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status, void* workspace,
                                    size_t workspace_bytes, s4c_stream_t stream) {
-    return s4c::qk_run(true, x, w_qkv, cache_len, parent, n_nodes, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C, rope_theta, status,
-                       workspace, workspace_bytes, stream);
+    return s4c::qk_run(true, x, w_qkv, cache_len, parent, n_nodes, nullptr, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C, rope_theta,
+                       status, workspace, workspace_bytes, stream);
+}
+
+extern "C" s4c_status s4c_qkv_rope_at(const void* x, const void* w_qkv, const int32_t* cache_len, const int32_t* position_base,
+                                      const int32_t* parent, const int32_t* n_nodes, void* q_out, void* k_cache, void* v_cache,
+                                      int B, int T, int H, int Hq, int Hkv, int d, int C, float rope_theta, int32_t* status,
+                                      void* workspace, size_t workspace_bytes, s4c_stream_t stream) {
+    if (!position_base) return S4C_ERR_NULL;
+    return s4c::qk_run(true, x, w_qkv, cache_len, parent, n_nodes, position_base, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C,
+                       rope_theta, status, workspace, workspace_bytes, stream);
 }
 
 extern "C" s4c_status s4c_qkv_rope_same_tree(const void* x, const void* w_qkv, void* q_out, void* k_cache, void* v_cache, int B,
                                              int T, int H, int Hq, int Hkv, int d, int C, int32_t* status, void* workspace,
                                              size_t workspace_bytes, s4c_stream_t stream) {
-    return s4c::qk_run(false, x, w_qkv, nullptr, nullptr, nullptr, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C, 10000.f, status,
+    return s4c::qk_run(false, x, w_qkv, nullptr, nullptr, nullptr, nullptr, q_out, k_cache, v_cache, B, T, H, Hq, Hkv, d, C, 10000.f, status,
                        workspace, workspace_bytes, stream);
 }

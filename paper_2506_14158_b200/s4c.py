@@ -25,7 +25,7 @@ EXPORTS = ["s4c_version", "s4c_status_string", "s4c_tree_attention_workspace_byt
            "s4c_launch_floor", "s4c_selftest_attention_timeout", "s4c_tree_build_workspace_bytes", "s4c_tree_build",
            "s4c_tree_attention_paged", "s4c_kv_compact_paged", "s4c_tree_accept_filtered_workspace_bytes",
            "s4c_tree_accept_filtered", "s4c_lm_head_greedy_workspace_bytes", "s4c_lm_head_greedy", "s4c_tree_accept_tokens",
-           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_qkv_rope_same_tree", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
+           "s4c_qkv_rope_workspace_bytes", "s4c_qkv_rope", "s4c_qkv_rope_at", "s4c_qkv_rope_same_tree", "s4c_lm_head_topk_workspace_bytes", "s4c_lm_head_topk",
            "s4c_tree_build_topk", "s4c_lm_head_logits_workspace_bytes", "s4c_lm_head_logits", "s4c_linear_workspace_bytes", "s4c_linear", "s4c_linear_rmsnorm", "s4c_rmsnorm", "s4c_embed_gather"]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
@@ -86,6 +86,8 @@ def _load() -> ctypes.CDLL:
     lib.s4c_qkv_rope_workspace_bytes.argtypes = [i, i, i]
     lib.s4c_qkv_rope.restype = i
     lib.s4c_qkv_rope.argtypes = [vp, vp, i32p, i32p, i32p, vp, vp, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
+    lib.s4c_qkv_rope_at.restype = i
+    lib.s4c_qkv_rope_at.argtypes = [vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp, i, i, i, i, i, i, i, f, i32p, vp, sz, vp]
     lib.s4c_qkv_rope_same_tree.restype = i
     lib.s4c_qkv_rope_same_tree.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i32p, vp, sz, vp]
     lib.s4c_lm_head_topk_workspace_bytes.restype = sz
@@ -502,7 +504,7 @@ def qkv_rope_workspace_bytes(B, T, d) -> int:
 
 
 def qkv_rope(x, w_qkv, cache_len, parent, q_out, k_cache, v_cache, n_nodes=None, rope_theta: float = 10000.0, status=None,
-             workspace=None, stream=None):
+             workspace=None, stream=None, position_base=None):
     """s4c_qkv_rope: q/k/v projections of the tree tokens, rotary embedding at position cache_len + depth, q into
     ``q_out`` [B,Hq,T,d], k and v into the caches' tree slots (``k_cache``, ``v_cache`` [B,Hkv,C,d], written in place)."""
     B, T, H = x.shape
@@ -513,13 +515,18 @@ def qkv_rope(x, w_qkv, cache_len, parent, q_out, k_cache, v_cache, n_nodes=None,
     if workspace is None:
         workspace = _workspace(int(_lib.s4c_qkv_rope_workspace_bytes(B, T, d)), dev, "qkv_rope")
     bf = torch.bfloat16
-    rc = _lib.s4c_qkv_rope(_dev(x, bf, "x"), _dev(w_qkv, bf, "w_qkv"), _dev(cache_len, torch.int32, "cache_len"),
-                           _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"), _dev(q_out, bf, "q_out"),
-                           _dev(k_cache, bf, "k_cache"), _dev(v_cache, bf, "v_cache"), B, T, H, Hq, Hkv, d, C, float(rope_theta),
-                           _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"),
-                           workspace.numel() * workspace.element_size(), _stream(stream))
+    tail = (_dev(q_out, bf, "q_out"), _dev(k_cache, bf, "k_cache"), _dev(v_cache, bf, "v_cache"), B, T, H, Hq, Hkv, d, C, float(rope_theta),
+            _dev(status, torch.int32, "status"), _dev(workspace, name="workspace"), workspace.numel() * workspace.element_size(),
+            _stream(stream))
+    if position_base is None:
+        rc = _lib.s4c_qkv_rope(_dev(x, bf, "x"), _dev(w_qkv, bf, "w_qkv"), _dev(cache_len, torch.int32, "cache_len"),
+                               _dev(parent, torch.int32, "parent"), _dev(n_nodes, torch.int32, "n_nodes"), *tail)
+    else:  # s4c_qkv_rope_at: positions count from position_base[b], slots from cache_len[b]
+        rc = _lib.s4c_qkv_rope_at(_dev(x, bf, "x"), _dev(w_qkv, bf, "w_qkv"), _dev(cache_len, torch.int32, "cache_len"),
+                                  _dev(position_base, torch.int32, "position_base"), _dev(parent, torch.int32, "parent"),
+                                  _dev(n_nodes, torch.int32, "n_nodes"), *tail)
     if rc:
-        raise S4CError("s4c_qkv_rope", rc)
+        raise S4CError("s4c_qkv_rope_at" if position_base is not None else "s4c_qkv_rope", rc)
     return dict(q=q_out, status=status)
 
 

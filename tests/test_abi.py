@@ -169,6 +169,11 @@ def test_bad_arguments_are_rejected_on_the_host(s4c_lib):
     assert qk(B=0) == 0
     assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) % 256 == 0 and lib.s4c_qkv_rope_workspace_bytes(4, 64, 128) > 0
     assert lib.s4c_qkv_rope_workspace_bytes(4, 64, 96) == 0
+    lib.s4c_qkv_rope_at.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp, vp, sz, vp]
+    qa = lambda **kw: lib.s4c_qkv_rope_at(*[kw.get(k, d) for k, d in [
+        ("x", P), ("w", P), ("cl", P), ("pb", P), ("par", P), ("nn", None), ("q", P), ("k", P), ("v", P), ("B", 1), ("T", 26), ("H", 4096),
+        ("Hq", 32), ("Hkv", 8), ("d", 128), ("C", 2048), ("theta", 10000.0), ("st", None), ("ws", None), ("wsb", 0), ("s", None)]])
+    assert qa(pb=None) == 1 and qa(cl=None) == 1 and qa(d=96) == 2 and qa(q=P + 2) == 4 and qa() == 5 and qa(B=0) == 0
     lib.s4c_qkv_rope_same_tree.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, vp, sz, vp]
     qs = lambda **kw: lib.s4c_qkv_rope_same_tree(*[kw.get(k, d) for k, d in [
         ("x", P), ("w", P), ("q", P), ("k", P), ("v", P), ("B", 1), ("T", 26), ("H", 4096), ("Hq", 32), ("Hkv", 8), ("d", 128),

@@ -20,7 +20,7 @@ def _bf16(a):
     return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16)
 
 
-def _run(x, w, cache_len, parent, Hq, Hkv, d, C, n_nodes=None, theta=10000.0, seed=0):
+def _run(x, w, cache_len, parent, Hq, Hkv, d, C, n_nodes=None, theta=10000.0, seed=0, position_base=None):
     from paper_2506_14158_b200 import s4c
 
     B, T, H = x.shape
@@ -31,12 +31,14 @@ def _run(x, w, cache_len, parent, Hq, Hkv, d, C, n_nodes=None, theta=10000.0, se
                 v=Guarded((B, Hkv, C, d), torch.bfloat16, src=v0.cuda()), status=Guarded((B,), torch.int32, fill=-9),
                 ws=Guarded((max(256, s4c.qkv_rope_workspace_bytes(B, T, d)),), torch.uint8, fill=0xCD))
     s4c.qkv_rope(x.cuda(), w.cuda(), dev(cache_len), dev(parent.astype(np.int32)), bufs["q"].t, bufs["k"].t, bufs["v"].t,
-                 None if n_nodes is None else dev(n_nodes), theta, status=bufs["status"].t, workspace=bufs["ws"].t)
+                 None if n_nodes is None else dev(n_nodes), theta, status=bufs["status"].t, workspace=bufs["ws"].t,
+                 position_base=None if position_base is None else dev(np.asarray(position_base, dtype=np.int32)))
     torch.cuda.synchronize()
     for name, buf in bufs.items():
         buf.check("s4c_qkv_rope " + name)
     kc, vc = k0.double().numpy().copy(), v0.double().numpy().copy()
-    ref = oracle.qkv_rope(x.double().numpy(), w.double().numpy(), cache_len, parent, Hq, Hkv, d, kc, vc, n_nodes, theta)
+    ref = oracle.qkv_rope(x.double().numpy(), w.double().numpy(), cache_len, parent, Hq, Hkv, d, kc, vc, n_nodes, theta,
+                          position_base=position_base)
     got = dict(q=bufs["q"].t.double().cpu().numpy(), k=bufs["k"].t.double().cpu().numpy(), v=bufs["v"].t.double().cpu().numpy(),
                status=bufs["status"].t.cpu().numpy())
     return got, dict(q=ref["q"], k=kc, v=vc, status=ref["status"]), (k0.double().numpy(), v0.double().numpy())
@@ -138,6 +140,22 @@ def test_another_layer_on_the_same_tree_reuses_the_tables(B, T, H, Hq, Hkv, d, C
     if B >= 5:
         assert st.tolist()[1] == oracle.SEQ_CAPACITY and st.tolist()[2] == oracle.SEQ_BAD_PARENT
         assert (q2.t[1] == -3.0).all() and torch.equal(k2.t[2], k0[2])
+
+
+def test_root_position_apart_from_the_cache_length():
+    # s4c_qkv_rope_at: positions count from position_base, slots from cache_len; a negative base flags its sequence
+    rng = np.random.default_rng(19)
+    B, T, H, Hq, Hkv, d, C = 4, 12, 256, 4, 2, 64, 40
+    parent = np.stack([W.random_tree(T, 5, rng, 1, 3) for _ in range(B)])
+    x, w = _bf16(rng.standard_normal((B, T, H))), _bf16(rng.standard_normal(((Hq + 2 * Hkv) * d, H)) / np.sqrt(H))
+    cache_len = np.array([5, 0, 28, 17], dtype=np.int32)
+    base = np.array([900, 3, -2, 17], dtype=np.int32)
+    got, ref, _ = _run(x, w, cache_len, parent, Hq, Hkv, d, C, position_base=base)
+    assert ref["status"].tolist() == [0, 0, oracle.SEQ_CAPACITY, 0]
+    _compare(got, ref, x, w, cache_len, None, T)
+    plain, _, _ = _run(x, w, cache_len, parent, Hq, Hkv, d, C)
+    np.testing.assert_array_equal(got["q"][3], plain["q"][3])          # base == cache length: the plain call
+    assert not np.array_equal(got["q"][0], plain["q"][0])
 
 
 def test_full_size_layer_then_attention_reads_what_was_written():
