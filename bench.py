@@ -501,7 +501,39 @@ def measure(cfg, args, device, rank, world, with_e2e):
         wbytes = sum(t.numel() * 2 for t in (wts.fc, wts.qkv, wts.o, wts.gate_up, wts.down, wts.lm_head))
         dr = dict(ms=ms_dr, rows=cfg.B * cfg.T, weight_bytes=wbytes, inter=inter, k=kk,
                   flops=2.0 * cfg.B * cfg.T * (wbytes / 2))
-        del wts, head, kc, vc
+        del head, kc, vc
+        # a whole drafting round: three heads (weights of their own; the target's embedding and LM head shared) fill a 21-node tree
+        # level by level (Section 3.1.1 + 3.2) -- rows 2, 6, 6 per sequence
+        if cfg.name in ("c2x32", "c4x32", "c2", "c4"):
+            br3, T3, k3 = [2, 3, 1, 1], 21, 3
+            w3 = [wts] + [drafter.random_weights(8, cfg.hid, cfg.Hq, cfg.Hkv, cfg.d, inter, device, seed=cfg.config_id + 100 + j) for j in (1, 2)]
+            for w_ in w3[1:]:
+                w_.embedding, w_.lm_head = wts.embedding, wts.lm_head
+            mh = drafter.MultiHeadDrafter(w3, cfg.B, T3, br3, cfg.Hq, cfg.Hkv, cfg.d, cfg.C, k3)
+            caches3 = []
+            for j in range(mh.n_passes):
+                nj = mh.levels[j][1] - mh.levels[j][0]
+                kc3 = torch.zeros((cfg.B * nj, cfg.Hkv, cfg.C, cfg.d), dtype=torch.bfloat16, device=device)
+                caches3.append((kc3, torch.zeros_like(kc3), step.cache_len0.repeat_interleave(nj).contiguous()))
+            root3, f03 = step.tokens[:, 0].contiguous(), step.feat_in[:, 0].contiguous()
+            cand3 = torch.arange(k3, dtype=torch.int32, device=device).repeat(cfg.B, 1).contiguous()
+            run_round = lambda: mh.draft(root3, f03, cand3, step.cache_len0, caches3)
+            sg = torch.cuda.Stream()
+            sg.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(sg):
+                run_round()
+            torch.cuda.current_stream().wait_stream(sg)
+            torch.cuda.synchronize()
+            g_mh = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_mh):
+                run_round()
+            for _ in range(3):
+                g_mh.replay()
+            dr["round_ms"] = time_graph(g_mh, K, torch)
+            dr["round_weight_bytes"] = 3 * (wbytes - wts.lm_head.numel() * 2) + 3 * wts.lm_head.numel() * 2  # each head streams the LM head again
+            dr["round_rows"] = [cfg.B * (e - s) for s, e in mh.levels[: mh.n_passes]]
+            del mh, caches3, w3
+        del wts
     # the whole greedy verify pass of the target (Section 3.2) composed from the library's calls: embedding of the tree tokens,
     # every decoder layer (q/k/v + rotary, tree attention, output projection, gated MLP), LM head with the greedy choice, walk,
     # compaction of every layer's cache -- random weights of the target's shapes, caches of its own (timed alone)
@@ -635,6 +667,13 @@ def roofline_records(cfg, args, rec, pk):
             bound="tensor" if dr["flops"] / dr["weight_bytes"] >= ridge else "hbm", gbs=dr["weight_bytes"] / t * 1e-9,
             frac_of_hbm_peak=dr["weight_bytes"] / t * 1e-9 / pk["hbm_gbs"], tflops=dr["flops"] / t * 1e-12,
             frac_of_tensor_peak=dr["flops"] / t * 1e-12 / pk["bf16_tflops"])
+        if "round_ms" in dr:
+            breakdown["drafter_round_3_heads_not_in_step"] = dr["round_ms"]
+            roofline["drafter_head"]["round_of_three_heads"] = dict(
+                what="three heads fill a 21-node tree level by level (rows per head below), tree rebuilt from the ranked choices after each",
+                rows_per_head=dr["round_rows"], us=dr["round_ms"] * 1e3, weight_bytes=dr["round_weight_bytes"],
+                gbs=dr["round_weight_bytes"] / (dr["round_ms"] * 1e-3) * 1e-9,
+                frac_of_hbm_peak=dr["round_weight_bytes"] / (dr["round_ms"] * 1e-3) * 1e-9 / pk["hbm_gbs"])
     if rec.get("vp") is not None:
         vp = rec["vp"]
         breakdown["full_verify_pass_not_in_step"] = vp["ms"]
