@@ -13,7 +13,7 @@
  *
  * Around them, the rest of the target's pass and the drafter's head (Section 3.1, Eq. 3-6), so
  * that a whole greedy round runs from these calls alone:
- *   per decoder layer:  s4c_qkv_rope (_same_tree)   q/k/v projections + rotary embedding into the
+ *   per decoder layer:  s4c_qkv_rope (_same_tree, _at)  q/k/v projections + rotary embedding into the
  *                                                   attention layout and the cache's tree slots
  *                       s4c_linear, s4c_linear_rmsnorm, s4c_rmsnorm   projections, gated MLP, norms
  *   once per step:      s4c_embed_gather            Eq. 6
@@ -21,7 +21,8 @@
  *                                                   the k ranked choices kept in the epilogue
  *                       s4c_tree_accept_tokens      the greedy walk on the choices
  *                       s4c_tree_build_topk         the tree from ranked choices
- * Variants: s4c_tree_attention_paged / s4c_kv_compact_paged (paged caches),
+ * Variants: s4c_tree_attention_rows (output as the rows the next projection reads), s4c_lm_head_logits
+ * (float32 logits for speculative sampling), s4c_tree_attention_paged / s4c_kv_compact_paged (paged caches),
  * s4c_tree_accept_filtered (top-k / nucleus filtered sampling), s4c_tree_accept_noalloc.
  *
  * Conventions for every entry point
