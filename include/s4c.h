@@ -60,7 +60,7 @@ typedef enum {
     S4C_ERR_DTYPE = 3,       /* unknown s4c_dtype */
     S4C_ERR_ALIGN = 4,       /* a tensor base pointer is not 16-byte aligned */
     S4C_ERR_WORKSPACE = 5,   /* workspace missing or smaller than the query says */
-    S4C_ERR_UNSUPPORTED = 6, /* valid request this build has no kernel for */
+    S4C_ERR_UNSUPPORTED = 6, /* valid request the library has no kernel for */
     S4C_ERR_CUDA = 7         /* a CUDA runtime call (launch, attribute) failed */
 } s4c_status;
 

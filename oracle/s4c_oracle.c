@@ -26,7 +26,7 @@
  *   s4c_oracle_accept_filtered the same walk against a top-k / nucleus filtered
  *                              target distribution (the sampling regime of the
  *                              temperature study, Section 4; the filter itself
- *                              is this build's statement of the usual samplers).
+ *                              is the usual chain of logit warpers, restated).
  *   s4c_oracle_kv_compact      Section 3.2, last paragraph (accepted tokens and
  *                              their features are kept for the next drafting
  *                              phase): a gather from a snapshot.
@@ -319,7 +319,7 @@ int s4c_oracle_accept_greedy(const float* logits, const int32_t* tokens, const i
 /*  F3  if top_p < 1: keep the shortest prefix, in rank order, whose          */
 /*      cumulative (renormalised) probability reaches top_p; renormalise.      */
 /* Every other token gets p = 0.  top_k = 0 leaves p as it is (top_p unused). */
-/* The paper does not define filtering; F1-F3 are this build's statement of   */
+/* The paper does not define filtering; F1-F3 restate, in their usual order,    */
 /* the usual top-k / nucleus samplers, and the accept / resample steps then    */
 /* preserve the FILTERED target distribution.                                  */
 static int accept_sampling(const float* logits, const float* dprobs, const int32_t* tokens,
