@@ -319,7 +319,7 @@ int s4c_oracle_accept_greedy(const float* logits, const int32_t* tokens, const i
 /*  F3  if top_p < 1: keep the shortest prefix, in rank order, whose          */
 /*      cumulative (renormalised) probability reaches top_p; renormalise.      */
 /* Every other token gets p = 0.  top_k = 0 leaves p as it is (top_p unused). */
-/* The paper does not define filtering; F1-F3 restate, in their usual order,    */
+/* The paper does not define filtering; F1-F3 restate, in their usual order,   */
 /* the usual top-k / nucleus samplers, and the accept / resample steps then    */
 /* preserve the FILTERED target distribution.                                  */
 static int accept_sampling(const float* logits, const float* dprobs, const int32_t* tokens,
